@@ -1,0 +1,242 @@
+/*
+ * aflex.h -- C ABI of the B200-native A/F decode-layer hot path.
+ *
+ * One decoder-layer decode step is split into an Attention side (A) and an FFN
+ * side (F) that exchange hidden states once per layer (paper Section 4.3,
+ * "Placement-aware A/F Data Path": the Attention group sends its outputs to the
+ * FFN group, which returns the hidden states) and run as M interleaved
+ * microbatches (Section 4.3, "Interleaved A/F Pipeline", Eq. 2).  The paper
+ * delegates the operators' arithmetic to its serving engine; the definitions
+ * implemented here are the standard ones and are restated at each entry point.
+ *
+ * Conventions (all entry points)
+ *  - Return value: aflex_status; 0 = OK.  Nothing throws, aborts or traps.
+ *  - Tensor pointers are DEVICE pointers unless the comment says "host".  They
+ *    are borrowed: the caller keeps them alive and unmodified until the work
+ *    enqueued by the call has finished on the stream; the library never frees
+ *    or reallocates them.  All base pointers must be 16-byte aligned.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *    stream).  Work is enqueued asynchronously; no call synchronises the
+ *    device unless its comment says so.
+ *  - bf16 tensors are raw 16-bit patterns, row-major, innermost dimension last.
+ *    Every fp32 -> bf16 store rounds to nearest even.
+ *  - Arguments are validated on the host before anything is enqueued: on a
+ *    non-OK return nothing was launched.  Shapes outside the supported
+ *    envelope return AFLEX_ERR_UNSUPPORTED (there is no slow path and no CPU
+ *    fallback).
+ *  - An aflex_ctx owns a device workspace, two internal streams and events
+ *    for aflex_layer_step, and a device status word.  A ctx is bound to one
+ *    device and must be used by one host thread at a time.  Calls that use the
+ *    same ctx must be stream-ordered with respect to each other (they share the
+ *    workspace); aflex_layer_step orders its own internal streams.
+ *  - Device-side waits are bounded: if one expires the kernel records
+ *    AFLEX_ERR_TIMEOUT in the ctx status word and exits cleanly; read it with
+ *    aflex_get_device_status.
+ *
+ * Supported envelope: head_dim in {64,128}; page_size 16; Hq/Hkv in {1,2,4,8};
+ * batch >= 1; every seq_len >= 1; hidden, inter and Hq*head_dim multiples of 8;
+ * num_experts <= 64 with top_k in {1,2} and top_k <= num_experts.
+ */
+#ifndef AFLEX_H_
+#define AFLEX_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define AFLEX_API __attribute__((visibility("default")))
+#else
+#define AFLEX_API
+#endif
+
+typedef enum {
+    AFLEX_OK = 0,
+    AFLEX_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, M > batch, ... */
+    AFLEX_ERR_UNSUPPORTED = 2, /* valid but outside the supported envelope */
+    AFLEX_ERR_WORKSPACE = 3,   /* ctx workspace too small for this call */
+    AFLEX_ERR_CUDA = 4,        /* a CUDA runtime/driver call failed (see aflex_last_error) */
+    AFLEX_ERR_TIMEOUT = 5,     /* a bounded device-side wait expired */
+    AFLEX_ERR_BOUNDS = 6       /* a device-side index check failed (page id / expert id out of range) */
+} aflex_status;
+
+typedef struct aflex_ctx aflex_ctx;
+
+/* Static string for a status code. */
+AFLEX_API const char* aflex_status_string(aflex_status s);
+
+/* Library version, major*10000 + minor*100 + patch. */
+AFLEX_API int aflex_version(void);
+
+/*
+ * Create a context on CUDA device `device`.  `workspace_bytes` is the size of
+ * the device workspace the ctx allocates (0 = library default, 256 MiB); use
+ * aflex_workspace_bytes to size it for a given layer.  Allocates device memory
+ * and creates streams/events: call it outside any timed or captured region.
+ * *out is owned by the caller and released with aflex_destroy.
+ */
+AFLEX_API aflex_status aflex_create(aflex_ctx** out, int device, size_t workspace_bytes);
+
+/* Synchronises the ctx's streams, frees everything the ctx owns. NULL is OK. */
+AFLEX_API aflex_status aflex_destroy(aflex_ctx* ctx);
+
+/* Host string describing the last non-OK return on this ctx (never NULL). */
+AFLEX_API const char* aflex_last_error(const aflex_ctx* ctx);
+
+/*
+ * Synchronises `stream`, then returns and clears the device status word:
+ * AFLEX_OK, AFLEX_ERR_TIMEOUT or AFLEX_ERR_BOUNDS as raised by kernels
+ * enqueued through this ctx.
+ */
+AFLEX_API aflex_status aflex_get_device_status(aflex_ctx* ctx, void* stream);
+
+/* ---- Attention side -------------------------------------------------------
+ *
+ * Decode attention (the operator the paper's Sections 1-2 describe as
+ * memory-bound on reads of the growing KV cache; one query token per
+ * sequence).  For sequence b with n = seq_lens[b] cached tokens and query head
+ * h reading KV head g = h / (Hq/Hkv):
+ *     s_j  = sm_scale * <q[b,h,:], K_j>            j = 0..n-1
+ *     p    = softmax(s)                            (fp32 scores and sums)
+ *     out[b,h,:] = sum_j p_j V_j                   -> bf16
+ *     lse[b,h]   = max_j s_j + ln sum_j exp(s_j - max)
+ * Token j of sequence b is stored in physical page page_table[b][j/16], slot
+ * j%16.  No mask (the n cached tokens include the one being decoded), no
+ * positional term.  Slots beyond a sequence's length and pages no sequence
+ * references may hold anything (including NaN) and do not affect the output.
+ * The work is split over KV chunks and merged by a combine pass; the result is
+ * deterministic run to run.
+ */
+typedef struct {
+    int num_q_heads;   /* Hq */
+    int num_kv_heads;  /* Hkv, divides Hq */
+    int head_dim;      /* D: 64 or 128 */
+    int page_size;     /* must be 16 */
+    float sm_scale;    /* 0 => 1/sqrt(D) */
+} aflex_attn_desc;
+
+typedef struct {
+    const void* k_cache;          /* bf16 [num_pages][Hkv][page_size][D] */
+    const void* v_cache;          /* bf16 [num_pages][Hkv][page_size][D] */
+    int64_t num_pages;            /* pages in each pool; page ids must be in [0, num_pages) */
+    const int32_t* page_table;    /* i32 [batch][max_pages_per_seq]; entries past ceil(len/16) are ignored */
+    int max_pages_per_seq;        /* row stride of page_table; also bounds every seq_len <= 16*max_pages_per_seq */
+    const int32_t* seq_lens;      /* i32 [batch], each >= 1 */
+    const int32_t* seq_lens_host; /* optional HOST copy of seq_lens (validated: each in [1, 16*max_pages_per_seq]); may be NULL */
+} aflex_kv;
+
+/*
+ * q   bf16 [batch][Hq][D]            (device, read)
+ * out bf16 [batch][Hq][D]            (device, written)
+ * lse fp32 [batch][Hq] or NULL       (device, written when non-NULL)
+ * Uses the ctx workspace for the per-chunk partial results.
+ * Errors: INVALID_ARG (null pointers, batch < 1, a host seq_len outside its
+ * range), UNSUPPORTED (envelope), WORKSPACE.
+ */
+AFLEX_API aflex_status aflex_attn_decode(aflex_ctx* ctx, const aflex_attn_desc* desc, const void* q,
+                                         const aflex_kv* kv, int batch, void* out, float* lse, void* stream);
+
+/* ---- FFN side -------------------------------------------------------------
+ *
+ * Dense SwiGLU FFN (the decode FFN operator of the paper's Section 1: weight
+ * streaming at small batch, tensor-core bound at large batch):
+ *     h = silu(x W_gate^T) .* (x W_up^T)     silu(z) = z / (1 + exp(-z))
+ *     y = h W_down^T
+ * x bf16 [T][H]; w_gate, w_up bf16 [I][H]; w_down bf16 [H][I]; y bf16 [T][H].
+ * fp32 accumulation; h is rounded to bf16 once between the two GEMMs.
+ * T >= 1; H and I multiples of 8 (otherwise UNSUPPORTED).
+ */
+AFLEX_API aflex_status aflex_ffn_dense(aflex_ctx* ctx, const void* x, const void* w_gate, const void* w_up,
+                                       const void* w_down, int T, int H, int I, void* y, void* stream);
+
+/*
+ * Top-k mixture-of-experts SwiGLU FFN (the sparse-expert FFN of the paper's
+ * Section 6.4 model family):
+ *   routing : idx[t][k], k < K = the K largest router logits of token t in
+ *             descending order; equal logits -> lower expert id first; a NaN
+ *             logit never wins.  gate[t][k] = softmax over the K selected
+ *             logits (fp32).
+ *   permute : assignments (t,k) sorted by (expert, t, k); counts per expert.
+ *   experts : per expert e, its rows go through that expert's SwiGLU FFN
+ *             (grouped GEMMs over the permuted rows).
+ *   combine : y[t] = sum_{k ascending} gate[t][k] * FFN_{idx[t][k]}(x[t]) in
+ *             fp32, then -> bf16.  No atomics: deterministic.
+ * Exactly one of router_logits (fp32 [T][E]) and w_router (bf16 [E][H]) is
+ * non-NULL; with w_router the logits are x W_router^T accumulated in fp32.
+ * w_gate, w_up bf16 [E][I][H]; w_down bf16 [E][H][I].
+ * Optional outputs (device, NULL to skip): topk_idx i32 [T][K], topk_gate fp32
+ * [T][K], expert_counts i32 [E].
+ * E <= 64, K in {1,2}, K <= E.
+ */
+AFLEX_API aflex_status aflex_ffn_moe(aflex_ctx* ctx, const void* x, const float* router_logits,
+                                     const void* w_router, const void* w_gate, const void* w_up,
+                                     const void* w_down, int T, int H, int I, int E, int top_k, void* y,
+                                     int32_t* topk_idx, float* topk_gate, int32_t* expert_counts, void* stream);
+
+/* ---- Layer step: A side, boundary, F side, as M interleaved microbatches ---
+ *
+ * Computes, for the whole batch,
+ *     a = attention(q, kv)                       bf16 [B][Hq*D]
+ *     x = a W_o^T   (x = a if w_o == NULL, which requires Hq*D == hidden)
+ *     y = dense FFN(x)  or  MoE FFN(x, router)   bf16 [B][hidden]
+ * scheduled as in the paper's interleaved A/F pipeline (Section 4.3, Eq. 2):
+ * the batch is cut into M contiguous microbatches; A_i (attention + W_o) is
+ * enqueued on the ctx's attention stream, F_i on its FFN stream as soon as A_i
+ * has finished, so A_{i+1} overlaps F_i.  M = 1 runs A then F serially.  Both
+ * "sides" live on one GPU here, so the transfer term of Eq. 2 is zero.
+ * The result does not depend on M or on the split.
+ */
+typedef struct {
+    aflex_attn_desc attn;
+    int hidden;            /* H */
+    int inter;             /* I */
+    int num_experts;       /* 0 => dense FFN */
+    int top_k;             /* MoE only */
+    const void* w_o;       /* bf16 [H][Hq*D], or NULL iff Hq*D == H */
+    const void* w_gate;    /* dense [I][H]  | MoE [E][I][H] */
+    const void* w_up;      /* dense [I][H]  | MoE [E][I][H] */
+    const void* w_down;    /* dense [H][I]  | MoE [E][H][I] */
+    const void* w_router;  /* MoE: bf16 [E][H] or NULL when router logits are passed */
+} aflex_layer_desc;
+
+/*
+ * q bf16 [B][Hq][D]; kv as for aflex_attn_decode (rows of page_table/seq_lens
+ * are per sequence, sliced per microbatch); router_logits fp32 [B][E] or NULL.
+ * microbatch_depth = M >= 1, M <= batch.  mb_offsets: HOST i32 [M+1],
+ * non-decreasing... strictly increasing from 0 to batch, or NULL for the
+ * near-equal split (the first batch % M microbatches get one extra row).
+ * attn_out bf16 [B][Hq][D]: optional copy of the A-side output (NULL => kept
+ * in the workspace).  y bf16 [B][hidden].
+ * `stream` is joined on entry (the internal streams wait for it) and on exit
+ * (it waits for the last A and F work).
+ */
+AFLEX_API aflex_status aflex_layer_step(aflex_ctx* ctx, const aflex_layer_desc* layer, const void* q,
+                                        const aflex_kv* kv, int batch, const float* router_logits,
+                                        int microbatch_depth, const int32_t* mb_offsets, void* attn_out,
+                                        void* y, void* stream);
+
+/*
+ * Workspace bytes that suffice for aflex_attn_decode / aflex_ffn_* /
+ * aflex_layer_step on this layer with up to max_batch rows and sequences of up
+ * to 16*max_pages_per_seq tokens.  Pure host computation.
+ */
+AFLEX_API size_t aflex_workspace_bytes(const aflex_layer_desc* layer, int max_batch, int max_pages_per_seq);
+
+/*
+ * Plain bf16 linear map y = x W^T with fp32 accumulation (the W_o boundary
+ * projection of aflex_layer_step, exposed for testing and benchmarking).
+ * x bf16 [T][K]; w bf16 [N][K]; y bf16 [T][N].  K, N multiples of 8.
+ */
+AFLEX_API aflex_status aflex_linear(aflex_ctx* ctx, const void* x, const void* w, int T, int K, int N,
+                                    void* y, void* stream);
+
+/* Tuning knob: tokens per split-KV chunk (multiple of 64; 0 = automatic). */
+AFLEX_API aflex_status aflex_set_attn_chunk(aflex_ctx* ctx, int chunk_tokens);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AFLEX_H_ */

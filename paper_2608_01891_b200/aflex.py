@@ -1,0 +1,210 @@
+"""Thin ctypes binding over the C-ABI CUDA library (``include/aflex.h``).
+
+Argument marshalling only: every step of the hot path runs inside libaflex's
+kernels.  PyTorch tensors are used as device-memory handles (``data_ptr()``) and
+for the current stream.  There is no CPU fallback: if the library cannot be
+loaded, or a call returns a non-OK status, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libaflex.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_BOUNDS = range(7)
+
+# Every symbol include/aflex.h declares.
+EXPORTS = (
+    "aflex_status_string", "aflex_version", "aflex_create", "aflex_destroy", "aflex_last_error",
+    "aflex_get_device_status", "aflex_attn_decode", "aflex_ffn_dense", "aflex_ffn_moe", "aflex_layer_step",
+    "aflex_workspace_bytes", "aflex_linear", "aflex_set_attn_chunk",
+)
+
+
+class AttnDesc(ctypes.Structure):
+    _fields_ = [("num_q_heads", ctypes.c_int), ("num_kv_heads", ctypes.c_int), ("head_dim", ctypes.c_int),
+                ("page_size", ctypes.c_int), ("sm_scale", ctypes.c_float)]
+
+
+class KV(ctypes.Structure):
+    _fields_ = [("k_cache", ctypes.c_void_p), ("v_cache", ctypes.c_void_p), ("num_pages", ctypes.c_int64),
+                ("page_table", ctypes.c_void_p), ("max_pages_per_seq", ctypes.c_int),
+                ("seq_lens", ctypes.c_void_p), ("seq_lens_host", ctypes.c_void_p)]
+
+
+class LayerDesc(ctypes.Structure):
+    _fields_ = [("attn", AttnDesc), ("hidden", ctypes.c_int), ("inter", ctypes.c_int),
+                ("num_experts", ctypes.c_int), ("top_k", ctypes.c_int), ("w_o", ctypes.c_void_p),
+                ("w_gate", ctypes.c_void_p), ("w_up", ctypes.c_void_p), ("w_down", ctypes.c_void_p),
+                ("w_router", ctypes.c_void_p)]
+
+
+class AflexError(RuntimeError):
+    def __init__(self, status: int, name: str, detail: str):
+        super().__init__(f"{name} ({status}): {detail}")
+        self.status = status
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """dlopen libaflex.so (built in-tree by ``build.py``).  Raises if missing."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} not found: build it with `python -m paper_2608_01891_b200.build` "
+                           "(there is no fallback path)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, ci, cs = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+    lib.aflex_status_string.restype = ctypes.c_char_p
+    lib.aflex_status_string.argtypes = [ci]
+    lib.aflex_version.restype = ci
+    lib.aflex_create.restype = ci
+    lib.aflex_create.argtypes = [ctypes.POINTER(vp), ci, cs]
+    lib.aflex_destroy.restype = ci
+    lib.aflex_destroy.argtypes = [vp]
+    lib.aflex_last_error.restype = ctypes.c_char_p
+    lib.aflex_last_error.argtypes = [vp]
+    lib.aflex_get_device_status.restype = ci
+    lib.aflex_get_device_status.argtypes = [vp, vp]
+    lib.aflex_set_attn_chunk.restype = ci
+    lib.aflex_set_attn_chunk.argtypes = [vp, ci]
+    lib.aflex_attn_decode.restype = ci
+    lib.aflex_attn_decode.argtypes = [vp, ctypes.POINTER(AttnDesc), vp, ctypes.POINTER(KV), ci, vp, vp, vp]
+    lib.aflex_linear.restype = ci
+    lib.aflex_linear.argtypes = [vp, vp, vp, ci, ci, ci, vp, vp]
+    lib.aflex_ffn_dense.restype = ci
+    lib.aflex_ffn_dense.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, vp, vp]
+    lib.aflex_ffn_moe.restype = ci
+    lib.aflex_ffn_moe.argtypes = [vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, vp, vp, vp, vp, vp]
+    lib.aflex_layer_step.restype = ci
+    lib.aflex_layer_step.argtypes = [vp, ctypes.POINTER(LayerDesc), vp, ctypes.POINTER(KV), ci, vp, ci,
+                                     ctypes.POINTER(ctypes.c_int32), vp, vp, vp]
+    lib.aflex_workspace_bytes.restype = cs
+    lib.aflex_workspace_bytes.argtypes = [ctypes.POINTER(LayerDesc), ci, ci]
+    _lib = lib
+    return lib
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    assert t.is_contiguous(), "tensors passed to aflex must be contiguous"
+    return t.data_ptr()
+
+
+def _stream(stream: Optional[torch.cuda.Stream]) -> int:
+    return (stream or torch.cuda.current_stream()).cuda_stream
+
+
+def attn_desc(num_q_heads: int, num_kv_heads: int, head_dim: int, sm_scale: float = 0.0) -> AttnDesc:
+    return AttnDesc(num_q_heads, num_kv_heads, head_dim, 16, sm_scale)
+
+
+def make_kv(k_cache: torch.Tensor, v_cache: torch.Tensor, page_table: torch.Tensor, seq_lens: torch.Tensor,
+            seq_lens_host: Optional[torch.Tensor] = None) -> KV:
+    """k_cache/v_cache bf16 CUDA [num_pages,Hkv,16,D]; page_table i32 CUDA [B,max_pages]; seq_lens i32 CUDA [B];
+    seq_lens_host optional i32 CPU [B].  The returned struct borrows the tensors: keep them alive."""
+    assert k_cache.dtype == torch.bfloat16 and v_cache.dtype == torch.bfloat16
+    assert page_table.dtype == torch.int32 and seq_lens.dtype == torch.int32
+    kv = KV(_ptr(k_cache), _ptr(v_cache), k_cache.shape[0], _ptr(page_table), page_table.shape[1],
+            _ptr(seq_lens), None)
+    if seq_lens_host is not None:
+        assert seq_lens_host.dtype == torch.int32 and seq_lens_host.device.type == "cpu"
+        kv.seq_lens_host = _ptr(seq_lens_host)
+    kv._keep = (k_cache, v_cache, page_table, seq_lens, seq_lens_host)
+    return kv
+
+
+def layer_desc(attn: AttnDesc, hidden: int, inter: int, w_o, w_gate, w_up, w_down, num_experts: int = 0,
+               top_k: int = 0, w_router=None) -> LayerDesc:
+    d = LayerDesc(attn, hidden, inter, num_experts, top_k, _ptr(w_o), _ptr(w_gate), _ptr(w_up), _ptr(w_down),
+                  _ptr(w_router))
+    d._keep = (w_o, w_gate, w_up, w_down, w_router)
+    return d
+
+
+def workspace_bytes(layer: LayerDesc, max_batch: int, max_pages_per_seq: int) -> int:
+    return int(load_library().aflex_workspace_bytes(ctypes.byref(layer), max_batch, max_pages_per_seq))
+
+
+class Context:
+    """Owns an aflex_ctx (device workspace, internal streams/events, status word)."""
+
+    def __init__(self, device: int = 0, workspace_bytes: int = 0):
+        self._lib = load_library()
+        self._h = ctypes.c_void_p()
+        st = self._lib.aflex_create(ctypes.byref(self._h), device, workspace_bytes)
+        if st != OK:
+            raise AflexError(st, self._lib.aflex_status_string(st).decode(), "aflex_create failed")
+        self.device = device
+
+    def close(self) -> None:
+        if getattr(self, "_h", None) and self._h.value:
+            self._lib.aflex_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, st: int) -> None:
+        if st != OK:
+            raise AflexError(st, self._lib.aflex_status_string(st).decode(),
+                             self._lib.aflex_last_error(self._h).decode())
+
+    def raw_call(self, name: str, *args) -> int:
+        """Call an entry point and return the raw status (for error-path tests)."""
+        return int(getattr(self._lib, name)(self._h, *args))
+
+    def last_error(self) -> str:
+        return self._lib.aflex_last_error(self._h).decode()
+
+    def device_status(self, stream=None) -> int:
+        return int(self._lib.aflex_get_device_status(self._h, _stream(stream)))
+
+    def set_attn_chunk(self, chunk_tokens: int) -> None:
+        self._check(self._lib.aflex_set_attn_chunk(self._h, chunk_tokens))
+
+    def attn_decode(self, desc: AttnDesc, q: torch.Tensor, kv: KV, out: torch.Tensor,
+                    lse: Optional[torch.Tensor] = None, stream=None) -> None:
+        self._check(self._lib.aflex_attn_decode(self._h, ctypes.byref(desc), _ptr(q), ctypes.byref(kv),
+                                                q.shape[0], _ptr(out), _ptr(lse), _stream(stream)))
+
+    def linear(self, x: torch.Tensor, w: torch.Tensor, y: torch.Tensor, stream=None) -> None:
+        T, K = x.shape
+        N = w.shape[0]
+        self._check(self._lib.aflex_linear(self._h, _ptr(x), _ptr(w), T, K, N, _ptr(y), _stream(stream)))
+
+    def ffn_dense(self, x, w_gate, w_up, w_down, y, stream=None) -> None:
+        T, H = x.shape
+        I = w_gate.shape[0]
+        self._check(self._lib.aflex_ffn_dense(self._h, _ptr(x), _ptr(w_gate), _ptr(w_up), _ptr(w_down), T, H, I,
+                                              _ptr(y), _stream(stream)))
+
+    def ffn_moe(self, x, w_gate, w_up, w_down, top_k: int, y, router_logits=None, w_router=None,
+                topk_idx=None, topk_gate=None, expert_counts=None, stream=None) -> None:
+        T, H = x.shape
+        E, I, _ = w_gate.shape
+        self._check(self._lib.aflex_ffn_moe(self._h, _ptr(x), _ptr(router_logits), _ptr(w_router), _ptr(w_gate),
+                                            _ptr(w_up), _ptr(w_down), T, H, I, E, top_k, _ptr(y), _ptr(topk_idx),
+                                            _ptr(topk_gate), _ptr(expert_counts), _stream(stream)))
+
+    def layer_step(self, layer: LayerDesc, q, kv: KV, y, microbatch_depth: int = 1,
+                   mb_offsets: Optional[Sequence[int]] = None, router_logits=None, attn_out=None,
+                   stream=None) -> None:
+        offs = None
+        if mb_offsets is not None:
+            offs = (ctypes.c_int32 * len(mb_offsets))(*[int(v) for v in mb_offsets])
+        self._check(self._lib.aflex_layer_step(self._h, ctypes.byref(layer), _ptr(q), ctypes.byref(kv), q.shape[0],
+                                               _ptr(router_logits), microbatch_depth, offs, _ptr(attn_out),
+                                               _ptr(y), _stream(stream)))

@@ -1,0 +1,466 @@
+// C-ABI entry points, the context and the A/F microbatch interleave.
+#include <cuda_bf16.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+
+#include "internal.h"
+
+namespace aflex {
+
+aflex_status set_error(aflex_ctx* ctx, aflex_status s, const char* fmt, ...) {
+    if (ctx) {
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(ctx->err, sizeof(ctx->err), fmt, ap);
+        va_end(ap);
+    }
+    return s;
+}
+
+aflex_status check_cuda(aflex_ctx* ctx, cudaError_t e, const char* what) {
+    if (e == cudaSuccess) return AFLEX_OK;
+    return set_error(ctx, AFLEX_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+bool encode_tmap_2d_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t row_stride_bytes,
+                         uint32_t box_rows, uint32_t box_cols, bool promote_l2_256) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {row_stride_bytes};
+    cuuint32_t box[2] = {box_cols, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                    promote_l2_256 ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+static aflex_status validate_attn(aflex_ctx* ctx, const aflex_attn_desc* d, const void* q, const aflex_kv* kv, int batch,
+                                  const void* out) {
+    if (!ctx) return AFLEX_ERR_INVALID_ARG;
+    if (!d || !q || !kv || !out) return set_error(ctx, AFLEX_ERR_INVALID_ARG, "attention: null argument");
+    if (!kv->k_cache || !kv->v_cache || !kv->page_table || !kv->seq_lens)
+        return set_error(ctx, AFLEX_ERR_INVALID_ARG, "attention: null KV argument");
+    if (batch < 1 || kv->num_pages < 1 || kv->max_pages_per_seq < 1)
+        return set_error(ctx, AFLEX_ERR_INVALID_ARG, "attention: batch, num_pages and max_pages_per_seq must be >= 1");
+    if (d->num_q_heads < 1 || d->num_kv_heads < 1 || d->num_q_heads % d->num_kv_heads != 0)
+        return set_error(ctx, AFLEX_ERR_INVALID_ARG, "attention: Hkv must divide Hq");
+    if (!aligned16(q) || !aligned16(out) || !aligned16(kv->k_cache) || !aligned16(kv->v_cache))
+        return set_error(ctx, AFLEX_ERR_INVALID_ARG, "attention: pointers must be 16-byte aligned");
+    const int G = d->num_q_heads / d->num_kv_heads;
+    if (d->head_dim != 64 && d->head_dim != 128)
+        return set_error(ctx, AFLEX_ERR_UNSUPPORTED, "attention: head_dim %d (supported: 64, 128)", d->head_dim);
+    if (d->page_size != 16) return set_error(ctx, AFLEX_ERR_UNSUPPORTED, "attention: page_size %d (supported: 16)", d->page_size);
+    if (G != 1 && G != 2 && G != 4 && G != 8)
+        return set_error(ctx, AFLEX_ERR_UNSUPPORTED, "attention: Hq/Hkv = %d (supported: 1, 2, 4, 8)", G);
+    if (batch > 65535) return set_error(ctx, AFLEX_ERR_UNSUPPORTED, "attention: batch > 65535");
+    if ((long long)kv->num_pages * d->num_kv_heads * 16 >= (1LL << 31))
+        return set_error(ctx, AFLEX_ERR_UNSUPPORTED, "attention: KV pool has more than 2^31 token rows");
+    if (kv->seq_lens_host) {
+        const long long max_len = (long long)kv->max_pages_per_seq * 16;
+        for (int b = 0; b < batch; ++b)
+            if (kv->seq_lens_host[b] < 1 || kv->seq_lens_host[b] > max_len)
+                return set_error(ctx, AFLEX_ERR_INVALID_ARG, "attention: seq_lens_host[%d] = %d outside [1, %lld]", b,
+                                 kv->seq_lens_host[b], max_len);
+    }
+    return AFLEX_OK;
+}
+
+static aflex_status validate_ffn_dims(aflex_ctx* ctx, int T, int H, int I) {
+    if (T < 1 || H < 1 || I < 1) return set_error(ctx, AFLEX_ERR_INVALID_ARG, "ffn: T, H, I must be >= 1");
+    if (H % 8 || I % 8) return set_error(ctx, AFLEX_ERR_UNSUPPORTED, "ffn: H and I must be multiples of 8");
+    return AFLEX_OK;
+}
+
+// ---- F side, shared by the stand-alone entry points and the layer step -----------------------
+static size_t dense_ws_bytes(int T, int H, int I, int num_sms) {
+    return align256((size_t)T * I * 2) + linear_workspace_bytes(T, I, H, num_sms);
+}
+
+static aflex_status dense_run(aflex_ctx* ctx, const void* x, const void* wg, const void* wu, const void* wd, int T,
+                              int H, int I, void* y, char* ws, size_t ws_bytes, cudaStream_t st) {
+    Arena arena(ws, ws_bytes);
+    __nv_bfloat16* h = arena.take<__nv_bfloat16>((size_t)T * I);
+    const size_t lin = linear_workspace_bytes(T, I, H, ctx->num_sms);
+    char* lws = lin ? arena.take<char>(lin) : nullptr;
+    if (arena.overflow)
+        return set_error(ctx, AFLEX_ERR_WORKSPACE, "dense ffn: need %zu workspace bytes, have %zu",
+                         dense_ws_bytes(T, H, I, ctx->num_sms), ws_bytes);
+    aflex_status s = gateup_launch(ctx, x, wg, wu, T, H, I, h, nullptr, 0, st);
+    if (s != AFLEX_OK) return s;
+    return linear_launch(ctx, h, wd, T, I, H, y, lws, lin, st);
+}
+
+static size_t moe_ws_bytes(int T, int H, int I, int E, int K, int num_sms) {
+    const size_t R = (size_t)T * K;
+    size_t b = 0;
+    b += align256(R * 4) * 3;                   // idx, gate, pos
+    b += align256((size_t)E * 4) + align256((size_t)(E + 1) * 4);
+    b += align256((size_t)T * E * 4);           // logits
+    b += align256(R * H * 2);                   // xp
+    b += align256(R * I * 2);                   // hp
+    b += align256(R * H * 4);                   // yp
+    b += grouped_workspace_bytes((int)R, T, I, H, E, num_sms);
+    return b;
+}
+
+static aflex_status moe_run(aflex_ctx* ctx, const void* x, const float* router_logits, const void* w_router,
+                            const void* wg, const void* wu, const void* wd, int T, int H, int I, int E, int K, void* y,
+                            int32_t* topk_idx, float* topk_gate, int32_t* expert_counts, char* ws, size_t ws_bytes,
+                            cudaStream_t st) {
+    const size_t R = (size_t)T * K;
+    Arena arena(ws, ws_bytes);
+    MoeBuffers mb;
+    mb.idx = arena.take<int32_t>(R);
+    mb.gate = arena.take<float>(R);
+    mb.pos = arena.take<int32_t>(R);
+    mb.counts = arena.take<int32_t>(E);
+    mb.offsets = arena.take<int32_t>(E + 1);
+    mb.logits = arena.take<float>((size_t)T * E);
+    __nv_bfloat16* xp = arena.take<__nv_bfloat16>(R * H);
+    __nv_bfloat16* hp = arena.take<__nv_bfloat16>(R * I);
+    float* yp = arena.take<float>(R * H);
+    const size_t gws = grouped_workspace_bytes((int)R, T, I, H, E, ctx->num_sms);
+    char* gw = gws ? arena.take<char>(gws) : nullptr;
+    if (arena.overflow)
+        return set_error(ctx, AFLEX_ERR_WORKSPACE, "moe ffn: need %zu workspace bytes, have %zu",
+                         moe_ws_bytes(T, H, I, E, K, ctx->num_sms), ws_bytes);
+    aflex_status s;
+    const float* logits = router_logits;
+    if (!logits) {
+        s = moe_router_logits_launch(ctx, x, w_router, T, H, E, mb.logits, st);
+        if (s != AFLEX_OK) return s;
+        logits = mb.logits;
+    }
+    s = moe_route_launch(ctx, logits, T, E, K, mb, st);
+    if (s != AFLEX_OK) return s;
+    s = moe_gather_launch(ctx, x, mb.pos, T, K, H, xp, st);
+    if (s != AFLEX_OK) return s;
+    // an expert receives at most one assignment per token => segments have at most T rows
+    s = grouped_gateup_launch(ctx, xp, wg, wu, mb.offsets, (int)R, T, H, I, E, hp, nullptr, 0, st);
+    if (s != AFLEX_OK) return s;
+    s = grouped_linear_launch(ctx, hp, wd, mb.offsets, (int)R, T, I, H, E, yp, gw, gws, st);
+    if (s != AFLEX_OK) return s;
+    s = moe_combine_launch(ctx, yp, mb.pos, mb.gate, T, K, H, y, st);
+    if (s != AFLEX_OK) return s;
+    if (topk_idx) { s = check_cuda(ctx, cudaMemcpyAsync(topk_idx, mb.idx, R * 4, cudaMemcpyDeviceToDevice, st), "copy topk_idx"); if (s != AFLEX_OK) return s; }
+    if (topk_gate) { s = check_cuda(ctx, cudaMemcpyAsync(topk_gate, mb.gate, R * 4, cudaMemcpyDeviceToDevice, st), "copy topk_gate"); if (s != AFLEX_OK) return s; }
+    if (expert_counts) { s = check_cuda(ctx, cudaMemcpyAsync(expert_counts, mb.counts, (size_t)E * 4, cudaMemcpyDeviceToDevice, st), "copy expert_counts"); if (s != AFLEX_OK) return s; }
+    return AFLEX_OK;
+}
+
+static aflex_status validate_moe(aflex_ctx* ctx, int T, int H, int I, int E, int K) {
+    aflex_status s = validate_ffn_dims(ctx, T, H, I);
+    if (s != AFLEX_OK) return s;
+    if (E < 1 || K < 1) return set_error(ctx, AFLEX_ERR_INVALID_ARG, "moe: E and top_k must be >= 1");
+    if (K > E) return set_error(ctx, AFLEX_ERR_INVALID_ARG, "moe: top_k > num_experts");
+    if (E > 64 || K > 2) return set_error(ctx, AFLEX_ERR_UNSUPPORTED, "moe: supported E <= 64, top_k in {1,2}");
+    return AFLEX_OK;
+}
+
+}  // namespace aflex
+
+using namespace aflex;
+
+extern "C" {
+
+const char* aflex_status_string(aflex_status s) {
+    switch (s) {
+        case AFLEX_OK: return "AFLEX_OK";
+        case AFLEX_ERR_INVALID_ARG: return "AFLEX_ERR_INVALID_ARG";
+        case AFLEX_ERR_UNSUPPORTED: return "AFLEX_ERR_UNSUPPORTED";
+        case AFLEX_ERR_WORKSPACE: return "AFLEX_ERR_WORKSPACE";
+        case AFLEX_ERR_CUDA: return "AFLEX_ERR_CUDA";
+        case AFLEX_ERR_TIMEOUT: return "AFLEX_ERR_TIMEOUT";
+        case AFLEX_ERR_BOUNDS: return "AFLEX_ERR_BOUNDS";
+    }
+    return "AFLEX_ERR_UNKNOWN";
+}
+
+int aflex_version(void) { return 100; }
+
+aflex_status aflex_create(aflex_ctx** out, int device, size_t workspace_bytes) {
+    if (!out) return AFLEX_ERR_INVALID_ARG;
+    *out = nullptr;
+    aflex_ctx* ctx = new (std::nothrow) aflex_ctx();
+    if (!ctx) return AFLEX_ERR_CUDA;
+    ctx->device = device;
+    ctx->ws_bytes = workspace_bytes ? align256(workspace_bytes) : kDefaultWorkspace;
+    cudaError_t e = cudaSetDevice(device);
+    cudaDeviceProp prop;
+    if (e == cudaSuccess) e = cudaGetDeviceProperties(&prop, device);
+    if (e == cudaSuccess) {
+        ctx->num_sms = prop.multiProcessorCount;
+        if (prop.major != 10) {
+            delete ctx;
+            return AFLEX_ERR_UNSUPPORTED;   // kernels are built for sm_100a only
+        }
+    }
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->ws, ctx->ws_bytes);
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->dev_status, sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(ctx->dev_status, 0, sizeof(int));
+    if (e == cudaSuccess) e = cudaMallocHost(&ctx->host_status, sizeof(int));
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->stream_a, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->stream_f, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_entry, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_a_done, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_f_done, cudaEventDisableTiming);
+    for (int i = 0; i < kMaxMicrobatches && e == cudaSuccess; ++i)
+        e = cudaEventCreateWithFlags(&ctx->ev_a[i], cudaEventDisableTiming);
+    if (e != cudaSuccess || !get_encode_fn()) {
+        aflex_destroy(ctx);
+        return AFLEX_ERR_CUDA;
+    }
+    *out = ctx;
+    return AFLEX_OK;
+}
+
+aflex_status aflex_destroy(aflex_ctx* ctx) {
+    if (!ctx) return AFLEX_OK;
+    cudaSetDevice(ctx->device);
+    if (ctx->stream_a) cudaStreamSynchronize(ctx->stream_a);
+    if (ctx->stream_f) cudaStreamSynchronize(ctx->stream_f);
+    for (int i = 0; i < kMaxMicrobatches; ++i) if (ctx->ev_a[i]) cudaEventDestroy(ctx->ev_a[i]);
+    if (ctx->ev_entry) cudaEventDestroy(ctx->ev_entry);
+    if (ctx->ev_a_done) cudaEventDestroy(ctx->ev_a_done);
+    if (ctx->ev_f_done) cudaEventDestroy(ctx->ev_f_done);
+    if (ctx->stream_a) cudaStreamDestroy(ctx->stream_a);
+    if (ctx->stream_f) cudaStreamDestroy(ctx->stream_f);
+    if (ctx->host_status) cudaFreeHost(ctx->host_status);
+    if (ctx->dev_status) cudaFree(ctx->dev_status);
+    if (ctx->ws) cudaFree(ctx->ws);
+    delete ctx;
+    return AFLEX_OK;
+}
+
+const char* aflex_last_error(const aflex_ctx* ctx) { return ctx ? ctx->err : "null context"; }
+
+aflex_status aflex_get_device_status(aflex_ctx* ctx, void* stream) {
+    if (!ctx) return AFLEX_ERR_INVALID_ARG;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(ctx->host_status, ctx->dev_status, sizeof(int), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(ctx->dev_status, 0, sizeof(int), st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return check_cuda(ctx, e, "aflex_get_device_status");
+    const int v = *ctx->host_status;
+    if (v != 0) set_error(ctx, (aflex_status)v, "device status word = %d (%s)", v, aflex_status_string((aflex_status)v));
+    return (aflex_status)v;
+}
+
+aflex_status aflex_set_attn_chunk(aflex_ctx* ctx, int chunk_tokens) {
+    if (!ctx || chunk_tokens < 0) return AFLEX_ERR_INVALID_ARG;
+    ctx->attn_chunk = chunk_tokens;
+    return AFLEX_OK;
+}
+
+aflex_status aflex_attn_decode(aflex_ctx* ctx, const aflex_attn_desc* desc, const void* q, const aflex_kv* kv, int batch,
+                               void* out, float* lse, void* stream) {
+    aflex_status s = validate_attn(ctx, desc, q, kv, batch, out);
+    if (s != AFLEX_OK) return s;
+    return attn_decode_launch(ctx, desc, q, kv, batch, out, lse, ctx->ws, ctx->ws_bytes,
+                              reinterpret_cast<cudaStream_t>(stream));
+}
+
+aflex_status aflex_linear(aflex_ctx* ctx, const void* x, const void* w, int T, int K, int N, void* y, void* stream) {
+    if (!ctx) return AFLEX_ERR_INVALID_ARG;
+    if (!x || !w || !y || T < 1 || K < 1 || N < 1) return set_error(ctx, AFLEX_ERR_INVALID_ARG, "linear: bad argument");
+    if (K % 8 || N % 8) return set_error(ctx, AFLEX_ERR_UNSUPPORTED, "linear: K and N must be multiples of 8");
+    if (!aligned16(x) || !aligned16(w) || !aligned16(y)) return set_error(ctx, AFLEX_ERR_INVALID_ARG, "linear: pointers must be 16-byte aligned");
+    return linear_launch(ctx, x, w, T, K, N, y, ctx->ws, ctx->ws_bytes, reinterpret_cast<cudaStream_t>(stream));
+}
+
+aflex_status aflex_ffn_dense(aflex_ctx* ctx, const void* x, const void* w_gate, const void* w_up, const void* w_down,
+                             int T, int H, int I, void* y, void* stream) {
+    if (!ctx) return AFLEX_ERR_INVALID_ARG;
+    if (!x || !w_gate || !w_up || !w_down || !y) return set_error(ctx, AFLEX_ERR_INVALID_ARG, "dense ffn: null argument");
+    aflex_status s = validate_ffn_dims(ctx, T, H, I);
+    if (s != AFLEX_OK) return s;
+    if (!aligned16(x) || !aligned16(w_gate) || !aligned16(w_up) || !aligned16(w_down) || !aligned16(y))
+        return set_error(ctx, AFLEX_ERR_INVALID_ARG, "dense ffn: pointers must be 16-byte aligned");
+    return dense_run(ctx, x, w_gate, w_up, w_down, T, H, I, y, ctx->ws, ctx->ws_bytes,
+                     reinterpret_cast<cudaStream_t>(stream));
+}
+
+aflex_status aflex_ffn_moe(aflex_ctx* ctx, const void* x, const float* router_logits, const void* w_router,
+                           const void* w_gate, const void* w_up, const void* w_down, int T, int H, int I, int E, int top_k,
+                           void* y, int32_t* topk_idx, float* topk_gate, int32_t* expert_counts, void* stream) {
+    if (!ctx) return AFLEX_ERR_INVALID_ARG;
+    if (!x || !w_gate || !w_up || !w_down || !y) return set_error(ctx, AFLEX_ERR_INVALID_ARG, "moe ffn: null argument");
+    if ((router_logits == nullptr) == (w_router == nullptr))
+        return set_error(ctx, AFLEX_ERR_INVALID_ARG, "moe ffn: exactly one of router_logits and w_router must be given");
+    aflex_status s = validate_moe(ctx, T, H, I, E, top_k);
+    if (s != AFLEX_OK) return s;
+    if (!aligned16(x) || !aligned16(w_gate) || !aligned16(w_up) || !aligned16(w_down) || !aligned16(y))
+        return set_error(ctx, AFLEX_ERR_INVALID_ARG, "moe ffn: pointers must be 16-byte aligned");
+    return moe_run(ctx, x, router_logits, w_router, w_gate, w_up, w_down, T, H, I, E, top_k, y, topk_idx, topk_gate,
+                   expert_counts, ctx->ws, ctx->ws_bytes, reinterpret_cast<cudaStream_t>(stream));
+}
+
+// Workspace layout of the layer step: [A region | attention output a | boundary x | F region].
+// The A region (attention partials, W_o split-K partials) is used only on the attention stream,
+// the F region only on the FFN stream; a and x are indexed by batch row, so microbatches touch
+// disjoint slices.
+namespace {
+struct LayerWs {
+    size_t a_attn, a_lin, a_total, attn_out, x, f_total, total;
+};
+// a_attn: bytes the attention partials need (the caller knows the chunk plan).
+LayerWs layer_ws(const aflex_layer_desc* L, int max_batch, size_t a_attn, int num_sms) {
+    LayerWs w;
+    const int A = L->attn.num_q_heads * L->attn.head_dim;
+    w.a_attn = a_attn;
+    w.a_lin = L->w_o ? linear_workspace_bytes(max_batch, A, L->hidden, num_sms) : 0;
+    // split-K plans depend on T; take the max over the microbatch sizes 1..max_batch that matter
+    if (L->w_o) {
+        for (int t = 1; t <= max_batch; t = t < 16 ? t + 1 : t + 16) {
+            size_t b = linear_workspace_bytes(t, A, L->hidden, num_sms);
+            if (b > w.a_lin) w.a_lin = b;
+        }
+    }
+    w.a_total = w.a_attn + w.a_lin;
+    w.attn_out = align256((size_t)max_batch * A * 2);
+    w.x = L->w_o ? align256((size_t)max_batch * L->hidden * 2) : 0;
+    size_t f = 0;
+    for (int t = 1; t <= max_batch; t = t < 16 ? t + 1 : t + 16) {
+        size_t b = L->num_experts == 0 ? dense_ws_bytes(t, L->hidden, L->inter, num_sms)
+                                       : moe_ws_bytes(t, L->hidden, L->inter, L->num_experts, L->top_k, num_sms);
+        if (b > f) f = b;
+    }
+    {
+        size_t b = L->num_experts == 0 ? dense_ws_bytes(max_batch, L->hidden, L->inter, num_sms)
+                                       : moe_ws_bytes(max_batch, L->hidden, L->inter, L->num_experts, L->top_k, num_sms);
+        if (b > f) f = b;
+    }
+    w.f_total = f;
+    w.total = w.a_total + w.attn_out + w.x + w.f_total + 1024;
+    return w;
+}
+}  // namespace
+
+size_t aflex_workspace_bytes(const aflex_layer_desc* layer, int max_batch, int max_pages_per_seq) {
+    if (!layer || max_batch < 1 || max_pages_per_seq < 1) return 0;
+    // the planner never picks a chunk below 128 tokens: size the partials for that worst case
+    const long long max_len = (long long)max_pages_per_seq * 16;
+    const int max_chunks = (int)((max_len + 127) / 128);
+    return layer_ws(layer, max_batch, attn_workspace_bytes(&layer->attn, max_batch, max_chunks), 148).total;
+}
+
+aflex_status aflex_layer_step(aflex_ctx* ctx, const aflex_layer_desc* L, const void* q, const aflex_kv* kv, int batch,
+                              const float* router_logits, int M, const int32_t* mb_offsets, void* attn_out, void* y,
+                              void* stream) {
+    if (!ctx) return AFLEX_ERR_INVALID_ARG;
+    if (!L || !y) return set_error(ctx, AFLEX_ERR_INVALID_ARG, "layer step: null argument");
+    aflex_status s = validate_attn(ctx, &L->attn, q, kv, batch, y);
+    if (s != AFLEX_OK) return s;
+    const int A = L->attn.num_q_heads * L->attn.head_dim;
+    const int H = L->hidden, I = L->inter, E = L->num_experts, K = L->top_k;
+    if (!L->w_gate || !L->w_up || !L->w_down) return set_error(ctx, AFLEX_ERR_INVALID_ARG, "layer step: null FFN weights");
+    if (!L->w_o && A != H) return set_error(ctx, AFLEX_ERR_INVALID_ARG, "layer step: w_o is required when Hq*D != hidden");
+    if (A % 8) return set_error(ctx, AFLEX_ERR_UNSUPPORTED, "layer step: Hq*D must be a multiple of 8");
+    if (E == 0) s = validate_ffn_dims(ctx, batch, H, I);
+    else {
+        s = validate_moe(ctx, batch, H, I, E, K);
+        if (s == AFLEX_OK && (router_logits == nullptr) == (L->w_router == nullptr))
+            s = set_error(ctx, AFLEX_ERR_INVALID_ARG, "layer step: exactly one of router_logits and w_router must be given");
+    }
+    if (s != AFLEX_OK) return s;
+    if (M < 1 || M > batch || M > kMaxMicrobatches)
+        return set_error(ctx, AFLEX_ERR_INVALID_ARG, "layer step: microbatch depth %d outside [1, min(batch, %d)]", M, kMaxMicrobatches);
+    int32_t offs[kMaxMicrobatches + 1];
+    if (mb_offsets) {
+        for (int i = 0; i <= M; ++i) offs[i] = mb_offsets[i];
+        if (offs[0] != 0 || offs[M] != batch) return set_error(ctx, AFLEX_ERR_INVALID_ARG, "layer step: mb_offsets must run from 0 to batch");
+        for (int i = 0; i < M; ++i)
+            if (offs[i + 1] <= offs[i]) return set_error(ctx, AFLEX_ERR_INVALID_ARG, "layer step: mb_offsets must be strictly increasing");
+    } else {
+        const int base = batch / M, extra = batch % M;
+        offs[0] = 0;
+        for (int i = 0; i < M; ++i) offs[i + 1] = offs[i] + base + (i < extra ? 1 : 0);
+    }
+
+    size_t a_attn = 0;
+    for (int i = 0; i < M; ++i) {
+        aflex_kv kvi = *kv;
+        kvi.seq_lens_host = kv->seq_lens_host ? kv->seq_lens_host + offs[i] : nullptr;
+        const int rows = offs[i + 1] - offs[i];
+        const AttnPlan plan = attn_make_plan(ctx, &L->attn, &kvi, rows);
+        const size_t b = attn_workspace_bytes(&L->attn, rows, plan.max_chunks);
+        if (b > a_attn) a_attn = b;
+    }
+    const LayerWs w = layer_ws(L, batch, a_attn, ctx->num_sms);
+    if (w.total > ctx->ws_bytes)
+        return set_error(ctx, AFLEX_ERR_WORKSPACE, "layer step: need %zu workspace bytes, have %zu", w.total, ctx->ws_bytes);
+    char* ws_a = ctx->ws;
+    char* ws_alin = ws_a + w.a_attn;
+    __nv_bfloat16* a_buf = attn_out ? reinterpret_cast<__nv_bfloat16*>(attn_out)
+                                    : reinterpret_cast<__nv_bfloat16*>(ctx->ws + w.a_total);
+    __nv_bfloat16* x_buf = L->w_o ? reinterpret_cast<__nv_bfloat16*>(ctx->ws + w.a_total + w.attn_out) : a_buf;
+    char* ws_f = ctx->ws + w.a_total + w.attn_out + w.x;
+
+    cudaStream_t user = reinterpret_cast<cudaStream_t>(stream);
+    cudaStream_t sa = ctx->stream_a, sf = ctx->stream_f;
+    cudaError_t e = cudaEventRecord(ctx->ev_entry, user);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(sa, ctx->ev_entry, 0);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(sf, ctx->ev_entry, 0);
+    if (e != cudaSuccess) return check_cuda(ctx, e, "layer step: entry join");
+
+    const int Hq = L->attn.num_q_heads, D = L->attn.head_dim;
+    for (int i = 0; i < M; ++i) {
+        const int r0 = offs[i], rows = offs[i + 1] - offs[i];
+        // ---- A_i on the attention stream
+        aflex_kv kvi = *kv;
+        kvi.page_table = kv->page_table + (size_t)r0 * kv->max_pages_per_seq;
+        kvi.seq_lens = kv->seq_lens + r0;
+        kvi.seq_lens_host = kv->seq_lens_host ? kv->seq_lens_host + r0 : nullptr;
+        const __nv_bfloat16* qi = reinterpret_cast<const __nv_bfloat16*>(q) + (size_t)r0 * Hq * D;
+        s = attn_decode_launch(ctx, &L->attn, qi, &kvi, rows, a_buf + (size_t)r0 * A, nullptr, ws_a, w.a_attn, sa);
+        if (s != AFLEX_OK) return s;
+        if (L->w_o) {
+            s = linear_launch(ctx, a_buf + (size_t)r0 * A, L->w_o, rows, A, H, x_buf + (size_t)r0 * H, ws_alin, w.a_lin, sa);
+            if (s != AFLEX_OK) return s;
+        }
+        e = cudaEventRecord(ctx->ev_a[i], sa);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(sf, ctx->ev_a[i], 0);
+        if (e != cudaSuccess) return check_cuda(ctx, e, "layer step: A->F event");
+        // ---- F_i on the FFN stream
+        __nv_bfloat16* yi = reinterpret_cast<__nv_bfloat16*>(y) + (size_t)r0 * H;
+        const __nv_bfloat16* xi = x_buf + (size_t)r0 * H;
+        if (E == 0) {
+            s = dense_run(ctx, xi, L->w_gate, L->w_up, L->w_down, rows, H, I, yi, ws_f, w.f_total, sf);
+        } else {
+            s = moe_run(ctx, xi, router_logits ? router_logits + (size_t)r0 * E : nullptr, L->w_router, L->w_gate,
+                        L->w_up, L->w_down, rows, H, I, E, K, yi, nullptr, nullptr, nullptr, ws_f, w.f_total, sf);
+        }
+        if (s != AFLEX_OK) return s;
+    }
+    e = cudaEventRecord(ctx->ev_a_done, sa);
+    if (e == cudaSuccess) e = cudaEventRecord(ctx->ev_f_done, sf);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(user, ctx->ev_a_done, 0);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(user, ctx->ev_f_done, 0);
+    return check_cuda(ctx, e, "layer step: exit join");
+}
+
+}  // extern "C"

@@ -1,0 +1,112 @@
+// Host-side internals shared by the translation units of libaflex: the context,
+// the workspace arena, tensor-map encoding and the launchers each .cu file exports.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/aflex.h"
+
+namespace aflex {
+
+constexpr int kMaxMicrobatches = 64;
+constexpr size_t kDefaultWorkspace = (size_t)256 << 20;
+constexpr int kMaxDynamicSmem = 227 * 1024;   // opt-in shared memory per CTA on sm_100
+
+}  // namespace aflex
+
+struct aflex_ctx {
+    int device = 0;
+    int num_sms = 148;
+    size_t ws_bytes = 0;
+    char* ws = nullptr;           // device workspace
+    int* dev_status = nullptr;    // device status word (0 = OK)
+    int* host_status = nullptr;   // pinned mirror used by aflex_get_device_status
+    cudaStream_t stream_a = nullptr, stream_f = nullptr;
+    cudaEvent_t ev_entry = nullptr;
+    cudaEvent_t ev_a[aflex::kMaxMicrobatches] = {};
+    cudaEvent_t ev_f_done = nullptr, ev_a_done = nullptr;
+    int attn_chunk = 0;           // 0 = automatic
+    bool gemm_attr_set[2] = {false, false};
+    bool attn_attr_set[2] = {false, false};
+    char err[512] = {0};
+};
+
+namespace aflex {
+
+aflex_status set_error(aflex_ctx* ctx, aflex_status s, const char* fmt, ...);
+aflex_status check_cuda(aflex_ctx* ctx, cudaError_t e, const char* what);
+
+// Bump allocator over a byte range of the ctx workspace (256-byte granules).
+struct Arena {
+    char* base;
+    size_t size;
+    size_t used = 0;
+    bool overflow = false;
+    Arena(char* b, size_t s) : base(b), size(s) {}
+    template <typename T>
+    T* take(size_t n) {
+        size_t bytes = (n * sizeof(T) + 255) & ~(size_t)255;
+        if (used + bytes > size) { overflow = true; return nullptr; }
+        T* p = reinterpret_cast<T*>(base + used);
+        used += bytes;
+        return p;
+    }
+};
+inline size_t align256(size_t b) { return (b + 255) & ~(size_t)255; }
+
+// Encode a 2-D bf16 tiled tensor map: rows x cols (cols contiguous), box_rows x box_cols,
+// 128-byte swizzle (box_cols * 2 must be 128).  Returns false on driver error.
+bool encode_tmap_2d_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t row_stride_bytes,
+                         uint32_t box_rows, uint32_t box_cols, bool promote_l2_256);
+
+// ---- attention (attn_decode.cu)
+struct AttnPlan {
+    int chunk_tokens;      // C, multiple of 64
+    int max_chunks;        // ceil(16*max_pages_per_seq / C)
+};
+AttnPlan attn_make_plan(const aflex_ctx* ctx, const aflex_attn_desc* d, const aflex_kv* kv, int batch);
+size_t attn_workspace_bytes(const aflex_attn_desc* d, int batch, int max_chunks);
+aflex_status attn_decode_launch(aflex_ctx* ctx, const aflex_attn_desc* d, const void* q, const aflex_kv* kv,
+                                int batch, void* out, float* lse, char* ws, size_t ws_bytes, cudaStream_t st);
+
+// ---- GEMM (gemm_tcgen05.cu)
+// y[T][N] = x[T][K] . w[N][K]^T (bf16 in, fp32 accumulate, bf16 out).
+size_t linear_workspace_bytes(int T, int K, int N, int num_sms);
+aflex_status linear_launch(aflex_ctx* ctx, const void* x, const void* w, int T, int K, int N, void* y, char* ws,
+                           size_t ws_bytes, cudaStream_t st);
+// h[T][I] = silu(x Wg^T) .* (x Wu^T)
+size_t gateup_workspace_bytes(int T, int H, int I, int num_sms);
+aflex_status gateup_launch(aflex_ctx* ctx, const void* x, const void* w_gate, const void* w_up, int T, int H, int I,
+                           void* h, char* ws, size_t ws_bytes, cudaStream_t st);
+
+// Grouped (per-expert) variants over permuted rows.  `offsets` is a device array [E+1]
+// (row segment of expert e = [offsets[e], offsets[e+1])); rows_max bounds any segment.
+size_t grouped_workspace_bytes(int rows_total, int rows_max, int K, int N, int E, int num_sms);
+aflex_status grouped_gateup_launch(aflex_ctx* ctx, const void* xp, const void* w_gate, const void* w_up,
+                                   const int32_t* offsets, int rows_total, int rows_max, int H, int I, int E,
+                                   void* hp, char* ws, size_t ws_bytes, cudaStream_t st);
+aflex_status grouped_linear_launch(aflex_ctx* ctx, const void* hp, const void* w_down, const int32_t* offsets,
+                                   int rows_total, int rows_max, int K, int N, int E, float* yp, char* ws,
+                                   size_t ws_bytes, cudaStream_t st);
+
+// ---- MoE glue (moe.cu)
+struct MoeBuffers {
+    int32_t* idx;      // [T][K]
+    float* gate;       // [T][K]
+    int32_t* counts;   // [E]
+    int32_t* offsets;  // [E+1]
+    int32_t* pos;      // [T][K]
+    float* logits;     // [T][E] (router GEMM output when w_router is used)
+};
+aflex_status moe_router_logits_launch(aflex_ctx* ctx, const void* x, const void* w_router, int T, int H, int E,
+                                      float* logits, cudaStream_t st);
+aflex_status moe_route_launch(aflex_ctx* ctx, const float* logits, int T, int E, int K, const MoeBuffers& mb,
+                              cudaStream_t st);
+aflex_status moe_gather_launch(aflex_ctx* ctx, const void* x, const int32_t* pos, int T, int K, int H, void* xp,
+                               cudaStream_t st);
+aflex_status moe_combine_launch(aflex_ctx* ctx, const float* yp, const int32_t* pos, const float* gate, int T,
+                                int K, int H, void* y, cudaStream_t st);
+
+}  // namespace aflex
