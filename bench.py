@@ -1,0 +1,371 @@
+#!/usr/bin/env python
+"""Benchmark of the A/F decode-layer hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config C] [--depth M]
+
+A "step" is one pass of the whole hot path -- aflex_layer_step: paged GQA decode attention,
+the W_o boundary projection and the dense (or MoE) SwiGLU FFN -- over one decode batch of
+seeded synthetic input.  The default workload is configuration 2 (Qwen3-32B-shaped layer,
+batch 32, context lengths U[512,4096], page size 16, shuffled page table), microbatch depth 1.
+Prints ONE JSON line:
+
+  value        decode-layer tokens/s, inputs resident in HBM, CUDA events around K steps
+  e2e          the same with q / page table / sequence lengths copied from pinned host memory
+               and y copied back, every step, inside the timed region
+  roofline     the dominant kernel's achieved HBM rate against the measured copy bandwidth
+  kernels      the same figures for every kernel kind of the step
+  cpu_baseline the fp64 oracle timed on this machine's host cores on a bounded sample
+
+With --gpus N > 1 (under torchrun) every rank runs an independent replica of the step on its
+own GPU (the path has no exchange step on one node); value = N * B / max-over-ranks time.
+--impl reference times the CPU oracle instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2608_01891_b200 import inputs as IN  # noqa: E402
+
+METRIC = "decode-layer tokens/s (Qwen3-32B shape); attn HBM GB/s & FFN TFLOPS % of peak"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "50", "-i", str(self.index)],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) >= 7:
+                self.rows.append(parts)
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.12)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def algorithmic_bytes(cfg, lens, M):
+    """Algorithmic HBM bytes per launch of each kernel kind (every K/V element and every weight read
+    once; activations, partial results and outputs once each).  Per step, per microbatch launch."""
+    B, Hq, D, H, I = cfg.batch, cfg.num_q_heads, cfg.head_dim, cfg.hidden, cfg.inter
+    A = Hq * D
+    kv = float(np.sum(lens.astype(np.int64)) * cfg.kv_bytes_per_token) + 2.0 * B * A * 2 + float(np.sum((lens + 15) // 16)) * 4
+    out = {"attn_partial": kv / M}
+    rows = B / M
+    out["linear_gemm"] = H * A * 2 + rows * (A + H) * 2
+    if cfg.num_experts == 0:
+        out["gateup_gemm"] = 2.0 * I * H * 2 + rows * (H + I) * 2
+        out["down_gemm"] = 1.0 * H * I * 2 + rows * (I + H) * 2
+    else:
+        E, K = cfg.num_experts, cfg.top_k
+        out["moe_gateup_gemm"] = 2.0 * E * I * H * 2 + rows * K * (H + I) * 2
+        out["moe_down_gemm"] = 1.0 * E * H * I * 2 + rows * K * (I * 2 + H * 4)
+    return out
+
+
+def algorithmic_flops(cfg, M):
+    B, Hq, D, H, I = cfg.batch, cfg.num_q_heads, cfg.head_dim, cfg.hidden, cfg.inter
+    rows = B / M
+    k = cfg.top_k if cfg.num_experts else 1
+    return {"linear_gemm": 2.0 * rows * H * Hq * D, "gateup_gemm": 4.0 * rows * H * I, "down_gemm": 2.0 * rows * H * I,
+            "moe_gateup_gemm": 4.0 * rows * k * H * I, "moe_down_gemm": 2.0 * rows * k * H * I}
+
+
+def build_workload(cfg, device):
+    """Everything resident in HBM before the timed region starts."""
+    from paper_2608_01891_b200 import aflex as AF
+    kvh = IN.make_paged_kv(cfg, device=device)
+    q = IN.make_q(cfg, device=device)
+    wo = IN.make_wo(cfg, device=device)
+    wg, wu, wd = IN.make_ffn_weights(cfg, device=device)
+    logits = IN.make_router_logits(cfg).to(device) if cfg.num_experts else None
+    table = kvh.page_table.to(device)
+    lens = kvh.seq_lens.to(device)
+    kv = AF.make_kv(kvh.k_cache, kvh.v_cache, table, lens, kvh.seq_lens)
+    layer = AF.layer_desc(AF.attn_desc(cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim), cfg.hidden, cfg.inter,
+                          wo, wg, wu, wd, cfg.num_experts, cfg.top_k)
+    y = torch.zeros(cfg.batch, cfg.hidden, dtype=torch.bfloat16, device=device)
+    return dict(kvh=kvh, q=q, wo=wo, wg=wg, wu=wu, wd=wd, logits=logits, table=table, lens=lens, kv=kv,
+                layer=layer, y=y)
+
+
+def oracle_sample(cfg, wl, rows):
+    """Time the fp64 oracle's layer step on the sampled batch rows.  Returns (seconds, threads)."""
+    from oracle import oracle as O
+    kvh = wl["kvh"]
+    table, lens = kvh.page_table.numpy(), kvh.seq_lens.numpy()
+    ids, new_rows, o = [], [], 0
+    mp = max((int(lens[b]) + 15) // 16 for b in rows)
+    for b in rows:
+        n = (int(lens[b]) + 15) // 16
+        ids.extend(table[b, :n].tolist())
+        r = np.zeros(mp, dtype=np.int32); r[:n] = np.arange(o, o + n); new_rows.append(r); o += n
+    sel = torch.as_tensor(np.asarray(ids, dtype=np.int64), device=kvh.k_cache.device)
+    u16 = lambda t: IN.bf16_bits(t.detach().cpu().contiguous())
+    k, v = u16(kvh.k_cache.index_select(0, sel)), u16(kvh.v_cache.index_select(0, sel))
+    q = u16(wl["q"][list(rows)])
+    wo, wg, wu, wd = u16(wl["wo"]), u16(wl["wg"]), u16(wl["wu"]), u16(wl["wd"])
+    logits = wl["logits"][list(rows)].cpu().numpy() if cfg.num_experts else None
+    t0 = time.perf_counter()
+    O.layer_step(q, k, v, np.stack(new_rows), lens[list(rows)].astype(np.int32), wo, wg, wu, wd,
+                 logits=logits, top_k=cfg.top_k)
+    return time.perf_counter() - t0, O.num_threads()
+
+
+def run_reference(args, cfg, rank, world):
+    """The CPU oracle as the reference arm: each step is a bounded sample of the workload."""
+    if rank != 0:
+        return
+    wl_cfg = cfg
+    kvh = IN.make_paged_kv(wl_cfg)
+    wl = dict(kvh=kvh, q=IN.make_q(wl_cfg), wo=IN.make_wo(wl_cfg), logits=IN.make_router_logits(wl_cfg) if wl_cfg.num_experts else None)
+    wl["wg"], wl["wu"], wl["wd"] = IN.make_ffn_weights(wl_cfg)
+    rows = list(range(min(args.ref_rows, cfg.batch)))
+    times, threads = [], 1
+    for i in range(args.warmup + args.steps):
+        dt, threads = oracle_sample(cfg, wl, rows)
+        if i >= args.warmup:
+            times.append(dt)
+    ms = 1e3 * float(np.mean(times))
+    value = len(rows) / (ms * 1e-3)
+    sample = f"layer step on batch rows {rows[0]}..{rows[-1]} of {cfg.batch} (rows are independent)"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"config {cfg.cfg_id}: {cfg.name}", "batch": cfg.batch, "microbatch_depth": 1,
+                       "sampled_rows": len(rows)},
+            "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=2, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--depth", type=int, default=1, help="microbatch depth M")
+    ap.add_argument("--attn-chunk", type=int, default=0)
+    ap.add_argument("--ref-rows", type=int, default=0,
+                    help="batch rows per reference/cpu-baseline sample (0 = about 15e9 multiply-adds of oracle work)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+
+    if args.ref_rows <= 0:
+        c = IN.CONFIGS[args.config]
+        macs_row = (c.num_q_heads * c.head_dim * (2 * (c.len_lo + c.len_hi) // 2 + c.hidden)
+                    + 3 * c.hidden * c.inter * max(1, c.top_k))
+        args.ref_rows = int(max(1, min(c.batch, 15e9 // macs_row)))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    cfg = IN.CONFIGS[args.config]
+
+    if args.impl == "reference":
+        run_reference(args, cfg, rank, world)
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    from paper_2608_01891_b200 import aflex as AF
+    torch.cuda.set_device(local_rank)
+    device = f"cuda:{local_rank}"
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(device))
+
+    peaks = load_peaks()
+    wl = build_workload(cfg, device)
+    lens_np = wl["kvh"].seq_lens.numpy()
+    M = args.depth
+    ws = AF.workspace_bytes(wl["layer"], cfg.batch, wl["kvh"].max_pages_per_seq)
+    ctx = AF.Context(local_rank, ws)
+    if args.attn_chunk:
+        ctx.set_attn_chunk(args.attn_chunk)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        ctx.layer_step(wl["layer"], wl["q"], wl["kv"], wl["y"], M, None, wl["logits"], None, stream)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            fn()
+        e1.record(stream)
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if dist is not None:
+            t = torch.tensor([ms], device=device)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    # ---- device-resident timing (the headline value)
+    for _ in range(args.warmup):
+        step()
+    launches0 = ctx.launch_count()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    ms_total = timed(step, args.steps)
+    launches = ctx.launch_count() - launches0
+    # the timed region can be shorter than one nvidia-smi sampling period: keep the same load
+    # running (untimed) until the sampler has seen it
+    if ms_total < 500:
+        timed(step, int(500 / max(ms_total / args.steps, 1e-3)) + 1)
+    clocks = sampler.stop()
+    ms_step = ms_total / args.steps
+    value = world * cfg.batch / (ms_step * 1e-3)
+    assert ctx.device_status() == AF.OK, ctx.last_error()
+
+    # ---- per-kernel durations: the same K steps with an event pair around every launch
+    psteps = max(1, min(args.steps, 8192 // max(1, launches // args.steps)))
+    ctx.profile_enable(True)
+    timed(step, psteps)
+    prof = ctx.profile_read()
+    ctx.profile_enable(False)
+    abytes = algorithmic_bytes(cfg, lens_np, M)
+    aflops = algorithmic_flops(cfg, M)
+    kernels = {}
+    for name, (ms, n) in prof.items():
+        avg_us = 1e3 * ms / n
+        k = {"launches_per_step": n // psteps, "avg_us": round(avg_us, 2)}
+        if name in abytes:
+            k["gbs"] = round(abytes[name] / (avg_us * 1e-6) / 1e9, 1)
+            k["frac_hbm"] = round(k["gbs"] / peaks["hbm_gbs"], 4)
+        if name in aflops:
+            k["tflops"] = round(aflops[name] / (avg_us * 1e-6) / 1e12, 2)
+        kernels[name] = k
+    dom = max((n for n in kernels if "gbs" in kernels[n]), key=lambda n: kernels[n]["avg_us"] * kernels[n]["launches_per_step"])
+    roofline = {"kernel": dom, "bound": "hbm", "achieved": kernels[dom]["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": kernels[dom]["frac_hbm"], "traffic": None, "peak_source": peaks["source"],
+                "algorithmic_bytes_per_launch": abytes[dom]}
+    ncu_traffic = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(ncu_traffic):
+        tr = json.load(open(ncu_traffic))
+        key = f"config{cfg.cfg_id}/{dom}"
+        if key in tr:
+            roofline["traffic"] = tr[key]
+
+    # ---- end to end: per-step inputs come from pinned host memory, the result goes back
+    hq = wl["q"].cpu().pin_memory()
+    htab = wl["kvh"].page_table.pin_memory()
+    hlens = wl["kvh"].seq_lens.pin_memory()
+    hlog = wl["logits"].cpu().pin_memory() if wl["logits"] is not None else None
+    hy = torch.empty(cfg.batch, cfg.hidden, dtype=torch.bfloat16).pin_memory()
+    h2d = hq.numel() * 2 + htab.numel() * 4 + hlens.numel() * 4 + (hlog.numel() * 4 if hlog is not None else 0)
+    d2h = hy.numel() * 2
+
+    def step_e2e():
+        wl["q"].copy_(hq, non_blocking=True)
+        wl["table"].copy_(htab, non_blocking=True)
+        wl["lens"].copy_(hlens, non_blocking=True)
+        if hlog is not None:
+            wl["logits"].copy_(hlog, non_blocking=True)
+        ctx.layer_step(wl["layer"], wl["q"], wl["kv"], wl["y"], M, None, wl["logits"], None, stream)
+        hy.copy_(wl["y"], non_blocking=True)
+        stream.synchronize()          # the caller consumes y before the next decode step
+
+    for _ in range(3):
+        step_e2e()
+    ms_e2e = timed(step_e2e, args.steps) / args.steps
+    e2e = {"value": world * cfg.batch / (ms_e2e * 1e-3), "unit": "tokens/s", "ms_per_step": ms_e2e,
+           "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+
+    # ---- CPU baseline: the oracle on a bounded sample, rank 0 at N = 1 only
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        rows = list(range(min(args.ref_rows, cfg.batch)))
+        dt, threads = oracle_sample(cfg, wl, rows)
+        cpu = {"value": len(rows) / dt, "unit": "tokens/s", "cores": threads, "kind": "oracle", "seconds": round(dt, 2),
+               "sample": f"fp64 oracle layer step on batch rows {rows[0]}..{rows[-1]} of {cfg.batch} (rows are independent)"}
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "config": {"workload": f"config {cfg.cfg_id}: {cfg.name}", "batch": cfg.batch, "microbatch_depth": M,
+                           "hq_hkv_d": [cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim], "hidden": cfg.hidden,
+                           "inter": cfg.inter, "experts": cfg.num_experts, "top_k": cfg.top_k,
+                           "context_tokens": int(lens_np.sum()), "page_size": 16,
+                           "l2": "inputs larger than L2 (KV + weights >> 126 MB), no flush",
+                           "parallelism": "replicas only" if world > 1 else "1 GPU"},
+                "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "kernels": kernels,
+                "cpu_baseline": cpu}
+        print(json.dumps(line), flush=True)
+    ctx.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -205,9 +205,9 @@ typedef struct {
 /*
  * q bf16 [B][Hq][D]; kv as for aflex_attn_decode (rows of page_table/seq_lens
  * are per sequence, sliced per microbatch); router_logits fp32 [B][E] or NULL.
- * microbatch_depth = M >= 1, M <= batch.  mb_offsets: HOST i32 [M+1],
- * non-decreasing... strictly increasing from 0 to batch, or NULL for the
- * near-equal split (the first batch % M microbatches get one extra row).
+ * microbatch_depth = M >= 1, M <= min(batch, 64).  mb_offsets: HOST i32 [M+1],
+ * strictly increasing from 0 to batch, or NULL for the near-equal split (the
+ * first batch % M microbatches get one extra row).
  * attn_out bf16 [B][Hq][D]: optional copy of the A-side output (NULL => kept
  * in the workspace).  y bf16 [B][hidden].
  * `stream` is joined on entry (the internal streams wait for it) and on exit
@@ -235,6 +235,25 @@ AFLEX_API aflex_status aflex_linear(aflex_ctx* ctx, const void* x, const void* w
 
 /* Tuning knob: tokens per split-KV chunk (multiple of 64; 0 = automatic). */
 AFLEX_API aflex_status aflex_set_attn_chunk(aflex_ctx* ctx, int chunk_tokens);
+
+/* ---- Measurement support (no counterpart in the paper's method; the per-operator latency
+ * profiling of its Section 4.1 is the motivation) --------------------------------------------
+ *
+ * The library launches a fixed set of kernel kinds (attention partial / combine, the GEMMs,
+ * the MoE glue).  Launches are always counted per kind.  With profiling enabled every launch
+ * is additionally bracketed by a CUDA event pair on the stream it runs on (at most 8192
+ * launches are kept per enable); aflex_profile_read waits for those events and sums the
+ * device time per kind.  Enabling allocates events: do it outside timed regions.
+ */
+AFLEX_API int aflex_num_kernel_kinds(void);
+AFLEX_API const char* aflex_kernel_name(int kind);
+/* Launches of `kind` since the ctx was created; kind < 0 => all kinds together. */
+AFLEX_API long long aflex_launch_count(const aflex_ctx* ctx, int kind);
+/* on != 0: clear collected samples and start collecting; on == 0: stop collecting. */
+AFLEX_API aflex_status aflex_profile_enable(aflex_ctx* ctx, int on);
+/* Blocks until the collected launches of `kind` have finished; returns their summed device
+ * time (ms) and their number. */
+AFLEX_API aflex_status aflex_profile_read(aflex_ctx* ctx, int kind, double* total_ms, long long* launches);
 
 #ifdef __cplusplus
 }

@@ -22,7 +22,8 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_
 EXPORTS = (
     "aflex_status_string", "aflex_version", "aflex_create", "aflex_destroy", "aflex_last_error",
     "aflex_get_device_status", "aflex_attn_decode", "aflex_ffn_dense", "aflex_ffn_moe", "aflex_layer_step",
-    "aflex_workspace_bytes", "aflex_linear", "aflex_set_attn_chunk",
+    "aflex_workspace_bytes", "aflex_linear", "aflex_set_attn_chunk", "aflex_num_kernel_kinds",
+    "aflex_kernel_name", "aflex_launch_count", "aflex_profile_enable", "aflex_profile_read",
 )
 
 
@@ -89,6 +90,15 @@ def load_library() -> ctypes.CDLL:
                                      ctypes.POINTER(ctypes.c_int32), vp, vp, vp]
     lib.aflex_workspace_bytes.restype = cs
     lib.aflex_workspace_bytes.argtypes = [ctypes.POINTER(LayerDesc), ci, ci]
+    lib.aflex_num_kernel_kinds.restype = ci
+    lib.aflex_kernel_name.restype = ctypes.c_char_p
+    lib.aflex_kernel_name.argtypes = [ci]
+    lib.aflex_launch_count.restype = ctypes.c_longlong
+    lib.aflex_launch_count.argtypes = [vp, ci]
+    lib.aflex_profile_enable.restype = ci
+    lib.aflex_profile_enable.argtypes = [vp, ci]
+    lib.aflex_profile_read.restype = ci
+    lib.aflex_profile_read.argtypes = [vp, ci, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_longlong)]
     _lib = lib
     return lib
 
@@ -171,6 +181,22 @@ class Context:
 
     def device_status(self, stream=None) -> int:
         return int(self._lib.aflex_get_device_status(self._h, _stream(stream)))
+
+    def launch_count(self, kind: int = -1) -> int:
+        return int(self._lib.aflex_launch_count(self._h, kind))
+
+    def profile_enable(self, on: bool) -> None:
+        self._check(self._lib.aflex_profile_enable(self._h, 1 if on else 0))
+
+    def profile_read(self) -> dict:
+        """{kernel kind name: (total device ms, launches)} for the launches collected since enable."""
+        out = {}
+        for k in range(self._lib.aflex_num_kernel_kinds()):
+            ms, n = ctypes.c_double(0.0), ctypes.c_longlong(0)
+            self._check(self._lib.aflex_profile_read(self._h, k, ctypes.byref(ms), ctypes.byref(n)))
+            if n.value:
+                out[self._lib.aflex_kernel_name(k).decode()] = (ms.value, n.value)
+        return out
 
     def set_attn_chunk(self, chunk_tokens: int) -> None:
         self._check(self._lib.aflex_set_attn_chunk(self._h, chunk_tokens))

@@ -111,7 +111,7 @@ static aflex_status dense_run(aflex_ctx* ctx, const void* x, const void* wg, con
                          dense_ws_bytes(T, H, I, ctx->num_sms), ws_bytes);
     aflex_status s = gateup_launch(ctx, x, wg, wu, T, H, I, h, nullptr, 0, st);
     if (s != AFLEX_OK) return s;
-    return linear_launch(ctx, h, wd, T, I, H, y, lws, lin, st);
+    return linear_launch(ctx, h, wd, T, I, H, y, lws, lin, st, kKDownGemm);
 }
 
 static size_t moe_ws_bytes(int T, int H, int I, int E, int K, int num_sms) {
@@ -249,6 +249,13 @@ aflex_status aflex_destroy(aflex_ctx* ctx) {
     if (ctx->ev_f_done) cudaEventDestroy(ctx->ev_f_done);
     if (ctx->stream_a) cudaStreamDestroy(ctx->stream_a);
     if (ctx->stream_f) cudaStreamDestroy(ctx->stream_f);
+    if (ctx->prof) {
+        for (int i = 0; i < kProfMaxSlots; ++i) {
+            if (ctx->prof[i].start) cudaEventDestroy(ctx->prof[i].start);
+            if (ctx->prof[i].stop) cudaEventDestroy(ctx->prof[i].stop);
+        }
+        delete[] ctx->prof;
+    }
     if (ctx->host_status) cudaFreeHost(ctx->host_status);
     if (ctx->dev_status) cudaFree(ctx->dev_status);
     if (ctx->ws) cudaFree(ctx->ws);
@@ -270,6 +277,54 @@ aflex_status aflex_get_device_status(aflex_ctx* ctx, void* stream) {
     return (aflex_status)v;
 }
 
+static const char* kKernelNames[kKKindCount] = {
+    "attn_partial", "attn_combine", "linear_gemm", "down_gemm", "gateup_gemm", "splitk_reduce", "router_logits",
+    "moe_route", "moe_gather", "moe_gateup_gemm", "moe_down_gemm", "moe_combine"};
+
+int aflex_num_kernel_kinds(void) { return kKKindCount; }
+
+const char* aflex_kernel_name(int kind) { return (kind >= 0 && kind < kKKindCount) ? kKernelNames[kind] : "?"; }
+
+long long aflex_launch_count(const aflex_ctx* ctx, int kind) {
+    if (!ctx) return 0;
+    if (kind >= 0 && kind < kKKindCount) return ctx->launches[kind];
+    long long t = 0;
+    for (int i = 0; i < kKKindCount; ++i) t += ctx->launches[i];
+    return t;
+}
+
+aflex_status aflex_profile_enable(aflex_ctx* ctx, int on) {
+    if (!ctx) return AFLEX_ERR_INVALID_ARG;
+    if (on && !ctx->prof) {
+        ctx->prof = new (std::nothrow) ProfSlot[kProfMaxSlots]();
+        if (!ctx->prof) return set_error(ctx, AFLEX_ERR_CUDA, "profile: out of host memory");
+        for (int i = 0; i < kProfMaxSlots; ++i) {
+            cudaError_t e = cudaEventCreate(&ctx->prof[i].start);
+            if (e == cudaSuccess) e = cudaEventCreate(&ctx->prof[i].stop);
+            if (e != cudaSuccess) return check_cuda(ctx, e, "profile: cudaEventCreate");
+        }
+    }
+    if (on) ctx->prof_used = 0;
+    ctx->profiling = on != 0;
+    return AFLEX_OK;
+}
+
+aflex_status aflex_profile_read(aflex_ctx* ctx, int kind, double* total_ms, long long* launches) {
+    if (!ctx || !total_ms || !launches || kind < 0 || kind >= kKKindCount) return AFLEX_ERR_INVALID_ARG;
+    *total_ms = 0.0;
+    *launches = 0;
+    for (int i = 0; i < ctx->prof_used; ++i) {
+        if (ctx->prof[i].kind != kind) continue;
+        cudaError_t e = cudaEventSynchronize(ctx->prof[i].stop);
+        float ms = 0.f;
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, ctx->prof[i].start, ctx->prof[i].stop);
+        if (e != cudaSuccess) return check_cuda(ctx, e, "profile: event read");
+        *total_ms += ms;
+        *launches += 1;
+    }
+    return AFLEX_OK;
+}
+
 aflex_status aflex_set_attn_chunk(aflex_ctx* ctx, int chunk_tokens) {
     if (!ctx || chunk_tokens < 0) return AFLEX_ERR_INVALID_ARG;
     ctx->attn_chunk = chunk_tokens;
@@ -289,7 +344,7 @@ aflex_status aflex_linear(aflex_ctx* ctx, const void* x, const void* w, int T, i
     if (!x || !w || !y || T < 1 || K < 1 || N < 1) return set_error(ctx, AFLEX_ERR_INVALID_ARG, "linear: bad argument");
     if (K % 8 || N % 8) return set_error(ctx, AFLEX_ERR_UNSUPPORTED, "linear: K and N must be multiples of 8");
     if (!aligned16(x) || !aligned16(w) || !aligned16(y)) return set_error(ctx, AFLEX_ERR_INVALID_ARG, "linear: pointers must be 16-byte aligned");
-    return linear_launch(ctx, x, w, T, K, N, y, ctx->ws, ctx->ws_bytes, reinterpret_cast<cudaStream_t>(stream));
+    return linear_launch(ctx, x, w, T, K, N, y, ctx->ws, ctx->ws_bytes, reinterpret_cast<cudaStream_t>(stream), kKLinearGemm);
 }
 
 aflex_status aflex_ffn_dense(aflex_ctx* ctx, const void* x, const void* w_gate, const void* w_up, const void* w_down,
@@ -439,7 +494,7 @@ aflex_status aflex_layer_step(aflex_ctx* ctx, const aflex_layer_desc* L, const v
         s = attn_decode_launch(ctx, &L->attn, qi, &kvi, rows, a_buf + (size_t)r0 * A, nullptr, ws_a, w.a_attn, sa);
         if (s != AFLEX_OK) return s;
         if (L->w_o) {
-            s = linear_launch(ctx, a_buf + (size_t)r0 * A, L->w_o, rows, A, H, x_buf + (size_t)r0 * H, ws_alin, w.a_lin, sa);
+            s = linear_launch(ctx, a_buf + (size_t)r0 * A, L->w_o, rows, A, H, x_buf + (size_t)r0 * H, ws_alin, w.a_lin, sa, kKLinearGemm);
             if (s != AFLEX_OK) return s;
         }
         e = cudaEventRecord(ctx->ev_a[i], sa);

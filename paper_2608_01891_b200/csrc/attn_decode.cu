@@ -372,9 +372,13 @@ static aflex_status attn_launch_t(aflex_ctx* ctx, const aflex_attn_desc* d, cons
         ctx->attn_attr_set[ti] = true;
     }
     dim3 grid((unsigned)plan.max_chunks, (unsigned)d->num_kv_heads, (unsigned)batch);
-    attn_partial_kernel<D><<<grid, kAttnThreads, smem, st>>>(tk, tv, p);
+    {
+        KernelScope scope(ctx, kKAttnPartial, st);
+        attn_partial_kernel<D><<<grid, kAttnThreads, smem, st>>>(tk, tv, p);
+    }
     aflex_status s = check_cuda(ctx, cudaGetLastError(), "attn_partial_kernel launch");
     if (s != AFLEX_OK) return s;
+    KernelScope scope(ctx, kKAttnCombine, st);
     attn_combine_kernel<D><<<batch * d->num_q_heads, D, 0, st>>>(p.o_part, p.ml_part, kv->seq_lens, d->num_q_heads,
                                                                plan.chunk_tokens, plan.max_chunks,
                                                                reinterpret_cast<__nv_bfloat16*>(out), lse);

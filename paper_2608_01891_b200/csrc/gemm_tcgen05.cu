@@ -368,13 +368,14 @@ static bool make_config(int mode, int T, int N, int K, int rows_max, int E, int 
 
 template <int MODE>
 static aflex_status launch_gemm(aflex_ctx* ctx, const GemmConfig& cfg, const CUtensorMap& ta0, const CUtensorMap& ta1,
-                                const CUtensorMap& tb, cudaStream_t st) {
+                                const CUtensorMap& tb, cudaStream_t st, int kind) {
     if (!ctx->gemm_attr_set[MODE]) {
         cudaError_t e = cudaFuncSetAttribute(gemm_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              kMaxDynamicSmem);
         if (e != cudaSuccess) return check_cuda(ctx, e, "cudaFuncSetAttribute(gemm)");
         ctx->gemm_attr_set[MODE] = true;
     }
+    KernelScope scope(ctx, kind, st);
     gemm_kernel<MODE><<<cfg.grid, kGemmThreads, cfg.smem_bytes, st>>>(ta0, ta1, tb, cfg.p);
     return check_cuda(ctx, cudaGetLastError(), "gemm_kernel launch");
 }
@@ -384,6 +385,7 @@ static aflex_status run_reduce(aflex_ctx* ctx, const float* part, int splits, si
     const int threads = 256;
     const size_t n4 = (TN + 3) / 4;
     const int blocks = (int)((n4 + threads - 1) / threads);
+    KernelScope scope(ctx, kKSplitKReduce, st);
     splitk_reduce_kernel<<<blocks, threads, 0, st>>>(part, splits, TN, (__nv_bfloat16*)out_bf16, out_f32);
     return check_cuda(ctx, cudaGetLastError(), "splitk_reduce launch");
 }
@@ -395,7 +397,7 @@ size_t linear_workspace_bytes(int T, int K, int N, int num_sms) {
 }
 
 aflex_status linear_launch(aflex_ctx* ctx, const void* x, const void* w, int T, int K, int N, void* y, char* ws,
-                           size_t ws_bytes, cudaStream_t st) {
+                           size_t ws_bytes, cudaStream_t st, int kind) {
     GemmConfig cfg;
     if (!make_config(kLinear, T, N, K, T, 0, ctx->num_sms, true, &cfg))
         return set_error(ctx, AFLEX_ERR_UNSUPPORTED, "linear: no tile configuration fits");
@@ -415,7 +417,7 @@ aflex_status linear_launch(aflex_ctx* ctx, const void* x, const void* w, int T, 
     if (!encode_tmap_2d_bf16(&ta, w, (uint64_t)N, (uint64_t)K, (uint64_t)K * 2, kBlockM, kBlockK, true) ||
         !encode_tmap_2d_bf16(&tb, x, (uint64_t)T, (uint64_t)K, (uint64_t)K * 2, (uint32_t)p.n_tile, kBlockK, false))
         return set_error(ctx, AFLEX_ERR_CUDA, "linear: cuTensorMapEncodeTiled failed");
-    aflex_status s = launch_gemm<kLinear>(ctx, cfg, ta, ta, tb, st);
+    aflex_status s = launch_gemm<kLinear>(ctx, cfg, ta, ta, tb, st, kind);
     if (s != AFLEX_OK) return s;
     if (p.splits > 1) return run_reduce(ctx, p.out_f32, p.splits, (size_t)T * N, y, nullptr, st);
     return AFLEX_OK;
@@ -438,7 +440,7 @@ aflex_status gateup_launch(aflex_ctx* ctx, const void* x, const void* w_gate, co
         !encode_tmap_2d_bf16(&tu, w_up, (uint64_t)I, (uint64_t)H, (uint64_t)H * 2, kBlockM, kBlockK, true) ||
         !encode_tmap_2d_bf16(&tb, x, (uint64_t)T, (uint64_t)H, (uint64_t)H * 2, (uint32_t)p.n_tile, kBlockK, false))
         return set_error(ctx, AFLEX_ERR_CUDA, "gate/up: cuTensorMapEncodeTiled failed");
-    return launch_gemm<kGateUp>(ctx, cfg, tg, tu, tb, st);
+    return launch_gemm<kGateUp>(ctx, cfg, tg, tu, tb, st, kKGateUpGemm);
 }
 
 size_t grouped_workspace_bytes(int rows_total, int rows_max, int K, int N, int E, int num_sms) {
@@ -464,7 +466,7 @@ aflex_status grouped_gateup_launch(aflex_ctx* ctx, const void* xp, const void* w
         !encode_tmap_2d_bf16(&tu, w_up, (uint64_t)E * I, (uint64_t)H, (uint64_t)H * 2, kBlockM, kBlockK, true) ||
         !encode_tmap_2d_bf16(&tb, xp, (uint64_t)rows_total, (uint64_t)H, (uint64_t)H * 2, (uint32_t)p.n_tile, kBlockK, false))
         return set_error(ctx, AFLEX_ERR_CUDA, "grouped gate/up: cuTensorMapEncodeTiled failed");
-    return launch_gemm<kGateUp>(ctx, cfg, tg, tu, tb, st);
+    return launch_gemm<kGateUp>(ctx, cfg, tg, tu, tb, st, kKMoeGateUpGemm);
 }
 
 aflex_status grouped_linear_launch(aflex_ctx* ctx, const void* hp, const void* w_down, const int32_t* offsets,
@@ -489,7 +491,7 @@ aflex_status grouped_linear_launch(aflex_ctx* ctx, const void* hp, const void* w
     if (!encode_tmap_2d_bf16(&ta, w_down, (uint64_t)E * N, (uint64_t)K, (uint64_t)K * 2, kBlockM, kBlockK, true) ||
         !encode_tmap_2d_bf16(&tb, hp, (uint64_t)rows_total, (uint64_t)K, (uint64_t)K * 2, (uint32_t)p.n_tile, kBlockK, false))
         return set_error(ctx, AFLEX_ERR_CUDA, "grouped linear: cuTensorMapEncodeTiled failed");
-    aflex_status s = launch_gemm<kLinear>(ctx, cfg, ta, ta, tb, st);
+    aflex_status s = launch_gemm<kLinear>(ctx, cfg, ta, ta, tb, st, kKMoeDownGemm);
     if (s != AFLEX_OK) return s;
     if (p.splits > 1) return run_reduce(ctx, p.out_f32, p.splits, (size_t)rows_total * N, nullptr, yp, st);
     return AFLEX_OK;

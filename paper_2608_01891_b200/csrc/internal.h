@@ -16,6 +16,16 @@ constexpr int kMaxDynamicSmem = 227 * 1024;   // opt-in shared memory per CTA on
 
 }  // namespace aflex
 
+namespace aflex {
+// Kernel kinds, for launch counting and optional per-kernel event timing.
+enum KernelKind {
+    kKAttnPartial = 0, kKAttnCombine, kKLinearGemm, kKDownGemm, kKGateUpGemm, kKSplitKReduce, kKRouterLogits,
+    kKMoeRoute, kKMoeGather, kKMoeGateUpGemm, kKMoeDownGemm, kKMoeCombine, kKKindCount
+};
+constexpr int kProfMaxSlots = 8192;
+struct ProfSlot { cudaEvent_t start, stop; int kind; };
+}  // namespace aflex
+
 struct aflex_ctx {
     int device = 0;
     int num_sms = 148;
@@ -31,12 +41,31 @@ struct aflex_ctx {
     bool gemm_attr_set[2] = {false, false};
     bool attn_attr_set[2] = {false, false};
     char err[512] = {0};
+    // launch counters (always on) and event-pair timing of every launch (when profiling is enabled)
+    long long launches[aflex::kKKindCount] = {};
+    bool profiling = false;
+    aflex::ProfSlot* prof = nullptr;   // kProfMaxSlots pre-created event pairs
+    int prof_used = 0;
 };
 
 namespace aflex {
 
 aflex_status set_error(aflex_ctx* ctx, aflex_status s, const char* fmt, ...);
 aflex_status check_cuda(aflex_ctx* ctx, cudaError_t e, const char* what);
+
+// Brackets one kernel launch: counts it, and records an event pair on its stream when profiling.
+struct KernelScope {
+    aflex_ctx* ctx; cudaStream_t st; int slot;
+    KernelScope(aflex_ctx* c, int kind, cudaStream_t s) : ctx(c), st(s), slot(-1) {
+        ctx->launches[kind]++;
+        if (ctx->profiling && ctx->prof_used < kProfMaxSlots) {
+            slot = ctx->prof_used++;
+            ctx->prof[slot].kind = kind;
+            cudaEventRecord(ctx->prof[slot].start, st);
+        }
+    }
+    ~KernelScope() { if (slot >= 0) cudaEventRecord(ctx->prof[slot].stop, st); }
+};
 
 // Bump allocator over a byte range of the ctx workspace (256-byte granules).
 struct Arena {
@@ -75,7 +104,7 @@ aflex_status attn_decode_launch(aflex_ctx* ctx, const aflex_attn_desc* d, const 
 // y[T][N] = x[T][K] . w[N][K]^T (bf16 in, fp32 accumulate, bf16 out).
 size_t linear_workspace_bytes(int T, int K, int N, int num_sms);
 aflex_status linear_launch(aflex_ctx* ctx, const void* x, const void* w, int T, int K, int N, void* y, char* ws,
-                           size_t ws_bytes, cudaStream_t st);
+                           size_t ws_bytes, cudaStream_t st, int kind);
 // h[T][I] = silu(x Wg^T) .* (x Wu^T)
 size_t gateup_workspace_bytes(int T, int H, int I, int num_sms);
 aflex_status gateup_launch(aflex_ctx* ctx, const void* x, const void* w_gate, const void* w_up, int T, int H, int I,

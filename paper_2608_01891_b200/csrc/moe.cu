@@ -157,6 +157,7 @@ aflex_status moe_router_logits_launch(aflex_ctx* ctx, const void* x, const void*
     const int warps = T * E;
     const int threads = 256;
     const int blocks = (warps * 32 + threads - 1) / threads;
+    KernelScope scope(ctx, kKRouterLogits, st);
     router_logits_kernel<<<blocks, threads, 0, st>>>((const __nv_bfloat16*)x, (const __nv_bfloat16*)w_router, T, H, E,
                                                      logits);
     return check_cuda(ctx, cudaGetLastError(), "router_logits_kernel launch");
@@ -164,6 +165,7 @@ aflex_status moe_router_logits_launch(aflex_ctx* ctx, const void* x, const void*
 
 aflex_status moe_route_launch(aflex_ctx* ctx, const float* logits, int T, int E, int K, const MoeBuffers& mb,
                               cudaStream_t st) {
+    KernelScope scope(ctx, kKMoeRoute, st);
     moe_route_kernel<<<1, kRouteThreads, 0, st>>>(logits, T, E, K, mb.idx, mb.gate, mb.counts, mb.offsets, mb.pos,
                                                   nullptr);
     return check_cuda(ctx, cudaGetLastError(), "moe_route_kernel launch");
@@ -171,12 +173,14 @@ aflex_status moe_route_launch(aflex_ctx* ctx, const float* logits, int T, int E,
 
 aflex_status moe_gather_launch(aflex_ctx* ctx, const void* x, const int32_t* pos, int T, int K, int H, void* xp,
                                cudaStream_t st) {
+    KernelScope scope(ctx, kKMoeGather, st);
     moe_gather_kernel<<<T * K, 128, 0, st>>>((const __nv_bfloat16*)x, pos, K, H, (__nv_bfloat16*)xp);
     return check_cuda(ctx, cudaGetLastError(), "moe_gather_kernel launch");
 }
 
 aflex_status moe_combine_launch(aflex_ctx* ctx, const float* yp, const int32_t* pos, const float* gate, int T, int K,
                                 int H, void* y, cudaStream_t st) {
+    KernelScope scope(ctx, kKMoeCombine, st);
     moe_combine_kernel<<<T, 256, 0, st>>>(yp, pos, gate, K, H, (__nv_bfloat16*)y);
     return check_cuda(ctx, cudaGetLastError(), "moe_combine_kernel launch");
 }
