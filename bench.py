@@ -100,6 +100,20 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def max_over_ranks(ms: float, dist, device) -> float:
+    """Slowest rank's time: the job is only as fast as its slowest replica."""
+    if dist is None:
+        return ms
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tokens_per_s(world: int, batch_per_rank: int, ms_per_step: float) -> float:
+    """Weak scaling over independent replicas: every rank decodes its own batch each step."""
+    return world * batch_per_rank / (ms_per_step * 1e-3)
+
+
 def algorithmic_bytes(cfg, lens, M):
     """Algorithmic HBM bytes per launch of each kernel kind (every K/V element and every weight read
     once; activations, partial results and outputs once each).  Per step, per microbatch launch."""
@@ -263,12 +277,7 @@ def main():
             fn()
         e1.record(stream)
         barrier()
-        ms = e0.elapsed_time(e1)
-        if dist is not None:
-            t = torch.tensor([ms], device=device)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return max_over_ranks(e0.elapsed_time(e1), dist, device)
 
     # ---- device-resident timing (the headline value)
     for _ in range(args.warmup):
@@ -284,7 +293,7 @@ def main():
         timed(step, int(500 / max(ms_total / args.steps, 1e-3)) + 1)
     clocks = sampler.stop()
     ms_step = ms_total / args.steps
-    value = world * cfg.batch / (ms_step * 1e-3)
+    value = whole_job_tokens_per_s(world, cfg.batch, ms_step)
     assert ctx.device_status() == AF.OK, ctx.last_error()
 
     # ---- per-kernel durations: the same K steps with an event pair around every launch
@@ -338,7 +347,7 @@ def main():
     for _ in range(3):
         step_e2e()
     ms_e2e = timed(step_e2e, args.steps) / args.steps
-    e2e = {"value": world * cfg.batch / (ms_e2e * 1e-3), "unit": "tokens/s", "ms_per_step": ms_e2e,
+    e2e = {"value": whole_job_tokens_per_s(world, cfg.batch, ms_e2e), "unit": "tokens/s", "ms_per_step": ms_e2e,
            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
 
     # ---- CPU baseline: the oracle on a bounded sample, rank 0 at N = 1 only
