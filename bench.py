@@ -120,7 +120,7 @@ def algorithmic_bytes(cfg, lens, M):
     B, Hq, D, H, I = cfg.batch, cfg.num_q_heads, cfg.head_dim, cfg.hidden, cfg.inter
     A = Hq * D
     kv = float(np.sum(lens.astype(np.int64)) * cfg.kv_bytes_per_token) + 2.0 * B * A * 2 + float(np.sum((lens + 15) // 16)) * 4
-    out = {"attn_partial": kv / M}
+    out = {"attn_decode": kv / M}
     rows = B / M
     out["linear_gemm"] = H * A * 2 + rows * (A + H) * 2
     if cfg.num_experts == 0:
@@ -218,7 +218,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2, choices=[1, 2, 3, 4, 5])
     ap.add_argument("--depth", type=int, default=1, help="microbatch depth M")
-    ap.add_argument("--attn-chunk", type=int, default=0)
+    ap.add_argument("--attn-ctas", type=int, default=0, help="persistent attention CTAs (0 = two per SM)")
     ap.add_argument("--ref-rows", type=int, default=0,
                     help="batch rows per reference/cpu-baseline sample (0 = about 15e9 multiply-adds of oracle work)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -256,8 +256,8 @@ def main():
     M = args.depth
     ws = AF.workspace_bytes(wl["layer"], cfg.batch, wl["kvh"].max_pages_per_seq)
     ctx = AF.Context(local_rank, ws)
-    if args.attn_chunk:
-        ctx.set_attn_chunk(args.attn_chunk)
+    if args.attn_ctas:
+        ctx.set_attn_ctas(args.attn_ctas)
     stream = torch.cuda.current_stream()
 
     def step():

@@ -107,8 +107,8 @@ AFLEX_API aflex_status aflex_get_device_status(aflex_ctx* ctx, void* stream);
  * j%16.  No mask (the n cached tokens include the one being decoded), no
  * positional term.  Slots beyond a sequence's length and pages no sequence
  * references may hold anything (including NaN) and do not affect the output.
- * The work is split over KV chunks and merged by a combine pass; the result is
- * deterministic run to run.
+ * The KV cache is split evenly over persistent CTAs and split sequences are merged in a fixed
+ * order; the result is deterministic run to run.
  */
 typedef struct {
     int num_q_heads;   /* Hq */
@@ -132,7 +132,7 @@ typedef struct {
  * q   bf16 [batch][Hq][D]            (device, read)
  * out bf16 [batch][Hq][D]            (device, written)
  * lse fp32 [batch][Hq] or NULL       (device, written when non-NULL)
- * Uses the ctx workspace for the per-chunk partial results.
+ * Uses the ctx workspace for per-CTA partial results (a few MB, independent of batch and context).
  * Errors: INVALID_ARG (null pointers, batch < 1, a host seq_len outside its
  * range), UNSUPPORTED (envelope), WORKSPACE.
  */
@@ -233,8 +233,9 @@ AFLEX_API size_t aflex_workspace_bytes(const aflex_layer_desc* layer, int max_ba
 AFLEX_API aflex_status aflex_linear(aflex_ctx* ctx, const void* x, const void* w, int T, int K, int N,
                                     void* y, void* stream);
 
-/* Tuning knob: tokens per split-KV chunk (multiple of 64; 0 = automatic). */
-AFLEX_API aflex_status aflex_set_attn_chunk(aflex_ctx* ctx, int chunk_tokens);
+/* Tuning knob: number of persistent attention CTAs per launch, 1..4096 (0 = automatic: two per
+ * SM).  It changes how the KV cache is split across CTAs, never the result beyond rounding. */
+AFLEX_API aflex_status aflex_set_attn_ctas(aflex_ctx* ctx, int ctas);
 
 /* ---- Measurement support (no counterpart in the paper's method; the per-operator latency
  * profiling of its Section 4.1 is the motivation) --------------------------------------------
@@ -254,6 +255,16 @@ AFLEX_API aflex_status aflex_profile_enable(aflex_ctx* ctx, int on);
 /* Blocks until the collected launches of `kind` have finished; returns their summed device
  * time (ms) and their number. */
 AFLEX_API aflex_status aflex_profile_read(aflex_ctx* ctx, int kind, double* total_ms, long long* launches);
+
+/*
+ * Timeline debugging.  When the ctx was created with the environment variable AFLEX_TRACE=1,
+ * the attention and GEMM kernels record a few %globaltimer stamps per CTA (CTA start, grid
+ * dependency satisfied, loads issued, last MMA issued, epilogue end) into a ring of 64 launch
+ * records of [4096 CTAs][8] uint64 each.  aflex_trace_read synchronises the device, copies the
+ * first `launches` records to host_out (launches * 4096 * 8 uint64), reports how many launches
+ * were recorded since the last read in *next_slot, and rewinds the ring.
+ */
+AFLEX_API aflex_status aflex_trace_read(aflex_ctx* ctx, unsigned long long* host_out, int launches, int* next_slot);
 
 #ifdef __cplusplus
 }

@@ -22,8 +22,9 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_
 EXPORTS = (
     "aflex_status_string", "aflex_version", "aflex_create", "aflex_destroy", "aflex_last_error",
     "aflex_get_device_status", "aflex_attn_decode", "aflex_ffn_dense", "aflex_ffn_moe", "aflex_layer_step",
-    "aflex_workspace_bytes", "aflex_linear", "aflex_set_attn_chunk", "aflex_num_kernel_kinds",
+    "aflex_workspace_bytes", "aflex_linear", "aflex_set_attn_ctas", "aflex_num_kernel_kinds",
     "aflex_kernel_name", "aflex_launch_count", "aflex_profile_enable", "aflex_profile_read",
+    "aflex_trace_read",
 )
 
 
@@ -75,8 +76,8 @@ def load_library() -> ctypes.CDLL:
     lib.aflex_last_error.argtypes = [vp]
     lib.aflex_get_device_status.restype = ci
     lib.aflex_get_device_status.argtypes = [vp, vp]
-    lib.aflex_set_attn_chunk.restype = ci
-    lib.aflex_set_attn_chunk.argtypes = [vp, ci]
+    lib.aflex_set_attn_ctas.restype = ci
+    lib.aflex_set_attn_ctas.argtypes = [vp, ci]
     lib.aflex_attn_decode.restype = ci
     lib.aflex_attn_decode.argtypes = [vp, ctypes.POINTER(AttnDesc), vp, ctypes.POINTER(KV), ci, vp, vp, vp]
     lib.aflex_linear.restype = ci
@@ -198,8 +199,17 @@ class Context:
                 out[self._lib.aflex_kernel_name(k).decode()] = (ms.value, n.value)
         return out
 
-    def set_attn_chunk(self, chunk_tokens: int) -> None:
-        self._check(self._lib.aflex_set_attn_chunk(self._h, chunk_tokens))
+    def trace_read(self, launches: int):
+        """(records uint64 [launches, 4096, 8], launches recorded since the last read); needs AFLEX_TRACE=1."""
+        import numpy as np
+        buf = np.zeros((launches, 4096, 8), dtype=np.uint64)
+        n = ctypes.c_int(0)
+        self._lib.aflex_trace_read.restype = ctypes.c_int
+        self._check(self._lib.aflex_trace_read(self._h, ctypes.c_void_p(buf.ctypes.data), launches, ctypes.byref(n)))
+        return buf, n.value
+
+    def set_attn_ctas(self, ctas: int) -> None:
+        self._check(self._lib.aflex_set_attn_ctas(self._h, ctas))
 
     def attn_decode(self, desc: AttnDesc, q: torch.Tensor, kv: KV, out: torch.Tensor,
                     lse: Optional[torch.Tensor] = None, stream=None) -> None:

@@ -2,6 +2,7 @@
 #include <cuda_bf16.h>
 #include <stdarg.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <new>
@@ -97,21 +98,24 @@ static aflex_status validate_ffn_dims(aflex_ctx* ctx, int T, int H, int I) {
 
 // ---- F side, shared by the stand-alone entry points and the layer step -----------------------
 static size_t dense_ws_bytes(int T, int H, int I, int num_sms) {
-    return align256((size_t)T * I * 2) + linear_workspace_bytes(T, I, H, num_sms);
+    const size_t gu = gateup_workspace_bytes(T, H, I, num_sms), dn = linear_workspace_bytes(T, I, H, num_sms);
+    return align256((size_t)T * I * 2) + (gu > dn ? gu : dn);
 }
 
 static aflex_status dense_run(aflex_ctx* ctx, const void* x, const void* wg, const void* wu, const void* wd, int T,
                               int H, int I, void* y, char* ws, size_t ws_bytes, cudaStream_t st) {
     Arena arena(ws, ws_bytes);
     __nv_bfloat16* h = arena.take<__nv_bfloat16>((size_t)T * I);
-    const size_t lin = linear_workspace_bytes(T, I, H, ctx->num_sms);
-    char* lws = lin ? arena.take<char>(lin) : nullptr;
+    // the two GEMMs run back to back on one stream: they share one scratch region and one counter array
+    const size_t gu = gateup_workspace_bytes(T, H, I, ctx->num_sms), dn = linear_workspace_bytes(T, I, H, ctx->num_sms);
+    const size_t scratch = gu > dn ? gu : dn;
+    char* sws = scratch ? arena.take<char>(scratch) : nullptr;
     if (arena.overflow)
         return set_error(ctx, AFLEX_ERR_WORKSPACE, "dense ffn: need %zu workspace bytes, have %zu",
                          dense_ws_bytes(T, H, I, ctx->num_sms), ws_bytes);
-    aflex_status s = gateup_launch(ctx, x, wg, wu, T, H, I, h, nullptr, 0, st);
+    aflex_status s = gateup_launch(ctx, x, wg, wu, T, H, I, h, sws, scratch, st, ctx->counters_f);
     if (s != AFLEX_OK) return s;
-    return linear_launch(ctx, h, wd, T, I, H, y, lws, lin, st, kKDownGemm);
+    return linear_launch(ctx, h, wd, T, I, H, y, sws, scratch, st, kKDownGemm, ctx->counters_f);
 }
 
 static size_t moe_ws_bytes(int T, int H, int I, int E, int K, int num_sms) {
@@ -123,7 +127,9 @@ static size_t moe_ws_bytes(int T, int H, int I, int E, int K, int num_sms) {
     b += align256(R * H * 2);                   // xp
     b += align256(R * I * 2);                   // hp
     b += align256(R * H * 4);                   // yp
-    b += grouped_workspace_bytes((int)R, T, I, H, E, num_sms);
+    const size_t gu = grouped_workspace_bytes(1, (int)R, T, H, I, E, num_sms);
+    const size_t dn = grouped_workspace_bytes(0, (int)R, T, I, H, E, num_sms);
+    b += gu > dn ? gu : dn;
     return b;
 }
 
@@ -143,7 +149,9 @@ static aflex_status moe_run(aflex_ctx* ctx, const void* x, const float* router_l
     __nv_bfloat16* xp = arena.take<__nv_bfloat16>(R * H);
     __nv_bfloat16* hp = arena.take<__nv_bfloat16>(R * I);
     float* yp = arena.take<float>(R * H);
-    const size_t gws = grouped_workspace_bytes((int)R, T, I, H, E, ctx->num_sms);
+    const size_t gu = grouped_workspace_bytes(1, (int)R, T, H, I, E, ctx->num_sms);
+    const size_t dn = grouped_workspace_bytes(0, (int)R, T, I, H, E, ctx->num_sms);
+    const size_t gws = gu > dn ? gu : dn;
     char* gw = gws ? arena.take<char>(gws) : nullptr;
     if (arena.overflow)
         return set_error(ctx, AFLEX_ERR_WORKSPACE, "moe ffn: need %zu workspace bytes, have %zu",
@@ -160,9 +168,9 @@ static aflex_status moe_run(aflex_ctx* ctx, const void* x, const float* router_l
     s = moe_gather_launch(ctx, x, mb.pos, T, K, H, xp, st);
     if (s != AFLEX_OK) return s;
     // an expert receives at most one assignment per token => segments have at most T rows
-    s = grouped_gateup_launch(ctx, xp, wg, wu, mb.offsets, (int)R, T, H, I, E, hp, nullptr, 0, st);
+    s = grouped_gateup_launch(ctx, xp, wg, wu, mb.offsets, (int)R, T, H, I, E, hp, gw, gws, st, ctx->counters_f);
     if (s != AFLEX_OK) return s;
-    s = grouped_linear_launch(ctx, hp, wd, mb.offsets, (int)R, T, I, H, E, yp, gw, gws, st);
+    s = grouped_linear_launch(ctx, hp, wd, mb.offsets, (int)R, T, I, H, E, yp, gw, gws, st, ctx->counters_f);
     if (s != AFLEX_OK) return s;
     s = moe_combine_launch(ctx, yp, mb.pos, mb.gate, T, K, H, y, st);
     if (s != AFLEX_OK) return s;
@@ -222,6 +230,17 @@ aflex_status aflex_create(aflex_ctx** out, int device, size_t workspace_bytes) {
     if (e == cudaSuccess) e = cudaMalloc(&ctx->ws, ctx->ws_bytes);
     if (e == cudaSuccess) e = cudaMalloc(&ctx->dev_status, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(ctx->dev_status, 0, sizeof(int));
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->counters_attn, kAttnCounterCap * sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(ctx->counters_attn, 0, kAttnCounterCap * sizeof(int));
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->counters_a, kStreamKMaxTiles * sizeof(int));
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->counters_f, kStreamKMaxTiles * sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(ctx->counters_a, 0, kStreamKMaxTiles * sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(ctx->counters_f, 0, kStreamKMaxTiles * sizeof(int));
+    if (e == cudaSuccess && getenv("AFLEX_TRACE") && atoi(getenv("AFLEX_TRACE")) > 0) {
+        const size_t tb = (size_t)kTraceKernels * kTraceStride * sizeof(unsigned long long);
+        e = cudaMalloc(&ctx->trace, tb);
+        if (e == cudaSuccess) e = cudaMemset(ctx->trace, 0, tb);
+    }
     if (e == cudaSuccess) e = cudaMallocHost(&ctx->host_status, sizeof(int));
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->stream_a, cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->stream_f, cudaStreamNonBlocking);
@@ -258,6 +277,10 @@ aflex_status aflex_destroy(aflex_ctx* ctx) {
     }
     if (ctx->host_status) cudaFreeHost(ctx->host_status);
     if (ctx->dev_status) cudaFree(ctx->dev_status);
+    if (ctx->trace) cudaFree(ctx->trace);
+    if (ctx->counters_attn) cudaFree(ctx->counters_attn);
+    if (ctx->counters_a) cudaFree(ctx->counters_a);
+    if (ctx->counters_f) cudaFree(ctx->counters_f);
     if (ctx->ws) cudaFree(ctx->ws);
     delete ctx;
     return AFLEX_OK;
@@ -273,12 +296,19 @@ aflex_status aflex_get_device_status(aflex_ctx* ctx, void* stream) {
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) return check_cuda(ctx, e, "aflex_get_device_status");
     const int v = *ctx->host_status;
+    if (v != 0) {
+        // a kernel that gave up may have left arrival counters half-way: restore the all-zero state
+        cudaMemsetAsync(ctx->counters_attn, 0, kAttnCounterCap * sizeof(int), st);
+        cudaMemsetAsync(ctx->counters_a, 0, kStreamKMaxTiles * sizeof(int), st);
+        cudaMemsetAsync(ctx->counters_f, 0, kStreamKMaxTiles * sizeof(int), st);
+        cudaStreamSynchronize(st);
+    }
     if (v != 0) set_error(ctx, (aflex_status)v, "device status word = %d (%s)", v, aflex_status_string((aflex_status)v));
     return (aflex_status)v;
 }
 
 static const char* kKernelNames[kKKindCount] = {
-    "attn_partial", "attn_combine", "linear_gemm", "down_gemm", "gateup_gemm", "splitk_reduce", "router_logits",
+    "attn_decode", "linear_gemm", "down_gemm", "gateup_gemm", "router_logits",
     "moe_route", "moe_gather", "moe_gateup_gemm", "moe_down_gemm", "moe_combine"};
 
 int aflex_num_kernel_kinds(void) { return kKKindCount; }
@@ -325,9 +355,20 @@ aflex_status aflex_profile_read(aflex_ctx* ctx, int kind, double* total_ms, long
     return AFLEX_OK;
 }
 
-aflex_status aflex_set_attn_chunk(aflex_ctx* ctx, int chunk_tokens) {
-    if (!ctx || chunk_tokens < 0) return AFLEX_ERR_INVALID_ARG;
-    ctx->attn_chunk = chunk_tokens;
+aflex_status aflex_trace_read(aflex_ctx* ctx, unsigned long long* host_out, int launches, int* next_slot) {
+    if (!ctx || !host_out || launches < 1 || launches > kTraceKernels) return AFLEX_ERR_INVALID_ARG;
+    if (!ctx->trace) return set_error(ctx, AFLEX_ERR_INVALID_ARG, "tracing is off (create the ctx with AFLEX_TRACE=1)");
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess)
+        e = cudaMemcpy(host_out, ctx->trace, (size_t)launches * kTraceStride * sizeof(unsigned long long), cudaMemcpyDeviceToHost);
+    if (next_slot) *next_slot = ctx->trace_slot;
+    ctx->trace_slot = 0;
+    return check_cuda(ctx, e, "aflex_trace_read");
+}
+
+aflex_status aflex_set_attn_ctas(aflex_ctx* ctx, int ctas) {
+    if (!ctx || ctas < 0 || ctas > 4096) return AFLEX_ERR_INVALID_ARG;
+    ctx->attn_ctas = ctas;
     return AFLEX_OK;
 }
 
@@ -344,7 +385,7 @@ aflex_status aflex_linear(aflex_ctx* ctx, const void* x, const void* w, int T, i
     if (!x || !w || !y || T < 1 || K < 1 || N < 1) return set_error(ctx, AFLEX_ERR_INVALID_ARG, "linear: bad argument");
     if (K % 8 || N % 8) return set_error(ctx, AFLEX_ERR_UNSUPPORTED, "linear: K and N must be multiples of 8");
     if (!aligned16(x) || !aligned16(w) || !aligned16(y)) return set_error(ctx, AFLEX_ERR_INVALID_ARG, "linear: pointers must be 16-byte aligned");
-    return linear_launch(ctx, x, w, T, K, N, y, ctx->ws, ctx->ws_bytes, reinterpret_cast<cudaStream_t>(stream), kKLinearGemm);
+    return linear_launch(ctx, x, w, T, K, N, y, ctx->ws, ctx->ws_bytes, reinterpret_cast<cudaStream_t>(stream), kKLinearGemm, ctx->counters_a);
 }
 
 aflex_status aflex_ffn_dense(aflex_ctx* ctx, const void* x, const void* w_gate, const void* w_up, const void* w_down,
@@ -417,10 +458,8 @@ LayerWs layer_ws(const aflex_layer_desc* L, int max_batch, size_t a_attn, int nu
 
 size_t aflex_workspace_bytes(const aflex_layer_desc* layer, int max_batch, int max_pages_per_seq) {
     if (!layer || max_batch < 1 || max_pages_per_seq < 1) return 0;
-    // the planner never picks a chunk below 128 tokens: size the partials for that worst case
-    const long long max_len = (long long)max_pages_per_seq * 16;
-    const int max_chunks = (int)((max_len + 127) / 128);
-    return layer_ws(layer, max_batch, attn_workspace_bytes(&layer->attn, max_batch, max_chunks), 148).total;
+    (void)max_pages_per_seq;   // the attention scratch is per CTA, not per context token
+    return layer_ws(layer, max_batch, attn_workspace_bytes(&layer->attn, 4096), 148).total;
 }
 
 aflex_status aflex_layer_step(aflex_ctx* ctx, const aflex_layer_desc* L, const void* q, const aflex_kv* kv, int batch,
@@ -456,15 +495,7 @@ aflex_status aflex_layer_step(aflex_ctx* ctx, const aflex_layer_desc* L, const v
         for (int i = 0; i < M; ++i) offs[i + 1] = offs[i] + base + (i < extra ? 1 : 0);
     }
 
-    size_t a_attn = 0;
-    for (int i = 0; i < M; ++i) {
-        aflex_kv kvi = *kv;
-        kvi.seq_lens_host = kv->seq_lens_host ? kv->seq_lens_host + offs[i] : nullptr;
-        const int rows = offs[i + 1] - offs[i];
-        const AttnPlan plan = attn_make_plan(ctx, &L->attn, &kvi, rows);
-        const size_t b = attn_workspace_bytes(&L->attn, rows, plan.max_chunks);
-        if (b > a_attn) a_attn = b;
-    }
+    const size_t a_attn = attn_workspace_bytes(&L->attn, attn_grid(ctx));
     const LayerWs w = layer_ws(L, batch, a_attn, ctx->num_sms);
     if (w.total > ctx->ws_bytes)
         return set_error(ctx, AFLEX_ERR_WORKSPACE, "layer step: need %zu workspace bytes, have %zu", w.total, ctx->ws_bytes);
@@ -476,11 +507,18 @@ aflex_status aflex_layer_step(aflex_ctx* ctx, const aflex_layer_desc* L, const v
     char* ws_f = ctx->ws + w.a_total + w.attn_out + w.x;
 
     cudaStream_t user = reinterpret_cast<cudaStream_t>(stream);
-    cudaStream_t sa = ctx->stream_a, sf = ctx->stream_f;
-    cudaError_t e = cudaEventRecord(ctx->ev_entry, user);
-    if (e == cudaSuccess) e = cudaStreamWaitEvent(sa, ctx->ev_entry, 0);
-    if (e == cudaSuccess) e = cudaStreamWaitEvent(sf, ctx->ev_entry, 0);
-    if (e != cudaSuccess) return check_cuda(ctx, e, "layer step: entry join");
+    // M = 1 is A then F in series (Eq. 2, first case): everything goes on the caller's stream, where
+    // consecutive kernels chain through programmatic dependent launch.  M >= 2 uses the ctx's
+    // attention and FFN streams, joined to the caller's stream on entry and exit.
+    const bool serial = (M == 1);
+    cudaStream_t sa = serial ? user : ctx->stream_a, sf = serial ? user : ctx->stream_f;
+    cudaError_t e = cudaSuccess;
+    if (!serial) {
+        e = cudaEventRecord(ctx->ev_entry, user);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(sa, ctx->ev_entry, 0);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(sf, ctx->ev_entry, 0);
+        if (e != cudaSuccess) return check_cuda(ctx, e, "layer step: entry join");
+    }
 
     const int Hq = L->attn.num_q_heads, D = L->attn.head_dim;
     for (int i = 0; i < M; ++i) {
@@ -494,12 +532,14 @@ aflex_status aflex_layer_step(aflex_ctx* ctx, const aflex_layer_desc* L, const v
         s = attn_decode_launch(ctx, &L->attn, qi, &kvi, rows, a_buf + (size_t)r0 * A, nullptr, ws_a, w.a_attn, sa);
         if (s != AFLEX_OK) return s;
         if (L->w_o) {
-            s = linear_launch(ctx, a_buf + (size_t)r0 * A, L->w_o, rows, A, H, x_buf + (size_t)r0 * H, ws_alin, w.a_lin, sa, kKLinearGemm);
+            s = linear_launch(ctx, a_buf + (size_t)r0 * A, L->w_o, rows, A, H, x_buf + (size_t)r0 * H, ws_alin, w.a_lin, sa, kKLinearGemm, ctx->counters_a);
             if (s != AFLEX_OK) return s;
         }
-        e = cudaEventRecord(ctx->ev_a[i], sa);
-        if (e == cudaSuccess) e = cudaStreamWaitEvent(sf, ctx->ev_a[i], 0);
-        if (e != cudaSuccess) return check_cuda(ctx, e, "layer step: A->F event");
+        if (!serial) {
+            e = cudaEventRecord(ctx->ev_a[i], sa);
+            if (e == cudaSuccess) e = cudaStreamWaitEvent(sf, ctx->ev_a[i], 0);
+            if (e != cudaSuccess) return check_cuda(ctx, e, "layer step: A->F event");
+        }
         // ---- F_i on the FFN stream
         __nv_bfloat16* yi = reinterpret_cast<__nv_bfloat16*>(y) + (size_t)r0 * H;
         const __nv_bfloat16* xi = x_buf + (size_t)r0 * H;
@@ -511,6 +551,7 @@ aflex_status aflex_layer_step(aflex_ctx* ctx, const aflex_layer_desc* L, const v
         }
         if (s != AFLEX_OK) return s;
     }
+    if (serial) return AFLEX_OK;
     e = cudaEventRecord(ctx->ev_a_done, sa);
     if (e == cudaSuccess) e = cudaEventRecord(ctx->ev_f_done, sf);
     if (e == cudaSuccess) e = cudaStreamWaitEvent(user, ctx->ev_a_done, 0);

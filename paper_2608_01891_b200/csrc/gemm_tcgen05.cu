@@ -15,13 +15,27 @@
 //   kGateUp : out = silu(x w_gate^T) .* (x w_up^T)          (two accumulators, fused SwiGLU epilogue)
 // Both have a grouped form for the mixture-of-experts FFN: the rows of x are the permuted
 // assignments, expert e owns rows [offsets[e], offsets[e+1]) and its own weight matrices.
-// kLinear optionally splits K across CTAs (fp32 partials + a fixed-order reduction kernel) so
-// that small-N projections still occupy every SM; the reduction order is fixed => deterministic.
+//
+// Scheduling.  A persistent CTA per SM.  With many tiles per CTA, whole tiles are taken
+// round-robin.  With few (the decode case: 200 gate/up tiles or 40 down-projection tiles on 148
+// SMs) the tile count is written as W * G + R for G CTAs: the R remainder tiles are cut along K
+// into one equal, contiguous share of 64-wide K blocks per CTA and are processed FIRST; then every
+// CTA takes its W whole tiles.  Every SM therefore streams the same number of weight bytes.  A
+// remainder tile whose K range is shared by several CTAs is finished by whichever of them arrives
+// last: each contributor stores its fp32 partial accumulator to the workspace and bumps the tile's
+// counter; the last one sums the partials IN CTA ORDER (the result does not depend on who was
+// last: bit-deterministic), applies the epilogue and resets the counter.  Because the shared
+// tiles come first, that fix-up overlaps the main loop of the CTA's next tile.
+//
+// Programmatic dependent launch: the kernel lets its successor start early and itself starts
+// before its predecessor has drained; weight tiles (which no kernel writes) are prefetched into
+// the pipeline before the grid-dependency wait, activation tiles only after it.
 //
 // CTA = 6 warps: warp 0 TMA producer, warp 1 MMA issuer (owns TMEM), warps 2..5 epilogue.
-// Persistent over a static round-robin tile list.  All waits are bounded.
+// All waits are bounded.
 #include <cuda_bf16.h>
 #include <stdio.h>
+#include <stdlib.h>
 
 #include "internal.h"
 #include "ptx.cuh"
@@ -43,16 +57,19 @@ struct GemmParams {
     int n_tile;       // token rows per tile, multiple of 16, <= 256
     int m_tiles;      // ceil(N / 128)
     int n_tiles;      // ceil(T / n_tile) (non-grouped)
-    int splits;       // K splits (kLinear only)
     int kblocks;      // ceil(K / 64)
     int stages;       // smem pipeline depth
     int nbuf;         // TMEM accumulator buffers (1 or 2)
     int num_experts;  // 0 => not grouped
     int tmem_cols;    // power of two >= 32
+    int streamk;      // 1 => equal contiguous shares of (tile, k-block) units per CTA
     const int32_t* offsets;   // grouped: device [E+1]
-    __nv_bfloat16* out_bf16;  // [T][N] (direct bf16 output) or nullptr
-    float* out_f32;           // [splits][T][N] fp32 partial sums, or nullptr
+    __nv_bfloat16* out_bf16;  // [T][N] bf16 output, or nullptr
+    float* out_f32;           // [T][N] fp32 output (MoE down projection), or nullptr
+    float* partials;          // shared tiles: [grid][2 slots][accumulators * n_tile / 4][128 rows] float4
+    int* counters;            // stream-K: one arrival counter per tile, zero on entry and on exit
     int* status;
+    unsigned long long* trace;   // optional [grid][8] timestamps (ns) for timeline debugging, or nullptr
 };
 
 struct TileCoord {
@@ -60,29 +77,26 @@ struct TileCoord {
     int a_row0;     // first row in the 2-D [(E*N)][K] weight view
     int b_row0;     // first token row
     int b_rows;     // valid token rows in this tile (<= n_tile)
-    int split;
     int out_row_limit;  // exclusive bound on token rows that may be stored
 };
 
-// Work list shared by all roles of a CTA.  Non-grouped: item = (m_tile, n_tile, split), n fastest.
-// Grouped: item = (expert, m_tile, chunk, split) over the experts' row segments, chunk fastest.
+// Tile list shared by all roles of a CTA.  Non-grouped: tile = (m_tile, n_tile), n fastest.
+// Grouped: tile = (expert, m_tile, chunk) over the experts' row segments, chunk fastest.
 struct TileIter {
     const GemmParams& p;
     const int* seg;       // smem copy of offsets (grouped)
     int total;
     __device__ TileIter(const GemmParams& p_, const int* seg_) : p(p_), seg(seg_) {
         if (p.num_experts == 0) {
-            total = p.m_tiles * p.n_tiles * p.splits;
+            total = p.m_tiles * p.n_tiles;
         } else {
             int chunks = 0;
             for (int e = 0; e < p.num_experts; ++e) chunks += (seg[e + 1] - seg[e] + p.n_tile - 1) / p.n_tile;
-            total = chunks * p.m_tiles * p.splits;
+            total = chunks * p.m_tiles;
         }
     }
     __device__ TileCoord get(int w) const {
         TileCoord c;
-        c.split = w % p.splits;
-        w /= p.splits;
         if (p.num_experts == 0) {
             int nt = w % p.n_tiles;
             c.m_tile = w / p.n_tiles;
@@ -92,12 +106,13 @@ struct TileIter {
             c.out_row_limit = p.T;
         } else {
             int e = 0;
-            for (; e < p.num_experts; ++e) {
+            for (; e < p.num_experts - 1; ++e) {
                 int items = ((seg[e + 1] - seg[e] + p.n_tile - 1) / p.n_tile) * p.m_tiles;
                 if (w < items) break;
                 w -= items;
             }
             int chunks = (seg[e + 1] - seg[e] + p.n_tile - 1) / p.n_tile;
+            if (chunks < 1) chunks = 1;
             int ch = w % chunks;
             c.m_tile = w / chunks;
             c.a_row0 = e * p.N + c.m_tile * kBlockM;
@@ -109,6 +124,72 @@ struct TileIter {
     }
 };
 
+// One unit of work for a CTA: K blocks [kb0, kb1) of one tile.  slot >= 0 => the unit does not
+// cover the whole K range and its partial accumulator goes to partial slot `slot` of this CTA.
+struct WorkUnit {
+    int tile, kb0, kb1, slot;
+};
+
+// Shape of the schedule, identical for every CTA and role.
+struct Schedule {
+    int kblocks;
+    int G;        // CTAs that take whole tiles
+    int R;        // remainder tiles (ids 0..R-1), shared along K
+    int Gr;       // CTAs that take a share of the remainder (every share non-empty)
+    int W;        // whole tiles per CTA (ids R + cta + i*G)
+    long long Ur; // R * kblocks
+    __device__ Schedule(const GemmParams& p, int total_tiles, int grid) {
+        kblocks = p.kblocks;
+        G = grid;
+        if (!p.streamk) { R = 0; W = (total_tiles + grid - 1) / grid; }
+        else { W = total_tiles / grid; R = total_tiles - W * grid; }
+        Ur = (long long)R * kblocks;
+        Gr = (int)(Ur < G ? Ur : G);
+        total = total_tiles;
+    }
+    int total;
+    __device__ long long share_begin(int c) const { return Ur * c / Gr; }
+    // CTA whose remainder share contains unit position x
+    __device__ int cta_of(long long x) const {
+        int c = (int)((x * Gr) / Ur);
+        if (c >= Gr) c = Gr - 1;
+        while (c > 0 && share_begin(c) > x) --c;
+        while (c + 1 < Gr && share_begin(c + 1) <= x) ++c;
+        return c;
+    }
+};
+
+// Walks the units of CTA `cta` in order; every role of the CTA walks the same sequence.
+struct UnitCursor {
+    const Schedule& sc;
+    int cta;
+    long long u, u_end;   // position in the remainder unit list
+    int i;                // index of the next whole tile
+    bool first;
+    __device__ UnitCursor(const Schedule& s, int cta_) : sc(s), cta(cta_), i(0), first(true) {
+        if (cta < sc.Gr) { u = sc.share_begin(cta); u_end = sc.share_begin(cta + 1); }
+        else { u = 0; u_end = 0; }
+    }
+    __device__ bool next(WorkUnit& out) {
+        if (u < u_end) {
+            out.tile = (int)(u / sc.kblocks);
+            out.kb0 = (int)(u % sc.kblocks);
+            out.kb1 = (int)min((long long)sc.kblocks, out.kb0 + (u_end - u));
+            const bool whole = out.kb0 == 0 && out.kb1 == sc.kblocks;
+            // at most two partial units per CTA: the first unit of its share (slot 0) and a later one (slot 1)
+            out.slot = whole ? -1 : (first ? 0 : 1);
+            first = false;
+            u += out.kb1 - out.kb0;
+            return true;
+        }
+        const int t = sc.R + cta + i * sc.G;
+        if (i >= sc.W || t >= sc.total) return false;
+        ++i;
+        out.tile = t; out.kb0 = 0; out.kb1 = sc.kblocks; out.slot = -1;
+        return true;
+    }
+};
+
 struct __align__(8) GemmBarriers {
     uint64_t full[kMaxStages];
     uint64_t empty[kMaxStages];
@@ -116,6 +197,7 @@ struct __align__(8) GemmBarriers {
     uint64_t tmem_empty[2];
     uint32_t tmem_base;
     volatile int abort;
+    int last_flag;
     int seg[kMaxExperts + 1];
 };
 
@@ -161,7 +243,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
 
     const uint32_t tmem_base = bars->tmem_base;
     const TileIter tiles(p, bars->seg);
-    const int acc_cols = (MODE == kGateUp ? 2 : 1) * p.n_tile;   // TMEM columns per accumulator buffer
+    constexpr int kAccs = (MODE == kGateUp) ? 2 : 1;
+    const int acc_cols = kAccs * p.n_tile;   // TMEM columns per accumulator buffer
+    const Schedule sched(p, tiles.total, (int)gridDim.x);
+    pdl_launch_dependents();
+    unsigned long long* tr = p.trace ? p.trace + (size_t)blockIdx.x * 8 : nullptr;
+    if (tr && threadIdx.x == 0) tr[0] = global_timer_ns();           // CTA running
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
@@ -170,11 +257,35 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
             const uint64_t pol_x = policy_evict_last();    // activations: re-read by every tile
             int s = 0; uint32_t ph = 0;
             const uint32_t tx = (uint32_t)(kNumA * kABytes + b_bytes);
-            for (int w = blockIdx.x; w < tiles.total && !bars->abort; w += gridDim.x) {
-                const TileCoord c = tiles.get(w);
-                const int kb0 = (int)(((long long)c.split * p.kblocks) / p.splits);
-                const int kb1 = (int)(((long long)(c.split + 1) * p.kblocks) / p.splits);
-                for (int kb = kb0; kb < kb1; ++kb) {
+            UnitCursor cur(sched, blockIdx.x);
+            WorkUnit wu;
+            // The first `stages` K blocks find the ring empty: their weight tiles are requested at once,
+            // before the grid-dependency wait; their activation tiles follow after it.
+            int primed = 0;
+            int pend_kb[kMaxStages], pend_row[kMaxStages];
+            bool waited = false;
+            while (!bars->abort && cur.next(wu)) {
+                const TileCoord c = tiles.get(wu.tile);
+                for (int kb = wu.kb0; kb < wu.kb1; ++kb) {
+                    if (primed < p.stages) {
+                        uint8_t* st = smem + (size_t)primed * stage_bytes;
+                        mbar_expect_tx(&bars->full[primed], tx);
+                        tma_load_2d_hint(st, &tmap_a0, kb * kBlockK, c.a_row0, &bars->full[primed], pol_w);
+                        if (MODE == kGateUp) tma_load_2d_hint(st + kABytes, &tmap_a1, kb * kBlockK, c.a_row0, &bars->full[primed], pol_w);
+                        pend_kb[primed] = kb; pend_row[primed] = c.b_row0;
+                        ++primed;
+                        if (++s == p.stages) { s = 0; ph ^= 1; }
+                        continue;
+                    }
+                    if (!waited) {
+                        if (tr) tr[1] = global_timer_ns();           // weights primed, about to wait
+                        pdl_wait();
+                        if (tr) tr[2] = global_timer_ns();           // dependency satisfied
+                        for (int i = 0; i < primed; ++i)
+                            tma_load_2d_hint(smem + (size_t)i * stage_bytes + kNumA * kABytes, &tmap_b, pend_kb[i] * kBlockK,
+                                             pend_row[i], &bars->full[i], pol_x);
+                        waited = true;
+                    }
                     if (!mbar_wait(&bars->empty[s], ph ^ 1)) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); break; }
                     uint8_t* st = smem + (size_t)s * stage_bytes;
                     mbar_expect_tx(&bars->full[s], tx);
@@ -184,8 +295,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
                     if (++s == p.stages) { s = 0; ph ^= 1; }
                 }
             }
-            // Drain: every load issued above has a consumer waiting on its full barrier unless the
-            // kernel aborted; on abort wait (bounded) for the loads in flight before leaving.
+            if (tr) tr[3] = global_timer_ns();                       // all loads issued
+            if (!waited) {
+                pdl_wait();
+                for (int i = 0; i < primed; ++i)
+                    tma_load_2d_hint(smem + (size_t)i * stage_bytes + kNumA * kABytes, &tmap_b, pend_kb[i] * kBlockK,
+                                     pend_row[i], &bars->full[i], pol_x);
+            }
+            // On abort wait (bounded) for loads still in flight before the CTA leaves.
             if (bars->abort) {
                 for (int i = 0; i < p.stages; ++i) (void)mbar_wait(&bars->full[i], 0);
             }
@@ -196,15 +313,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
             const uint32_t idesc = umma_idesc_bf16(kBlockM, (uint32_t)p.n_tile);
             int s = 0; uint32_t ph = 0;
             int buf = 0; uint32_t acc_ph = 0;
-            bool issued_any = false;
-            for (int w = blockIdx.x; w < tiles.total && !bars->abort; w += gridDim.x) {
-                const TileCoord c = tiles.get(w);
-                const int kb0 = (int)(((long long)c.split * p.kblocks) / p.splits);
-                const int kb1 = (int)(((long long)(c.split + 1) * p.kblocks) / p.splits);
+            UnitCursor cur(sched, blockIdx.x);
+            WorkUnit wu;
+            while (!bars->abort && cur.next(wu)) {
                 if (!mbar_wait(&bars->tmem_empty[buf], acc_ph ^ 1)) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); break; }
                 tc_fence_after();
                 const uint32_t d0 = tmem_base + (uint32_t)(buf * acc_cols);
-                for (int kb = kb0; kb < kb1; ++kb) {
+                for (int kb = wu.kb0; kb < wu.kb1; ++kb) {
                     if (!mbar_wait(&bars->full[s], ph)) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); break; }
                     tc_fence_after();
                     const uint32_t a_addr = smem_u32(smem + (size_t)s * stage_bytes);
@@ -212,7 +327,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
                     const uint64_t db = umma_desc_k_sw128(a_addr + kNumA * kABytes);
 #pragma unroll
                     for (int k = 0; k < kBlockK / 16; ++k) {
-                        const uint32_t acc = (kb > kb0 || k > 0) ? 1u : 0u;
+                        const uint32_t acc = (kb > wu.kb0 || k > 0) ? 1u : 0u;
                         // advancing 16 bf16 along K inside the swizzled row = +32 bytes = +2 in 16-byte units
                         umma_bf16(d0, da0 + 2 * k, db + 2 * k, idesc, acc);
                         if (MODE == kGateUp) {
@@ -221,87 +336,171 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
                         }
                     }
                     umma_commit(&bars->empty[s]);   // smem stage reusable once these MMAs retire
-                    issued_any = true;
                     if (++s == p.stages) { s = 0; ph ^= 1; }
                 }
                 if (bars->abort) break;
                 umma_commit(&bars->tmem_full[buf]);  // accumulator complete
+                if (tr) tr[4] = global_timer_ns();                   // last MMA of the unit issued
                 if (++buf == p.nbuf) { buf = 0; acc_ph ^= 1; }
             }
-            (void)issued_any;
         }
     } else {
         // ------------------------------------------------------------ epilogue (warps 2..5)
         const int lane_grp = warp & 3;                 // TMEM lanes [32*lane_grp, +32) belong to this warp
+        const int row = lane_grp * 32 + lane;          // accumulator row = weight row inside the tile
+        const int etid = threadIdx.x - 64;             // 0..127 among the epilogue threads
+        const int cols = kAccs * p.n_tile;             // fp32 values per accumulator row
+        const size_t slot_floats = (size_t)cols * kBlockM;
         int buf = 0; uint32_t acc_ph = 0;
-        for (int w = blockIdx.x; w < tiles.total && !bars->abort; w += gridDim.x) {
-            const TileCoord c = tiles.get(w);
+        UnitCursor cur(sched, blockIdx.x);
+        WorkUnit wu;
+        pdl_wait();   // nothing is written before the predecessor grid has completed
+        while (!bars->abort && cur.next(wu)) {
+            const TileCoord c = tiles.get(wu.tile);
             if (!mbar_wait(&bars->tmem_full[buf], acc_ph)) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); break; }
             tc_fence_after();
-            const int n_local = c.m_tile * kBlockM + lane_grp * 32 + lane;    // output feature inside the expert
+            const int n_local = c.m_tile * kBlockM + row;    // output feature inside the expert
             const bool n_ok = n_local < p.N;
             const uint32_t t0 = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(buf * acc_cols);
-            for (int c0 = 0; c0 < c.b_rows; c0 += 16) {
-                uint32_t g[16];
-                tmem_ld_32x32b_x16(t0 + (uint32_t)c0, g);
-                if (MODE == kGateUp) {
-                    uint32_t u[16];
-                    tmem_ld_32x32b_x16(t0 + (uint32_t)(p.n_tile + c0), u);
-                    tmem_ld_wait();
+            if (wu.slot < 0) {
+                // ---- whole K range in this CTA: epilogue straight from TMEM
+                for (int c0 = 0; c0 < c.b_rows; c0 += 16) {
+                    uint32_t g[16];
+                    tmem_ld_32x32b_x16(t0 + (uint32_t)c0, g);
+                    if (MODE == kGateUp) {
+                        uint32_t u[16];
+                        tmem_ld_32x32b_x16(t0 + (uint32_t)(p.n_tile + c0), u);
+                        tmem_ld_wait();
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const int t = c.b_row0 + c0 + j;
-                        if (n_ok && t < c.out_row_limit) {
-                            const float hv = silu_f32(__uint_as_float(g[j])) * __uint_as_float(u[j]);
-                            p.out_bf16[(size_t)t * p.N + n_local] = __float2bfloat16_rn(hv);
+                        for (int j = 0; j < 16; ++j) {
+                            const int t = c.b_row0 + c0 + j;
+                            if (n_ok && t < c.out_row_limit) {
+                                const float hv = silu_f32(__uint_as_float(g[j])) * __uint_as_float(u[j]);
+                                p.out_bf16[(size_t)t * p.N + n_local] = __float2bfloat16_rn(hv);
+                            }
                         }
-                    }
-                } else {
-                    tmem_ld_wait();
+                    } else {
+                        tmem_ld_wait();
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const int t = c.b_row0 + c0 + j;
-                        if (n_ok && t < c.out_row_limit) {
-                            const float v = __uint_as_float(g[j]);
-                            if (p.out_f32) p.out_f32[((size_t)c.split * p.T + t) * p.N + n_local] = v;
-                            else p.out_bf16[(size_t)t * p.N + n_local] = __float2bfloat16_rn(v);
+                        for (int j = 0; j < 16; ++j) {
+                            const int t = c.b_row0 + c0 + j;
+                            if (n_ok && t < c.out_row_limit) {
+                                const float v = __uint_as_float(g[j]);
+                                if (p.out_f32) p.out_f32[(size_t)t * p.N + n_local] = v;
+                                else p.out_bf16[(size_t)t * p.N + n_local] = __float2bfloat16_rn(v);
+                            }
                         }
                     }
                 }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars->tmem_empty[buf]);
+            } else {
+                // ---- partial K range: park the fp32 accumulator as [column group of 4][row] float4 (a warp
+                //      stores / loads 512 contiguous bytes per instruction); the last arriver finishes the tile
+                uint4* mine = reinterpret_cast<uint4*>(p.partials + ((size_t)blockIdx.x * 2 + wu.slot) * slot_floats) + row;
+                for (int c0 = 0; c0 < cols; c0 += 16) {
+                    if ((c0 % p.n_tile) >= c.b_rows) continue;   // token columns beyond the tile's valid rows
+                    uint32_t g[16];
+                    tmem_ld_32x32b_x16(t0 + (uint32_t)c0, g);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 16; j += 4)
+                        mine[(size_t)((c0 + j) >> 2) * kBlockM] = make_uint4(g[j], g[j + 1], g[j + 2], g[j + 3]);
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars->tmem_empty[buf]);   // TMEM buffer is free again
+                // publish: all 128 rows stored (CTA barrier), then one thread releases them device-wide
+                // and bumps the tile counter
+                asm volatile("bar.sync 2, 128;" ::: "memory");
+                const long long x0 = (long long)wu.tile * p.kblocks;
+                const int cf = sched.cta_of(x0);
+                const int cl = sched.cta_of(x0 + p.kblocks - 1);
+                if (etid == 0) {
+                    if (tr) tr[6] = global_timer_ns();               // partial stored, about to publish
+                    __threadfence();
+                    const int prev = atomicAdd(&p.counters[wu.tile], 1);
+                    bars->last_flag = (prev == cl - cf) ? 1 : 0;
+                    if (tr) tr[7] = global_timer_ns();               // published
+                }
+                asm volatile("bar.sync 2, 128;" ::: "memory");
+                if (bars->last_flag) {
+                    __threadfence();
+                    const bool cf_early = sched.share_begin(cf) < x0;
+                    // 32 token columns per pass; the partials of a batch of pieces (4, or 2 for gate/up) are
+                    // all requested before any is used, so a pass costs one memory round trip per batch.
+                    constexpr int kPB = (MODE == kGateUp) ? 2 : 4;
+                    for (int c0 = 0; c0 < c.b_rows; c0 += 32) {
+                        const bool hi = c0 + 16 < c.b_rows;          // second 16-column half is live
+                        float4 g[8], u[8];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) { g[j] = make_float4(0.f, 0.f, 0.f, 0.f); u[j] = g[j]; }
+                        for (int cb = cf; cb <= cl; cb += kPB) {
+                            float4 a[kPB][8], bq[kPB][8];
+#pragma unroll
+                            for (int q = 0; q < kPB; ++q) {
+                                const int cc = cb + q;
+                                if (cc <= cl) {
+                                    // only the first contributor's share can begin before the tile: then the piece
+                                    // is a later unit of that CTA (slot 1); every other piece is a first unit (slot 0)
+                                    const int sl = (cc == cf && cf_early) ? 1 : 0;
+                                    const float4* part = reinterpret_cast<const float4*>(p.partials + ((size_t)cc * 2 + sl) * slot_floats) +
+                                                         (size_t)(c0 >> 2) * kBlockM + row;
+#pragma unroll
+                                    for (int j = 0; j < 8; ++j) {
+                                        if (j < 4 || hi) {
+                                            a[q][j] = __ldcg(part + (size_t)j * kBlockM);
+                                            if (MODE == kGateUp) bq[q][j] = __ldcg(part + (size_t)(j + (p.n_tile >> 2)) * kBlockM);
+                                        }
+                                    }
+                                }
+                            }
+#pragma unroll
+                            for (int q = 0; q < kPB; ++q) {
+                                if (cb + q <= cl) {
+#pragma unroll
+                                    for (int j = 0; j < 8; ++j) {
+                                        if (j < 4 || hi) {
+                                            g[j].x += a[q][j].x; g[j].y += a[q][j].y; g[j].z += a[q][j].z; g[j].w += a[q][j].w;
+                                            if (MODE == kGateUp) {
+                                                u[j].x += bq[q][j].x; u[j].y += bq[q][j].y; u[j].z += bq[q][j].z; u[j].w += bq[q][j].w;
+                                            }
+                                        }
+                                    }
+                                }
+                            }
+                        }
+                        const float* gf = reinterpret_cast<const float*>(g);
+                        const float* uf = reinterpret_cast<const float*>(u);
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const int t = c.b_row0 + c0 + j;
+                            if ((j < 16 || hi) && n_ok && t < c.out_row_limit) {
+                                if (MODE == kGateUp) {
+                                    p.out_bf16[(size_t)t * p.N + n_local] = __float2bfloat16_rn(silu_f32(gf[j]) * uf[j]);
+                                } else if (p.out_f32) {
+                                    p.out_f32[(size_t)t * p.N + n_local] = gf[j];
+                                } else {
+                                    p.out_bf16[(size_t)t * p.N + n_local] = __float2bfloat16_rn(gf[j]);
+                                }
+                            }
+                        }
+                    }
+                    if (etid == 0) p.counters[wu.tile] = 0;   // leave the counter clean for the next launch
+                }
+                asm volatile("bar.sync 2, 128;" ::: "memory");   // last_flag may be rewritten by the next unit
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&bars->tmem_empty[buf]);
             if (++buf == p.nbuf) { buf = 0; acc_ph ^= 1; }
         }
     }
 
+    if (tr && threadIdx.x == 64) tr[5] = global_timer_ns();          // epilogue finished
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
-    }
-}
-
-// out[t][n] = sum_s part[s][t][n]  (fixed order s = 0,1,..) -> bf16 or fp32
-__global__ void splitk_reduce_kernel(const float* __restrict__ part, int splits, size_t TN, __nv_bfloat16* out_bf16,
-                                     float* out_f32) {
-    const size_t i4 = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
-    if (i4 >= TN) return;
-    float4 acc = *reinterpret_cast<const float4*>(part + i4);
-    for (int s = 1; s < splits; ++s) {
-        const float4 v = *reinterpret_cast<const float4*>(part + (size_t)s * TN + i4);
-        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
-    }
-    if (out_bf16) {
-        __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
-        uint2 pk;
-        pk.x = *reinterpret_cast<uint32_t*>(&lo);
-        pk.y = *reinterpret_cast<uint32_t*>(&hi);
-        *reinterpret_cast<uint2*>(out_bf16 + i4) = pk;
-    } else {
-        *reinterpret_cast<float4*>(out_f32 + i4) = acc;
     }
 }
 
@@ -313,31 +512,28 @@ static int pick_n_tile(int rows_max) {
     return n > 256 ? 256 : n;
 }
 
-// Choose the K split so that the static round-robin list fills whole waves of CTAs.
-static int pick_splits(int base_items, int kblocks, int num_sms, bool allow) {
-    if (!allow || base_items >= 2 * num_sms) return 1;
-    int best = 1;
-    double best_score = -1.0;
-    for (int s = 1; s <= 16; ++s) {
-        if (kblocks / s < 8) break;
-        const int items = base_items * s;
-        const int waves = (items + num_sms - 1) / num_sms;
-        double eff = (double)items / ((double)waves * num_sms);
-        // prefer fewer splits when efficiency is close (partials cost traffic)
-        const double score = eff - 0.004 * s;
-        if (score > best_score) { best_score = score; best = s; }
-    }
-    return best;
-}
-
 struct GemmConfig {
     GemmParams p;
     size_t smem_bytes;
+    size_t partial_bytes;
     int grid;
 };
 
-static bool make_config(int mode, int T, int N, int K, int rows_max, int E, int num_sms, bool allow_split,
-                        GemmConfig* cfg) {
+// Shared-memory budget of a CTA in the few-tiles (weight-streaming) regime.  Half of the SM, so the
+// first CTAs of the next kernel in the stream can become resident (and prefetch weights) while this
+// kernel's CTAs are still in their epilogue.  AFLEX_GEMM_SMEM_KB overrides it (tuning).
+static int streaming_smem_budget() {
+    static int kb = -1;
+    if (kb < 0) {
+        const char* e = getenv("AFLEX_GEMM_SMEM_KB");
+        kb = e ? atoi(e) : 150;
+        if (kb < 48) kb = 48;
+        if (kb > 227) kb = 227;
+    }
+    return kb * 1024;
+}
+
+static bool make_config(int mode, int T, int N, int K, int rows_max, int E, int num_sms, GemmConfig* cfg) {
     GemmParams& p = cfg->p;
     p.T = T; p.N = N; p.K = K;
     p.n_tile = pick_n_tile(rows_max);
@@ -345,24 +541,32 @@ static bool make_config(int mode, int T, int N, int K, int rows_max, int E, int 
     p.n_tiles = (T + p.n_tile - 1) / p.n_tile;
     p.kblocks = (K + kBlockK - 1) / kBlockK;
     p.num_experts = E;
-    const int base_items = (E == 0) ? p.m_tiles * p.n_tiles : p.m_tiles * E * ((rows_max + p.n_tile - 1) / p.n_tile);
-    p.splits = (mode == kLinear) ? pick_splits(base_items, p.kblocks, num_sms, allow_split) : 1;
-    const int acc_cols = (mode == kGateUp ? 2 : 1) * p.n_tile;
+    // upper bound on tiles (exact for the non-grouped form; the grouped form knows its tile count
+    // only on the device: every expert can add one ragged chunk)
+    const long long tiles_hi = (E == 0) ? (long long)p.m_tiles * p.n_tiles
+                                        : (long long)p.m_tiles * ((T + p.n_tile - 1) / p.n_tile + E);
+    const int accs = (mode == kGateUp ? 2 : 1);
+    const int acc_cols = accs * p.n_tile;
     p.nbuf = (2 * acc_cols <= 512) ? 2 : 1;
     int cols = 32;
     while (cols < p.nbuf * acc_cols) cols <<= 1;
     p.tmem_cols = cols;
-    const int a_bytes = (mode == kGateUp ? 2 : 1) * kBlockM * kBlockK * 2;
+    const int a_bytes = accs * kBlockM * kBlockK * 2;
     const int stage_bytes = a_bytes + round_up(p.n_tile * kBlockK * 2, 1024);
-    const int budget = 227 * 1024 - 1024 /*alignment slack*/ - (int)sizeof(GemmBarriers) - 256;
+    // few tiles per SM: share the remainder tiles along K; many: whole tiles round-robin
+    p.streamk = (tiles_hi < 8LL * num_sms && tiles_hi <= kStreamKMaxTiles) ? 1 : 0;
+    const int cap = (p.streamk && p.n_tile <= 64) ? streaming_smem_budget() : kMaxDynamicSmem;
+    const int budget = cap - 1024 /*alignment slack*/ - (int)sizeof(GemmBarriers) - 256;
     int stages = budget / stage_bytes;
     if (stages > kMaxStages) stages = kMaxStages;
-    if (stages < 2) return false;
+    if (stages < 2) stages = 2;
     p.stages = stages;
     cfg->smem_bytes = (size_t)stages * stage_bytes + sizeof(GemmBarriers) + 1024 + 128;
-    int items = base_items * p.splits;
-    cfg->grid = items < num_sms ? items : num_sms;
+    if (cfg->smem_bytes > (size_t)kMaxDynamicSmem) return false;
+    long long units = tiles_hi * p.kblocks;
+    cfg->grid = (int)(units < num_sms ? units : num_sms);
     if (cfg->grid < 1) cfg->grid = 1;
+    cfg->partial_bytes = p.streamk ? align256((size_t)cfg->grid * 2 * accs * p.n_tile * kBlockM * sizeof(float)) : 0;
     return true;
 }
 
@@ -376,65 +580,75 @@ static aflex_status launch_gemm(aflex_ctx* ctx, const GemmConfig& cfg, const CUt
         ctx->gemm_attr_set[MODE] = true;
     }
     KernelScope scope(ctx, kind, st);
-    gemm_kernel<MODE><<<cfg.grid, kGemmThreads, cfg.smem_bytes, st>>>(ta0, ta1, tb, cfg.p);
-    return check_cuda(ctx, cudaGetLastError(), "gemm_kernel launch");
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3((unsigned)cfg.grid);
+    lc.blockDim = dim3(kGemmThreads);
+    lc.dynamicSmemBytes = cfg.smem_bytes;
+    lc.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    return check_cuda(ctx, cudaLaunchKernelEx(&lc, gemm_kernel<MODE>, ta0, ta1, tb, cfg.p), "gemm_kernel launch");
 }
 
-static aflex_status run_reduce(aflex_ctx* ctx, const float* part, int splits, size_t TN, void* out_bf16, float* out_f32,
-                               cudaStream_t st) {
-    const int threads = 256;
-    const size_t n4 = (TN + 3) / 4;
-    const int blocks = (int)((n4 + threads - 1) / threads);
-    KernelScope scope(ctx, kKSplitKReduce, st);
-    splitk_reduce_kernel<<<blocks, threads, 0, st>>>(part, splits, TN, (__nv_bfloat16*)out_bf16, out_f32);
-    return check_cuda(ctx, cudaGetLastError(), "splitk_reduce launch");
+static aflex_status bind_scratch(aflex_ctx* ctx, GemmConfig& cfg, char* ws, size_t ws_bytes, int* counters,
+                                 const char* who) {
+    GemmParams& p = cfg.p;
+    p.status = ctx->dev_status;
+    p.trace = ctx->trace ? ctx->trace + (size_t)(ctx->trace_slot++ % kTraceKernels) * kTraceStride : nullptr;
+    p.counters = counters;
+    p.partials = nullptr;
+    if (p.streamk) {
+        if (cfg.partial_bytes > ws_bytes || ws == nullptr)
+            return set_error(ctx, AFLEX_ERR_WORKSPACE, "%s: need %zu workspace bytes, have %zu", who, cfg.partial_bytes, ws_bytes);
+        p.partials = reinterpret_cast<float*>(ws);
+    }
+    return AFLEX_OK;
 }
 
 size_t linear_workspace_bytes(int T, int K, int N, int num_sms) {
     GemmConfig cfg;
-    if (!make_config(kLinear, T, N, K, T, 0, num_sms, true, &cfg)) return 0;
-    return cfg.p.splits > 1 ? align256((size_t)cfg.p.splits * T * N * sizeof(float)) : 0;
+    if (!make_config(kLinear, T, N, K, T, 0, num_sms, &cfg)) return 0;
+    return cfg.partial_bytes;
 }
 
 aflex_status linear_launch(aflex_ctx* ctx, const void* x, const void* w, int T, int K, int N, void* y, char* ws,
-                           size_t ws_bytes, cudaStream_t st, int kind) {
+                           size_t ws_bytes, cudaStream_t st, int kind, int* counters) {
     GemmConfig cfg;
-    if (!make_config(kLinear, T, N, K, T, 0, ctx->num_sms, true, &cfg))
+    if (!make_config(kLinear, T, N, K, T, 0, ctx->num_sms, &cfg))
         return set_error(ctx, AFLEX_ERR_UNSUPPORTED, "linear: no tile configuration fits");
     GemmParams& p = cfg.p;
     p.offsets = nullptr;
-    p.status = ctx->dev_status;
-    if (p.splits > 1) {
-        const size_t need = (size_t)p.splits * T * N * sizeof(float);
-        if (need > ws_bytes) return set_error(ctx, AFLEX_ERR_WORKSPACE, "linear: need %zu workspace bytes, have %zu", need, ws_bytes);
-        p.out_f32 = reinterpret_cast<float*>(ws);
-        p.out_bf16 = nullptr;
-    } else {
-        p.out_f32 = nullptr;
-        p.out_bf16 = reinterpret_cast<__nv_bfloat16*>(y);
-    }
+    p.out_f32 = nullptr;
+    p.out_bf16 = reinterpret_cast<__nv_bfloat16*>(y);
+    aflex_status s = bind_scratch(ctx, cfg, ws, ws_bytes, counters, "linear");
+    if (s != AFLEX_OK) return s;
     CUtensorMap ta, tb;
     if (!encode_tmap_2d_bf16(&ta, w, (uint64_t)N, (uint64_t)K, (uint64_t)K * 2, kBlockM, kBlockK, true) ||
         !encode_tmap_2d_bf16(&tb, x, (uint64_t)T, (uint64_t)K, (uint64_t)K * 2, (uint32_t)p.n_tile, kBlockK, false))
         return set_error(ctx, AFLEX_ERR_CUDA, "linear: cuTensorMapEncodeTiled failed");
-    aflex_status s = launch_gemm<kLinear>(ctx, cfg, ta, ta, tb, st, kind);
-    if (s != AFLEX_OK) return s;
-    if (p.splits > 1) return run_reduce(ctx, p.out_f32, p.splits, (size_t)T * N, y, nullptr, st);
-    return AFLEX_OK;
+    return launch_gemm<kLinear>(ctx, cfg, ta, ta, tb, st, kind);
 }
 
-size_t gateup_workspace_bytes(int, int, int, int) { return 0; }
+size_t gateup_workspace_bytes(int T, int H, int I, int num_sms) {
+    GemmConfig cfg;
+    if (!make_config(kGateUp, T, I, H, T, 0, num_sms, &cfg)) return 0;
+    return cfg.partial_bytes;
+}
 
 aflex_status gateup_launch(aflex_ctx* ctx, const void* x, const void* w_gate, const void* w_up, int T, int H, int I,
-                           void* h, char*, size_t, cudaStream_t st) {
+                           void* h, char* ws, size_t ws_bytes, cudaStream_t st, int* counters) {
     GemmConfig cfg;
-    if (!make_config(kGateUp, T, I, H, T, 0, ctx->num_sms, false, &cfg))
+    if (!make_config(kGateUp, T, I, H, T, 0, ctx->num_sms, &cfg))
         return set_error(ctx, AFLEX_ERR_UNSUPPORTED, "gate/up: no tile configuration fits");
     GemmParams& p = cfg.p;
     p.offsets = nullptr;
-    p.status = ctx->dev_status;
     p.out_f32 = nullptr;
     p.out_bf16 = reinterpret_cast<__nv_bfloat16*>(h);
+    aflex_status s = bind_scratch(ctx, cfg, ws, ws_bytes, counters, "gate/up");
+    if (s != AFLEX_OK) return s;
     CUtensorMap tg, tu, tb;
     if (!encode_tmap_2d_bf16(&tg, w_gate, (uint64_t)I, (uint64_t)H, (uint64_t)H * 2, kBlockM, kBlockK, true) ||
         !encode_tmap_2d_bf16(&tu, w_up, (uint64_t)I, (uint64_t)H, (uint64_t)H * 2, kBlockM, kBlockK, true) ||
@@ -443,24 +657,25 @@ aflex_status gateup_launch(aflex_ctx* ctx, const void* x, const void* w_gate, co
     return launch_gemm<kGateUp>(ctx, cfg, tg, tu, tb, st, kKGateUpGemm);
 }
 
-size_t grouped_workspace_bytes(int rows_total, int rows_max, int K, int N, int E, int num_sms) {
+size_t grouped_workspace_bytes(int mode_gateup, int rows_total, int rows_max, int K, int N, int E, int num_sms) {
     GemmConfig cfg;
-    if (!make_config(kLinear, rows_total, N, K, rows_max, E, num_sms, true, &cfg)) return 0;
-    return cfg.p.splits > 1 ? align256((size_t)cfg.p.splits * rows_total * N * sizeof(float)) : 0;
+    if (!make_config(mode_gateup ? kGateUp : kLinear, rows_total, N, K, rows_max, E, num_sms, &cfg)) return 0;
+    return cfg.partial_bytes;
 }
 
 aflex_status grouped_gateup_launch(aflex_ctx* ctx, const void* xp, const void* w_gate, const void* w_up,
                                    const int32_t* offsets, int rows_total, int rows_max, int H, int I, int E,
-                                   void* hp, char*, size_t, cudaStream_t st) {
+                                   void* hp, char* ws, size_t ws_bytes, cudaStream_t st, int* counters) {
     if (E > kMaxExperts) return set_error(ctx, AFLEX_ERR_UNSUPPORTED, "num_experts > %d", kMaxExperts);
     GemmConfig cfg;
-    if (!make_config(kGateUp, rows_total, I, H, rows_max, E, ctx->num_sms, false, &cfg))
+    if (!make_config(kGateUp, rows_total, I, H, rows_max, E, ctx->num_sms, &cfg))
         return set_error(ctx, AFLEX_ERR_UNSUPPORTED, "grouped gate/up: no tile configuration fits");
     GemmParams& p = cfg.p;
     p.offsets = offsets;
-    p.status = ctx->dev_status;
     p.out_f32 = nullptr;
     p.out_bf16 = reinterpret_cast<__nv_bfloat16*>(hp);
+    aflex_status s = bind_scratch(ctx, cfg, ws, ws_bytes, counters, "grouped gate/up");
+    if (s != AFLEX_OK) return s;
     CUtensorMap tg, tu, tb;
     if (!encode_tmap_2d_bf16(&tg, w_gate, (uint64_t)E * I, (uint64_t)H, (uint64_t)H * 2, kBlockM, kBlockK, true) ||
         !encode_tmap_2d_bf16(&tu, w_up, (uint64_t)E * I, (uint64_t)H, (uint64_t)H * 2, kBlockM, kBlockK, true) ||
@@ -471,30 +686,22 @@ aflex_status grouped_gateup_launch(aflex_ctx* ctx, const void* xp, const void* w
 
 aflex_status grouped_linear_launch(aflex_ctx* ctx, const void* hp, const void* w_down, const int32_t* offsets,
                                    int rows_total, int rows_max, int K, int N, int E, float* yp, char* ws,
-                                   size_t ws_bytes, cudaStream_t st) {
+                                   size_t ws_bytes, cudaStream_t st, int* counters) {
     if (E > kMaxExperts) return set_error(ctx, AFLEX_ERR_UNSUPPORTED, "num_experts > %d", kMaxExperts);
     GemmConfig cfg;
-    if (!make_config(kLinear, rows_total, N, K, rows_max, E, ctx->num_sms, true, &cfg))
+    if (!make_config(kLinear, rows_total, N, K, rows_max, E, ctx->num_sms, &cfg))
         return set_error(ctx, AFLEX_ERR_UNSUPPORTED, "grouped linear: no tile configuration fits");
     GemmParams& p = cfg.p;
     p.offsets = offsets;
-    p.status = ctx->dev_status;
     p.out_bf16 = nullptr;
-    if (p.splits > 1) {
-        const size_t need = (size_t)p.splits * rows_total * N * sizeof(float);
-        if (need > ws_bytes) return set_error(ctx, AFLEX_ERR_WORKSPACE, "grouped linear: need %zu workspace bytes, have %zu", need, ws_bytes);
-        p.out_f32 = reinterpret_cast<float*>(ws);
-    } else {
-        p.out_f32 = yp;
-    }
+    p.out_f32 = yp;
+    aflex_status s = bind_scratch(ctx, cfg, ws, ws_bytes, counters, "grouped linear");
+    if (s != AFLEX_OK) return s;
     CUtensorMap ta, tb;
     if (!encode_tmap_2d_bf16(&ta, w_down, (uint64_t)E * N, (uint64_t)K, (uint64_t)K * 2, kBlockM, kBlockK, true) ||
         !encode_tmap_2d_bf16(&tb, hp, (uint64_t)rows_total, (uint64_t)K, (uint64_t)K * 2, (uint32_t)p.n_tile, kBlockK, false))
         return set_error(ctx, AFLEX_ERR_CUDA, "grouped linear: cuTensorMapEncodeTiled failed");
-    aflex_status s = launch_gemm<kLinear>(ctx, cfg, ta, ta, tb, st, kKMoeDownGemm);
-    if (s != AFLEX_OK) return s;
-    if (p.splits > 1) return run_reduce(ctx, p.out_f32, p.splits, (size_t)rows_total * N, nullptr, yp, st);
-    return AFLEX_OK;
+    return launch_gemm<kLinear>(ctx, cfg, ta, ta, tb, st, kKMoeDownGemm);
 }
 
 }  // namespace aflex

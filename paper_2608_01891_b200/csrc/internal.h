@@ -13,13 +13,17 @@ namespace aflex {
 constexpr int kMaxMicrobatches = 64;
 constexpr size_t kDefaultWorkspace = (size_t)256 << 20;
 constexpr int kMaxDynamicSmem = 227 * 1024;   // opt-in shared memory per CTA on sm_100
+constexpr int kAttnCounterCap = 1 << 20;       // (sequence, KV head) arrival counters
+constexpr int kTraceKernels = 64;              // timeline debugging: ring of per-launch records
+constexpr int kTraceStride = 4096 * 8;         // u64 per launch record: [cta < 4096][8 stamps]
+constexpr int kStreamKMaxTiles = 16384;       // capacity of each per-tile arrival-counter array
 
 }  // namespace aflex
 
 namespace aflex {
 // Kernel kinds, for launch counting and optional per-kernel event timing.
 enum KernelKind {
-    kKAttnPartial = 0, kKAttnCombine, kKLinearGemm, kKDownGemm, kKGateUpGemm, kKSplitKReduce, kKRouterLogits,
+    kKAttnDecode = 0, kKLinearGemm, kKDownGemm, kKGateUpGemm, kKRouterLogits,
     kKMoeRoute, kKMoeGather, kKMoeGateUpGemm, kKMoeDownGemm, kKMoeCombine, kKKindCount
 };
 constexpr int kProfMaxSlots = 8192;
@@ -33,11 +37,14 @@ struct aflex_ctx {
     char* ws = nullptr;           // device workspace
     int* dev_status = nullptr;    // device status word (0 = OK)
     int* host_status = nullptr;   // pinned mirror used by aflex_get_device_status
+    int* counters_attn = nullptr; // per-(sequence, KV head) chunk arrival counters (zero between launches)
+    int* counters_a = nullptr;    // per-tile arrival counters, attention-stream GEMMs (zero between launches)
+    int* counters_f = nullptr;    // per-tile arrival counters, FFN-stream GEMMs
     cudaStream_t stream_a = nullptr, stream_f = nullptr;
     cudaEvent_t ev_entry = nullptr;
     cudaEvent_t ev_a[aflex::kMaxMicrobatches] = {};
     cudaEvent_t ev_f_done = nullptr, ev_a_done = nullptr;
-    int attn_chunk = 0;           // 0 = automatic
+    int attn_ctas = 0;            // persistent attention CTAs per launch; 0 = two per SM
     bool gemm_attr_set[2] = {false, false};
     bool attn_attr_set[2] = {false, false};
     char err[512] = {0};
@@ -46,6 +53,8 @@ struct aflex_ctx {
     bool profiling = false;
     aflex::ProfSlot* prof = nullptr;   // kProfMaxSlots pre-created event pairs
     int prof_used = 0;
+    unsigned long long* trace = nullptr;   // device buffer, allocated when AFLEX_TRACE=1
+    int trace_slot = 0;
 };
 
 namespace aflex {
@@ -91,34 +100,31 @@ bool encode_tmap_2d_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint
                          uint32_t box_rows, uint32_t box_cols, bool promote_l2_256);
 
 // ---- attention (attn_decode.cu)
-struct AttnPlan {
-    int chunk_tokens;      // C, multiple of 64
-    int max_chunks;        // ceil(16*max_pages_per_seq / C)
-};
-AttnPlan attn_make_plan(const aflex_ctx* ctx, const aflex_attn_desc* d, const aflex_kv* kv, int batch);
-size_t attn_workspace_bytes(const aflex_attn_desc* d, int batch, int max_chunks);
+int attn_grid(const aflex_ctx* ctx);                                    // persistent CTAs per launch
+size_t attn_workspace_bytes(const aflex_attn_desc* d, int grid);        // per-CTA partial slots
 aflex_status attn_decode_launch(aflex_ctx* ctx, const aflex_attn_desc* d, const void* q, const aflex_kv* kv,
                                 int batch, void* out, float* lse, char* ws, size_t ws_bytes, cudaStream_t st);
 
 // ---- GEMM (gemm_tcgen05.cu)
 // y[T][N] = x[T][K] . w[N][K]^T (bf16 in, fp32 accumulate, bf16 out).
+// `counters`: kStreamKMaxTiles zeroed ints not used by any launch that may run concurrently.
 size_t linear_workspace_bytes(int T, int K, int N, int num_sms);
 aflex_status linear_launch(aflex_ctx* ctx, const void* x, const void* w, int T, int K, int N, void* y, char* ws,
-                           size_t ws_bytes, cudaStream_t st, int kind);
+                           size_t ws_bytes, cudaStream_t st, int kind, int* counters);
 // h[T][I] = silu(x Wg^T) .* (x Wu^T)
 size_t gateup_workspace_bytes(int T, int H, int I, int num_sms);
 aflex_status gateup_launch(aflex_ctx* ctx, const void* x, const void* w_gate, const void* w_up, int T, int H, int I,
-                           void* h, char* ws, size_t ws_bytes, cudaStream_t st);
+                           void* h, char* ws, size_t ws_bytes, cudaStream_t st, int* counters);
 
 // Grouped (per-expert) variants over permuted rows.  `offsets` is a device array [E+1]
 // (row segment of expert e = [offsets[e], offsets[e+1])); rows_max bounds any segment.
-size_t grouped_workspace_bytes(int rows_total, int rows_max, int K, int N, int E, int num_sms);
+size_t grouped_workspace_bytes(int mode_gateup, int rows_total, int rows_max, int K, int N, int E, int num_sms);
 aflex_status grouped_gateup_launch(aflex_ctx* ctx, const void* xp, const void* w_gate, const void* w_up,
                                    const int32_t* offsets, int rows_total, int rows_max, int H, int I, int E,
-                                   void* hp, char* ws, size_t ws_bytes, cudaStream_t st);
+                                   void* hp, char* ws, size_t ws_bytes, cudaStream_t st, int* counters);
 aflex_status grouped_linear_launch(aflex_ctx* ctx, const void* hp, const void* w_down, const int32_t* offsets,
                                    int rows_total, int rows_max, int K, int N, int E, float* yp, char* ws,
-                                   size_t ws_bytes, cudaStream_t st);
+                                   size_t ws_bytes, cudaStream_t st, int* counters);
 
 // ---- MoE glue (moe.cu)
 struct MoeBuffers {

@@ -59,32 +59,32 @@ def test_attention_config1_matches_oracle(ctx):
 
 @pytest.mark.parametrize("Hq,Hkv,D", [(64, 8, 128), (32, 8, 128), (8, 8, 128), (4, 2, 64), (16, 2, 64)])
 def test_attention_ragged_lengths_every_residue(ctx, Hq, Hkv, D):
-    """Lengths 1..3 pages at every residue mod 16, plus chunk boundaries +-1, with NaN poison in
-    every unreferenced slot; several chunks and a ragged tail per sequence."""
+    """Lengths 1..3 pages at every residue mod 16, plus 64-token unit boundaries +-1, with NaN poison in
+    every unreferenced slot; sequences split across several CTAs and ragged tails."""
     lens = list(range(1, 50)) + [63, 64, 65, 127, 128, 129, 255, 256, 257, 300, 511, 512, 513, 777, 1024, 1100]
     q, kv = make_case(len(lens), Hq, Hkv, D, lens, seed=1, poison=True)
     want, want_lse = O.attn_decode(u16(q), u16(kv.k_cache), u16(kv.v_cache), kv.page_table.numpy(), kv.seq_lens.numpy())
-    for chunk in (0, 64, 256):
-        ctx.set_attn_chunk(chunk)
+    for ctas in (0, 1, 37, 2000):     # different splits of the same KV: one CTA .. more CTAs than 64-token units of most items
+        ctx.set_attn_ctas(ctas)
         got, lse = run_attention(ctx, q, kv.k_cache, kv.v_cache, kv.page_table, kv.seq_lens, Hq, Hkv, D)
-        assert row_rel_err(got, want) <= TOL_ATTN, chunk
-        assert np.abs(lse - want_lse).max() <= TOL_LSE, chunk
-    ctx.set_attn_chunk(0)
+        assert row_rel_err(got, want) <= TOL_ATTN, ctas
+        assert np.abs(lse - want_lse).max() <= TOL_LSE, ctas
+    ctx.set_attn_ctas(0)
     # n = 1: the output is that token's V row, bit for bit
     b = lens.index(1)
     vrow = f64(kv.v_cache[int(kv.page_table[b, 0]), :, 0, :])            # [Hkv, D]
     assert (got[b] == np.repeat(vrow, Hq // Hkv, axis=0)).all()
 
 
-def test_attention_chunking_does_not_change_result(ctx):
+def test_attention_split_does_not_change_result(ctx):
     lens = [37, 500, 1999, 4096, 2048, 1]
     q, kv = make_case(len(lens), 16, 2, 128, lens, seed=2)
     outs = []
-    for chunk in (64, 128, 512, 4096):
-        ctx.set_attn_chunk(chunk)
+    for ctas in (1, 2, 5, 64, 296, 4096):
+        ctx.set_attn_ctas(ctas)
         outs.append(run_attention(ctx, q, kv.k_cache, kv.v_cache, kv.page_table, kv.seq_lens, 16, 2, 128,
                                   with_host_lens=False)[0])
-    ctx.set_attn_chunk(0)
+    ctx.set_attn_ctas(0)
     want, _ = O.attn_decode(u16(q), u16(kv.k_cache), u16(kv.v_cache), kv.page_table.numpy(), kv.seq_lens.numpy())
     for o in outs:
         assert row_rel_err(o, want) <= TOL_ATTN
