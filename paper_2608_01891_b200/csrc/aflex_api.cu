@@ -232,10 +232,10 @@ aflex_status aflex_create(aflex_ctx** out, int device, size_t workspace_bytes) {
     if (e == cudaSuccess) e = cudaMemset(ctx->dev_status, 0, sizeof(int));
     if (e == cudaSuccess) e = cudaMalloc(&ctx->counters_attn, kAttnCounterCap * sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(ctx->counters_attn, 0, kAttnCounterCap * sizeof(int));
-    if (e == cudaSuccess) e = cudaMalloc(&ctx->counters_a, kStreamKMaxTiles * sizeof(int));
-    if (e == cudaSuccess) e = cudaMalloc(&ctx->counters_f, kStreamKMaxTiles * sizeof(int));
-    if (e == cudaSuccess) e = cudaMemset(ctx->counters_a, 0, kStreamKMaxTiles * sizeof(int));
-    if (e == cudaSuccess) e = cudaMemset(ctx->counters_f, 0, kStreamKMaxTiles * sizeof(int));
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->counters_a, 2 * kStreamKMaxTiles * sizeof(int));
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->counters_f, 2 * kStreamKMaxTiles * sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(ctx->counters_a, 0, 2 * kStreamKMaxTiles * sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(ctx->counters_f, 0, 2 * kStreamKMaxTiles * sizeof(int));
     if (e == cudaSuccess && getenv("AFLEX_TRACE") && atoi(getenv("AFLEX_TRACE")) > 0) {
         const size_t tb = (size_t)kTraceKernels * kTraceStride * sizeof(unsigned long long);
         e = cudaMalloc(&ctx->trace, tb);
@@ -299,8 +299,8 @@ aflex_status aflex_get_device_status(aflex_ctx* ctx, void* stream) {
     if (v != 0) {
         // a kernel that gave up may have left arrival counters half-way: restore the all-zero state
         cudaMemsetAsync(ctx->counters_attn, 0, kAttnCounterCap * sizeof(int), st);
-        cudaMemsetAsync(ctx->counters_a, 0, kStreamKMaxTiles * sizeof(int), st);
-        cudaMemsetAsync(ctx->counters_f, 0, kStreamKMaxTiles * sizeof(int), st);
+        cudaMemsetAsync(ctx->counters_a, 0, 2 * kStreamKMaxTiles * sizeof(int), st);
+        cudaMemsetAsync(ctx->counters_f, 0, 2 * kStreamKMaxTiles * sizeof(int), st);
         cudaStreamSynchronize(st);
     }
     if (v != 0) set_error(ctx, (aflex_status)v, "device status word = %d (%s)", v, aflex_status_string((aflex_status)v));

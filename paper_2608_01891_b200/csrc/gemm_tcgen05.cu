@@ -21,11 +21,11 @@
 // SMs) the tile count is written as W * G + R for G CTAs: the R remainder tiles are cut along K
 // into one equal, contiguous share of 64-wide K blocks per CTA and are processed FIRST; then every
 // CTA takes its W whole tiles.  Every SM therefore streams the same number of weight bytes.  A
-// remainder tile whose K range is shared by several CTAs is finished by whichever of them arrives
-// last: each contributor stores its fp32 partial accumulator to the workspace and bumps the tile's
-// counter; the last one sums the partials IN CTA ORDER (the result does not depend on who was
-// last: bit-deterministic), applies the epilogue and resets the counter.  Because the shared
-// tiles come first, that fix-up overlaps the main loop of the CTA's next tile.
+// remainder tile whose K range is shared by several CTAs is finished by those CTAs together: each
+// contributor stores its fp32 partial accumulator to the workspace and bumps the tile's counter;
+// when all pieces are there, contributor i sums the i-th slice of the tile over the pieces IN CTA
+// ORDER (bit-deterministic), applies the epilogue and writes that slice.  Because the shared tiles
+// come first, this fix-up overlaps the main loop of the CTA's next tile.
 //
 // Programmatic dependent launch: the kernel lets its successor start early and itself starts
 // before its predecessor has drained; weight tiles (which no kernel writes) are prefetched into
@@ -67,7 +67,7 @@ struct GemmParams {
     __nv_bfloat16* out_bf16;  // [T][N] bf16 output, or nullptr
     float* out_f32;           // [T][N] fp32 output (MoE down projection), or nullptr
     float* partials;          // shared tiles: [grid][2 slots][accumulators * n_tile / 4][128 rows] float4
-    int* counters;            // stream-K: one arrival counter per tile, zero on entry and on exit
+    int* counters;            // shared tiles: [2][kStreamKMaxTiles] arrival / completion counters, zero on entry and exit
     int* status;
     unsigned long long* trace;   // optional [grid][8] timestamps (ns) for timeline debugging, or nullptr
 };
@@ -355,8 +355,109 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
         UnitCursor cur(sched, blockIdx.x);
         WorkUnit wu;
         pdl_wait();   // nothing is written before the predecessor grid has completed
+
+        // A shared tile is finished by ALL its contributors together: once every piece is published
+        // (arrival counter == number of pieces; bounded spin), contributor i sums the i-th slice of the
+        // tile over all pieces, in CTA order, and writes that slice of the output.  A second counter
+        // tells the last finisher to reset both counters.  Contributors of a tile run concurrently (the
+        // grid never exceeds the SM count and shared tiles are everyone's first units), so the spin is short.
+        struct PendingTile { int tile; TileCoord c; };
+        PendingTile pend[2];
+        int npend = 0;
+        auto run_reduce = [&](const PendingTile& pd) {
+            const long long x0 = (long long)pd.tile * p.kblocks;
+            const int cf = sched.cta_of(x0);
+            const int cl = sched.cta_of(x0 + p.kblocks - 1);
+            const int np = cl - cf + 1, me = (int)blockIdx.x - cf;
+            if (etid == 0) {
+                const long long t_start = clock64();
+                int seen;
+                do {
+                    asm volatile("ld.acquire.gpu.b32 %0, [%1];" : "=r"(seen) : "l"(p.counters + pd.tile) : "memory");
+                    if (seen >= np) break;
+                    __nanosleep(64);
+                } while (clock64() - t_start < kWaitBudgetCycles);
+                if (seen < np) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); }
+            }
+            asm volatile("bar.sync 2, 128;" ::: "memory");
+            if (bars->abort) return;
+            __threadfence();
+            const bool cf_early = sched.share_begin(cf) < x0;
+            const int n4 = ((pd.c.b_rows + 15) / 16) * 4 * kBlockM;     // float4 slots of one accumulator that were stored
+            const int lo = (int)((long long)n4 * me / np), hi = (int)((long long)n4 * (me + 1) / np);
+            const int up_off = (p.n_tile >> 2) * kBlockM;               // float4 offset of the "up" accumulator
+            for (int i0 = lo + etid; i0 < hi; i0 += 2 * 128) {
+                const int i1 = i0 + 128;
+                const bool two = i1 < hi;
+                float4 g0 = make_float4(0.f, 0.f, 0.f, 0.f), g1 = g0, u0 = g0, u1 = g0;
+                for (int cb = cf; cb <= cl; cb += 4) {
+                    float4 a0[4], a1[4], b0[4], b1[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const int cc = cb + q;
+                        if (cc <= cl) {
+                            // only the first contributor's share can begin before the tile: then its piece is a
+                            // later unit of that CTA (slot 1); every other piece is a first unit (slot 0)
+                            const int sl = (cc == cf && cf_early) ? 1 : 0;
+                            const float4* part = reinterpret_cast<const float4*>(p.partials + ((size_t)cc * 2 + sl) * slot_floats);
+                            a0[q] = __ldcg(part + i0);
+                            if (two) a1[q] = __ldcg(part + i1);
+                            if (MODE == kGateUp) {
+                                b0[q] = __ldcg(part + up_off + i0);
+                                if (two) b1[q] = __ldcg(part + up_off + i1);
+                            }
+                        }
+                    }
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        if (cb + q <= cl) {
+                            g0.x += a0[q].x; g0.y += a0[q].y; g0.z += a0[q].z; g0.w += a0[q].w;
+                            if (two) { g1.x += a1[q].x; g1.y += a1[q].y; g1.z += a1[q].z; g1.w += a1[q].w; }
+                            if (MODE == kGateUp) {
+                                u0.x += b0[q].x; u0.y += b0[q].y; u0.z += b0[q].z; u0.w += b0[q].w;
+                                if (two) { u1.x += b1[q].x; u1.y += b1[q].y; u1.z += b1[q].z; u1.w += b1[q].w; }
+                            }
+                        }
+                    }
+                }
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    if (h == 1 && !two) break;
+                    const int idx = h ? i1 : i0;
+                    const float4 gv = h ? g1 : g0, uv = h ? u1 : u0;
+                    const float gf[4] = {gv.x, gv.y, gv.z, gv.w}, uf[4] = {uv.x, uv.y, uv.z, uv.w};
+                    const int r = idx & (kBlockM - 1), cg = idx / kBlockM;
+                    const int nl = pd.c.m_tile * kBlockM + r;
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const int t = pd.c.b_row0 + cg * 4 + k;
+                        if (nl < p.N && t < pd.c.out_row_limit) {
+                            if (MODE == kGateUp) p.out_bf16[(size_t)t * p.N + nl] = __float2bfloat16_rn(silu_f32(gf[k]) * uf[k]);
+                            else if (p.out_f32) p.out_f32[(size_t)t * p.N + nl] = gf[k];
+                            else p.out_bf16[(size_t)t * p.N + nl] = __float2bfloat16_rn(gf[k]);
+                        }
+                    }
+                }
+            }
+            asm volatile("bar.sync 2, 128;" ::: "memory");
+            if (etid == 0) {
+                const int done = atomicAdd(&p.counters[kStreamKMaxTiles + pd.tile], 1);
+                if (done == np - 1) {   // every contributor has read what it needs: clean up for the next launch
+                    p.counters[pd.tile] = 0;
+                    p.counters[kStreamKMaxTiles + pd.tile] = 0;
+                }
+            }
+        };
+
         while (!bars->abort && cur.next(wu)) {
             const TileCoord c = tiles.get(wu.tile);
+            if (wu.slot < 0 && npend > 0) {
+                // shared tiles come first: before waiting for the first whole tile, finish this CTA's part
+                // of the shared tiles (the main loop of the whole tile runs meanwhile)
+                for (int i = 0; i < npend; ++i) run_reduce(pend[i]);
+                npend = 0;
+                if (bars->abort) break;
+            }
             if (!mbar_wait(&bars->tmem_full[buf], acc_ph)) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); break; }
             tc_fence_after();
             const int n_local = c.m_tile * kBlockM + row;    // output feature inside the expert
@@ -412,87 +513,21 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&bars->tmem_empty[buf]);   // TMEM buffer is free again
                 // publish: all 128 rows stored (CTA barrier), then one thread releases them device-wide
-                // and bumps the tile counter
+                // and bumps the tile counter.  The reduction itself is deferred (see run_reduce).
                 asm volatile("bar.sync 2, 128;" ::: "memory");
-                const long long x0 = (long long)wu.tile * p.kblocks;
-                const int cf = sched.cta_of(x0);
-                const int cl = sched.cta_of(x0 + p.kblocks - 1);
                 if (etid == 0) {
                     if (tr) tr[6] = global_timer_ns();               // partial stored, about to publish
                     __threadfence();
-                    const int prev = atomicAdd(&p.counters[wu.tile], 1);
-                    bars->last_flag = (prev == cl - cf) ? 1 : 0;
+                    atomicAdd(&p.counters[wu.tile], 1);
                     if (tr) tr[7] = global_timer_ns();               // published
                 }
-                asm volatile("bar.sync 2, 128;" ::: "memory");
-                if (bars->last_flag) {
-                    __threadfence();
-                    const bool cf_early = sched.share_begin(cf) < x0;
-                    // 32 token columns per pass; the partials of a batch of pieces (4, or 2 for gate/up) are
-                    // all requested before any is used, so a pass costs one memory round trip per batch.
-                    constexpr int kPB = (MODE == kGateUp) ? 2 : 4;
-                    for (int c0 = 0; c0 < c.b_rows; c0 += 32) {
-                        const bool hi = c0 + 16 < c.b_rows;          // second 16-column half is live
-                        float4 g[8], u[8];
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) { g[j] = make_float4(0.f, 0.f, 0.f, 0.f); u[j] = g[j]; }
-                        for (int cb = cf; cb <= cl; cb += kPB) {
-                            float4 a[kPB][8], bq[kPB][8];
-#pragma unroll
-                            for (int q = 0; q < kPB; ++q) {
-                                const int cc = cb + q;
-                                if (cc <= cl) {
-                                    // only the first contributor's share can begin before the tile: then the piece
-                                    // is a later unit of that CTA (slot 1); every other piece is a first unit (slot 0)
-                                    const int sl = (cc == cf && cf_early) ? 1 : 0;
-                                    const float4* part = reinterpret_cast<const float4*>(p.partials + ((size_t)cc * 2 + sl) * slot_floats) +
-                                                         (size_t)(c0 >> 2) * kBlockM + row;
-#pragma unroll
-                                    for (int j = 0; j < 8; ++j) {
-                                        if (j < 4 || hi) {
-                                            a[q][j] = __ldcg(part + (size_t)j * kBlockM);
-                                            if (MODE == kGateUp) bq[q][j] = __ldcg(part + (size_t)(j + (p.n_tile >> 2)) * kBlockM);
-                                        }
-                                    }
-                                }
-                            }
-#pragma unroll
-                            for (int q = 0; q < kPB; ++q) {
-                                if (cb + q <= cl) {
-#pragma unroll
-                                    for (int j = 0; j < 8; ++j) {
-                                        if (j < 4 || hi) {
-                                            g[j].x += a[q][j].x; g[j].y += a[q][j].y; g[j].z += a[q][j].z; g[j].w += a[q][j].w;
-                                            if (MODE == kGateUp) {
-                                                u[j].x += bq[q][j].x; u[j].y += bq[q][j].y; u[j].z += bq[q][j].z; u[j].w += bq[q][j].w;
-                                            }
-                                        }
-                                    }
-                                }
-                            }
-                        }
-                        const float* gf = reinterpret_cast<const float*>(g);
-                        const float* uf = reinterpret_cast<const float*>(u);
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            const int t = c.b_row0 + c0 + j;
-                            if ((j < 16 || hi) && n_ok && t < c.out_row_limit) {
-                                if (MODE == kGateUp) {
-                                    p.out_bf16[(size_t)t * p.N + n_local] = __float2bfloat16_rn(silu_f32(gf[j]) * uf[j]);
-                                } else if (p.out_f32) {
-                                    p.out_f32[(size_t)t * p.N + n_local] = gf[j];
-                                } else {
-                                    p.out_bf16[(size_t)t * p.N + n_local] = __float2bfloat16_rn(gf[j]);
-                                }
-                            }
-                        }
-                    }
-                    if (etid == 0) p.counters[wu.tile] = 0;   // leave the counter clean for the next launch
-                }
-                asm volatile("bar.sync 2, 128;" ::: "memory");   // last_flag may be rewritten by the next unit
+                pend[npend].tile = wu.tile;
+                pend[npend].c = c;
+                ++npend;
             }
             if (++buf == p.nbuf) { buf = 0; acc_ph ^= 1; }
         }
+        for (int i = 0; i < npend; ++i) run_reduce(pend[i]);
     }
 
     if (tr && threadIdx.x == 64) tr[5] = global_timer_ns();          // epilogue finished
