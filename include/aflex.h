@@ -139,6 +139,37 @@ typedef struct {
 AFLEX_API aflex_status aflex_attn_decode(aflex_ctx* ctx, const aflex_attn_desc* desc, const void* q,
                                          const aflex_kv* kv, int batch, void* out, float* lse, void* stream);
 
+/*
+ * Decode attention for callers that cannot allocate device memory (no counterpart in the
+ * paper: it serves the integration, not the method).
+ *
+ * Who needs it: a process whose memory pool has already claimed the whole GPU so that any
+ * later cudaMalloc fails, a plugin that must stay inside a host application's allocator, or a
+ * latency-critical path where an allocation -- an implicit device-wide synchronisation -- is
+ * not acceptable.  aflex_create allocates, so such callers cannot hold an aflex_ctx.  This
+ * entry point takes no ctx and calls no allocating routine: the kernel's scratch (per-CTA
+ * partial results, arrival counters, a status word) is a fixed ~2.7 MB array inside the
+ * library's device image, present on every GPU that loads the library until the process
+ * exits.  The caller still passes every input and output.
+ *
+ * Same arguments, layouts, arithmetic and result as aflex_attn_decode.  Limits of the fixed
+ * scratch: batch * num_kv_heads <= 16384 (otherwise AFLEX_ERR_WORKSPACE is returned and
+ * nothing is launched) and at most 320 persistent CTAs are used.  Other errors:
+ * AFLEX_ERR_INVALID_ARG / AFLEX_ERR_UNSUPPORTED as for aflex_attn_decode, AFLEX_ERR_CUDA.
+ * There is no error string (no ctx to keep it in).
+ *
+ * The first call on a device looks up the scratch array's device address and raises the
+ * kernel's shared-memory limit for that device; make that first call with the device
+ * current and before any stream capture.  Later calls only enqueue work.
+ * All calls share the one array, which keeps the previous call's contents: each call
+ * re-zeroes the counters and the status word on `stream` before the kernel.  Two calls
+ * that overlap on the GPU (different streams, or different host threads without ordering)
+ * race on the scratch and give wrong results: order them on one stream or with events.
+ * Not thread-safe on the host for first calls on the same device.
+ */
+AFLEX_API aflex_status aflex_attn_decode_static(const aflex_attn_desc* desc, const void* q, const aflex_kv* kv,
+                                                int batch, void* out, float* lse, void* stream);
+
 /* ---- FFN side -------------------------------------------------------------
  *
  * Dense SwiGLU FFN (the decode FFN operator of the paper's Section 1: weight

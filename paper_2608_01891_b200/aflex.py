@@ -24,7 +24,7 @@ EXPORTS = (
     "aflex_get_device_status", "aflex_attn_decode", "aflex_ffn_dense", "aflex_ffn_moe", "aflex_layer_step",
     "aflex_workspace_bytes", "aflex_linear", "aflex_set_attn_ctas", "aflex_num_kernel_kinds",
     "aflex_kernel_name", "aflex_launch_count", "aflex_profile_enable", "aflex_profile_read",
-    "aflex_trace_read",
+    "aflex_trace_read", "aflex_attn_decode_static",
 )
 
 
@@ -100,6 +100,8 @@ def load_library() -> ctypes.CDLL:
     lib.aflex_profile_enable.argtypes = [vp, ci]
     lib.aflex_profile_read.restype = ci
     lib.aflex_profile_read.argtypes = [vp, ci, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_longlong)]
+    lib.aflex_attn_decode_static.restype = ci
+    lib.aflex_attn_decode_static.argtypes = [ctypes.POINTER(AttnDesc), vp, ctypes.POINTER(KV), ci, vp, vp, vp]
     _lib = lib
     return lib
 
@@ -144,6 +146,27 @@ def layer_desc(attn: AttnDesc, hidden: int, inter: int, w_o, w_gate, w_up, w_dow
 
 def workspace_bytes(layer: LayerDesc, max_batch: int, max_pages_per_seq: int) -> int:
     return int(load_library().aflex_workspace_bytes(ctypes.byref(layer), max_batch, max_pages_per_seq))
+
+
+_STATIC_ERRORS = {
+    ERR_INVALID_ARG: "null / misaligned pointer, batch < 1, or Hkv does not divide Hq",
+    ERR_UNSUPPORTED: "outside the supported envelope (head_dim 64|128, page_size 16, Hq/Hkv in 1,2,4,8)",
+    ERR_WORKSPACE: "batch * num_kv_heads exceeds the fixed scratch capacity (16384)",
+    ERR_CUDA: "a CUDA call failed",
+}
+
+
+def attn_decode_static(desc: AttnDesc, q: torch.Tensor, kv: KV, out: torch.Tensor,
+                       lse: Optional[torch.Tensor] = None, stream=None) -> None:
+    """Decode attention through the allocation-free entry point: no Context, no workspace; the
+    kernel's scratch is a fixed array inside the library.  For callers that cannot allocate device
+    memory (a pool that owns the whole GPU, a host application's allocator rules, a path that must not
+    synchronise).  Calls must not overlap on the GPU: they share that one scratch array."""
+    lib = load_library()
+    st = lib.aflex_attn_decode_static(ctypes.byref(desc), _ptr(q), ctypes.byref(kv), q.shape[0], _ptr(out), _ptr(lse),
+                                      _stream(stream))
+    if st != OK:
+        raise AflexError(st, lib.aflex_status_string(st).decode(), _STATIC_ERRORS.get(st, "unknown error"))
 
 
 class Context:

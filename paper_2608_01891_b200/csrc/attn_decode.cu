@@ -564,3 +564,125 @@ aflex_status attn_decode_launch(aflex_ctx* ctx, const aflex_attn_desc* d, const 
 }
 
 }  // namespace aflex
+
+// ------------------------------------------------------------------------------------------------
+// Allocation-free decode attention.
+//
+// Some callers must not allocate device memory at all: a serving process whose memory pool has
+// already claimed the whole GPU (every later cudaMalloc fails), a plugin that runs inside
+// someone else's allocator discipline, or code on a latency-critical path where an allocation
+// (an implicit device synchronisation) is not acceptable.  aflex_create allocates a workspace, so
+// those callers cannot use the ctx-based entry points.  This entry point needs no ctx: the
+// kernel's scratch (per-CTA partial results, arrival counters, a status word) lives in the
+// file-scope device array below, which every GPU that loads the library holds until exit.
+//
+// Limits (stated maxima of the fixed scratch): at most kStaticMaxCtas persistent CTAs are
+// launched and batch * num_kv_heads must not exceed kStaticMaxItems.  Everything else follows
+// aflex_attn_decode (same kernel, same arithmetic).
+namespace aflex {
+
+constexpr int kStaticMaxCtas = 320;        // >= 2 CTAs per SM on a 148-SM part
+constexpr int kStaticMaxItems = 16384;     // (sequence, KV head) pairs per call
+constexpr size_t kStaticOPartFloats = (size_t)kStaticMaxCtas * 2 * 8 * 128;
+constexpr size_t kStaticMlFloats = (size_t)kStaticMaxCtas * 2 * 8 * 2;
+constexpr size_t kStaticScratchBytes =
+    (kStaticOPartFloats + kStaticMlFloats) * sizeof(float) + (size_t)kStaticMaxItems * sizeof(int) + 256;   // ~2.7 MB
+
+// Layout: [o_part floats | ml_part floats | counters ints | status word].
+static __device__ __align__(256) unsigned char g_attn_static_scratch[kStaticScratchBytes];
+
+struct StaticDeviceState {
+    unsigned char* scratch = nullptr;   // device address of g_attn_static_scratch on this device
+    int num_sms = 0;
+    bool attr_set[2] = {false, false};
+};
+static StaticDeviceState g_static_state[64];
+
+template <int D>
+static aflex_status attn_static_launch(StaticDeviceState& stt, const aflex_attn_desc* d, const void* q, const aflex_kv* kv,
+                                       int batch, void* out, float* lse, cudaStream_t st) {
+    int grid = 2 * stt.num_sms;
+    if (grid > kStaticMaxCtas) grid = kStaticMaxCtas;
+    float* o_part = reinterpret_cast<float*>(stt.scratch);
+    float* ml_part = o_part + kStaticOPartFloats;
+    int* counters = reinterpret_cast<int*>(ml_part + kStaticMlFloats);
+    int* status = counters + kStaticMaxItems;
+    // The array keeps whatever the previous call left: the arrival counters and the status word must
+    // start at zero (a call that was cut short could have left them dirty).
+    cudaError_t e = cudaMemsetAsync(counters, 0, ((size_t)batch * d->num_kv_heads) * sizeof(int), st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(status, 0, sizeof(int), st);
+    if (e != cudaSuccess) return AFLEX_ERR_CUDA;
+
+    AttnParams p;
+    p.o_part = o_part;
+    p.ml_part = ml_part;
+    p.q = reinterpret_cast<const __nv_bfloat16*>(q);
+    p.page_table = kv->page_table;
+    p.seq_lens = kv->seq_lens;
+    p.batch = batch;
+    p.max_pages = kv->max_pages_per_seq;
+    p.Hq = d->num_q_heads; p.Hkv = d->num_kv_heads; p.G = d->num_q_heads / d->num_kv_heads;
+    p.num_pages = kv->num_pages;
+    const float scale = d->sm_scale != 0.f ? d->sm_scale : 1.0f / sqrtf((float)D);
+    p.scale_log2 = scale * 1.4426950408889634f;
+    p.status = status;
+    p.out = reinterpret_cast<__nv_bfloat16*>(out);
+    p.lse = lse;
+    p.counters = counters;
+    p.trace = nullptr;
+
+    const uint64_t rows = (uint64_t)kv->num_pages * d->num_kv_heads * kPage;
+    CUtensorMap tk, tv;
+    if (!encode_tmap_2d_bf16(&tk, kv->k_cache, rows, D, (uint64_t)D * 2, kPage, 64, true) ||
+        !encode_tmap_2d_bf16(&tv, kv->v_cache, rows, D, (uint64_t)D * 2, kPage, 64, true))
+        return AFLEX_ERR_CUDA;
+    constexpr int kStageBytes = 2 * kPagesPerStage * kPage * D * 2;
+    constexpr int kStateFloats = 4 * (D / 16) + 4;
+    const size_t smem = (size_t)kAttnStages * kStageBytes + 3 * kStateFloats * 32 * sizeof(float) + sizeof(AttnShared) + 1024;
+    const int ti = (D == 128) ? 1 : 0;
+    if (!stt.attr_set[ti]) {
+        e = cudaFuncSetAttribute(attn_decode_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return AFLEX_ERR_CUDA;
+        stt.attr_set[ti] = true;
+    }
+    attn_decode_kernel<D><<<grid, kAttnThreads, smem, st>>>(tk, tv, p);
+    return cudaGetLastError() == cudaSuccess ? AFLEX_OK : AFLEX_ERR_CUDA;
+}
+
+}  // namespace aflex
+
+extern "C" aflex_status aflex_attn_decode_static(const aflex_attn_desc* desc, const void* q, const aflex_kv* kv, int batch,
+                                                 void* out, float* lse, void* stream) {
+    using namespace aflex;
+    if (!desc || !q || !kv || !out || !kv->k_cache || !kv->v_cache || !kv->page_table || !kv->seq_lens)
+        return AFLEX_ERR_INVALID_ARG;
+    if (batch < 1 || kv->num_pages < 1 || kv->max_pages_per_seq < 1) return AFLEX_ERR_INVALID_ARG;
+    if (desc->num_q_heads < 1 || desc->num_kv_heads < 1 || desc->num_q_heads % desc->num_kv_heads != 0)
+        return AFLEX_ERR_INVALID_ARG;
+    const int G = desc->num_q_heads / desc->num_kv_heads;
+    if ((desc->head_dim != 64 && desc->head_dim != 128) || desc->page_size != 16 || (G != 1 && G != 2 && G != 4 && G != 8))
+        return AFLEX_ERR_UNSUPPORTED;
+    if ((long long)kv->num_pages * desc->num_kv_heads * 16 >= (1LL << 31)) return AFLEX_ERR_UNSUPPORTED;
+    if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(out) | reinterpret_cast<uintptr_t>(kv->k_cache) |
+         reinterpret_cast<uintptr_t>(kv->v_cache)) & 15)
+        return AFLEX_ERR_INVALID_ARG;
+    // beyond the fixed scratch: refuse, never spill into an allocation
+    if ((long long)batch * desc->num_kv_heads > kStaticMaxItems) return AFLEX_ERR_WORKSPACE;
+
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return AFLEX_ERR_CUDA;
+    StaticDeviceState& stt = g_static_state[dev];
+    if (stt.scratch == nullptr) {
+        // One-time set-up for this device (it is the current device): in host code the array's name is
+        // only a stand-in, the kernel needs its device address.
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_attn_static_scratch) != cudaSuccess || ptr == nullptr) return AFLEX_ERR_CUDA;
+        int sms = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) return AFLEX_ERR_CUDA;
+        stt.num_sms = sms;
+        stt.scratch = static_cast<unsigned char*>(ptr);
+    }
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    if (desc->head_dim == 128) return attn_static_launch<128>(stt, desc, q, kv, batch, out, lse, st);
+    return attn_static_launch<64>(stt, desc, q, kv, batch, out, lse, st);
+}
