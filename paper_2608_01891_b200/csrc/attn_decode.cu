@@ -131,7 +131,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
 
     pdl_launch_dependents();
     unsigned long long* tr = (p.trace && cta < 4096) ? p.trace + (size_t)cta * 8 : nullptr;
-    if (tr && threadIdx.x == 0) { tr[0] = global_timer_ns(); tr[5] = 0; }
+    if (tr && threadIdx.x == 0) { tr[0] = global_timer_ns(); tr[3] = 0; tr[5] = 0; }
     if (threadIdx.x == 0) {
         for (int s = 0; s < kAttnStages; ++s) {
             mbar_init(&sh->full[s], 1);
@@ -174,6 +174,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         sh->start_prefix = pre;
     }
     __syncthreads();
+    if (tr && threadIdx.x == 0) tr[1] = global_timer_ns();            // share located
 
     if (warp == kAttnConsumerWarps) {
         // ------------------------------------------------------------------ producer warp
@@ -260,6 +261,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                     aborted = true;
                     break;
                 }
+                if (tr && threadIdx.x == 0 && tr[3] == 0) tr[3] = global_timer_ns();     // first data landed
                 const int nvalid = min(kPage, len - (u * kUnitTokens + warp * kPage));   // tokens of this warp's page
                 if (nvalid > 0) {
                     const uint32_t kpage = smem_u32(smem + s * kStageBytes + warp * kPageBytes);
@@ -325,6 +327,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                 if (++s == kAttnStages) { s = 0; ph ^= 1; }
             }
 
+            if (tr && threadIdx.x == 0) tr[4] = global_timer_ns();      // units of this piece consumed
             // ---- end of piece: warps 1..3 hand (O, m, l) to warp 0
 #pragma unroll
             for (int off = 4; off < 32; off <<= 1) {

@@ -190,6 +190,17 @@ struct UnitCursor {
     }
 };
 
+// Activation (B operand) tensor maps with box heights 16, 32, 64, 128, 256 token rows: a tile loads
+// (and multiplies) only as many token rows as it has, rounded up to the next of these sizes; a cold
+// expert with 18 rows costs an N = 32 MMA and a 4 KB load per K block, not the widest tile's.
+struct TmapSetB {
+    CUtensorMap m[5];
+};
+__host__ __device__ __forceinline__ int box_index(int rows) { return rows <= 16 ? 0 : rows <= 32 ? 1 : rows <= 64 ? 2 : rows <= 128 ? 3 : 4; }
+// Box height actually used for a tile with `rows` token rows: never more than the tile (the stage's
+// activation buffer and the TMEM accumulator are sized for n_tile rows).
+__host__ __device__ __forceinline__ int box_rows(int rows, int n_tile) { const int b = 16 << box_index(rows); return b < n_tile ? b : n_tile; }
+
 struct __align__(8) GemmBarriers {
     uint64_t full[kMaxStages];
     uint64_t empty[kMaxStages];
@@ -206,14 +217,13 @@ __device__ __forceinline__ float silu_f32(float z) { return z / (1.0f + __expf(-
 template <int MODE>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__ CUtensorMap tmap_a1,
-            const __grid_constant__ CUtensorMap tmap_b, const GemmParams p) {
+            const __grid_constant__ TmapSetB tmaps_b, const GemmParams p) {
     extern __shared__ uint8_t smem_raw[];
     // 1024-byte alignment: the 128-byte swizzle pattern is a function of address bits [7,10).
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     constexpr int kNumA = (MODE == kGateUp) ? 2 : 1;
     constexpr int kABytes = kBlockM * kBlockK * 2;           // 16 KB
-    const int b_bytes = p.n_tile * kBlockK * 2;
-    const int stage_bytes = kNumA * kABytes + ((b_bytes + 1023) & ~1023);
+    const int stage_bytes = kNumA * kABytes + ((p.n_tile * kBlockK * 2 + 1023) & ~1023);
     GemmBarriers* bars = reinterpret_cast<GemmBarriers*>(smem + (size_t)p.stages * stage_bytes);
 
     const int warp = threadIdx.x >> 5;
@@ -235,7 +245,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
     if (warp == 0 && lane == 0) {
         prefetch_tmap(&tmap_a0);
         if (MODE == kGateUp) prefetch_tmap(&tmap_a1);
-        prefetch_tmap(&tmap_b);
+        for (int i = 0; i <= box_index(p.n_tile); ++i) prefetch_tmap(&tmaps_b.m[i]);
     }
     tc_fence_before();
     __syncthreads();
@@ -256,23 +266,24 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
             const uint64_t pol_w = policy_evict_first();   // weights: streamed once
             const uint64_t pol_x = policy_evict_last();    // activations: re-read by every tile
             int s = 0; uint32_t ph = 0;
-            const uint32_t tx = (uint32_t)(kNumA * kABytes + b_bytes);
             UnitCursor cur(sched, blockIdx.x);
             WorkUnit wu;
             // The first `stages` K blocks find the ring empty: their weight tiles are requested at once,
             // before the grid-dependency wait; their activation tiles follow after it.
             int primed = 0;
-            int pend_kb[kMaxStages], pend_row[kMaxStages];
+            int pend_kb[kMaxStages], pend_row[kMaxStages], pend_box[kMaxStages];
             bool waited = false;
             while (!bars->abort && cur.next(wu)) {
                 const TileCoord c = tiles.get(wu.tile);
+                const int bi = box_index(c.b_rows);
+                const uint32_t tx = (uint32_t)(kNumA * kABytes + box_rows(c.b_rows, p.n_tile) * kBlockK * 2);
                 for (int kb = wu.kb0; kb < wu.kb1; ++kb) {
                     if (primed < p.stages) {
                         uint8_t* st = smem + (size_t)primed * stage_bytes;
                         mbar_expect_tx(&bars->full[primed], tx);
                         tma_load_2d_hint(st, &tmap_a0, kb * kBlockK, c.a_row0, &bars->full[primed], pol_w);
                         if (MODE == kGateUp) tma_load_2d_hint(st + kABytes, &tmap_a1, kb * kBlockK, c.a_row0, &bars->full[primed], pol_w);
-                        pend_kb[primed] = kb; pend_row[primed] = c.b_row0;
+                        pend_kb[primed] = kb; pend_row[primed] = c.b_row0; pend_box[primed] = bi;
                         ++primed;
                         if (++s == p.stages) { s = 0; ph ^= 1; }
                         continue;
@@ -282,8 +293,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
                         pdl_wait();
                         if (tr) tr[2] = global_timer_ns();           // dependency satisfied
                         for (int i = 0; i < primed; ++i)
-                            tma_load_2d_hint(smem + (size_t)i * stage_bytes + kNumA * kABytes, &tmap_b, pend_kb[i] * kBlockK,
-                                             pend_row[i], &bars->full[i], pol_x);
+                            tma_load_2d_hint(smem + (size_t)i * stage_bytes + kNumA * kABytes, &tmaps_b.m[pend_box[i]],
+                                             pend_kb[i] * kBlockK, pend_row[i], &bars->full[i], pol_x);
                         waited = true;
                     }
                     if (!mbar_wait(&bars->empty[s], ph ^ 1)) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); break; }
@@ -291,7 +302,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
                     mbar_expect_tx(&bars->full[s], tx);
                     tma_load_2d_hint(st, &tmap_a0, kb * kBlockK, c.a_row0, &bars->full[s], pol_w);
                     if (MODE == kGateUp) tma_load_2d_hint(st + kABytes, &tmap_a1, kb * kBlockK, c.a_row0, &bars->full[s], pol_w);
-                    tma_load_2d_hint(st + kNumA * kABytes, &tmap_b, kb * kBlockK, c.b_row0, &bars->full[s], pol_x);
+                    tma_load_2d_hint(st + kNumA * kABytes, &tmaps_b.m[bi], kb * kBlockK, c.b_row0, &bars->full[s], pol_x);
                     if (++s == p.stages) { s = 0; ph ^= 1; }
                 }
             }
@@ -299,8 +310,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
             if (!waited) {
                 pdl_wait();
                 for (int i = 0; i < primed; ++i)
-                    tma_load_2d_hint(smem + (size_t)i * stage_bytes + kNumA * kABytes, &tmap_b, pend_kb[i] * kBlockK,
-                                     pend_row[i], &bars->full[i], pol_x);
+                    tma_load_2d_hint(smem + (size_t)i * stage_bytes + kNumA * kABytes, &tmaps_b.m[pend_box[i]],
+                                     pend_kb[i] * kBlockK, pend_row[i], &bars->full[i], pol_x);
             }
             // On abort wait (bounded) for loads still in flight before the CTA leaves.
             if (bars->abort) {
@@ -310,12 +321,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            const uint32_t idesc = umma_idesc_bf16(kBlockM, (uint32_t)p.n_tile);
             int s = 0; uint32_t ph = 0;
             int buf = 0; uint32_t acc_ph = 0;
             UnitCursor cur(sched, blockIdx.x);
             WorkUnit wu;
             while (!bars->abort && cur.next(wu)) {
+                const uint32_t idesc = umma_idesc_bf16(kBlockM, (uint32_t)box_rows(tiles.get(wu.tile).b_rows, p.n_tile));
                 if (!mbar_wait(&bars->tmem_empty[buf], acc_ph ^ 1)) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); break; }
                 tc_fence_after();
                 const uint32_t d0 = tmem_base + (uint32_t)(buf * acc_cols);
@@ -572,6 +583,10 @@ static bool make_config(int mode, int T, int N, int K, int rows_max, int E, int 
     GemmParams& p = cfg->p;
     p.T = T; p.N = N; p.K = K;
     p.n_tile = pick_n_tile(rows_max);
+    // Grouped form: cap the tile at 128 token rows so the two gate/up accumulators stay double-buffered
+    // in TMEM; a hot expert with more rows becomes two adjacent tiles whose weight tiles are read by
+    // neighbouring CTAs at the same time (the second read is an L2 hit).
+    if (E > 0 && p.n_tile > 128) p.n_tile = 128;
     p.m_tiles = (N + kBlockM - 1) / kBlockM;
     p.n_tiles = (T + p.n_tile - 1) / p.n_tile;
     p.kblocks = (K + kBlockK - 1) / kBlockK;
@@ -605,9 +620,17 @@ static bool make_config(int mode, int T, int N, int K, int rows_max, int E, int 
     return true;
 }
 
+static bool encode_b_set(TmapSetB* set, const void* base, uint64_t rows, uint64_t K, int n_tile) {
+    for (int i = 0; i < 5; ++i) {
+        const uint32_t box = (uint32_t)((16 << i) < n_tile ? (16 << i) : n_tile);   // same rule as box_rows()
+        if (!encode_tmap_2d_bf16(&set->m[i], base, rows, K, K * 2, box, kBlockK, false)) return false;
+    }
+    return true;
+}
+
 template <int MODE>
 static aflex_status launch_gemm(aflex_ctx* ctx, const GemmConfig& cfg, const CUtensorMap& ta0, const CUtensorMap& ta1,
-                                const CUtensorMap& tb, cudaStream_t st, int kind) {
+                                const TmapSetB& tb, cudaStream_t st, int kind) {
     if (!ctx->gemm_attr_set[MODE]) {
         cudaError_t e = cudaFuncSetAttribute(gemm_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              kMaxDynamicSmem);
@@ -660,9 +683,10 @@ aflex_status linear_launch(aflex_ctx* ctx, const void* x, const void* w, int T, 
     p.out_bf16 = reinterpret_cast<__nv_bfloat16*>(y);
     aflex_status s = bind_scratch(ctx, cfg, ws, ws_bytes, counters, "linear");
     if (s != AFLEX_OK) return s;
-    CUtensorMap ta, tb;
+    CUtensorMap ta;
+    TmapSetB tb;
     if (!encode_tmap_2d_bf16(&ta, w, (uint64_t)N, (uint64_t)K, (uint64_t)K * 2, kBlockM, kBlockK, true) ||
-        !encode_tmap_2d_bf16(&tb, x, (uint64_t)T, (uint64_t)K, (uint64_t)K * 2, (uint32_t)p.n_tile, kBlockK, false))
+        !encode_b_set(&tb, x, (uint64_t)T, (uint64_t)K, p.n_tile))
         return set_error(ctx, AFLEX_ERR_CUDA, "linear: cuTensorMapEncodeTiled failed");
     return launch_gemm<kLinear>(ctx, cfg, ta, ta, tb, st, kind);
 }
@@ -684,10 +708,11 @@ aflex_status gateup_launch(aflex_ctx* ctx, const void* x, const void* w_gate, co
     p.out_bf16 = reinterpret_cast<__nv_bfloat16*>(h);
     aflex_status s = bind_scratch(ctx, cfg, ws, ws_bytes, counters, "gate/up");
     if (s != AFLEX_OK) return s;
-    CUtensorMap tg, tu, tb;
+    CUtensorMap tg, tu;
+    TmapSetB tb;
     if (!encode_tmap_2d_bf16(&tg, w_gate, (uint64_t)I, (uint64_t)H, (uint64_t)H * 2, kBlockM, kBlockK, true) ||
         !encode_tmap_2d_bf16(&tu, w_up, (uint64_t)I, (uint64_t)H, (uint64_t)H * 2, kBlockM, kBlockK, true) ||
-        !encode_tmap_2d_bf16(&tb, x, (uint64_t)T, (uint64_t)H, (uint64_t)H * 2, (uint32_t)p.n_tile, kBlockK, false))
+        !encode_b_set(&tb, x, (uint64_t)T, (uint64_t)H, p.n_tile))
         return set_error(ctx, AFLEX_ERR_CUDA, "gate/up: cuTensorMapEncodeTiled failed");
     return launch_gemm<kGateUp>(ctx, cfg, tg, tu, tb, st, kKGateUpGemm);
 }
@@ -711,10 +736,11 @@ aflex_status grouped_gateup_launch(aflex_ctx* ctx, const void* xp, const void* w
     p.out_bf16 = reinterpret_cast<__nv_bfloat16*>(hp);
     aflex_status s = bind_scratch(ctx, cfg, ws, ws_bytes, counters, "grouped gate/up");
     if (s != AFLEX_OK) return s;
-    CUtensorMap tg, tu, tb;
+    CUtensorMap tg, tu;
+    TmapSetB tb;
     if (!encode_tmap_2d_bf16(&tg, w_gate, (uint64_t)E * I, (uint64_t)H, (uint64_t)H * 2, kBlockM, kBlockK, true) ||
         !encode_tmap_2d_bf16(&tu, w_up, (uint64_t)E * I, (uint64_t)H, (uint64_t)H * 2, kBlockM, kBlockK, true) ||
-        !encode_tmap_2d_bf16(&tb, xp, (uint64_t)rows_total, (uint64_t)H, (uint64_t)H * 2, (uint32_t)p.n_tile, kBlockK, false))
+        !encode_b_set(&tb, xp, (uint64_t)rows_total, (uint64_t)H, p.n_tile))
         return set_error(ctx, AFLEX_ERR_CUDA, "grouped gate/up: cuTensorMapEncodeTiled failed");
     return launch_gemm<kGateUp>(ctx, cfg, tg, tu, tb, st, kKMoeGateUpGemm);
 }
@@ -732,9 +758,10 @@ aflex_status grouped_linear_launch(aflex_ctx* ctx, const void* hp, const void* w
     p.out_f32 = yp;
     aflex_status s = bind_scratch(ctx, cfg, ws, ws_bytes, counters, "grouped linear");
     if (s != AFLEX_OK) return s;
-    CUtensorMap ta, tb;
+    CUtensorMap ta;
+    TmapSetB tb;
     if (!encode_tmap_2d_bf16(&ta, w_down, (uint64_t)E * N, (uint64_t)K, (uint64_t)K * 2, kBlockM, kBlockK, true) ||
-        !encode_tmap_2d_bf16(&tb, hp, (uint64_t)rows_total, (uint64_t)K, (uint64_t)K * 2, (uint32_t)p.n_tile, kBlockK, false))
+        !encode_b_set(&tb, hp, (uint64_t)rows_total, (uint64_t)K, p.n_tile))
         return set_error(ctx, AFLEX_ERR_CUDA, "grouped linear: cuTensorMapEncodeTiled failed");
     return launch_gemm<kLinear>(ctx, cfg, ta, ta, tb, st, kKMoeDownGemm);
 }
