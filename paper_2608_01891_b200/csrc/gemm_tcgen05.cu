@@ -603,8 +603,10 @@ static bool make_config(int mode, int T, int N, int K, int rows_max, int E, int 
     p.tmem_cols = cols;
     const int a_bytes = accs * kBlockM * kBlockK * 2;
     const int stage_bytes = a_bytes + round_up(p.n_tile * kBlockK * 2, 1024);
-    // few tiles per SM: share the remainder tiles along K; many: whole tiles round-robin
-    p.streamk = (tiles_hi < 8LL * num_sms && tiles_hi <= kStreamKMaxTiles) ? 1 : 0;
+    // few tiles per SM: share the remainder tiles along K; many: whole tiles round-robin.  Wide tiles
+    // (large T, compute-bound) make the shared tiles' partials big, so they are shared only when whole
+    // tiles alone would leave most SMs idle.
+    p.streamk = (tiles_hi < 8LL * num_sms && tiles_hi <= kStreamKMaxTiles && (p.n_tile <= 128 || tiles_hi < 2LL * num_sms)) ? 1 : 0;
     const int cap = (p.streamk && p.n_tile <= 64) ? streaming_smem_budget() : kMaxDynamicSmem;
     const int budget = cap - 1024 /*alignment slack*/ - (int)sizeof(GemmBarriers) - 256;
     int stages = budget / stage_bytes;
