@@ -42,8 +42,33 @@ static EncodeTiledFn get_encode_fn() {
     return fn;
 }
 
+// Encoding a tensor map costs a driver call (~1-2 us) and a decode step launches ~20 loads' worth of
+// maps over the same few tensors every time: keep the encoded maps in a small per-thread cache keyed
+// by everything the encoding depends on (address, extents, stride, box, promotion).
+namespace {
+struct TmapKey {
+    const void* base; uint64_t rows, cols, stride; uint32_t box_rows, box_cols; bool promote;
+    bool operator==(const TmapKey& o) const {
+        return base == o.base && rows == o.rows && cols == o.cols && stride == o.stride && box_rows == o.box_rows &&
+               box_cols == o.box_cols && promote == o.promote;
+    }
+};
+struct TmapCache {
+    static constexpr int kEntries = 128;
+    TmapKey keys[kEntries];
+    CUtensorMap maps[kEntries];
+    int used = 0, next = 0;
+};
+thread_local TmapCache g_tmap_cache;
+}  // namespace
+
 bool encode_tmap_2d_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t row_stride_bytes,
                          uint32_t box_rows, uint32_t box_cols, bool promote_l2_256) {
+    TmapCache& cache = g_tmap_cache;
+    const TmapKey key{base, rows, cols, row_stride_bytes, box_rows, box_cols, promote_l2_256};
+    for (int i = 0; i < cache.used; ++i) {
+        if (cache.keys[i] == key) { *out = cache.maps[i]; return true; }
+    }
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return false;
     cuuint64_t dims[2] = {cols, rows};
@@ -54,7 +79,11 @@ bool encode_tmap_2d_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                     promote_l2_256 ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS;
+    if (r != CUDA_SUCCESS) return false;
+    const int slot = cache.used < TmapCache::kEntries ? cache.used++ : (cache.next = (cache.next + 1) % TmapCache::kEntries);
+    cache.keys[slot] = key;
+    cache.maps[slot] = *out;
+    return true;
 }
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
