@@ -31,6 +31,7 @@
 // replaced (not multiplied) by -inf and their V rows are zeroed in shared memory before use.
 #include <cuda_bf16.h>
 #include <math.h>
+#include <stdlib.h>
 
 #include "internal.h"
 #include "ptx.cuh"
@@ -59,17 +60,30 @@ struct AttnParams {
     __nv_bfloat16* out;    // [B][Hq][D]
     float* lse;            // [B][Hq] or nullptr
     int* counters;         // [B][Hkv] piece-arrival counters, zero on entry and on exit
+    int* ticket;           // [2]: next dynamic chunk, CTAs finished; zero on entry and on exit (unused if dyn_pct == 0)
+    int dyn_pct;           // percent of the unit list handed out dynamically (0 = static shares only)
+    int dyn_chunks;        // target number of dynamic chunks per CTA
     int* status;
     unsigned long long* trace;
 };
 
+// A contiguous run of the unit list handed to a CTA: its static share (rid = CTA index) or a
+// dynamically claimed chunk (rid = grid + chunk index).  x0 == x1 ends the CTA's work.
+struct AttnRange {
+    long long x0, x1;        // unit positions
+    long long prefix;        // units (per KV head) of the sequences before b
+    int b;                   // sequence that contains x0
+    int rid;                 // partial-slot owner id of the range
+};
+constexpr int kRangeRing = 4;
+
 struct __align__(8) AttnShared {
     uint64_t full[kAttnStages];
     uint64_t empty[kAttnStages];
+    uint64_t rng_ready[kRangeRing];
+    AttnRange rng[kRangeRing];
     volatile int abort;
-    int start_b;             // first sequence of this CTA's share
-    long long start_prefix;  // units (per KV head) of the sequences before start_b
-    int scan[kAttnThreads];
+    int scan[kAttnThreads];  // exclusive prefix (units per KV head) of the sequences before each thread's segment
 };
 
 // Position in the (sequence, head, unit) list; every warp of a CTA walks the same sequence of pieces.
@@ -79,11 +93,11 @@ struct Walker {
     long long pos, end;   // unit positions in the global list
     long long prefix;     // units (per head) of the sequences before b
     int b, g, u, nu, len;
-    __device__ void init(const AttnParams& p, const AttnShared* sh, long long begin, long long end_) {
-        lens = p.seq_lens; Hkv = p.Hkv; pos = begin; end = end_;
-        b = sh->start_b; prefix = sh->start_prefix;
+    __device__ void init(const AttnParams& p, const AttnRange& r) {
+        lens = p.seq_lens; Hkv = p.Hkv; pos = r.x0; end = r.x1;
+        b = r.b; prefix = r.prefix;
         len = lens[b]; nu = (len + kUnitTokens - 1) / kUnitTokens;
-        const long long rel = begin - prefix * Hkv;
+        const long long rel = pos - prefix * Hkv;
         g = (int)(rel / nu); u = (int)(rel % nu);
     }
     __device__ bool done() const { return pos >= end; }
@@ -97,6 +111,31 @@ struct Walker {
                 if (pos < end) { len = lens[b]; nu = (len + kUnitTokens - 1) / kUnitTokens; }
             }
         }
+    }
+};
+
+// How the unit list [0, U) is handed out: [0, U1) as one static share per CTA (Ge1 CTAs take part),
+// [U1, U) as n2 chunks of K2 units claimed through a ticket counter by whichever CTA is free.
+struct AttnSplit {
+    long long U, U1;
+    int Ge1, K2, n2;
+    __device__ AttnSplit(long long U_, int grid, int dyn_pct, int dyn_chunks) {
+        U = U_;
+        long long U2 = dyn_pct > 0 ? U * dyn_pct / 100 : 0;
+        // A chunk costs a fixed ~2-3 us (claim, hand-over, an extra partial piece to publish and merge):
+        // chunks below ~12 units (~0.4 MB at D = 128) do not pay, so small launches stay purely static.
+        if (U2 > 0 && U2 / ((long long)dyn_chunks * grid) < 12) U2 = 0;
+        if (U2 > 0) {
+            long long k = (U2 + (long long)dyn_chunks * grid - 1) / ((long long)dyn_chunks * grid);
+            K2 = (int)(k < 2 ? 2 : (k > 64 ? 64 : k));
+            n2 = (int)((U2 + K2 - 1) / K2);
+            // keep the slot count bounded: never more than dyn_chunks * grid + 1 chunks
+            if (n2 > dyn_chunks * grid + 1) { n2 = dyn_chunks * grid + 1; }
+            U2 = min(U2, (long long)n2 * K2);
+        } else { K2 = 1; n2 = 0; }
+        U1 = U - U2;
+        n2 = U2 > 0 ? (int)((U2 + K2 - 1) / K2) : 0;
+        Ge1 = (int)min((long long)grid, U1);
     }
 };
 
@@ -137,6 +176,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             mbar_init(&sh->full[s], 1);
             mbar_init(&sh->empty[s], kAttnConsumerWarps);
         }
+        for (int i = 0; i < kRangeRing; ++i) mbar_init(&sh->rng_ready[i], 1);
         sh->abort = 0;
         fence_mbar_init();
         prefetch_tmap(&tmap_k);
@@ -145,41 +185,55 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     pdl_wait();   // q, the page table and the lengths may come from the preceding kernel
     if (tr && threadIdx.x == 0) tr[2] = global_timer_ns();
 
-    // ---- share of this CTA: block-wide prefix over ceil(len/64), then locate the first sequence
+    // ---- block-wide exclusive prefix over ceil(len/64): thread t owns sequences [t*per_thread, ...)
     const int per_thread = (p.batch + kAttnThreads - 1) / kAttnThreads;
-    const int b_lo = min(p.batch, (int)threadIdx.x * per_thread), b_hi = min(p.batch, b_lo + per_thread);
-    int local = 0;
-    for (int b = b_lo; b < b_hi; ++b) local += (p.seq_lens[b] + kUnitTokens - 1) / kUnitTokens;
-    sh->scan[threadIdx.x] = local;
-    __syncthreads();
-    long long before = 0, total = 0;
-    for (int t = 0; t < kAttnThreads; ++t) {
-        const int v = sh->scan[t];
-        if (t < (int)threadIdx.x) before += v;
-        total += v;
-    }
-    const long long U = total * p.Hkv;
-    const int Ge = (int)min((long long)gridDim.x, U);
-    if (cta >= Ge) return;                                    // uniform for the whole CTA
-    const long long x_begin = share_begin(U, cta, Ge), x_end = share_begin(U, cta + 1, Ge);
-    if (local > 0 && before * p.Hkv <= x_begin && x_begin < (before + local) * p.Hkv) {
-        long long pre = before;
-        int b = b_lo;
-        for (; b < b_hi; ++b) {
-            const int nu = (p.seq_lens[b] + kUnitTokens - 1) / kUnitTokens;
-            if (x_begin < (pre + nu) * p.Hkv) break;
-            pre += nu;
+    {
+        const int b_lo = min(p.batch, (int)threadIdx.x * per_thread), b_hi = min(p.batch, b_lo + per_thread);
+        int local = 0;
+        for (int b = b_lo; b < b_hi; ++b) local += (p.seq_lens[b] + kUnitTokens - 1) / kUnitTokens;
+        // inclusive warp scan, then warp totals through shared memory
+        int incl = local;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, off);
+            if (lane >= off) incl += v;
         }
-        sh->start_b = b;
-        sh->start_prefix = pre;
+        __shared__ int warp_tot[kAttnConsumerWarps + 1];
+        if (lane == 31) warp_tot[warp] = incl;
+        __syncthreads();
+        int base = 0;
+        for (int w = 0; w < warp; ++w) base += warp_tot[w];
+        sh->scan[threadIdx.x] = base + incl - local;
+        if (threadIdx.x == kAttnThreads - 1) sh->rng[0].x0 = base + incl;   // grand total, parked for everyone
+        __syncthreads();
     }
+    const long long U = sh->rng[0].x0 * (long long)p.Hkv;
     __syncthreads();
-    if (tr && threadIdx.x == 0) tr[1] = global_timer_ns();            // share located
+    const AttnSplit sp(U, (int)gridDim.x, p.dyn_pct, p.dyn_chunks);
+    if (tr && threadIdx.x == 0) tr[1] = global_timer_ns();            // prefix ready
+
+    // Sequence that contains unit position x (cooperative over the 32 lanes of one warp).
+    auto locate = [&](long long x, int& b_out, long long& prefix_out) {
+        int best = 0;
+#pragma unroll
+        for (int k = 0; k < kAttnThreads / 32; ++k) {
+            const int t = lane * (kAttnThreads / 32) + k;
+            if ((long long)sh->scan[t] * p.Hkv <= x) best = t;      // scan is non-decreasing
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) best = max(best, __shfl_xor_sync(0xffffffffu, best, off));
+        int b = min(p.batch - 1, best * per_thread);
+        long long pre = sh->scan[best];
+        while (b + 1 < p.batch) {
+            const int nu = (p.seq_lens[b] + kUnitTokens - 1) / kUnitTokens;
+            if (x < (pre + nu) * p.Hkv) break;
+            pre += nu; ++b;
+        }
+        b_out = b; prefix_out = pre;
+    };
 
     if (warp == kAttnConsumerWarps) {
         // ------------------------------------------------------------------ producer warp
-        Walker wk;
-        wk.init(p, sh, x_begin, x_end);
         const int pg = lane / (2 * kHalves);
         const int kv = (lane / kHalves) & 1;
         const int hf = lane % kHalves;
@@ -188,42 +242,91 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             const int idx = w.u * kPagesPerStage + pg;
             return (op_lane && idx * kPage < w.len) ? p.page_table[(size_t)w.b * p.max_pages + idx] : 0;
         };
-        int pid = page_id(wk);
         int s = 0;
         uint32_t ph = 0;
-        while (!wk.done()) {
-            const int g = wk.g, u = wk.u, len = wk.len;
-            wk.advance(1);
-            const int pid_next = wk.done() ? 0 : page_id(wk);   // one unit ahead of the ring
-            bool ok = mbar_wait(&sh->empty[s], ph ^ 1);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok || sh->abort) {
-                if (lane == 0) { sh->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); }
-                break;
+        int r = 0;                       // ranges published so far
+        bool aborted = false;
+        // range 0: the static share; later ranges: claimed chunks
+        long long x0 = 0, x1 = 0;
+        int rid = cta;
+        if (cta < sp.Ge1) { x0 = share_begin(sp.U1, cta, sp.Ge1); x1 = share_begin(sp.U1, cta + 1, sp.Ge1); }
+        int next_ticket = -1;
+        while (true) {
+            if (sp.n2 > 0) {             // claim the chunk after this range now: the round trip hides behind the range
+                if (lane == 0) next_ticket = atomicAdd(&p.ticket[0], 1);
+                next_ticket = __shfl_sync(0xffffffffu, next_ticket, 0);
             }
-            const int np = min(kPagesPerStage, (len - u * kUnitTokens + kPage - 1) / kPage);
-            if (lane == 0) mbar_expect_tx(&sh->full[s], (uint32_t)(np * 2 * kPageBytes));
-            __syncwarp();
-            if (op_lane && pg < np) {
-                int id = pid;
-                if (id < 0 || id >= p.num_pages) { atomicExch(p.status, AFLEX_ERR_BOUNDS); id = 0; }
-                uint8_t* dst = smem + s * kStageBytes + kv * (kPagesPerStage * kPageBytes) + pg * kPageBytes + hf * (kPage * 128);
-                const int row = (id * p.Hkv + g) * kPage;
-                tma_load_2d(dst, kv ? &tmap_v : &tmap_k, hf * 64, row, &sh->full[s]);
+            if (x1 > x0) {
+                AttnRange rg;
+                rg.x0 = x0; rg.x1 = x1; rg.rid = rid;
+                locate(x0, rg.b, rg.prefix);
+                if (lane == 0) { sh->rng[r % kRangeRing] = rg; mbar_arrive(&sh->rng_ready[r % kRangeRing]); }
+                ++r;
+                Walker wk;
+                wk.init(p, rg);
+                int pid = page_id(wk);
+                while (!wk.done()) {
+                    const int g = wk.g, u = wk.u, len = wk.len;
+                    wk.advance(1);
+                    const int pid_next = wk.done() ? 0 : page_id(wk);   // one unit ahead of the ring
+                    bool ok = mbar_wait(&sh->empty[s], ph ^ 1);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok || sh->abort) {
+                        if (lane == 0) { sh->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); }
+                        aborted = true;
+                        break;
+                    }
+                    const int np = min(kPagesPerStage, (len - u * kUnitTokens + kPage - 1) / kPage);
+                    if (lane == 0) mbar_expect_tx(&sh->full[s], (uint32_t)(np * 2 * kPageBytes));
+                    __syncwarp();
+                    if (op_lane && pg < np) {
+                        int id = pid;
+                        if (id < 0 || id >= p.num_pages) { atomicExch(p.status, AFLEX_ERR_BOUNDS); id = 0; }
+                        uint8_t* dst = smem + s * kStageBytes + kv * (kPagesPerStage * kPageBytes) + pg * kPageBytes + hf * (kPage * 128);
+                        const int row = (id * p.Hkv + g) * kPage;
+                        tma_load_2d(dst, kv ? &tmap_v : &tmap_k, hf * 64, row, &sh->full[s]);
+                    }
+                    pid = pid_next;
+                    if (++s == kAttnStages) { s = 0; ph ^= 1; }
+                }
             }
-            pid = pid_next;
-            if (++s == kAttnStages) { s = 0; ph ^= 1; }
+            if (aborted || sp.n2 == 0 || next_ticket >= sp.n2) break;
+            x0 = sp.U1 + (long long)next_ticket * sp.K2;
+            x1 = min(sp.U, x0 + sp.K2);
+            rid = (int)gridDim.x + next_ticket;
+        }
+        // end marker for the consumers
+        if (lane == 0) {
+            AttnRange rg;
+            rg.x0 = 0; rg.x1 = 0; rg.prefix = 0; rg.b = 0; rg.rid = -1;
+            sh->rng[r % kRangeRing] = rg;
+            mbar_arrive(&sh->rng_ready[r % kRangeRing]);
+            if (sp.n2 > 0) {
+                // last CTA out resets the ticket counters (every CTA has made its final claim by now)
+                __threadfence();
+                if (atomicAdd(&p.ticket[1], 1) == (int)gridDim.x - 1) { p.ticket[0] = 0; p.ticket[1] = 0; }
+            }
         }
     } else {
         // ------------------------------------------------------------------ consumer warps
-        Walker wk;
-        wk.init(p, sh, x_begin, x_end);
         const int mi = lane >> 3, r8 = lane & 7;
         const int h0 = 2 * (lane & 3);          // this lane's two heads of the group: h0, h0 + 1
         int s = 0;
         uint32_t ph = 0;
-        bool first_piece = true;                // a partial piece uses slot 0 if it is the CTA's first piece, else 1
         bool aborted = false;
+        const int G = (int)gridDim.x;
+
+        for (int r = 0; !aborted; ++r) {
+            // ---- next range of this CTA
+            if (!mbar_wait(&sh->rng_ready[r % kRangeRing], (uint32_t)((r / kRangeRing) & 1))) {
+                if (lane == 0) { sh->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); }
+                break;
+            }
+            const AttnRange rg = sh->rng[r % kRangeRing];
+            if (rg.x1 <= rg.x0) break;
+            Walker wk;
+            wk.init(p, rg);
+            bool first_piece = true;            // a partial piece uses slot 0 if it is the range's first piece, else 1
 
         while (!wk.done() && !aborted) {
             // ---- one piece: units [u0, u0 + n) of item (b, g)
@@ -394,10 +497,10 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                 }
                 continue;
             }
-            // ---- partial piece: park it in this CTA's next slot, bump the item's counter
+            // ---- partial piece: park it in the range's slot, bump the item's counter
             {
-                float* op = p.o_part + ((size_t)cta * 2 + slot) * 8 * D;
-                float* mlp = p.ml_part + ((size_t)cta * 2 + slot) * 8 * 2;
+                float* op = p.o_part + ((size_t)rg.rid * 2 + slot) * 8 * D;
+                float* mlp = p.ml_part + ((size_t)rg.rid * 2 + slot) * 8 * 2;
 #pragma unroll
                 for (int mt = 0; mt < kKSteps; ++mt) {
                     op[(h0) * D + mt * 16 + dr] = o[mt][0];
@@ -411,18 +514,30 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                 }
             }
             __syncwarp();
-            const int cf = cta_of_unit(item_x0, U, Ge);
-            const int cl = cta_of_unit(item_x0 + nu - 1, U, Ge);
+            // pieces of this item: static shares cf..cl over [item_x0, min(item_x1, U1)), then dynamic chunks jf..jl
+            const long long item_x1 = item_x0 + nu;
+            int cf = 0, cl = -1, jf = 0, jl = -1;
+            if (item_x0 < sp.U1) {
+                cf = cta_of_unit(item_x0, sp.U1, sp.Ge1);
+                cl = cta_of_unit(min(item_x1, sp.U1) - 1, sp.U1, sp.Ge1);
+            }
+            const long long dyn_x0 = max(item_x0, sp.U1);
+            if (item_x1 > sp.U1) {
+                jf = (int)((dyn_x0 - sp.U1) / sp.K2);
+                jl = (int)((item_x1 - 1 - sp.U1) / sp.K2);
+            }
+            const int expected = (cl - cf + 1) + (jl - jf + 1);
             int last = 0;
             if (lane == 0) {
                 __threadfence();
-                last = (atomicAdd(&p.counters[b * p.Hkv + g], 1) == cl - cf) ? 1 : 0;
+                last = (atomicAdd(&p.counters[b * p.Hkv + g], 1) == expected - 1) ? 1 : 0;
             }
             last = __shfl_sync(0xffffffffu, last, 0);
             if (!last) continue;
-            // ---- last arriver: merge the item's pieces in CTA order cf..cl (one pass, running maximum).
+            // ---- last arriver: merge the item's pieces in list order (one pass, running maximum).
             // Lane owns d = 4*lane + 128*j .. +3 of every head: all loads of a piece are independent.
-            // Only the first piece can belong to a CTA whose share began before the item (its slot 1).
+            // A piece sits in slot 0 of its range unless other units of the range precede it (slot 1):
+            // that can only happen for the first static share and for the first dynamic chunk.
             __threadfence();
             constexpr int kVec = D / 128 > 0 ? D / 128 : 1;      // float4 per head per lane (D = 64: lanes 16.. idle)
             const bool lane_on = lane * 4 < D;
@@ -434,9 +549,18 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
 #pragma unroll
                 for (int j = 0; j < kVec; ++j) acc[h][j] = make_float4(0.f, 0.f, 0.f, 0.f);
             }
-            for (int c = cf; c <= cl; ++c) {
-                const int sl = (c == cf && share_begin(U, cf, Ge) < item_x0) ? 1 : 0;
-                const size_t base = ((size_t)c * 2 + sl) * 8;
+            const int n_static = cl - cf + 1;
+            for (int i = 0; i < expected; ++i) {
+                int rid_i, sl;
+                if (i < n_static) {
+                    rid_i = cf + i;
+                    sl = (i == 0 && share_begin(sp.U1, cf, sp.Ge1) < item_x0) ? 1 : 0;
+                } else {
+                    const int j = jf + (i - n_static);
+                    rid_i = G + j;
+                    sl = (j == jf && sp.U1 + (long long)jf * sp.K2 < dyn_x0) ? 1 : 0;
+                }
+                const size_t base = ((size_t)rid_i * 2 + sl) * 8;
                 float2 ml[8];
                 float4 o4[8][kVec];
 #pragma unroll
@@ -488,6 +612,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             }
             if (lane == 0) p.counters[b * p.Hkv + g] = 0;   // clean for the next launch
         }
+        }
         if (tr && threadIdx.x == 0) tr[5] = global_timer_ns();
     }
 }
@@ -499,8 +624,24 @@ int attn_grid(const aflex_ctx* ctx) {
     return g;
 }
 
+// Dynamic hand-out of the tail of the unit list (tuning: AFLEX_ATTN_DYN_PCT, AFLEX_ATTN_DYN_CHUNKS).
+static int attn_dyn_pct() {
+    static int v = -1;
+    if (v < 0) { const char* e = getenv("AFLEX_ATTN_DYN_PCT"); v = e ? atoi(e) : 15; if (v < 0) v = 0; if (v > 90) v = 90; }
+    return v;
+}
+static int attn_dyn_chunks() {
+    static int v = -1;
+    if (v < 0) { const char* e = getenv("AFLEX_ATTN_DYN_CHUNKS"); v = e ? atoi(e) : 4; if (v < 1) v = 1; if (v > 64) v = 64; }
+    return v;
+}
+
+// Partial slots: two per range id; range ids = one static share per CTA plus at most
+// dyn_chunks * grid + 1 dynamic chunks.
+static size_t attn_slots(int grid) { return ((size_t)grid * (1 + attn_dyn_chunks()) + 2) * 2; }
+
 size_t attn_workspace_bytes(const aflex_attn_desc* d, int grid) {
-    return align256((size_t)grid * 2 * 8 * d->head_dim * sizeof(float)) + align256((size_t)grid * 2 * 8 * 2 * sizeof(float));
+    return align256(attn_slots(grid) * 8 * d->head_dim * sizeof(float)) + align256(attn_slots(grid) * 8 * 2 * sizeof(float));
 }
 
 template <int D>
@@ -514,8 +655,8 @@ static aflex_status attn_launch_t(aflex_ctx* ctx, const aflex_attn_desc* d, cons
         return set_error(ctx, AFLEX_ERR_WORKSPACE, "attention: need %zu workspace bytes, have %zu", need, ws_bytes);
     Arena arena(ws, ws_bytes);
     AttnParams p;
-    p.o_part = arena.take<float>((size_t)grid * 2 * 8 * D);
-    p.ml_part = arena.take<float>((size_t)grid * 2 * 8 * 2);
+    p.o_part = arena.take<float>(attn_slots(grid) * 8 * D);
+    p.ml_part = arena.take<float>(attn_slots(grid) * 8 * 2);
     p.q = reinterpret_cast<const __nv_bfloat16*>(q);
     p.page_table = kv->page_table;
     p.seq_lens = kv->seq_lens;
@@ -525,6 +666,9 @@ static aflex_status attn_launch_t(aflex_ctx* ctx, const aflex_attn_desc* d, cons
     p.num_pages = kv->num_pages;
     const float scale = d->sm_scale != 0.f ? d->sm_scale : 1.0f / sqrtf((float)D);
     p.scale_log2 = scale * 1.4426950408889634f;
+    p.ticket = ctx->counters_attn + kAttnCounterCap;      // two ints past the per-item counters
+    p.dyn_pct = attn_dyn_pct();
+    p.dyn_chunks = attn_dyn_chunks();
     p.status = ctx->dev_status;
     p.out = reinterpret_cast<__nv_bfloat16*>(out);
     p.lse = lse;
@@ -632,6 +776,9 @@ static aflex_status attn_static_launch(StaticDeviceState& stt, const aflex_attn_
     p.out = reinterpret_cast<__nv_bfloat16*>(out);
     p.lse = lse;
     p.counters = counters;
+    p.ticket = nullptr;     // static shares only: the fixed scratch has two slots per CTA
+    p.dyn_pct = 0;
+    p.dyn_chunks = 1;
     p.trace = nullptr;
 
     const uint64_t rows = (uint64_t)kv->num_pages * d->num_kv_heads * kPage;
