@@ -236,6 +236,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
         fence_mbar_init();
     }
     if (p.num_experts > 0) {
+        // the expert segment offsets come from an earlier kernel of the same chain: they are only
+        // valid once the grid dependency has resolved (so the grouped form cannot prefetch weights early)
+        pdl_wait();
         for (int i = threadIdx.x; i <= p.num_experts; i += blockDim.x) bars->seg[i] = p.offsets[i];
     }
     if (warp == 1) {

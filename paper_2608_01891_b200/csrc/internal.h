@@ -76,6 +76,23 @@ struct KernelScope {
     ~KernelScope() { if (slot >= 0) cudaEventRecord(ctx->prof[slot].stop, st); }
 };
 
+// Launch with programmatic stream serialization: the kernel may start while its predecessor in the
+// stream is still draining; it must execute griddepcontrol.wait before touching the predecessor's output.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = grid;
+    lc.blockDim = block;
+    lc.dynamicSmemBytes = smem;
+    lc.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    return cudaLaunchKernelEx(&lc, kernel, static_cast<KArgs>(args)...);
+}
+
 // Bump allocator over a byte range of the ctx workspace (256-byte granules).
 struct Arena {
     char* base;

@@ -5,6 +5,7 @@
 #include <cuda_bf16.h>
 
 #include "internal.h"
+#include "ptx.cuh"
 
 namespace aflex {
 
@@ -16,6 +17,8 @@ constexpr int kRouteMaxExperts = 64;
 // then butterfly, order).  One warp per (t, e).
 __global__ void router_logits_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ w,
                                      int T, int H, int E, float* __restrict__ logits) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     if (gw >= T * E) return;
@@ -53,7 +56,9 @@ moe_route_kernel(const float* __restrict__ logits, int T, int E, int K, int32_t*
     __shared__ int s_running[kRouteMaxExperts];
     __shared__ int s_warp[kRouteWarps][kRouteMaxExperts];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    pdl_launch_dependents();
     if (tid < kRouteMaxExperts) { s_count[tid] = 0; s_running[tid] = 0; }
+    pdl_wait();
     __syncthreads();
 
     for (int t = tid; t < T; t += kRouteThreads) {
@@ -125,6 +130,8 @@ moe_route_kernel(const float* __restrict__ logits, int T, int E, int K, int32_t*
 // xp[pos[t][k]][:] = x[t][:]
 __global__ void moe_gather_kernel(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ pos, int K, int H,
                                   __nv_bfloat16* __restrict__ xp) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int a = blockIdx.x;          // assignment index t*K + k
     const int t = a / K;
     const uint4* src = reinterpret_cast<const uint4*>(x + (size_t)t * H);
@@ -135,6 +142,8 @@ __global__ void moe_gather_kernel(const __nv_bfloat16* __restrict__ x, const int
 // y[t][:] = sum_{k ascending} gate[t][k] * yp[pos[t][k]][:]   (fp32) -> bf16
 __global__ void moe_combine_kernel(const float* __restrict__ yp, const int32_t* __restrict__ pos,
                                    const float* __restrict__ gate, int K, int H, __nv_bfloat16* __restrict__ y) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int t = blockIdx.x;
     for (int i = threadIdx.x; i < H / 4; i += blockDim.x) {
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -158,31 +167,32 @@ aflex_status moe_router_logits_launch(aflex_ctx* ctx, const void* x, const void*
     const int threads = 256;
     const int blocks = (warps * 32 + threads - 1) / threads;
     KernelScope scope(ctx, kKRouterLogits, st);
-    router_logits_kernel<<<blocks, threads, 0, st>>>((const __nv_bfloat16*)x, (const __nv_bfloat16*)w_router, T, H, E,
-                                                     logits);
-    return check_cuda(ctx, cudaGetLastError(), "router_logits_kernel launch");
+    return check_cuda(ctx, launch_pdl(router_logits_kernel, dim3(blocks), dim3(threads), 0, st, (const __nv_bfloat16*)x,
+                                      (const __nv_bfloat16*)w_router, T, H, E, logits),
+                      "router_logits_kernel launch");
 }
 
 aflex_status moe_route_launch(aflex_ctx* ctx, const float* logits, int T, int E, int K, const MoeBuffers& mb,
                               cudaStream_t st) {
     KernelScope scope(ctx, kKMoeRoute, st);
-    moe_route_kernel<<<1, kRouteThreads, 0, st>>>(logits, T, E, K, mb.idx, mb.gate, mb.counts, mb.offsets, mb.pos,
-                                                  nullptr);
-    return check_cuda(ctx, cudaGetLastError(), "moe_route_kernel launch");
+    return check_cuda(ctx, launch_pdl(moe_route_kernel, dim3(1), dim3(kRouteThreads), 0, st, logits, T, E, K, mb.idx, mb.gate,
+                                      mb.counts, mb.offsets, mb.pos, (int32_t*)nullptr),
+                      "moe_route_kernel launch");
 }
 
 aflex_status moe_gather_launch(aflex_ctx* ctx, const void* x, const int32_t* pos, int T, int K, int H, void* xp,
                                cudaStream_t st) {
     KernelScope scope(ctx, kKMoeGather, st);
-    moe_gather_kernel<<<T * K, 128, 0, st>>>((const __nv_bfloat16*)x, pos, K, H, (__nv_bfloat16*)xp);
-    return check_cuda(ctx, cudaGetLastError(), "moe_gather_kernel launch");
+    return check_cuda(ctx, launch_pdl(moe_gather_kernel, dim3(T * K), dim3(128), 0, st, (const __nv_bfloat16*)x, pos, K, H,
+                                      (__nv_bfloat16*)xp),
+                      "moe_gather_kernel launch");
 }
 
 aflex_status moe_combine_launch(aflex_ctx* ctx, const float* yp, const int32_t* pos, const float* gate, int T, int K,
                                 int H, void* y, cudaStream_t st) {
     KernelScope scope(ctx, kKMoeCombine, st);
-    moe_combine_kernel<<<T, 256, 0, st>>>(yp, pos, gate, K, H, (__nv_bfloat16*)y);
-    return check_cuda(ctx, cudaGetLastError(), "moe_combine_kernel launch");
+    return check_cuda(ctx, launch_pdl(moe_combine_kernel, dim3(T), dim3(256), 0, st, yp, pos, gate, K, H, (__nv_bfloat16*)y),
+                      "moe_combine_kernel launch");
 }
 
 }  // namespace aflex
