@@ -141,6 +141,34 @@ def algorithmic_flops(cfg, M):
             "moe_gateup_gemm": 4.0 * rows * k * H * I, "moe_down_gemm": 2.0 * rows * k * H * I}
 
 
+def measure_energy(step, barrier, gpu_index, tokens_per_step, ms_step):
+    """Joules per token from nvmlDeviceGetTotalEnergyConsumption around a >= 2 s loop of the step, at the
+    clocks the GPU is found at (GPU settings are never changed).  Returns a dict, or a reason string."""
+    try:
+        import pynvml
+        pynvml.nvmlInit()
+        # NVML enumerates physical GPUs; map through CUDA_VISIBLE_DEVICES when it is a plain index list
+        vis = os.environ.get("CUDA_VISIBLE_DEVICES", "")
+        idx = gpu_index
+        if vis and all(v.strip().isdigit() for v in vis.split(",")):
+            idx = int(vis.split(",")[gpu_index])
+        h = pynvml.nvmlDeviceGetHandleByIndex(idx)
+        steps = max(50, int(2000.0 / max(ms_step, 1e-3)))
+        barrier()
+        e0 = pynvml.nvmlDeviceGetTotalEnergyConsumption(h)
+        t0 = time.perf_counter()
+        for _ in range(steps):
+            step()
+        barrier()
+        dt = time.perf_counter() - t0
+        e1 = pynvml.nvmlDeviceGetTotalEnergyConsumption(h)
+        joules = (e1 - e0) / 1000.0
+        return {"joules_per_token": joules / (steps * tokens_per_step), "watts_avg": joules / dt, "seconds": round(dt, 2),
+                "steps": steps, "clocks": "as found (locked-clock sweep: changing GPU settings is closed on this pool)"}
+    except Exception as exc:   # no NVML, no permission, unsupported counter
+        return {"unavailable": str(exc)[:200]}
+
+
 def build_workload(cfg, device):
     """Everything resident in HBM before the timed region starts."""
     from paper_2608_01891_b200 import aflex as AF
@@ -222,6 +250,8 @@ def main():
     ap.add_argument("--ref-rows", type=int, default=0,
                     help="batch rows per reference/cpu-baseline sample (0 = about 15e9 multiply-adds of oracle work)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--energy", action="store_true",
+                    help="also read the NVML energy counter around a >= 2 s loop of the step (default clocks)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
@@ -350,6 +380,11 @@ def main():
     e2e = {"value": whole_job_tokens_per_s(world, cfg.batch, ms_e2e), "unit": "tokens/s", "ms_per_step": ms_e2e,
            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
 
+    # ---- energy per token at default clocks (read-only NVML; the paper's metric, Section 6.1)
+    energy = None
+    if args.energy and rank == 0:
+        energy = measure_energy(step, barrier, local_rank, cfg.batch, ms_step)
+
     # ---- CPU baseline: the oracle on a bounded sample, rank 0 at N = 1 only
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -370,6 +405,8 @@ def main():
                            "parallelism": "replicas only" if world > 1 else "1 GPU"},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "kernels": kernels,
                 "cpu_baseline": cpu}
+        if energy is not None:
+            line["energy"] = energy
         print(json.dumps(line), flush=True)
     ctx.close()
     if dist is not None:

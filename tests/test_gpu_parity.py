@@ -293,3 +293,90 @@ def test_argument_validation_returns_status_without_launching(ctx):
         small.close()
     torch.cuda.synchronize()
     assert ctx.device_status() == AF.OK
+
+
+# ------------------------------------------------------------------------------- edge cases
+def test_attention_single_sequence_and_very_long_context(ctx):
+    """B = 1 with the longest context of the benchmark set (16384 tokens) and B = 1 with one token."""
+    for lens in ([16384], [1], [16383, 2]):
+        q, kv = make_case(len(lens), 32, 8, 128, lens, seed=7)
+        got, lse = run_attention(ctx, q, kv.k_cache, kv.v_cache, kv.page_table, kv.seq_lens, 32, 8, 128)
+        want, want_lse = O.attn_decode(u16(q), u16(kv.k_cache), u16(kv.v_cache), kv.page_table.numpy(), kv.seq_lens.numpy())
+        assert row_rel_err(got, want) <= TOL_ATTN
+        assert np.abs(lse - want_lse).max() <= TOL_LSE
+
+
+def test_attention_many_short_sequences(ctx):
+    """More (sequence, head) items than 64-token units per CTA: most pieces are whole items."""
+    rng = np.random.default_rng(5)
+    lens = rng.integers(1, 90, size=700).tolist()
+    q, kv = make_case(len(lens), 8, 2, 64, lens, seed=8, poison=True)
+    got, _ = run_attention(ctx, q, kv.k_cache, kv.v_cache, kv.page_table, kv.seq_lens, 8, 2, 64)
+    want, _ = O.attn_decode(u16(q), u16(kv.k_cache), u16(kv.v_cache), kv.page_table.numpy(), kv.seq_lens.numpy())
+    assert row_rel_err(got, want) <= TOL_ATTN
+
+
+def test_attention_gqa_groups_1_and_2(ctx):
+    for Hq, Hkv in ((4, 4), (8, 4)):
+        lens = [5, 200, 64, 333]
+        q, kv = make_case(len(lens), Hq, Hkv, 128, lens, seed=9)
+        got, _ = run_attention(ctx, q, kv.k_cache, kv.v_cache, kv.page_table, kv.seq_lens, Hq, Hkv, 128)
+        want, _ = O.attn_decode(u16(q), u16(kv.k_cache), u16(kv.v_cache), kv.page_table.numpy(), kv.seq_lens.numpy())
+        assert row_rel_err(got, want) <= TOL_ATTN
+
+
+def test_out_of_range_page_id_is_reported_not_dereferenced(ctx):
+    """A page id beyond the pool sets AFLEX_ERR_BOUNDS in the device status word; the load is redirected
+    to page 0 (no fault) and the context stays usable."""
+    lens = [40, 70]
+    q, kv = make_case(2, 8, 2, 64, lens, seed=10)
+    table = kv.page_table.clone()
+    table[1, 2] = kv.num_pages + 12345
+    run_attention(ctx, q, kv.k_cache, kv.v_cache, table, kv.seq_lens, 8, 2, 64)
+    assert ctx.device_status() == AF.ERR_BOUNDS
+    assert ctx.device_status() == AF.OK            # reading clears it
+    got, _ = run_attention(ctx, q, kv.k_cache, kv.v_cache, kv.page_table, kv.seq_lens, 8, 2, 64)
+    want, _ = O.attn_decode(u16(q), u16(kv.k_cache), u16(kv.v_cache), kv.page_table.numpy(), kv.seq_lens.numpy())
+    assert row_rel_err(got, want) <= TOL_ATTN
+
+
+def test_moe_many_experts_top1_and_empty_experts(ctx):
+    """E = 64 experts with 5 tokens: almost every expert is empty; K = 1 and K = 2."""
+    T, H, I, E = 5, 128, 256, 64
+    x = rand_bf16((T, H), 1.0, 1)
+    wg, wu, wd = rand_bf16((E, I, H), 0.1, 2), rand_bf16((E, I, H), 0.1, 3), rand_bf16((E, H, I), 0.1, 4)
+    logits = torch.randn(T, E, generator=torch.Generator().manual_seed(11))
+    for K in (1, 2):
+        y, idx, gate, counts = run_moe(ctx, x, logits, wg, wu, wd, K)
+        want_y, want_idx, want_gate = O.ffn_moe(u16(x), logits.numpy(), u16(wg), u16(wu), u16(wd), K)
+        assert (idx == want_idx).all() and counts.sum() == T * K
+        assert np.abs(gate - want_gate).max() <= TOL_GATE
+        assert row_rel_err(y, want_y) <= TOL_FFN
+
+
+def test_moe_all_tokens_to_one_expert(ctx):
+    """Degenerate load: one expert receives every token (its segment spans several token chunks)."""
+    T, H, I, E = 300, 128, 256, 8
+    x = rand_bf16((T, H), 1.0, 1)
+    wg, wu, wd = rand_bf16((E, I, H), 0.1, 2), rand_bf16((E, I, H), 0.1, 3), rand_bf16((E, H, I), 0.1, 4)
+    logits = torch.zeros(T, E)
+    logits[:, 5] = 4.0
+    logits[:, 2] = 1.0
+    y, idx, gate, counts = run_moe(ctx, x, logits, wg, wu, wd, 2)
+    want_y, want_idx, _ = O.ffn_moe(u16(x), logits.numpy(), u16(wg), u16(wu), u16(wd), 2)
+    assert (idx == want_idx).all() and counts[5] == T and counts[2] == T
+    assert row_rel_err(y, want_y) <= TOL_FFN
+
+
+def test_dense_ffn_large_token_count_uses_whole_tile_path(ctx):
+    """T = 1100 at a small FFN: several 256-token tiles per weight tile (the compute-bound schedule)."""
+    T, H, I = 1100, 256, 1024
+    x = rand_bf16((T, H), 1.0, 1)
+    wg, wu, wd = rand_bf16((I, H), 0.08, 2), rand_bf16((I, H), 0.08, 3), rand_bf16((H, I), 0.08, 4)
+    y = torch.full((T, H), float("nan"), dtype=torch.bfloat16, device=DEV)
+    ctx.ffn_dense(x.to(DEV), wg.to(DEV), wu.to(DEV), wd.to(DEV), y)
+    torch.cuda.synchronize()
+    rows = [0, 1, 255, 256, 257, 511, 512, 1023, 1024, 1099]
+    want = O.ffn_dense(u16(x[rows]), u16(wg), u16(wu), u16(wd))
+    assert row_rel_err(f64(y[rows]), want) <= TOL_FFN
+    assert torch.isfinite(y.float()).all()
