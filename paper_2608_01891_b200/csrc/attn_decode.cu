@@ -63,6 +63,7 @@ struct AttnParams {
     int* ticket;           // [2]: next dynamic chunk, CTAs finished; zero on entry and on exit (unused if dyn_pct == 0)
     int dyn_pct;           // percent of the unit list handed out dynamically (0 = static shares only)
     int dyn_chunks;        // target number of dynamic chunks per CTA
+    int piece_cost;        // list positions charged per item start (balances the fixed cost of a piece)
     int* status;
     unsigned long long* trace;
 };
@@ -87,16 +88,19 @@ struct __align__(8) AttnShared {
 };
 
 // Position in the (sequence, head, unit) list; every warp of a CTA walks the same sequence of pieces.
+// The list is "virtual": every item is preceded by `cost` empty positions, so that cutting the list
+// into equal shares balances units AND item starts (each start costs a warp merge, a publish, maybe a
+// cross-CTA merge).  Position u of an item is real unit u - cost; positions below `cost` hold no work.
 struct Walker {
     const int32_t* lens;
-    int Hkv;
+    int Hkv, cost;
     long long pos, end;   // unit positions in the global list
     long long prefix;     // units (per head) of the sequences before b
     int b, g, u, nu, len;
     __device__ void init(const AttnParams& p, const AttnRange& r) {
-        lens = p.seq_lens; Hkv = p.Hkv; pos = r.x0; end = r.x1;
+        lens = p.seq_lens; Hkv = p.Hkv; cost = p.piece_cost; pos = r.x0; end = r.x1;
         b = r.b; prefix = r.prefix;
-        len = lens[b]; nu = (len + kUnitTokens - 1) / kUnitTokens;
+        len = lens[b]; nu = (len + kUnitTokens - 1) / kUnitTokens + cost;
         const long long rel = pos - prefix * Hkv;
         g = (int)(rel / nu); u = (int)(rel % nu);
     }
@@ -108,7 +112,7 @@ struct Walker {
             u = 0;
             if (++g == Hkv) {
                 g = 0; prefix += nu; ++b;
-                if (pos < end) { len = lens[b]; nu = (len + kUnitTokens - 1) / kUnitTokens; }
+                if (pos < end) { len = lens[b]; nu = (len + kUnitTokens - 1) / kUnitTokens + cost; }
             }
         }
     }
@@ -170,7 +174,12 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
 
     pdl_launch_dependents();
     unsigned long long* tr = (p.trace && cta < 4096) ? p.trace + (size_t)cta * 8 : nullptr;
-    if (tr && threadIdx.x == 0) { tr[0] = global_timer_ns(); tr[3] = 0; tr[5] = 0; }
+    if (tr && threadIdx.x == 0) {
+        tr[0] = global_timer_ns(); tr[3] = 0; tr[5] = 0;
+        unsigned smid;
+        asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+        tr[6] = smid;
+    }
     if (threadIdx.x == 0) {
         for (int s = 0; s < kAttnStages; ++s) {
             mbar_init(&sh->full[s], 1);
@@ -190,7 +199,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     {
         const int b_lo = min(p.batch, (int)threadIdx.x * per_thread), b_hi = min(p.batch, b_lo + per_thread);
         int local = 0;
-        for (int b = b_lo; b < b_hi; ++b) local += (p.seq_lens[b] + kUnitTokens - 1) / kUnitTokens;
+        for (int b = b_lo; b < b_hi; ++b) local += (p.seq_lens[b] + kUnitTokens - 1) / kUnitTokens + p.piece_cost;
         // inclusive warp scan, then warp totals through shared memory
         int incl = local;
 #pragma unroll
@@ -225,7 +234,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         int b = min(p.batch - 1, best * per_thread);
         long long pre = sh->scan[best];
         while (b + 1 < p.batch) {
-            const int nu = (p.seq_lens[b] + kUnitTokens - 1) / kUnitTokens;
+            const int nu = (p.seq_lens[b] + kUnitTokens - 1) / kUnitTokens + p.piece_cost;
             if (x < (pre + nu) * p.Hkv) break;
             pre += nu; ++b;
         }
@@ -239,7 +248,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         const int hf = lane % kHalves;
         const bool op_lane = lane < kOpsPerStage;
         auto page_id = [&](const Walker& w) -> int {
-            const int idx = w.u * kPagesPerStage + pg;
+            const int idx = (w.u - w.cost) * kPagesPerStage + pg;
             return (op_lane && idx * kPage < w.len) ? p.page_table[(size_t)w.b * p.max_pages + idx] : 0;
         };
         int s = 0;
@@ -260,14 +269,20 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                 AttnRange rg;
                 rg.x0 = x0; rg.x1 = x1; rg.rid = rid;
                 locate(x0, rg.b, rg.prefix);
-                if (lane == 0) { sh->rng[r % kRangeRing] = rg; mbar_arrive(&sh->rng_ready[r % kRangeRing]); }
-                ++r;
                 Walker wk;
                 wk.init(p, rg);
-                int pid = page_id(wk);
+                while (!wk.done() && wk.u < wk.cost) wk.advance(1);     // positions without work
+                // a range without any real unit is not handed to the consumers at all (every published
+                // range then holds at least one ring stage, which is what bounds the range ring)
+                if (!wk.done()) {
+                    if (lane == 0) { sh->rng[r % kRangeRing] = rg; mbar_arrive(&sh->rng_ready[r % kRangeRing]); }
+                    ++r;
+                }
+                int pid = wk.done() ? 0 : page_id(wk);
                 while (!wk.done()) {
-                    const int g = wk.g, u = wk.u, len = wk.len;
+                    const int g = wk.g, u = wk.u - wk.cost, len = wk.len;
                     wk.advance(1);
+                    while (!wk.done() && wk.u < wk.cost) wk.advance(1);
                     const int pid_next = wk.done() ? 0 : page_id(wk);   // one unit ahead of the ring
                     bool ok = mbar_wait(&sh->empty[s], ph ^ 1);
                     ok = __all_sync(0xffffffffu, ok);
@@ -330,10 +345,15 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
 
         while (!wk.done() && !aborted) {
             // ---- one piece: units [u0, u0 + n) of item (b, g)
-            const int b = wk.b, g = wk.g, u0 = wk.u, len = wk.len, nu = wk.nu;
-            const long long item_x0 = wk.prefix * p.Hkv + (long long)g * nu;
-            const int n = (int)min((long long)(nu - u0), wk.end - wk.pos);
-            wk.advance(n);
+            const int b = wk.b, g = wk.g, len = wk.len, cost = wk.cost;
+            const int nu = wk.nu - cost;                                     // real units of the item
+            const long long item_v0 = wk.prefix * p.Hkv + (long long)g * wk.nu;   // list position where the item starts
+            const long long item_x0 = item_v0 + cost;                        // ... where its real units start
+            const int nv = (int)min((long long)(wk.nu - wk.u), wk.end - wk.pos);
+            const int u0 = max(wk.u, cost) - cost;                           // real unit range [u0, u0 + n)
+            const int n = max(wk.u + nv, cost) - cost - u0;
+            wk.advance(nv);
+            if (n <= 0) continue;                                            // only empty positions: no piece
             const int slot = first_piece ? 0 : 1;
             first_piece = false;
 
@@ -554,11 +574,11 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                 int rid_i, sl;
                 if (i < n_static) {
                     rid_i = cf + i;
-                    sl = (i == 0 && share_begin(sp.U1, cf, sp.Ge1) < item_x0) ? 1 : 0;
+                    sl = (i == 0 && share_begin(sp.U1, cf, sp.Ge1) < item_v0) ? 1 : 0;
                 } else {
                     const int j = jf + (i - n_static);
                     rid_i = G + j;
-                    sl = (j == jf && sp.U1 + (long long)jf * sp.K2 < dyn_x0) ? 1 : 0;
+                    sl = (j == jf && sp.U1 + (long long)jf * sp.K2 < max(item_v0, sp.U1)) ? 1 : 0;
                 }
                 const size_t base = ((size_t)rid_i * 2 + sl) * 8;
                 float2 ml[8];
@@ -636,6 +656,13 @@ static int attn_dyn_chunks() {
     return v;
 }
 
+// List positions charged per item start when the unit list is cut into equal shares (tuning).
+static int attn_piece_cost() {
+    static int v = -1;
+    if (v < 0) { const char* e = getenv("AFLEX_ATTN_PIECE_COST"); v = e ? atoi(e) : 2; if (v < 0) v = 0; if (v > 16) v = 16; }
+    return v;
+}
+
 // Partial slots: two per range id; range ids = one static share per CTA plus at most
 // dyn_chunks * grid + 1 dynamic chunks.
 static size_t attn_slots(int grid) { return ((size_t)grid * (1 + attn_dyn_chunks()) + 2) * 2; }
@@ -669,6 +696,7 @@ static aflex_status attn_launch_t(aflex_ctx* ctx, const aflex_attn_desc* d, cons
     p.ticket = ctx->counters_attn + kAttnCounterCap;      // two ints past the per-item counters
     p.dyn_pct = attn_dyn_pct();
     p.dyn_chunks = attn_dyn_chunks();
+    p.piece_cost = attn_piece_cost();
     p.status = ctx->dev_status;
     p.out = reinterpret_cast<__nv_bfloat16*>(out);
     p.lse = lse;
@@ -779,6 +807,7 @@ static aflex_status attn_static_launch(StaticDeviceState& stt, const aflex_attn_
     p.ticket = nullptr;     // static shares only: the fixed scratch has two slots per CTA
     p.dyn_pct = 0;
     p.dyn_chunks = 1;
+    p.piece_cost = 0;
     p.trace = nullptr;
 
     const uint64_t rows = (uint64_t)kv->num_pages * d->num_kv_heads * kPage;
