@@ -169,6 +169,54 @@ def measure_energy(step, barrier, gpu_index, tokens_per_step, ms_step):
         return {"unavailable": str(exc)[:200]}
 
 
+def run_ffn_sweep(args, cfg, local_rank, device, peaks):
+    """Dense SwiGLU FFN at the configuration's (H, I) over a range of token counts: where the FFN stops being
+    a weight-streaming kernel and becomes a tensor-core kernel (arithmetic intensity ~ T flop per weight byte)."""
+    from paper_2608_01891_b200 import aflex as AF
+    H, I = cfg.hidden, cfg.inter
+    dense = dataclasses_replace_dense(cfg)
+    wg, wu, wd = IN.make_ffn_weights(dense, device=device)
+    ctx = AF.Context(local_rank, 6 << 30)
+    stream = torch.cuda.current_stream()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    rows = []
+    for T in (32, 64, 128, 256, 512, 1024, 2048, 4096, 8192):
+        x = IN.make_x(dense, device=device, tokens=T)
+        y = torch.empty(T, H, dtype=torch.bfloat16, device=device)
+        for _ in range(max(3, args.warmup)):
+            ctx.ffn_dense(x, wg, wu, wd, y, stream)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n = max(10, args.steps // 2)
+        e0.record(stream)
+        for _ in range(n):
+            ctx.ffn_dense(x, wg, wu, wd, y, stream)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        us = 1e3 * e0.elapsed_time(e1) / n
+        flops = 6.0 * T * H * I
+        wbytes = 3.0 * H * I * 2 + 2.0 * T * H * 2 + 2.0 * T * I * 2
+        rows.append({"T": T, "us": round(us, 1), "tflops": round(flops / us / 1e6, 1),
+                     "frac_bf16_burst": round(flops / us / 1e6 / peaks["bf16_tflops"], 4),
+                     "frac_bf16_sustained": round(flops / us / 1e6 / peaks["bf16_tflops_sustained"], 4),
+                     "weight_stream_gbs": round(wbytes / us / 1e3, 1),
+                     "frac_hbm": round(wbytes / us / 1e3 / peaks["hbm_gbs"], 4)})
+    assert ctx.device_status() == AF.OK
+    line = {"metric": "dense FFN throughput vs tokens (Qwen3-32B FFN shape)" if cfg.cfg_id in (2, 3) else
+            f"dense FFN throughput vs tokens (H={H}, I={I})", "unit": "TFLOP/s", "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"ffn token sweep, H={H}, I={I}", "l2": "weights (>= 786 MB) larger than L2, no flush"},
+            "peaks": peaks, "clocks": sampler.stop(), "sweep": rows}
+    print(json.dumps(line), flush=True)
+    ctx.close()
+
+
+def dataclasses_replace_dense(cfg):
+    """The configuration's FFN shape as a dense FFN (MoE configurations: one expert's shape)."""
+    import dataclasses
+    return dataclasses.replace(cfg, num_experts=0, top_k=0)
+
+
 def build_workload(cfg, device):
     """Everything resident in HBM before the timed region starts."""
     from paper_2608_01891_b200 import aflex as AF
@@ -250,6 +298,9 @@ def main():
     ap.add_argument("--ref-rows", type=int, default=0,
                     help="batch rows per reference/cpu-baseline sample (0 = about 15e9 multiply-adds of oracle work)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--ffn-sweep", action="store_true",
+                    help="instead of the layer step: dense FFN (aflex_ffn_dense) at the configuration's weight shape "
+                         "for T = 32..8192 tokens, TFLOP/s against the measured bf16 peak; prints one JSON line")
     ap.add_argument("--energy", action="store_true",
                     help="also read the NVML energy counter around a >= 2 s loop of the step (default clocks)")
     args = ap.parse_args()
@@ -281,6 +332,10 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device(device))
 
     peaks = load_peaks()
+    if args.ffn_sweep:
+        if rank == 0:
+            run_ffn_sweep(args, cfg, local_rank, device, peaks)
+        return
     wl = build_workload(cfg, device)
     lens_np = wl["kvh"].seq_lens.numpy()
     M = args.depth

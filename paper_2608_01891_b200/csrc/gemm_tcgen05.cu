@@ -212,7 +212,7 @@ struct __align__(8) GemmBarriers {
     int seg[kMaxExperts + 1];
 };
 
-__device__ __forceinline__ float silu_f32(float z) { return z / (1.0f + __expf(-z)); }
+__device__ __forceinline__ float silu_f32(float z) { return __fdividef(z, 1.0f + __expf(-z)); }
 
 template <int MODE>
 __global__ void __launch_bounds__(kGemmThreads, 1)
