@@ -208,7 +208,6 @@ struct __align__(8) GemmBarriers {
     uint64_t tmem_empty[2];
     uint32_t tmem_base;
     volatile int abort;
-    int last_flag;
     int seg[kMaxExperts + 1];
 };
 

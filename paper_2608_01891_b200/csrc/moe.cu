@@ -50,7 +50,7 @@ __global__ void router_logits_kernel(const __nv_bfloat16* __restrict__ x, const 
 __global__ void __launch_bounds__(kRouteThreads)
 moe_route_kernel(const float* __restrict__ logits, int T, int E, int K, int32_t* __restrict__ idx,
                  float* __restrict__ gate, int32_t* __restrict__ counts, int32_t* __restrict__ offsets,
-                 int32_t* __restrict__ pos, int32_t* __restrict__ counts_out) {
+                 int32_t* __restrict__ pos) {
     __shared__ int s_count[kRouteMaxExperts];
     __shared__ int s_offset[kRouteMaxExperts + 1];
     __shared__ int s_running[kRouteMaxExperts];
@@ -101,10 +101,7 @@ moe_route_kernel(const float* __restrict__ logits, int T, int E, int K, int32_t*
     }
     __syncthreads();
     if (tid <= E) offsets[tid] = s_offset[tid];
-    if (tid < E) {
-        counts[tid] = s_count[tid];
-        if (counts_out) counts_out[tid] = s_count[tid];
-    }
+    if (tid < E) counts[tid] = s_count[tid];
 
     const int total = T * K;
     for (int base = 0; base < total; base += kRouteThreads) {
@@ -176,7 +173,7 @@ aflex_status moe_route_launch(aflex_ctx* ctx, const float* logits, int T, int E,
                               cudaStream_t st) {
     KernelScope scope(ctx, kKMoeRoute, st);
     return check_cuda(ctx, launch_pdl(moe_route_kernel, dim3(1), dim3(kRouteThreads), 0, st, logits, T, E, K, mb.idx, mb.gate,
-                                      mb.counts, mb.offsets, mb.pos, (int32_t*)nullptr),
+                                      mb.counts, mb.offsets, mb.pos),
                       "moe_route_kernel launch");
 }
 
