@@ -410,22 +410,38 @@ def main():
         if key in tr:
             roofline["traffic"] = tr[key]
 
-    # ---- end to end: per-step inputs come from pinned host memory, the result goes back
-    hq = wl["q"].cpu().pin_memory()
-    htab = wl["kvh"].page_table.pin_memory()
-    hlens = wl["kvh"].seq_lens.pin_memory()
-    hlog = wl["logits"].cpu().pin_memory() if wl["logits"] is not None else None
+    # ---- end to end: per-step inputs come from pinned host memory, the result goes back.
+    # The per-step inputs (q, page table, sequence lengths, router logits) are packed into one pinned
+    # staging buffer and travel in ONE host-to-device copy into one device buffer the tensors are views of.
+    def carve(total_specs):
+        off, out = 0, []
+        for shape, dtype in total_specs:
+            n = int(np.prod(shape)) * torch.empty((), dtype=dtype).element_size()
+            out.append((off, n, shape, dtype))
+            off = (off + n + 255) & ~255
+        return off, out
+    specs = [(tuple(wl["q"].shape), torch.bfloat16), (tuple(wl["kvh"].page_table.shape), torch.int32),
+             (tuple(wl["kvh"].seq_lens.shape), torch.int32)]
+    if wl["logits"] is not None:
+        specs.append((tuple(wl["logits"].shape), torch.float32))
+    nbytes, layout = carve(specs)
+    host_blob = torch.empty(nbytes, dtype=torch.uint8).pin_memory()
+    dev_blob = torch.empty(nbytes, dtype=torch.uint8, device=device)
+    views_h = [host_blob[o:o + n].view(dt).view(sh) for o, n, sh, dt in layout]
+    views_d = [dev_blob[o:o + n].view(dt).view(sh) for o, n, sh, dt in layout]
+    views_h[0].copy_(wl["q"].cpu()); views_h[1].copy_(wl["kvh"].page_table); views_h[2].copy_(wl["kvh"].seq_lens)
+    if wl["logits"] is not None:
+        views_h[3].copy_(wl["logits"].cpu())
+    dq, dtab, dlens = views_d[0], views_d[1], views_d[2]
+    dlog = views_d[3] if wl["logits"] is not None else None
+    kv_e2e = AF.make_kv(wl["kvh"].k_cache, wl["kvh"].v_cache, dtab, dlens, wl["kvh"].seq_lens)
     hy = torch.empty(cfg.batch, cfg.hidden, dtype=torch.bfloat16).pin_memory()
-    h2d = hq.numel() * 2 + htab.numel() * 4 + hlens.numel() * 4 + (hlog.numel() * 4 if hlog is not None else 0)
+    h2d = sum(n for _, n, _, _ in layout)
     d2h = hy.numel() * 2
 
     def step_e2e():
-        wl["q"].copy_(hq, non_blocking=True)
-        wl["table"].copy_(htab, non_blocking=True)
-        wl["lens"].copy_(hlens, non_blocking=True)
-        if hlog is not None:
-            wl["logits"].copy_(hlog, non_blocking=True)
-        ctx.layer_step(wl["layer"], wl["q"], wl["kv"], wl["y"], M, None, wl["logits"], None, stream)
+        dev_blob.copy_(host_blob, non_blocking=True)
+        ctx.layer_step(wl["layer"], dq, kv_e2e, wl["y"], M, None, dlog, None, stream)
         hy.copy_(wl["y"], non_blocking=True)
         stream.synchronize()          # the caller consumes y before the next decode step
 

@@ -251,6 +251,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             const int idx = (w.u - w.cost) * kPagesPerStage + pg;
             return (op_lane && idx * kPage < w.len) ? p.page_table[(size_t)w.b * p.max_pages + idx] : 0;
         };
+        const uint64_t pol_kv = policy_evict_first();    // KV is read once: do not let it push reusable lines out of L2
         int s = 0;
         uint32_t ph = 0;
         int r = 0;                       // ranges published so far
@@ -299,7 +300,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                         if (id < 0 || id >= p.num_pages) { atomicExch(p.status, AFLEX_ERR_BOUNDS); id = 0; }
                         uint8_t* dst = smem + s * kStageBytes + kv * (kPagesPerStage * kPageBytes) + pg * kPageBytes + hf * (kPage * 128);
                         const int row = (id * p.Hkv + g) * kPage;
-                        tma_load_2d(dst, kv ? &tmap_v : &tmap_k, hf * 64, row, &sh->full[s]);
+                        tma_load_2d_hint(dst, kv ? &tmap_v : &tmap_k, hf * 64, row, &sh->full[s], pol_kv);
                     }
                     pid = pid_next;
                     if (++s == kAttnStages) { s = 0; ph ^= 1; }
