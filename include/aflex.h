@@ -124,7 +124,8 @@ typedef struct {
     int64_t num_pages;            /* pages in each pool; page ids must be in [0, num_pages) */
     const int32_t* page_table;    /* i32 [batch][max_pages_per_seq]; entries past ceil(len/16) are ignored */
     int max_pages_per_seq;        /* row stride of page_table; also bounds every seq_len <= 16*max_pages_per_seq */
-    const int32_t* seq_lens;      /* i32 [batch], each >= 1 */
+    const int32_t* seq_lens;      /* i32 [batch], each in [1, 16*max_pages_per_seq]; a value outside that range is clamped on
+                                     the device and reported as AFLEX_ERR_BOUNDS (a sequence clamped to 0 gets no output) */
     const int32_t* seq_lens_host; /* optional HOST copy of seq_lens (validated: each in [1, 16*max_pages_per_seq]); may be NULL */
 } aflex_kv;
 

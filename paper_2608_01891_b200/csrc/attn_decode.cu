@@ -87,20 +87,27 @@ struct __align__(8) AttnShared {
     int scan[kAttnThreads];  // exclusive prefix (units per KV head) of the sequences before each thread's segment
 };
 
+// A sequence length as the kernel uses it: never beyond what the page-table row can address (a
+// longer value would walk off the row).  Out-of-range lengths are reported by the prologue.
+__device__ __forceinline__ int usable_len(int raw, int max_pages) {
+    const int cap = max_pages * kPage;
+    return raw < 0 ? 0 : (raw > cap ? cap : raw);
+}
+
 // Position in the (sequence, head, unit) list; every warp of a CTA walks the same sequence of pieces.
 // The list is "virtual": every item is preceded by `cost` empty positions, so that cutting the list
 // into equal shares balances units AND item starts (each start costs a warp merge, a publish, maybe a
 // cross-CTA merge).  Position u of an item is real unit u - cost; positions below `cost` hold no work.
 struct Walker {
     const int32_t* lens;
-    int Hkv, cost;
+    int Hkv, cost, max_pages;
     long long pos, end;   // unit positions in the global list
     long long prefix;     // units (per head) of the sequences before b
     int b, g, u, nu, len;
     __device__ void init(const AttnParams& p, const AttnRange& r) {
-        lens = p.seq_lens; Hkv = p.Hkv; cost = p.piece_cost; pos = r.x0; end = r.x1;
+        lens = p.seq_lens; Hkv = p.Hkv; cost = p.piece_cost; max_pages = p.max_pages; pos = r.x0; end = r.x1;
         b = r.b; prefix = r.prefix;
-        len = lens[b]; nu = (len + kUnitTokens - 1) / kUnitTokens + cost;
+        len = usable_len(lens[b], max_pages); nu = (len + kUnitTokens - 1) / kUnitTokens + cost;
         const long long rel = pos - prefix * Hkv;
         g = (int)(rel / nu); u = (int)(rel % nu);
     }
@@ -112,7 +119,7 @@ struct Walker {
             u = 0;
             if (++g == Hkv) {
                 g = 0; prefix += nu; ++b;
-                if (pos < end) { len = lens[b]; nu = (len + kUnitTokens - 1) / kUnitTokens + cost; }
+                if (pos < end) { len = usable_len(lens[b], max_pages); nu = (len + kUnitTokens - 1) / kUnitTokens + cost; }
             }
         }
     }
@@ -199,7 +206,11 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     {
         const int b_lo = min(p.batch, (int)threadIdx.x * per_thread), b_hi = min(p.batch, b_lo + per_thread);
         int local = 0;
-        for (int b = b_lo; b < b_hi; ++b) local += (p.seq_lens[b] + kUnitTokens - 1) / kUnitTokens + p.piece_cost;
+        for (int b = b_lo; b < b_hi; ++b) {
+            const int raw = p.seq_lens[b];
+            if ((raw < 1 || raw > p.max_pages * kPage) && cta == 0) atomicExch(p.status, AFLEX_ERR_BOUNDS);
+            local += (usable_len(raw, p.max_pages) + kUnitTokens - 1) / kUnitTokens + p.piece_cost;
+        }
         // inclusive warp scan, then warp totals through shared memory
         int incl = local;
 #pragma unroll
@@ -234,7 +245,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         int b = min(p.batch - 1, best * per_thread);
         long long pre = sh->scan[best];
         while (b + 1 < p.batch) {
-            const int nu = (p.seq_lens[b] + kUnitTokens - 1) / kUnitTokens + p.piece_cost;
+            const int nu = (usable_len(p.seq_lens[b], p.max_pages) + kUnitTokens - 1) / kUnitTokens + p.piece_cost;
             if (x < (pre + nu) * p.Hkv) break;
             pre += nu; ++b;
         }

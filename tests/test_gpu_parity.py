@@ -380,3 +380,17 @@ def test_dense_ffn_large_token_count_uses_whole_tile_path(ctx):
     want = O.ffn_dense(u16(x[rows]), u16(wg), u16(wu), u16(wd))
     assert row_rel_err(f64(y[rows]), want) <= TOL_FFN
     assert torch.isfinite(y.float()).all()
+
+
+def test_sequence_length_beyond_the_page_table_row_is_clamped_and_reported(ctx):
+    """A device-side length larger than 16 * max_pages_per_seq must not walk off the page-table row."""
+    lens = [40, 70]
+    q, kv = make_case(2, 8, 2, 64, lens, seed=12)
+    bad = kv.seq_lens.clone()
+    bad[1] = 16 * kv.page_table.shape[1] + 500
+    run_attention(ctx, q, kv.k_cache, kv.v_cache, kv.page_table, bad, 8, 2, 64, with_host_lens=False)
+    assert ctx.device_status() == AF.ERR_BOUNDS
+    got, _ = run_attention(ctx, q, kv.k_cache, kv.v_cache, kv.page_table, kv.seq_lens, 8, 2, 64)
+    want, _ = O.attn_decode(u16(q), u16(kv.k_cache), u16(kv.v_cache), kv.page_table.numpy(), kv.seq_lens.numpy())
+    assert row_rel_err(got, want) <= TOL_ATTN
+    assert ctx.device_status() == AF.OK
