@@ -317,3 +317,192 @@ ORACLE_API double oracle_eq2_layer_time(double t_a, double t_f, double t_comm, i
     if (M <= 1) return t_a + t_f + t_comm;
     return (t_a > t_f ? t_a : t_f) + t_comm / (double)M;
 }
+
+/* ========================================================================= */
+/* The rest of the decoder layer around the A/F hot path (the Attention       */
+/* group's own operators and the residual stream), so that whole layers can   */
+/* be chained as in the interleaved pipeline of Section 4.3 (A of layer l+1   */
+/* starts from what F of layer l returns).  The paper leaves these operators   */
+/* to the two model families it serves (Section 6.1); what follows is their    */
+/* public definition: pre-norm residual blocks, RMS normalisation, rotary      */
+/* position embedding in the rotate-half convention, optional per-head         */
+/* normalisation of queries and keys, K/V of the decoded token appended to     */
+/* the paged cache in the cache's storage type (bf16).                         */
+/* ========================================================================= */
+
+/* double -> bf16 bit pattern, round to nearest even, one rounding. */
+static uint16_t f64_to_bf16(double d) {
+    if (d != d) return 0x7fc0;
+    const uint16_t sign = signbit(d) ? 0x8000 : 0;
+    const double a = fabs(d);
+    if (a == 0.0) return sign;
+    if (isinf(a)) return (uint16_t)(sign | 0x7f80);
+    int e;
+    (void)frexp(a, &e);                 /* a = m * 2^e, m in [0.5, 1) */
+    int qe = e - 8;                     /* quantum 2^qe leaves 8 significant bits */
+    if (e - 1 < -126) qe = -126 - 7;    /* subnormal range: fixed quantum */
+    const double r = ldexp(nearbyint(ldexp(a, -qe)), qe);   /* default rounding mode: to nearest even */
+    const float f = (float)r;           /* exact: r has at most 8 significant bits */
+    if (isinf(f) || r > 3.3895313892515355e38) return (uint16_t)(sign | 0x7f80);
+    uint32_t u;
+    memcpy(&u, &f, sizeof u);
+    return (uint16_t)(sign | (u >> 16));
+}
+
+ORACLE_API uint16_t oracle_f64_to_bf16(double d) { return f64_to_bf16(d); }
+
+/* ------------------------------------------------------------------------- */
+/* RMS normalisation over the last axis:                                      */
+/*   y[t][i] = x[t][i] / sqrt( (1/H) sum_j x[t][j]^2 + eps ) * w[i].           */
+/*   x f64 [T][H]; w bf16 [H] (NULL = all ones); y f64 [T][H].                 */
+/* ------------------------------------------------------------------------- */
+ORACLE_API void oracle_rmsnorm(const double* x, const uint16_t* w, int T, int H, double eps, double* y) {
+    for (int t = 0; t < T; ++t) {
+        double ss = 0.0;
+        for (int j = 0; j < H; ++j) ss += x[(size_t)t * H + j] * x[(size_t)t * H + j];
+        const double r = 1.0 / sqrt(ss / (double)H + eps);
+        for (int i = 0; i < H; ++i)
+            y[(size_t)t * H + i] = x[(size_t)t * H + i] * r * (w ? bf16_to_f64(w[i]) : 1.0);
+    }
+}
+
+/* ------------------------------------------------------------------------- */
+/* Rotary position embedding, rotate-half convention, on one head vector:     */
+/*   for i < D/2:  angle_i = pos * theta^(-2i/D)                               */
+/*     out[i]       = v[i] cos(angle_i) - v[i + D/2] sin(angle_i)              */
+/*     out[i + D/2] = v[i + D/2] cos(angle_i) + v[i] sin(angle_i)              */
+/* ------------------------------------------------------------------------- */
+ORACLE_API void oracle_rope(const double* v, int D, double pos, double theta, double* out) {
+    const int half = D / 2;
+    for (int i = 0; i < half; ++i) {
+        const double ang = pos * pow(theta, -2.0 * (double)i / (double)D);
+        const double c = cos(ang), s = sin(ang);
+        const double a = v[i], b = v[i + half];
+        out[i] = a * c - b * s;
+        out[i + half] = b * c + a * s;
+    }
+}
+
+/* Paged GQA decode attention with the queries given in double ([B][Hq][D]). */
+ORACLE_API void oracle_attn_decode_f64q(const double* q, const uint16_t* k_cache, const uint16_t* v_cache,
+                                        const int32_t* page_table, int max_pages, const int32_t* seq_lens,
+                                        int B, int Hq, int Hkv, int D, int P, double scale,
+                                        double* out, double* lse) {
+    const int G = Hq / Hkv;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int b = 0; b < B; ++b) {
+        for (int h = 0; h < Hq; ++h) {
+            const int n = seq_lens[b];
+            const int g = h / G;
+            double* keys = (double*)malloc(sizeof(double) * (size_t)n * D);
+            double* vals = (double*)malloc(sizeof(double) * (size_t)n * D);
+            for (int j = 0; j < n; ++j) {
+                const int64_t page = page_table[(size_t)b * max_pages + j / P];
+                const size_t base = (((size_t)page * Hkv + g) * P + (size_t)(j % P)) * (size_t)D;
+                for (int d = 0; d < D; ++d) {
+                    keys[(size_t)j * D + d] = bf16_to_f64(k_cache[base + d]);
+                    vals[(size_t)j * D + d] = bf16_to_f64(v_cache[base + d]);
+                }
+            }
+            oracle_attn_one_query_f64(q + ((size_t)b * Hq + h) * D, keys, vals, n, D, scale,
+                                      out + ((size_t)b * Hq + h) * D, lse ? lse + (size_t)b * Hq + h : NULL);
+            free(keys); free(vals);
+        }
+    }
+}
+
+/* ------------------------------------------------------------------------- */
+/* The Attention group's work before the attention operator, for the token    */
+/* being decoded (position seq_lens[b] - 1 of sequence b):                     */
+/*   xn  = rmsnorm(x, w_ln)                                                    */
+/*   qkv = xn W_qkv^T, rows of W_qkv ordered [Hq query heads | Hkv key heads   */
+/*         | Hkv value heads], D rows per head                                 */
+/*   q_h = rope(norm_q(qkv_h), pos),  k_g = rope(norm_k(qkv_{Hq+g}), pos)      */
+/*         (norm_* = RMS normalisation over the D entries of the head with      */
+/*          weights w_qn / w_kn; skipped when the pointer is NULL)             */
+/*   cache[page_table[b][pos / P]][g][pos % P] = bf16(k_g), bf16(v_g)          */
+/* q_out f64 [B][Hq][D].  The caches are updated in place.                     */
+/* ------------------------------------------------------------------------- */
+ORACLE_API void oracle_qkv_rope_append(const double* x, const uint16_t* w_ln, const uint16_t* w_qkv,
+                                       const uint16_t* w_qn, const uint16_t* w_kn, double eps, double theta,
+                                       uint16_t* k_cache, uint16_t* v_cache,
+                                       const int32_t* page_table, int max_pages, const int32_t* seq_lens,
+                                       int B, int H, int Hq, int Hkv, int D, int P, double* q_out) {
+    const int N = (Hq + 2 * Hkv) * D;
+    double* xn = (double*)malloc(sizeof(double) * (size_t)B * H);
+    double* qkv = (double*)malloc(sizeof(double) * (size_t)B * N);
+    double* tmp = (double*)malloc(sizeof(double) * (size_t)D);
+    double* rot = (double*)malloc(sizeof(double) * (size_t)D);
+    oracle_rmsnorm(x, w_ln, B, H, eps, xn);
+    oracle_linear(xn, w_qkv, B, H, N, qkv);
+    for (int b = 0; b < B; ++b) {
+        const int pos = seq_lens[b] - 1;
+        const int64_t page = page_table[(size_t)b * max_pages + pos / P];
+        for (int h = 0; h < Hq; ++h) {
+            const double* v = qkv + (size_t)b * N + (size_t)h * D;
+            if (w_qn) { oracle_rmsnorm(v, w_qn, 1, D, eps, tmp); v = tmp; }
+            oracle_rope(v, D, (double)pos, theta, q_out + ((size_t)b * Hq + h) * D);
+        }
+        for (int g = 0; g < Hkv; ++g) {
+            const size_t base = (((size_t)page * Hkv + g) * P + (size_t)(pos % P)) * (size_t)D;
+            const double* kk = qkv + (size_t)b * N + (size_t)(Hq + g) * D;
+            const double* vv = qkv + (size_t)b * N + (size_t)(Hq + Hkv + g) * D;
+            if (w_kn) { oracle_rmsnorm(kk, w_kn, 1, D, eps, tmp); kk = tmp; }
+            oracle_rope(kk, D, (double)pos, theta, rot);
+            for (int d = 0; d < D; ++d) {
+                k_cache[base + d] = f64_to_bf16(rot[d]);
+                v_cache[base + d] = f64_to_bf16(vv[d]);
+            }
+        }
+    }
+    free(xn); free(qkv); free(tmp); free(rot);
+}
+
+/* ------------------------------------------------------------------------- */
+/* One whole pre-norm decoder layer, decode step, in double:                  */
+/*   A group:  q, cache append  (oracle_qkv_rope_append on x with w_ln_attn)   */
+/*             a  = attention(q, cache)                                        */
+/*             h1 = x + a W_o^T                  (what A sends to F)           */
+/*   F group:  out = h1 + FFN(rmsnorm(h1, w_ln_ffn))  (what F returns)          */
+/* FFN = dense SwiGLU (E == 0) or top-K mixture of experts with router         */
+/* logits = rmsnorm(h1) W_r^T (or the given logits when w_router is NULL).     */
+/* No intermediate is rounded except the cache entries (bf16 storage).         */
+/* ------------------------------------------------------------------------- */
+ORACLE_API void oracle_decoder_layer(const double* x, const uint16_t* w_ln_attn, const uint16_t* w_qkv,
+                                     const uint16_t* w_qn, const uint16_t* w_kn, double eps, double theta,
+                                     uint16_t* k_cache, uint16_t* v_cache,
+                                     const int32_t* page_table, int max_pages, const int32_t* seq_lens,
+                                     int B, int H, int Hq, int Hkv, int D, int P, double scale,
+                                     const uint16_t* w_o, const uint16_t* w_ln_ffn, int I, int E, int K,
+                                     const uint16_t* w_gate, const uint16_t* w_up, const uint16_t* w_down,
+                                     const uint16_t* w_router, const float* logits,
+                                     double* q_out, double* h1_out, double* out) {
+    const int A = Hq * D;
+    double* q = q_out ? q_out : (double*)malloc(sizeof(double) * (size_t)B * A);
+    double* a = (double*)malloc(sizeof(double) * (size_t)B * A);
+    double* h1 = h1_out ? h1_out : (double*)malloc(sizeof(double) * (size_t)B * H);
+    double* xn = (double*)malloc(sizeof(double) * (size_t)B * H);
+    double* f = (double*)malloc(sizeof(double) * (size_t)B * H);
+    oracle_qkv_rope_append(x, w_ln_attn, w_qkv, w_qn, w_kn, eps, theta, k_cache, v_cache, page_table, max_pages,
+                           seq_lens, B, H, Hq, Hkv, D, P, q);
+    oracle_attn_decode_f64q(q, k_cache, v_cache, page_table, max_pages, seq_lens, B, Hq, Hkv, D, P, scale, a, NULL);
+    oracle_linear(a, w_o, B, A, H, h1);
+    for (size_t i = 0; i < (size_t)B * H; ++i) h1[i] += x[i];
+    oracle_rmsnorm(h1, w_ln_ffn, B, H, eps, xn);
+    if (E == 0) {
+        oracle_ffn_dense_f64x(xn, w_gate, w_up, w_down, B, H, I, f);
+    } else if (w_router) {
+        double* ld = (double*)malloc(sizeof(double) * (size_t)B * E);
+        float* lf = (float*)malloc(sizeof(float) * (size_t)B * E);
+        oracle_router_logits(xn, w_router, B, H, E, ld);
+        for (size_t i = 0; i < (size_t)B * E; ++i) lf[i] = (float)ld[i];   /* routing takes fp32 logits */
+        oracle_ffn_moe_f64x(xn, lf, w_gate, w_up, w_down, B, H, I, E, K, f, NULL, NULL);
+        free(ld); free(lf);
+    } else {
+        oracle_ffn_moe_f64x(xn, logits, w_gate, w_up, w_down, B, H, I, E, K, f, NULL, NULL);
+    }
+    for (size_t i = 0; i < (size_t)B * H; ++i) out[i] = h1[i] + f[i];
+    if (!q_out) free(q);
+    if (!h1_out) free(h1);
+    free(a); free(xn); free(f);
+}

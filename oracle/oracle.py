@@ -230,3 +230,128 @@ def layer_step(q, k_cache, v_cache, page_table, seq_lens, w_o, w_gate, w_up, w_d
                               _p(w_gate, _u16p), _p(w_up, _u16p), _p(w_down, _u16p),
                               _p(logits, _f32p) if E else None, _p(a, _f64p), _p(y, _f64p))
     return a, y
+
+
+# --------------------------------------------------------------------------- whole decoder layer
+def f64_to_bf16(values) -> np.ndarray:
+    """f64 array -> bf16 bit patterns (u16), round to nearest even in one rounding."""
+    values = np.ascontiguousarray(values, dtype=np.float64)
+    lib = _load()
+    lib.oracle_f64_to_bf16.restype = ctypes.c_uint16
+    lib.oracle_f64_to_bf16.argtypes = [ctypes.c_double]
+    out = np.zeros(values.shape, dtype=np.uint16)
+    flat_in, flat_out = values.reshape(-1), out.reshape(-1)
+    for i in range(flat_in.size):
+        flat_out[i] = lib.oracle_f64_to_bf16(float(flat_in[i]))
+    return out
+
+
+def rmsnorm(x, w, eps: float) -> np.ndarray:
+    """x f64 [T,H]; w u16 [H] or None (ones) -> f64 [T,H]."""
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    T, H = x.shape
+    if w is not None:
+        w = _u16(w)
+        assert w.shape == (H,)
+    y = np.zeros((T, H), dtype=np.float64)
+    _load().oracle_rmsnorm(_p(x, _f64p), _p(w, _u16p), T, H, ctypes.c_double(eps), _p(y, _f64p))
+    return y
+
+
+def rope(v, pos: float, theta: float) -> np.ndarray:
+    """One head vector f64 [D] rotated to position pos (rotate-half convention)."""
+    v = np.ascontiguousarray(v, dtype=np.float64)
+    (D,) = v.shape
+    assert D % 2 == 0
+    out = np.zeros(D, dtype=np.float64)
+    _load().oracle_rope(_p(v, _f64p), D, ctypes.c_double(pos), ctypes.c_double(theta), _p(out, _f64p))
+    return out
+
+
+def attn_decode_f64q(q, k_cache, v_cache, page_table, seq_lens, scale: Optional[float] = None):
+    """As attn_decode with the queries in f64 [B,Hq,D]."""
+    q = np.ascontiguousarray(q, dtype=np.float64)
+    k_cache, v_cache = _u16(k_cache), _u16(v_cache)
+    page_table = np.ascontiguousarray(page_table, dtype=np.int32)
+    seq_lens = np.ascontiguousarray(seq_lens, dtype=np.int32)
+    B, Hq, D = q.shape
+    _, Hkv, P, _ = k_cache.shape
+    if scale is None:
+        scale = 1.0 / np.sqrt(float(D))
+    out = np.zeros((B, Hq, D), dtype=np.float64)
+    lse = np.zeros((B, Hq), dtype=np.float64)
+    _load().oracle_attn_decode_f64q(_p(q, _f64p), _p(k_cache, _u16p), _p(v_cache, _u16p),
+                                    _p(page_table, _i32p), int(page_table.shape[1]), _p(seq_lens, _i32p),
+                                    B, Hq, Hkv, D, P, ctypes.c_double(scale), _p(out, _f64p), _p(lse, _f64p))
+    return out, lse
+
+
+def qkv_rope_append(x, w_ln, w_qkv, w_qn, w_kn, eps: float, theta: float, k_cache, v_cache, page_table,
+                    seq_lens, num_q_heads: int) -> np.ndarray:
+    """Attention-group operators in front of the attention itself.  x f64 [B,H]; w_ln u16 [H];
+    w_qkv u16 [(Hq+2Hkv)*D, H]; w_qn, w_kn u16 [D] or None.  Updates k_cache / v_cache (u16
+    [num_pages,Hkv,P,D]) IN PLACE at position seq_lens[b]-1 and returns q f64 [B,Hq,D]."""
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    B, H = x.shape
+    assert k_cache.dtype == np.uint16 and k_cache.flags["C_CONTIGUOUS"] and k_cache.flags["WRITEABLE"]
+    assert v_cache.dtype == np.uint16 and v_cache.flags["C_CONTIGUOUS"] and v_cache.flags["WRITEABLE"]
+    _, Hkv, P, D = k_cache.shape
+    Hq = int(num_q_heads)
+    w_ln, w_qkv = _u16(w_ln), _u16(w_qkv)
+    assert w_qkv.shape == ((Hq + 2 * Hkv) * D, H) and w_ln.shape == (H,)
+    w_qn = None if w_qn is None else _u16(w_qn)
+    w_kn = None if w_kn is None else _u16(w_kn)
+    page_table = np.ascontiguousarray(page_table, dtype=np.int32)
+    seq_lens = np.ascontiguousarray(seq_lens, dtype=np.int32)
+    q = np.zeros((B, Hq, D), dtype=np.float64)
+    _load().oracle_qkv_rope_append(_p(x, _f64p), _p(w_ln, _u16p), _p(w_qkv, _u16p), _p(w_qn, _u16p),
+                                   _p(w_kn, _u16p), ctypes.c_double(eps), ctypes.c_double(theta),
+                                   _p(k_cache, _u16p), _p(v_cache, _u16p), _p(page_table, _i32p),
+                                   int(page_table.shape[1]), _p(seq_lens, _i32p), B, H, Hq, Hkv, D, P,
+                                   _p(q, _f64p))
+    return q
+
+
+def decoder_layer(x, w, k_cache, v_cache, page_table, seq_lens, num_q_heads: int, eps: float, theta: float,
+                  top_k: int = 0, logits=None, scale: Optional[float] = None):
+    """One whole pre-norm decoder layer (decode step) in fp64.
+
+    x f64 [B,H] (the residual stream); ``w`` is a dict of u16 arrays: ln_attn [H], qkv
+    [(Hq+2Hkv)*D,H], q_norm / k_norm [D] or None, o [H,Hq*D], ln_ffn [H], gate / up ([I,H] dense,
+    [E,I,H] MoE), down ([H,I] / [E,H,I]), router [E,H] or None (then ``logits`` f32 [B,E] is used).
+    The caches are updated IN PLACE.  Returns (q f64 [B,Hq,D], h1 f64 [B,H], out f64 [B,H])."""
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    B, H = x.shape
+    assert k_cache.dtype == np.uint16 and k_cache.flags["C_CONTIGUOUS"] and k_cache.flags["WRITEABLE"]
+    assert v_cache.dtype == np.uint16 and v_cache.flags["C_CONTIGUOUS"] and v_cache.flags["WRITEABLE"]
+    _, Hkv, P, D = k_cache.shape
+    Hq = int(num_q_heads)
+    page_table = np.ascontiguousarray(page_table, dtype=np.int32)
+    seq_lens = np.ascontiguousarray(seq_lens, dtype=np.int32)
+    g = {k: (None if v is None else _u16(v)) for k, v in w.items()}
+    assert g["qkv"].shape == ((Hq + 2 * Hkv) * D, H) and g["o"].shape == (H, Hq * D)
+    if g["gate"].ndim == 3:
+        E, I, _ = g["gate"].shape
+        assert top_k >= 1
+        if g.get("router") is None:
+            logits = np.ascontiguousarray(logits, dtype=np.float32)
+            assert logits.shape == (B, E)
+    else:
+        E = 0
+        I = g["gate"].shape[0]
+    if scale is None:
+        scale = 1.0 / np.sqrt(float(D))
+    q = np.zeros((B, Hq, D), dtype=np.float64)
+    h1 = np.zeros((B, H), dtype=np.float64)
+    out = np.zeros((B, H), dtype=np.float64)
+    _load().oracle_decoder_layer(_p(x, _f64p), _p(g["ln_attn"], _u16p), _p(g["qkv"], _u16p),
+                                 _p(g.get("q_norm"), _u16p), _p(g.get("k_norm"), _u16p),
+                                 ctypes.c_double(eps), ctypes.c_double(theta),
+                                 _p(k_cache, _u16p), _p(v_cache, _u16p), _p(page_table, _i32p),
+                                 int(page_table.shape[1]), _p(seq_lens, _i32p), B, H, Hq, Hkv, D, P,
+                                 ctypes.c_double(scale), _p(g["o"], _u16p), _p(g["ln_ffn"], _u16p),
+                                 I, E, int(top_k), _p(g["gate"], _u16p), _p(g["up"], _u16p), _p(g["down"], _u16p),
+                                 _p(g.get("router"), _u16p) if E else None,
+                                 _p(logits, _f32p) if (E and g.get("router") is None) else None,
+                                 _p(q, _f64p), _p(h1, _f64p), _p(out, _f64p))
+    return q, h1, out

@@ -49,6 +49,10 @@ class LayerConfig:
     len_sigma: float = 0.7        # lognormal only
     microbatch_depths: Tuple[int, ...] = (1,)
     zipf_s: float = 0.0           # > 0 => skewed expert load
+    # the rest of the decoder layer (whole-layer entry points)
+    rms_eps: float = 1e-6
+    rope_theta: float = 1.0e6
+    qk_norm: bool = True          # per-head RMS normalisation of queries and keys
 
     @property
     def group(self) -> int:
@@ -61,7 +65,7 @@ class LayerConfig:
 
 CONFIGS = {
     1: LayerConfig(1, "tiny-dense", 4, 8, 2, 64, 512, 1376,
-                   len_dist="uniform", len_lo=16, len_hi=128),
+                   len_dist="uniform", len_lo=16, len_hi=128, rope_theta=1.0e4),
     2: LayerConfig(2, "qwen3-32b-shape", 32, 64, 8, 128, 5120, 25600,
                    len_dist="uniform", len_lo=512, len_hi=4096),
     3: LayerConfig(3, "qwen3-32b-shape-interleaved", 128, 64, 8, 128, 5120, 25600,
@@ -69,11 +73,11 @@ CONFIGS = {
                    microbatch_depths=(1, 2, 4)),
     4: LayerConfig(4, "mixtral-8x7b-shape", 64, 32, 8, 128, 4096, 14336,
                    num_experts=8, top_k=2,
-                   len_dist="uniform", len_lo=1024, len_hi=8192),
+                   len_dist="uniform", len_lo=1024, len_hi=8192, rms_eps=1e-5, qk_norm=False),
     5: LayerConfig(5, "mixtral-8x7b-shape-loaded", 256, 32, 8, 128, 4096, 14336,
                    num_experts=8, top_k=2,
                    len_dist="lognormal", len_lo=512, len_hi=16384, len_median=4096,
-                   microbatch_depths=(1, 2, 3, 4), zipf_s=1.2),
+                   microbatch_depths=(1, 2, 3, 4), zipf_s=1.2, rms_eps=1e-5, qk_norm=False),
 }
 
 # Tensor indices k inside a configuration (seed = 1000*cfg + k).
@@ -223,6 +227,58 @@ def make_ffn_weights(cfg: LayerConfig, device: str = "cpu"):
 
 def make_router_weight(cfg: LayerConfig, device: str = "cpu") -> torch.Tensor:
     return _randn_bf16((cfg.num_experts, cfg.hidden), 0.02, _seed(cfg, _K_WR), device)
+
+
+@dataclasses.dataclass
+class DecoderWeights:
+    """Weights of one whole decoder layer (bf16).  Index 100*layer + k seeds tensor k of a layer."""
+    ln_attn: torch.Tensor                 # [H]            ~ 1 + N(0, 0.1)
+    qkv: torch.Tensor                     # [(Hq+2Hkv)*D, H] rows: query heads, key heads, value heads
+    q_norm: Optional[torch.Tensor]        # [D] or None    ~ 1 + N(0, 0.1)
+    k_norm: Optional[torch.Tensor]        # [D] or None
+    o: torch.Tensor                       # [H, Hq*D]
+    ln_ffn: torch.Tensor                  # [H]
+    gate: torch.Tensor
+    up: torch.Tensor
+    down: torch.Tensor
+    router: Optional[torch.Tensor]        # [E, H] (MoE only)
+
+
+def _gain_bf16(n: int, seed: int, device: str) -> torch.Tensor:
+    g = _gen(seed, device)
+    t = torch.randn(n, generator=g, device=device, dtype=torch.float32).mul_(0.1).add_(1.0)
+    return t.to(torch.bfloat16)
+
+
+def make_decoder_weights(cfg: LayerConfig, layer: int = 0, device: str = "cpu") -> DecoderWeights:
+    """All weights of decoder layer `layer`: projections ~N(0,0.02), normalisation gains ~1+N(0,0.1).
+    Layer 0 reuses the FFN and W_o draws of the hot-path benchmarks; further layers get their own."""
+    H, I, E, D = cfg.hidden, cfg.inter, cfg.num_experts, cfg.head_dim
+    base = 1000 * cfg.cfg_id + 100 * (layer + 1)
+    n_qkv = (cfg.num_q_heads + 2 * cfg.num_kv_heads) * D
+    lead = (E,) if E > 0 else ()
+    if layer == 0:
+        gate, up, down = make_ffn_weights(cfg, device)
+        o = make_wo(cfg, device)
+        router = make_router_weight(cfg, device) if E > 0 else None
+    else:
+        gate = _randn_bf16(lead + (I, H), 0.02, base + 0, device)
+        up = _randn_bf16(lead + (I, H), 0.02, base + 1, device)
+        down = _randn_bf16(lead + (H, I), 0.02, base + 2, device)
+        o = _randn_bf16((H, cfg.num_q_heads * D), 0.02, base + 3, device)
+        router = _randn_bf16((E, H), 0.02, base + 4, device) if E > 0 else None
+    qkv = _randn_bf16((n_qkv, H), 0.02, base + 5, device)
+    ln_attn = _gain_bf16(H, base + 6, device)
+    ln_ffn = _gain_bf16(H, base + 7, device)
+    q_norm = _gain_bf16(D, base + 8, device) if cfg.qk_norm else None
+    k_norm = _gain_bf16(D, base + 9, device) if cfg.qk_norm else None
+    return DecoderWeights(ln_attn, qkv, q_norm, k_norm, o, ln_ffn, gate, up, down, router)
+
+
+def make_hidden(cfg: LayerConfig, device: str = "cpu", batch: Optional[int] = None) -> torch.Tensor:
+    """Residual-stream input [B, H] ~N(0,1) of the first decoder layer."""
+    B = cfg.batch if batch is None else batch
+    return _randn_bf16((B, cfg.hidden), 1.0, 1000 * cfg.cfg_id + 50, device)
 
 
 def make_router_logits(cfg: LayerConfig, tokens: Optional[int] = None) -> torch.Tensor:
