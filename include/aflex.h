@@ -269,6 +269,74 @@ AFLEX_API aflex_status aflex_linear(aflex_ctx* ctx, const void* x, const void* w
  * SM).  It changes how the KV cache is split across CTAs, never the result beyond rounding. */
 AFLEX_API aflex_status aflex_set_attn_ctas(aflex_ctx* ctx, int ctas);
 
+/* ---- Whole decoder layers, chained (Section 4.3, "Interleaved A/F Pipeline") -------------
+ *
+ * The interleaved pipeline launches A of layer l+1 for microbatch i as soon as F of layer l has
+ * returned that microbatch's hidden states, without waiting for the layer's other microbatches.
+ * To chain layers the Attention group needs its remaining operators (the paper leaves them to
+ * the two model families it serves, Section 6.1; these are their public definitions):
+ *
+ *   A_{l,i}:  r   = hidden state entering the layer (the residual stream), bf16 [rows][H]
+ *             xn  = rmsnorm(r, w_ln_attn)            rmsnorm(v, g)_j = v_j / sqrt(mean(v^2) + eps) * g_j
+ *             qkv = xn W_qkv^T                       rows of W_qkv: Hq query heads, Hkv key heads,
+ *                                                    Hkv value heads, D rows per head
+ *             q_h = rope(norm_q(qkv_h), pos), k_g = rope(norm_k(qkv_{Hq+g}), pos), pos = seq_len - 1
+ *                   norm_* = rmsnorm over the head's D entries with gains w_q_norm / w_k_norm
+ *                   (skipped when NULL); rope: for i < D/2, angle = pos * theta^(-2i/D),
+ *                   (v_i, v_{i+D/2}) <- (v_i cos - v_{i+D/2} sin, v_{i+D/2} cos + v_i sin)
+ *             K/V cache slot (page_table[b][pos/16], g, pos%16) <- bf16(k_g), bf16(v_g)
+ *             a   = attention(q, cache)              as aflex_attn_decode; the new token takes part
+ *             h1  = r + a W_o^T                      what A sends to F
+ *   F_{l,i}:  out = h1 + FFN(rmsnorm(h1, w_ln_ffn))  what F returns; dense SwiGLU or top-k MoE
+ *                                                    (router logits = rmsnorm(h1) W_router^T)
+ *
+ * Intermediate tensors are bf16 (each store rounds to nearest even); sums, norms and the rotary
+ * angles are formed in fp32 / fp64.  seq_lens[b] counts the token being decoded: its K/V slot is
+ * WRITTEN by this call (the k_cache / v_cache pointers of aflex_kv are written through), every
+ * earlier slot is read.  Two sequences must not share the page of their last token.
+ */
+typedef struct {
+    aflex_layer_desc layer;   /* attention shape, hidden, inter, experts, W_o, FFN weights, router;
+                                 w_o is required; MoE layers require w_router */
+    const void* w_qkv;        /* bf16 [(Hq + 2 Hkv) * D][H] */
+    const void* w_ln_attn;    /* bf16 [H] */
+    const void* w_ln_ffn;     /* bf16 [H] */
+    const void* w_q_norm;     /* bf16 [D], or NULL: queries are not normalised */
+    const void* w_k_norm;     /* bf16 [D], or NULL */
+    float rms_eps;
+    float rope_theta;
+} aflex_decoder_desc;
+
+/*
+ * Runs num_layers >= 1 decoder layers on hidden states x_in bf16 [B][H] -> x_out bf16 [B][H]
+ * (x_out may alias x_in).  layers: HOST array [num_layers]; kvs: HOST array [num_layers], one
+ * cache per layer (page_table and seq_lens may be shared between them).  Microbatching as in
+ * aflex_layer_step (depth M, host offsets or NULL); with M >= 2, A_{l+1,i} waits only for
+ * F_{l,i}.  The result does not depend on M or on the split.  All layers must have the same
+ * hidden size.  Device-side length or page-id violations raise AFLEX_ERR_BOUNDS in the status
+ * word and skip the offending write.
+ */
+AFLEX_API aflex_status aflex_decoder_layers(aflex_ctx* ctx, const aflex_decoder_desc* layers, const aflex_kv* kvs,
+                                            int num_layers, const void* x_in, int batch, int microbatch_depth,
+                                            const int32_t* mb_offsets, void* x_out, void* stream);
+
+/* Workspace bytes that suffice for aflex_decoder_layers on this layer shape.  Pure host computation. */
+AFLEX_API size_t aflex_decoder_workspace_bytes(const aflex_decoder_desc* layer, int max_batch);
+
+/*
+ * The two small operators of the chain on their own (testing, benchmarking).
+ * aflex_add_rmsnorm: s = res (+ add when add != NULL), bf16 [T][H] each, summed in fp32;
+ *   res_out (optional, may alias res or add) = bf16(s); y (optional) = bf16(rmsnorm(s, w)).
+ *   H multiple of 8; w bf16 [H], required when y != NULL.
+ * aflex_rope_append: the q / k / v step of A_{l,i} above on qkv bf16 [B][(Hq+2Hkv)*D]:
+ *   writes q_out bf16 [B][Hq][D] and the decoded token's K/V cache slots.
+ */
+AFLEX_API aflex_status aflex_add_rmsnorm(aflex_ctx* ctx, const void* res, const void* add, const void* w, int T, int H,
+                                         float eps, void* res_out, void* y, void* stream);
+AFLEX_API aflex_status aflex_rope_append(aflex_ctx* ctx, const aflex_attn_desc* desc, const void* qkv,
+                                         const aflex_kv* kv, int batch, const void* w_q_norm, const void* w_k_norm,
+                                         float rms_eps, float rope_theta, void* q_out, void* stream);
+
 /* ---- Measurement support (no counterpart in the paper's method; the per-operator latency
  * profiling of its Section 4.1 is the motivation) --------------------------------------------
  *

@@ -24,7 +24,8 @@ EXPORTS = (
     "aflex_get_device_status", "aflex_attn_decode", "aflex_ffn_dense", "aflex_ffn_moe", "aflex_layer_step",
     "aflex_workspace_bytes", "aflex_linear", "aflex_set_attn_ctas", "aflex_num_kernel_kinds",
     "aflex_kernel_name", "aflex_launch_count", "aflex_profile_enable", "aflex_profile_read",
-    "aflex_trace_read", "aflex_attn_decode_static",
+    "aflex_trace_read", "aflex_attn_decode_static", "aflex_decoder_layers", "aflex_decoder_workspace_bytes",
+    "aflex_add_rmsnorm", "aflex_rope_append",
 )
 
 
@@ -44,6 +45,12 @@ class LayerDesc(ctypes.Structure):
                 ("num_experts", ctypes.c_int), ("top_k", ctypes.c_int), ("w_o", ctypes.c_void_p),
                 ("w_gate", ctypes.c_void_p), ("w_up", ctypes.c_void_p), ("w_down", ctypes.c_void_p),
                 ("w_router", ctypes.c_void_p)]
+
+
+class DecoderDesc(ctypes.Structure):
+    _fields_ = [("layer", LayerDesc), ("w_qkv", ctypes.c_void_p), ("w_ln_attn", ctypes.c_void_p),
+                ("w_ln_ffn", ctypes.c_void_p), ("w_q_norm", ctypes.c_void_p), ("w_k_norm", ctypes.c_void_p),
+                ("rms_eps", ctypes.c_float), ("rope_theta", ctypes.c_float)]
 
 
 class AflexError(RuntimeError):
@@ -100,6 +107,16 @@ def load_library() -> ctypes.CDLL:
     lib.aflex_profile_enable.argtypes = [vp, ci]
     lib.aflex_profile_read.restype = ci
     lib.aflex_profile_read.argtypes = [vp, ci, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_longlong)]
+    lib.aflex_decoder_layers.restype = ci
+    lib.aflex_decoder_layers.argtypes = [vp, ctypes.POINTER(DecoderDesc), ctypes.POINTER(KV), ci, vp, ci, ci,
+                                         ctypes.POINTER(ctypes.c_int32), vp, vp]
+    lib.aflex_decoder_workspace_bytes.restype = cs
+    lib.aflex_decoder_workspace_bytes.argtypes = [ctypes.POINTER(DecoderDesc), ci]
+    lib.aflex_add_rmsnorm.restype = ci
+    lib.aflex_add_rmsnorm.argtypes = [vp, vp, vp, vp, ci, ci, ctypes.c_float, vp, vp, vp]
+    lib.aflex_rope_append.restype = ci
+    lib.aflex_rope_append.argtypes = [vp, ctypes.POINTER(AttnDesc), vp, ctypes.POINTER(KV), ci, vp, vp,
+                                      ctypes.c_float, ctypes.c_float, vp, vp]
     lib.aflex_attn_decode_static.restype = ci
     lib.aflex_attn_decode_static.argtypes = [ctypes.POINTER(AttnDesc), vp, ctypes.POINTER(KV), ci, vp, vp, vp]
     _lib = lib
@@ -142,6 +159,18 @@ def layer_desc(attn: AttnDesc, hidden: int, inter: int, w_o, w_gate, w_up, w_dow
                   _ptr(w_router))
     d._keep = (w_o, w_gate, w_up, w_down, w_router)
     return d
+
+
+def decoder_desc(layer: LayerDesc, w_qkv, w_ln_attn, w_ln_ffn, w_q_norm, w_k_norm, rms_eps: float,
+                 rope_theta: float) -> DecoderDesc:
+    d = DecoderDesc(layer, _ptr(w_qkv), _ptr(w_ln_attn), _ptr(w_ln_ffn), _ptr(w_q_norm), _ptr(w_k_norm),
+                    rms_eps, rope_theta)
+    d._keep = (layer, w_qkv, w_ln_attn, w_ln_ffn, w_q_norm, w_k_norm)
+    return d
+
+
+def decoder_workspace_bytes(layer: DecoderDesc, max_batch: int) -> int:
+    return int(load_library().aflex_decoder_workspace_bytes(ctypes.byref(layer), max_batch))
 
 
 def workspace_bytes(layer: LayerDesc, max_batch: int, max_pages_per_seq: int) -> int:
@@ -267,3 +296,26 @@ class Context:
         self._check(self._lib.aflex_layer_step(self._h, ctypes.byref(layer), _ptr(q), ctypes.byref(kv), q.shape[0],
                                                _ptr(router_logits), microbatch_depth, offs, _ptr(attn_out),
                                                _ptr(y), _stream(stream)))
+
+    def decoder_layers(self, layers: Sequence[DecoderDesc], kvs: Sequence[KV], x_in, x_out,
+                       microbatch_depth: int = 1, mb_offsets: Optional[Sequence[int]] = None, stream=None) -> None:
+        """Runs len(layers) whole decoder layers on x_in bf16 [B,H] -> x_out; kvs[l] is layer l's cache
+        (its decoded-token slots are written)."""
+        assert len(layers) == len(kvs) and len(layers) >= 1
+        offs = None
+        if mb_offsets is not None:
+            offs = (ctypes.c_int32 * len(mb_offsets))(*[int(v) for v in mb_offsets])
+        la = (DecoderDesc * len(layers))(*layers)
+        ka = (KV * len(kvs))(*kvs)
+        self._check(self._lib.aflex_decoder_layers(self._h, la, ka, len(layers), _ptr(x_in), x_in.shape[0],
+                                                   microbatch_depth, offs, _ptr(x_out), _stream(stream)))
+
+    def add_rmsnorm(self, res, add, w, eps: float, res_out=None, y=None, stream=None) -> None:
+        self._check(self._lib.aflex_add_rmsnorm(self._h, _ptr(res), _ptr(add), _ptr(w), res.shape[0], res.shape[1],
+                                                eps, _ptr(res_out), _ptr(y), _stream(stream)))
+
+    def rope_append(self, desc: AttnDesc, qkv, kv: KV, q_out, w_q_norm, w_k_norm, rms_eps: float, rope_theta: float,
+                    stream=None) -> None:
+        self._check(self._lib.aflex_rope_append(self._h, ctypes.byref(desc), _ptr(qkv), ctypes.byref(kv),
+                                                qkv.shape[0], _ptr(w_q_norm), _ptr(w_k_norm), rms_eps, rope_theta,
+                                                _ptr(q_out), _stream(stream)))

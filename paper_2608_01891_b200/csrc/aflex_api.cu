@@ -278,6 +278,8 @@ aflex_status aflex_create(aflex_ctx** out, int device, size_t workspace_bytes) {
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_f_done, cudaEventDisableTiming);
     for (int i = 0; i < kMaxMicrobatches && e == cudaSuccess; ++i)
         e = cudaEventCreateWithFlags(&ctx->ev_a[i], cudaEventDisableTiming);
+    for (int i = 0; i < kMaxMicrobatches && e == cudaSuccess; ++i)
+        e = cudaEventCreateWithFlags(&ctx->ev_f[i], cudaEventDisableTiming);
     if (e != cudaSuccess || !get_encode_fn()) {
         aflex_destroy(ctx);
         return AFLEX_ERR_CUDA;
@@ -292,6 +294,7 @@ aflex_status aflex_destroy(aflex_ctx* ctx) {
     if (ctx->stream_a) cudaStreamSynchronize(ctx->stream_a);
     if (ctx->stream_f) cudaStreamSynchronize(ctx->stream_f);
     for (int i = 0; i < kMaxMicrobatches; ++i) if (ctx->ev_a[i]) cudaEventDestroy(ctx->ev_a[i]);
+    for (int i = 0; i < kMaxMicrobatches; ++i) if (ctx->ev_f[i]) cudaEventDestroy(ctx->ev_f[i]);
     if (ctx->ev_entry) cudaEventDestroy(ctx->ev_entry);
     if (ctx->ev_a_done) cudaEventDestroy(ctx->ev_a_done);
     if (ctx->ev_f_done) cudaEventDestroy(ctx->ev_f_done);
@@ -338,7 +341,8 @@ aflex_status aflex_get_device_status(aflex_ctx* ctx, void* stream) {
 
 static const char* kKernelNames[kKKindCount] = {
     "attn_decode", "linear_gemm", "down_gemm", "gateup_gemm", "router_logits",
-    "moe_route", "moe_gather", "moe_gateup_gemm", "moe_down_gemm", "moe_combine"};
+    "moe_route", "moe_gather", "moe_gateup_gemm", "moe_down_gemm", "moe_combine",
+    "add_rmsnorm", "qkv_gemm", "rope_append"};
 
 int aflex_num_kernel_kinds(void) { return kKKindCount; }
 
@@ -586,6 +590,197 @@ aflex_status aflex_layer_step(aflex_ctx* ctx, const aflex_layer_desc* L, const v
     if (e == cudaSuccess) e = cudaStreamWaitEvent(user, ctx->ev_a_done, 0);
     if (e == cudaSuccess) e = cudaStreamWaitEvent(user, ctx->ev_f_done, 0);
     return check_cuda(ctx, e, "layer step: exit join");
+}
+
+// ---- whole decoder layers ------------------------------------------------------------------
+// Workspace: [A scratch | resid | xn | qkv | q | a | o | xn2 | y | F scratch].  The row-indexed
+// buffers are touched by microbatch i only in rows of i, in the order A_{l,i} -> F_{l,i} ->
+// A_{l+1,i} that the events enforce; the A scratch is used on the attention stream only, the F
+// scratch on the FFN stream only.
+namespace {
+struct DecoderWs {
+    size_t a_attn, a_lin, rows_h, rows_qkv, rows_a, f_total, total;
+};
+DecoderWs decoder_ws(const aflex_decoder_desc* d, int max_batch, size_t a_attn, int num_sms) {
+    const aflex_layer_desc* L = &d->layer;
+    const int D = L->attn.head_dim, A = L->attn.num_q_heads * D, H = L->hidden;
+    const int NQ = (L->attn.num_q_heads + 2 * L->attn.num_kv_heads) * D;
+    DecoderWs w;
+    w.a_attn = a_attn;
+    w.a_lin = 0;
+    for (int t = 1; t <= max_batch; t = (t < 16 ? t + 1 : t + 16)) {
+        const size_t b0 = linear_workspace_bytes(t, A, H, num_sms), b1 = linear_workspace_bytes(t, H, NQ, num_sms);
+        if (b0 > w.a_lin) w.a_lin = b0;
+        if (b1 > w.a_lin) w.a_lin = b1;
+    }
+    {
+        const size_t b0 = linear_workspace_bytes(max_batch, A, H, num_sms), b1 = linear_workspace_bytes(max_batch, H, NQ, num_sms);
+        if (b0 > w.a_lin) w.a_lin = b0;
+        if (b1 > w.a_lin) w.a_lin = b1;
+    }
+    w.rows_h = align256((size_t)max_batch * H * 2);
+    w.rows_qkv = align256((size_t)max_batch * NQ * 2);
+    w.rows_a = align256((size_t)max_batch * A * 2);
+    w.f_total = layer_ws(L, max_batch, 0, num_sms).f_total;
+    w.total = w.a_attn + w.a_lin + 5 * w.rows_h + w.rows_qkv + 2 * w.rows_a + w.f_total + 1024;
+    return w;
+}
+}  // namespace
+
+size_t aflex_decoder_workspace_bytes(const aflex_decoder_desc* layer, int max_batch) {
+    if (!layer || max_batch < 1) return 0;
+    return decoder_ws(layer, max_batch, attn_workspace_bytes(&layer->layer.attn, 4096), 148).total;
+}
+
+aflex_status aflex_add_rmsnorm(aflex_ctx* ctx, const void* res, const void* add, const void* w, int T, int H, float eps,
+                               void* res_out, void* y, void* stream) {
+    if (!ctx) return AFLEX_ERR_INVALID_ARG;
+    if (!res || (!res_out && !y) || (y && !w) || T < 1 || H < 1)
+        return set_error(ctx, AFLEX_ERR_INVALID_ARG, "add_rmsnorm: bad argument");
+    if (H % 8) return set_error(ctx, AFLEX_ERR_UNSUPPORTED, "add_rmsnorm: H must be a multiple of 8");
+    if (!aligned16(res) || !aligned16(add) || !aligned16(w) || !aligned16(res_out) || !aligned16(y))
+        return set_error(ctx, AFLEX_ERR_INVALID_ARG, "add_rmsnorm: pointers must be 16-byte aligned");
+    return add_rmsnorm_launch(ctx, res, add, w, T, H, eps, res_out, y, reinterpret_cast<cudaStream_t>(stream));
+}
+
+aflex_status aflex_rope_append(aflex_ctx* ctx, const aflex_attn_desc* desc, const void* qkv, const aflex_kv* kv, int batch,
+                               const void* w_q_norm, const void* w_k_norm, float rms_eps, float rope_theta, void* q_out,
+                               void* stream) {
+    aflex_status s = validate_attn(ctx, desc, qkv, kv, batch, q_out);
+    if (s != AFLEX_OK) return s;
+    if (!(rope_theta > 0.f)) return set_error(ctx, AFLEX_ERR_INVALID_ARG, "rope_append: rope_theta must be > 0");
+    return rope_append_launch(ctx, desc, qkv, kv, batch, w_q_norm, w_k_norm, rms_eps, rope_theta, q_out,
+                              reinterpret_cast<cudaStream_t>(stream));
+}
+
+aflex_status aflex_decoder_layers(aflex_ctx* ctx, const aflex_decoder_desc* layers, const aflex_kv* kvs, int num_layers,
+                                  const void* x_in, int batch, int M, const int32_t* mb_offsets, void* x_out,
+                                  void* stream) {
+    if (!ctx) return AFLEX_ERR_INVALID_ARG;
+    if (!layers || !kvs || !x_in || !x_out || num_layers < 1)
+        return set_error(ctx, AFLEX_ERR_INVALID_ARG, "decoder layers: null argument or num_layers < 1");
+    if (!aligned16(x_in) || !aligned16(x_out))
+        return set_error(ctx, AFLEX_ERR_INVALID_ARG, "decoder layers: pointers must be 16-byte aligned");
+    const int H = layers[0].layer.hidden;
+    aflex_status s;
+    size_t need = 0;
+    for (int l = 0; l < num_layers; ++l) {
+        const aflex_decoder_desc* d = &layers[l];
+        const aflex_layer_desc* L = &d->layer;
+        s = validate_attn(ctx, &L->attn, x_in, &kvs[l], batch, x_out);
+        if (s != AFLEX_OK) return s;
+        if (L->hidden != H) return set_error(ctx, AFLEX_ERR_INVALID_ARG, "decoder layers: layer %d has another hidden size", l);
+        if (!d->w_qkv || !d->w_ln_attn || !d->w_ln_ffn || !L->w_o || !L->w_gate || !L->w_up || !L->w_down)
+            return set_error(ctx, AFLEX_ERR_INVALID_ARG, "decoder layers: layer %d has a null weight", l);
+        if (!aligned16(d->w_qkv) || !aligned16(d->w_ln_attn) || !aligned16(d->w_ln_ffn) || !aligned16(L->w_o) ||
+            !aligned16(L->w_gate) || !aligned16(L->w_up) || !aligned16(L->w_down))
+            return set_error(ctx, AFLEX_ERR_INVALID_ARG, "decoder layers: pointers must be 16-byte aligned");
+        if (!(d->rope_theta > 0.f) || !(d->rms_eps >= 0.f))
+            return set_error(ctx, AFLEX_ERR_INVALID_ARG, "decoder layers: rope_theta must be > 0 and rms_eps >= 0");
+        if (L->num_experts == 0) s = validate_ffn_dims(ctx, batch, H, L->inter);
+        else {
+            s = validate_moe(ctx, batch, H, L->inter, L->num_experts, L->top_k);
+            if (s == AFLEX_OK && !L->w_router) s = set_error(ctx, AFLEX_ERR_INVALID_ARG, "decoder layers: MoE layer %d needs w_router", l);
+        }
+        if (s != AFLEX_OK) return s;
+        const DecoderWs w = decoder_ws(d, batch, attn_workspace_bytes(&L->attn, attn_grid(ctx)), ctx->num_sms);
+        if (w.total > need) need = w.total;
+    }
+    if (need > ctx->ws_bytes)
+        return set_error(ctx, AFLEX_ERR_WORKSPACE, "decoder layers: need %zu workspace bytes, have %zu", need, ctx->ws_bytes);
+    if (M < 1 || M > batch || M > kMaxMicrobatches)
+        return set_error(ctx, AFLEX_ERR_INVALID_ARG, "decoder layers: microbatch depth %d outside [1, min(batch, %d)]", M, kMaxMicrobatches);
+    int32_t offs[kMaxMicrobatches + 1];
+    if (mb_offsets) {
+        for (int i = 0; i <= M; ++i) offs[i] = mb_offsets[i];
+        if (offs[0] != 0 || offs[M] != batch) return set_error(ctx, AFLEX_ERR_INVALID_ARG, "decoder layers: mb_offsets must run from 0 to batch");
+        for (int i = 0; i < M; ++i)
+            if (offs[i + 1] <= offs[i]) return set_error(ctx, AFLEX_ERR_INVALID_ARG, "decoder layers: mb_offsets must be strictly increasing");
+    } else {
+        const int base = batch / M, extra = batch % M;
+        offs[0] = 0;
+        for (int i = 0; i < M; ++i) offs[i + 1] = offs[i] + base + (i < extra ? 1 : 0);
+    }
+
+    cudaStream_t user = reinterpret_cast<cudaStream_t>(stream);
+    const bool serial = (M == 1);
+    cudaStream_t sa = serial ? user : ctx->stream_a, sf = serial ? user : ctx->stream_f;
+    cudaError_t e = cudaSuccess;
+    if (!serial) {
+        e = cudaEventRecord(ctx->ev_entry, user);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(sa, ctx->ev_entry, 0);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(sf, ctx->ev_entry, 0);
+        if (e != cudaSuccess) return check_cuda(ctx, e, "decoder layers: entry join");
+    }
+    typedef __nv_bfloat16 bf;
+    for (int l = 0; l < num_layers; ++l) {
+        const aflex_decoder_desc* d = &layers[l];
+        const aflex_layer_desc* L = &d->layer;
+        const int Hq = L->attn.num_q_heads, Hkv = L->attn.num_kv_heads, D = L->attn.head_dim;
+        const int A = Hq * D, NQ = (Hq + 2 * Hkv) * D, I = L->inter, E = L->num_experts;
+        const DecoderWs w = decoder_ws(d, batch, attn_workspace_bytes(&L->attn, attn_grid(ctx)), ctx->num_sms);
+        char* p = ctx->ws;
+        char* ws_attn = p; p += w.a_attn;
+        char* ws_lin = p; p += w.a_lin;
+        bf* resid = reinterpret_cast<bf*>(p); p += w.rows_h;
+        bf* xn = reinterpret_cast<bf*>(p); p += w.rows_h;
+        bf* qkv = reinterpret_cast<bf*>(p); p += w.rows_qkv;
+        bf* qb = reinterpret_cast<bf*>(p); p += w.rows_a;
+        bf* ab = reinterpret_cast<bf*>(p); p += w.rows_a;
+        bf* ob = reinterpret_cast<bf*>(p); p += w.rows_h;
+        bf* xn2 = reinterpret_cast<bf*>(p); p += w.rows_h;
+        bf* yb = reinterpret_cast<bf*>(p); p += w.rows_h;
+        char* ws_f = p;
+        for (int i = 0; i < M; ++i) {
+            const int r0 = offs[i], rows = offs[i + 1] - offs[i];
+            const size_t oh = (size_t)r0 * H;
+            // ---- A_{l,i}
+            if (l > 0 && !serial) {
+                e = cudaStreamWaitEvent(sa, ctx->ev_f[i], 0);     // F_{l-1,i} has returned this microbatch
+                if (e != cudaSuccess) return check_cuda(ctx, e, "decoder layers: F->A event");
+            }
+            if (l == 0) s = add_rmsnorm_launch(ctx, reinterpret_cast<const bf*>(x_in) + oh, nullptr, d->w_ln_attn, rows, H, d->rms_eps, resid + oh, xn + oh, sa);
+            else s = add_rmsnorm_launch(ctx, resid + oh, yb + oh, d->w_ln_attn, rows, H, d->rms_eps, resid + oh, xn + oh, sa);
+            if (s != AFLEX_OK) return s;
+            s = linear_launch(ctx, xn + oh, d->w_qkv, rows, H, NQ, qkv + (size_t)r0 * NQ, ws_lin, w.a_lin, sa, kKQkvGemm, ctx->counters_a);
+            if (s != AFLEX_OK) return s;
+            aflex_kv kvi = kvs[l];
+            kvi.page_table = kvs[l].page_table + (size_t)r0 * kvs[l].max_pages_per_seq;
+            kvi.seq_lens = kvs[l].seq_lens + r0;
+            kvi.seq_lens_host = kvs[l].seq_lens_host ? kvs[l].seq_lens_host + r0 : nullptr;
+            s = rope_append_launch(ctx, &L->attn, qkv + (size_t)r0 * NQ, &kvi, rows, d->w_q_norm, d->w_k_norm, d->rms_eps, d->rope_theta, qb + (size_t)r0 * A, sa);
+            if (s != AFLEX_OK) return s;
+            s = attn_decode_launch(ctx, &L->attn, qb + (size_t)r0 * A, &kvi, rows, ab + (size_t)r0 * A, nullptr, ws_attn, w.a_attn, sa);
+            if (s != AFLEX_OK) return s;
+            s = linear_launch(ctx, ab + (size_t)r0 * A, L->w_o, rows, A, H, ob + oh, ws_lin, w.a_lin, sa, kKLinearGemm, ctx->counters_a);
+            if (s != AFLEX_OK) return s;
+            if (!serial) {
+                e = cudaEventRecord(ctx->ev_a[i], sa);
+                if (e == cudaSuccess) e = cudaStreamWaitEvent(sf, ctx->ev_a[i], 0);
+                if (e != cudaSuccess) return check_cuda(ctx, e, "decoder layers: A->F event");
+            }
+            // ---- F_{l,i}
+            s = add_rmsnorm_launch(ctx, resid + oh, ob + oh, d->w_ln_ffn, rows, H, d->rms_eps, resid + oh, xn2 + oh, sf);
+            if (s != AFLEX_OK) return s;
+            if (E == 0) s = dense_run(ctx, xn2 + oh, L->w_gate, L->w_up, L->w_down, rows, H, I, yb + oh, ws_f, w.f_total, sf);
+            else s = moe_run(ctx, xn2 + oh, nullptr, L->w_router, L->w_gate, L->w_up, L->w_down, rows, H, I, E, L->top_k, yb + oh,
+                             nullptr, nullptr, nullptr, ws_f, w.f_total, sf);
+            if (s != AFLEX_OK) return s;
+            if (l == num_layers - 1) {     // hidden states leaving the last layer
+                s = add_rmsnorm_launch(ctx, resid + oh, yb + oh, nullptr, rows, H, 0.f, reinterpret_cast<bf*>(x_out) + oh, nullptr, sf);
+                if (s != AFLEX_OK) return s;
+            } else if (!serial) {
+                e = cudaEventRecord(ctx->ev_f[i], sf);
+                if (e != cudaSuccess) return check_cuda(ctx, e, "decoder layers: F event");
+            }
+        }
+    }
+    if (serial) return AFLEX_OK;
+    e = cudaEventRecord(ctx->ev_a_done, sa);
+    if (e == cudaSuccess) e = cudaEventRecord(ctx->ev_f_done, sf);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(user, ctx->ev_a_done, 0);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(user, ctx->ev_f_done, 0);
+    return check_cuda(ctx, e, "decoder layers: exit join");
 }
 
 }  // extern "C"

@@ -18,16 +18,19 @@ constexpr int kTraceKernels = 64;              // timeline debugging: ring of pe
 constexpr int kTraceStride = 4096 * 8;         // u64 per launch record: [cta < 4096][8 stamps]
 constexpr int kStreamKMaxTiles = 16384;       // capacity of each per-tile arrival-counter array
 
+
 }  // namespace aflex
 
 namespace aflex {
 // Kernel kinds, for launch counting and optional per-kernel event timing.
 enum KernelKind {
     kKAttnDecode = 0, kKLinearGemm, kKDownGemm, kKGateUpGemm, kKRouterLogits,
-    kKMoeRoute, kKMoeGather, kKMoeGateUpGemm, kKMoeDownGemm, kKMoeCombine, kKKindCount
+    kKMoeRoute, kKMoeGather, kKMoeGateUpGemm, kKMoeDownGemm, kKMoeCombine,
+    kKAddRmsNorm, kKQkvGemm, kKRopeAppend, kKKindCount
 };
 constexpr int kProfMaxSlots = 8192;
 struct ProfSlot { cudaEvent_t start, stop; int kind; };
+
 }  // namespace aflex
 
 struct aflex_ctx {
@@ -43,6 +46,7 @@ struct aflex_ctx {
     cudaStream_t stream_a = nullptr, stream_f = nullptr;
     cudaEvent_t ev_entry = nullptr;
     cudaEvent_t ev_a[aflex::kMaxMicrobatches] = {};
+    cudaEvent_t ev_f[aflex::kMaxMicrobatches] = {};   // F_{l,i} done (decoder chain)
     cudaEvent_t ev_f_done = nullptr, ev_a_done = nullptr;
     int attn_ctas = 0;            // persistent attention CTAs per launch; 0 = two per SM
     bool gemm_attr_set[2] = {false, false};
@@ -160,5 +164,12 @@ aflex_status moe_gather_launch(aflex_ctx* ctx, const void* x, const int32_t* pos
                                cudaStream_t st);
 aflex_status moe_combine_launch(aflex_ctx* ctx, const float* yp, const int32_t* pos, const float* gate, int T,
                                 int K, int H, void* y, cudaStream_t st);
+
+
+// ---- decoder-layer glue (decoder.cu)
+aflex_status add_rmsnorm_launch(aflex_ctx* ctx, const void* res, const void* add, const void* w, int T, int H, float eps,
+                                void* res_out, void* y, cudaStream_t st);
+aflex_status rope_append_launch(aflex_ctx* ctx, const aflex_attn_desc* d, const void* qkv, const aflex_kv* kv, int batch,
+                                const void* w_qn, const void* w_kn, float eps, float theta, void* q_out, cudaStream_t st);
 
 }  // namespace aflex
