@@ -211,6 +211,62 @@ def run_ffn_sweep(args, cfg, local_rank, device, peaks):
     ctx.close()
 
 
+def run_decoder_chain(args, cfg, local_rank, device, peaks):
+    """Whole decoder layers chained (aflex_decoder_layers): L layers, each with its own weights and KV cache,
+    at every microbatch depth of the configuration.  One JSON line: time per layer, tokens/s, the share of the
+    measured HBM bandwidth the layer's algorithmic bytes reach, and the per-kernel times of the M = 1 chain."""
+    from paper_2608_01891_b200 import aflex as AF
+    L = args.decoder_layers
+    kvh = IN.make_paged_kv(cfg, device=device)
+    table, lens = kvh.page_table.to(device), kvh.seq_lens.to(device)
+    attn = AF.attn_desc(cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim)
+    descs, kvs, keep = [], [], []
+    for l in range(L):
+        w = IN.make_decoder_weights(cfg, l, device=device)
+        layer = AF.layer_desc(attn, cfg.hidden, cfg.inter, w.o, w.gate, w.up, w.down, cfg.num_experts, cfg.top_k, w.router)
+        descs.append(AF.decoder_desc(layer, w.qkv, w.ln_attn, w.ln_ffn, w.q_norm, w.k_norm, cfg.rms_eps, cfg.rope_theta))
+        kc, vc = (kvh.k_cache, kvh.v_cache) if l == 0 else (kvh.k_cache.clone(), kvh.v_cache.clone())
+        kvs.append(AF.make_kv(kc, vc, table, lens, kvh.seq_lens))
+        keep.append((w, kc, vc))
+    x = IN.make_hidden(cfg, device=device)
+    y = torch.empty_like(x)
+    ctx = AF.Context(local_rank, max(AF.decoder_workspace_bytes(d, cfg.batch) for d in descs))
+    stream = torch.cuda.current_stream()
+    n_qkv = (cfg.num_q_heads + 2 * cfg.num_kv_heads) * cfg.head_dim
+    extra = 2.0 * n_qkv * cfg.hidden                      # W_qkv bytes on top of the hot path's
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    rows = []
+    for M in cfg.microbatch_depths:
+        for _ in range(max(3, args.warmup)):
+            ctx.decoder_layers(descs, kvs, x, y, M, None, stream)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(args.steps):
+            ctx.decoder_layers(descs, kvs, x, y, M, None, stream)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        us_layer = 1e3 * e0.elapsed_time(e1) / args.steps / L
+        byts = M * (sum(algorithmic_bytes(cfg, kvh.seq_lens.numpy(), M).values()) + extra)
+        rows.append({"M": M, "us_per_layer": round(us_layer, 1), "tokens_per_s": round(cfg.batch / us_layer * 1e6),
+                     "algorithmic_gbs": round(byts / us_layer / 1e3, 1),
+                     "frac_hbm": round(byts / us_layer / 1e3 / peaks["hbm_gbs"], 4)})
+    ctx.profile_enable(True)
+    for _ in range(5):
+        ctx.decoder_layers(descs, kvs, x, y, 1, None, stream)
+    prof = ctx.profile_read()
+    ctx.profile_enable(False)
+    assert ctx.device_status() == AF.OK
+    line = {"metric": "whole decoder layer, chained: tokens/s per layer", "unit": "tokens/s", "dtype": "bf16",
+            "data": "synthetic", "config": {"workload": f"config {cfg.cfg_id}: {cfg.name}, {L} chained decoder layers",
+                                            "batch": cfg.batch, "l2": "per-layer weights + KV larger than L2, no flush"},
+            "peaks": peaks, "clocks": sampler.stop(), "depths": rows,
+            "kernel_us_event_pairs_M1": {k: round(1e3 * v[0] / v[1], 1) for k, v in prof.items()}}
+    print(json.dumps(line), flush=True)
+    ctx.close()
+
+
 def dataclasses_replace_dense(cfg):
     """The configuration's FFN shape as a dense FFN (MoE configurations: one expert's shape)."""
     import dataclasses
@@ -301,6 +357,9 @@ def main():
     ap.add_argument("--ffn-sweep", action="store_true",
                     help="instead of the layer step: dense FFN (aflex_ffn_dense) at the configuration's weight shape "
                          "for T = 32..8192 tokens, TFLOP/s against the measured bf16 peak; prints one JSON line")
+    ap.add_argument("--decoder-layers", type=int, default=0,
+                    help="instead of the layer step: chain this many whole decoder layers (aflex_decoder_layers) at "
+                         "every microbatch depth of the configuration; prints one JSON line")
     ap.add_argument("--energy", action="store_true",
                     help="also read the NVML energy counter around a >= 2 s loop of the step (default clocks)")
     args = ap.parse_args()
@@ -335,6 +394,10 @@ def main():
     if args.ffn_sweep:
         if rank == 0:
             run_ffn_sweep(args, cfg, local_rank, device, peaks)
+        return
+    if args.decoder_layers > 0:
+        if rank == 0:
+            run_decoder_chain(args, cfg, local_rank, device, peaks)
         return
     wl = build_workload(cfg, device)
     lens_np = wl["kvh"].seq_lens.numpy()

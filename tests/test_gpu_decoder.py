@@ -243,6 +243,40 @@ def test_decoder_layers_match_oracle(cfg, L):
         ctx.close()
 
 
+def test_decoder_layers_attention_sees_the_token_it_just_appended():
+    """Sequences of 1-3 tokens: the appended K/V carries most of the softmax weight, so an attention
+    that read the cache before the append would be far off."""
+    cfg = IN.CONFIGS[1]
+    ch = Chain(cfg, 2, seq_lens=np.array([1, 2, 1, 3], dtype=np.int32))
+    ctx = AF.Context(0, ch.workspace())
+    try:
+        outs, _, _ = ch.oracle()
+        for M in (1, 2, 4):
+            x_out = _run_chain(ctx, ch, M)
+            assert row_rel_err(f64(x_out), outs[-1]) <= TOL_FFN * 2, M
+        # the stand-alone attention after a stand-alone append agrees with the oracle on the same cache
+        ch.reset_caches()
+        B, Hq, Hkv, D = cfg.batch, cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim
+        g = torch.Generator().manual_seed(9)
+        qkv = torch.randn(B, (Hq + 2 * Hkv) * D, generator=g).to(torch.bfloat16).to(DEV)
+        q = torch.empty(B, Hq, D, dtype=torch.bfloat16, device=DEV)
+        out = torch.empty_like(q)
+        desc = AF.attn_desc(Hq, Hkv, D)
+        ctx.rope_append(desc, qkv, ch.kvs[0], q, None, None, cfg.rms_eps, cfg.rope_theta)
+        ctx.attn_decode(desc, q, ch.kvs[0], out)
+        torch.cuda.synchronize()
+        kc, vc = ch.caches[0]
+        want, _ = O.attn_decode(u16(q), u16(kc), u16(vc), ch.kvh.page_table.numpy(), ch.kvh.seq_lens.numpy())
+        assert row_rel_err(f64(out), want) <= TOL_ATTN
+        # sequences of one token return exactly the value rows just stored
+        v_new = qkv.view(B, Hq + 2 * Hkv, D)[:, Hq + Hkv:, :]
+        for b in (0, 2):
+            got = out[b].view(Hkv, Hq // Hkv, D)
+            assert torch.equal(got, v_new[b][:, None, :].expand(Hkv, Hq // Hkv, D))
+    finally:
+        ctx.close()
+
+
 def test_decoder_layers_in_place_and_argument_checks():
     cfg = IN.CONFIGS[1]
     ch = Chain(cfg, 2)
