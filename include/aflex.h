@@ -337,6 +337,80 @@ AFLEX_API aflex_status aflex_rope_append(aflex_ctx* ctx, const aflex_attn_desc* 
                                          const aflex_kv* kv, int batch, const void* w_q_norm, const void* w_k_norm,
                                          float rms_eps, float rope_theta, void* q_out, void* stream);
 
+/* ---- Host-side decisions of the data plane and the DVFS controller ------------------------
+ *
+ * Pure host computation on HOST pointers: nothing is launched and no GPU setting is read or
+ * changed (applying a chosen frequency is the caller's business).  Times are in one unit of the
+ * caller's choice (microseconds in the tests).
+ */
+
+/* Eq. 2 (Section 4.3): depth 1 -> t_a + t_f + t_comm; depth >= 2 -> max(t_a, t_f) + t_comm / depth. */
+AFLEX_API double aflex_eq2_layer_time(double t_a, double t_f, double t_comm, int depth);
+
+/* A profiled latency curve: n >= 1 points, x strictly ascending; piecewise linear, the end
+ * segments extended beyond the profiled range, a single point is a constant. */
+typedef struct { int n; const double* x; const double* y; } aflex_curve;
+AFLEX_API double aflex_curve_eval(const aflex_curve* curve, double x);   /* NaN on a malformed curve */
+
+/* Predicted stage times of one microbatch ("profiled Attention/FFN latency curves", Section 4.3):
+ *   t_A = attn_vs_tokens(sum of its context lengths) + attn_vs_rows(rows),  t_F = ffn_vs_rows(rows),
+ *   one hidden-state transfer, either direction = comm_fixed + comm_per_row * rows;
+ *   t_A and t_F are clamped at zero where an extended curve goes negative.
+ * shared_memory_system != 0: both sides run on one GPU; stages then queue on one engine (they do
+ * not overlap) and transfers cost nothing. */
+typedef struct {
+    aflex_curve attn_vs_tokens, attn_vs_rows, ffn_vs_rows;
+    double comm_fixed, comm_per_row;
+    int shared_memory_system;
+} aflex_pipeline_model;
+
+/*
+ * Completion time of `layers` chained layers cut into `depth` microbatches at host offsets
+ * [depth+1] under the interleaved schedule of Section 4.3: stages A, transfer, F, transfer back of
+ * every (layer, microbatch); each of the four engines serves its stages in (layer, microbatch)
+ * order; A of layer l+1 starts for a microbatch once its hidden states are back.  With depth 1 this
+ * is layers * Eq. 2 (t_comm = both transfers).  Returns NaN on invalid arguments.
+ */
+AFLEX_API double aflex_pipeline_makespan(const aflex_pipeline_model* model, const int32_t* seq_lens_host, int batch,
+                                         int depth, const int32_t* offsets, int layers);
+
+/*
+ * "Dynamic microbatch depth" and "adaptive request batching" (Section 4.3): among the candidate
+ * depths[n_depths] and all contiguous splits whose boundaries are multiples of `granularity` rows,
+ * the pair with the lowest aflex_pipeline_makespan.  Ties keep the smaller depth, then the
+ * lexicographically smaller offsets.  best_offsets: HOST i32 [max depth + 1].  The search is
+ * exhaustive; more than 4e6 candidate splits return AFLEX_ERR_UNSUPPORTED (raise the granularity).
+ */
+AFLEX_API aflex_status aflex_plan_microbatches(const aflex_pipeline_model* model, const int32_t* seq_lens_host,
+                                               int batch, int layers, const int* depths, int n_depths,
+                                               int granularity, int* best_depth, int32_t* best_offsets,
+                                               double* predicted);
+
+/* Window size of the decode DVFS controller (Section 4.4): max(w_min, round(kappa * t_switch / t_iter)),
+ * halves rounded away from zero. */
+AFLEX_API int aflex_dvfs_window(int w_min, double kappa, double t_switch, double t_iter);
+
+/* Algorithm 1 (window-based decode DVFS).  Frequencies are indices into the caller's ascending
+ * DA / DF lists (the last index is f_max).  t_hat / e_hat: HOST [n_da][n_df] predicted iteration
+ * time and energy of every pair for the current decode state and microbatch depth. */
+typedef struct { int n_da, n_df; double tau; double delta_b; int window; double t_switch; } aflex_dvfs_params;
+typedef struct { int i_da, i_df; int w; int b_last; } aflex_dvfs_state;
+/* One decode iteration with batch size batch_now and measured time t_iter.  Returns 0: window still
+ * open, state.w advanced; 1: searched, pair kept; 2: searched, pair changed (the caller applies
+ * it); -1: invalid arguments.  Among equal-energy feasible pairs the first in (DA, DF) order wins. */
+AFLEX_API int aflex_dvfs_decode_step(const aflex_dvfs_params* params, const double* t_hat, const double* e_hat,
+                                     int batch_now, double t_iter, aflex_dvfs_state* state);
+
+/* Prefill pair (Section 4.4): lowest-energy pair whose predicted time, plus t_switch when it
+ * differs from the current pair, fits `budget` (the tightest remaining TTFT slack).  Returns flags:
+ * AFLEX_DVFS_ESCALATED when the pair exceeds the global plan's baseline in either domain,
+ * AFLEX_DVFS_INFEASIBLE when nothing fits (then the pair is (f_max, f_max)); -1 on invalid arguments. */
+#define AFLEX_DVFS_ESCALATED 1
+#define AFLEX_DVFS_INFEASIBLE 2
+AFLEX_API int aflex_dvfs_prefill_pair(int n_pa, int n_pf, const double* t_hat, const double* e_hat, double budget,
+                                      double t_switch, int cur_pa, int cur_pf, int base_pa, int base_pf,
+                                      int* out_pa, int* out_pf);
+
 /* ---- Measurement support (no counterpart in the paper's method; the per-operator latency
  * profiling of its Section 4.1 is the motivation) --------------------------------------------
  *

@@ -48,17 +48,18 @@ class Model:
     t_A = attn_tokens(sum of its context lengths) + attn_rows(rows);  t_F = ffn_rows(rows);
     one hidden-state transfer (either direction) = comm_fixed + comm_per_row * rows.
     shared = True: both sides run on one GPU and share its memory system; stages then do not
-    overlap (reading: the measured one-GPU step times add up), and transfers cost nothing."""
+    overlap (reading: the measured one-GPU step times add up), and transfers cost nothing.
+    A curve extended below zero predicts no time at all: stage times are clamped at zero."""
 
     def __init__(self, attn_tokens, attn_rows, ffn_rows, comm_fixed=0.0, comm_per_row=0.0, shared=False):
         self.attn_tokens, self.attn_rows, self.ffn_rows = attn_tokens, attn_rows, ffn_rows
         self.comm_fixed, self.comm_per_row, self.shared = comm_fixed, comm_per_row, shared
 
     def t_a(self, lens: Sequence[int]) -> float:
-        return curve_eval(*self.attn_tokens, float(sum(lens))) + curve_eval(*self.attn_rows, float(len(lens)))
+        return max(0.0, curve_eval(*self.attn_tokens, float(sum(lens))) + curve_eval(*self.attn_rows, float(len(lens))))
 
     def t_f(self, rows: int) -> float:
-        return curve_eval(*self.ffn_rows, float(rows))
+        return max(0.0, curve_eval(*self.ffn_rows, float(rows)))
 
     def t_x(self, rows: int) -> float:
         return 0.0 if self.shared else self.comm_fixed + self.comm_per_row * rows

@@ -25,7 +25,9 @@ EXPORTS = (
     "aflex_workspace_bytes", "aflex_linear", "aflex_set_attn_ctas", "aflex_num_kernel_kinds",
     "aflex_kernel_name", "aflex_launch_count", "aflex_profile_enable", "aflex_profile_read",
     "aflex_trace_read", "aflex_attn_decode_static", "aflex_decoder_layers", "aflex_decoder_workspace_bytes",
-    "aflex_add_rmsnorm", "aflex_rope_append",
+    "aflex_add_rmsnorm", "aflex_rope_append", "aflex_eq2_layer_time", "aflex_curve_eval",
+    "aflex_pipeline_makespan", "aflex_plan_microbatches", "aflex_dvfs_window", "aflex_dvfs_decode_step",
+    "aflex_dvfs_prefill_pair",
 )
 
 
@@ -51,6 +53,28 @@ class DecoderDesc(ctypes.Structure):
     _fields_ = [("layer", LayerDesc), ("w_qkv", ctypes.c_void_p), ("w_ln_attn", ctypes.c_void_p),
                 ("w_ln_ffn", ctypes.c_void_p), ("w_q_norm", ctypes.c_void_p), ("w_k_norm", ctypes.c_void_p),
                 ("rms_eps", ctypes.c_float), ("rope_theta", ctypes.c_float)]
+
+
+class Curve(ctypes.Structure):
+    _fields_ = [("n", ctypes.c_int), ("x", ctypes.POINTER(ctypes.c_double)), ("y", ctypes.POINTER(ctypes.c_double))]
+
+
+class PipelineModel(ctypes.Structure):
+    _fields_ = [("attn_vs_tokens", Curve), ("attn_vs_rows", Curve), ("ffn_vs_rows", Curve),
+                ("comm_fixed", ctypes.c_double), ("comm_per_row", ctypes.c_double),
+                ("shared_memory_system", ctypes.c_int)]
+
+
+class DvfsParams(ctypes.Structure):
+    _fields_ = [("n_da", ctypes.c_int), ("n_df", ctypes.c_int), ("tau", ctypes.c_double),
+                ("delta_b", ctypes.c_double), ("window", ctypes.c_int), ("t_switch", ctypes.c_double)]
+
+
+class DvfsState(ctypes.Structure):
+    _fields_ = [("i_da", ctypes.c_int), ("i_df", ctypes.c_int), ("w", ctypes.c_int), ("b_last", ctypes.c_int)]
+
+
+DVFS_ESCALATED, DVFS_INFEASIBLE = 1, 2
 
 
 class AflexError(RuntimeError):
@@ -117,6 +141,23 @@ def load_library() -> ctypes.CDLL:
     lib.aflex_rope_append.restype = ci
     lib.aflex_rope_append.argtypes = [vp, ctypes.POINTER(AttnDesc), vp, ctypes.POINTER(KV), ci, vp, vp,
                                       ctypes.c_float, ctypes.c_float, vp, vp]
+    cd, dp, ip = ctypes.c_double, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_int32)
+    lib.aflex_eq2_layer_time.restype = cd
+    lib.aflex_eq2_layer_time.argtypes = [cd, cd, cd, ci]
+    lib.aflex_curve_eval.restype = cd
+    lib.aflex_curve_eval.argtypes = [ctypes.POINTER(Curve), cd]
+    lib.aflex_pipeline_makespan.restype = cd
+    lib.aflex_pipeline_makespan.argtypes = [ctypes.POINTER(PipelineModel), ip, ci, ci, ip, ci]
+    lib.aflex_plan_microbatches.restype = ci
+    lib.aflex_plan_microbatches.argtypes = [ctypes.POINTER(PipelineModel), ip, ci, ci, ctypes.POINTER(ci), ci, ci,
+                                            ctypes.POINTER(ci), ip, dp]
+    lib.aflex_dvfs_window.restype = ci
+    lib.aflex_dvfs_window.argtypes = [ci, cd, cd, cd]
+    lib.aflex_dvfs_decode_step.restype = ci
+    lib.aflex_dvfs_decode_step.argtypes = [ctypes.POINTER(DvfsParams), dp, dp, ci, cd, ctypes.POINTER(DvfsState)]
+    lib.aflex_dvfs_prefill_pair.restype = ci
+    lib.aflex_dvfs_prefill_pair.argtypes = [ci, ci, dp, dp, cd, cd, ci, ci, ci, ci, ctypes.POINTER(ci),
+                                            ctypes.POINTER(ci)]
     lib.aflex_attn_decode_static.restype = ci
     lib.aflex_attn_decode_static.argtypes = [ctypes.POINTER(AttnDesc), vp, ctypes.POINTER(KV), ci, vp, vp, vp]
     _lib = lib
@@ -196,6 +237,81 @@ def attn_decode_static(desc: AttnDesc, q: torch.Tensor, kv: KV, out: torch.Tenso
                                       _stream(stream))
     if st != OK:
         raise AflexError(st, lib.aflex_status_string(st).decode(), _STATIC_ERRORS.get(st, "unknown error"))
+
+
+# --------------------------------------------------------------------------- host-side decisions
+def _dbl(values):
+    return (ctypes.c_double * len(values))(*[float(v) for v in values])
+
+
+def curve(xs, ys) -> Curve:
+    assert len(xs) == len(ys) >= 1
+    ax, ay = _dbl(xs), _dbl(ys)
+    c = Curve(len(xs), ax, ay)
+    c._keep = (ax, ay)
+    return c
+
+
+def pipeline_model(attn_vs_tokens, attn_vs_rows, ffn_vs_rows, comm_fixed=0.0, comm_per_row=0.0,
+                   shared_memory_system=False) -> PipelineModel:
+    """Each curve is an (xs, ys) pair of profiled points."""
+    cs = [curve(*attn_vs_tokens), curve(*attn_vs_rows), curve(*ffn_vs_rows)]
+    m = PipelineModel(cs[0], cs[1], cs[2], comm_fixed, comm_per_row, 1 if shared_memory_system else 0)
+    m._keep = cs
+    return m
+
+
+def eq2_layer_time(t_a: float, t_f: float, t_comm: float, depth: int) -> float:
+    return float(load_library().aflex_eq2_layer_time(t_a, t_f, t_comm, depth))
+
+
+def curve_eval(c: Curve, x: float) -> float:
+    return float(load_library().aflex_curve_eval(ctypes.byref(c), x))
+
+
+def pipeline_makespan(model: PipelineModel, seq_lens, offsets, layers: int) -> float:
+    lens = (ctypes.c_int32 * len(seq_lens))(*[int(v) for v in seq_lens])
+    offs = (ctypes.c_int32 * len(offsets))(*[int(v) for v in offsets])
+    return float(load_library().aflex_pipeline_makespan(ctypes.byref(model), lens, len(seq_lens), len(offsets) - 1,
+                                                        offs, layers))
+
+
+def plan_microbatches(model: PipelineModel, seq_lens, layers: int, depths, granularity: int = 1):
+    """-> (depth, offsets, predicted time).  Raises AflexError on a non-OK status."""
+    lib = load_library()
+    lens = (ctypes.c_int32 * len(seq_lens))(*[int(v) for v in seq_lens])
+    ds = (ctypes.c_int * len(depths))(*[int(v) for v in depths])
+    best = ctypes.c_int(0)
+    offs = (ctypes.c_int32 * (max(depths) + 1))()
+    pred = ctypes.c_double(0.0)
+    st = lib.aflex_plan_microbatches(ctypes.byref(model), lens, len(seq_lens), layers, ds, len(depths), granularity,
+                                     ctypes.byref(best), offs, ctypes.byref(pred))
+    if st != OK:
+        raise AflexError(st, lib.aflex_status_string(st).decode(), "aflex_plan_microbatches")
+    return best.value, list(offs[:best.value + 1]), pred.value
+
+
+def dvfs_window(w_min: int, kappa: float, t_switch: float, t_iter: float) -> int:
+    return int(load_library().aflex_dvfs_window(w_min, kappa, t_switch, t_iter))
+
+
+def dvfs_decode_step(params: DvfsParams, t_hat, e_hat, batch_now: int, t_iter: float, state: DvfsState) -> int:
+    """t_hat / e_hat: nested [n_da][n_df] lists.  Updates `state` in place; returns the library's code."""
+    flat_t = _dbl([v for row in t_hat for v in row])
+    flat_e = _dbl([v for row in e_hat for v in row])
+    return int(load_library().aflex_dvfs_decode_step(ctypes.byref(params), flat_t, flat_e, batch_now, t_iter,
+                                                     ctypes.byref(state)))
+
+
+def dvfs_prefill_pair(t_hat, e_hat, budget: float, t_switch: float, current, base):
+    """-> ((pa, pf), flags)."""
+    flat_t = _dbl([v for row in t_hat for v in row])
+    flat_e = _dbl([v for row in e_hat for v in row])
+    pa, pf = ctypes.c_int(0), ctypes.c_int(0)
+    flags = load_library().aflex_dvfs_prefill_pair(len(t_hat), len(t_hat[0]), flat_t, flat_e, budget, t_switch,
+                                                   current[0], current[1], base[0], base[1], ctypes.byref(pa),
+                                                   ctypes.byref(pf))
+    return (pa.value, pf.value), int(flags)
 
 
 class Context:
