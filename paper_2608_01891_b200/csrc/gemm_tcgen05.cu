@@ -555,8 +555,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
 // ----------------------------------------------------------------------------------------- host side
 static int round_up(int a, int b) { return (a + b - 1) / b * b; }
 
+// Token-tile width: the fewest tiles of at most 256 rows, all of (nearly) the same width, so that
+// e.g. 384 rows become 192 + 192 rather than 256 + 128.
 static int pick_n_tile(int rows_max) {
-    int n = round_up(rows_max < 16 ? 16 : rows_max, 16);
+    const int rows = rows_max < 16 ? 16 : rows_max;
+    const int tiles = (rows + 255) / 256;
+    const int n = round_up((rows + tiles - 1) / tiles, 16);
     return n > 256 ? 256 : n;
 }
 
@@ -589,6 +593,11 @@ static bool make_config(int mode, int T, int N, int K, int rows_max, int E, int 
     // in TMEM; a hot expert with more rows becomes two adjacent tiles whose weight tiles are read by
     // neighbouring CTAs at the same time (the second read is an L2 hit).
     if (E > 0 && p.n_tile > 128) p.n_tile = 128;
+    {
+        static int cap = -1;
+        if (cap < 0) { const char* e = getenv("AFLEX_GEMM_NTILE_CAP"); cap = e ? atoi(e) : 0; }
+        if (cap >= 16 && p.n_tile > cap) p.n_tile = cap / 16 * 16;
+    }
     p.m_tiles = (N + kBlockM - 1) / kBlockM;
     p.n_tiles = (T + p.n_tile - 1) / p.n_tile;
     p.kblocks = (K + kBlockK - 1) / kBlockK;

@@ -109,7 +109,7 @@ def test_attention_custom_scale_and_zero_query(ctx):
 
 # ------------------------------------------------------------------------------- GEMMs / dense FFN
 @pytest.mark.parametrize("T,K,N", [(1, 64, 128), (4, 512, 512), (32, 1376, 512), (33, 520, 264), (130, 8192, 640),
-                                   (300, 256, 136)])
+                                   (300, 256, 136), (384, 320, 264), (700, 128, 136)])
 def test_linear_matches_oracle(ctx, T, K, N):
     x, w = rand_bf16((T, K), 1.0, 1), rand_bf16((N, K), 0.05, 2)
     y = torch.full((T, N), float("nan"), dtype=torch.bfloat16, device=DEV)
@@ -119,7 +119,7 @@ def test_linear_matches_oracle(ctx, T, K, N):
     assert row_rel_err(f64(y), want) <= TOL_FFN
 
 
-@pytest.mark.parametrize("T", [1, 3, 4, 32, 33, 300])
+@pytest.mark.parametrize("T", [1, 3, 4, 32, 33, 300, 384, 530])
 def test_dense_ffn_config1_shapes(ctx, T):
     cfg = IN.CONFIGS[1]
     x = IN.make_x(cfg, tokens=T)
