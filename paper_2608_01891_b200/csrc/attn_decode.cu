@@ -63,6 +63,7 @@ struct AttnParams {
     int* ticket;           // [2]: next dynamic chunk, CTAs finished; zero on entry and on exit (unused if dyn_pct == 0)
     int dyn_pct;           // percent of the unit list handed out dynamically (0 = static shares only)
     int dyn_chunks;        // target number of dynamic chunks per CTA
+    int kv_policy;         // 0: evict-first KV loads, 1: normal priority (tuning)
     int piece_cost;        // list positions charged per item start (balances the fixed cost of a piece)
     int* status;
     unsigned long long* trace;
@@ -262,7 +263,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             const int idx = (w.u - w.cost) * kPagesPerStage + pg;
             return (op_lane && idx * kPage < w.len) ? p.page_table[(size_t)w.b * p.max_pages + idx] : 0;
         };
-        const uint64_t pol_kv = policy_evict_first();    // KV is read once: do not let it push reusable lines out of L2
+        const uint64_t pol_kv = p.kv_policy == 1 ? policy_evict_normal() : policy_evict_first();    // KV is read once: do not let it push reusable lines out of L2
         int s = 0;
         uint32_t ph = 0;
         int r = 0;                       // ranges published so far
@@ -709,6 +710,7 @@ static aflex_status attn_launch_t(aflex_ctx* ctx, const aflex_attn_desc* d, cons
     p.dyn_pct = attn_dyn_pct();
     p.dyn_chunks = attn_dyn_chunks();
     p.piece_cost = attn_piece_cost();
+    { static int v = -1; if (v < 0) { const char* e = getenv("AFLEX_ATTN_KVPOL"); v = e ? atoi(e) : 0; } p.kv_policy = v; }
     p.status = ctx->dev_status;
     p.out = reinterpret_cast<__nv_bfloat16*>(out);
     p.lse = lse;
@@ -819,6 +821,7 @@ static aflex_status attn_static_launch(StaticDeviceState& stt, const aflex_attn_
     p.ticket = nullptr;     // static shares only: the fixed scratch has two slots per CTA
     p.dyn_pct = 0;
     p.dyn_chunks = 1;
+    p.kv_policy = 0;
     p.piece_cost = 0;
     p.trace = nullptr;
 
