@@ -199,8 +199,11 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         prefetch_tmap(&tmap_k);
         prefetch_tmap(&tmap_v);
     }
-    pdl_wait();   // q, the page table and the lengths may come from the preceding kernel
-    if (tr && threadIdx.x == 0) tr[2] = global_timer_ns();
+    // The lengths and the page table are inputs of the step, never written by a kernel of this library,
+    // so the plan (prefix scan, this CTA's share, its first page ids) is made while the preceding kernel
+    // is still draining.  q and the KV cache may come from that kernel (the K/V append), and the partial
+    // slots, counters and ticket may still be in use by an earlier attention launch: everything that
+    // touches those waits for the grid dependency (pdl_wait below, per role).
 
     // ---- block-wide exclusive prefix over ceil(len/64): thread t owns sequences [t*per_thread, ...)
     const int per_thread = (p.batch + kAttnThreads - 1) / kAttnThreads;
@@ -273,6 +276,19 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         int rid = cta;
         if (cta < sp.Ge1) { x0 = share_begin(sp.U1, cta, sp.Ge1); x1 = share_begin(sp.U1, cta + 1, sp.Ge1); }
         int next_ticket = -1;
+        // the static share's start, located before the grid dependency resolves
+        AttnRange rg0;
+        rg0.x0 = x0; rg0.x1 = x1; rg0.rid = rid; rg0.b = 0; rg0.prefix = 0;
+        int pid0 = 0;
+        if (x1 > x0) {
+            locate(x0, rg0.b, rg0.prefix);
+            Walker w0;
+            w0.init(p, rg0);
+            while (!w0.done() && w0.u < w0.cost) w0.advance(1);
+            pid0 = w0.done() ? 0 : page_id(w0);          // also warms the page-table line
+        }
+        pdl_wait();
+        bool first_range = true;
         while (true) {
             if (sp.n2 > 0) {             // claim the chunk after this range now: the round trip hides behind the range
                 if (lane == 0) next_ticket = atomicAdd(&p.ticket[0], 1);
@@ -280,8 +296,8 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             }
             if (x1 > x0) {
                 AttnRange rg;
-                rg.x0 = x0; rg.x1 = x1; rg.rid = rid;
-                locate(x0, rg.b, rg.prefix);
+                if (first_range) { rg = rg0; }
+                else { rg.x0 = x0; rg.x1 = x1; rg.rid = rid; locate(x0, rg.b, rg.prefix); }
                 Walker wk;
                 wk.init(p, rg);
                 while (!wk.done() && wk.u < wk.cost) wk.advance(1);     // positions without work
@@ -291,7 +307,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                     if (lane == 0) { sh->rng[r % kRangeRing] = rg; mbar_arrive(&sh->rng_ready[r % kRangeRing]); }
                     ++r;
                 }
-                int pid = wk.done() ? 0 : page_id(wk);
+                int pid = wk.done() ? 0 : (first_range ? pid0 : page_id(wk));
                 while (!wk.done()) {
                     const int g = wk.g, u = wk.u - wk.cost, len = wk.len;
                     wk.advance(1);
@@ -318,6 +334,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                     if (++s == kAttnStages) { s = 0; ph ^= 1; }
                 }
             }
+            first_range = false;
             if (aborted || sp.n2 == 0 || next_ticket >= sp.n2) break;
             x0 = sp.U1 + (long long)next_ticket * sp.K2;
             x1 = min(sp.U, x0 + sp.K2);
@@ -337,6 +354,8 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         }
     } else {
         // ------------------------------------------------------------------ consumer warps
+        pdl_wait();   // q, the partial slots and the counters
+        if (tr && threadIdx.x == 0) tr[2] = global_timer_ns();
         const int mi = lane >> 3, r8 = lane & 7;
         const int h0 = 2 * (lane & 3);          // this lane's two heads of the group: h0, h0 + 1
         int s = 0;
