@@ -287,13 +287,23 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             while (!w0.done() && w0.u < w0.cost) w0.advance(1);
             pid0 = w0.done() ? 0 : page_id(w0);          // also warms the page-table line
         }
-        pdl_wait();
+        // KV loads do not wait for the grid dependency: the only kernel of this library that writes the
+        // cache (the K/V append) does not release its dependents early, so whatever precedes this launch
+        // in the stream has left the cache final.  The ticket, like everything else in global memory that
+        // an earlier attention launch may still be using, is touched only after pdl_wait.
+        bool waited = false;
+        auto claim = [&]() {
+            if (!waited) { pdl_wait(); waited = true; }
+            if (lane == 0) next_ticket = atomicAdd(&p.ticket[0], 1);
+            next_ticket = __shfl_sync(0xffffffffu, next_ticket, 0);
+        };
         bool first_range = true;
         while (true) {
-            if (sp.n2 > 0) {             // claim the chunk after this range now: the round trip hides behind the range
-                if (lane == 0) next_ticket = atomicAdd(&p.ticket[0], 1);
-                next_ticket = __shfl_sync(0xffffffffu, next_ticket, 0);
-            }
+            // claim the chunk after this range while the range streams (the round trip hides behind it);
+            // in the first range only once the ring has been filled
+            bool claimed = sp.n2 == 0;
+            if (!claimed && waited) { claim(); claimed = true; }
+            int issued = 0;
             if (x1 > x0) {
                 AttnRange rg;
                 if (first_range) { rg = rg0; }
@@ -313,6 +323,8 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                     wk.advance(1);
                     while (!wk.done() && wk.u < wk.cost) wk.advance(1);
                     const int pid_next = wk.done() ? 0 : page_id(wk);   // one unit ahead of the ring
+                    if (!claimed && issued >= kAttnStages) { claim(); claimed = true; }
+                    ++issued;
                     bool ok = mbar_wait(&sh->empty[s], ph ^ 1);
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok || sh->abort) {
@@ -335,6 +347,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                 }
             }
             first_range = false;
+            if (!claimed && !aborted) { claim(); claimed = true; }
             if (aborted || sp.n2 == 0 || next_ticket >= sp.n2) break;
             x0 = sp.U1 + (long long)next_ticket * sp.K2;
             x1 = min(sp.U, x0 + sp.K2);
@@ -348,6 +361,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             mbar_arrive(&sh->rng_ready[r % kRangeRing]);
             if (sp.n2 > 0) {
                 // last CTA out resets the ticket counters (every CTA has made its final claim by now)
+                if (!waited) pdl_wait();
                 __threadfence();
                 if (atomicAdd(&p.ticket[1], 1) == (int)gridDim.x - 1) { p.ticket[0] = 0; p.ticket[1] = 0; }
             }

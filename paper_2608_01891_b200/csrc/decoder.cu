@@ -116,7 +116,9 @@ struct RopeParams {
 // double: at positions of 10^4 and more an fp32 angle would already be off by 10^-3 rad.
 constexpr int kRopeWarps = 4;
 __global__ void __launch_bounds__(kRopeWarps * 32) rope_append_kernel(const RopeParams p) {
-    pdl_launch_dependents();
+    // No early release of the dependents here: the attention kernel streams the KV cache without waiting
+    // for the grid dependency, which is sound only if the kernel that writes the cache has finished (and
+    // flushed) before anything later in the stream starts.
     pdl_wait();
     const int lane = threadIdx.x & 31;
     const int head = blockIdx.y * kRopeWarps + (threadIdx.x >> 5);
