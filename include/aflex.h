@@ -29,6 +29,13 @@
  *    device and must be used by one host thread at a time.  Calls that use the
  *    same ctx must be stream-ordered with respect to each other (they share the
  *    workspace); aflex_layer_step orders its own internal streams.
+ *  - Kernels are launched with programmatic stream serialization and read their
+ *    INPUT tensors (q, KV cache, page table, lengths, weights) before the grid
+ *    dependency resolves.  This is invisible to ordinary callers (a preceding
+ *    kernel, copy or event wait in the stream completes first, as usual); only a
+ *    caller's own kernel that releases its dependents early
+ *    (cudaTriggerProgrammaticLaunchCompletion) must not be the producer of those
+ *    inputs.  Outputs and scratch are touched only after the dependency resolves.
  *  - Device-side waits are bounded: if one expires the kernel records
  *    AFLEX_ERR_TIMEOUT in the ctx status word and exits cleanly; read it with
  *    aflex_get_device_status.

@@ -64,6 +64,7 @@ struct AttnParams {
     int dyn_pct;           // percent of the unit list handed out dynamically (0 = static shares only)
     int dyn_chunks;        // target number of dynamic chunks per CTA
     int kv_policy;         // 0: evict-first KV loads, 1: normal priority (tuning)
+    int dyn_min;           // smallest chunk (units) for which the dynamic tail is used
     int piece_cost;        // list positions charged per item start (balances the fixed cost of a piece)
     int* status;
     unsigned long long* trace;
@@ -131,12 +132,12 @@ struct Walker {
 struct AttnSplit {
     long long U, U1;
     int Ge1, K2, n2;
-    __device__ AttnSplit(long long U_, int grid, int dyn_pct, int dyn_chunks) {
+    __device__ AttnSplit(long long U_, int grid, int dyn_pct, int dyn_chunks, int dyn_min = 12) {
         U = U_;
         long long U2 = dyn_pct > 0 ? U * dyn_pct / 100 : 0;
         // A chunk costs a fixed ~2-3 us (claim, hand-over, an extra partial piece to publish and merge):
         // chunks below ~12 units (~0.4 MB at D = 128) do not pay, so small launches stay purely static.
-        if (U2 > 0 && U2 / ((long long)dyn_chunks * grid) < 12) U2 = 0;
+        if (U2 > 0 && U2 / ((long long)dyn_chunks * grid) < dyn_min) U2 = 0;
         if (U2 > 0) {
             long long k = (U2 + (long long)dyn_chunks * grid - 1) / ((long long)dyn_chunks * grid);
             K2 = (int)(k < 2 ? 2 : (k > 64 ? 64 : k));
@@ -233,7 +234,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     }
     const long long U = sh->rng[0].x0 * (long long)p.Hkv;
     __syncthreads();
-    const AttnSplit sp(U, (int)gridDim.x, p.dyn_pct, p.dyn_chunks);
+    const AttnSplit sp(U, (int)gridDim.x, p.dyn_pct, p.dyn_chunks, p.dyn_min);
     if (tr && threadIdx.x == 0) tr[1] = global_timer_ns();            // prefix ready
 
     // Sequence that contains unit position x (cooperative over the 32 lanes of one warp).
@@ -368,8 +369,10 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         }
     } else {
         // ------------------------------------------------------------------ consumer warps
-        pdl_wait();   // q, the partial slots and the counters
-        if (tr && threadIdx.x == 0) tr[2] = global_timer_ns();
+        // q is final when this kernel starts (an input of the step, or written by the K/V append kernel,
+        // which does not release its dependents early), so pages are processed at once; the grid
+        // dependency is awaited before this warp's first write to global memory.
+        bool dep_ok = false;
         const int mi = lane >> 3, r8 = lane & 7;
         const int h0 = 2 * (lane & 3);          // this lane's two heads of the group: h0, h0 + 1
         int s = 0;
@@ -539,6 +542,11 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                     o[mt][2] = o[mt][2] * a0 + src[(mt * 4 + 2) * 32] * b0;
                     o[mt][3] = o[mt][3] * a1 + src[(mt * 4 + 3) * 32] * b1;
                 }
+            }
+            if (!dep_ok) {
+                pdl_wait();   // output rows, partial slots and counters may still be in use by earlier kernels
+                dep_ok = true;
+                if (tr && threadIdx.x == 0) tr[2] = global_timer_ns();
             }
             const int dr = lane >> 2;
             const size_t hq0 = (size_t)g * p.G + h0;
@@ -743,6 +751,7 @@ static aflex_status attn_launch_t(aflex_ctx* ctx, const aflex_attn_desc* d, cons
     p.dyn_pct = attn_dyn_pct();
     p.dyn_chunks = attn_dyn_chunks();
     p.piece_cost = attn_piece_cost();
+    { static int v = -1; if (v < 0) { const char* e = getenv("AFLEX_ATTN_DYN_MIN"); v = e ? atoi(e) : 12; if (v < 1) v = 1; } p.dyn_min = v; }
     { static int v = -1; if (v < 0) { const char* e = getenv("AFLEX_ATTN_KVPOL"); v = e ? atoi(e) : 0; } p.kv_policy = v; }
     p.status = ctx->dev_status;
     p.out = reinterpret_cast<__nv_bfloat16*>(out);
@@ -855,6 +864,7 @@ static aflex_status attn_static_launch(StaticDeviceState& stt, const aflex_attn_
     p.dyn_pct = 0;
     p.dyn_chunks = 1;
     p.kv_policy = 0;
+    p.dyn_min = 12;
     p.piece_cost = 0;
     p.trace = nullptr;
 
