@@ -223,6 +223,10 @@ def run_decoder_chain(args, cfg, local_rank, device, peaks):
     descs, kvs, keep = [], [], []
     for l in range(L):
         w = IN.make_decoder_weights(cfg, l, device=device)
+        if args.af_pair and args.ffn_device >= 0 and args.ffn_device != local_rank:
+            fdev = f"cuda:{args.ffn_device}"                 # role-specific weights: the FFN's live on the FFN GPU
+            w.gate, w.up, w.down, w.ln_ffn = w.gate.to(fdev), w.up.to(fdev), w.down.to(fdev), w.ln_ffn.to(fdev)
+            w.router = None if w.router is None else w.router.to(fdev)
         layer = AF.layer_desc(attn, cfg.hidden, cfg.inter, w.o, w.gate, w.up, w.down, cfg.num_experts, cfg.top_k, w.router)
         descs.append(AF.decoder_desc(layer, w.qkv, w.ln_attn, w.ln_ffn, w.q_norm, w.k_norm, cfg.rms_eps, cfg.rope_theta))
         kc, vc = (kvh.k_cache, kvh.v_cache) if l == 0 else (kvh.k_cache.clone(), kvh.v_cache.clone())
@@ -230,8 +234,19 @@ def run_decoder_chain(args, cfg, local_rank, device, peaks):
         keep.append((w, kc, vc))
     x = IN.make_hidden(cfg, device=device)
     y = torch.empty_like(x)
-    ctx = AF.Context(local_rank, max(AF.decoder_workspace_bytes(d, cfg.batch) for d in descs))
     stream = torch.cuda.current_stream()
+    if args.af_pair:
+        # Attention side on this GPU, FFN side on --ffn-device (the same GPU by default: the hand-over copies are
+        # then device-local and the two sides share one memory system)
+        ctx = AF.Context(local_rank, max(AF.af_workspace_bytes(d, cfg.batch, False) for d in descs))
+        ctx_f = AF.Context(args.ffn_device if args.ffn_device >= 0 else local_rank,
+                           max(AF.af_workspace_bytes(d, cfg.batch, True) for d in descs))
+        torch.cuda.set_device(local_rank)
+        run = lambda M: AF.af_decoder_layers(ctx, ctx_f, descs, kvs, x, y, M, None, stream)
+    else:
+        ctx = AF.Context(local_rank, max(AF.decoder_workspace_bytes(d, cfg.batch) for d in descs))
+        ctx_f = None
+        run = lambda M: ctx.decoder_layers(descs, kvs, x, y, M, None, stream)
     n_qkv = (cfg.num_q_heads + 2 * cfg.num_kv_heads) * cfg.head_dim
     extra = 2.0 * n_qkv * cfg.hidden                      # W_qkv bytes on top of the hot path's
     sampler = ClockSampler(local_rank)
@@ -239,12 +254,12 @@ def run_decoder_chain(args, cfg, local_rank, device, peaks):
     rows = []
     for M in cfg.microbatch_depths:
         for _ in range(max(3, args.warmup)):
-            ctx.decoder_layers(descs, kvs, x, y, M, None, stream)
+            run(M)
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
         for _ in range(args.steps):
-            ctx.decoder_layers(descs, kvs, x, y, M, None, stream)
+            run(M)
         e1.record(stream)
         torch.cuda.synchronize()
         us_layer = 1e3 * e0.elapsed_time(e1) / args.steps / L
@@ -254,17 +269,21 @@ def run_decoder_chain(args, cfg, local_rank, device, peaks):
                      "frac_hbm": round(byts / us_layer / 1e3 / peaks["hbm_gbs"], 4)})
     ctx.profile_enable(True)
     for _ in range(5):
-        ctx.decoder_layers(descs, kvs, x, y, 1, None, stream)
+        run(1)
     prof = ctx.profile_read()
     ctx.profile_enable(False)
-    assert ctx.device_status() == AF.OK
+    assert ctx.device_status() == AF.OK and (ctx_f is None or ctx_f.device_status() == AF.OK)
     line = {"metric": "whole decoder layer, chained: tokens/s per layer", "unit": "tokens/s", "dtype": "bf16",
-            "data": "synthetic", "config": {"workload": f"config {cfg.cfg_id}: {cfg.name}, {L} chained decoder layers",
+            "data": "synthetic", "config": {"workload": f"config {cfg.cfg_id}: {cfg.name}, {L} chained decoder layers"
+                                            + (f", A/F pair (attention GPU {local_rank}, FFN GPU "
+                                               f"{args.ffn_device if args.ffn_device >= 0 else local_rank})" if args.af_pair else ""),
                                             "batch": cfg.batch, "l2": "per-layer weights + KV larger than L2, no flush"},
             "peaks": peaks, "clocks": sampler.stop(), "depths": rows,
             "kernel_us_event_pairs_M1": {k: round(1e3 * v[0] / v[1], 1) for k, v in prof.items()}}
     print(json.dumps(line), flush=True)
     ctx.close()
+    if ctx_f is not None:
+        ctx_f.close()
 
 
 def dataclasses_replace_dense(cfg):
@@ -360,6 +379,11 @@ def main():
     ap.add_argument("--decoder-layers", type=int, default=0,
                     help="instead of the layer step: chain this many whole decoder layers (aflex_decoder_layers) at "
                          "every microbatch depth of the configuration; prints one JSON line")
+    ap.add_argument("--af-pair", action="store_true",
+                    help="with --decoder-layers: run the Attention side and the FFN side as an A/F pair "
+                         "(aflex_af_decoder_layers), hidden states handed over by peer copies")
+    ap.add_argument("--ffn-device", type=int, default=-1,
+                    help="with --af-pair: CUDA device of the FFN side (default: the same GPU as the attention side)")
     ap.add_argument("--energy", action="store_true",
                     help="also read the NVML energy counter around a >= 2 s loop of the step (default clocks)")
     args = ap.parse_args()

@@ -330,6 +330,35 @@ AFLEX_API aflex_status aflex_decoder_layers(aflex_ctx* ctx, const aflex_decoder_
 /* Workspace bytes that suffice for aflex_decoder_layers on this layer shape.  Pure host computation. */
 AFLEX_API size_t aflex_decoder_workspace_bytes(const aflex_decoder_desc* layer, int max_batch);
 
+/* ---- A/F pair: the Attention side on one GPU, the FFN side on another -----------------------
+ *
+ * The paper's data plane (Section 4.3, "Placement-aware A/F Data Path"; Section 5: within a node
+ * the hidden states move by peer copies over NVLink): at every A/F boundary the Attention group
+ * sends one [rows][H] hidden-state tensor to the FFN group, which returns one [rows][H] tensor for
+ * the next layer.  Here one process drives both GPUs:
+ *
+ *   A_{l,i} on ctx_a's device:  h1 = r + attention-side(r)      (as aflex_decoder_layers)
+ *                               peer copy h1 rows -> ctx_f's device, event
+ *   F_{l,i} on ctx_f's device:  out = h1 + FFN(rmsnorm(h1, w_ln_ffn))
+ *                               peer copy out rows -> ctx_a's device, event
+ *   A_{l+1,i} starts when the rows of microbatch i are back (interleaved schedule, Eq. 2 with a
+ *   real t_comm).  The copies are plain cudaMemcpyPeerAsync calls on the producing side's stream:
+ *   the payload is in the consumer's own memory before any of its kernels reads it.
+ *
+ * Placement: w_qkv, w_ln_attn, w_q_norm, w_k_norm, layer.w_o, the KV caches, x_in and x_out live on
+ * ctx_a's device; w_ln_ffn, layer.w_gate / w_up / w_down / w_router on ctx_f's device ("each
+ * worker loads only its role-specific weights", Section 5).  The two contexts may be on the same
+ * device (then the copies are device-local); both must outlive the call's work.  `stream` belongs
+ * to ctx_a's device and is joined on entry and exit.  Results equal aflex_decoder_layers up to
+ * one extra bf16 rounding of the returned hidden states per layer.
+ */
+AFLEX_API aflex_status aflex_af_decoder_layers(aflex_ctx* ctx_a, aflex_ctx* ctx_f, const aflex_decoder_desc* layers,
+                                               const aflex_kv* kvs, int num_layers, const void* x_in, int batch,
+                                               int microbatch_depth, const int32_t* mb_offsets, void* x_out,
+                                               void* stream);
+/* Workspace bytes each side needs for aflex_af_decoder_layers (pure host computation). */
+AFLEX_API size_t aflex_af_workspace_bytes(const aflex_decoder_desc* layer, int max_batch, int ffn_side);
+
 /*
  * The two small operators of the chain on their own (testing, benchmarking).
  * aflex_add_rmsnorm: s = res (+ add when add != NULL), bf16 [T][H] each, summed in fp32;

@@ -25,7 +25,8 @@ EXPORTS = (
     "aflex_workspace_bytes", "aflex_linear", "aflex_set_attn_ctas", "aflex_num_kernel_kinds",
     "aflex_kernel_name", "aflex_launch_count", "aflex_profile_enable", "aflex_profile_read",
     "aflex_trace_read", "aflex_attn_decode_static", "aflex_decoder_layers", "aflex_decoder_workspace_bytes",
-    "aflex_add_rmsnorm", "aflex_rope_append", "aflex_eq2_layer_time", "aflex_curve_eval",
+    "aflex_add_rmsnorm", "aflex_rope_append", "aflex_af_decoder_layers", "aflex_af_workspace_bytes",
+    "aflex_eq2_layer_time", "aflex_curve_eval",
     "aflex_pipeline_makespan", "aflex_plan_microbatches", "aflex_dvfs_window", "aflex_dvfs_decode_step",
     "aflex_dvfs_prefill_pair",
 )
@@ -136,6 +137,11 @@ def load_library() -> ctypes.CDLL:
                                          ctypes.POINTER(ctypes.c_int32), vp, vp]
     lib.aflex_decoder_workspace_bytes.restype = cs
     lib.aflex_decoder_workspace_bytes.argtypes = [ctypes.POINTER(DecoderDesc), ci]
+    lib.aflex_af_decoder_layers.restype = ci
+    lib.aflex_af_decoder_layers.argtypes = [vp, vp, ctypes.POINTER(DecoderDesc), ctypes.POINTER(KV), ci, vp, ci, ci,
+                                            ctypes.POINTER(ctypes.c_int32), vp, vp]
+    lib.aflex_af_workspace_bytes.restype = cs
+    lib.aflex_af_workspace_bytes.argtypes = [ctypes.POINTER(DecoderDesc), ci, ci]
     lib.aflex_add_rmsnorm.restype = ci
     lib.aflex_add_rmsnorm.argtypes = [vp, vp, vp, vp, ci, ci, ctypes.c_float, vp, vp, vp]
     lib.aflex_rope_append.restype = ci
@@ -212,6 +218,25 @@ def decoder_desc(layer: LayerDesc, w_qkv, w_ln_attn, w_ln_ffn, w_q_norm, w_k_nor
 
 def decoder_workspace_bytes(layer: DecoderDesc, max_batch: int) -> int:
     return int(load_library().aflex_decoder_workspace_bytes(ctypes.byref(layer), max_batch))
+
+
+def af_workspace_bytes(layer: DecoderDesc, max_batch: int, ffn_side: bool) -> int:
+    return int(load_library().aflex_af_workspace_bytes(ctypes.byref(layer), max_batch, 1 if ffn_side else 0))
+
+
+def af_decoder_layers(ctx_a: "Context", ctx_f: "Context", layers: Sequence[DecoderDesc], kvs: Sequence[KV], x_in, x_out,
+                      microbatch_depth: int = 1, mb_offsets: Optional[Sequence[int]] = None, stream=None) -> None:
+    """Chained decoder layers with the Attention side on ctx_a's GPU and the FFN side on ctx_f's (see the header
+    for which weights live where).  `stream` is a stream of ctx_a's device (default: its current stream)."""
+    assert len(layers) == len(kvs) and len(layers) >= 1
+    offs = None
+    if mb_offsets is not None:
+        offs = (ctypes.c_int32 * len(mb_offsets))(*[int(v) for v in mb_offsets])
+    la = (DecoderDesc * len(layers))(*layers)
+    ka = (KV * len(kvs))(*kvs)
+    st = stream.cuda_stream if stream is not None else torch.cuda.current_stream(x_in.device).cuda_stream
+    ctx_a._check(ctx_a._lib.aflex_af_decoder_layers(ctx_a._h, ctx_f._h, la, ka, len(layers), _ptr(x_in), x_in.shape[0],
+                                                    microbatch_depth, offs, _ptr(x_out), st))
 
 
 def workspace_bytes(layer: LayerDesc, max_batch: int, max_pages_per_seq: int) -> int:

@@ -653,21 +653,19 @@ aflex_status aflex_rope_append(aflex_ctx* ctx, const aflex_attn_desc* desc, cons
                               reinterpret_cast<cudaStream_t>(stream));
 }
 
-aflex_status aflex_decoder_layers(aflex_ctx* ctx, const aflex_decoder_desc* layers, const aflex_kv* kvs, int num_layers,
-                                  const void* x_in, int batch, int M, const int32_t* mb_offsets, void* x_out,
-                                  void* stream) {
-    if (!ctx) return AFLEX_ERR_INVALID_ARG;
+namespace {
+// Argument checks shared by the single-GPU chain and the A/F pair.  Errors are recorded on ctx.
+aflex_status validate_decoder_args(aflex_ctx* ctx, const aflex_decoder_desc* layers, const aflex_kv* kvs, int num_layers,
+                                   const void* x_in, int batch, const void* x_out) {
     if (!layers || !kvs || !x_in || !x_out || num_layers < 1)
         return set_error(ctx, AFLEX_ERR_INVALID_ARG, "decoder layers: null argument or num_layers < 1");
     if (!aligned16(x_in) || !aligned16(x_out))
         return set_error(ctx, AFLEX_ERR_INVALID_ARG, "decoder layers: pointers must be 16-byte aligned");
     const int H = layers[0].layer.hidden;
-    aflex_status s;
-    size_t need = 0;
     for (int l = 0; l < num_layers; ++l) {
         const aflex_decoder_desc* d = &layers[l];
         const aflex_layer_desc* L = &d->layer;
-        s = validate_attn(ctx, &L->attn, x_in, &kvs[l], batch, x_out);
+        aflex_status s = validate_attn(ctx, &L->attn, x_in, &kvs[l], batch, x_out);
         if (s != AFLEX_OK) return s;
         if (L->hidden != H) return set_error(ctx, AFLEX_ERR_INVALID_ARG, "decoder layers: layer %d has another hidden size", l);
         if (!d->w_qkv || !d->w_ln_attn || !d->w_ln_ffn || !L->w_o || !L->w_gate || !L->w_up || !L->w_down)
@@ -683,24 +681,45 @@ aflex_status aflex_decoder_layers(aflex_ctx* ctx, const aflex_decoder_desc* laye
             if (s == AFLEX_OK && !L->w_router) s = set_error(ctx, AFLEX_ERR_INVALID_ARG, "decoder layers: MoE layer %d needs w_router", l);
         }
         if (s != AFLEX_OK) return s;
-        const DecoderWs w = decoder_ws(d, batch, attn_workspace_bytes(&L->attn, attn_grid(ctx)), ctx->num_sms);
-        if (w.total > need) need = w.total;
     }
-    if (need > ctx->ws_bytes)
-        return set_error(ctx, AFLEX_ERR_WORKSPACE, "decoder layers: need %zu workspace bytes, have %zu", need, ctx->ws_bytes);
+    return AFLEX_OK;
+}
+
+// Microbatch offsets: the caller's (validated) or the near-equal split.
+aflex_status make_offsets(aflex_ctx* ctx, int batch, int M, const int32_t* mb_offsets, int32_t* offs) {
     if (M < 1 || M > batch || M > kMaxMicrobatches)
-        return set_error(ctx, AFLEX_ERR_INVALID_ARG, "decoder layers: microbatch depth %d outside [1, min(batch, %d)]", M, kMaxMicrobatches);
-    int32_t offs[kMaxMicrobatches + 1];
+        return set_error(ctx, AFLEX_ERR_INVALID_ARG, "microbatch depth %d outside [1, min(batch, %d)]", M, kMaxMicrobatches);
     if (mb_offsets) {
         for (int i = 0; i <= M; ++i) offs[i] = mb_offsets[i];
-        if (offs[0] != 0 || offs[M] != batch) return set_error(ctx, AFLEX_ERR_INVALID_ARG, "decoder layers: mb_offsets must run from 0 to batch");
+        if (offs[0] != 0 || offs[M] != batch) return set_error(ctx, AFLEX_ERR_INVALID_ARG, "mb_offsets must run from 0 to batch");
         for (int i = 0; i < M; ++i)
-            if (offs[i + 1] <= offs[i]) return set_error(ctx, AFLEX_ERR_INVALID_ARG, "decoder layers: mb_offsets must be strictly increasing");
+            if (offs[i + 1] <= offs[i]) return set_error(ctx, AFLEX_ERR_INVALID_ARG, "mb_offsets must be strictly increasing");
     } else {
         const int base = batch / M, extra = batch % M;
         offs[0] = 0;
         for (int i = 0; i < M; ++i) offs[i + 1] = offs[i] + base + (i < extra ? 1 : 0);
     }
+    return AFLEX_OK;
+}
+}  // namespace
+
+aflex_status aflex_decoder_layers(aflex_ctx* ctx, const aflex_decoder_desc* layers, const aflex_kv* kvs, int num_layers,
+                                  const void* x_in, int batch, int M, const int32_t* mb_offsets, void* x_out,
+                                  void* stream) {
+    if (!ctx) return AFLEX_ERR_INVALID_ARG;
+    aflex_status s = validate_decoder_args(ctx, layers, kvs, num_layers, x_in, batch, x_out);
+    if (s != AFLEX_OK) return s;
+    const int H = layers[0].layer.hidden;
+    size_t need = 0;
+    for (int l = 0; l < num_layers; ++l) {
+        const DecoderWs w = decoder_ws(&layers[l], batch, attn_workspace_bytes(&layers[l].layer.attn, attn_grid(ctx)), ctx->num_sms);
+        if (w.total > need) need = w.total;
+    }
+    if (need > ctx->ws_bytes)
+        return set_error(ctx, AFLEX_ERR_WORKSPACE, "decoder layers: need %zu workspace bytes, have %zu", need, ctx->ws_bytes);
+    int32_t offs[kMaxMicrobatches + 1];
+    s = make_offsets(ctx, batch, M, mb_offsets, offs);
+    if (s != AFLEX_OK) return s;
 
     cudaStream_t user = reinterpret_cast<cudaStream_t>(stream);
     const bool serial = (M == 1);
@@ -781,6 +800,145 @@ aflex_status aflex_decoder_layers(aflex_ctx* ctx, const aflex_decoder_desc* laye
     if (e == cudaSuccess) e = cudaStreamWaitEvent(user, ctx->ev_a_done, 0);
     if (e == cudaSuccess) e = cudaStreamWaitEvent(user, ctx->ev_f_done, 0);
     return check_cuda(ctx, e, "decoder layers: exit join");
+}
+
+// ---- A/F pair: Attention side on ctx_a's device, FFN side on ctx_f's device ----------------
+// A-side workspace: [attn scratch | linear scratch | xn | qkv | q | a | o | h1 | back]
+// F-side workspace: [h1_f | xn2 | y | out_f | F scratch]
+namespace {
+struct PairWs {
+    size_t a_attn, a_lin, rows_h, rows_qkv, rows_a, a_total, f_scratch, f_total;
+};
+PairWs pair_ws(const aflex_decoder_desc* d, int max_batch, size_t a_attn, int num_sms) {
+    const DecoderWs w = decoder_ws(d, max_batch, a_attn, num_sms);
+    PairWs p;
+    p.a_attn = w.a_attn; p.a_lin = w.a_lin; p.rows_h = w.rows_h; p.rows_qkv = w.rows_qkv; p.rows_a = w.rows_a;
+    p.a_total = w.a_attn + w.a_lin + 4 * w.rows_h + w.rows_qkv + 2 * w.rows_a + 1024;
+    p.f_scratch = w.f_total;
+    p.f_total = 4 * w.rows_h + w.f_total + 1024;
+    return p;
+}
+struct DeviceGuard {
+    int saved = -1;
+    DeviceGuard() { cudaGetDevice(&saved); }
+    ~DeviceGuard() { if (saved >= 0) cudaSetDevice(saved); }
+};
+}  // namespace
+
+size_t aflex_af_workspace_bytes(const aflex_decoder_desc* layer, int max_batch, int ffn_side) {
+    if (!layer || max_batch < 1) return 0;
+    const PairWs w = pair_ws(layer, max_batch, attn_workspace_bytes(&layer->layer.attn, 4096), 148);
+    return ffn_side ? w.f_total : w.a_total;
+}
+
+aflex_status aflex_af_decoder_layers(aflex_ctx* ca, aflex_ctx* cf, const aflex_decoder_desc* layers, const aflex_kv* kvs,
+                                     int num_layers, const void* x_in, int batch, int M, const int32_t* mb_offsets,
+                                     void* x_out, void* stream) {
+    if (!ca || !cf) return AFLEX_ERR_INVALID_ARG;
+    if (ca == cf) return set_error(ca, AFLEX_ERR_INVALID_ARG, "A/F pair: the two sides need separate contexts");
+    aflex_status s = validate_decoder_args(ca, layers, kvs, num_layers, x_in, batch, x_out);
+    if (s != AFLEX_OK) return s;
+    const int H = layers[0].layer.hidden;
+    size_t need_a = 0, need_f = 0;
+    for (int l = 0; l < num_layers; ++l) {
+        const PairWs w = pair_ws(&layers[l], batch, attn_workspace_bytes(&layers[l].layer.attn, attn_grid(ca)), ca->num_sms);
+        if (w.a_total > need_a) need_a = w.a_total;
+        if (w.f_total > need_f) need_f = w.f_total;
+    }
+    if (need_a > ca->ws_bytes)
+        return set_error(ca, AFLEX_ERR_WORKSPACE, "A/F pair: attention side needs %zu workspace bytes, has %zu", need_a, ca->ws_bytes);
+    if (need_f > cf->ws_bytes)
+        return set_error(ca, AFLEX_ERR_WORKSPACE, "A/F pair: FFN side needs %zu workspace bytes, has %zu", need_f, cf->ws_bytes);
+    int32_t offs[kMaxMicrobatches + 1];
+    s = make_offsets(ca, batch, M, mb_offsets, offs);
+    if (s != AFLEX_OK) return s;
+
+    DeviceGuard guard;                                    // the caller's current device is restored on return
+    const int dev_a = ca->device, dev_f = cf->device;
+    cudaStream_t user = reinterpret_cast<cudaStream_t>(stream);
+    cudaStream_t sa = ca->stream_a, sf = cf->stream_f;
+    cudaError_t e = cudaSetDevice(dev_a);
+    if (e == cudaSuccess) e = cudaEventRecord(ca->ev_entry, user);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(sa, ca->ev_entry, 0);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(sf, ca->ev_entry, 0);
+    if (e != cudaSuccess) return check_cuda(ca, e, "A/F pair: entry join");
+
+    typedef __nv_bfloat16 bf;
+    for (int l = 0; l < num_layers; ++l) {
+        const aflex_decoder_desc* d = &layers[l];
+        const aflex_layer_desc* L = &d->layer;
+        const int Hq = L->attn.num_q_heads, Hkv = L->attn.num_kv_heads, D = L->attn.head_dim;
+        const int A = Hq * D, NQ = (Hq + 2 * Hkv) * D, I = L->inter, E = L->num_experts;
+        const PairWs w = pair_ws(d, batch, attn_workspace_bytes(&L->attn, attn_grid(ca)), ca->num_sms);
+        char* p = ca->ws;
+        char* ws_attn = p; p += w.a_attn;
+        char* ws_lin = p; p += w.a_lin;
+        bf* xn = reinterpret_cast<bf*>(p); p += w.rows_h;
+        bf* qkv = reinterpret_cast<bf*>(p); p += w.rows_qkv;
+        bf* qb = reinterpret_cast<bf*>(p); p += w.rows_a;
+        bf* ab = reinterpret_cast<bf*>(p); p += w.rows_a;
+        bf* ob = reinterpret_cast<bf*>(p); p += w.rows_h;
+        bf* h1 = reinterpret_cast<bf*>(p); p += w.rows_h;
+        bf* back = reinterpret_cast<bf*>(p); p += w.rows_h;
+        char* pf = cf->ws;
+        bf* h1f = reinterpret_cast<bf*>(pf); pf += w.rows_h;
+        bf* xn2 = reinterpret_cast<bf*>(pf); pf += w.rows_h;
+        bf* yb = reinterpret_cast<bf*>(pf); pf += w.rows_h;
+        bf* outf = reinterpret_cast<bf*>(pf); pf += w.rows_h;
+        char* ws_f = pf;
+        for (int i = 0; i < M; ++i) {
+            const int r0 = offs[i], rows = offs[i + 1] - offs[i];
+            const size_t oh = (size_t)r0 * H;
+            const size_t row_bytes = (size_t)rows * H * sizeof(bf);
+            // ---- A_{l,i} on the attention GPU
+            e = cudaSetDevice(dev_a);
+            if (e == cudaSuccess && l > 0) e = cudaStreamWaitEvent(sa, cf->ev_f[i], 0);   // the rows are back
+            if (e != cudaSuccess) return check_cuda(ca, e, "A/F pair: F->A event");
+            const bf* r = (l == 0 ? reinterpret_cast<const bf*>(x_in) : back) + oh;        // residual stream entering the layer
+            s = add_rmsnorm_launch(ca, r, nullptr, d->w_ln_attn, rows, H, d->rms_eps, nullptr, xn + oh, sa);
+            if (s != AFLEX_OK) return s;
+            s = linear_launch(ca, xn + oh, d->w_qkv, rows, H, NQ, qkv + (size_t)r0 * NQ, ws_lin, w.a_lin, sa, kKQkvGemm, ca->counters_a);
+            if (s != AFLEX_OK) return s;
+            aflex_kv kvi = kvs[l];
+            kvi.page_table = kvs[l].page_table + (size_t)r0 * kvs[l].max_pages_per_seq;
+            kvi.seq_lens = kvs[l].seq_lens + r0;
+            kvi.seq_lens_host = kvs[l].seq_lens_host ? kvs[l].seq_lens_host + r0 : nullptr;
+            s = rope_append_launch(ca, &L->attn, qkv + (size_t)r0 * NQ, &kvi, rows, d->w_q_norm, d->w_k_norm, d->rms_eps, d->rope_theta, qb + (size_t)r0 * A, sa);
+            if (s != AFLEX_OK) return s;
+            s = attn_decode_launch(ca, &L->attn, qb + (size_t)r0 * A, &kvi, rows, ab + (size_t)r0 * A, nullptr, ws_attn, w.a_attn, sa);
+            if (s != AFLEX_OK) return s;
+            s = linear_launch(ca, ab + (size_t)r0 * A, L->w_o, rows, A, H, ob + oh, ws_lin, w.a_lin, sa, kKLinearGemm, ca->counters_a);
+            if (s != AFLEX_OK) return s;
+            s = add_rmsnorm_launch(ca, r, ob + oh, nullptr, rows, H, 0.f, h1 + oh, nullptr, sa);     // h1 = r + a W_o^T
+            if (s != AFLEX_OK) return s;
+            // what A sends to F: into the FFN GPU's own memory, then the event
+            e = cudaMemcpyPeerAsync(h1f + oh, dev_f, h1 + oh, dev_a, row_bytes, sa);
+            if (e == cudaSuccess) e = cudaEventRecord(ca->ev_a[i], sa);
+            if (e != cudaSuccess) return check_cuda(ca, e, "A/F pair: A->F transfer");
+            // ---- F_{l,i} on the FFN GPU
+            e = cudaSetDevice(dev_f);
+            if (e == cudaSuccess) e = cudaStreamWaitEvent(sf, ca->ev_a[i], 0);
+            if (e != cudaSuccess) return check_cuda(ca, e, "A/F pair: A->F event");
+            s = add_rmsnorm_launch(cf, h1f + oh, nullptr, d->w_ln_ffn, rows, H, d->rms_eps, nullptr, xn2 + oh, sf);
+            if (s == AFLEX_OK) {
+                if (E == 0) s = dense_run(cf, xn2 + oh, L->w_gate, L->w_up, L->w_down, rows, H, I, yb + oh, ws_f, w.f_scratch, sf);
+                else s = moe_run(cf, xn2 + oh, nullptr, L->w_router, L->w_gate, L->w_up, L->w_down, rows, H, I, E, L->top_k, yb + oh,
+                                 nullptr, nullptr, nullptr, ws_f, w.f_scratch, sf);
+            }
+            if (s == AFLEX_OK) s = add_rmsnorm_launch(cf, h1f + oh, yb + oh, nullptr, rows, H, 0.f, outf + oh, nullptr, sf);   // out = h1 + FFN
+            if (s != AFLEX_OK) return set_error(ca, s, "A/F pair: FFN side: %s", cf->err);
+            // what F returns: into the attention GPU's memory (the last layer's rows go straight to x_out)
+            bf* dst = (l == num_layers - 1 ? reinterpret_cast<bf*>(x_out) : back) + oh;
+            e = cudaMemcpyPeerAsync(dst, dev_a, outf + oh, dev_f, row_bytes, sf);
+            if (e == cudaSuccess) e = cudaEventRecord(cf->ev_f[i], sf);
+            if (e != cudaSuccess) return check_cuda(ca, e, "A/F pair: F->A transfer");
+        }
+    }
+    e = cudaSetDevice(dev_a);
+    if (e == cudaSuccess) e = cudaEventRecord(ca->ev_a_done, sa);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(user, ca->ev_a_done, 0);
+    for (int i = 0; i < M && e == cudaSuccess; ++i) e = cudaStreamWaitEvent(user, cf->ev_f[i], 0);
+    return check_cuda(ca, e, "A/F pair: exit join");
 }
 
 }  // extern "C"

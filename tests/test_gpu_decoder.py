@@ -277,6 +277,52 @@ def test_decoder_layers_attention_sees_the_token_it_just_appended():
         ctx.close()
 
 
+@pytest.mark.parametrize("cfg,L", [(IN.CONFIGS[1], 3), (TINY_MOE, 2)], ids=lambda v: getattr(v, "name", str(v)))
+def test_af_pair_matches_oracle_and_single_context_chain(cfg, L):
+    """Attention side and FFN side in two contexts (here on the same GPU: the peer copies are then
+    device-local), hidden states handed over once each way per layer and microbatch."""
+    ch = Chain(cfg, L)
+    ctx = AF.Context(0, ch.workspace())
+    ca = AF.Context(0, max(AF.af_workspace_bytes(d, cfg.batch, False) for d in ch.descs))
+    cf = AF.Context(0, max(AF.af_workspace_bytes(d, cfg.batch, True) for d in ch.descs))
+    try:
+        outs, _, margins = ch.oracle()
+        keep = np.ones(cfg.batch, dtype=bool)
+        for m in margins:
+            keep &= m > 0.02
+        single = _run_chain(ctx, ch, 1)
+        for M in (1, 2, cfg.batch):
+            ch.reset_caches()
+            x_out = torch.full_like(ch.x, float("nan"), device=DEV)
+            AF.af_decoder_layers(ca, cf, ch.descs, ch.kvs, ch.x.to(DEV), x_out, M)
+            torch.cuda.synchronize()
+            assert ca.device_status() == AF.OK and cf.device_status() == AF.OK
+            assert row_rel_err(f64(x_out)[keep], outs[-1][keep]) <= TOL_FFN * L, (cfg.name, M)
+            assert row_rel_err(f64(x_out)[keep], f64(single)[keep]) <= 1e-2 * L, (cfg.name, M)
+        # the same call twice gives the same bits
+        ch.reset_caches()
+        a = torch.empty_like(x_out)
+        AF.af_decoder_layers(ca, cf, ch.descs, ch.kvs, ch.x.to(DEV), a, 2)
+        ch.reset_caches()
+        b = torch.empty_like(x_out)
+        AF.af_decoder_layers(ca, cf, ch.descs, ch.kvs, ch.x.to(DEV), b, 2)
+        torch.cuda.synchronize()
+        assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+        with pytest.raises(AF.AflexError):
+            AF.af_decoder_layers(ca, ca, ch.descs, ch.kvs, ch.x.to(DEV), a, 1)
+        small = AF.Context(0, 1 << 16)
+        try:
+            with pytest.raises(AF.AflexError) as ei:
+                AF.af_decoder_layers(ca, small, ch.descs, ch.kvs, ch.x.to(DEV), a, 1)
+            assert ei.value.status == AF.ERR_WORKSPACE
+        finally:
+            small.close()
+    finally:
+        ctx.close()
+        ca.close()
+        cf.close()
+
+
 def test_decoder_layers_in_place_and_argument_checks():
     cfg = IN.CONFIGS[1]
     ch = Chain(cfg, 2)
