@@ -7,7 +7,7 @@
 //
 //   work        = the list of 64-token units (4 pages) of every (sequence, KV head) item, in
 //                 (sequence, head, unit) order.  It is cut into one contiguous, equal share per CTA
-//                 (2 CTAs per SM), computed on the device from the sequence lengths: no host plan,
+//                 (2 CTAs per SM), located on the device from the sequence lengths: no host plan,
 //                 no wave quantisation, no per-chunk launch overhead.  A CTA's share is a run of
 //                 "pieces": unit ranges of consecutive items.
 //   data path   = a producer warp walks the share and issues tiled TMA loads (128-byte swizzle) of
@@ -19,13 +19,17 @@
 //                 padding: S^T = K Q^T, then O^T += V^T P^T with P^T obtained from the S^T
 //                 accumulator by movmatrix.  The flop/byte ratio (8 at G = 8) is above what the
 //                 fp32 pipes sustain at full HBM rate, which is the only reason MMAs are used.
-//   softmax     = online, fp32, base-2 exponentials; each of the 4 consumer warps owns one page
-//                 of a unit and its own running (m, l, O); at the end of a piece warps 1-3 hand
-//                 their state to warp 0 through shared memory.
+//   softmax     = online, fp32, base-2 exponentials; each of the 4 compute warps owns one page of a
+//                 unit and its own running (m, l, O).  At the last unit of a piece every compute warp
+//                 parks its state in its own K/V pages of that stage and goes on to the next piece
+//                 without waiting; an epilogue warp that walks the same pieces folds the four states
+//                 (fixed order), releases the stage and does everything that touches global memory.
 //   combine     = a piece that covers its whole item is written straight to the output.  Otherwise
-//                 the piece's unnormalised (O, m, l) goes to a per-CTA slot and the item's arrival
-//                 counter is bumped; the CTA that arrives last merges the item's pieces, always in
-//                 CTA order, so the result does not depend on which CTA was last (deterministic).
+//                 the piece's unnormalised (O, m, l) goes to one of the range's two partial slots and
+//                 the item's arrival counter is bumped; the warp that arrives last merges the item's
+//                 pieces, always in list order, so the result does not depend on which was last.
+//   tail        = on launches large enough for one 16-unit chunk per CTA, the last quarter of the
+//                 list is handed out as ticket-claimed chunks, so faster CTAs take more.
 //
 // Unreferenced slots (beyond a sequence's length) may hold NaN: scores of such tokens are
 // replaced (not multiplied) by -inf and their V rows are zeroed in shared memory before use.
@@ -43,7 +47,7 @@ constexpr int kPagesPerStage = 4;
 constexpr int kUnitTokens = kPage * kPagesPerStage;   // 64
 constexpr int kAttnStages = 3;
 constexpr int kAttnConsumerWarps = 4;
-constexpr int kAttnThreads = (kAttnConsumerWarps + 1) * 32;
+constexpr int kAttnThreads = (kAttnConsumerWarps + 2) * 32;   // compute warps, producer warp, epilogue warp
 constexpr float kNegBig = -1.0e30f;
 
 struct AttnParams {
@@ -64,7 +68,7 @@ struct AttnParams {
     int dyn_pct;           // percent of the unit list handed out dynamically (0 = static shares only)
     int dyn_chunks;        // target number of dynamic chunks per CTA
     int kv_policy;         // 0: evict-first KV loads, 1: normal priority (tuning)
-    int dyn_min;           // smallest chunk (units) for which the dynamic tail is used
+    int dyn_min;           // chunk size (units) the dynamic tail aims at
     int piece_cost;        // list positions charged per item start (balances the fixed cost of a piece)
     int* status;
     unsigned long long* trace;
@@ -83,6 +87,7 @@ constexpr int kRangeRing = 4;
 struct __align__(8) AttnShared {
     uint64_t full[kAttnStages];
     uint64_t empty[kAttnStages];
+    uint64_t xready[kAttnStages];   // the compute warps' states of a finished piece are parked in this stage
     uint64_t rng_ready[kRangeRing];
     AttnRange rng[kRangeRing];
     volatile int abort;
@@ -132,22 +137,23 @@ struct Walker {
 struct AttnSplit {
     long long U, U1;
     int Ge1, K2, n2;
-    __device__ AttnSplit(long long U_, int grid, int dyn_pct, int dyn_chunks, int dyn_min = 12) {
+    // dyn_pct: share of the list handed out dynamically; dyn_chunks: most chunks per CTA (bounds the partial
+    // slots); dyn_units: chunk size aimed at.  A chunk costs a claim, a hand-over and an extra partial piece
+    // to publish and merge, so chunks stay at dyn_units or more, and the tail is dynamic only when it yields
+    // at least one chunk per CTA (small launches stay purely static).
+    __device__ AttnSplit(long long U_, int grid, int dyn_pct, int dyn_chunks, int dyn_units = 16) {
         U = U_;
         long long U2 = dyn_pct > 0 ? U * dyn_pct / 100 : 0;
-        // A chunk costs a fixed ~2-3 us (claim, hand-over, an extra partial piece to publish and merge):
-        // chunks below ~12 units (~0.4 MB at D = 128) do not pay, so small launches stay purely static.
-        if (U2 > 0 && U2 / ((long long)dyn_chunks * grid) < dyn_min) U2 = 0;
+        K2 = 1; n2 = 0;
         if (U2 > 0) {
             long long k = (U2 + (long long)dyn_chunks * grid - 1) / ((long long)dyn_chunks * grid);
-            K2 = (int)(k < 2 ? 2 : (k > 64 ? 64 : k));
+            if (k < dyn_units) k = dyn_units;
+            if (k > (1 << 20)) k = 1 << 20;
+            K2 = (int)k;
             n2 = (int)((U2 + K2 - 1) / K2);
-            // keep the slot count bounded: never more than dyn_chunks * grid + 1 chunks
-            if (n2 > dyn_chunks * grid + 1) { n2 = dyn_chunks * grid + 1; }
-            U2 = min(U2, (long long)n2 * K2);
-        } else { K2 = 1; n2 = 0; }
+            if (n2 < grid) { U2 = 0; n2 = 0; K2 = 1; }
+        }
         U1 = U - U2;
-        n2 = U2 > 0 ? (int)((U2 + K2 - 1) / K2) : 0;
         Ge1 = (int)min((long long)grid, U1);
     }
 };
@@ -170,12 +176,10 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     constexpr int kStageBytes = 2 * kPagesPerStage * kPageBytes;
     constexpr int kOpsPerStage = 2 * kPagesPerStage * kHalves;
     constexpr int kKSteps = D / 16;
-    constexpr int kStateFloats = 4 * kKSteps + 4;   // per lane: O fragments + m0, m1, l0, l1
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    float* xchg = reinterpret_cast<float*>(smem + kAttnStages * kStageBytes);           // [3 warps][kStateFloats][32]
-    AttnShared* sh = reinterpret_cast<AttnShared*>(xchg + 3 * kStateFloats * 32);
+    AttnShared* sh = reinterpret_cast<AttnShared*>(smem + kAttnStages * kStageBytes);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -193,6 +197,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         for (int s = 0; s < kAttnStages; ++s) {
             mbar_init(&sh->full[s], 1);
             mbar_init(&sh->empty[s], kAttnConsumerWarps);
+            mbar_init(&sh->xready[s], kAttnConsumerWarps);
         }
         for (int i = 0; i < kRangeRing; ++i) mbar_init(&sh->rng_ready[i], 1);
         sh->abort = 0;
@@ -367,18 +372,16 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                 if (atomicAdd(&p.ticket[1], 1) == (int)gridDim.x - 1) { p.ticket[0] = 0; p.ticket[1] = 0; }
             }
         }
-    } else {
-        // ------------------------------------------------------------------ consumer warps
+    } else if (warp < kAttnConsumerWarps) {
+        // ------------------------------------------------------------------ compute warps
         // q is final when this kernel starts (an input of the step, or written by the K/V append kernel,
-        // which does not release its dependents early), so pages are processed at once; the grid
-        // dependency is awaited before this warp's first write to global memory.
-        bool dep_ok = false;
+        // which does not release its dependents early), so pages are processed at once.  These warps
+        // never write to global memory: a finished piece's state goes to the epilogue warp through the
+        // piece's last stage buffer.
         const int mi = lane >> 3, r8 = lane & 7;
-        const int h0 = 2 * (lane & 3);          // this lane's two heads of the group: h0, h0 + 1
         int s = 0;
         uint32_t ph = 0;
         bool aborted = false;
-        const int G = (int)gridDim.x;
 
         for (int r = 0; !aborted; ++r) {
             // ---- next range of this CTA
@@ -390,7 +393,6 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             if (rg.x1 <= rg.x0) break;
             Walker wk;
             wk.init(p, rg);
-            bool first_piece = true;            // a partial piece uses slot 0 if it is the range's first piece, else 1
 
         while (!wk.done() && !aborted) {
             // ---- one piece: units [u0, u0 + n) of item (b, g)
@@ -403,8 +405,6 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             const int n = max(wk.u + nv, cost) - cost - u0;
             wk.advance(nv);
             if (n <= 0) continue;                                            // only empty positions: no piece
-            const int slot = first_piece ? 0 : 1;
-            first_piece = false;
 
             // Q^T as the MMA's B operand: lane holds head (lane/4), d = 16*ks + 2*(lane%4) + {0,1} (+8)
             uint32_t qb[kKSteps][2];
@@ -495,58 +495,124 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                     if (nvalid < kPage) fence_proxy_async();   // order the zeroing stores before the next TMA write
                 }
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&sh->empty[s]);
+                if (u + 1 < u0 + n) {
+                    if (lane == 0) mbar_arrive(&sh->empty[s]);
+                } else {
+                    // ---- last unit of the piece: park (O, m, l) in this warp's own pages of the stage (the O
+                    // fragments fill the K page exactly, m and l go to the V page) and tell the epilogue warp;
+                    // it releases the stage once it has read the four states.  No warp waits for another.
+#pragma unroll
+                    for (int off = 4; off < 32; off <<= 1) {
+                        l0 += __shfl_xor_sync(0xffffffffu, l0, off);
+                        l1 += __shfl_xor_sync(0xffffffffu, l1, off);
+                    }
+                    float* kdst = reinterpret_cast<float*>(smem + s * kStageBytes + warp * kPageBytes) + lane;
+                    float* vdst = reinterpret_cast<float*>(smem + s * kStageBytes + (kPagesPerStage + warp) * kPageBytes) + lane;
+#pragma unroll
+                    for (int mt = 0; mt < kKSteps; ++mt) {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) kdst[(mt * 4 + j) * 32] = o[mt][j];
+                    }
+                    vdst[0] = m0; vdst[32] = m1; vdst[64] = l0; vdst[96] = l1;
+                    fence_proxy_async();                 // these stores precede the stage's next TMA write
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sh->xready[s]);
+                }
                 if (++s == kAttnStages) { s = 0; ph ^= 1; }
             }
 
             if (tr && threadIdx.x == 0) tr[4] = global_timer_ns();      // units of this piece consumed
-            // ---- end of piece: warps 1..3 hand (O, m, l) to warp 0
-#pragma unroll
-            for (int off = 4; off < 32; off <<= 1) {
-                l0 += __shfl_xor_sync(0xffffffffu, l0, off);
-                l1 += __shfl_xor_sync(0xffffffffu, l1, off);
-            }
-            // (A) warp 0 has finished reading the exchange area of the previous piece
-            asm volatile("bar.sync 1, %0;" ::"n"(kAttnConsumerWarps * 32) : "memory");
-            if (warp > 0) {
-                float* dst = xchg + (size_t)(warp - 1) * kStateFloats * 32 + lane;
-#pragma unroll
-                for (int mt = 0; mt < kKSteps; ++mt) {
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) dst[(mt * 4 + j) * 32] = o[mt][j];
-                }
-                dst[(4 * kKSteps + 0) * 32] = m0; dst[(4 * kKSteps + 1) * 32] = m1;
-                dst[(4 * kKSteps + 2) * 32] = l0; dst[(4 * kKSteps + 3) * 32] = l1;
-            }
-            // (B) states of warps 1..3 are in shared memory
-            asm volatile("bar.sync 1, %0;" ::"n"(kAttnConsumerWarps * 32) : "memory");
-            if (sh->abort) { aborted = true; break; }
-            if (warp != 0) continue;
+        }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue warp
+        // Walks the same ranges and pieces as the compute warps.  For every piece it waits until the four
+        // states are parked in the piece's last stage, folds them (fixed order 0, 1, 2, 3), releases the
+        // stage to the producer, and then does everything that touches global memory: the output row of a
+        // whole item, or the partial slot, the arrival counter and - for the last arriver - the merge.
+        // The compute warps stream on meanwhile; only the stage that holds the states waits for this warp.
+        bool dep_ok = false;
+        const int h0 = 2 * (lane & 3);          // this lane's two heads of the group: h0, h0 + 1
+        int s = 0;
+        uint32_t xph = 0;                       // phase bit of xready[] per stage
+        bool aborted = false;
+        const int G = (int)gridDim.x;
 
-            // ---- warp 0: merge the three states into its own (fixed order 1, 2, 3)
-#pragma unroll
-            for (int w = 0; w < kAttnConsumerWarps - 1; ++w) {
-                const float* src = xchg + (size_t)w * kStateFloats * 32 + lane;
-                const float om0 = src[(4 * kKSteps + 0) * 32], om1 = src[(4 * kKSteps + 1) * 32];
-                const float ol0 = src[(4 * kKSteps + 2) * 32], ol1 = src[(4 * kKSteps + 3) * 32];
-                const float mn0 = fmaxf(m0, om0), mn1 = fmaxf(m1, om1);
-                const float a0 = fast_exp2(m0 - mn0), a1 = fast_exp2(m1 - mn1);
-                const float b0 = fast_exp2(om0 - mn0), b1 = fast_exp2(om1 - mn1);
-                m0 = mn0; m1 = mn1;
-                l0 = l0 * a0 + ol0 * b0;
-                l1 = l1 * a1 + ol1 * b1;
+        for (int r = 0; !aborted; ++r) {
+            // ---- next range of this CTA
+            if (!mbar_wait(&sh->rng_ready[r % kRangeRing], (uint32_t)((r / kRangeRing) & 1))) {
+                if (lane == 0) { sh->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); }
+                break;
+            }
+            const AttnRange rg = sh->rng[r % kRangeRing];
+            if (rg.x1 <= rg.x0) break;
+            Walker wk;
+            wk.init(p, rg);
+            bool first_piece = true;            // a partial piece uses slot 0 if it is the range's first piece, else 1
+
+        while (!wk.done() && !aborted) {
+            // ---- one piece: units [u0, u0 + n) of item (b, g)
+            const int b = wk.b, g = wk.g, len = wk.len, cost = wk.cost;
+            const int nu = wk.nu - cost;                                     // real units of the item
+            const long long item_v0 = wk.prefix * p.Hkv + (long long)g * wk.nu;   // list position where the item starts
+            const long long item_x0 = item_v0 + cost;                        // ... where its real units start
+            const int nv = (int)min((long long)(wk.nu - wk.u), wk.end - wk.pos);
+            const int u0 = max(wk.u, cost) - cost;                           // real unit range [u0, u0 + n)
+            const int n = max(wk.u + nv, cost) - cost - u0;
+            wk.advance(nv);
+            if (n <= 0) continue;                                            // only empty positions: no piece
+            const int slot = first_piece ? 0 : 1;
+            first_piece = false;
+
+            const int s_last = (s + n - 1) % kAttnStages;
+            s = (s + n) % kAttnStages;
+            {
+                bool ok = mbar_wait(&sh->xready[s_last], (xph >> s_last) & 1u);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok || sh->abort) {
+                    if (lane == 0) { sh->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); }
+                    aborted = true;
+                    break;
+                }
+                xph ^= 1u << s_last;
+            }
+            float o[kKSteps][4];
+            float m0, m1, l0, l1;
+            {
+                const float* ksrc = reinterpret_cast<const float*>(smem + s_last * kStageBytes) + lane;
+                const float* vsrc = reinterpret_cast<const float*>(smem + s_last * kStageBytes + kPagesPerStage * kPageBytes) + lane;
 #pragma unroll
                 for (int mt = 0; mt < kKSteps; ++mt) {
-                    o[mt][0] = o[mt][0] * a0 + src[(mt * 4 + 0) * 32] * b0;
-                    o[mt][1] = o[mt][1] * a1 + src[(mt * 4 + 1) * 32] * b1;
-                    o[mt][2] = o[mt][2] * a0 + src[(mt * 4 + 2) * 32] * b0;
-                    o[mt][3] = o[mt][3] * a1 + src[(mt * 4 + 3) * 32] * b1;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) o[mt][j] = ksrc[(mt * 4 + j) * 32];
+                }
+                m0 = vsrc[0]; m1 = vsrc[32]; l0 = vsrc[64]; l1 = vsrc[96];
+#pragma unroll
+                for (int w = 1; w < kAttnConsumerWarps; ++w) {
+                    const float* ks = ksrc + w * (kPageBytes / 4);
+                    const float* vs = vsrc + w * (kPageBytes / 4);
+                    const float om0 = vs[0], om1 = vs[32], ol0 = vs[64], ol1 = vs[96];
+                    const float mn0 = fmaxf(m0, om0), mn1 = fmaxf(m1, om1);
+                    const float a0 = fast_exp2(m0 - mn0), a1 = fast_exp2(m1 - mn1);
+                    const float b0 = fast_exp2(om0 - mn0), b1 = fast_exp2(om1 - mn1);
+                    m0 = mn0; m1 = mn1;
+                    l0 = l0 * a0 + ol0 * b0;
+                    l1 = l1 * a1 + ol1 * b1;
+#pragma unroll
+                    for (int mt = 0; mt < kKSteps; ++mt) {
+                        o[mt][0] = o[mt][0] * a0 + ks[(mt * 4 + 0) * 32] * b0;
+                        o[mt][1] = o[mt][1] * a1 + ks[(mt * 4 + 1) * 32] * b1;
+                        o[mt][2] = o[mt][2] * a0 + ks[(mt * 4 + 2) * 32] * b0;
+                        o[mt][3] = o[mt][3] * a1 + ks[(mt * 4 + 3) * 32] * b1;
+                    }
                 }
             }
+            __syncwarp();
+            if (lane == 0) mbar_arrive_n(&sh->empty[s_last], kAttnConsumerWarps);    // the stage may be refilled
             if (!dep_ok) {
                 pdl_wait();   // output rows, partial slots and counters may still be in use by earlier kernels
                 dep_ok = true;
-                if (tr && threadIdx.x == 0) tr[2] = global_timer_ns();
+                if (tr && lane == 0) tr[2] = global_timer_ns();
             }
             const int dr = lane >> 2;
             const size_t hq0 = (size_t)g * p.G + h0;
@@ -687,7 +753,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             if (lane == 0) p.counters[b * p.Hkv + g] = 0;   // clean for the next launch
         }
         }
-        if (tr && threadIdx.x == 0) tr[5] = global_timer_ns();
+        if (tr && lane == 0) tr[5] = global_timer_ns();
     }
 }
 
@@ -701,19 +767,19 @@ int attn_grid(const aflex_ctx* ctx) {
 // Dynamic hand-out of the tail of the unit list (tuning: AFLEX_ATTN_DYN_PCT, AFLEX_ATTN_DYN_CHUNKS).
 static int attn_dyn_pct() {
     static int v = -1;
-    if (v < 0) { const char* e = getenv("AFLEX_ATTN_DYN_PCT"); v = e ? atoi(e) : 15; if (v < 0) v = 0; if (v > 90) v = 90; }
+    if (v < 0) { const char* e = getenv("AFLEX_ATTN_DYN_PCT"); v = e ? atoi(e) : 25; if (v < 0) v = 0; if (v > 90) v = 90; }
     return v;
 }
 static int attn_dyn_chunks() {
     static int v = -1;
-    if (v < 0) { const char* e = getenv("AFLEX_ATTN_DYN_CHUNKS"); v = e ? atoi(e) : 4; if (v < 1) v = 1; if (v > 64) v = 64; }
+    if (v < 0) { const char* e = getenv("AFLEX_ATTN_DYN_CHUNKS"); v = e ? atoi(e) : 8; if (v < 1) v = 1; if (v > 64) v = 64; }
     return v;
 }
 
 // List positions charged per item start when the unit list is cut into equal shares (tuning).
 static int attn_piece_cost() {
     static int v = -1;
-    if (v < 0) { const char* e = getenv("AFLEX_ATTN_PIECE_COST"); v = e ? atoi(e) : 2; if (v < 0) v = 0; if (v > 16) v = 16; }
+    if (v < 0) { const char* e = getenv("AFLEX_ATTN_PIECE_COST"); v = e ? atoi(e) : 1; if (v < 0) v = 0; if (v > 16) v = 16; }
     return v;
 }
 
@@ -751,7 +817,7 @@ static aflex_status attn_launch_t(aflex_ctx* ctx, const aflex_attn_desc* d, cons
     p.dyn_pct = attn_dyn_pct();
     p.dyn_chunks = attn_dyn_chunks();
     p.piece_cost = attn_piece_cost();
-    { static int v = -1; if (v < 0) { const char* e = getenv("AFLEX_ATTN_DYN_MIN"); v = e ? atoi(e) : 12; if (v < 1) v = 1; } p.dyn_min = v; }
+    { static int v = -1; if (v < 0) { const char* e = getenv("AFLEX_ATTN_DYN_UNITS"); v = e ? atoi(e) : 16; if (v < 1) v = 1; } p.dyn_min = v; }
     { static int v = -1; if (v < 0) { const char* e = getenv("AFLEX_ATTN_KVPOL"); v = e ? atoi(e) : 0; } p.kv_policy = v; }
     p.status = ctx->dev_status;
     p.out = reinterpret_cast<__nv_bfloat16*>(out);
@@ -766,8 +832,7 @@ static aflex_status attn_launch_t(aflex_ctx* ctx, const aflex_attn_desc* d, cons
         return set_error(ctx, AFLEX_ERR_CUDA, "attention: cuTensorMapEncodeTiled failed");
 
     constexpr int kStageBytes = 2 * kPagesPerStage * kPage * D * 2;
-    constexpr int kStateFloats = 4 * (D / 16) + 4;
-    const size_t smem = (size_t)kAttnStages * kStageBytes + 3 * kStateFloats * 32 * sizeof(float) + sizeof(AttnShared) + 1024;
+    const size_t smem = (size_t)kAttnStages * kStageBytes + sizeof(AttnShared) + 1024;
     const int ti = (D == 128) ? 1 : 0;
     if (!ctx->attn_attr_set[ti]) {
         cudaError_t e = cudaFuncSetAttribute(attn_decode_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -874,8 +939,7 @@ static aflex_status attn_static_launch(StaticDeviceState& stt, const aflex_attn_
         !encode_tmap_2d_bf16(&tv, kv->v_cache, rows, D, (uint64_t)D * 2, kPage, 64, true))
         return AFLEX_ERR_CUDA;
     constexpr int kStageBytes = 2 * kPagesPerStage * kPage * D * 2;
-    constexpr int kStateFloats = 4 * (D / 16) + 4;
-    const size_t smem = (size_t)kAttnStages * kStageBytes + 3 * kStateFloats * 32 * sizeof(float) + sizeof(AttnShared) + 1024;
+    const size_t smem = (size_t)kAttnStages * kStageBytes + sizeof(AttnShared) + 1024;
     const int ti = (D == 128) ? 1 : 0;
     if (!stt.attr_set[ti]) {
         e = cudaFuncSetAttribute(attn_decode_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
