@@ -13,6 +13,8 @@
 // Variants (template MODE):
 //   kLinear : out = x w^T                                   (W_o projection, down projection)
 //   kGateUp : out = silu(x w_gate^T) .* (x w_up^T)          (two accumulators, fused SwiGLU epilogue)
+//   kLinear2: kLinear with two weight-row tiles (256 rows) per CTA tile sharing one activation tile:
+//             half the activation traffic per weight byte, used at 64..128 token rows
 // Both have a grouped form for the mixture-of-experts FFN: the rows of x are the permuted
 // assignments, expert e owns rows [offsets[e], offsets[e+1]) and its own weight matrices.
 //
@@ -42,7 +44,7 @@
 
 namespace aflex {
 
-enum GemmMode { kLinear = 0, kGateUp = 1 };
+enum GemmMode { kLinear = 0, kGateUp = 1, kLinear2 = 2 };
 
 constexpr int kBlockM = 128;   // weight rows per tile (UMMA M)
 constexpr int kBlockK = 64;    // bf16 elements per 128-byte swizzled row
@@ -55,7 +57,8 @@ struct GemmParams {
     int N;            // weight rows (output features) per expert
     int K;
     int n_tile;       // token rows per tile, multiple of 16, <= 256
-    int m_tiles;      // ceil(N / 128)
+    int m_tiles;      // ceil(N / tile_rows)
+    int tile_rows;    // weight rows per tile: 128, or 256 in kLinear2
     int n_tiles;      // ceil(T / n_tile) (non-grouped)
     int kblocks;      // ceil(K / 64)
     int stages;       // smem pipeline depth
@@ -101,7 +104,7 @@ struct TileIter {
         if (p.num_experts == 0) {
             int nt = w % p.n_tiles;
             c.m_tile = w / p.n_tiles;
-            c.a_row0 = c.m_tile * kBlockM;
+            c.a_row0 = c.m_tile * p.tile_rows;
             c.b_row0 = nt * p.n_tile;
             c.b_rows = min(p.n_tile, p.T - c.b_row0);
             c.out_row_limit = p.T;
@@ -221,7 +224,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
     extern __shared__ uint8_t smem_raw[];
     // 1024-byte alignment: the 128-byte swizzle pattern is a function of address bits [7,10).
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    constexpr int kNumA = (MODE == kGateUp) ? 2 : 1;
+    constexpr int kNumA = (MODE == kLinear) ? 1 : 2;
     constexpr int kABytes = kBlockM * kBlockK * 2;           // 16 KB
     const int stage_bytes = kNumA * kABytes + ((p.n_tile * kBlockK * 2 + 1023) & ~1023);
     GemmBarriers* bars = reinterpret_cast<GemmBarriers*>(smem + (size_t)p.stages * stage_bytes);
@@ -256,7 +259,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
 
     const uint32_t tmem_base = bars->tmem_base;
     const TileIter tiles(p, bars->seg);
-    constexpr int kAccs = (MODE == kGateUp) ? 2 : 1;
+    constexpr int kAccs = (MODE == kLinear) ? 1 : 2;
     const int acc_cols = kAccs * p.n_tile;   // TMEM columns per accumulator buffer
     const Schedule sched(p, tiles.total, (int)gridDim.x);
     pdl_launch_dependents();
@@ -286,7 +289,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
                         uint8_t* st = smem + (size_t)primed * stage_bytes;
                         mbar_expect_tx(&bars->full[primed], tx);
                         tma_load_2d_hint(st, &tmap_a0, kb * kBlockK, c.a_row0, &bars->full[primed], pol_w);
-                        if (MODE == kGateUp) tma_load_2d_hint(st + kABytes, &tmap_a1, kb * kBlockK, c.a_row0, &bars->full[primed], pol_w);
+                        if (kNumA == 2) tma_load_2d_hint(st + kABytes, MODE == kGateUp ? &tmap_a1 : &tmap_a0, kb * kBlockK,
+                                                         c.a_row0 + (MODE == kGateUp ? 0 : kBlockM), &bars->full[primed], pol_w);
                         pend_kb[primed] = kb; pend_row[primed] = c.b_row0; pend_box[primed] = bi;
                         ++primed;
                         if (++s == p.stages) { s = 0; ph ^= 1; }
@@ -305,7 +309,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
                     uint8_t* st = smem + (size_t)s * stage_bytes;
                     mbar_expect_tx(&bars->full[s], tx);
                     tma_load_2d_hint(st, &tmap_a0, kb * kBlockK, c.a_row0, &bars->full[s], pol_w);
-                    if (MODE == kGateUp) tma_load_2d_hint(st + kABytes, &tmap_a1, kb * kBlockK, c.a_row0, &bars->full[s], pol_w);
+                    if (kNumA == 2) tma_load_2d_hint(st + kABytes, MODE == kGateUp ? &tmap_a1 : &tmap_a0, kb * kBlockK,
+                                                     c.a_row0 + (MODE == kGateUp ? 0 : kBlockM), &bars->full[s], pol_w);
                     tma_load_2d_hint(st + kNumA * kABytes, &tmaps_b.m[bi], kb * kBlockK, c.b_row0, &bars->full[s], pol_x);
                     if (++s == p.stages) { s = 0; ph ^= 1; }
                 }
@@ -345,7 +350,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
                         const uint32_t acc = (kb > wu.kb0 || k > 0) ? 1u : 0u;
                         // advancing 16 bf16 along K inside the swizzled row = +32 bytes = +2 in 16-byte units
                         umma_bf16(d0, da0 + 2 * k, db + 2 * k, idesc, acc);
-                        if (MODE == kGateUp) {
+                        if (kNumA == 2) {
                             const uint64_t da1 = umma_desc_k_sw128(a_addr + kABytes);
                             umma_bf16(d0 + (uint32_t)p.n_tile, da1 + 2 * k, db + 2 * k, idesc, acc);
                         }
@@ -417,7 +422,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
                             const float4* part = reinterpret_cast<const float4*>(p.partials + ((size_t)cc * 2 + sl) * slot_floats);
                             a0[q] = __ldcg(part + i0);
                             if (two) a1[q] = __ldcg(part + i1);
-                            if (MODE == kGateUp) {
+                            if (kAccs == 2) {
                                 b0[q] = __ldcg(part + up_off + i0);
                                 if (two) b1[q] = __ldcg(part + up_off + i1);
                             }
@@ -428,7 +433,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
                         if (cb + q <= cl) {
                             g0.x += a0[q].x; g0.y += a0[q].y; g0.z += a0[q].z; g0.w += a0[q].w;
                             if (two) { g1.x += a1[q].x; g1.y += a1[q].y; g1.z += a1[q].z; g1.w += a1[q].w; }
-                            if (MODE == kGateUp) {
+                            if (kAccs == 2) {
                                 u0.x += b0[q].x; u0.y += b0[q].y; u0.z += b0[q].z; u0.w += b0[q].w;
                                 if (two) { u1.x += b1[q].x; u1.y += b1[q].y; u1.z += b1[q].z; u1.w += b1[q].w; }
                             }
@@ -442,12 +447,16 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
                     const float4 gv = h ? g1 : g0, uv = h ? u1 : u0;
                     const float gf[4] = {gv.x, gv.y, gv.z, gv.w}, uf[4] = {uv.x, uv.y, uv.z, uv.w};
                     const int r = idx & (kBlockM - 1), cg = idx / kBlockM;
-                    const int nl = pd.c.m_tile * kBlockM + r;
+                    const int nl = pd.c.m_tile * p.tile_rows + r;
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {
                         const int t = pd.c.b_row0 + cg * 4 + k;
                         if (nl < p.N && t < pd.c.out_row_limit) {
                             if (MODE == kGateUp) p.out_bf16[(size_t)t * p.N + nl] = __float2bfloat16_rn(silu_f32(gf[k]) * uf[k]);
+                            else if (MODE == kLinear2) {
+                                p.out_bf16[(size_t)t * p.N + nl] = __float2bfloat16_rn(gf[k]);
+                                if (nl + kBlockM < p.N) p.out_bf16[(size_t)t * p.N + nl + kBlockM] = __float2bfloat16_rn(uf[k]);
+                            }
                             else if (p.out_f32) p.out_f32[(size_t)t * p.N + nl] = gf[k];
                             else p.out_bf16[(size_t)t * p.N + nl] = __float2bfloat16_rn(gf[k]);
                         }
@@ -475,7 +484,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
             }
             if (!mbar_wait(&bars->tmem_full[buf], acc_ph)) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); break; }
             tc_fence_after();
-            const int n_local = c.m_tile * kBlockM + row;    // output feature inside the expert
+            const int n_local = c.m_tile * p.tile_rows + row;    // output feature inside the expert
             const bool n_ok = n_local < p.N;
             const uint32_t t0 = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(buf * acc_cols);
             if (wu.slot < 0) {
@@ -493,6 +502,19 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
                             if (n_ok && t < c.out_row_limit) {
                                 const float hv = silu_f32(__uint_as_float(g[j])) * __uint_as_float(u[j]);
                                 p.out_bf16[(size_t)t * p.N + n_local] = __float2bfloat16_rn(hv);
+                            }
+                        }
+                    } else if (MODE == kLinear2) {
+                        uint32_t u[16];
+                        tmem_ld_32x32b_x16(t0 + (uint32_t)(p.n_tile + c0), u);
+                        tmem_ld_wait();
+                        const bool n2_ok = n_local + kBlockM < p.N;        // the tile's second 128 weight rows
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const int t = c.b_row0 + c0 + j;
+                            if (t < c.out_row_limit) {
+                                if (n_ok) p.out_bf16[(size_t)t * p.N + n_local] = __float2bfloat16_rn(__uint_as_float(g[j]));
+                                if (n2_ok) p.out_bf16[(size_t)t * p.N + n_local + kBlockM] = __float2bfloat16_rn(__uint_as_float(u[j]));
                             }
                         }
                     } else {
@@ -587,6 +609,21 @@ static int streaming_smem_budget() {
     return kb * 1024;
 }
 
+// Plain linear GEMMs take two weight-row tiles per CTA tile (kLinear2) when the activation tile is as
+// large as a weight tile's K slice or close to it (64..128 token rows) and the weight matrix is large:
+// the activation bytes that go from L2 to shared memory per weight byte are halved.  AFLEX_GEMM_DUAL = 0 / 1 forces it off / on (tuning).
+static int linear_mode(int T, int N, int K) {
+    static int force = -2;
+    if (force == -2) { const char* e = getenv("AFLEX_GEMM_DUAL"); force = e ? atoi(e) : -1; }
+    if (N < 2 * kBlockM) return kLinear;
+    if (force == 0) return kLinear;
+    if (force == 1) return kLinear2;
+    const int n_tile = pick_n_tile(T);
+    // measured at the Qwen3-32B shapes: pays on the long down projection (70.6 -> 66.3 us at 128 rows), not on
+    // the short W_o / QKV projections, whose time is fixed cost rather than streaming
+    return (n_tile >= 64 && n_tile <= 128 && (long long)N * K >= (64LL << 20)) ? kLinear2 : kLinear;
+}
+
 static bool make_config(int mode, int T, int N, int K, int rows_max, int E, int num_sms, GemmConfig* cfg) {
     GemmParams& p = cfg->p;
     p.T = T; p.N = N; p.K = K;
@@ -600,7 +637,8 @@ static bool make_config(int mode, int T, int N, int K, int rows_max, int E, int 
         if (cap < 0) { const char* e = getenv("AFLEX_GEMM_NTILE_CAP"); cap = e ? atoi(e) : 0; }
         if (cap >= 16 && p.n_tile > cap) p.n_tile = cap / 16 * 16;
     }
-    p.m_tiles = (N + kBlockM - 1) / kBlockM;
+    p.tile_rows = (mode == kLinear2) ? 2 * kBlockM : kBlockM;
+    p.m_tiles = (N + p.tile_rows - 1) / p.tile_rows;
     p.n_tiles = (T + p.n_tile - 1) / p.n_tile;
     p.kblocks = (K + kBlockK - 1) / kBlockK;
     p.num_experts = E;
@@ -617,7 +655,7 @@ static bool make_config(int mode, int T, int N, int K, int rows_max, int E, int 
     // only on the device: every expert can add one ragged chunk)
     const long long tiles_hi = (E == 0) ? (long long)p.m_tiles * p.n_tiles
                                         : (long long)p.m_tiles * ((T + p.n_tile - 1) / p.n_tile + E);
-    const int accs = (mode == kGateUp ? 2 : 1);
+    const int accs = (mode == kLinear ? 1 : 2);
     const int acc_cols = accs * p.n_tile;
     p.nbuf = (2 * acc_cols <= 512) ? 2 : 1;
     int cols = 32;
@@ -629,7 +667,7 @@ static bool make_config(int mode, int T, int N, int K, int rows_max, int E, int 
     // (large T, compute-bound) make the shared tiles' partials big, so they are shared only when whole
     // tiles alone would leave most SMs idle.
     p.streamk = (tiles_hi < 8LL * num_sms && tiles_hi <= kStreamKMaxTiles && (p.n_tile <= 128 || tiles_hi < 2LL * num_sms)) ? 1 : 0;
-    const int cap = (p.streamk && p.n_tile <= 64) ? streaming_smem_budget() : kMaxDynamicSmem;
+    const int cap = (p.streamk && p.n_tile <= 64 && mode != kLinear2) ? streaming_smem_budget() : kMaxDynamicSmem;
     const int budget = cap - 1024 /*alignment slack*/ - (int)sizeof(GemmBarriers) - 256;
     int stages = budget / stage_bytes;
     if (stages > kMaxStages) stages = kMaxStages;
@@ -692,14 +730,15 @@ static aflex_status bind_scratch(aflex_ctx* ctx, GemmConfig& cfg, char* ws, size
 
 size_t linear_workspace_bytes(int T, int K, int N, int num_sms) {
     GemmConfig cfg;
-    if (!make_config(kLinear, T, N, K, T, 0, num_sms, &cfg)) return 0;
+    if (!make_config(linear_mode(T, N, K), T, N, K, T, 0, num_sms, &cfg)) return 0;
     return cfg.partial_bytes;
 }
 
 aflex_status linear_launch(aflex_ctx* ctx, const void* x, const void* w, int T, int K, int N, void* y, char* ws,
                            size_t ws_bytes, cudaStream_t st, int kind, int* counters) {
     GemmConfig cfg;
-    if (!make_config(kLinear, T, N, K, T, 0, ctx->num_sms, &cfg))
+    const int mode = linear_mode(T, N, K);
+    if (!make_config(mode, T, N, K, T, 0, ctx->num_sms, &cfg))
         return set_error(ctx, AFLEX_ERR_UNSUPPORTED, "linear: no tile configuration fits");
     GemmParams& p = cfg.p;
     p.offsets = nullptr;
@@ -712,6 +751,7 @@ aflex_status linear_launch(aflex_ctx* ctx, const void* x, const void* w, int T, 
     if (!encode_tmap_2d_bf16(&ta, w, (uint64_t)N, (uint64_t)K, (uint64_t)K * 2, kBlockM, kBlockK, true) ||
         !encode_b_set(&tb, x, (uint64_t)T, (uint64_t)K, p.n_tile))
         return set_error(ctx, AFLEX_ERR_CUDA, "linear: cuTensorMapEncodeTiled failed");
+    if (mode == kLinear2) return launch_gemm<kLinear2>(ctx, cfg, ta, ta, tb, st, kind);
     return launch_gemm<kLinear>(ctx, cfg, ta, ta, tb, st, kind);
 }
 

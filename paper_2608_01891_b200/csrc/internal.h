@@ -49,7 +49,7 @@ struct aflex_ctx {
     cudaEvent_t ev_f[aflex::kMaxMicrobatches] = {};   // F_{l,i} done (decoder chain)
     cudaEvent_t ev_f_done = nullptr, ev_a_done = nullptr;
     int attn_ctas = 0;            // persistent attention CTAs per launch; 0 = two per SM
-    bool gemm_attr_set[2] = {false, false};
+    bool gemm_attr_set[3] = {false, false, false};
     bool attn_attr_set[2] = {false, false};
     char err[512] = {0};
     // launch counters (always on) and event-pair timing of every launch (when profiling is enabled)

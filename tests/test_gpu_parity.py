@@ -109,7 +109,8 @@ def test_attention_custom_scale_and_zero_query(ctx):
 
 # ------------------------------------------------------------------------------- GEMMs / dense FFN
 @pytest.mark.parametrize("T,K,N", [(1, 64, 128), (4, 512, 512), (32, 1376, 512), (33, 520, 264), (130, 8192, 640),
-                                   (300, 256, 136), (384, 320, 264), (700, 128, 136)])
+                                   (300, 256, 136), (384, 320, 264), (700, 128, 136),
+                                   (100, 16384, 4104), (64, 8200, 8328)])   # large weights: two weight tiles per CTA tile
 def test_linear_matches_oracle(ctx, T, K, N):
     x, w = rand_bf16((T, K), 1.0, 1), rand_bf16((N, K), 0.05, 2)
     y = torch.full((T, N), float("nan"), dtype=torch.bfloat16, device=DEV)
