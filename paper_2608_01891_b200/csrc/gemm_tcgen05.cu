@@ -406,12 +406,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
             const int n4 = ((pd.c.b_rows + 15) / 16) * 4 * kBlockM;     // float4 slots of one accumulator that were stored
             const int lo = (int)((long long)n4 * me / np), hi = (int)((long long)n4 * (me + 1) / np);
             const int up_off = (p.n_tile >> 2) * kBlockM;               // float4 offset of the "up" accumulator
-            for (int i0 = lo + etid; i0 < hi; i0 += 2 * 128) {
-                const int i1 = i0 + 128;
-                const bool two = i1 < hi;
-                float4 g0 = make_float4(0.f, 0.f, 0.f, 0.f), g1 = g0, u0 = g0, u1 = g0;
+            // kElems float4 per thread and round, all pieces' loads of a round in flight together (the loop is
+            // bound by L2 latency, not bandwidth)
+            constexpr int kElems = (kAccs == 1) ? 4 : 2;
+            for (int i0 = lo + etid; i0 < hi; i0 += kElems * 128) {
+                float4 g[kElems], u[kElems];
+#pragma unroll
+                for (int e = 0; e < kElems; ++e) g[e] = u[e] = make_float4(0.f, 0.f, 0.f, 0.f);
                 for (int cb = cf; cb <= cl; cb += 4) {
-                    float4 a0[4], a1[4], b0[4], b1[4];
+                    float4 a[kElems][4], b[kElems][4];
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
                         const int cc = cb + q;
@@ -420,32 +423,33 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
                             // later unit of that CTA (slot 1); every other piece is a first unit (slot 0)
                             const int sl = (cc == cf && cf_early) ? 1 : 0;
                             const float4* part = reinterpret_cast<const float4*>(p.partials + ((size_t)cc * 2 + sl) * slot_floats);
-                            a0[q] = __ldcg(part + i0);
-                            if (two) a1[q] = __ldcg(part + i1);
-                            if (kAccs == 2) {
-                                b0[q] = __ldcg(part + up_off + i0);
-                                if (two) b1[q] = __ldcg(part + up_off + i1);
+#pragma unroll
+                            for (int e = 0; e < kElems; ++e) {
+                                if (i0 + e * 128 < hi) {
+                                    a[e][q] = __ldcg(part + i0 + e * 128);
+                                    if (kAccs == 2) b[e][q] = __ldcg(part + up_off + i0 + e * 128);
+                                }
                             }
                         }
                     }
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
                         if (cb + q <= cl) {
-                            g0.x += a0[q].x; g0.y += a0[q].y; g0.z += a0[q].z; g0.w += a0[q].w;
-                            if (two) { g1.x += a1[q].x; g1.y += a1[q].y; g1.z += a1[q].z; g1.w += a1[q].w; }
-                            if (kAccs == 2) {
-                                u0.x += b0[q].x; u0.y += b0[q].y; u0.z += b0[q].z; u0.w += b0[q].w;
-                                if (two) { u1.x += b1[q].x; u1.y += b1[q].y; u1.z += b1[q].z; u1.w += b1[q].w; }
+#pragma unroll
+                            for (int e = 0; e < kElems; ++e) {
+                                if (i0 + e * 128 < hi) {
+                                    g[e].x += a[e][q].x; g[e].y += a[e][q].y; g[e].z += a[e][q].z; g[e].w += a[e][q].w;
+                                    if (kAccs == 2) { u[e].x += b[e][q].x; u[e].y += b[e][q].y; u[e].z += b[e][q].z; u[e].w += b[e][q].w; }
+                                }
                             }
                         }
                     }
                 }
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    if (h == 1 && !two) break;
-                    const int idx = h ? i1 : i0;
-                    const float4 gv = h ? g1 : g0, uv = h ? u1 : u0;
-                    const float gf[4] = {gv.x, gv.y, gv.z, gv.w}, uf[4] = {uv.x, uv.y, uv.z, uv.w};
+                for (int e = 0; e < kElems; ++e) {
+                    const int idx = i0 + e * 128;
+                    if (idx >= hi) break;
+                    const float gf[4] = {g[e].x, g[e].y, g[e].z, g[e].w}, uf[4] = {u[e].x, u[e].y, u[e].z, u[e].w};
                     const int r = idx & (kBlockM - 1), cg = idx / kBlockM;
                     const int nl = pd.c.m_tile * p.tile_rows + r;
 #pragma unroll
