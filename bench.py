@@ -169,6 +169,58 @@ def measure_energy(step, barrier, gpu_index, tokens_per_step, ms_step):
         return {"unavailable": str(exc)[:200]}
 
 
+def run_energy_ops(args, cfg, local_rank, device, peaks):
+    """Per-operator time and energy per token at the clocks the GPU is found at (the per-operator side of the paper's
+    Section 3.2 frequency-sensitivity study; the clock sweep itself would need GPU settings to be changed)."""
+    from paper_2608_01891_b200 import aflex as AF
+    wl = build_workload(cfg, device)
+    ctx = AF.Context(local_rank, max(AF.workspace_bytes(wl["layer"], cfg.batch, wl["kvh"].max_pages_per_seq), 6 << 30))
+    stream = torch.cuda.current_stream()
+    dense = dataclasses_replace_dense(cfg)
+    H = cfg.hidden
+    desc = AF.attn_desc(cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim)
+    a_out = torch.empty_like(wl["q"])
+    ops = [("attn_decode", cfg.batch, lambda: ctx.attn_decode(desc, wl["q"], wl["kv"], a_out, None, stream))]
+    if cfg.num_experts == 0:
+        wg, wu, wd = wl["wg"], wl["wu"], wl["wd"]
+    else:
+        wg, wu, wd = IN.make_ffn_weights(dense, device=device)
+    for T in (32, 2048):
+        x = IN.make_x(dense, device=device, tokens=T)
+        y = torch.empty(T, H, dtype=torch.bfloat16, device=device)
+        ops.append((f"ffn_dense(T={T})", T, (lambda x=x, y=y: ctx.ffn_dense(x, wg, wu, wd, y, stream))))
+    ops.append(("layer_step(M=1)", cfg.batch,
+                lambda: ctx.layer_step(wl["layer"], wl["q"], wl["kv"], wl["y"], 1, None, wl["logits"], None, stream)))
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    rows = []
+    for name, tokens, fn in ops:
+        for _ in range(5):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(20):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / 20
+        en = measure_energy(fn, torch.cuda.synchronize, local_rank, tokens, ms)
+        row = {"operator": name, "tokens": tokens, "us": round(ms * 1e3, 1)}
+        if "joules_per_token" in en:
+            row.update({"mj_per_token": round(en["joules_per_token"] * 1e3, 3), "watts_avg": round(en["watts_avg"], 1)})
+        else:
+            row.update(en)
+        rows.append(row)
+    assert ctx.device_status() == AF.OK
+    line = {"metric": "per-operator time and energy per token at default clocks", "unit": "mJ/token", "dtype": "bf16",
+            "data": "synthetic", "config": {"workload": f"config {cfg.cfg_id}: {cfg.name}, operators alone"},
+            "clocks": sampler.stop(), "locked_clock_sweep": "closed on this pool (GPU settings are never changed)",
+            "operators": rows}
+    print(json.dumps(line), flush=True)
+    ctx.close()
+
+
 def run_ffn_sweep(args, cfg, local_rank, device, peaks):
     """Dense SwiGLU FFN at the configuration's (H, I) over a range of token counts: where the FFN stops being
     a weight-streaming kernel and becomes a tensor-core kernel (arithmetic intensity ~ T flop per weight byte)."""
@@ -384,6 +436,9 @@ def main():
                          "(aflex_af_decoder_layers), hidden states handed over by peer copies")
     ap.add_argument("--ffn-device", type=int, default=-1,
                     help="with --af-pair: CUDA device of the FFN side (default: the same GPU as the attention side)")
+    ap.add_argument("--energy-ops", action="store_true",
+                    help="instead of the layer step: time and NVML energy per token of attention, the dense FFN at "
+                         "T = 32 and T = 2048 and the layer step, each alone, at the clocks the GPU is found at")
     ap.add_argument("--energy", action="store_true",
                     help="also read the NVML energy counter around a >= 2 s loop of the step (default clocks)")
     args = ap.parse_args()
@@ -422,6 +477,10 @@ def main():
     if args.decoder_layers > 0:
         if rank == 0:
             run_decoder_chain(args, cfg, local_rank, device, peaks)
+        return
+    if args.energy_ops:
+        if rank == 0:
+            run_energy_ops(args, cfg, local_rank, device, peaks)
         return
     wl = build_workload(cfg, device)
     lens_np = wl["kvh"].seq_lens.numpy()
