@@ -608,7 +608,15 @@ def main():
         rows = list(range(min(args.ref_rows, cfg.batch)))
         dt, threads = oracle_sample(cfg, wl, rows)
         cpu = {"value": len(rows) / dt, "unit": "tokens/s", "cores": threads, "kind": "oracle", "seconds": round(dt, 2),
+               "host_cpus": os.cpu_count(),
                "sample": f"fp64 oracle layer step on batch rows {rows[0]}..{rows[-1]} of {cfg.batch} (rows are independent)"}
+        if cfg.cfg_id == 1:
+            # the tiny configuration also gets a single-thread figure
+            from oracle import oracle as O
+            O.set_num_threads(1)
+            dt1, _ = oracle_sample(cfg, wl, rows)
+            O.set_num_threads(threads)
+            cpu["value_1_thread"] = len(rows) / dt1
 
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
