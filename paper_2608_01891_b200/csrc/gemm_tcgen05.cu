@@ -670,7 +670,9 @@ static bool make_config(int mode, int T, int N, int K, int rows_max, int E, int 
     // few tiles per SM: share the remainder tiles along K; many: whole tiles round-robin.  Wide tiles
     // (large T, compute-bound) make the shared tiles' partials big, so they are shared only when whole
     // tiles alone would leave most SMs idle.
-    p.streamk = (tiles_hi < 8LL * num_sms && tiles_hi <= kStreamKMaxTiles && (p.n_tile <= 128 || tiles_hi < 2LL * num_sms)) ? 1 : 0;
+    static int nostream = -1;   // AFLEX_GEMM_NOSTREAMK=1: whole tiles only (measurement of per-SM streaming rates)
+    if (nostream < 0) { const char* e = getenv("AFLEX_GEMM_NOSTREAMK"); nostream = e ? atoi(e) : 0; }
+    p.streamk = nostream ? 0 : (tiles_hi < 8LL * num_sms && tiles_hi <= kStreamKMaxTiles && (p.n_tile <= 128 || tiles_hi < 2LL * num_sms)) ? 1 : 0;
     const int cap = (p.streamk && p.n_tile <= 64 && mode != kLinear2) ? streaming_smem_budget() : kMaxDynamicSmem;
     const int budget = cap - 1024 /*alignment slack*/ - (int)sizeof(GemmBarriers) - 256;
     int stages = budget / stage_bytes;
