@@ -487,6 +487,9 @@ def main():
     M = args.depth
     ws = AF.workspace_bytes(wl["layer"], cfg.batch, wl["kvh"].max_pages_per_seq)
     ctx = AF.Context(local_rank, ws)
+    # q is a resident tensor (value) or arrives by a host-to-device copy (e2e), never as the output of the library
+    # kernel enqueued just before the step: the documented promise that lets attention read it with its other inputs
+    ctx.set_attn_q_final(True)
     if args.attn_ctas:
         ctx.set_attn_ctas(args.attn_ctas)
     stream = torch.cuda.current_stream()

@@ -29,9 +29,9 @@
  *    device and must be used by one host thread at a time.  Calls that use the
  *    same ctx must be stream-ordered with respect to each other (they share the
  *    workspace); aflex_layer_step orders its own internal streams.
- *  - Kernels are launched with programmatic stream serialization and read their
- *    INPUT tensors (q, KV cache, page table, lengths, weights) before the grid
- *    dependency resolves.  This is invisible to ordinary callers (a preceding
+ *  - Kernels are launched with programmatic stream serialization and read some
+ *    INPUT tensors (KV cache, page table, lengths, weights - not activations such
+ *    as q or x) before the grid dependency resolves.  This is invisible to ordinary callers (a preceding
  *    kernel, copy or event wait in the stream completes first, as usual); only a
  *    caller's own kernel that releases its dependents early
  *    (cudaTriggerProgrammaticLaunchCompletion) must not be the producer of those
@@ -275,6 +275,13 @@ AFLEX_API aflex_status aflex_linear(aflex_ctx* ctx, const void* x, const void* w
 /* Tuning knob: number of persistent attention CTAs per launch, 1..4096 (0 = automatic: two per
  * SM).  It changes how the KV cache is split across CTAs, never the result beyond rounding. */
 AFLEX_API aflex_status aflex_set_attn_ctas(aflex_ctx* ctx, int ctas);
+
+/* A promise about q in aflex_attn_decode / aflex_layer_step on this ctx (default off).  on != 0: q is never the
+ * output of the library kernel enqueued directly before the call (aflex_linear, aflex_ffn_*, aflex_layer_step);
+ * the attention kernel may then read q before its grid dependency resolves, like its other inputs, and starts
+ * computing while the preceding kernel drains.  q written by aflex_rope_append, by a caller's kernel, by a copy,
+ * or resident from earlier work satisfies the promise. */
+AFLEX_API aflex_status aflex_set_attn_q_final(aflex_ctx* ctx, int on);
 
 /* ---- Whole decoder layers, chained (Section 4.3, "Interleaved A/F Pipeline") -------------
  *

@@ -399,6 +399,12 @@ aflex_status aflex_trace_read(aflex_ctx* ctx, unsigned long long* host_out, int 
     return check_cuda(ctx, e, "aflex_trace_read");
 }
 
+aflex_status aflex_set_attn_q_final(aflex_ctx* ctx, int on) {
+    if (!ctx) return AFLEX_ERR_INVALID_ARG;
+    ctx->attn_q_final = on != 0;
+    return AFLEX_OK;
+}
+
 aflex_status aflex_set_attn_ctas(aflex_ctx* ctx, int ctas) {
     if (!ctx || ctas < 0 || ctas > 4096) return AFLEX_ERR_INVALID_ARG;
     ctx->attn_ctas = ctas;
@@ -769,6 +775,7 @@ aflex_status aflex_decoder_layers(aflex_ctx* ctx, const aflex_decoder_desc* laye
             kvi.seq_lens_host = kvs[l].seq_lens_host ? kvs[l].seq_lens_host + r0 : nullptr;
             s = rope_append_launch(ctx, &L->attn, qkv + (size_t)r0 * NQ, &kvi, rows, d->w_q_norm, d->w_k_norm, d->rms_eps, d->rope_theta, qb + (size_t)r0 * A, sa);
             if (s != AFLEX_OK) return s;
+            ctx->attn_q_final_once = true;      // q was written by the append kernel, which does not release its dependents early
             s = attn_decode_launch(ctx, &L->attn, qb + (size_t)r0 * A, &kvi, rows, ab + (size_t)r0 * A, nullptr, ws_attn, w.a_attn, sa);
             if (s != AFLEX_OK) return s;
             s = linear_launch(ctx, ab + (size_t)r0 * A, L->w_o, rows, A, H, ob + oh, ws_lin, w.a_lin, sa, kKLinearGemm, ctx->counters_a);
@@ -905,6 +912,7 @@ aflex_status aflex_af_decoder_layers(aflex_ctx* ca, aflex_ctx* cf, const aflex_d
             kvi.seq_lens_host = kvs[l].seq_lens_host ? kvs[l].seq_lens_host + r0 : nullptr;
             s = rope_append_launch(ca, &L->attn, qkv + (size_t)r0 * NQ, &kvi, rows, d->w_q_norm, d->w_k_norm, d->rms_eps, d->rope_theta, qb + (size_t)r0 * A, sa);
             if (s != AFLEX_OK) return s;
+            ca->attn_q_final_once = true;
             s = attn_decode_launch(ca, &L->attn, qb + (size_t)r0 * A, &kvi, rows, ab + (size_t)r0 * A, nullptr, ws_attn, w.a_attn, sa);
             if (s != AFLEX_OK) return s;
             s = linear_launch(ca, ab + (size_t)r0 * A, L->w_o, rows, A, H, ob + oh, ws_lin, w.a_lin, sa, kKLinearGemm, ca->counters_a);

@@ -68,6 +68,7 @@ struct AttnParams {
     int dyn_pct;           // percent of the unit list handed out dynamically (0 = static shares only)
     int dyn_chunks;        // target number of dynamic chunks per CTA
     int kv_policy;         // 0: evict-first KV loads, 1: normal priority (tuning)
+    int q_final;           // 1: q is final when the kernel starts (its first loads need not wait for the grid dependency)
     int dyn_min;           // chunk size (units) the dynamic tail aims at
     int piece_cost;        // list positions charged per item start (balances the fixed cost of a piece)
     int* status;
@@ -374,10 +375,12 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         }
     } else if (warp < kAttnConsumerWarps) {
         // ------------------------------------------------------------------ compute warps
-        // q is final when this kernel starts (an input of the step, or written by the K/V append kernel,
-        // which does not release its dependents early), so pages are processed at once.  These warps
-        // never write to global memory: a finished piece's state goes to the epilogue warp through the
-        // piece's last stage buffer.
+        // q may be the output of the kernel just before this one (a projection GEMM of this library releases
+        // its dependents early), so unless the launcher knows better (q written by the K/V append kernel, which
+        // does not release early, or the caller's promise) these warps wait for the grid dependency before
+        // their first q load; the ring fills meanwhile.  They never write to global memory: a finished
+        // piece's state goes to the epilogue warp through the piece's last stage buffer.
+        if (!p.q_final) pdl_wait();
         const int mi = lane >> 3, r8 = lane & 7;
         int s = 0;
         uint32_t ph = 0;
@@ -817,6 +820,8 @@ static aflex_status attn_launch_t(aflex_ctx* ctx, const aflex_attn_desc* d, cons
     p.dyn_pct = attn_dyn_pct();
     p.dyn_chunks = attn_dyn_chunks();
     p.piece_cost = attn_piece_cost();
+    p.q_final = (ctx->attn_q_final || ctx->attn_q_final_once) ? 1 : 0;
+    ctx->attn_q_final_once = false;
     { static int v = -1; if (v < 0) { const char* e = getenv("AFLEX_ATTN_DYN_UNITS"); v = e ? atoi(e) : 16; if (v < 1) v = 1; } p.dyn_min = v; }
     { static int v = -1; if (v < 0) { const char* e = getenv("AFLEX_ATTN_KVPOL"); v = e ? atoi(e) : 0; } p.kv_policy = v; }
     p.status = ctx->dev_status;
@@ -929,6 +934,7 @@ static aflex_status attn_static_launch(StaticDeviceState& stt, const aflex_attn_
     p.dyn_pct = 0;
     p.dyn_chunks = 1;
     p.kv_policy = 0;
+    p.q_final = 0;
     p.dyn_min = 12;
     p.piece_cost = 0;
     p.trace = nullptr;

@@ -395,3 +395,31 @@ def test_sequence_length_beyond_the_page_table_row_is_clamped_and_reported(ctx):
     want, _ = O.attn_decode(u16(q), u16(kv.k_cache), u16(kv.v_cache), kv.page_table.numpy(), kv.seq_lens.numpy())
     assert row_rel_err(got, want) <= TOL_ATTN
     assert ctx.device_status() == AF.OK
+
+
+def test_attention_waits_for_a_query_produced_by_the_preceding_gemm(ctx):
+    """q = x Wq^T by aflex_linear, attention enqueued right behind it: the projection releases its dependents
+    early, so the attention kernel must not read q before the grid dependency resolves (default behaviour)."""
+    cfg = IN.CONFIGS[1]
+    B, Hq, Hkv, D = 64, cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim
+    lens = np.random.default_rng(5).integers(1, 200, size=B).astype(np.int32)
+    kvh = IN.make_paged_kv(cfg, lens)
+    kv = AF.make_kv(kvh.k_cache.to(DEV), kvh.v_cache.to(DEV), kvh.page_table.to(DEV), kvh.seq_lens.to(DEV), kvh.seq_lens)
+    K = 16384                                            # long enough for the GEMM to still run when attention starts
+    x = rand_bf16((B, K), 1.0, 11).to(DEV)
+    wq = rand_bf16((Hq * D, K), 0.01, 12).to(DEV)
+    desc = AF.attn_desc(Hq, Hkv, D)
+    q_ref = torch.empty(B, Hq * D, dtype=torch.bfloat16, device=DEV)
+    ctx.linear(x, wq, q_ref)
+    torch.cuda.synchronize()
+    out_ref = torch.empty(B, Hq, D, dtype=torch.bfloat16, device=DEV)
+    ctx.attn_decode(desc, q_ref.view(B, Hq, D), kv, out_ref)
+    torch.cuda.synchronize()
+    for _ in range(20):
+        q = torch.full((B, Hq * D), float("nan"), dtype=torch.bfloat16, device=DEV)
+        out = torch.empty_like(out_ref)
+        ctx.linear(x, wq, q)
+        ctx.attn_decode(desc, q.view(B, Hq, D), kv, out)
+        torch.cuda.synchronize()
+        assert torch.equal(out.view(torch.int16), out_ref.view(torch.int16))
+    assert ctx.device_status() == AF.OK
