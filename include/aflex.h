@@ -36,6 +36,10 @@
  *    caller's own kernel that releases its dependents early
  *    (cudaTriggerProgrammaticLaunchCompletion) must not be the producer of those
  *    inputs.  Outputs and scratch are touched only after the dependency resolves.
+ *  - The enqueueing calls (aflex_attn_decode, aflex_ffn_*, aflex_layer_step, aflex_decoder_layers, ...) can be
+ *    captured into a CUDA graph on `stream` after one un-captured warm-up call with the same shapes (the first
+ *    call sets kernel attributes and fills the host-side tensor-map cache); with a microbatch depth >= 2 the
+ *    ctx's internal streams are forked from and joined to `stream`, so they become part of the capture.
  *  - Device-side waits are bounded: if one expires the kernel records
  *    AFLEX_ERR_TIMEOUT in the ctx status word and exits cleanly; read it with
  *    aflex_get_device_status.

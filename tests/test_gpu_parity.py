@@ -423,3 +423,30 @@ def test_attention_waits_for_a_query_produced_by_the_preceding_gemm(ctx):
         torch.cuda.synchronize()
         assert torch.equal(out.view(torch.int16), out_ref.view(torch.int16))
     assert ctx.device_status() == AF.OK
+
+
+@pytest.mark.parametrize("M", [1, 2])
+def test_layer_step_replays_from_a_cuda_graph(ctx, M):
+    """The layer step (one stream at M = 1, the ctx's two streams joined to the caller's at M >= 2) captured
+    into a CUDA graph after a warm-up call, replayed twice: same bits as the eager call."""
+    cfg = IN.CONFIGS[1]
+    kvh = IN.make_paged_kv(cfg)
+    kv = AF.make_kv(kvh.k_cache.to(DEV), kvh.v_cache.to(DEV), kvh.page_table.to(DEV), kvh.seq_lens.to(DEV), kvh.seq_lens)
+    q, wo = IN.make_q(cfg).to(DEV), IN.make_wo(cfg).to(DEV)
+    wg, wu, wd = (t.to(DEV) for t in IN.make_ffn_weights(cfg))
+    layer = AF.layer_desc(AF.attn_desc(cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim), cfg.hidden, cfg.inter, wo, wg, wu, wd)
+    y = torch.zeros(cfg.batch, cfg.hidden, dtype=torch.bfloat16, device=DEV)
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        ctx.layer_step(layer, q, kv, y, M, None, None, None, s)      # warm-up: sets kernel attributes, fills caches
+        s.synchronize()
+        want = y.clone()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            ctx.layer_step(layer, q, kv, y, M, None, None, None, s)
+        for _ in range(2):
+            y.zero_()
+            g.replay()
+            s.synchronize()
+            assert torch.equal(y.view(torch.int16), want.view(torch.int16))
+    assert ctx.device_status() == AF.OK
