@@ -506,3 +506,49 @@ ORACLE_API void oracle_decoder_layer(const double* x, const uint16_t* w_ln_attn,
     if (!h1_out) free(h1);
     free(a); free(xn); free(f);
 }
+
+/* ------------------------------------------------------------------------- */
+/* Prefill (causal) attention over the paged cache, the attention operator of  */
+/* the prefill phase (the paper's PA pool).  Sequence b has n = seq_lens[b]     */
+/* cached tokens of which the last m = q_offsets[b+1] - q_offsets[b] are the    */
+/* ones being prefilled; query i (0 <= i < m) sits at position n - m + i and    */
+/* attends to the cached tokens 0 .. n - m + i (itself included), nothing       */
+/* later:                                                                       */
+/*   s_j = scale * <q_i, k_j>, p = softmax over j <= pos_i, o_i = sum_j p_j v_j */
+/*   q bf16 [T][Hq][D] (T = q_offsets[B], queries of sequence b at rows          */
+/*   q_offsets[b] ..); caches, page table as for decode; out f64 [T][Hq][D].     */
+/* ------------------------------------------------------------------------- */
+ORACLE_API void oracle_attn_prefill(const uint16_t* q, const uint16_t* k_cache, const uint16_t* v_cache,
+                                    const int32_t* page_table, int max_pages, const int32_t* seq_lens,
+                                    const int32_t* q_offsets, int B, int Hq, int Hkv, int D, int P, double scale,
+                                    double* out) {
+    const int G = Hq / Hkv;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int b = 0; b < B; ++b) {
+        const int n = seq_lens[b];
+        const int m = q_offsets[b + 1] - q_offsets[b];
+        double* keys = (double*)malloc(sizeof(double) * (size_t)n * D);
+        double* vals = (double*)malloc(sizeof(double) * (size_t)n * D);
+        double* qd = (double*)malloc(sizeof(double) * (size_t)D);
+        for (int g = 0; g < Hkv; ++g) {
+            for (int j = 0; j < n; ++j) {
+                const int64_t page = page_table[(size_t)b * max_pages + j / P];
+                const size_t base = (((size_t)page * Hkv + g) * P + (size_t)(j % P)) * (size_t)D;
+                for (int d = 0; d < D; ++d) {
+                    keys[(size_t)j * D + d] = bf16_to_f64(k_cache[base + d]);
+                    vals[(size_t)j * D + d] = bf16_to_f64(v_cache[base + d]);
+                }
+            }
+            for (int i = 0; i < m; ++i) {
+                const int visible = n - m + i + 1;          /* keys 0 .. pos_i */
+                const size_t row = (size_t)q_offsets[b] + i;
+                for (int hh = 0; hh < G; ++hh) {
+                    const int h = g * G + hh;
+                    for (int d = 0; d < D; ++d) qd[d] = bf16_to_f64(q[(row * Hq + h) * D + d]);
+                    oracle_attn_one_query_f64(qd, keys, vals, visible, D, scale, out + (row * Hq + h) * D, NULL);
+                }
+            }
+        }
+        free(keys); free(vals); free(qd);
+    }
+}

@@ -355,3 +355,25 @@ def decoder_layer(x, w, k_cache, v_cache, page_table, seq_lens, num_q_heads: int
                                  _p(logits, _f32p) if (E and g.get("router") is None) else None,
                                  _p(q, _f64p), _p(h1, _f64p), _p(out, _f64p))
     return q, h1, out
+
+
+def attn_prefill(q, k_cache, v_cache, page_table, seq_lens, q_offsets, scale: Optional[float] = None) -> np.ndarray:
+    """Causal attention of the last q_len tokens of every sequence over its paged cache.
+    q u16 [T,Hq,D] (T = q_offsets[-1]); seq_lens i32 [B] (cached tokens incl. the prefilled ones);
+    q_offsets i32 [B+1] -> out f64 [T,Hq,D]."""
+    q, k_cache, v_cache = _u16(q), _u16(k_cache), _u16(v_cache)
+    page_table = np.ascontiguousarray(page_table, dtype=np.int32)
+    seq_lens = np.ascontiguousarray(seq_lens, dtype=np.int32)
+    q_offsets = np.ascontiguousarray(q_offsets, dtype=np.int32)
+    T, Hq, D = q.shape
+    _, Hkv, P, _ = k_cache.shape
+    B = seq_lens.shape[0]
+    assert q_offsets.shape == (B + 1,) and q_offsets[0] == 0 and q_offsets[-1] == T
+    assert ((q_offsets[1:] - q_offsets[:-1]) <= seq_lens).all() and ((q_offsets[1:] - q_offsets[:-1]) >= 0).all()
+    if scale is None:
+        scale = 1.0 / np.sqrt(float(D))
+    out = np.zeros((T, Hq, D), dtype=np.float64)
+    _load().oracle_attn_prefill(_p(q, _u16p), _p(k_cache, _u16p), _p(v_cache, _u16p), _p(page_table, _i32p),
+                                int(page_table.shape[1]), _p(seq_lens, _i32p), _p(q_offsets, _i32p), B, Hq, Hkv, D, P,
+                                ctypes.c_double(scale), _p(out, _f64p))
+    return out

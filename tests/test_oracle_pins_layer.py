@@ -245,3 +245,57 @@ def test_decoder_layer_one_expert_equals_dense():
     wd = dict(w, gate=w["gate"][0], up=w["up"][0], down=w["down"][0], router=None)
     _, _, out_dense = O.decoder_layer(x, wd, k2, v2, table, lens, 4, 1e-6, 1e4)
     np.testing.assert_allclose(out_moe, out_dense, rtol=0, atol=1e-13)
+
+
+# --------------------------------------------------------------------------- prefill (causal) attention
+def _prefill_case(rng, lens, q_lens, Hq=4, Hkv=2, D=8):
+    P = IN.PAGE_SIZE
+    lens = np.asarray(lens, dtype=np.int32)
+    pages = (lens + P - 1) // P
+    num_pages = int(pages.sum()) + 2
+    perm = rng.permutation(num_pages)
+    table = np.zeros((len(lens), int(pages.max())), dtype=np.int32)
+    o = 0
+    for b in range(len(lens)):
+        table[b, :pages[b]] = perm[o:o + pages[b]]
+        o += int(pages[b])
+    k = bf16(rng.standard_normal((num_pages, Hkv, P, D)))
+    v = bf16(rng.standard_normal((num_pages, Hkv, P, D)))
+    q_off = np.concatenate([[0], np.cumsum(q_lens)]).astype(np.int32)
+    q = bf16(rng.standard_normal((int(q_off[-1]), Hq, D)))
+    return q, k, v, table, lens, q_off
+
+
+def test_prefill_with_one_query_per_sequence_is_decode_attention():
+    rng = np.random.default_rng(20)
+    q, k, v, table, lens, q_off = _prefill_case(rng, (5, 33, 16), (1, 1, 1))
+    got = O.attn_prefill(q, k, v, table, lens, q_off)
+    want, _ = O.attn_decode(q, k, v, table, lens)
+    np.testing.assert_array_equal(got, want)
+
+
+def test_prefill_is_causal_row_by_row():
+    # query i of a sequence sees exactly the cached tokens up to its own position: the same as decoding with a
+    # sequence length cut at that position
+    rng = np.random.default_rng(21)
+    q, k, v, table, lens, q_off = _prefill_case(rng, (20, 37), (20, 9))
+    got = O.attn_prefill(q, k, v, table, lens, q_off)
+    for b in range(2):
+        m = int(q_off[b + 1] - q_off[b])
+        for i in range(m):
+            row = int(q_off[b]) + i
+            cut = np.array([int(lens[b]) - m + i + 1], dtype=np.int32)
+            want, _ = O.attn_decode(q[row:row + 1], k, v, table[b:b + 1], cut)
+            np.testing.assert_array_equal(got[row], want[0])
+    # the first token of a full prefill attends to itself only: its output is its own value row
+    vals = bf16_to_f64(v)
+    first = vals[table[0, 0], :, 0, :]                      # [Hkv, D]
+    np.testing.assert_array_equal(got[0], np.repeat(first, 2, axis=0))
+    # a later key cannot influence an earlier query
+    k2, v2 = k.copy(), v.copy()
+    last_page, last_slot = table[0, 19 // 16], 19 % 16
+    k2[last_page, :, last_slot] = bf16(np.full((2, 8), 50.0))
+    v2[last_page, :, last_slot] = bf16(np.full((2, 8), -7.0))
+    got2 = O.attn_prefill(q, k2, v2, table, lens, q_off)
+    np.testing.assert_array_equal(got2[:19], got[:19])
+    assert np.abs(got2[19] - got[19]).max() > 1e-3
