@@ -182,6 +182,23 @@ AFLEX_API aflex_status aflex_attn_decode(aflex_ctx* ctx, const aflex_attn_desc* 
 AFLEX_API aflex_status aflex_attn_decode_static(const aflex_attn_desc* desc, const void* q, const aflex_kv* kv,
                                                 int batch, void* out, float* lse, void* stream);
 
+/*
+ * Prefill (causal) attention: the attention operator of the prefill phase (the paper's "PA" pool; Section 1: in
+ * prefill both operators are dominated by matrix multiplications).  Sequence b has n = seq_lens[b] cached tokens,
+ * of which the last m = q_offsets[b+1] - q_offsets[b] are being prefilled (m = n: a whole prompt; m < n: a chunk
+ * behind an existing context).  Query i (0 <= i < m) sits at position n - m + i and attends to the cached tokens
+ * 0 .. n - m + i, itself included:
+ *     s_j = sm_scale * <q_i, K_j>,  p = softmax over j <= n - m + i,  out_i = sum_j p_j V_j  -> bf16
+ * q, out: bf16 [T][Hq][D] with T = q_offsets[batch], the queries of sequence b at rows q_offsets[b] ..;
+ * q_offsets: DEVICE i32 [batch + 1]; q_offsets_host: HOST copy of the same (sizes the launch); kv as for
+ * aflex_attn_decode, the K/V of the prefilled tokens already in the cache.  Runs on the tcgen05 tensor cores
+ * (fp32 scores and accumulation, P rounded to bf16 before the P V product).  Errors as aflex_attn_decode, plus
+ * INVALID_ARG for inconsistent offsets.
+ */
+AFLEX_API aflex_status aflex_attn_prefill(aflex_ctx* ctx, const aflex_attn_desc* desc, const void* q, const aflex_kv* kv,
+                                          int batch, const int32_t* q_offsets, const int32_t* q_offsets_host, void* out,
+                                          void* stream);
+
 /* ---- FFN side -------------------------------------------------------------
  *
  * Dense SwiGLU FFN (the decode FFN operator of the paper's Section 1: weight

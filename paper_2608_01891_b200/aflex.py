@@ -25,7 +25,7 @@ EXPORTS = (
     "aflex_workspace_bytes", "aflex_linear", "aflex_set_attn_ctas", "aflex_set_attn_q_final", "aflex_num_kernel_kinds",
     "aflex_kernel_name", "aflex_launch_count", "aflex_profile_enable", "aflex_profile_read",
     "aflex_trace_read", "aflex_attn_decode_static", "aflex_decoder_layers", "aflex_decoder_workspace_bytes",
-    "aflex_add_rmsnorm", "aflex_rope_append", "aflex_af_decoder_layers", "aflex_af_workspace_bytes",
+    "aflex_add_rmsnorm", "aflex_rope_append", "aflex_attn_prefill", "aflex_af_decoder_layers", "aflex_af_workspace_bytes",
     "aflex_eq2_layer_time", "aflex_curve_eval",
     "aflex_pipeline_makespan", "aflex_plan_microbatches", "aflex_dvfs_window", "aflex_dvfs_decode_step",
     "aflex_dvfs_prefill_pair",
@@ -114,6 +114,8 @@ def load_library() -> ctypes.CDLL:
     lib.aflex_set_attn_q_final.argtypes = [vp, ci]
     lib.aflex_attn_decode.restype = ci
     lib.aflex_attn_decode.argtypes = [vp, ctypes.POINTER(AttnDesc), vp, ctypes.POINTER(KV), ci, vp, vp, vp]
+    lib.aflex_attn_prefill.restype = ci
+    lib.aflex_attn_prefill.argtypes = [vp, ctypes.POINTER(AttnDesc), vp, ctypes.POINTER(KV), ci, vp, vp, vp, vp]
     lib.aflex_linear.restype = ci
     lib.aflex_linear.argtypes = [vp, vp, vp, ci, ci, ci, vp, vp]
     lib.aflex_ffn_dense.restype = ci
@@ -414,6 +416,15 @@ class Context:
                     lse: Optional[torch.Tensor] = None, stream=None) -> None:
         self._check(self._lib.aflex_attn_decode(self._h, ctypes.byref(desc), _ptr(q), ctypes.byref(kv),
                                                 q.shape[0], _ptr(out), _ptr(lse), _stream(stream)))
+
+    def attn_prefill(self, desc: AttnDesc, q: torch.Tensor, kv: KV, q_offsets: torch.Tensor,
+                     q_offsets_host: torch.Tensor, out: torch.Tensor, stream=None) -> None:
+        """Causal attention of the last q_len tokens of every sequence over its paged cache.  q, out bf16
+        [T,Hq,D]; q_offsets i32 CUDA [B+1]; q_offsets_host the same on the CPU."""
+        assert q_offsets.dtype == torch.int32 and q_offsets_host.dtype == torch.int32 and q_offsets_host.device.type == "cpu"
+        self._check(self._lib.aflex_attn_prefill(self._h, ctypes.byref(desc), _ptr(q), ctypes.byref(kv),
+                                                 q_offsets_host.shape[0] - 1, _ptr(q_offsets), _ptr(q_offsets_host),
+                                                 _ptr(out), _stream(stream)))
 
     def linear(self, x: torch.Tensor, w: torch.Tensor, y: torch.Tensor, stream=None) -> None:
         T, K = x.shape

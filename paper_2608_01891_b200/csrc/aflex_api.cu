@@ -342,7 +342,7 @@ aflex_status aflex_get_device_status(aflex_ctx* ctx, void* stream) {
 static const char* kKernelNames[kKKindCount] = {
     "attn_decode", "linear_gemm", "down_gemm", "gateup_gemm", "router_logits",
     "moe_route", "moe_gather", "moe_gateup_gemm", "moe_down_gemm", "moe_combine",
-    "add_rmsnorm", "qkv_gemm", "rope_append"};
+    "add_rmsnorm", "qkv_gemm", "rope_append", "attn_prefill"};
 
 int aflex_num_kernel_kinds(void) { return kKKindCount; }
 
@@ -417,6 +417,19 @@ aflex_status aflex_attn_decode(aflex_ctx* ctx, const aflex_attn_desc* desc, cons
     if (s != AFLEX_OK) return s;
     return attn_decode_launch(ctx, desc, q, kv, batch, out, lse, ctx->ws, ctx->ws_bytes,
                               reinterpret_cast<cudaStream_t>(stream));
+}
+
+aflex_status aflex_attn_prefill(aflex_ctx* ctx, const aflex_attn_desc* desc, const void* q, const aflex_kv* kv, int batch,
+                                const int32_t* q_offsets, const int32_t* q_offsets_host, void* out, void* stream) {
+    aflex_status s = validate_attn(ctx, desc, q, kv, batch, out);
+    if (s != AFLEX_OK) return s;
+    if (!q_offsets || !q_offsets_host) return set_error(ctx, AFLEX_ERR_INVALID_ARG, "prefill attention: null q_offsets");
+    if (kv->seq_lens_host) {
+        for (int b = 0; b < batch; ++b)
+            if (q_offsets_host[b + 1] - q_offsets_host[b] > kv->seq_lens_host[b])
+                return set_error(ctx, AFLEX_ERR_INVALID_ARG, "prefill attention: sequence %d has more queries than cached tokens", b);
+    }
+    return attn_prefill_launch(ctx, desc, q, kv, batch, q_offsets, q_offsets_host, out, reinterpret_cast<cudaStream_t>(stream));
 }
 
 aflex_status aflex_linear(aflex_ctx* ctx, const void* x, const void* w, int T, int K, int N, void* y, void* stream) {

@@ -1,0 +1,397 @@
+// Prefill (causal) attention over the paged KV cache: the attention operator of the prefill phase
+// (the paper's PA pool; Section 1: during prefill both operators are dominated by matrix
+// multiplications).  Compute-bound, so it runs on the 5th-generation tensor cores:
+//
+//   tile        = 128 consecutive query tokens of one query head against 128 cached tokens at a time
+//   S = Q K^T   tcgen05.mma, both operands K-major (Q tile and K tile rows of D contiguous elements,
+//               128-byte swizzle as TMA writes them), fp32 accumulator in TMEM, double-buffered
+//   softmax     four warps, one query row per thread: tcgen05.ld of its S row, causal mask, online
+//               max / sum in base 2, P rounded to bf16 into shared memory as the next MMA's A operand
+//   O += P V    tcgen05.mma with V exactly as the cache stores it ([token][D]: an MN-major B operand),
+//               accumulator in TMEM; rescaled in place (tcgen05.ld / st) when a row's maximum moves
+//   pipeline    a producer warp issues the TMA loads of the K and V pages of the next tile (2 stages)
+//               while one thread issues MMAs and S of tile t+1 is computed during the softmax of tile t
+//
+// Query i of a sequence with n cached tokens of which the last m are being prefilled sits at position
+// n - m + i and sees cached tokens 0 .. n - m + i.  Cache slots beyond n may hold anything (NaN too):
+// their scores are replaced by -inf and their V rows are zeroed in shared memory before use.
+#include <cuda_bf16.h>
+#include <math.h>
+
+#include "internal.h"
+#include "ptx.cuh"
+
+namespace aflex {
+namespace pa {
+
+constexpr int kBM = 128;          // query rows per tile
+constexpr int kBN = 128;          // cached tokens per step
+constexpr int kPage = 16;
+constexpr int kPagesPerTile = kBN / kPage;
+constexpr int kStages = 2;
+constexpr int kThreads = 6 * 32;  // producer, MMA issuer, four softmax warps
+constexpr float kNegBig = -1.0e30f;
+
+struct Params {
+    const int32_t* page_table;
+    const int32_t* seq_lens;      // cached tokens per sequence, the prefilled ones included
+    const int32_t* q_offsets;     // [B+1] first query row of every sequence
+    int batch, max_pages, Hq, Hkv, G;
+    long long num_pages;
+    int total_tiles;              // sum over sequences of ceil(q_len / 128)
+    float scale_log2;
+    __nv_bfloat16* out;           // [T][Hq][D]
+    int* status;
+};
+
+struct __align__(8) Shared {
+    uint64_t q_full;
+    uint64_t kv_full[kStages], kv_empty[kStages];
+    uint64_t s_ready[2], s_free[2];
+    uint64_t p_ready, pv_done;
+    uint32_t tmem_base;
+    volatile int abort;
+};
+
+__device__ __forceinline__ void tmem_st_32x32b_x16(uint32_t taddr, const uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// Shared-memory descriptor of an MN-major bf16 operand stored as [K rows][64 MN elements] blocks of 128-byte
+// swizzled rows: 8-row groups 1024 B apart (stride byte offset), 64-element MN blocks `mn_block_bytes` apart
+// (leading byte offset).
+__device__ __forceinline__ uint64_t umma_desc_mn_sw128(uint32_t smem_addr, uint32_t mn_block_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFF) >> 4);
+    d |= (uint64_t)((mn_block_bytes >> 4) & 0x3FFF) << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+
+template <int D>
+__global__ void __launch_bounds__(kThreads, 1)
+attn_prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
+                    const __grid_constant__ CUtensorMap tmap_v, const Params p) {
+    constexpr int kHalves = D / 64;
+    constexpr int kHalfBytes = kBN * 128;               // 128 rows of 128 B
+    constexpr int kQBytes = kHalves * kHalfBytes;
+    constexpr int kKVStage = 2 * kHalves * kHalfBytes;   // K then V
+    constexpr int kPBytes = 2 * kHalfBytes;
+    constexpr uint32_t kSCol = 0, kOCol = 2 * kBN;       // TMEM columns: S buffers at 0 and 128, O after them
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t* sq = smem;
+    uint8_t* skv = sq + kQBytes;
+    uint8_t* sp = skv + kStages * kKVStage;
+    Shared* sh = reinterpret_cast<Shared*>(sp + kPBytes);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    // ---- which tile: query head fastest (the heads of a group share K/V tiles in L2), long tiles first
+    const int h = blockIdx.x % p.Hq;
+    const int tile_id = p.total_tiles - 1 - (int)(blockIdx.x / p.Hq);
+    int b = 0, tile_in_seq = 0;
+    {
+        int acc = 0;
+        for (b = 0; b < p.batch; ++b) {
+            const int m = p.q_offsets[b + 1] - p.q_offsets[b];
+            const int nt = (m + kBM - 1) / kBM;
+            if (tile_id < acc + nt) { tile_in_seq = tile_id - acc; break; }
+            acc += nt;
+        }
+        if (b >= p.batch) return;                       // cannot happen with a consistent total_tiles
+    }
+    const int q_row0 = p.q_offsets[b] + tile_in_seq * kBM;
+    const int q_len = p.q_offsets[b + 1] - p.q_offsets[b];
+    const int rows_valid = min(kBM, q_len - tile_in_seq * kBM);
+    int n_cached = p.seq_lens[b];
+    {
+        const int cap = p.max_pages * kPage;
+        if (n_cached > cap || n_cached < q_len) { if (threadIdx.x == 0) atomicExch(p.status, AFLEX_ERR_BOUNDS); n_cached = max(min(n_cached, cap), q_len); }
+    }
+    const int pos0 = n_cached - q_len + tile_in_seq * kBM;          // position of the tile's first query
+    const int kv_end = pos0 + rows_valid;                           // cached tokens visible to the tile's last query
+    const int n_steps = (kv_end + kBN - 1) / kBN;
+    const int g = h / p.G;
+
+    if (threadIdx.x == 0) {
+        mbar_init(&sh->q_full, 1);
+        for (int s = 0; s < kStages; ++s) { mbar_init(&sh->kv_full[s], 1); mbar_init(&sh->kv_empty[s], 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(&sh->s_ready[i], 1); mbar_init(&sh->s_free[i], 4); }
+        mbar_init(&sh->p_ready, 4);
+        mbar_init(&sh->pv_done, 1);
+        sh->abort = 0;
+        fence_mbar_init();
+        prefetch_tmap(&tmap_q); prefetch_tmap(&tmap_k); prefetch_tmap(&tmap_v);
+    }
+    if (warp == 1) { tmem_alloc(&sh->tmem_base, 512); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = sh->tmem_base;
+    pdl_launch_dependents();
+    pdl_wait();
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ producer warp
+        if (lane == 0) {
+            mbar_expect_tx(&sh->q_full, (uint32_t)kQBytes);
+            for (int hf = 0; hf < kHalves; ++hf)
+                tma_load_2d(sq + hf * kHalfBytes, &tmap_q, h * D + hf * 64, q_row0, &sh->q_full);
+        }
+        // one lane per (K | V, 64-column half, page) box of a step
+        const int page = lane % kPagesPerTile;
+        const int hf = (lane / kPagesPerTile) % kHalves;
+        const int isv = lane / (kPagesPerTile * kHalves);
+        const bool op_lane = lane < 2 * kHalves * kPagesPerTile;
+        auto page_id = [&](int t) -> int {
+            const int idx = t * kPagesPerTile + page;
+            return (op_lane && idx * kPage < kv_end) ? p.page_table[(size_t)b * p.max_pages + idx] : 0;
+        };
+        int id = page_id(0);
+        for (int t = 0; t < n_steps; ++t) {
+            const int id_next = (t + 1 < n_steps) ? page_id(t + 1) : 0;      // one step ahead of the ring
+            const int s = t % kStages;
+            bool ok = mbar_wait(&sh->kv_empty[s], ((t / kStages) & 1) ^ 1);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok || sh->abort) { if (lane == 0) { sh->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); } break; }
+            const int np = min(kPagesPerTile, (kv_end - t * kBN + kPage - 1) / kPage);
+            if (lane == 0) mbar_expect_tx(&sh->kv_full[s], (uint32_t)(np * 2 * kHalves * kPage * 128));
+            __syncwarp();
+            if (op_lane && page < np) {
+                int pid = id;
+                if (pid < 0 || pid >= p.num_pages) { atomicExch(p.status, AFLEX_ERR_BOUNDS); pid = 0; }
+                uint8_t* dst = skv + s * kKVStage + isv * (kHalves * kHalfBytes) + hf * kHalfBytes + page * (kPage * 128);
+                tma_load_2d(dst, isv ? &tmap_v : &tmap_k, hf * 64, (pid * p.Hkv + g) * kPage, &sh->kv_full[s]);
+            }
+            id = id_next;
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc_s = umma_idesc_bf16(kBM, kBN);
+            const uint32_t idesc_pv = umma_idesc_bf16(kBM, D) | (1u << 16);      // B operand (V) is MN-major
+            bool ok = mbar_wait(&sh->q_full, 0);
+            auto issue_s = [&](int t) {
+                const int s = t % kStages, buf = t & 1;
+                ok = ok && mbar_wait(&sh->kv_full[s], (t / kStages) & 1);
+                ok = ok && mbar_wait(&sh->s_free[buf], ((t >> 1) & 1) ^ 1);
+                if (!ok) return;
+                tc_fence_after();
+                const uint32_t kaddr = smem_u32(skv + s * kKVStage);
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks) {
+                    const uint64_t da = umma_desc_k_sw128(smem_u32(sq) + (ks / 4) * kHalfBytes + (ks % 4) * 32);
+                    const uint64_t db = umma_desc_k_sw128(kaddr + (ks / 4) * kHalfBytes + (ks % 4) * 32);
+                    umma_bf16(tmem + kSCol + (uint32_t)(buf * kBN), da, db, idesc_s, ks > 0 ? 1u : 0u);
+                }
+                umma_commit(&sh->s_ready[buf]);
+            };
+            issue_s(0);
+            for (int t = 0; t < n_steps && ok && !sh->abort; ++t) {
+                if (t + 1 < n_steps) issue_s(t + 1);                           // S of the next step runs under this step's softmax
+                ok = ok && mbar_wait(&sh->p_ready, t & 1);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t vaddr = smem_u32(skv + (t % kStages) * kKVStage + kHalves * kHalfBytes);
+#pragma unroll
+                for (int ks = 0; ks < kBN / 16; ++ks) {
+                    const uint64_t da = umma_desc_k_sw128(smem_u32(sp) + (ks / 4) * kHalfBytes + (ks % 4) * 32);
+                    const uint64_t db = umma_desc_mn_sw128(vaddr + ks * 2048, kHalfBytes);
+                    umma_bf16(tmem + kOCol, da, db, idesc_pv, (t > 0 || ks > 0) ? 1u : 0u);
+                }
+                umma_commit(&sh->kv_empty[t % kStages]);
+                umma_commit(&sh->pv_done);
+            }
+            if (!ok) { sh->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); }
+        }
+    } else {
+        // ------------------------------------------------------------------ softmax warps: one query row per thread
+        const int w = warp & 3;                       // TMEM lane quadrant of this warp
+        const int row = w * 32 + lane;
+        const bool row_ok = row < rows_valid;
+        const int pos = pos0 + row;                   // position of this row's query
+        const uint32_t lane_base = tmem + ((uint32_t)(w * 32) << 16);
+        float m = kNegBig, l = 0.f;
+        bool ok = true;
+        for (int t = 0; t < n_steps; ++t) {
+            const int buf = t & 1;
+            ok = mbar_wait(&sh->s_ready[buf], (t >> 1) & 1);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok || sh->abort) break;
+            tc_fence_after();
+            const uint32_t s_addr = lane_base + kSCol + (uint32_t)(buf * kBN);
+            const int col0 = t * kBN;
+            // ---- pass 1: row maximum of the visible scores
+            float mx = -INFINITY;
+            for (int c0 = 0; c0 < kBN; c0 += 16) {
+                uint32_t r[16];
+                tmem_ld_32x32b_x16(s_addr + (uint32_t)c0, r);
+                tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const bool vis = row_ok && (col0 + c0 + j <= pos);
+                    mx = fmaxf(mx, vis ? __uint_as_float(r[j]) * p.scale_log2 : -INFINITY);
+                }
+            }
+            const float m_new = fmaxf(m, mx);
+            const float corr = fast_exp2(m - m_new);
+            // ---- the previous step's P V must have retired before O is rescaled and P overwritten
+            if (t > 0) {
+                ok = mbar_wait(&sh->pv_done, (t - 1) & 1);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after();
+                if (__any_sync(0xffffffffu, corr != 1.0f)) {
+                    for (int c0 = 0; c0 < D; c0 += 16) {
+                        uint32_t r[16];
+                        tmem_ld_32x32b_x16(lane_base + kOCol + (uint32_t)c0, r);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * corr);
+                        tmem_st_32x32b_x16(lane_base + kOCol + (uint32_t)c0, r);
+                    }
+                    tmem_st_wait();
+                }
+            }
+            // ---- V rows that were not loaded or lie past the sequence's end: zero them, whatever they hold
+            {
+                // rows of the step's V tile that hold real tokens: loaded pages only, and only up to the sequence's end
+                const int np = min(kPagesPerTile, (kv_end - col0 + kPage - 1) / kPage);
+                const int n_here = max(0, min(n_cached - col0, np * kPage));
+                if (n_here < kBN) {
+                    uint8_t* vbase = skv + (t % kStages) * kKVStage + kHalves * kHalfBytes;
+                    for (int i = threadIdx.x - 64; i < (kBN - n_here) * kHalves * 8; i += 128) {
+                        const int r_ = n_here + i / (kHalves * 8), c_ = i % (kHalves * 8);
+                        *reinterpret_cast<uint4*>(vbase + (c_ / 8) * kHalfBytes + r_ * 128 + (c_ % 8) * 16) = make_uint4(0, 0, 0, 0);
+                    }
+                }
+            }
+            // ---- pass 2: p = 2^(s - m), row sum, P (bf16) into shared memory as the A operand of P V
+            float lsum = 0.f;
+            for (int c0 = 0; c0 < kBN; c0 += 16) {
+                uint32_t r[16];
+                tmem_ld_32x32b_x16(s_addr + (uint32_t)c0, r);
+                tmem_ld_wait();
+                uint32_t pk[8];
+#pragma unroll
+                for (int j = 0; j < 16; j += 2) {
+                    const bool v0 = row_ok && (col0 + c0 + j <= pos), v1 = row_ok && (col0 + c0 + j + 1 <= pos);
+                    const float p0 = v0 ? fast_exp2(__uint_as_float(r[j]) * p.scale_log2 - m_new) : 0.f;
+                    const float p1 = v1 ? fast_exp2(__uint_as_float(r[j + 1]) * p.scale_log2 - m_new) : 0.f;
+                    lsum += p0 + p1;
+                    pk[j >> 1] = pack_bf16x2(p0, p1);
+                }
+#pragma unroll
+                for (int q4 = 0; q4 < 2; ++q4) {
+                    const int cc = c0 / 8 + q4;                      // 16-byte chunk of the row: 8 kv columns
+                    uint8_t* dst = sp + (cc / 8) * kHalfBytes + row * 128 + (((cc % 8) ^ (row & 7)) << 4);
+                    *reinterpret_cast<uint4*>(dst) = make_uint4(pk[4 * q4], pk[4 * q4 + 1], pk[4 * q4 + 2], pk[4 * q4 + 3]);
+                }
+            }
+            l = l * corr + lsum;
+            m = m_new;
+            // S buffer read, P (and zeroed V rows) written: hand both to the MMA issuer
+            fence_proxy_async();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) { mbar_arrive(&sh->s_free[buf]); mbar_arrive(&sh->p_ready); }
+        }
+        if (ok && !sh->abort) {
+            ok = mbar_wait(&sh->pv_done, (n_steps - 1) & 1);
+            ok = __all_sync(0xffffffffu, ok);
+        }
+        if (ok && !sh->abort) {
+            tc_fence_after();
+            const float inv = row_ok ? 1.0f / l : 0.f;
+            __nv_bfloat16* orow = p.out + ((size_t)(q_row0 + row) * p.Hq + h) * D;
+            for (int c0 = 0; c0 < D; c0 += 16) {
+                uint32_t r[16];
+                tmem_ld_32x32b_x16(lane_base + kOCol + (uint32_t)c0, r);
+                tmem_ld_wait();
+                if (row_ok) {
+                    uint32_t pk[8];
+#pragma unroll
+                    for (int j = 0; j < 16; j += 2)
+                        pk[j >> 1] = pack_bf16x2(__uint_as_float(r[j]) * inv, __uint_as_float(r[j + 1]) * inv);
+                    *reinterpret_cast<uint4*>(orow + c0) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    *reinterpret_cast<uint4*>(orow + c0 + 8) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                }
+            }
+        } else if (lane == 0 && !sh->abort) {
+            sh->abort = 1;
+            atomicExch(p.status, AFLEX_ERR_TIMEOUT);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem, 512); }
+}
+
+template <int D>
+static aflex_status launch_t(aflex_ctx* ctx, const aflex_attn_desc* d, const void* q, const aflex_kv* kv, int batch,
+                             const int32_t* q_offsets, int total_rows, int total_tiles, void* out, cudaStream_t st) {
+    Params p;
+    p.page_table = kv->page_table;
+    p.seq_lens = kv->seq_lens;
+    p.q_offsets = q_offsets;
+    p.batch = batch;
+    p.max_pages = kv->max_pages_per_seq;
+    p.Hq = d->num_q_heads; p.Hkv = d->num_kv_heads; p.G = d->num_q_heads / d->num_kv_heads;
+    p.num_pages = kv->num_pages;
+    p.total_tiles = total_tiles;
+    const float scale = d->sm_scale != 0.f ? d->sm_scale : 1.0f / sqrtf((float)D);
+    p.scale_log2 = scale * 1.4426950408889634f;
+    p.out = reinterpret_cast<__nv_bfloat16*>(out);
+    p.status = ctx->dev_status;
+    CUtensorMap tq, tk, tv;
+    const uint64_t rows = (uint64_t)kv->num_pages * d->num_kv_heads * kPage;
+    const uint64_t qcols = (uint64_t)d->num_q_heads * D;
+    if (!encode_tmap_2d_bf16(&tq, q, (uint64_t)total_rows, qcols, qcols * 2, kBM, 64, false) ||
+        !encode_tmap_2d_bf16(&tk, kv->k_cache, rows, D, (uint64_t)D * 2, kPage, 64, true) ||
+        !encode_tmap_2d_bf16(&tv, kv->v_cache, rows, D, (uint64_t)D * 2, kPage, 64, true))
+        return set_error(ctx, AFLEX_ERR_CUDA, "prefill attention: cuTensorMapEncodeTiled failed");
+    constexpr int kHalfBytes = kBN * 128;
+    const size_t smem = (size_t)(D / 64) * kHalfBytes * (1 + 2 * kStages) + 2 * kHalfBytes + sizeof(Shared) + 1024;
+    static bool attr_set[2] = {false, false};
+    const int ti = (D == 128) ? 1 : 0;
+    if (!attr_set[ti]) {
+        cudaError_t e = cudaFuncSetAttribute(attn_prefill_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return check_cuda(ctx, e, "cudaFuncSetAttribute(prefill attention)");
+        attr_set[ti] = true;
+    }
+    KernelScope scope(ctx, kKAttnPrefill, st);
+    return check_cuda(ctx,
+                      launch_pdl(attn_prefill_kernel<D>, dim3((unsigned)total_tiles * (unsigned)d->num_q_heads), dim3(kThreads),
+                                 smem, st, tq, tk, tv, p),
+                      "attn_prefill_kernel launch");
+}
+
+}  // namespace pa
+
+aflex_status attn_prefill_launch(aflex_ctx* ctx, const aflex_attn_desc* d, const void* q, const aflex_kv* kv, int batch,
+                                 const int32_t* q_offsets, const int32_t* q_offsets_host, void* out, cudaStream_t st) {
+    long long tiles = 0;
+    for (int b = 0; b < batch; ++b) {
+        const int m = q_offsets_host[b + 1] - q_offsets_host[b];
+        if (m < 0) return set_error(ctx, AFLEX_ERR_INVALID_ARG, "prefill attention: q_offsets_host must not decrease");
+        tiles += (m + pa::kBM - 1) / pa::kBM;
+    }
+    const int total_rows = q_offsets_host[batch];
+    if (q_offsets_host[0] != 0 || total_rows < 1 || tiles < 1)
+        return set_error(ctx, AFLEX_ERR_INVALID_ARG, "prefill attention: q_offsets_host must start at 0 and hold at least one query");
+    if (tiles * d->num_q_heads > 0x7fffffffLL) return set_error(ctx, AFLEX_ERR_UNSUPPORTED, "prefill attention: too many tiles");
+    if (d->head_dim == 128) return pa::launch_t<128>(ctx, d, q, kv, batch, q_offsets, total_rows, (int)tiles, out, st);
+    return pa::launch_t<64>(ctx, d, q, kv, batch, q_offsets, total_rows, (int)tiles, out, st);
+}
+
+}  // namespace aflex

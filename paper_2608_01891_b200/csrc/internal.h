@@ -26,7 +26,7 @@ namespace aflex {
 enum KernelKind {
     kKAttnDecode = 0, kKLinearGemm, kKDownGemm, kKGateUpGemm, kKRouterLogits,
     kKMoeRoute, kKMoeGather, kKMoeGateUpGemm, kKMoeDownGemm, kKMoeCombine,
-    kKAddRmsNorm, kKQkvGemm, kKRopeAppend, kKKindCount
+    kKAddRmsNorm, kKQkvGemm, kKRopeAppend, kKAttnPrefill, kKKindCount
 };
 constexpr int kProfMaxSlots = 8192;
 struct ProfSlot { cudaEvent_t start, stop; int kind; };
@@ -167,6 +167,10 @@ aflex_status moe_gather_launch(aflex_ctx* ctx, const void* x, const int32_t* pos
 aflex_status moe_combine_launch(aflex_ctx* ctx, const float* yp, const int32_t* pos, const float* gate, int T,
                                 int K, int H, void* y, cudaStream_t st);
 
+
+// ---- prefill attention (attn_prefill.cu)
+aflex_status attn_prefill_launch(aflex_ctx* ctx, const aflex_attn_desc* d, const void* q, const aflex_kv* kv, int batch,
+                                 const int32_t* q_offsets, const int32_t* q_offsets_host, void* out, cudaStream_t st);
 
 // ---- decoder-layer glue (decoder.cu)
 aflex_status add_rmsnorm_launch(aflex_ctx* ctx, const void* res, const void* add, const void* w, int T, int H, float eps,
