@@ -231,18 +231,25 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
             tc_fence_after();
             const uint32_t s_addr = lane_base + kSCol + (uint32_t)(buf * kBN);
             const int col0 = t * kBN;
-            // ---- pass 1: row maximum of the visible scores
-            float mx = -INFINITY;
-            for (int c0 = 0; c0 < kBN; c0 += 16) {
-                uint32_t r[16];
-                tmem_ld_32x32b_x16(s_addr + (uint32_t)c0, r);
-                tmem_ld_wait();
+            // ---- this thread's S row into registers (one wait for all eight loads); the buffer is free at once
+            float sv[kBN];
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const bool vis = row_ok && (col0 + c0 + j <= pos);
-                    mx = fmaxf(mx, vis ? __uint_as_float(r[j]) * p.scale_log2 : -INFINITY);
-                }
+            for (int c0 = 0; c0 < kBN; c0 += 16)
+                tmem_ld_32x32b_x16(s_addr + (uint32_t)c0, *reinterpret_cast<uint32_t(*)[16]>(&sv[c0]));
+            tmem_ld_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh->s_free[buf]);
+            // causal mask: only steps that reach past the tile's first query need it
+            if (col0 + kBN - 1 > pos0 || !row_ok) {
+#pragma unroll
+                for (int j = 0; j < kBN; ++j)
+                    if (!(row_ok && col0 + j <= pos)) sv[j] = -INFINITY;
             }
+            float mx = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < kBN; ++j) mx = fmaxf(mx, sv[j]);
+            mx *= p.scale_log2;
             const float m_new = fmaxf(m, mx);
             const float corr = fast_exp2(m - m_new);
             // ---- the previous step's P V must have retired before O is rescaled and P overwritten
@@ -276,35 +283,29 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
                     }
                 }
             }
-            // ---- pass 2: p = 2^(s - m), row sum, P (bf16) into shared memory as the A operand of P V
+            // ---- p = 2^(s * scale - m), row sum, P (bf16) into shared memory as the A operand of P V
             float lsum = 0.f;
-            for (int c0 = 0; c0 < kBN; c0 += 16) {
-                uint32_t r[16];
-                tmem_ld_32x32b_x16(s_addr + (uint32_t)c0, r);
-                tmem_ld_wait();
-                uint32_t pk[8];
 #pragma unroll
-                for (int j = 0; j < 16; j += 2) {
-                    const bool v0 = row_ok && (col0 + c0 + j <= pos), v1 = row_ok && (col0 + c0 + j + 1 <= pos);
-                    const float p0 = v0 ? fast_exp2(__uint_as_float(r[j]) * p.scale_log2 - m_new) : 0.f;
-                    const float p1 = v1 ? fast_exp2(__uint_as_float(r[j + 1]) * p.scale_log2 - m_new) : 0.f;
+            for (int c0 = 0; c0 < kBN; c0 += 8) {
+                uint32_t pk[4];
+#pragma unroll
+                for (int j = 0; j < 8; j += 2) {
+                    const float p0 = fast_exp2(fmaf(sv[c0 + j], p.scale_log2, -m_new));
+                    const float p1 = fast_exp2(fmaf(sv[c0 + j + 1], p.scale_log2, -m_new));
                     lsum += p0 + p1;
                     pk[j >> 1] = pack_bf16x2(p0, p1);
                 }
-#pragma unroll
-                for (int q4 = 0; q4 < 2; ++q4) {
-                    const int cc = c0 / 8 + q4;                      // 16-byte chunk of the row: 8 kv columns
-                    uint8_t* dst = sp + (cc / 8) * kHalfBytes + row * 128 + (((cc % 8) ^ (row & 7)) << 4);
-                    *reinterpret_cast<uint4*>(dst) = make_uint4(pk[4 * q4], pk[4 * q4 + 1], pk[4 * q4 + 2], pk[4 * q4 + 3]);
-                }
+                const int cc = c0 / 8;                               // 16-byte chunk of the row: 8 kv columns
+                uint8_t* dst = sp + (cc / 8) * kHalfBytes + row * 128 + (((cc % 8) ^ (row & 7)) << 4);
+                *reinterpret_cast<uint4*>(dst) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
             }
             l = l * corr + lsum;
             m = m_new;
-            // S buffer read, P (and zeroed V rows) written: hand both to the MMA issuer
+            // P (and zeroed V rows) written: hand them to the MMA issuer
             fence_proxy_async();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) { mbar_arrive(&sh->s_free[buf]); mbar_arrive(&sh->p_ready); }
+            if (lane == 0) mbar_arrive(&sh->p_ready);
         }
         if (ok && !sh->abort) {
             ok = mbar_wait(&sh->pv_done, (n_steps - 1) & 1);
