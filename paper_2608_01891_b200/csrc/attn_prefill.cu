@@ -2,15 +2,17 @@
 // (the paper's PA pool; Section 1: during prefill both operators are dominated by matrix
 // multiplications).  Compute-bound, so it runs on the 5th-generation tensor cores:
 //
-//   tile        = 128 consecutive query tokens of one query head against 128 cached tokens at a time
+//   CTA         = two tiles of 128 consecutive query tokens of one query head; both walk the same cached tokens,
+//               64 at a step, share the K/V stages and alternate on the tensor pipe (one tile's softmax runs
+//               while the other tile's MMAs do)
 //   S = Q K^T   tcgen05.mma, both operands K-major (Q tile and K tile rows of D contiguous elements,
-//               128-byte swizzle as TMA writes them), fp32 accumulator in TMEM, double-buffered
+//               128-byte swizzle as TMA writes them), fp32 accumulator in TMEM, double-buffered per tile
 //   softmax     four warps, one query row per thread: tcgen05.ld of its S row, causal mask, online
 //               max / sum in base 2, P rounded to bf16 into shared memory as the next MMA's A operand
 //   O += P V    tcgen05.mma with V exactly as the cache stores it ([token][D]: an MN-major B operand),
 //               accumulator in TMEM; rescaled in place (tcgen05.ld / st) when a row's maximum moves
-//   pipeline    a producer warp issues the TMA loads of the K and V pages of the next tile (2 stages)
-//               while one thread issues MMAs and S of tile t+1 is computed during the softmax of tile t
+//   pipeline    a producer warp issues the TMA loads of the K and V pages of the coming steps (3 stages)
+//               while one thread issues MMAs; S of step t+1 is computed during the softmax of step t
 //
 // Query i of a sequence with n cached tokens of which the last m are being prefilled sits at position
 // n - m + i and sees cached tokens 0 .. n - m + i.  Cache slots beyond n may hold anything (NaN too):
@@ -25,11 +27,12 @@ namespace aflex {
 namespace pa {
 
 constexpr int kBM = 128;          // query rows per tile
-constexpr int kBN = 128;          // cached tokens per step
+constexpr int kQT = 2;            // query tiles per CTA (they share the K/V stages and alternate on the tensor pipe)
+constexpr int kBN = 64;           // cached tokens per step
 constexpr int kPage = 16;
-constexpr int kPagesPerTile = kBN / kPage;
-constexpr int kStages = 2;
-constexpr int kThreads = 6 * 32;  // producer, MMA issuer, four softmax warps
+constexpr int kPagesPerStep = kBN / kPage;
+constexpr int kStages = 3;
+constexpr int kThreads = (2 + 4 * kQT) * 32;   // producer, MMA issuer, four softmax warps per query tile
 constexpr float kNegBig = -1.0e30f;
 
 struct Params {
@@ -38,7 +41,7 @@ struct Params {
     const int32_t* q_offsets;     // [B+1] first query row of every sequence
     int batch, max_pages, Hq, Hkv, G;
     long long num_pages;
-    int total_tiles;              // sum over sequences of ceil(q_len / 128)
+    int total_blocks;             // sum over sequences of ceil(q_len / 256)
     float scale_log2;
     __nv_bfloat16* out;           // [T][Hq][D]
     int* status;
@@ -47,8 +50,8 @@ struct Params {
 struct __align__(8) Shared {
     uint64_t q_full;
     uint64_t kv_full[kStages], kv_empty[kStages];
-    uint64_t s_ready[2], s_free[2];
-    uint64_t p_ready, pv_done;
+    uint64_t s_ready[kQT][2], s_free[kQT][2];
+    uint64_t p_ready[kQT], pv_done[kQT];
     uint32_t tmem_base;
     volatile int abort;
 };
@@ -81,54 +84,65 @@ __global__ void __launch_bounds__(kThreads, 1)
 attn_prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                     const __grid_constant__ CUtensorMap tmap_v, const Params p) {
     constexpr int kHalves = D / 64;
-    constexpr int kHalfBytes = kBN * 128;               // 128 rows of 128 B
-    constexpr int kQBytes = kHalves * kHalfBytes;
-    constexpr int kKVStage = 2 * kHalves * kHalfBytes;   // K then V
-    constexpr int kPBytes = 2 * kHalfBytes;
-    constexpr uint32_t kSCol = 0, kOCol = 2 * kBN;       // TMEM columns: S buffers at 0 and 128, O after them
+    constexpr int kQHalf = kBM * 128;                    // 128 query rows of 128 B
+    constexpr int kQBytes = kHalves * kQHalf;            // one query tile
+    constexpr int kKVHalf = kBN * 128;                   // 64 cached tokens of 128 B
+    constexpr int kKVStage = 2 * kHalves * kKVHalf;      // K then V
+    constexpr int kPBytes = kBM * 128;                   // P of one query tile: 128 rows x 64 tokens
+    constexpr uint32_t kOCol = kQT * 2 * kBN;            // TMEM: S[tile][buffer] first, then O[tile]
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* sq = smem;
-    uint8_t* skv = sq + kQBytes;
+    uint8_t* skv = sq + kQT * kQBytes;
     uint8_t* sp = skv + kStages * kKVStage;
-    Shared* sh = reinterpret_cast<Shared*>(sp + kPBytes);
+    Shared* sh = reinterpret_cast<Shared*>(sp + kQT * kPBytes);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-    // ---- which tile: query head fastest (the heads of a group share K/V tiles in L2), long tiles first
+    // ---- which block of 256 query rows: query head fastest (the heads of a group share K/V in L2), long blocks first
     const int h = blockIdx.x % p.Hq;
-    const int tile_id = p.total_tiles - 1 - (int)(blockIdx.x / p.Hq);
-    int b = 0, tile_in_seq = 0;
+    const int block_id = p.total_blocks - 1 - (int)(blockIdx.x / p.Hq);
+    int b = 0, block_in_seq = 0;
     {
         int acc = 0;
         for (b = 0; b < p.batch; ++b) {
             const int m = p.q_offsets[b + 1] - p.q_offsets[b];
-            const int nt = (m + kBM - 1) / kBM;
-            if (tile_id < acc + nt) { tile_in_seq = tile_id - acc; break; }
-            acc += nt;
+            const int nb = (m + kQT * kBM - 1) / (kQT * kBM);
+            if (block_id < acc + nb) { block_in_seq = block_id - acc; break; }
+            acc += nb;
         }
-        if (b >= p.batch) return;                       // cannot happen with a consistent total_tiles
+        if (b >= p.batch) return;                        // cannot happen with a consistent total_blocks
     }
-    const int q_row0 = p.q_offsets[b] + tile_in_seq * kBM;
     const int q_len = p.q_offsets[b + 1] - p.q_offsets[b];
-    const int rows_valid = min(kBM, q_len - tile_in_seq * kBM);
     int n_cached = p.seq_lens[b];
     {
         const int cap = p.max_pages * kPage;
         if (n_cached > cap || n_cached < q_len) { if (threadIdx.x == 0) atomicExch(p.status, AFLEX_ERR_BOUNDS); n_cached = max(min(n_cached, cap), q_len); }
     }
-    const int pos0 = n_cached - q_len + tile_in_seq * kBM;          // position of the tile's first query
-    const int kv_end = pos0 + rows_valid;                           // cached tokens visible to the tile's last query
-    const int n_steps = (kv_end + kBN - 1) / kBN;
+    // per query tile: rows, position of the first query, cached tokens visible to the last query, steps
+    int rows_valid[kQT], pos0[kQT], kv_end[kQT], n_steps[kQT];
+#pragma unroll
+    for (int i = 0; i < kQT; ++i) {
+        const int first = (block_in_seq * kQT + i) * kBM;
+        rows_valid[i] = max(0, min(kBM, q_len - first));
+        pos0[i] = n_cached - q_len + first;
+        kv_end[i] = rows_valid[i] > 0 ? pos0[i] + rows_valid[i] : 0;
+        n_steps[i] = (kv_end[i] + kBN - 1) / kBN;
+    }
+    const int q_row0 = p.q_offsets[b] + block_in_seq * kQT * kBM;
+    const int kv_end_all = max(kv_end[0], kv_end[1]);
+    const int steps_all = max(n_steps[0], n_steps[1]);
     const int g = h / p.G;
 
     if (threadIdx.x == 0) {
         mbar_init(&sh->q_full, 1);
         for (int s = 0; s < kStages; ++s) { mbar_init(&sh->kv_full[s], 1); mbar_init(&sh->kv_empty[s], 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(&sh->s_ready[i], 1); mbar_init(&sh->s_free[i], 4); }
-        mbar_init(&sh->p_ready, 4);
-        mbar_init(&sh->pv_done, 1);
+        for (int i = 0; i < kQT; ++i) {
+            for (int k = 0; k < 2; ++k) { mbar_init(&sh->s_ready[i][k], 1); mbar_init(&sh->s_free[i][k], 4); }
+            mbar_init(&sh->p_ready[i], 4);
+            mbar_init(&sh->pv_done[i], 1);
+        }
         sh->abort = 0;
         fence_mbar_init();
         prefetch_tmap(&tmap_q); prefetch_tmap(&tmap_k); prefetch_tmap(&tmap_v);
@@ -144,33 +158,34 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     if (warp == 0) {
         // ------------------------------------------------------------------ producer warp
         if (lane == 0) {
-            mbar_expect_tx(&sh->q_full, (uint32_t)kQBytes);
-            for (int hf = 0; hf < kHalves; ++hf)
-                tma_load_2d(sq + hf * kHalfBytes, &tmap_q, h * D + hf * 64, q_row0, &sh->q_full);
+            mbar_expect_tx(&sh->q_full, (uint32_t)(kQT * kQBytes));
+            for (int i = 0; i < kQT; ++i)
+                for (int hf = 0; hf < kHalves; ++hf)
+                    tma_load_2d(sq + i * kQBytes + hf * kQHalf, &tmap_q, h * D + hf * 64, q_row0 + i * kBM, &sh->q_full);
         }
         // one lane per (K | V, 64-column half, page) box of a step
-        const int page = lane % kPagesPerTile;
-        const int hf = (lane / kPagesPerTile) % kHalves;
-        const int isv = lane / (kPagesPerTile * kHalves);
-        const bool op_lane = lane < 2 * kHalves * kPagesPerTile;
+        const int page = lane % kPagesPerStep;
+        const int hf = (lane / kPagesPerStep) % kHalves;
+        const int isv = lane / (kPagesPerStep * kHalves);
+        const bool op_lane = lane < 2 * kHalves * kPagesPerStep;
         auto page_id = [&](int t) -> int {
-            const int idx = t * kPagesPerTile + page;
-            return (op_lane && idx * kPage < kv_end) ? p.page_table[(size_t)b * p.max_pages + idx] : 0;
+            const int idx = t * kPagesPerStep + page;
+            return (op_lane && idx * kPage < kv_end_all) ? p.page_table[(size_t)b * p.max_pages + idx] : 0;
         };
         int id = page_id(0);
-        for (int t = 0; t < n_steps; ++t) {
-            const int id_next = (t + 1 < n_steps) ? page_id(t + 1) : 0;      // one step ahead of the ring
+        for (int t = 0; t < steps_all; ++t) {
+            const int id_next = (t + 1 < steps_all) ? page_id(t + 1) : 0;     // one step ahead of the ring
             const int s = t % kStages;
             bool ok = mbar_wait(&sh->kv_empty[s], ((t / kStages) & 1) ^ 1);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok || sh->abort) { if (lane == 0) { sh->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); } break; }
-            const int np = min(kPagesPerTile, (kv_end - t * kBN + kPage - 1) / kPage);
+            const int np = min(kPagesPerStep, (kv_end_all - t * kBN + kPage - 1) / kPage);
             if (lane == 0) mbar_expect_tx(&sh->kv_full[s], (uint32_t)(np * 2 * kHalves * kPage * 128));
             __syncwarp();
             if (op_lane && page < np) {
                 int pid = id;
                 if (pid < 0 || pid >= p.num_pages) { atomicExch(p.status, AFLEX_ERR_BOUNDS); pid = 0; }
-                uint8_t* dst = skv + s * kKVStage + isv * (kHalves * kHalfBytes) + hf * kHalfBytes + page * (kPage * 128);
+                uint8_t* dst = skv + s * kKVStage + isv * (kHalves * kKVHalf) + hf * kKVHalf + page * (kPage * 128);
                 tma_load_2d(dst, isv ? &tmap_v : &tmap_k, hf * 64, (pid * p.Hkv + g) * kPage, &sh->kv_full[s]);
             }
             id = id_next;
@@ -181,57 +196,69 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
             const uint32_t idesc_s = umma_idesc_bf16(kBM, kBN);
             const uint32_t idesc_pv = umma_idesc_bf16(kBM, D) | (1u << 16);      // B operand (V) is MN-major
             bool ok = mbar_wait(&sh->q_full, 0);
+            // S of step t for both query tiles (needs the step's K/V and the tiles' free S buffers)
             auto issue_s = [&](int t) {
                 const int s = t % kStages, buf = t & 1;
                 ok = ok && mbar_wait(&sh->kv_full[s], (t / kStages) & 1);
-                ok = ok && mbar_wait(&sh->s_free[buf], ((t >> 1) & 1) ^ 1);
-                if (!ok) return;
-                tc_fence_after();
                 const uint32_t kaddr = smem_u32(skv + s * kKVStage);
+                for (int i = 0; i < kQT && ok; ++i) {
+                    if (t >= n_steps[i]) continue;
+                    ok = ok && mbar_wait(&sh->s_free[i][buf], ((t >> 1) & 1) ^ 1);
+                    if (!ok) break;
+                    tc_fence_after();
 #pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks) {
-                    const uint64_t da = umma_desc_k_sw128(smem_u32(sq) + (ks / 4) * kHalfBytes + (ks % 4) * 32);
-                    const uint64_t db = umma_desc_k_sw128(kaddr + (ks / 4) * kHalfBytes + (ks % 4) * 32);
-                    umma_bf16(tmem + kSCol + (uint32_t)(buf * kBN), da, db, idesc_s, ks > 0 ? 1u : 0u);
+                    for (int ks = 0; ks < D / 16; ++ks) {
+                        const uint64_t da = umma_desc_k_sw128(smem_u32(sq + i * kQBytes) + (ks / 4) * kQHalf + (ks % 4) * 32);
+                        const uint64_t db = umma_desc_k_sw128(kaddr + (ks / 4) * kKVHalf + (ks % 4) * 32);
+                        umma_bf16(tmem + (uint32_t)((i * 2 + buf) * kBN), da, db, idesc_s, ks > 0 ? 1u : 0u);
+                    }
+                    umma_commit(&sh->s_ready[i][buf]);
                 }
-                umma_commit(&sh->s_ready[buf]);
             };
             issue_s(0);
-            for (int t = 0; t < n_steps && ok && !sh->abort; ++t) {
-                if (t + 1 < n_steps) issue_s(t + 1);                           // S of the next step runs under this step's softmax
-                ok = ok && mbar_wait(&sh->p_ready, t & 1);
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t vaddr = smem_u32(skv + (t % kStages) * kKVStage + kHalves * kHalfBytes);
+            for (int t = 0; t < steps_all && ok && !sh->abort; ++t) {
+                if (t + 1 < steps_all) issue_s(t + 1);                        // runs under this step's softmax
+                const uint32_t vaddr = smem_u32(skv + (t % kStages) * kKVStage + kHalves * kKVHalf);
+                for (int i = 0; i < kQT && ok; ++i) {
+                    if (t >= n_steps[i]) continue;
+                    ok = ok && mbar_wait(&sh->p_ready[i], t & 1);
+                    if (!ok) break;
+                    tc_fence_after();
 #pragma unroll
-                for (int ks = 0; ks < kBN / 16; ++ks) {
-                    const uint64_t da = umma_desc_k_sw128(smem_u32(sp) + (ks / 4) * kHalfBytes + (ks % 4) * 32);
-                    const uint64_t db = umma_desc_mn_sw128(vaddr + ks * 2048, kHalfBytes);
-                    umma_bf16(tmem + kOCol, da, db, idesc_pv, (t > 0 || ks > 0) ? 1u : 0u);
+                    for (int ks = 0; ks < kBN / 16; ++ks) {
+                        const uint64_t da = umma_desc_k_sw128(smem_u32(sp + i * kPBytes) + ks * 32);
+                        const uint64_t db = umma_desc_mn_sw128(vaddr + ks * 2048, kKVHalf);
+                        umma_bf16(tmem + kOCol + (uint32_t)(i * D), da, db, idesc_pv, (t > 0 || ks > 0) ? 1u : 0u);
+                    }
+                    umma_commit(&sh->pv_done[i]);
                 }
                 umma_commit(&sh->kv_empty[t % kStages]);
-                umma_commit(&sh->pv_done);
             }
             if (!ok) { sh->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); }
         }
     } else {
         // ------------------------------------------------------------------ softmax warps: one query row per thread
+        const int i = (warp - 2) / 4;                 // query tile of this warp
         const int w = warp & 3;                       // TMEM lane quadrant of this warp
         const int row = w * 32 + lane;
-        const bool row_ok = row < rows_valid;
-        const int pos = pos0 + row;                   // position of this row's query
+        const bool row_ok = row < rows_valid[i];
+        const int pos = pos0[i] + row;                // position of this row's query
         const uint32_t lane_base = tmem + ((uint32_t)(w * 32) << 16);
+        const uint32_t o_addr = lane_base + kOCol + (uint32_t)(i * D);
+        uint8_t* my_p = sp + i * kPBytes;
+        const int steps = n_steps[i];
+        const int tid = (warp - 2 - 4 * i) * 32 + lane;   // 0..127 inside the tile's warps
         float m = kNegBig, l = 0.f;
         bool ok = true;
-        for (int t = 0; t < n_steps; ++t) {
+        for (int t = 0; t < steps; ++t) {
             const int buf = t & 1;
-            ok = mbar_wait(&sh->s_ready[buf], (t >> 1) & 1);
+            ok = mbar_wait(&sh->s_ready[i][buf], (t >> 1) & 1);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok || sh->abort) break;
             tc_fence_after();
-            const uint32_t s_addr = lane_base + kSCol + (uint32_t)(buf * kBN);
+            const uint32_t s_addr = lane_base + (uint32_t)((i * 2 + buf) * kBN);
             const int col0 = t * kBN;
-            // ---- this thread's S row into registers (one wait for all eight loads); the buffer is free at once
+            // ---- this thread's S row into registers (one wait for all loads); the buffer is free at once
             float sv[kBN];
 #pragma unroll
             for (int c0 = 0; c0 < kBN; c0 += 16)
@@ -239,9 +266,9 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
             tmem_ld_wait();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&sh->s_free[buf]);
+            if (lane == 0) mbar_arrive(&sh->s_free[i][buf]);
             // causal mask: only steps that reach past the tile's first query need it
-            if (col0 + kBN - 1 > pos0 || !row_ok) {
+            if (col0 + kBN - 1 > pos0[i] || !row_ok) {
 #pragma unroll
                 for (int j = 0; j < kBN; ++j)
                     if (!(row_ok && col0 + j <= pos)) sv[j] = -INFINITY;
@@ -254,32 +281,33 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
             const float corr = fast_exp2(m - m_new);
             // ---- the previous step's P V must have retired before O is rescaled and P overwritten
             if (t > 0) {
-                ok = mbar_wait(&sh->pv_done, (t - 1) & 1);
+                ok = mbar_wait(&sh->pv_done[i], (t - 1) & 1);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after();
                 if (__any_sync(0xffffffffu, corr != 1.0f)) {
+#pragma unroll
                     for (int c0 = 0; c0 < D; c0 += 16) {
                         uint32_t r[16];
-                        tmem_ld_32x32b_x16(lane_base + kOCol + (uint32_t)c0, r);
+                        tmem_ld_32x32b_x16(o_addr + (uint32_t)c0, r);
                         tmem_ld_wait();
 #pragma unroll
                         for (int j = 0; j < 16; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * corr);
-                        tmem_st_32x32b_x16(lane_base + kOCol + (uint32_t)c0, r);
+                        tmem_st_32x32b_x16(o_addr + (uint32_t)c0, r);
                     }
                     tmem_st_wait();
                 }
             }
             // ---- V rows that were not loaded or lie past the sequence's end: zero them, whatever they hold
+            //      (by the warps of both query tiles: each tile's P V waits only for its own warps, zeros are idempotent)
             {
-                // rows of the step's V tile that hold real tokens: loaded pages only, and only up to the sequence's end
-                const int np = min(kPagesPerTile, (kv_end - col0 + kPage - 1) / kPage);
+                const int np = min(kPagesPerStep, (kv_end_all - col0 + kPage - 1) / kPage);
                 const int n_here = max(0, min(n_cached - col0, np * kPage));
                 if (n_here < kBN) {
-                    uint8_t* vbase = skv + (t % kStages) * kKVStage + kHalves * kHalfBytes;
-                    for (int i = threadIdx.x - 64; i < (kBN - n_here) * kHalves * 8; i += 128) {
-                        const int r_ = n_here + i / (kHalves * 8), c_ = i % (kHalves * 8);
-                        *reinterpret_cast<uint4*>(vbase + (c_ / 8) * kHalfBytes + r_ * 128 + (c_ % 8) * 16) = make_uint4(0, 0, 0, 0);
+                    uint8_t* vbase = skv + (t % kStages) * kKVStage + kHalves * kKVHalf;
+                    for (int k = tid; k < (kBN - n_here) * kHalves * 8; k += 128) {
+                        const int r_ = n_here + k / (kHalves * 8), c_ = k % (kHalves * 8);
+                        *reinterpret_cast<uint4*>(vbase + (c_ / 8) * kKVHalf + r_ * 128 + (c_ % 8) * 16) = make_uint4(0, 0, 0, 0);
                     }
                 }
             }
@@ -296,8 +324,7 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
                     pk[j >> 1] = pack_bf16x2(p0, p1);
                 }
                 const int cc = c0 / 8;                               // 16-byte chunk of the row: 8 kv columns
-                uint8_t* dst = sp + (cc / 8) * kHalfBytes + row * 128 + (((cc % 8) ^ (row & 7)) << 4);
-                *reinterpret_cast<uint4*>(dst) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                *reinterpret_cast<uint4*>(my_p + row * 128 + ((cc ^ (row & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
             }
             l = l * corr + lsum;
             m = m_new;
@@ -305,19 +332,20 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
             fence_proxy_async();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&sh->p_ready);
+            if (lane == 0) mbar_arrive(&sh->p_ready[i]);
         }
-        if (ok && !sh->abort) {
-            ok = mbar_wait(&sh->pv_done, (n_steps - 1) & 1);
+        if (steps > 0 && ok && !sh->abort) {
+            ok = mbar_wait(&sh->pv_done[i], (steps - 1) & 1);
             ok = __all_sync(0xffffffffu, ok);
         }
-        if (ok && !sh->abort) {
+        if (steps > 0 && ok && !sh->abort) {
             tc_fence_after();
             const float inv = row_ok ? 1.0f / l : 0.f;
-            __nv_bfloat16* orow = p.out + ((size_t)(q_row0 + row) * p.Hq + h) * D;
+            __nv_bfloat16* orow = p.out + ((size_t)(q_row0 + i * kBM + row) * p.Hq + h) * D;
+#pragma unroll
             for (int c0 = 0; c0 < D; c0 += 16) {
                 uint32_t r[16];
-                tmem_ld_32x32b_x16(lane_base + kOCol + (uint32_t)c0, r);
+                tmem_ld_32x32b_x16(o_addr + (uint32_t)c0, r);
                 tmem_ld_wait();
                 if (row_ok) {
                     uint32_t pk[8];
@@ -328,7 +356,7 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
                     *reinterpret_cast<uint4*>(orow + c0 + 8) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
                 }
             }
-        } else if (lane == 0 && !sh->abort) {
+        } else if (steps > 0 && lane == 0 && !sh->abort) {
             sh->abort = 1;
             atomicExch(p.status, AFLEX_ERR_TIMEOUT);
         }
@@ -340,7 +368,7 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
 
 template <int D>
 static aflex_status launch_t(aflex_ctx* ctx, const aflex_attn_desc* d, const void* q, const aflex_kv* kv, int batch,
-                             const int32_t* q_offsets, int total_rows, int total_tiles, void* out, cudaStream_t st) {
+                             const int32_t* q_offsets, int total_rows, int total_blocks, void* out, cudaStream_t st) {
     Params p;
     p.page_table = kv->page_table;
     p.seq_lens = kv->seq_lens;
@@ -349,7 +377,7 @@ static aflex_status launch_t(aflex_ctx* ctx, const aflex_attn_desc* d, const voi
     p.max_pages = kv->max_pages_per_seq;
     p.Hq = d->num_q_heads; p.Hkv = d->num_kv_heads; p.G = d->num_q_heads / d->num_kv_heads;
     p.num_pages = kv->num_pages;
-    p.total_tiles = total_tiles;
+    p.total_blocks = total_blocks;
     const float scale = d->sm_scale != 0.f ? d->sm_scale : 1.0f / sqrtf((float)D);
     p.scale_log2 = scale * 1.4426950408889634f;
     p.out = reinterpret_cast<__nv_bfloat16*>(out);
@@ -361,8 +389,8 @@ static aflex_status launch_t(aflex_ctx* ctx, const aflex_attn_desc* d, const voi
         !encode_tmap_2d_bf16(&tk, kv->k_cache, rows, D, (uint64_t)D * 2, kPage, 64, true) ||
         !encode_tmap_2d_bf16(&tv, kv->v_cache, rows, D, (uint64_t)D * 2, kPage, 64, true))
         return set_error(ctx, AFLEX_ERR_CUDA, "prefill attention: cuTensorMapEncodeTiled failed");
-    constexpr int kHalfBytes = kBN * 128;
-    const size_t smem = (size_t)(D / 64) * kHalfBytes * (1 + 2 * kStages) + 2 * kHalfBytes + sizeof(Shared) + 1024;
+    const size_t smem = (size_t)kQT * (D / 64) * kBM * 128 + (size_t)kStages * 2 * (D / 64) * kBN * 128 + (size_t)kQT * kBM * 128 +
+                        sizeof(Shared) + 1024;
     static bool attr_set[2] = {false, false};
     const int ti = (D == 128) ? 1 : 0;
     if (!attr_set[ti]) {
@@ -372,7 +400,7 @@ static aflex_status launch_t(aflex_ctx* ctx, const aflex_attn_desc* d, const voi
     }
     KernelScope scope(ctx, kKAttnPrefill, st);
     return check_cuda(ctx,
-                      launch_pdl(attn_prefill_kernel<D>, dim3((unsigned)total_tiles * (unsigned)d->num_q_heads), dim3(kThreads),
+                      launch_pdl(attn_prefill_kernel<D>, dim3((unsigned)total_blocks * (unsigned)d->num_q_heads), dim3(kThreads),
                                  smem, st, tq, tk, tv, p),
                       "attn_prefill_kernel launch");
 }
@@ -385,7 +413,7 @@ aflex_status attn_prefill_launch(aflex_ctx* ctx, const aflex_attn_desc* d, const
     for (int b = 0; b < batch; ++b) {
         const int m = q_offsets_host[b + 1] - q_offsets_host[b];
         if (m < 0) return set_error(ctx, AFLEX_ERR_INVALID_ARG, "prefill attention: q_offsets_host must not decrease");
-        tiles += (m + pa::kBM - 1) / pa::kBM;
+        tiles += (m + pa::kQT * pa::kBM - 1) / (pa::kQT * pa::kBM);
     }
     const int total_rows = q_offsets_host[batch];
     if (q_offsets_host[0] != 0 || total_rows < 1 || tiles < 1)
