@@ -277,7 +277,10 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
 #pragma unroll
             for (int j = 0; j < kBN; ++j) mx = fmaxf(mx, sv[j]);
             mx *= p.scale_log2;
-            const float m_new = fmaxf(m, mx);
+            // The reference maximum m moves only when some row of the warp outgrows it by more than 2^8: until
+            // then p = 2^(s - m) stays below 256 (harmless in bf16 / fp32) and O needs no rescaling.
+            const bool grow = __any_sync(0xffffffffu, mx > m + 8.0f);
+            const float m_new = grow ? fmaxf(m, mx) : m;
             const float corr = fast_exp2(m - m_new);
             // ---- the previous step's P V must have retired before O is rescaled and P overwritten
             if (t > 0) {
@@ -285,7 +288,7 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after();
-                if (__any_sync(0xffffffffu, corr != 1.0f)) {
+                if (grow) {
 #pragma unroll
                     for (int c0 = 0; c0 < D; c0 += 16) {
                         uint32_t r[16];
