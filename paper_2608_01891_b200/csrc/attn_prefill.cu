@@ -31,7 +31,7 @@ constexpr int kQT = 2;            // query tiles per CTA (they share the K/V sta
 constexpr int kBN = 64;           // cached tokens per step
 constexpr int kPage = 16;
 constexpr int kPagesPerStep = kBN / kPage;
-constexpr int kStages = 3;
+constexpr int kStages = 4;
 constexpr int kThreads = (2 + 4 * kQT) * 32;   // producer, MMA issuer, four softmax warps per query tile
 constexpr float kNegBig = -1.0e30f;
 
@@ -79,6 +79,33 @@ __device__ __forceinline__ uint64_t umma_desc_mn_sw128(uint32_t smem_addr, uint3
     return d;
 }
 
+// The MMA issuer keeps descriptors as a low word (start address in 16-byte units, leading byte offset at bit 16) that
+// it advances by adding byte offsets >> 4, and one upper word shared by every operand here (8-row groups 1024 B apart,
+// descriptor version 1, 128-byte swizzle).
+constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint32_t desc_lo(uint32_t smem_addr, uint32_t lbo_bytes) {
+    return ((smem_addr & 0x3FFFF) >> 4) | ((lbo_bytes >> 4) << 16);
+}
+__device__ __forceinline__ void umma_ss(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "mov.b64 da, {%1, %5};\n\t"
+        "mov.b64 db, {%2, %5};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}"
+        ::"r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHi)
+        : "memory");
+}
+__device__ __forceinline__ void umma_ts(uint32_t tmem_d, uint32_t tmem_a, uint32_t b_lo, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "mov.b64 db, {%2, %5};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %3, p;\n\t}"
+        ::"r"(tmem_d), "r"(tmem_a), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHi)
+        : "memory");
+}
+
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
@@ -88,15 +115,13 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     constexpr int kQBytes = kHalves * kQHalf;            // one query tile
     constexpr int kKVHalf = kBN * 128;                   // 64 cached tokens of 128 B
     constexpr int kKVStage = 2 * kHalves * kKVHalf;      // K then V
-    constexpr int kPBytes = kBM * 128;                   // P of one query tile: 128 rows x 64 tokens
     constexpr uint32_t kOCol = kQT * 2 * kBN;            // TMEM: S[tile][buffer] first, then O[tile]
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* sq = smem;
     uint8_t* skv = sq + kQT * kQBytes;
-    uint8_t* sp = skv + kStages * kKVStage;
-    Shared* sh = reinterpret_cast<Shared*>(sp + kQT * kPBytes);
+    Shared* sh = reinterpret_cast<Shared*>(skv + kStages * kKVStage);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -200,36 +225,33 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
             auto issue_s = [&](int t) {
                 const int s = t % kStages, buf = t & 1;
                 ok = ok && mbar_wait(&sh->kv_full[s], (t / kStages) & 1);
-                const uint32_t kaddr = smem_u32(skv + s * kKVStage);
+                const uint32_t k_lo = desc_lo(smem_u32(skv + s * kKVStage), 16);
                 for (int i = 0; i < kQT && ok; ++i) {
                     if (t >= n_steps[i]) continue;
                     ok = ok && mbar_wait(&sh->s_free[i][buf], ((t >> 1) & 1) ^ 1);
                     if (!ok) break;
                     tc_fence_after();
+                    const uint32_t q_lo = desc_lo(smem_u32(sq + i * kQBytes), 16);
 #pragma unroll
-                    for (int ks = 0; ks < D / 16; ++ks) {
-                        const uint64_t da = umma_desc_k_sw128(smem_u32(sq + i * kQBytes) + (ks / 4) * kQHalf + (ks % 4) * 32);
-                        const uint64_t db = umma_desc_k_sw128(kaddr + (ks / 4) * kKVHalf + (ks % 4) * 32);
-                        umma_bf16(tmem + (uint32_t)((i * 2 + buf) * kBN), da, db, idesc_s, ks > 0 ? 1u : 0u);
-                    }
+                    for (int ks = 0; ks < D / 16; ++ks)
+                        umma_ss(tmem + (uint32_t)((i * 2 + buf) * kBN), q_lo + (uint32_t)(((ks / 4) * kQHalf + (ks % 4) * 32) >> 4),
+                                k_lo + (uint32_t)(((ks / 4) * kKVHalf + (ks % 4) * 32) >> 4), idesc_s, ks > 0 ? 1u : 0u);
                     umma_commit(&sh->s_ready[i][buf]);
                 }
             };
             issue_s(0);
             for (int t = 0; t < steps_all && ok && !sh->abort; ++t) {
                 if (t + 1 < steps_all) issue_s(t + 1);                        // runs under this step's softmax
-                const uint32_t vaddr = smem_u32(skv + (t % kStages) * kKVStage + kHalves * kKVHalf);
+                const uint32_t v_lo = desc_lo(smem_u32(skv + (t % kStages) * kKVStage + kHalves * kKVHalf), kKVHalf);
                 for (int i = 0; i < kQT && ok; ++i) {
                     if (t >= n_steps[i]) continue;
                     ok = ok && mbar_wait(&sh->p_ready[i], t & 1);
                     if (!ok) break;
                     tc_fence_after();
 #pragma unroll
-                    for (int ks = 0; ks < kBN / 16; ++ks) {
-                        const uint64_t da = umma_desc_k_sw128(smem_u32(sp + i * kPBytes) + ks * 32);
-                        const uint64_t db = umma_desc_mn_sw128(vaddr + ks * 2048, kKVHalf);
-                        umma_bf16(tmem + kOCol + (uint32_t)(i * D), da, db, idesc_pv, (t > 0 || ks > 0) ? 1u : 0u);
-                    }
+                    for (int ks = 0; ks < kBN / 16; ++ks)
+                        umma_ts(tmem + kOCol + (uint32_t)(i * D), tmem + (uint32_t)((i * 2 + (t & 1)) * kBN + ks * 8),
+                                v_lo + (uint32_t)((ks * 2048) >> 4), idesc_pv, (t > 0 || ks > 0) ? 1u : 0u);
                     umma_commit(&sh->pv_done[i]);
                 }
                 umma_commit(&sh->kv_empty[t % kStages]);
@@ -245,7 +267,6 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         const int pos = pos0[i] + row;                // position of this row's query
         const uint32_t lane_base = tmem + ((uint32_t)(w * 32) << 16);
         const uint32_t o_addr = lane_base + kOCol + (uint32_t)(i * D);
-        uint8_t* my_p = sp + i * kPBytes;
         const int steps = n_steps[i];
         const int tid = (warp - 2 - 4 * i) * 32 + lane;   // 0..127 inside the tile's warps
         float m = kNegBig, l = 0.f;
@@ -282,13 +303,13 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
             const bool grow = __any_sync(0xffffffffu, mx > m + 8.0f);
             const float m_new = grow ? fmaxf(m, mx) : m;
             const float corr = fast_exp2(m - m_new);
-            // ---- the previous step's P V must have retired before O is rescaled and P overwritten
-            if (t > 0) {
+            // ---- O is rescaled only after the previous step's P V has retired (rare: see `grow`)
+            if (t > 0 && grow) {
                 ok = mbar_wait(&sh->pv_done[i], (t - 1) & 1);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after();
-                if (grow) {
+                {
 #pragma unroll
                     for (int c0 = 0; c0 < D; c0 += 16) {
                         uint32_t r[16];
@@ -314,21 +335,22 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
                     }
                 }
             }
-            // ---- p = 2^(s * scale - m), row sum, P (bf16) into shared memory as the A operand of P V
+            // ---- p = 2^(s * scale - m), row sum; P (bf16, two per column) goes back over the S buffer it came from
+            //      as the A operand of P V: the tensor pipe runs in order, so S of step t + 2 lands there after P V read it
             float lsum = 0.f;
 #pragma unroll
-            for (int c0 = 0; c0 < kBN; c0 += 8) {
-                uint32_t pk[4];
+            for (int c0 = 0; c0 < kBN; c0 += 32) {
+                uint32_t pk[16];
 #pragma unroll
-                for (int j = 0; j < 8; j += 2) {
+                for (int j = 0; j < 32; j += 2) {
                     const float p0 = fast_exp2(fmaf(sv[c0 + j], p.scale_log2, -m_new));
                     const float p1 = fast_exp2(fmaf(sv[c0 + j + 1], p.scale_log2, -m_new));
                     lsum += p0 + p1;
                     pk[j >> 1] = pack_bf16x2(p0, p1);
                 }
-                const int cc = c0 / 8;                               // 16-byte chunk of the row: 8 kv columns
-                *reinterpret_cast<uint4*>(my_p + row * 128 + ((cc ^ (row & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                tmem_st_32x32b_x16(s_addr + (uint32_t)(c0 / 2), pk);
             }
+            tmem_st_wait();
             l = l * corr + lsum;
             m = m_new;
             // P (and zeroed V rows) written: hand them to the MMA issuer
@@ -392,7 +414,7 @@ static aflex_status launch_t(aflex_ctx* ctx, const aflex_attn_desc* d, const voi
         !encode_tmap_2d_bf16(&tk, kv->k_cache, rows, D, (uint64_t)D * 2, kPage, 64, true) ||
         !encode_tmap_2d_bf16(&tv, kv->v_cache, rows, D, (uint64_t)D * 2, kPage, 64, true))
         return set_error(ctx, AFLEX_ERR_CUDA, "prefill attention: cuTensorMapEncodeTiled failed");
-    const size_t smem = (size_t)kQT * (D / 64) * kBM * 128 + (size_t)kStages * 2 * (D / 64) * kBN * 128 + (size_t)kQT * kBM * 128 +
+    const size_t smem = (size_t)kQT * (D / 64) * kBM * 128 + (size_t)kStages * 2 * (D / 64) * kBN * 128 +
                         sizeof(Shared) + 1024;
     static bool attr_set[2] = {false, false};
     const int ti = (D == 128) ? 1 : 0;
