@@ -3,16 +3,20 @@
 // multiplications).  Compute-bound, so it runs on the 5th-generation tensor cores:
 //
 //   CTA         = two tiles of 128 consecutive query tokens of one query head; both walk the same cached tokens,
-//               64 at a step, share the K/V stages and alternate on the tensor pipe (one tile's softmax runs
+//               128 at a step, share the K/V ring and alternate on the tensor pipe (one tile's softmax runs
 //               while the other tile's MMAs do)
-//   S = Q K^T   tcgen05.mma, both operands K-major (Q tile and K tile rows of D contiguous elements,
-//               128-byte swizzle as TMA writes them), fp32 accumulator in TMEM, double-buffered per tile
-//   softmax     four warps, one query row per thread: tcgen05.ld of its S row, causal mask, online
-//               max / sum in base 2, P rounded to bf16 into shared memory as the next MMA's A operand
-//   O += P V    tcgen05.mma with V exactly as the cache stores it ([token][D]: an MN-major B operand),
-//               accumulator in TMEM; rescaled in place (tcgen05.ld / st) when a row's maximum moves
-//   pipeline    a producer warp issues the TMA loads of the K and V pages of the coming steps (3 stages)
-//               while one thread issues MMAs; S of step t+1 is computed during the softmax of step t
+//   S = Q K^T   tcgen05.mma (128 x 128 x 16: issuing an MMA costs about as much as a 128-wide one takes, so
+//               narrower steps starve the pipe), both operands K-major (Q tile and K rows of D contiguous
+//               elements, 128-byte swizzle as TMA writes them), fp32 accumulator in TMEM, one per tile
+//   softmax     four warps per tile, one query row per thread: tcgen05.ld of its S row, causal mask, online
+//               max / sum in base 2, P rounded to bf16 and stored back over the S columns (tcgen05.st)
+//   O += P V    tcgen05.mma with A = P read from TMEM and B = V exactly as the cache stores it ([token][D]:
+//               an MN-major operand); accumulator in TMEM, rescaled in place only when a row's maximum
+//               outgrows the reference by 2^8
+//   pipeline    a producer warp issues the TMA loads of the K rows and the V rows of the coming steps into a
+//               ring of slots (K(0) V(0) K(1) V(1) ...: a slot is free as soon as its own MMAs retire);
+//               one thread issues MMAs in the order P V(t), S(t+1) per tile, so the pipe's in-order execution
+//               keeps S(t+1) from landing on P(t) before it was read
 //
 // Query i of a sequence with n cached tokens of which the last m are being prefilled sits at position
 // n - m + i and sees cached tokens 0 .. n - m + i.  Cache slots beyond n may hold anything (NaN too):
@@ -28,10 +32,11 @@ namespace pa {
 
 constexpr int kBM = 128;          // query rows per tile
 constexpr int kQT = 2;            // query tiles per CTA (they share the K/V stages and alternate on the tensor pipe)
-constexpr int kBN = 64;           // cached tokens per step
+constexpr int kBN = 128;          // cached tokens per step
 constexpr int kPage = 16;
 constexpr int kPagesPerStep = kBN / kPage;
-constexpr int kStages = 4;
+constexpr int kMaxSlots = 6;
+constexpr int slots_for(int D) { return D == 128 ? 5 : 6; }   // K or V rows of one step per slot (32 KB at D = 128)
 constexpr int kThreads = (2 + 4 * kQT) * 32;   // producer, MMA issuer, four softmax warps per query tile
 constexpr float kNegBig = -1.0e30f;
 
@@ -49,9 +54,8 @@ struct Params {
 
 struct __align__(8) Shared {
     uint64_t q_full;
-    uint64_t kv_full[kStages], kv_empty[kStages];
-    uint64_t s_ready[kQT][2], s_free[kQT][2];
-    uint64_t p_ready[kQT], pv_done[kQT];
+    uint64_t kv_full[kMaxSlots], kv_empty[kMaxSlots];
+    uint64_t s_ready[kQT], p_ready[kQT], pv_done[kQT];
     uint32_t tmem_base;
     volatile int abort;
 };
@@ -113,15 +117,16 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     constexpr int kHalves = D / 64;
     constexpr int kQHalf = kBM * 128;                    // 128 query rows of 128 B
     constexpr int kQBytes = kHalves * kQHalf;            // one query tile
-    constexpr int kKVHalf = kBN * 128;                   // 64 cached tokens of 128 B
-    constexpr int kKVStage = 2 * kHalves * kKVHalf;      // K then V
-    constexpr uint32_t kOCol = kQT * 2 * kBN;            // TMEM: S[tile][buffer] first, then O[tile]
+    constexpr int kKVHalf = kBN * 128;                   // 128 cached tokens of 128 B
+    constexpr int kSlotBytes = kHalves * kKVHalf;        // the K rows, or the V rows, of one step
+    constexpr int kSlots = slots_for(D);                 // ring of K and V slots: K(0) V(0) K(1) V(1) ...
+    constexpr uint32_t kOCol = kQT * kBN;                // TMEM: S[tile] (P over it) first, then O[tile]
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* sq = smem;
     uint8_t* skv = sq + kQT * kQBytes;
-    Shared* sh = reinterpret_cast<Shared*>(skv + kStages * kKVStage);
+    Shared* sh = reinterpret_cast<Shared*>(skv + kSlots * kSlotBytes);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -162,9 +167,9 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
 
     if (threadIdx.x == 0) {
         mbar_init(&sh->q_full, 1);
-        for (int s = 0; s < kStages; ++s) { mbar_init(&sh->kv_full[s], 1); mbar_init(&sh->kv_empty[s], 1); }
+        for (int s = 0; s < kSlots; ++s) { mbar_init(&sh->kv_full[s], 1); mbar_init(&sh->kv_empty[s], 1); }
         for (int i = 0; i < kQT; ++i) {
-            for (int k = 0; k < 2; ++k) { mbar_init(&sh->s_ready[i][k], 1); mbar_init(&sh->s_free[i][k], 4); }
+            mbar_init(&sh->s_ready[i], 1);
             mbar_init(&sh->p_ready[i], 4);
             mbar_init(&sh->pv_done[i], 1);
         }
@@ -188,11 +193,10 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
                 for (int hf = 0; hf < kHalves; ++hf)
                     tma_load_2d(sq + i * kQBytes + hf * kQHalf, &tmap_q, h * D + hf * 64, q_row0 + i * kBM, &sh->q_full);
         }
-        // one lane per (K | V, 64-column half, page) box of a step
+        // one lane per (64-column half, page) box of a slot; slot 2t holds the K rows of step t, slot 2t + 1 its V rows
         const int page = lane % kPagesPerStep;
-        const int hf = (lane / kPagesPerStep) % kHalves;
-        const int isv = lane / (kPagesPerStep * kHalves);
-        const bool op_lane = lane < 2 * kHalves * kPagesPerStep;
+        const int hf = lane / kPagesPerStep;
+        const bool op_lane = lane < kHalves * kPagesPerStep;
         auto page_id = [&](int t) -> int {
             const int idx = t * kPagesPerStep + page;
             return (op_lane && idx * kPage < kv_end_all) ? p.page_table[(size_t)b * p.max_pages + idx] : 0;
@@ -200,19 +204,22 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         int id = page_id(0);
         for (int t = 0; t < steps_all; ++t) {
             const int id_next = (t + 1 < steps_all) ? page_id(t + 1) : 0;     // one step ahead of the ring
-            const int s = t % kStages;
-            bool ok = mbar_wait(&sh->kv_empty[s], ((t / kStages) & 1) ^ 1);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok || sh->abort) { if (lane == 0) { sh->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); } break; }
             const int np = min(kPagesPerStep, (kv_end_all - t * kBN + kPage - 1) / kPage);
-            if (lane == 0) mbar_expect_tx(&sh->kv_full[s], (uint32_t)(np * 2 * kHalves * kPage * 128));
-            __syncwarp();
-            if (op_lane && page < np) {
-                int pid = id;
-                if (pid < 0 || pid >= p.num_pages) { atomicExch(p.status, AFLEX_ERR_BOUNDS); pid = 0; }
-                uint8_t* dst = skv + s * kKVStage + isv * (kHalves * kKVHalf) + hf * kKVHalf + page * (kPage * 128);
-                tma_load_2d(dst, isv ? &tmap_v : &tmap_k, hf * 64, (pid * p.Hkv + g) * kPage, &sh->kv_full[s]);
+            int pid = id;
+            if (op_lane && page < np && (pid < 0 || pid >= p.num_pages)) { atomicExch(p.status, AFLEX_ERR_BOUNDS); pid = 0; }
+            bool ok = true;
+            for (int isv = 0; isv < 2 && ok; ++isv) {
+                const int j = 2 * t + isv, s = j % kSlots;
+                ok = mbar_wait(&sh->kv_empty[s], ((j / kSlots) & 1) ^ 1);
+                ok = __all_sync(0xffffffffu, ok) && !sh->abort;
+                if (!ok) break;
+                if (lane == 0) mbar_expect_tx(&sh->kv_full[s], (uint32_t)(np * kHalves * kPage * 128));
+                __syncwarp();
+                if (op_lane && page < np)
+                    tma_load_2d(skv + s * kSlotBytes + hf * kKVHalf + page * (kPage * 128), isv ? &tmap_v : &tmap_k, hf * 64,
+                                (pid * p.Hkv + g) * kPage, &sh->kv_full[s]);
             }
+            if (!ok) { if (lane == 0) { sh->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); } break; }
             id = id_next;
         }
     } else if (warp == 1) {
@@ -221,40 +228,43 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
             const uint32_t idesc_s = umma_idesc_bf16(kBM, kBN);
             const uint32_t idesc_pv = umma_idesc_bf16(kBM, D) | (1u << 16);      // B operand (V) is MN-major
             bool ok = mbar_wait(&sh->q_full, 0);
-            // S of step t for both query tiles (needs the step's K/V and the tiles' free S buffers)
-            auto issue_s = [&](int t) {
-                const int s = t % kStages, buf = t & 1;
-                ok = ok && mbar_wait(&sh->kv_full[s], (t / kStages) & 1);
-                const uint32_t k_lo = desc_lo(smem_u32(skv + s * kKVStage), 16);
-                for (int i = 0; i < kQT && ok; ++i) {
-                    if (t >= n_steps[i]) continue;
-                    ok = ok && mbar_wait(&sh->s_free[i][buf], ((t >> 1) & 1) ^ 1);
-                    if (!ok) break;
-                    tc_fence_after();
-                    const uint32_t q_lo = desc_lo(smem_u32(sq + i * kQBytes), 16);
+            // S of step t of query tile i (needs the step's K rows; the tile's S / P columns are free once its
+            // previous P V has been issued: the tensor pipe runs in order)
+            auto issue_s = [&](int t, int i) {
+                if (t >= n_steps[i]) return;
+                const int j = 2 * t, s = j % kSlots;
+                ok = ok && mbar_wait(&sh->kv_full[s], (j / kSlots) & 1);
+                if (!ok) return;
+                tc_fence_after();
+                const uint32_t k_lo = desc_lo(smem_u32(skv + s * kSlotBytes), 16);
+                const uint32_t q_lo = desc_lo(smem_u32(sq + i * kQBytes), 16);
 #pragma unroll
-                    for (int ks = 0; ks < D / 16; ++ks)
-                        umma_ss(tmem + (uint32_t)((i * 2 + buf) * kBN), q_lo + (uint32_t)(((ks / 4) * kQHalf + (ks % 4) * 32) >> 4),
-                                k_lo + (uint32_t)(((ks / 4) * kKVHalf + (ks % 4) * 32) >> 4), idesc_s, ks > 0 ? 1u : 0u);
-                    umma_commit(&sh->s_ready[i][buf]);
-                }
+                for (int ks = 0; ks < D / 16; ++ks)
+                    umma_ss(tmem + (uint32_t)(i * kBN), q_lo + (uint32_t)(((ks / 4) * kQHalf + (ks % 4) * 32) >> 4),
+                            k_lo + (uint32_t)(((ks / 4) * kKVHalf + (ks % 4) * 32) >> 4), idesc_s, ks > 0 ? 1u : 0u);
+                umma_commit(&sh->s_ready[i]);
             };
-            issue_s(0);
+            for (int i = 0; i < kQT; ++i) issue_s(0, i);
+            if (steps_all > 0 && ok) umma_commit(&sh->kv_empty[0]);
             for (int t = 0; t < steps_all && ok && !sh->abort; ++t) {
-                if (t + 1 < steps_all) issue_s(t + 1);                        // runs under this step's softmax
-                const uint32_t v_lo = desc_lo(smem_u32(skv + (t % kStages) * kKVStage + kHalves * kKVHalf), kKVHalf);
+                const int jv = 2 * t + 1, sv_ = jv % kSlots;
                 for (int i = 0; i < kQT && ok; ++i) {
                     if (t >= n_steps[i]) continue;
                     ok = ok && mbar_wait(&sh->p_ready[i], t & 1);
+                    ok = ok && mbar_wait(&sh->kv_full[sv_], (jv / kSlots) & 1);
                     if (!ok) break;
                     tc_fence_after();
+                    const uint32_t v_lo = desc_lo(smem_u32(skv + sv_ * kSlotBytes), kKVHalf);
 #pragma unroll
                     for (int ks = 0; ks < kBN / 16; ++ks)
-                        umma_ts(tmem + kOCol + (uint32_t)(i * D), tmem + (uint32_t)((i * 2 + (t & 1)) * kBN + ks * 8),
-                                v_lo + (uint32_t)((ks * 2048) >> 4), idesc_pv, (t > 0 || ks > 0) ? 1u : 0u);
+                        umma_ts(tmem + kOCol + (uint32_t)(i * D), tmem + (uint32_t)(i * kBN + ks * 8), v_lo + (uint32_t)((ks * 2048) >> 4),
+                                idesc_pv, (t > 0 || ks > 0) ? 1u : 0u);
                     umma_commit(&sh->pv_done[i]);
+                    issue_s(t + 1, i);                                       // runs under the other tile's softmax
                 }
-                umma_commit(&sh->kv_empty[t % kStages]);
+                if (!ok) break;
+                umma_commit(&sh->kv_empty[sv_]);                             // V of this step
+                if (t + 1 < steps_all) umma_commit(&sh->kv_empty[(2 * t + 2) % kSlots]);   // K of the next
             }
             if (!ok) { sh->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); }
         }
@@ -266,38 +276,36 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         const bool row_ok = row < rows_valid[i];
         const int pos = pos0[i] + row;                // position of this row's query
         const uint32_t lane_base = tmem + ((uint32_t)(w * 32) << 16);
+        const uint32_t s_addr = lane_base + (uint32_t)(i * kBN);
         const uint32_t o_addr = lane_base + kOCol + (uint32_t)(i * D);
         const int steps = n_steps[i];
         const int tid = (warp - 2 - 4 * i) * 32 + lane;   // 0..127 inside the tile's warps
         float m = kNegBig, l = 0.f;
         bool ok = true;
         for (int t = 0; t < steps; ++t) {
-            const int buf = t & 1;
-            ok = mbar_wait(&sh->s_ready[i][buf], (t >> 1) & 1);
+            ok = mbar_wait(&sh->s_ready[i], t & 1);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok || sh->abort) break;
             tc_fence_after();
-            const uint32_t s_addr = lane_base + (uint32_t)((i * 2 + buf) * kBN);
             const int col0 = t * kBN;
-            // ---- this thread's S row into registers (one wait for all loads); the buffer is free at once
+            // ---- this thread's S row into registers (one wait for all loads)
             float sv[kBN];
 #pragma unroll
             for (int c0 = 0; c0 < kBN; c0 += 16)
                 tmem_ld_32x32b_x16(s_addr + (uint32_t)c0, *reinterpret_cast<uint32_t(*)[16]>(&sv[c0]));
             tmem_ld_wait();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sh->s_free[i][buf]);
             // causal mask: only steps that reach past the tile's first query need it
             if (col0 + kBN - 1 > pos0[i] || !row_ok) {
 #pragma unroll
                 for (int j = 0; j < kBN; ++j)
                     if (!(row_ok && col0 + j <= pos)) sv[j] = -INFINITY;
             }
-            float mx = -INFINITY;
+            float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-            for (int j = 0; j < kBN; ++j) mx = fmaxf(mx, sv[j]);
-            mx *= p.scale_log2;
+            for (int j = 0; j < kBN; j += 4) {
+                mx0 = fmaxf(mx0, sv[j]); mx1 = fmaxf(mx1, sv[j + 1]); mx2 = fmaxf(mx2, sv[j + 2]); mx3 = fmaxf(mx3, sv[j + 3]);
+            }
+            const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2;
             // The reference maximum m moves only when some row of the warp outgrows it by more than 2^8: until
             // then p = 2^(s - m) stays below 256 (harmless in bf16 / fp32) and O needs no rescaling.
             const bool grow = __any_sync(0xffffffffu, mx > m + 8.0f);
@@ -309,17 +317,14 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after();
-                {
 #pragma unroll
-                    for (int c0 = 0; c0 < D; c0 += 16) {
-                        uint32_t r[16];
-                        tmem_ld_32x32b_x16(o_addr + (uint32_t)c0, r);
-                        tmem_ld_wait();
+                for (int c0 = 0; c0 < D; c0 += 16) {
+                    uint32_t r[16];
+                    tmem_ld_32x32b_x16(o_addr + (uint32_t)c0, r);
+                    tmem_ld_wait();
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * corr);
-                        tmem_st_32x32b_x16(o_addr + (uint32_t)c0, r);
-                    }
-                    tmem_st_wait();
+                    for (int j = 0; j < 16; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * corr);
+                    tmem_st_32x32b_x16(o_addr + (uint32_t)c0, r);
                 }
             }
             // ---- V rows that were not loaded or lie past the sequence's end: zero them, whatever they hold
@@ -328,16 +333,21 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
                 const int np = min(kPagesPerStep, (kv_end_all - col0 + kPage - 1) / kPage);
                 const int n_here = max(0, min(n_cached - col0, np * kPage));
                 if (n_here < kBN) {
-                    uint8_t* vbase = skv + (t % kStages) * kKVStage + kHalves * kKVHalf;
+                    const int jv = 2 * t + 1, sv_ = jv % kSlots;
+                    ok = mbar_wait(&sh->kv_full[sv_], (jv / kSlots) & 1);        // the loaded rows must have landed first
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    uint8_t* vbase = skv + sv_ * kSlotBytes;
                     for (int k = tid; k < (kBN - n_here) * kHalves * 8; k += 128) {
                         const int r_ = n_here + k / (kHalves * 8), c_ = k % (kHalves * 8);
                         *reinterpret_cast<uint4*>(vbase + (c_ / 8) * kKVHalf + r_ * 128 + (c_ % 8) * 16) = make_uint4(0, 0, 0, 0);
                     }
+                    fence_proxy_async();
                 }
             }
-            // ---- p = 2^(s * scale - m), row sum; P (bf16, two per column) goes back over the S buffer it came from
-            //      as the A operand of P V: the tensor pipe runs in order, so S of step t + 2 lands there after P V read it
-            float lsum = 0.f;
+            // ---- p = 2^(s * scale - m), row sum; P (bf16, two per column) goes back over the S columns it came
+            //      from as the A operand of P V (the tensor pipe runs in order: the next S lands there after P V read it)
+            float l0 = 0.f, l1 = 0.f;
 #pragma unroll
             for (int c0 = 0; c0 < kBN; c0 += 32) {
                 uint32_t pk[16];
@@ -345,16 +355,15 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
                 for (int j = 0; j < 32; j += 2) {
                     const float p0 = fast_exp2(fmaf(sv[c0 + j], p.scale_log2, -m_new));
                     const float p1 = fast_exp2(fmaf(sv[c0 + j + 1], p.scale_log2, -m_new));
-                    lsum += p0 + p1;
+                    l0 += p0; l1 += p1;
                     pk[j >> 1] = pack_bf16x2(p0, p1);
                 }
                 tmem_st_32x32b_x16(s_addr + (uint32_t)(c0 / 2), pk);
             }
             tmem_st_wait();
-            l = l * corr + lsum;
+            l = l * corr + (l0 + l1);
             m = m_new;
             // P (and zeroed V rows) written: hand them to the MMA issuer
-            fence_proxy_async();
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&sh->p_ready[i]);
@@ -414,7 +423,7 @@ static aflex_status launch_t(aflex_ctx* ctx, const aflex_attn_desc* d, const voi
         !encode_tmap_2d_bf16(&tk, kv->k_cache, rows, D, (uint64_t)D * 2, kPage, 64, true) ||
         !encode_tmap_2d_bf16(&tv, kv->v_cache, rows, D, (uint64_t)D * 2, kPage, 64, true))
         return set_error(ctx, AFLEX_ERR_CUDA, "prefill attention: cuTensorMapEncodeTiled failed");
-    const size_t smem = (size_t)kQT * (D / 64) * kBM * 128 + (size_t)kStages * 2 * (D / 64) * kBN * 128 +
+    const size_t smem = (size_t)kQT * (D / 64) * kBM * 128 + (size_t)slots_for(D) * (D / 64) * kBN * 128 +
                         sizeof(Shared) + 1024;
     static bool attr_set[2] = {false, false};
     const int ti = (D == 128) ? 1 : 0;
