@@ -37,7 +37,9 @@ constexpr int kPage = 16;
 constexpr int kPagesPerStep = kBN / kPage;
 constexpr int kMaxSlots = 6;
 constexpr int slots_for(int D) { return D == 128 ? 5 : 6; }   // K or V rows of one step per slot (32 KB at D = 128)
-constexpr int kThreads = (2 + 4 * kQT) * 32;   // producer, MMA issuer, four softmax warps per query tile
+constexpr int kSoftmaxWarps = 4 * kQT;         // warp groups 0 and 1: four softmax warps per query tile
+constexpr int kThreads = (kSoftmaxWarps + 4) * 32;   // warp group 2: producer, MMA issuer, two idle warps
+constexpr int kRegsSoftmax = 216, kRegsIssue = 72;   // registers per thread after the warp groups trade them
 constexpr float kNegBig = -1.0e30f;
 
 struct Params {
@@ -177,7 +179,7 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         fence_mbar_init();
         prefetch_tmap(&tmap_q); prefetch_tmap(&tmap_k); prefetch_tmap(&tmap_v);
     }
-    if (warp == 1) { tmem_alloc(&sh->tmem_base, 512); tmem_relinquish(); }
+    if (warp == kSoftmaxWarps + 1) { tmem_alloc(&sh->tmem_base, 512); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -185,7 +187,9 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     pdl_launch_dependents();
     pdl_wait();
 
-    if (warp == 0) {
+    if (warp >= kSoftmaxWarps) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsIssue));
+    if (warp == kSoftmaxWarps) {
         // ------------------------------------------------------------------ producer warp
         if (lane == 0) {
             mbar_expect_tx(&sh->q_full, (uint32_t)(kQT * kQBytes));
@@ -222,7 +226,7 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
             if (!ok) { if (lane == 0) { sh->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); } break; }
             id = id_next;
         }
-    } else if (warp == 1) {
+    } else if (warp == kSoftmaxWarps + 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             const uint32_t idesc_s = umma_idesc_bf16(kBM, kBN);
@@ -268,9 +272,11 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
             }
             if (!ok) { sh->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); }
         }
+    }
     } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
         // ------------------------------------------------------------------ softmax warps: one query row per thread
-        const int i = (warp - 2) / 4;                 // query tile of this warp
+        const int i = warp / 4;                       // query tile of this warp
         const int w = warp & 3;                       // TMEM lane quadrant of this warp
         const int row = w * 32 + lane;
         const bool row_ok = row < rows_valid[i];
@@ -279,7 +285,7 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         const uint32_t s_addr = lane_base + (uint32_t)(i * kBN);
         const uint32_t o_addr = lane_base + kOCol + (uint32_t)(i * D);
         const int steps = n_steps[i];
-        const int tid = (warp - 2 - 4 * i) * 32 + lane;   // 0..127 inside the tile's warps
+        const int tid = (warp & 3) * 32 + lane;       // 0..127 inside the tile's warps
         float m = kNegBig, l = 0.f;
         bool ok = true;
         for (int t = 0; t < steps; ++t) {
@@ -397,7 +403,7 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem, 512); }
+    if (warp == kSoftmaxWarps + 1) { tc_fence_after(); tmem_dealloc(tmem, 512); }
 }
 
 template <int D>
