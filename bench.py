@@ -23,6 +23,7 @@ own GPU (the path has no exchange step on one node); value = N * B / max-over-ra
 from __future__ import annotations
 
 import argparse
+import dataclasses
 import json
 import os
 import subprocess
@@ -263,6 +264,66 @@ def run_ffn_sweep(args, cfg, local_rank, device, peaks):
     ctx.close()
 
 
+def run_prefill(args, cfg, local_rank, device, peaks):
+    """Prefill (causal) attention over the paged cache at the configuration's head shape: whole prompts of several
+    lengths, a ragged batch and a chunk appended to a long cached prefix.  Compute-bound, so each row reports
+    TFLOP/s of the causal flops (4 Hq D per visible query-key pair) against the measured dense bf16 peaks."""
+    from paper_2608_01891_b200 import aflex as AF
+    Hq, Hkv, D = cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim
+    ctx = AF.Context(local_rank, 1 << 26)
+    stream = torch.cuda.current_stream()
+    desc = AF.attn_desc(Hq, Hkv, D)
+    rng = np.random.default_rng(20260801)
+    cases = [("whole prompts 8 x 1024", [1024] * 8, None), ("whole prompts 8 x 2048", [2048] * 8, None),
+             ("whole prompts 4 x 4096", [4096] * 4, None), ("whole prompts 2 x 8192", [8192] * 2, None),
+             ("whole prompt 1 x 16384", [16384], None),
+             ("ragged prompts, 8 lengths in [512, 4096]", [int(v) for v in rng.integers(512, 4097, size=8)], None),
+             ("chunk of 2048 onto 8192 cached, 2 sequences", [10240] * 2, [2048] * 2)]
+    if args.prefill_case >= 0:
+        cases = cases[args.prefill_case:args.prefill_case + 1]
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    rows = []
+    for name, cached, new in cases:
+        new = cached if new is None else new
+        B = len(cached)
+        c = dataclasses.replace(cfg, batch=B)
+        lens = np.asarray(cached, dtype=np.int32)
+        kvh = IN.make_paged_kv(c, lens, device=device)
+        kv = AF.make_kv(kvh.k_cache, kvh.v_cache, kvh.page_table.to(device), kvh.seq_lens.to(device), kvh.seq_lens)
+        qo = torch.zeros(B + 1, dtype=torch.int32)
+        qo[1:] = torch.cumsum(torch.tensor(new, dtype=torch.int32), 0)
+        qod = qo.to(device)
+        T = int(qo[-1])
+        q = (torch.randn(T, Hq, D, device=device) * 1.0).to(torch.bfloat16)
+        out = torch.empty_like(q)
+        pairs = sum(m * (n - m) + m * (m + 1) // 2 for n, m in zip(cached, new))
+        flops = 4.0 * Hq * D * pairs
+        for _ in range(max(3, args.warmup)):
+            ctx.attn_prefill(desc, q, kv, qod, qo, out, stream)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(args.steps):
+            ctx.attn_prefill(desc, q, kv, qod, qo, out, stream)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        us = 1e3 * e0.elapsed_time(e1) / args.steps
+        tf = flops / us / 1e6
+        rows.append({"case": name, "query_tokens": T, "us": round(us, 1), "tflops": round(tf, 1),
+                     "frac_bf16_burst": round(tf / peaks["bf16_tflops"], 4),
+                     "frac_bf16_sustained": round(tf / peaks["bf16_tflops_sustained"], 4)})
+        del kvh, kv, q, out
+    assert ctx.device_status() == AF.OK
+    line = {"metric": "prefill attention throughput (causal flops)", "unit": "TFLOP/s", "dtype": "bf16", "data": "synthetic",
+            "steps": args.steps, "warmup": max(3, args.warmup),
+            "config": {"workload": f"causal attention over the paged cache, Hq={Hq}, Hkv={Hkv}, D={D}",
+                       "l2": "q, out and K/V of a case exceed L2 together; no flush between iterations"},
+            "peaks": peaks, "clocks": sampler.stop(), "cases": rows}
+    print(json.dumps(line), flush=True)
+    ctx.close()
+
+
 def run_decoder_chain(args, cfg, local_rank, device, peaks):
     """Whole decoder layers chained (aflex_decoder_layers): L layers, each with its own weights and KV cache,
     at every microbatch depth of the configuration.  One JSON line: time per layer, tokens/s, the share of the
@@ -439,6 +500,11 @@ def main():
     ap.add_argument("--energy-ops", action="store_true",
                     help="instead of the layer step: time and NVML energy per token of attention, the dense FFN at "
                          "T = 32 and T = 2048 and the layer step, each alone, at the clocks the GPU is found at")
+    ap.add_argument("--prefill", action="store_true",
+                    help="instead of the layer step: prefill (causal) attention at the configuration's head shape over "
+                         "several prompt mixes, TFLOP/s against the measured bf16 peaks")
+    ap.add_argument("--prefill-case", type=int, default=-1,
+                    help="with --prefill: run only this case of the list (a small single-kernel run for a profiler)")
     ap.add_argument("--energy", action="store_true",
                     help="also read the NVML energy counter around a >= 2 s loop of the step (default clocks)")
     args = ap.parse_args()
@@ -481,6 +547,10 @@ def main():
     if args.energy_ops:
         if rank == 0:
             run_energy_ops(args, cfg, local_rank, device, peaks)
+        return
+    if args.prefill:
+        if rank == 0:
+            run_prefill(args, cfg, local_rank, device, peaks)
         return
     wl = build_workload(cfg, device)
     lens_np = wl["kvh"].seq_lens.numpy()

@@ -93,3 +93,67 @@ def test_prefill_argument_checks(ctx):
     with pytest.raises(AF.AflexError):
         ctx.attn_prefill(AF.attn_desc(8, 2, 128), q, kv, bad.to(DEV), bad, out)
     assert ctx.device_status() == AF.OK
+
+
+@pytest.mark.parametrize("direction", ["rising", "falling"])
+def test_prefill_scores_that_ramp_along_the_sequence(ctx, direction):
+    """Keys built so that every query's score ramps by about 37 (base 2) per 128 cached tokens.  Rising: each step's
+    maximum outgrows the standing reference, so the accumulator is rescaled at every step; falling: everything after
+    the first steps underflows to zero.  Both are exact cases for an online softmax, and a worst case for one that
+    moves its reference lazily."""
+    Hq, Hkv, D = 8, 2, 128
+    lens = np.asarray([1000, 333], dtype=np.int32)
+    cfg = IN.LayerConfig(41, "prefill-ramp", len(lens), Hq, Hkv, D, 64, 64)
+    kvh = IN.make_paged_kv(cfg, lens, poison=True)
+    g = torch.Generator().manual_seed(41)
+    u = torch.randn(Hkv, D, generator=g)
+    u = u / u.norm(dim=-1, keepdim=True)
+    table = kvh.page_table.numpy()
+    for b, n in enumerate(lens):
+        j = torch.arange(int(n), dtype=torch.float32)
+        ramp = 0.29 * 11.3 * (j if direction == "rising" else (float(n) - j))      # q.k * scale grows by 0.2 per token
+        k = (u[None, :, :] * ramp[:, None, None] / 8.0 + 0.05 * torch.randn(int(n), Hkv, D, generator=g)).to(torch.bfloat16)
+        pages = torch.from_numpy(table[b, : (int(n) + 15) // 16].astype(np.int64))
+        for t0 in range(0, int(n), 16):
+            w = min(16, int(n) - t0)
+            kvh.k_cache[pages[t0 // 16], :, :w, :] = k[t0:t0 + w].transpose(0, 1)
+    q_off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    T = int(q_off[-1])
+    q = (8.0 * u.repeat_interleave(Hq // Hkv, dim=0)[None, :, :] + 0.1 * torch.randn(T, Hq, D, generator=g)).to(torch.bfloat16)
+    kv = AF.make_kv(kvh.k_cache.to(DEV), kvh.v_cache.to(DEV), kvh.page_table.to(DEV), kvh.seq_lens.to(DEV), kvh.seq_lens)
+    out = torch.full((T, Hq, D), float("nan"), dtype=torch.bfloat16, device=DEV)
+    qo = torch.from_numpy(q_off)
+    ctx.attn_prefill(AF.attn_desc(Hq, Hkv, D), q.to(DEV), kv, qo.to(DEV), qo, out)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == AF.OK
+    want = O.attn_prefill(u16(q), u16(kvh.k_cache), u16(kvh.v_cache), table, lens, q_off)
+    assert row_rel_err(f64(out), want) <= TOL_ATTN
+
+
+def test_prefill_full_size_sampled_rows(ctx):
+    """The head shape and prompt lengths bench.py times (64 query heads, 8 KV heads, head size 128; 16 384 and 4 099
+    tokens), checked on sampled query rows: a prefill row is decode attention over the sequence cut after that row."""
+    Hq, Hkv, D = 64, 8, 128
+    lens = np.asarray([16384, 4099], dtype=np.int32)
+    cfg = IN.LayerConfig(42, "prefill-full", len(lens), Hq, Hkv, D, 64, 64)
+    kvh = IN.make_paged_kv(cfg, lens, device=DEV)
+    q_off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    T = int(q_off[-1])
+    g = torch.Generator(device=DEV).manual_seed(42)
+    q = torch.randn(T, Hq, D, generator=g, device=DEV).to(torch.bfloat16)
+    kv = AF.make_kv(kvh.k_cache, kvh.v_cache, kvh.page_table.to(DEV), kvh.seq_lens.to(DEV), kvh.seq_lens)
+    out = torch.full((T, Hq, D), float("nan"), dtype=torch.bfloat16, device=DEV)
+    qo = torch.from_numpy(q_off)
+    ctx.attn_prefill(AF.attn_desc(Hq, Hkv, D), q, kv, qo.to(DEV), qo, out)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == AF.OK
+    assert torch.isfinite(out.float()).all()
+    rng = np.random.default_rng(42)
+    rows = [(0, 0), (0, 1), (0, 127), (0, 128), (0, 255), (0, 256), (0, 16383), (1, 0), (1, 4095), (1, 4096), (1, 4098)]
+    rows += [(0, int(r)) for r in rng.integers(0, 16384, size=12)] + [(1, int(r)) for r in rng.integers(0, 4099, size=6)]
+    table = kvh.page_table.numpy()
+    q_s = torch.stack([q[int(q_off[b]) + r] for b, r in rows]).cpu()
+    got = torch.stack([out[int(q_off[b]) + r] for b, r in rows]).cpu()
+    want, _ = O.attn_decode(u16(q_s), u16(kvh.k_cache.cpu()), u16(kvh.v_cache.cpu()),
+                            np.stack([table[b] for b, _ in rows]), np.asarray([r + 1 for _, r in rows], dtype=np.int32))
+    assert row_rel_err(f64(got), want) <= TOL_ATTN
