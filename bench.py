@@ -324,6 +324,51 @@ def run_prefill(args, cfg, local_rank, device, peaks):
     ctx.close()
 
 
+def run_moe_sweep(args, cfg, local_rank, device, peaks):
+    """Top-k MoE FFN (router logits given) at the configuration's (H, I, E, K) over a range of token counts: from the
+    decode regime (every expert's weights streamed for a handful of rows) to the prefill regime (hundreds to thousands
+    of rows per expert, tensor-core bound)."""
+    from paper_2608_01891_b200 import aflex as AF
+    H, I, E, K = cfg.hidden, cfg.inter, cfg.num_experts, cfg.top_k
+    wg, wu, wd = IN.make_ffn_weights(cfg, device=device)
+    ctx = AF.Context(local_rank, 8 << 30)
+    stream = torch.cuda.current_stream()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    rows = []
+    for T in (64, 256, 512, 1024, 2048, 4096, 8192):
+        x = IN.make_x(cfg, device=device, tokens=T)
+        logits = IN.make_router_logits(cfg, tokens=T).to(device)
+        y = torch.empty(T, H, dtype=torch.bfloat16, device=device)
+        counts = torch.zeros(E, dtype=torch.int32, device=device)
+        for _ in range(max(3, args.warmup)):
+            ctx.ffn_moe(x, wg, wu, wd, K, y, router_logits=logits, expert_counts=counts, stream=stream)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n = max(10, args.steps // 2)
+        e0.record(stream)
+        for _ in range(n):
+            ctx.ffn_moe(x, wg, wu, wd, K, y, router_logits=logits, expert_counts=counts, stream=stream)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        us = 1e3 * e0.elapsed_time(e1) / n
+        flops = 6.0 * T * K * H * I
+        wbytes = 3.0 * E * H * I * 2 + 2.0 * T * K * H * 2 + 2.0 * T * K * I * 2
+        rows.append({"T": T, "rows_per_expert": counts.cpu().tolist(), "us": round(us, 1), "tflops": round(flops / us / 1e6, 1),
+                     "frac_bf16_burst": round(flops / us / 1e6 / peaks["bf16_tflops"], 4),
+                     "frac_bf16_sustained": round(flops / us / 1e6 / peaks["bf16_tflops_sustained"], 4),
+                     "weight_stream_gbs": round(wbytes / us / 1e3, 1),
+                     "frac_hbm": round(wbytes / us / 1e3 / peaks["hbm_gbs"], 4)})
+    assert ctx.device_status() == AF.OK
+    line = {"metric": f"MoE FFN throughput vs tokens (H={H}, I={I}, E={E}, top-{K})", "unit": "TFLOP/s", "dtype": "bf16",
+            "data": "synthetic",
+            "config": {"workload": f"moe ffn token sweep, config {cfg.cfg_id} routing, H={H}, I={I}, E={E}, K={K}",
+                       "l2": "expert weights (2.8 GB) larger than L2, no flush"},
+            "peaks": peaks, "clocks": sampler.stop(), "sweep": rows}
+    print(json.dumps(line), flush=True)
+    ctx.close()
+
+
 def run_decoder_chain(args, cfg, local_rank, device, peaks):
     """Whole decoder layers chained (aflex_decoder_layers): L layers, each with its own weights and KV cache,
     at every microbatch depth of the configuration.  One JSON line: time per layer, tokens/s, the share of the
@@ -538,7 +583,7 @@ def main():
     peaks = load_peaks()
     if args.ffn_sweep:
         if rank == 0:
-            run_ffn_sweep(args, cfg, local_rank, device, peaks)
+            (run_moe_sweep if cfg.num_experts > 0 else run_ffn_sweep)(args, cfg, local_rank, device, peaks)
         return
     if args.decoder_layers > 0:
         if rank == 0:

@@ -585,6 +585,7 @@ static int round_up(int a, int b) { return (a + b - 1) / b * b; }
 
 // Token-tile width: the fewest tiles of at most 256 rows, all of (nearly) the same width, so that
 // e.g. 384 rows become 192 + 192 rather than 256 + 128.
+constexpr int kGroupedWideRowsLinear = 128, kGroupedWideRowsGateUp = 512;
 static int pick_n_tile(int rows_max) {
     const int rows = rows_max < 16 ? 16 : rows_max;
     const int tiles = (rows + 255) / 256;
@@ -635,7 +636,18 @@ static bool make_config(int mode, int T, int N, int K, int rows_max, int E, int 
     // Grouped form: cap the tile at 128 token rows so the two gate/up accumulators stay double-buffered
     // in TMEM; a hot expert with more rows becomes two adjacent tiles whose weight tiles are read by
     // neighbouring CTAs at the same time (the second read is an L2 hit).
-    if (E > 0 && p.n_tile > 128) p.n_tile = 128;
+    // That is the decode regime (tens of rows per expert).  With hundreds of rows per expert (prefill) the grouped
+    // form is a tensor-core kernel like the dense one, and a 128-row tile's MMAs read as many shared-memory bytes per
+    // cycle as the SM delivers.  Measured at the Mixtral shape: the down projection (one accumulator, still double-
+    // buffered at 256 rows) gains from an average of 128 rows per expert on (328 -> 289 us at 256, 2388 -> 1582 us at
+    // 2048); gate/up (two accumulators: 256 rows fill TMEM, no double buffering) only from about 512 on
+    // (536 -> 593 us at 256 rows per expert, 3612 -> 3384 us at 2048).  AFLEX_GEMM_GROUP_WIDE overrides both (tuning).
+    {
+        static int wide = -1;
+        if (wide < 0) { const char* e = getenv("AFLEX_GEMM_GROUP_WIDE"); wide = e ? atoi(e) : 0; }
+        const int from = wide > 0 ? wide : (mode == kGateUp ? kGroupedWideRowsGateUp : kGroupedWideRowsLinear);
+        if (E > 0 && p.n_tile > 128 && T / E < from) p.n_tile = 128;
+    }
     {
         static int cap = -1;
         if (cap < 0) { const char* e = getenv("AFLEX_GEMM_NTILE_CAP"); cap = e ? atoi(e) : 0; }

@@ -369,6 +369,23 @@ def test_moe_all_tokens_to_one_expert(ctx):
     assert row_rel_err(y, want_y) <= TOL_FFN
 
 
+def test_moe_skewed_load_at_prefill_size(ctx):
+    """Hundreds of rows per expert on average (the grouped GEMMs then take 256-row token tiles) with a strongly
+    skewed load: segments from a few rows to more than a thousand, ragged last chunks everywhere."""
+    T, H, I, E, K = 1300, 256, 384, 8, 2
+    x = rand_bf16((T, H), 1.0, 11)
+    wg, wu, wd = rand_bf16((E, I, H), 0.08, 12), rand_bf16((E, I, H), 0.08, 13), rand_bf16((E, H, I), 0.08, 14)
+    g = torch.Generator().manual_seed(15)
+    logits = torch.randn(T, E, generator=g) + torch.tensor([3.0, -2.5, 1.0, -1.0, 0.0, -3.0, 2.0, -0.5])
+    y, idx, gate, counts = run_moe(ctx, x, logits, wg, wu, wd, K)
+    want_y, want_idx, want_gate = O.ffn_moe(u16(x), logits.numpy(), u16(wg), u16(wu), u16(wd), K)
+    assert (idx == want_idx).all()
+    assert (counts == np.bincount(want_idx.ravel(), minlength=E)).all()
+    assert counts.max() > 1000 and counts.min() < 40
+    assert np.abs(gate - want_gate).max() <= TOL_GATE
+    assert row_rel_err(y, want_y) <= TOL_FFN
+
+
 def test_dense_ffn_large_token_count_uses_whole_tile_path(ctx):
     """T = 1100 at a small FFN: several 256-token tiles per weight tile (the compute-bound schedule)."""
     T, H, I = 1100, 256, 1024
