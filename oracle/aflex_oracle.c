@@ -552,3 +552,136 @@ ORACLE_API void oracle_attn_prefill(const uint16_t* q, const uint16_t* k_cache, 
         free(keys); free(vals); free(qd);
     }
 }
+
+/* ------------------------------------------------------------------------- */
+/* The same with the queries in double (the layer oracle does not round q).    */
+/* ------------------------------------------------------------------------- */
+ORACLE_API void oracle_attn_prefill_f64q(const double* q, const uint16_t* k_cache, const uint16_t* v_cache,
+                                         const int32_t* page_table, int max_pages, const int32_t* seq_lens,
+                                         const int32_t* q_offsets, int B, int Hq, int Hkv, int D, int P, double scale,
+                                         double* out) {
+    const int G = Hq / Hkv;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int b = 0; b < B; ++b) {
+        const int n = seq_lens[b];
+        const int m = q_offsets[b + 1] - q_offsets[b];
+        double* keys = (double*)malloc(sizeof(double) * (size_t)n * D);
+        double* vals = (double*)malloc(sizeof(double) * (size_t)n * D);
+        for (int g = 0; g < Hkv; ++g) {
+            for (int j = 0; j < n; ++j) {
+                const int64_t page = page_table[(size_t)b * max_pages + j / P];
+                const size_t base = (((size_t)page * Hkv + g) * P + (size_t)(j % P)) * (size_t)D;
+                for (int d = 0; d < D; ++d) {
+                    keys[(size_t)j * D + d] = bf16_to_f64(k_cache[base + d]);
+                    vals[(size_t)j * D + d] = bf16_to_f64(v_cache[base + d]);
+                }
+            }
+            for (int i = 0; i < m; ++i) {
+                const int visible = n - m + i + 1;          /* keys 0 .. pos_i */
+                const size_t row = (size_t)q_offsets[b] + i;
+                for (int hh = 0; hh < G; ++hh) {
+                    const int h = g * G + hh;
+                    oracle_attn_one_query_f64(q + (row * Hq + h) * D, keys, vals, visible, D, scale,
+                                              out + (row * Hq + h) * D, NULL);
+                }
+            }
+        }
+        free(keys); free(vals);
+    }
+}
+
+/* ------------------------------------------------------------------------- */
+/* The Attention group's work before the attention operator for the tokens    */
+/* being prefilled: row q_offsets[b] + i of x is token i of the last            */
+/* m = q_offsets[b+1] - q_offsets[b] tokens of sequence b and sits at position  */
+/* pos = seq_lens[b] - m + i.  Per row exactly what oracle_qkv_rope_append      */
+/* does for its one token: rmsnorm, QKV projection, head norms, rotary          */
+/* embedding at pos, K and V rounded to bf16 into the cache slot of pos.        */
+/* q_out f64 [T][Hq][D].                                                        */
+/* ------------------------------------------------------------------------- */
+ORACLE_API void oracle_qkv_rope_append_prefill(const double* x, const uint16_t* w_ln, const uint16_t* w_qkv,
+                                               const uint16_t* w_qn, const uint16_t* w_kn, double eps, double theta,
+                                               uint16_t* k_cache, uint16_t* v_cache,
+                                               const int32_t* page_table, int max_pages, const int32_t* seq_lens,
+                                               const int32_t* q_offsets, int B, int H, int Hq, int Hkv, int D, int P,
+                                               double* q_out) {
+    const int N = (Hq + 2 * Hkv) * D;
+    const int T = q_offsets[B];
+    double* xn = (double*)malloc(sizeof(double) * (size_t)T * H);
+    double* qkv = (double*)malloc(sizeof(double) * (size_t)T * N);
+    double* tmp = (double*)malloc(sizeof(double) * (size_t)D);
+    double* rot = (double*)malloc(sizeof(double) * (size_t)D);
+    oracle_rmsnorm(x, w_ln, T, H, eps, xn);
+    oracle_linear(xn, w_qkv, T, H, N, qkv);
+    for (int b = 0; b < B; ++b) {
+        const int m = q_offsets[b + 1] - q_offsets[b];
+        for (int i = 0; i < m; ++i) {
+            const size_t r = (size_t)q_offsets[b] + i;
+            const int pos = seq_lens[b] - m + i;
+            const int64_t page = page_table[(size_t)b * max_pages + pos / P];
+            for (int h = 0; h < Hq; ++h) {
+                const double* v = qkv + r * N + (size_t)h * D;
+                if (w_qn) { oracle_rmsnorm(v, w_qn, 1, D, eps, tmp); v = tmp; }
+                oracle_rope(v, D, (double)pos, theta, q_out + (r * Hq + h) * D);
+            }
+            for (int g = 0; g < Hkv; ++g) {
+                const size_t base = (((size_t)page * Hkv + g) * P + (size_t)(pos % P)) * (size_t)D;
+                const double* kk = qkv + r * N + (size_t)(Hq + g) * D;
+                const double* vv = qkv + r * N + (size_t)(Hq + Hkv + g) * D;
+                if (w_kn) { oracle_rmsnorm(kk, w_kn, 1, D, eps, tmp); kk = tmp; }
+                oracle_rope(kk, D, (double)pos, theta, rot);
+                for (int d = 0; d < D; ++d) {
+                    k_cache[base + d] = f64_to_bf16(rot[d]);
+                    v_cache[base + d] = f64_to_bf16(vv[d]);
+                }
+            }
+        }
+    }
+    free(xn); free(qkv); free(tmp); free(rot);
+}
+
+/* ------------------------------------------------------------------------- */
+/* One whole pre-norm decoder layer over the tokens being prefilled (the       */
+/* paper's PA and PF groups): the decode layer's arithmetic row by row, with    */
+/* causal attention over the cache that now also holds the rows' own K / V.     */
+/*   x, h1_out, out f64 [T][H], T = q_offsets[B]; logits f32 [T][E] when given. */
+/* ------------------------------------------------------------------------- */
+ORACLE_API void oracle_prefill_layer(const double* x, const uint16_t* w_ln_attn, const uint16_t* w_qkv,
+                                     const uint16_t* w_qn, const uint16_t* w_kn, double eps, double theta,
+                                     uint16_t* k_cache, uint16_t* v_cache,
+                                     const int32_t* page_table, int max_pages, const int32_t* seq_lens,
+                                     const int32_t* q_offsets, int B, int H, int Hq, int Hkv, int D, int P, double scale,
+                                     const uint16_t* w_o, const uint16_t* w_ln_ffn, int I, int E, int K,
+                                     const uint16_t* w_gate, const uint16_t* w_up, const uint16_t* w_down,
+                                     const uint16_t* w_router, const float* logits,
+                                     double* q_out, double* h1_out, double* out) {
+    const int A = Hq * D;
+    const int T = q_offsets[B];
+    double* q = q_out ? q_out : (double*)malloc(sizeof(double) * (size_t)T * A);
+    double* a = (double*)malloc(sizeof(double) * (size_t)T * A);
+    double* h1 = h1_out ? h1_out : (double*)malloc(sizeof(double) * (size_t)T * H);
+    double* xn = (double*)malloc(sizeof(double) * (size_t)T * H);
+    double* f = (double*)malloc(sizeof(double) * (size_t)T * H);
+    oracle_qkv_rope_append_prefill(x, w_ln_attn, w_qkv, w_qn, w_kn, eps, theta, k_cache, v_cache, page_table, max_pages,
+                                   seq_lens, q_offsets, B, H, Hq, Hkv, D, P, q);
+    oracle_attn_prefill_f64q(q, k_cache, v_cache, page_table, max_pages, seq_lens, q_offsets, B, Hq, Hkv, D, P, scale, a);
+    oracle_linear(a, w_o, T, A, H, h1);
+    for (size_t i = 0; i < (size_t)T * H; ++i) h1[i] += x[i];
+    oracle_rmsnorm(h1, w_ln_ffn, T, H, eps, xn);
+    if (E == 0) {
+        oracle_ffn_dense_f64x(xn, w_gate, w_up, w_down, T, H, I, f);
+    } else if (w_router) {
+        double* ld = (double*)malloc(sizeof(double) * (size_t)T * E);
+        float* lf = (float*)malloc(sizeof(float) * (size_t)T * E);
+        oracle_router_logits(xn, w_router, T, H, E, ld);
+        for (size_t i = 0; i < (size_t)T * E; ++i) lf[i] = (float)ld[i];   /* routing takes fp32 logits */
+        oracle_ffn_moe_f64x(xn, lf, w_gate, w_up, w_down, T, H, I, E, K, f, NULL, NULL);
+        free(ld); free(lf);
+    } else {
+        oracle_ffn_moe_f64x(xn, logits, w_gate, w_up, w_down, T, H, I, E, K, f, NULL, NULL);
+    }
+    for (size_t i = 0; i < (size_t)T * H; ++i) out[i] = h1[i] + f[i];
+    if (!q_out) free(q);
+    if (!h1_out) free(h1);
+    free(a); free(xn); free(f);
+}

@@ -357,6 +357,55 @@ def decoder_layer(x, w, k_cache, v_cache, page_table, seq_lens, num_q_heads: int
     return q, h1, out
 
 
+def prefill_layer(x, w, k_cache, v_cache, page_table, seq_lens, q_offsets, num_q_heads: int, eps: float, theta: float,
+                  top_k: int = 0, logits=None, scale: Optional[float] = None):
+    """One whole pre-norm decoder layer over the tokens being prefilled, in fp64.
+
+    x f64 [T,H] (T = q_offsets[-1]): row q_offsets[b] + i is token i of the last q_offsets[b+1] - q_offsets[b]
+    tokens of sequence b (seq_lens counts them already).  ``w`` as for decoder_layer; ``logits`` f32 [T,E].
+    The caches are updated IN PLACE.  Returns (q f64 [T,Hq,D], h1 f64 [T,H], out f64 [T,H])."""
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    T, H = x.shape
+    assert k_cache.dtype == np.uint16 and k_cache.flags["C_CONTIGUOUS"] and k_cache.flags["WRITEABLE"]
+    assert v_cache.dtype == np.uint16 and v_cache.flags["C_CONTIGUOUS"] and v_cache.flags["WRITEABLE"]
+    _, Hkv, P, D = k_cache.shape
+    Hq = int(num_q_heads)
+    page_table = np.ascontiguousarray(page_table, dtype=np.int32)
+    seq_lens = np.ascontiguousarray(seq_lens, dtype=np.int32)
+    q_offsets = np.ascontiguousarray(q_offsets, dtype=np.int32)
+    B = seq_lens.shape[0]
+    assert q_offsets.shape == (B + 1,) and q_offsets[0] == 0 and q_offsets[-1] == T
+    m = q_offsets[1:] - q_offsets[:-1]
+    assert (m >= 0).all() and (m <= seq_lens).all()
+    g = {k: (None if v is None else _u16(v)) for k, v in w.items()}
+    assert g["qkv"].shape == ((Hq + 2 * Hkv) * D, H) and g["o"].shape == (H, Hq * D)
+    if g["gate"].ndim == 3:
+        E, I, _ = g["gate"].shape
+        assert top_k >= 1
+        if g.get("router") is None:
+            logits = np.ascontiguousarray(logits, dtype=np.float32)
+            assert logits.shape == (T, E)
+    else:
+        E = 0
+        I = g["gate"].shape[0]
+    if scale is None:
+        scale = 1.0 / np.sqrt(float(D))
+    q = np.zeros((T, Hq, D), dtype=np.float64)
+    h1 = np.zeros((T, H), dtype=np.float64)
+    out = np.zeros((T, H), dtype=np.float64)
+    _load().oracle_prefill_layer(_p(x, _f64p), _p(g["ln_attn"], _u16p), _p(g["qkv"], _u16p),
+                                 _p(g.get("q_norm"), _u16p), _p(g.get("k_norm"), _u16p),
+                                 ctypes.c_double(eps), ctypes.c_double(theta),
+                                 _p(k_cache, _u16p), _p(v_cache, _u16p), _p(page_table, _i32p),
+                                 int(page_table.shape[1]), _p(seq_lens, _i32p), _p(q_offsets, _i32p), B, H, Hq, Hkv, D, P,
+                                 ctypes.c_double(scale), _p(g["o"], _u16p), _p(g["ln_ffn"], _u16p),
+                                 I, E, int(top_k), _p(g["gate"], _u16p), _p(g["up"], _u16p), _p(g["down"], _u16p),
+                                 _p(g.get("router"), _u16p) if E else None,
+                                 _p(logits, _f32p) if (E and g.get("router") is None) else None,
+                                 _p(q, _f64p), _p(h1, _f64p), _p(out, _f64p))
+    return q, h1, out
+
+
 def attn_prefill(q, k_cache, v_cache, page_table, seq_lens, q_offsets, scale: Optional[float] = None) -> np.ndarray:
     """Causal attention of the last q_len tokens of every sequence over its paged cache.
     q u16 [T,Hq,D] (T = q_offsets[-1]); seq_lens i32 [B] (cached tokens incl. the prefilled ones);

@@ -299,3 +299,58 @@ def test_prefill_is_causal_row_by_row():
     got2 = O.attn_prefill(q, k2, v2, table, lens, q_off)
     np.testing.assert_array_equal(got2[:19], got[:19])
     assert np.abs(got2[19] - got[19]).max() > 1e-3
+
+
+# --------------------------------------------------------------------------- prefill layer
+def _prompt_rows(q_off, b, i):
+    return int(q_off[b]) + i
+
+
+def test_prefill_layer_equals_the_decode_layer_fed_one_token_at_a_time():
+    """A layer's output for a prompt token depends on the earlier tokens only through the cache, so prefilling a
+    prompt must give, row by row, what the (separately pinned) decode layer gives when the same rows are fed one
+    position at a time.  Dense and mixture-of-experts FFN, two ragged prompts, one of them behind a cached prefix."""
+    for E in (0, 4):
+        rng = np.random.default_rng(21 + E)
+        Hq, eps, theta = 4, 1e-5, 1e4
+        lens = np.asarray([7, 21], dtype=np.int32)
+        new = np.asarray([7, 5], dtype=np.int32)            # sequence 1 already holds 16 cached tokens
+        _, w, k, v, table, _ = _tiny_layer(rng, lens=tuple(lens), E=E)
+        q_off = np.concatenate([[0], np.cumsum(new)]).astype(np.int32)
+        T = int(q_off[-1])
+        x = rng.standard_normal((T, 32))
+        kp, vp = k.copy(), v.copy()
+        q, h1, out = O.prefill_layer(x, w, kp, vp, table, lens, q_off, Hq, eps, theta, top_k=2 if E else 0)
+        kd, vd = k.copy(), v.copy()
+        for b in range(2):
+            for i in range(int(new[b])):
+                r = _prompt_rows(q_off, b, i)
+                cur = np.asarray([lens[b] - new[b] + i + 1], dtype=np.int32)
+                q1, h11, out1 = O.decoder_layer(x[r:r + 1], w, kd, vd, table[b:b + 1], cur, Hq, eps, theta,
+                                                top_k=2 if E else 0)
+                np.testing.assert_allclose(q[r], q1[0], rtol=0, atol=1e-13)
+                np.testing.assert_allclose(h1[r], h11[0], rtol=0, atol=1e-12)
+                np.testing.assert_allclose(out[r], out1[0], rtol=0, atol=1e-11)
+        assert (kp == kd).all() and (vp == vd).all()         # the same cache slots, bit for bit
+        assert (kp != k).any()
+
+
+def test_prefill_layer_in_two_chunks_equals_one_pass():
+    rng = np.random.default_rng(31)
+    Hq, eps, theta = 4, 1e-5, 1e6
+    lens = np.asarray([19, 6], dtype=np.int32)
+    _, w, k, v, table, _ = _tiny_layer(rng, lens=tuple(lens))
+    q_off = np.asarray([0, 19, 25], dtype=np.int32)
+    x = rng.standard_normal((25, 32))
+    k1, v1 = k.copy(), v.copy()
+    _, _, out = O.prefill_layer(x, w, k1, v1, table, lens, q_off, Hq, eps, theta)
+    # first 11 / 2 tokens, then the rest
+    first = np.asarray([11, 2], dtype=np.int32)
+    k2, v2 = k.copy(), v.copy()
+    rows_a = np.r_[0:11, 19:21]
+    rows_b = np.r_[11:19, 21:25]
+    _, _, out_a = O.prefill_layer(x[rows_a], w, k2, v2, table, first, np.asarray([0, 11, 13], dtype=np.int32), Hq, eps, theta)
+    _, _, out_b = O.prefill_layer(x[rows_b], w, k2, v2, table, lens, np.asarray([0, 8, 12], dtype=np.int32), Hq, eps, theta)
+    np.testing.assert_allclose(out[rows_a], out_a, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(out[rows_b], out_b, rtol=0, atol=1e-12)
+    assert (k1 == k2).all() and (v1 == v2).all()
