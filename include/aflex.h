@@ -358,6 +358,24 @@ AFLEX_API aflex_status aflex_decoder_layers(aflex_ctx* ctx, const aflex_decoder_
 /* Workspace bytes that suffice for aflex_decoder_layers on this layer shape.  Pure host computation. */
 AFLEX_API size_t aflex_decoder_workspace_bytes(const aflex_decoder_desc* layer, int max_batch);
 
+/*
+ * The same layers over the tokens being PREFILLED (the paper's PA and PF pools: Section 1, prefill runs the two
+ * operators on whole prompts, both dominated by matrix multiplications).  Row q_offsets[b] + i of x_in is token i of
+ * the last m = q_offsets[b+1] - q_offsets[b] tokens of sequence b; kvs[l].seq_lens[b] = n counts them already
+ * (m = n: a whole prompt; m < n: a chunk behind a cached prefix), the token sits at position n - m + i.  Per layer:
+ *   PA:  r = hidden states; qkv = rmsnorm(r) W_qkv^T; per row q / k head norms and rotary embedding at the row's
+ *        position; the row's K / V cache slot is WRITTEN; a = causal attention over the cache (aflex_attn_prefill);
+ *        h1 = r + a W_o^T
+ *   PF:  out = h1 + FFN(rmsnorm(h1))      dense SwiGLU or top-k MoE (router logits from w_router)
+ * x_in, x_out: bf16 [T][H], T = q_offsets_host[batch] (x_out may alias x_in); q_offsets: DEVICE i32 [batch + 1];
+ * q_offsets_host: HOST copy.  One stream, no microbatching (both groups are compute-bound here).  Workspace from
+ * aflex_prefill_workspace_bytes(layer, T).  Errors as aflex_decoder_layers and aflex_attn_prefill.
+ */
+AFLEX_API aflex_status aflex_prefill_layers(aflex_ctx* ctx, const aflex_decoder_desc* layers, const aflex_kv* kvs,
+                                            int num_layers, const void* x_in, int batch, const int32_t* q_offsets,
+                                            const int32_t* q_offsets_host, void* x_out, void* stream);
+AFLEX_API size_t aflex_prefill_workspace_bytes(const aflex_decoder_desc* layer, int max_tokens);
+
 /* ---- A/F pair: the Attention side on one GPU, the FFN side on another -----------------------
  *
  * The paper's data plane (Section 4.3, "Placement-aware A/F Data Path"; Section 5: within a node

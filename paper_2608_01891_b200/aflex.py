@@ -26,6 +26,7 @@ EXPORTS = (
     "aflex_kernel_name", "aflex_launch_count", "aflex_profile_enable", "aflex_profile_read",
     "aflex_trace_read", "aflex_attn_decode_static", "aflex_decoder_layers", "aflex_decoder_workspace_bytes",
     "aflex_add_rmsnorm", "aflex_rope_append", "aflex_attn_prefill", "aflex_af_decoder_layers", "aflex_af_workspace_bytes",
+    "aflex_prefill_layers", "aflex_prefill_workspace_bytes",
     "aflex_eq2_layer_time", "aflex_curve_eval",
     "aflex_pipeline_makespan", "aflex_plan_microbatches", "aflex_dvfs_window", "aflex_dvfs_decode_step",
     "aflex_dvfs_prefill_pair",
@@ -141,6 +142,10 @@ def load_library() -> ctypes.CDLL:
                                          ctypes.POINTER(ctypes.c_int32), vp, vp]
     lib.aflex_decoder_workspace_bytes.restype = cs
     lib.aflex_decoder_workspace_bytes.argtypes = [ctypes.POINTER(DecoderDesc), ci]
+    lib.aflex_prefill_layers.restype = ci
+    lib.aflex_prefill_layers.argtypes = [vp, ctypes.POINTER(DecoderDesc), ctypes.POINTER(KV), ci, vp, ci, vp, vp, vp, vp]
+    lib.aflex_prefill_workspace_bytes.restype = cs
+    lib.aflex_prefill_workspace_bytes.argtypes = [ctypes.POINTER(DecoderDesc), ci]
     lib.aflex_af_decoder_layers.restype = ci
     lib.aflex_af_decoder_layers.argtypes = [vp, vp, ctypes.POINTER(DecoderDesc), ctypes.POINTER(KV), ci, vp, ci, ci,
                                             ctypes.POINTER(ctypes.c_int32), vp, vp]
@@ -222,6 +227,10 @@ def decoder_desc(layer: LayerDesc, w_qkv, w_ln_attn, w_ln_ffn, w_q_norm, w_k_nor
 
 def decoder_workspace_bytes(layer: DecoderDesc, max_batch: int) -> int:
     return int(load_library().aflex_decoder_workspace_bytes(ctypes.byref(layer), max_batch))
+
+
+def prefill_workspace_bytes(layer: DecoderDesc, max_tokens: int) -> int:
+    return int(load_library().aflex_prefill_workspace_bytes(ctypes.byref(layer), max_tokens))
 
 
 def af_workspace_bytes(layer: DecoderDesc, max_batch: int, ffn_side: bool) -> int:
@@ -467,6 +476,19 @@ class Context:
         ka = (KV * len(kvs))(*kvs)
         self._check(self._lib.aflex_decoder_layers(self._h, la, ka, len(layers), _ptr(x_in), x_in.shape[0],
                                                    microbatch_depth, offs, _ptr(x_out), _stream(stream)))
+
+    def prefill_layers(self, layers: Sequence[DecoderDesc], kvs: Sequence[KV], x_in, q_offsets: torch.Tensor,
+                       q_offsets_host: torch.Tensor, x_out, stream=None) -> None:
+        """Runs len(layers) whole decoder layers over the tokens being prefilled: x_in bf16 [T,H] -> x_out, row
+        q_offsets[b] + i = token i of the last q_offsets[b+1] - q_offsets[b] tokens of sequence b (the caches'
+        seq_lens count them already; their K / V slots are written).  q_offsets i32 CUDA [B+1], q_offsets_host
+        the same on the CPU."""
+        assert len(layers) == len(kvs) and len(layers) >= 1
+        assert q_offsets.dtype == torch.int32 and q_offsets_host.dtype == torch.int32 and q_offsets_host.device.type == "cpu"
+        la = (DecoderDesc * len(layers))(*layers)
+        ka = (KV * len(kvs))(*kvs)
+        self._check(self._lib.aflex_prefill_layers(self._h, la, ka, len(layers), _ptr(x_in), q_offsets_host.shape[0] - 1,
+                                                   _ptr(q_offsets), _ptr(q_offsets_host), _ptr(x_out), _stream(stream)))
 
     def add_rmsnorm(self, res, add, w, eps: float, res_out=None, y=None, stream=None) -> None:
         self._check(self._lib.aflex_add_rmsnorm(self._h, _ptr(res), _ptr(add), _ptr(w), res.shape[0], res.shape[1],

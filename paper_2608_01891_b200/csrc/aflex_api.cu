@@ -822,6 +822,107 @@ aflex_status aflex_decoder_layers(aflex_ctx* ctx, const aflex_decoder_desc* laye
     return check_cuda(ctx, e, "decoder layers: exit join");
 }
 
+// ---- whole decoder layers over the tokens being prefilled -----------------------------------
+// Workspace: [linear scratch | resid | xn | qkv | q | a | o | xn2 | y | F scratch], rows = prompt tokens.
+namespace {
+struct PrefillWs {
+    size_t a_lin, rows_h, rows_qkv, rows_a, f_total, total;
+};
+PrefillWs prefill_ws(const aflex_decoder_desc* d, int T, int num_sms) {
+    const aflex_layer_desc* L = &d->layer;
+    const int D = L->attn.head_dim, A = L->attn.num_q_heads * D, H = L->hidden;
+    const int NQ = (L->attn.num_q_heads + 2 * L->attn.num_kv_heads) * D;
+    PrefillWs w;
+    const size_t b0 = linear_workspace_bytes(T, A, H, num_sms), b1 = linear_workspace_bytes(T, H, NQ, num_sms);
+    w.a_lin = b0 > b1 ? b0 : b1;
+    w.rows_h = align256((size_t)T * H * 2);
+    w.rows_qkv = align256((size_t)T * NQ * 2);
+    w.rows_a = align256((size_t)T * A * 2);
+    w.f_total = L->num_experts == 0 ? dense_ws_bytes(T, H, L->inter, num_sms)
+                                    : moe_ws_bytes(T, H, L->inter, L->num_experts, L->top_k, num_sms);
+    w.total = w.a_lin + 5 * w.rows_h + w.rows_qkv + 2 * w.rows_a + w.f_total + 1024;
+    return w;
+}
+}  // namespace
+
+size_t aflex_prefill_workspace_bytes(const aflex_decoder_desc* layer, int max_tokens) {
+    if (!layer || max_tokens < 1) return 0;
+    return prefill_ws(layer, max_tokens, 148).total;
+}
+
+aflex_status aflex_prefill_layers(aflex_ctx* ctx, const aflex_decoder_desc* layers, const aflex_kv* kvs, int num_layers,
+                                  const void* x_in, int batch, const int32_t* q_offsets, const int32_t* q_offsets_host,
+                                  void* x_out, void* stream) {
+    if (!ctx) return AFLEX_ERR_INVALID_ARG;
+    if (!q_offsets || !q_offsets_host) return set_error(ctx, AFLEX_ERR_INVALID_ARG, "prefill layers: null q_offsets");
+    if (batch < 1 || q_offsets_host[0] != 0)
+        return set_error(ctx, AFLEX_ERR_INVALID_ARG, "prefill layers: batch must be >= 1 and q_offsets_host start at 0");
+    for (int b = 0; b < batch; ++b)
+        if (q_offsets_host[b + 1] < q_offsets_host[b])
+            return set_error(ctx, AFLEX_ERR_INVALID_ARG, "prefill layers: q_offsets_host must not decrease");
+    const int T = q_offsets_host[batch];
+    if (T < 1) return set_error(ctx, AFLEX_ERR_INVALID_ARG, "prefill layers: no token to prefill");
+    aflex_status s = validate_decoder_args(ctx, layers, kvs, num_layers, x_in, batch, x_out);
+    if (s != AFLEX_OK) return s;
+    const int H = layers[0].layer.hidden;
+    size_t need = 0;
+    for (int l = 0; l < num_layers; ++l) {
+        if (kvs[l].seq_lens_host)
+            for (int b = 0; b < batch; ++b)
+                if (q_offsets_host[b + 1] - q_offsets_host[b] > kvs[l].seq_lens_host[b])
+                    return set_error(ctx, AFLEX_ERR_INVALID_ARG, "prefill layers: sequence %d has more new tokens than cached tokens", b);
+        const PrefillWs w = prefill_ws(&layers[l], T, ctx->num_sms);
+        if (w.total > need) need = w.total;
+    }
+    if (need > ctx->ws_bytes)
+        return set_error(ctx, AFLEX_ERR_WORKSPACE, "prefill layers: need %zu workspace bytes, have %zu", need, ctx->ws_bytes);
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    typedef __nv_bfloat16 bf;
+    for (int l = 0; l < num_layers; ++l) {
+        const aflex_decoder_desc* d = &layers[l];
+        const aflex_layer_desc* L = &d->layer;
+        const int Hq = L->attn.num_q_heads, Hkv = L->attn.num_kv_heads, D = L->attn.head_dim;
+        const int A = Hq * D, NQ = (Hq + 2 * Hkv) * D, I = L->inter, E = L->num_experts;
+        const PrefillWs w = prefill_ws(d, T, ctx->num_sms);
+        char* p = ctx->ws;
+        char* ws_lin = p; p += w.a_lin;
+        bf* resid = reinterpret_cast<bf*>(p); p += w.rows_h;
+        bf* xn = reinterpret_cast<bf*>(p); p += w.rows_h;
+        bf* qkv = reinterpret_cast<bf*>(p); p += w.rows_qkv;
+        bf* qb = reinterpret_cast<bf*>(p); p += w.rows_a;
+        bf* ab = reinterpret_cast<bf*>(p); p += w.rows_a;
+        bf* ob = reinterpret_cast<bf*>(p); p += w.rows_h;
+        bf* xn2 = reinterpret_cast<bf*>(p); p += w.rows_h;
+        bf* yb = reinterpret_cast<bf*>(p); p += w.rows_h;
+        char* ws_f = p;
+        // ---- PA
+        if (l == 0) s = add_rmsnorm_launch(ctx, x_in, nullptr, d->w_ln_attn, T, H, d->rms_eps, resid, xn, st);
+        else s = add_rmsnorm_launch(ctx, resid, yb, d->w_ln_attn, T, H, d->rms_eps, resid, xn, st);
+        if (s != AFLEX_OK) return s;
+        s = linear_launch(ctx, xn, d->w_qkv, T, H, NQ, qkv, ws_lin, w.a_lin, st, kKQkvGemm, ctx->counters_a);
+        if (s != AFLEX_OK) return s;
+        s = rope_append_launch(ctx, &L->attn, qkv, &kvs[l], batch, d->w_q_norm, d->w_k_norm, d->rms_eps, d->rope_theta, qb, st,
+                               q_offsets, T);
+        if (s != AFLEX_OK) return s;
+        s = attn_prefill_launch(ctx, &L->attn, qb, &kvs[l], batch, q_offsets, q_offsets_host, ab, st);
+        if (s != AFLEX_OK) return s;
+        s = linear_launch(ctx, ab, L->w_o, T, A, H, ob, ws_lin, w.a_lin, st, kKLinearGemm, ctx->counters_a);
+        if (s != AFLEX_OK) return s;
+        // ---- PF
+        s = add_rmsnorm_launch(ctx, resid, ob, d->w_ln_ffn, T, H, d->rms_eps, resid, xn2, st);
+        if (s != AFLEX_OK) return s;
+        if (E == 0) s = dense_run(ctx, xn2, L->w_gate, L->w_up, L->w_down, T, H, I, yb, ws_f, w.f_total, st);
+        else s = moe_run(ctx, xn2, nullptr, L->w_router, L->w_gate, L->w_up, L->w_down, T, H, I, E, L->top_k, yb, nullptr, nullptr,
+                         nullptr, ws_f, w.f_total, st);
+        if (s != AFLEX_OK) return s;
+        if (l == num_layers - 1) {
+            s = add_rmsnorm_launch(ctx, resid, yb, nullptr, T, H, 0.f, x_out, nullptr, st);
+            if (s != AFLEX_OK) return s;
+        }
+    }
+    return AFLEX_OK;
+}
+
 // ---- A/F pair: Attention side on ctx_a's device, FFN side on ctx_f's device ----------------
 // A-side workspace: [attn scratch | linear scratch | xn | qkv | q | a | o | h1 | back]
 // F-side workspace: [h1_f | xn2 | y | out_f | F scratch]

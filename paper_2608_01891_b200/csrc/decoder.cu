@@ -101,7 +101,10 @@ struct RopeParams {
     const __nv_bfloat16* w_kn;     // [D] or null
     const int32_t* page_table;     // [B][max_pages]
     const int32_t* seq_lens;       // [B]
-    __nv_bfloat16* q_out;          // [B][Hq][D]
+    const int32_t* q_offsets;      // null: one row per sequence, the token being decoded; else [B + 1]: row
+                                   // q_offsets[b] + i is token i of the last q_offsets[b+1] - q_offsets[b] of sequence b
+    int batch;
+    __nv_bfloat16* q_out;          // [rows][Hq][D]
     __nv_bfloat16* k_cache;        // [num_pages][Hkv][16][D]
     __nv_bfloat16* v_cache;
     long long num_pages;
@@ -122,24 +125,38 @@ __global__ void __launch_bounds__(kRopeWarps * 32) rope_append_kernel(const Rope
     pdl_wait();
     const int lane = threadIdx.x & 31;
     const int head = blockIdx.y * kRopeWarps + (threadIdx.x >> 5);
-    const int b = blockIdx.x;
+    const int row = blockIdx.x;
     const int heads = p.Hq + 2 * p.Hkv;
     if (head >= heads) return;
     const int D = p.D, half = D / 2;
+    int b = row, back = 0;                         // sequence of this row; tokens of the sequence that follow it
+    if (p.q_offsets != nullptr) {
+        int lo = 0, hi = p.batch;                  // largest b with q_offsets[b] <= row
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) / 2;
+            if (p.q_offsets[mid] <= row) lo = mid; else hi = mid;
+        }
+        b = lo;
+        back = p.q_offsets[b + 1] - 1 - row;
+        if (back < 0) {                            // offsets that do not cover this row
+            if (lane == 0) atomicExch(p.status, AFLEX_ERR_BOUNDS);
+            return;
+        }
+    }
     const int len = p.seq_lens[b];
-    if (len < 1 || len > p.max_pages * 16) {
+    if (len - back < 1 || len > p.max_pages * 16) {
         if (lane == 0) atomicExch(p.status, AFLEX_ERR_BOUNDS);
         return;                                    // no position to write to
     }
-    const int pos = len - 1;
-    const __nv_bfloat16* src = p.qkv + ((size_t)b * heads + head) * D;
+    const int pos = len - 1 - back;
+    const __nv_bfloat16* src = p.qkv + ((size_t)row * heads + head) * D;
     const bool is_q = head < p.Hq, is_k = !is_q && head < p.Hq + p.Hkv;
     const __nv_bfloat16* gain = is_q ? p.w_qn : (is_k ? p.w_kn : nullptr);
 
     // destination row
     __nv_bfloat16* dst;
     if (is_q) {
-        dst = p.q_out + ((size_t)b * p.Hq + head) * D;
+        dst = p.q_out + ((size_t)row * p.Hq + head) * D;
     } else {
         const int page = p.page_table[(size_t)b * p.max_pages + pos / 16];
         if (page < 0 || page >= p.num_pages) {
@@ -206,8 +223,11 @@ aflex_status add_rmsnorm_launch(aflex_ctx* ctx, const void* res, const void* add
 }
 
 aflex_status rope_append_launch(aflex_ctx* ctx, const aflex_attn_desc* d, const void* qkv, const aflex_kv* kv, int batch,
-                                const void* w_qn, const void* w_kn, float eps, float theta, void* q_out, cudaStream_t st) {
+                                const void* w_qn, const void* w_kn, float eps, float theta, void* q_out, cudaStream_t st,
+                                const int32_t* q_offsets, int rows) {
     RopeParams p;
+    p.q_offsets = q_offsets;
+    p.batch = batch;
     p.qkv = (const __nv_bfloat16*)qkv;
     p.w_qn = (const __nv_bfloat16*)w_qn;
     p.w_kn = (const __nv_bfloat16*)w_kn;
@@ -225,7 +245,7 @@ aflex_status rope_append_launch(aflex_ctx* ctx, const aflex_attn_desc* d, const 
     const int heads = p.Hq + 2 * p.Hkv;
     KernelScope scope(ctx, kKRopeAppend, st);
     return check_cuda(ctx,
-                      launch_pdl(rope_append_kernel, dim3(batch, (heads + kRopeWarps - 1) / kRopeWarps), dim3(kRopeWarps * 32),
+                      launch_pdl(rope_append_kernel, dim3(q_offsets ? rows : batch, (heads + kRopeWarps - 1) / kRopeWarps), dim3(kRopeWarps * 32),
                                  0, st, p),
                       "rope_append_kernel launch");
 }

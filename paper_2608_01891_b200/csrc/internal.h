@@ -176,6 +176,7 @@ aflex_status attn_prefill_launch(aflex_ctx* ctx, const aflex_attn_desc* d, const
 aflex_status add_rmsnorm_launch(aflex_ctx* ctx, const void* res, const void* add, const void* w, int T, int H, float eps,
                                 void* res_out, void* y, cudaStream_t st);
 aflex_status rope_append_launch(aflex_ctx* ctx, const aflex_attn_desc* d, const void* qkv, const aflex_kv* kv, int batch,
-                                const void* w_qn, const void* w_kn, float eps, float theta, void* q_out, cudaStream_t st);
+                                const void* w_qn, const void* w_kn, float eps, float theta, void* q_out, cudaStream_t st,
+                                const int32_t* q_offsets = nullptr, int rows = 0);
 
 }  // namespace aflex
