@@ -369,6 +369,82 @@ def run_moe_sweep(args, cfg, local_rank, device, peaks):
     ctx.close()
 
 
+def run_prefill_layers(args, cfg, local_rank, device, peaks):
+    """Whole decoder layers over prompts (aflex_prefill_layers: the paper's PA and PF operators chained): L layers,
+    each with its own weights and KV cache, over several prompt mixes.  One JSON line: time per layer, prompt
+    tokens/s, TFLOP/s of the layer's algorithmic flops against the measured bf16 peaks, per-kernel times."""
+    from paper_2608_01891_b200 import aflex as AF
+    L = args.prefill_layers
+    Hq, Hkv, D, H, I = cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim, cfg.hidden, cfg.inter
+    A, NQ = Hq * D, (Hq + 2 * Hkv) * D
+    attn = AF.attn_desc(Hq, Hkv, D)
+    weights = [IN.make_decoder_weights(cfg, l, device=device) for l in range(L)]
+    cases = [("whole prompts 8 x 1024", [1024] * 8, None), ("whole prompts 4 x 4096", [4096] * 4, None),
+             ("whole prompt 1 x 16384", [16384], None),
+             ("chunk of 2048 onto 8192 cached, 2 sequences", [10240] * 2, [2048] * 2)]
+    if args.prefill_case >= 0:
+        cases = cases[args.prefill_case:args.prefill_case + 1]
+    stream = torch.cuda.current_stream()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    rows, prof = [], {}
+    for name, cached, new in cases:
+        new = cached if new is None else new
+        B = len(cached)
+        c = dataclasses.replace(cfg, batch=B)
+        kvh = IN.make_paged_kv(c, np.asarray(cached, dtype=np.int32), device=device)
+        table, lens = kvh.page_table.to(device), kvh.seq_lens.to(device)
+        descs, kvs, keep = [], [], []
+        for l, w in enumerate(weights):
+            layer = AF.layer_desc(attn, H, I, w.o, w.gate, w.up, w.down, cfg.num_experts, cfg.top_k, w.router)
+            descs.append(AF.decoder_desc(layer, w.qkv, w.ln_attn, w.ln_ffn, w.q_norm, w.k_norm, cfg.rms_eps, cfg.rope_theta))
+            kc, vc = (kvh.k_cache, kvh.v_cache) if l == 0 else (kvh.k_cache.clone(), kvh.v_cache.clone())
+            kvs.append(AF.make_kv(kc, vc, table, lens, kvh.seq_lens))
+            keep.append((kc, vc))
+        qo = torch.zeros(B + 1, dtype=torch.int32)
+        qo[1:] = torch.cumsum(torch.tensor(new, dtype=torch.int32), 0)
+        qod = qo.to(device)
+        T = int(qo[-1])
+        x = IN.make_x(dataclasses.replace(cfg, num_experts=0), device=device, tokens=T)
+        y = torch.empty_like(x)
+        ctx = AF.Context(local_rank, max(AF.prefill_workspace_bytes(d, T) for d in descs))
+        run = lambda: ctx.prefill_layers(descs, kvs, x, qod, qo, y, stream)
+        for _ in range(max(3, args.warmup)):
+            run()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(args.steps):
+            run()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        us_layer = 1e3 * e0.elapsed_time(e1) / args.steps / L
+        pairs = sum(m * (n - m) + m * (m + 1) // 2 for n, m in zip(cached, new))
+        ffn_flops = 6.0 * T * H * I * (cfg.top_k if cfg.num_experts else 1)
+        flops = 2.0 * T * H * NQ + 2.0 * T * A * H + ffn_flops + 4.0 * Hq * D * pairs
+        tf = flops / us_layer / 1e6
+        rows.append({"case": name, "prompt_tokens": T, "us_per_layer": round(us_layer, 1),
+                     "tokens_per_s_per_layer": round(T / us_layer * 1e6), "tflops": round(tf, 1),
+                     "frac_bf16_burst": round(tf / peaks["bf16_tflops"], 4),
+                     "frac_bf16_sustained": round(tf / peaks["bf16_tflops_sustained"], 4)})
+        ctx.profile_enable(True)
+        for _ in range(3):
+            run()
+        pr = ctx.profile_read()
+        ctx.profile_enable(False)
+        prof[name] = {k: round(1e3 * v[0] / v[1], 1) for k, v in pr.items()}
+        assert ctx.device_status() == AF.OK
+        ctx.close()
+        del kvh, kvs, keep, x, y
+        torch.cuda.empty_cache()
+    line = {"metric": "whole decoder layer over prompts (prefill): tokens/s per layer", "unit": "tokens/s", "dtype": "bf16",
+            "data": "synthetic", "steps": args.steps, "warmup": max(3, args.warmup),
+            "config": {"workload": f"config {cfg.cfg_id}: {cfg.name}, {L} chained layers over prompt tokens",
+                       "l2": "per-layer weights and activations larger than L2, no flush"},
+            "peaks": peaks, "clocks": sampler.stop(), "cases": rows, "kernel_us_event_pairs": prof}
+    print(json.dumps(line), flush=True)
+
+
 def run_decoder_chain(args, cfg, local_rank, device, peaks):
     """Whole decoder layers chained (aflex_decoder_layers): L layers, each with its own weights and KV cache,
     at every microbatch depth of the configuration.  One JSON line: time per layer, tokens/s, the share of the
@@ -548,8 +624,11 @@ def main():
     ap.add_argument("--prefill", action="store_true",
                     help="instead of the layer step: prefill (causal) attention at the configuration's head shape over "
                          "several prompt mixes, TFLOP/s against the measured bf16 peaks")
+    ap.add_argument("--prefill-layers", type=int, default=0,
+                    help="instead of the layer step: this many whole decoder layers chained over prompt tokens "
+                         "(aflex_prefill_layers), several prompt mixes")
     ap.add_argument("--prefill-case", type=int, default=-1,
-                    help="with --prefill: run only this case of the list (a small single-kernel run for a profiler)")
+                    help="with --prefill / --prefill-layers: run only this case of the list (a small single-kernel run for a profiler)")
     ap.add_argument("--energy", action="store_true",
                     help="also read the NVML energy counter around a >= 2 s loop of the step (default clocks)")
     args = ap.parse_args()
@@ -596,6 +675,10 @@ def main():
     if args.prefill:
         if rank == 0:
             run_prefill(args, cfg, local_rank, device, peaks)
+        return
+    if args.prefill_layers > 0:
+        if rank == 0:
+            run_prefill_layers(args, cfg, local_rank, device, peaks)
         return
     wl = build_workload(cfg, device)
     lens_np = wl["kvh"].seq_lens.numpy()

@@ -109,14 +109,17 @@ struct RopeParams {
     __nv_bfloat16* v_cache;
     long long num_pages;
     int max_pages, Hq, Hkv, D;
+    int heads_per_warp;            // 1 for a decode batch (every head its own warp); more for prompt rows, so that a
+                                   // warp's position lookup and rotation serve several heads
     float eps;
-    double log2_theta;
+    double inv_freq[64];           // theta^(-2 i / D), i < D / 2 (D <= 128), formed in double on the host
     int* status;
 };
 
-// One warp per (sequence, head) of the concatenated q | k | v heads.  Lane handles the rotary pairs
-// (i, i + D/2), i = lane, lane + 32, ...  The angle pos * theta^(-2i/D) is formed and reduced in
-// double: at positions of 10^4 and more an fp32 angle would already be off by 10^-3 rad.
+// One warp per (row, head) of the concatenated q | k | v heads.  Lane handles the rotary pairs
+// (i, i + D/2), i = lane, lane + 32, ...  The angle pos * theta^(-2i/D) is formed and reduced to
+// [-pi, pi] in double (at positions of 10^4 and more an fp32 angle would already be off by 10^-3 rad; the
+// frequencies come from the host as doubles); only the sine and cosine of the remainder are fp32.
 constexpr int kRopeWarps = 4;
 __global__ void __launch_bounds__(kRopeWarps * 32) rope_append_kernel(const RopeParams p) {
     // No early release of the dependents here: the attention kernel streams the KV cache without waiting
@@ -124,10 +127,10 @@ __global__ void __launch_bounds__(kRopeWarps * 32) rope_append_kernel(const Rope
     // flushed) before anything later in the stream starts.
     pdl_wait();
     const int lane = threadIdx.x & 31;
-    const int head = blockIdx.y * kRopeWarps + (threadIdx.x >> 5);
+    const int head0 = (blockIdx.y * kRopeWarps + (threadIdx.x >> 5)) * p.heads_per_warp;
     const int row = blockIdx.x;
     const int heads = p.Hq + 2 * p.Hkv;
-    if (head >= heads) return;
+    if (head0 >= heads) return;
     const int D = p.D, half = D / 2;
     int b = row, back = 0;                         // sequence of this row; tokens of the sequence that follow it
     if (p.q_offsets != nullptr) {
@@ -149,64 +152,77 @@ __global__ void __launch_bounds__(kRopeWarps * 32) rope_append_kernel(const Rope
         return;                                    // no position to write to
     }
     const int pos = len - 1 - back;
-    const __nv_bfloat16* src = p.qkv + ((size_t)row * heads + head) * D;
-    const bool is_q = head < p.Hq, is_k = !is_q && head < p.Hq + p.Hkv;
-    const __nv_bfloat16* gain = is_q ? p.w_qn : (is_k ? p.w_kn : nullptr);
-
-    // destination row
-    __nv_bfloat16* dst;
-    if (is_q) {
-        dst = p.q_out + ((size_t)row * p.Hq + head) * D;
-    } else {
-        const int page = p.page_table[(size_t)b * p.max_pages + pos / 16];
-        if (page < 0 || page >= p.num_pages) {
-            if (lane == 0) atomicExch(p.status, AFLEX_ERR_BOUNDS);
-            return;
-        }
-        const int g = is_k ? head - p.Hq : head - p.Hq - p.Hkv;
-        dst = (is_k ? p.k_cache : p.v_cache) + (((size_t)page * p.Hkv + g) * 16 + (pos & 15)) * D;
-    }
-    if (!is_q && !is_k) {                          // values are stored as they are
-        for (int i = lane; i < D / 2; i += 32)
-            reinterpret_cast<uint32_t*>(dst)[i] = reinterpret_cast<const uint32_t*>(src)[i];
-        return;
-    }
-    float lo[2], hi[2];                            // D <= 128: at most two pairs per lane
-    float ss = 0.f;
+    const int page = p.page_table[(size_t)b * p.max_pages + pos / 16];
+    const bool page_ok = page >= 0 && page < p.num_pages;
+    // the row's rotation: the same for every head (D <= 128: at most two pairs per lane)
+    float cs[2], sn[2];
 #pragma unroll
     for (int k = 0; k < 2; ++k) {
         const int i = lane + 32 * k;
-        lo[k] = hi[k] = 0.f;
+        cs[k] = 1.f; sn[k] = 0.f;
         if (i < half) {
-            lo[k] = __bfloat162float(src[i]);
-            hi[k] = __bfloat162float(src[i + half]);
-            ss = fmaf(lo[k], lo[k], ss);
-            ss = fmaf(hi[k], hi[k], ss);
+            // angle and its reduction to [-pi, pi] in double (two-term 2 pi), sine and cosine of the remainder in fp32
+            const double ang = (double)pos * p.inv_freq[i];
+            const double turns = rint(ang * 0.15915494309189535);
+            const double red = fma(-turns, 2.4492935982947064e-16, fma(-turns, 6.283185307179586, ang));
+            sincosf((float)red, &sn[k], &cs[k]);
         }
     }
-    if (gain != nullptr) {
+    const int head_end = min(heads, head0 + p.heads_per_warp);
+    for (int head = head0; head < head_end; ++head) {
+        const __nv_bfloat16* src = p.qkv + ((size_t)row * heads + head) * D;
+        const bool is_q = head < p.Hq, is_k = !is_q && head < p.Hq + p.Hkv;
+        const __nv_bfloat16* gain = is_q ? p.w_qn : (is_k ? p.w_kn : nullptr);
+        // destination row
+        __nv_bfloat16* dst;
+        if (is_q) {
+            dst = p.q_out + ((size_t)row * p.Hq + head) * D;
+        } else {
+            if (!page_ok) {
+                if (lane == 0) atomicExch(p.status, AFLEX_ERR_BOUNDS);
+                continue;
+            }
+            const int g = is_k ? head - p.Hq : head - p.Hq - p.Hkv;
+            dst = (is_k ? p.k_cache : p.v_cache) + (((size_t)page * p.Hkv + g) * 16 + (pos & 15)) * D;
+        }
+        if (!is_q && !is_k) {                      // values are stored as they are
+            for (int i = lane; i < D / 2; i += 32)
+                reinterpret_cast<uint32_t*>(dst)[i] = reinterpret_cast<const uint32_t*>(src)[i];
+            continue;
+        }
+        float lo[2], hi[2];
+        float ss = 0.f;
 #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
-        const float rinv = rsqrtf(ss / (float)D + p.eps);
+        for (int k = 0; k < 2; ++k) {
+            const int i = lane + 32 * k;
+            lo[k] = hi[k] = 0.f;
+            if (i < half) {
+                lo[k] = __bfloat162float(src[i]);
+                hi[k] = __bfloat162float(src[i + half]);
+                ss = fmaf(lo[k], lo[k], ss);
+                ss = fmaf(hi[k], hi[k], ss);
+            }
+        }
+        if (gain != nullptr) {
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
+            const float rinv = rsqrtf(ss / (float)D + p.eps);
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {
+                const int i = lane + 32 * k;
+                if (i < half) {
+                    lo[k] = lo[k] * rinv * __bfloat162float(gain[i]);
+                    hi[k] = hi[k] * rinv * __bfloat162float(gain[i + half]);
+                }
+            }
+        }
 #pragma unroll
         for (int k = 0; k < 2; ++k) {
             const int i = lane + 32 * k;
             if (i < half) {
-                lo[k] = lo[k] * rinv * __bfloat162float(gain[i]);
-                hi[k] = hi[k] * rinv * __bfloat162float(gain[i + half]);
+                dst[i] = __float2bfloat16_rn(lo[k] * cs[k] - hi[k] * sn[k]);
+                dst[i + half] = __float2bfloat16_rn(hi[k] * cs[k] + lo[k] * sn[k]);
             }
-        }
-    }
-#pragma unroll
-    for (int k = 0; k < 2; ++k) {
-        const int i = lane + 32 * k;
-        if (i < half) {
-            const double ang = (double)pos * exp2(-2.0 * (double)i / (double)D * p.log2_theta);
-            double sn, cs;
-            sincos(ang, &sn, &cs);
-            const float c = (float)cs, s = (float)sn;
-            dst[i] = __float2bfloat16_rn(lo[k] * c - hi[k] * s);
-            dst[i + half] = __float2bfloat16_rn(hi[k] * c + lo[k] * s);
         }
     }
 }
@@ -240,12 +256,14 @@ aflex_status rope_append_launch(aflex_ctx* ctx, const aflex_attn_desc* d, const 
     p.max_pages = kv->max_pages_per_seq;
     p.Hq = d->num_q_heads; p.Hkv = d->num_kv_heads; p.D = d->head_dim;
     p.eps = eps;
-    p.log2_theta = log2((double)theta);
+    for (int i = 0; i < 64; ++i) p.inv_freq[i] = i < d->head_dim / 2 ? pow((double)theta, -2.0 * i / (double)d->head_dim) : 0.0;
     p.status = ctx->dev_status;
     const int heads = p.Hq + 2 * p.Hkv;
+    p.heads_per_warp = (q_offsets && rows >= 1024) ? 8 : 1;
+    const int warps = (heads + p.heads_per_warp - 1) / p.heads_per_warp;
     KernelScope scope(ctx, kKRopeAppend, st);
     return check_cuda(ctx,
-                      launch_pdl(rope_append_kernel, dim3(q_offsets ? rows : batch, (heads + kRopeWarps - 1) / kRopeWarps), dim3(kRopeWarps * 32),
+                      launch_pdl(rope_append_kernel, dim3(q_offsets ? rows : batch, (warps + kRopeWarps - 1) / kRopeWarps), dim3(kRopeWarps * 32),
                                  0, st, p),
                       "rope_append_kernel launch");
 }

@@ -63,6 +63,7 @@ CASES = [
     (IN.CONFIGS[1], 2, [40, 1, 129, 300], [40, 1, 129, 300]),          # whole prompts, ragged
     (IN.CONFIGS[1], 1, [500, 130, 77, 64], [100, 130, 1, 0]),           # chunks behind prefixes, a decode row, nothing
     (TINY_D128, 2, [257, 16, 33, 5, 700], [257, 16, 20, 5, 188]),
+    (IN.CONFIGS[1], 1, [1100, 30, 5, 200], [1100, 30, 5, 200]),        # more than 1024 rows: several heads per warp in the append kernel
     (TINY_MOE, 1, [90, 17, 128, 3, 260, 31], [90, 17, 100, 3, 200, 31]),
 ]
 
