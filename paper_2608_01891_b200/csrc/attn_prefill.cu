@@ -431,12 +431,11 @@ static aflex_status launch_t(aflex_ctx* ctx, const aflex_attn_desc* d, const voi
         return set_error(ctx, AFLEX_ERR_CUDA, "prefill attention: cuTensorMapEncodeTiled failed");
     const size_t smem = (size_t)kQT * (D / 64) * kBM * 128 + (size_t)slots_for(D) * (D / 64) * kBN * 128 +
                         sizeof(Shared) + 1024;
-    static bool attr_set[2] = {false, false};
     const int ti = (D == 128) ? 1 : 0;
-    if (!attr_set[ti]) {
+    if (!ctx->prefill_attr_set[ti]) {
         cudaError_t e = cudaFuncSetAttribute(attn_prefill_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return check_cuda(ctx, e, "cudaFuncSetAttribute(prefill attention)");
-        attr_set[ti] = true;
+        ctx->prefill_attr_set[ti] = true;
     }
     KernelScope scope(ctx, kKAttnPrefill, st);
     return check_cuda(ctx,

@@ -53,6 +53,7 @@ struct aflex_ctx {
     bool attn_q_final_once = false;   // set by the layer chains for their own attention launch (q comes from the append kernel)
     bool gemm_attr_set[3] = {false, false, false};
     bool attn_attr_set[2] = {false, false};
+    bool prefill_attr_set[2] = {false, false};   // shared-memory limit raised for attn_prefill_kernel<64 / 128> on this device
     char err[512] = {0};
     // launch counters (always on) and event-pair timing of every launch (when profiling is enabled)
     long long launches[aflex::kKKindCount] = {};
