@@ -150,3 +150,37 @@ def test_prefill_layers_argument_checks():
         assert ctx.device_status() == AF.OK
     finally:
         ctx.close()
+
+
+def test_prefill_layers_replay_from_a_cuda_graph():
+    """The prefill chain only enqueues work on the caller's stream (tensor maps are kernel parameters, no
+    synchronisation, no allocation): captured into a CUDA graph after a warm-up call and replayed, it gives the
+    bits of the eager call."""
+    cfg = IN.CONFIGS[1]
+    lens = np.asarray([70, 33, 129, 16], dtype=np.int32)
+    ch = Chain(cfg, 2, seq_lens=lens)
+    q_off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    T = int(q_off[-1])
+    x = prompt_hidden(T, cfg.hidden, 5).to(DEV)
+    qo = torch.from_numpy(q_off)
+    qod = qo.to(DEV)
+    out = torch.zeros(T, cfg.hidden, dtype=torch.bfloat16, device=DEV)
+    ctx = AF.Context(0, max(AF.prefill_workspace_bytes(d, T) for d in ch.descs))
+    try:
+        s = torch.cuda.Stream()
+        with torch.cuda.stream(s):
+            ch.reset_caches()
+            ctx.prefill_layers(ch.descs, ch.kvs, x, qod, qo, out, s)        # warm-up: sets kernel attributes
+            s.synchronize()
+            want = out.clone()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=s):
+                ctx.prefill_layers(ch.descs, ch.kvs, x, qod, qo, out, s)
+            for _ in range(2):
+                out.zero_()
+                g.replay()
+                s.synchronize()
+                assert torch.equal(out.view(torch.int16), want.view(torch.int16))
+        assert ctx.device_status() == AF.OK
+    finally:
+        ctx.close()
