@@ -376,10 +376,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
         WorkUnit wu;
         pdl_wait();   // nothing is written before the predecessor grid has completed
 
-        // A shared tile is finished by ALL its contributors together: once every piece is published
-        // (arrival counter == number of pieces; bounded spin), contributor i sums the i-th slice of the
-        // tile over all pieces, in CTA order, and writes that slice of the output.  A second counter
-        // tells the last finisher to reset both counters.  Contributors of a tile run concurrently (the
+        // A shared tile is finished by its contributors together (all of them but a last one that has another
+        // shared tile to finish): once every piece is published (arrival counter == number of pieces; bounded
+        // spin), reducer i sums the i-th slice of the tile over all pieces, in CTA order, and writes that slice
+        // of the output.  A second counter tells the last finisher to reset both counters.  Contributors of a tile run concurrently (the
         // grid never exceeds the SM count and shared tiles are everyone's first units), so the spin is short.
         struct PendingTile { int tile; TileCoord c; };
         PendingTile pend[2];
@@ -389,6 +389,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
             const int cf = sched.cta_of(x0);
             const int cl = sched.cta_of(x0 + p.kblocks - 1);
             const int np = cl - cf + 1, me = (int)blockIdx.x - cf;
+            // A last contributor whose share runs on into the next tile has a second shared tile to finish (as that
+            // tile's first contributor): it is excused here, so that no CTA does two reductions one after the other
+            // at the very end, where everybody else waits for the kernel's last CTA.
+            const int nred = (np > 1 && sched.share_begin(cl + 1) > x0 + p.kblocks) ? np - 1 : np;
+            if (me >= nred) return;
             if (etid == 0) {
                 const long long t_start = clock64();
                 int seen;
@@ -404,7 +409,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
             __threadfence();
             const bool cf_early = sched.share_begin(cf) < x0;
             const int n4 = ((pd.c.b_rows + 15) / 16) * 4 * kBlockM;     // float4 slots of one accumulator that were stored
-            const int lo = (int)((long long)n4 * me / np), hi = (int)((long long)n4 * (me + 1) / np);
+            const int lo = (int)((long long)n4 * me / nred), hi = (int)((long long)n4 * (me + 1) / nred);
             const int up_off = (p.n_tile >> 2) * kBlockM;               // float4 offset of the "up" accumulator
             // kElems float4 per thread and round, all pieces' loads of a round in flight together (the loop is
             // bound by L2 latency, not bandwidth)
@@ -470,7 +475,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
             asm volatile("bar.sync 2, 128;" ::: "memory");
             if (etid == 0) {
                 const int done = atomicAdd(&p.counters[kStreamKMaxTiles + pd.tile], 1);
-                if (done == np - 1) {   // every contributor has read what it needs: clean up for the next launch
+                if (done == nred - 1) {   // every reducer has read what it needs: clean up for the next launch
                     p.counters[pd.tile] = 0;
                     p.counters[kStreamKMaxTiles + pd.tile] = 0;
                 }
