@@ -157,3 +157,56 @@ def test_prefill_full_size_sampled_rows(ctx):
     want, _ = O.attn_decode(u16(q_s), u16(kvh.k_cache.cpu()), u16(kvh.v_cache.cpu()),
                             np.stack([table[b] for b, _ in rows]), np.asarray([r + 1 for _, r in rows], dtype=np.int32))
     assert row_rel_err(f64(got), want) <= TOL_ATTN
+
+
+def test_prefill_lengths_on_tile_and_step_boundaries(ctx):
+    """Prompt lengths that end exactly on the kernel's natural boundaries (16-token pages, 128-token steps, 128-row
+    query tiles, 256-row blocks) and one token beyond them; a non-default softmax scale."""
+    lens = [128, 129, 256, 257, 512, 16, 127, 384]
+    Hq, Hkv, D = 8, 2, 128
+    cfg = IN.LayerConfig(43, "prefill-bounds", len(lens), Hq, Hkv, D, 64, 64)
+    l = np.asarray(lens, dtype=np.int32)
+    kvh = IN.make_paged_kv(cfg, l, poison=True)
+    q_off = np.concatenate([[0], np.cumsum(l)]).astype(np.int32)
+    T = int(q_off[-1])
+    g = torch.Generator().manual_seed(43)
+    q = torch.randn(T, Hq, D, generator=g).to(torch.bfloat16)
+    kv = AF.make_kv(kvh.k_cache.to(DEV), kvh.v_cache.to(DEV), kvh.page_table.to(DEV), kvh.seq_lens.to(DEV), kvh.seq_lens)
+    out = torch.full((T, Hq, D), float("nan"), dtype=torch.bfloat16, device=DEV)
+    qo = torch.from_numpy(q_off)
+    desc = AF.attn_desc(Hq, Hkv, D, sm_scale=0.05)
+    ctx.attn_prefill(desc, q.to(DEV), kv, qo.to(DEV), qo, out)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == AF.OK
+    want = O.attn_prefill(u16(q), u16(kvh.k_cache), u16(kvh.v_cache), kvh.page_table.numpy(), l, q_off, scale=0.05)
+    assert row_rel_err(f64(out), want) <= TOL_ATTN
+
+
+def test_prefill_with_equal_keys_is_the_running_mean_of_the_values(ctx):
+    """Closed form, no oracle: when every cached key of a sequence is the same vector, every query weighs the tokens
+    it may see equally, so row i of the output is the mean of V over positions 0 .. pos_i."""
+    Hq, Hkv, D = 4, 2, 64
+    lens = np.asarray([300, 45], dtype=np.int32)
+    new = np.asarray([300, 20], dtype=np.int32)
+    cfg = IN.LayerConfig(44, "prefill-mean", len(lens), Hq, Hkv, D, 64, 64)
+    kvh = IN.make_paged_kv(cfg, lens)
+    kvh.k_cache[:] = torch.randn(D, generator=torch.Generator().manual_seed(44)).to(torch.bfloat16)
+    q_off = np.concatenate([[0], np.cumsum(new)]).astype(np.int32)
+    T = int(q_off[-1])
+    q = torch.randn(T, Hq, D, generator=torch.Generator().manual_seed(45)).to(torch.bfloat16)
+    kv = AF.make_kv(kvh.k_cache.to(DEV), kvh.v_cache.to(DEV), kvh.page_table.to(DEV), kvh.seq_lens.to(DEV), kvh.seq_lens)
+    out = torch.full((T, Hq, D), float("nan"), dtype=torch.bfloat16, device=DEV)
+    qo = torch.from_numpy(q_off)
+    ctx.attn_prefill(AF.attn_desc(Hq, Hkv, D), q.to(DEV), kv, qo.to(DEV), qo, out)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == AF.OK
+    table = kvh.page_table.numpy()
+    v = kvh.v_cache.to(torch.float64).numpy()
+    want = np.zeros((T, Hq, D))
+    for b in range(2):
+        vs = np.stack([v[table[b, j // 16], :, j % 16, :] for j in range(int(lens[b]))])      # [n, Hkv, D]
+        run = np.cumsum(vs, axis=0) / np.arange(1, int(lens[b]) + 1)[:, None, None]
+        for i in range(int(new[b])):
+            pos = int(lens[b] - new[b]) + i
+            want[q_off[b] + i] = np.repeat(run[pos], Hq // Hkv, axis=0)
+    assert row_rel_err(f64(out), want) <= TOL_ATTN
