@@ -72,19 +72,10 @@ __device__ __forceinline__ void tmem_st_32x32b_x16(uint32_t taddr, const uint32_
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-// Shared-memory descriptor of an MN-major bf16 operand stored as [K rows][64 MN elements] blocks of 128-byte
-// swizzled rows: 8-row groups 1024 B apart (stride byte offset), 64-element MN blocks `mn_block_bytes` apart
-// (leading byte offset).
-__device__ __forceinline__ uint64_t umma_desc_mn_sw128(uint32_t smem_addr, uint32_t mn_block_bytes) {
-    uint64_t d = 0;
-    d |= (uint64_t)((smem_addr & 0x3FFFF) >> 4);
-    d |= (uint64_t)((mn_block_bytes >> 4) & 0x3FFF) << 16;
-    d |= (uint64_t)(1024 >> 4) << 32;
-    d |= (uint64_t)1 << 46;
-    d |= (uint64_t)2 << 61;
-    return d;
-}
-
+// Shared-memory operand descriptors, all with the 128-byte swizzle TMA writes (8-row groups 1024 B apart: the
+// stride byte offset).  K-major operands (Q, K: rows of 64 contiguous K elements) leave the leading byte offset at
+// its unused value 16; the MN-major operand (V as the cache stores it, [token = K row][64 D columns] blocks) puts the
+// distance between its 64-column blocks there and advances by 2048 B per 16 token rows.
 // The MMA issuer keeps descriptors as a low word (start address in 16-byte units, leading byte offset at bit 16) that
 // it advances by adding byte offsets >> 4, and one upper word shared by every operand here (8-row groups 1024 B apart,
 // descriptor version 1, 128-byte swizzle).
