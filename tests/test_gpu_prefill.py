@@ -210,3 +210,39 @@ def test_prefill_with_equal_keys_is_the_running_mean_of_the_values(ctx):
             pos = int(lens[b] - new[b]) + i
             want[q_off[b] + i] = np.repeat(run[pos], Hq // Hkv, axis=0)
     assert row_rel_err(f64(out), want) <= TOL_ATTN
+
+
+def test_prefill_random_shapes(ctx):
+    """Seeded sweep over head shapes (D 64 / 128, 1 - 4 KV heads, group sizes 1 - 8), batch sizes, ragged cached
+    lengths and query counts (whole prompts, arbitrary chunks, short tails, sequences without a query), with and
+    without the host copy of the lengths."""
+    rng = np.random.default_rng(7)
+    worst = 0.0
+    for case in range(24):
+        D, Hkv, G = int(rng.choice([64, 128])), int(rng.choice([1, 2, 4])), int(rng.choice([1, 2, 4, 8]))
+        B = int(rng.integers(1, 6))
+        lens = rng.integers(1, 700, size=B).astype(np.int32)
+        mode = int(rng.integers(0, 3))
+        if mode == 0:
+            new = lens.copy()
+        elif mode == 1:
+            new = np.array([int(rng.integers(0, n + 1)) for n in lens], dtype=np.int32)
+        else:
+            new = np.minimum(lens, rng.integers(1, 40, size=B)).astype(np.int32)
+        if new.sum() == 0:
+            new[0] = 1
+        cfg = IN.LayerConfig(100 + case, "prefill-sweep", B, Hkv * G, Hkv, D, 64, 64)
+        kvh = IN.make_paged_kv(cfg, lens, poison=True)
+        q_off = np.concatenate([[0], np.cumsum(new)]).astype(np.int32)
+        T = int(q_off[-1])
+        q = torch.randn(T, Hkv * G, D, generator=torch.Generator().manual_seed(case)).to(torch.bfloat16)
+        kv = AF.make_kv(kvh.k_cache.to(DEV), kvh.v_cache.to(DEV), kvh.page_table.to(DEV), kvh.seq_lens.to(DEV),
+                        kvh.seq_lens if case % 2 else None)
+        out = torch.full((T, Hkv * G, D), float("nan"), dtype=torch.bfloat16, device=DEV)
+        qo = torch.from_numpy(q_off)
+        ctx.attn_prefill(AF.attn_desc(Hkv * G, Hkv, D), q.to(DEV), kv, qo.to(DEV), qo, out)
+        torch.cuda.synchronize()
+        assert ctx.device_status() == AF.OK, case
+        want = O.attn_prefill(u16(q), u16(kvh.k_cache), u16(kvh.v_cache), kvh.page_table.numpy(), lens, q_off)
+        worst = max(worst, row_rel_err(f64(out), want))
+    assert worst <= TOL_ATTN
