@@ -467,3 +467,47 @@ def test_layer_step_replays_from_a_cuda_graph(ctx, M):
             s.synchronize()
             assert torch.equal(y.view(torch.int16), want.view(torch.int16))
     assert ctx.device_status() == AF.OK
+
+
+def test_seeded_sweep_over_shapes(ctx):
+    """Decode attention, dense FFN and MoE FFN over seeded random shapes: head sizes and group sizes, ragged
+    batches up to 3000 cached tokens, token counts from 1 to several hundred, feature sizes that are odd multiples
+    of 8, 2 - 16 experts with top-1 / top-2."""
+    rng = np.random.default_rng(11)
+    worst = {"attn": 0.0, "ffn": 0.0, "moe": 0.0}
+    for case in range(16):
+        # ---- attention
+        D, Hkv, G = int(rng.choice([64, 128])), int(rng.choice([1, 2, 4, 8])), int(rng.choice([1, 2, 4, 8]))
+        B = int(rng.integers(1, 40))
+        lens = rng.integers(1, int(rng.choice([40, 400, 3000])), size=B).astype(np.int32)
+        cfg = IN.LayerConfig(200 + case, "sweep", B, Hkv * G, Hkv, D, 64, 64)
+        kvh = IN.make_paged_kv(cfg, lens, poison=True)
+        q = rand_bf16((B, Hkv * G, D), 1.0, 3 * case)
+        kv = AF.make_kv(kvh.k_cache.to(DEV), kvh.v_cache.to(DEV), kvh.page_table.to(DEV), kvh.seq_lens.to(DEV),
+                        kvh.seq_lens if case % 2 else None)
+        out = torch.full((B, Hkv * G, D), float("nan"), dtype=torch.bfloat16, device=DEV)
+        ctx.attn_decode(AF.attn_desc(Hkv * G, Hkv, D), q.to(DEV), kv, out)
+        torch.cuda.synchronize()
+        want, _ = O.attn_decode(u16(q), u16(kvh.k_cache), u16(kvh.v_cache), kvh.page_table.numpy(), lens)
+        worst["attn"] = max(worst["attn"], row_rel_err(f64(out), want))
+        # ---- dense FFN
+        T = int(rng.integers(1, int(rng.choice([40, 300, 900]))))
+        H, I = 8 * int(rng.integers(4, 80)), 8 * int(rng.integers(4, 120))
+        x = rand_bf16((T, H), 1.0, 3 * case + 1)
+        wg, wu, wd = rand_bf16((I, H), 0.08, 5), rand_bf16((I, H), 0.08, 6), rand_bf16((H, I), 0.08, 7)
+        y = torch.full((T, H), float("nan"), dtype=torch.bfloat16, device=DEV)
+        ctx.ffn_dense(x.to(DEV), wg.to(DEV), wu.to(DEV), wd.to(DEV), y)
+        torch.cuda.synchronize()
+        worst["ffn"] = max(worst["ffn"], row_rel_err(f64(y), O.ffn_dense(u16(x), u16(wg), u16(wu), u16(wd))))
+        # ---- MoE FFN
+        E, K, T = int(rng.choice([2, 4, 8, 16])), int(rng.choice([1, 2])), int(rng.integers(1, 400))
+        H, I = 8 * int(rng.integers(4, 40)), 8 * int(rng.integers(4, 60))
+        x = rand_bf16((T, H), 1.0, 3 * case + 2)
+        wg, wu, wd = rand_bf16((E, I, H), 0.08, 8), rand_bf16((E, I, H), 0.08, 9), rand_bf16((E, H, I), 0.08, 10)
+        logits = torch.randn(T, E, generator=torch.Generator().manual_seed(case))
+        ym, idx, _, _ = run_moe(ctx, x, logits, wg, wu, wd, K)
+        want_y, want_idx, _ = O.ffn_moe(u16(x), logits.numpy(), u16(wg), u16(wu), u16(wd), K)
+        assert (idx == want_idx).all(), case
+        worst["moe"] = max(worst["moe"], row_rel_err(ym, want_y))
+        assert ctx.device_status() == AF.OK, case
+    assert worst["attn"] <= TOL_ATTN and worst["ffn"] <= TOL_FFN and worst["moe"] <= TOL_FFN, worst
