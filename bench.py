@@ -757,6 +757,39 @@ def main():
         if key in tr:
             roofline["traffic"] = tr[key]
 
+    # ---- the two operators on their own (back-to-back calls of the public entry points; with programmatic dependent
+    #      launch a call's ramp overlaps its predecessor's tail, so these are the streaming rates the step is built from)
+    operators = {}
+    if rank == 0:
+        a_out = torch.empty_like(wl["q"])
+        x_ffn = IN.make_x(cfg, device=device)
+        y_ffn = torch.empty_like(x_ffn)
+
+        def attn_alone():
+            ctx.attn_decode(wl["layer"].attn, wl["q"], wl["kv"], a_out, None, stream)
+
+        def ffn_alone():
+            if cfg.num_experts == 0:
+                ctx.ffn_dense(x_ffn, wl["wg"], wl["wu"], wl["wd"], y_ffn, stream)
+            else:
+                ctx.ffn_moe(x_ffn, wl["wg"], wl["wu"], wl["wd"], cfg.top_k, y_ffn, router_logits=wl["logits"], stream=stream)
+
+        for name, fn in (("attn_decode", attn_alone), ("ffn", ffn_alone)):
+            for _ in range(3):
+                fn()
+            us = 1e3 * timed(fn, args.steps) / args.steps
+            if name == "attn_decode":
+                byts = abytes["attn_decode"] * M
+                operators[name] = {"us": round(us, 2), "gbs": round(byts / us / 1e3, 1),
+                                   "frac_hbm_measured": round(byts / us / 1e3 / peaks["hbm_gbs"], 4),
+                                   "frac_hbm_nominal_8tbs": round(byts / us / 1e3 / 8000.0, 4)}
+            else:
+                g, d = ("gateup_gemm", "down_gemm") if cfg.num_experts == 0 else ("moe_gateup_gemm", "moe_down_gemm")
+                byts, fl = (abytes[g] + abytes[d]) * M, (aflops[g] + aflops[d]) * M
+                operators[name] = {"us": round(us, 2), "weight_stream_gbs": round(byts / us / 1e3, 1),
+                                   "frac_hbm_measured": round(byts / us / 1e3 / peaks["hbm_gbs"], 4),
+                                   "tflops": round(fl / us / 1e6, 1), "frac_bf16_burst": round(fl / us / 1e6 / peaks["bf16_tflops"], 4)}
+
     # ---- end to end: per-step inputs come from pinned host memory, the result goes back.
     # The per-step inputs (q, page table, sequence lengths, router logits) are packed into one pinned
     # staging buffer and travel in ONE host-to-device copy into one device buffer the tensors are views of.
@@ -829,7 +862,7 @@ def main():
                            "context_tokens": int(lens_np.sum()), "page_size": 16,
                            "l2": "inputs larger than L2 (KV + weights >> 126 MB), no flush",
                            "parallelism": "replicas only" if world > 1 else "1 GPU"},
-                "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "kernels": kernels,
+                "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "kernels": kernels, "operators_alone": operators,
                 "cpu_baseline": cpu}
         if energy is not None:
             line["energy"] = energy
