@@ -50,6 +50,19 @@ def test_makespan_matches_the_longest_path_oracle():
         assert AF.pipeline_makespan(lm, lens, offs, L) == pytest.approx(C.pipeline_makespan(om, lens, offs, L), rel=1e-12)
 
 
+def test_library_clamps_the_stage_time_as_a_whole():
+    # the hand-computed cases that pin the oracle's reading (a stage's time, i.e. the SUM of the token term and the
+    # row term, is clamped at zero; the curves themselves are not), here against the library
+    tokens = ([100.0, 200.0], [10.0, 30.0])                    # 20 tokens -> -6
+    const = lambda v: ([0.0], [v])
+    m = AF.pipeline_model(tokens, const(4.0), const(3.0), 0.0, 0.0, True)
+    assert AF.pipeline_makespan(m, [20], [0, 1], 1) == pytest.approx(3.0)            # t_A = max(0, -6 + 4) = 0
+    m = AF.pipeline_model(tokens, const(10.0), const(3.0), 0.0, 0.0, True)
+    assert AF.pipeline_makespan(m, [20], [0, 1], 2) == pytest.approx(14.0)           # t_A = -6 + 10 = 4, not 0 + 10
+    m = AF.pipeline_model(tokens, const(10.0), ([10.0, 20.0], [5.0, 25.0]), 0.0, 0.0, True)
+    assert AF.pipeline_makespan(m, [20], [0, 1], 1) == pytest.approx(4.0)            # t_F(1 row) = max(0, -13) = 0
+
+
 def test_makespan_rejects_bad_arguments():
     _, lm = random_model(np.random.default_rng(2))
     assert math.isnan(AF.pipeline_makespan(lm, [5, 5], [0, 1], 1))          # offsets do not end at the batch

@@ -75,6 +75,31 @@ def test_stage_times_follow_the_curves():
     assert C.pipeline_makespan(m, [10, 30, 60], [0, 2, 3], 1) == pytest.approx(6.0 + 4.0 + 7.5 + 3.0)
 
 
+def test_stage_time_is_clamped_at_zero_as_a_whole_not_curve_by_curve():
+    # Reading (the paper's "profiled Attention/FFN latency curves" says nothing about extrapolation): a stage's
+    # duration is the physical quantity and cannot be negative, while the two terms of t_A are only a fit whose
+    # parts may have either sign (a negative token-term offset by a positive row-term is a legitimate fit).  So the
+    # SUM is clamped, not each curve.  Numbers by hand: the token curve through (100, 10), (200, 30) has slope 0.2,
+    # so 20 tokens give 10 - 80 * 0.2 = -6.
+    tokens = ([100.0, 200.0], [10.0, 30.0])
+    assert C.curve_eval(*tokens, 20.0) == pytest.approx(-6.0)
+    # (a) row term +4: -6 + 4 = -2 -> the stage takes 0 (unclamped: -2; clamped curve by curve: 0 + 4 = 4)
+    m = C.Model(tokens, CONST(4.0), CONST(3.0), shared=True)
+    assert m.t_a([20]) == 0.0
+    assert C.pipeline_makespan(m, [20], [0, 1], 1) == pytest.approx(0.0 + 3.0)
+    # (b) row term +10: -6 + 10 = 4 stays 4 (clamped curve by curve: 0 + 10 = 10)
+    m = C.Model(tokens, CONST(10.0), CONST(3.0), shared=True)
+    assert m.t_a([20]) == pytest.approx(4.0)
+    assert C.pipeline_makespan(m, [20], [0, 1], 2) == pytest.approx(2 * (4.0 + 3.0))
+    # (c) the FFN curve through (10, 5), (20, 25) has slope 2: one row gives 5 - 18 = -13 -> 0 (unclamped: 4 - 13 = -9)
+    m = C.Model(tokens, CONST(10.0), ([10.0, 20.0], [5.0, 25.0]), shared=True)
+    assert m.t_f(1) == 0.0 and m.t_f(15) == pytest.approx(15.0)
+    assert C.pipeline_makespan(m, [20], [0, 1], 1) == pytest.approx(4.0)
+    # separate pools: the clamped stage still occupies no time on its engine (A0 0-0, F0 0-3, A1 0-0, F1 3-6)
+    m = C.Model(tokens, CONST(4.0), CONST(3.0))
+    assert C.pipeline_makespan(m, [20, 20], [0, 1, 2], 1) == pytest.approx(6.0)
+
+
 def test_plan_prefers_depth_one_on_a_shared_memory_system():
     # fixed cost per stage launch (curves with an intercept): splitting only adds cost
     m = C.Model(([0.0, 1000.0], [10.0, 110.0]), CONST(5.0), ([0.0, 64.0], [100.0, 110.0]), shared=True)
