@@ -164,7 +164,10 @@ AFLEX_API aflex_status aflex_attn_decode(aflex_ctx* ctx, const aflex_attn_desc* 
  * library's device image, present on every GPU that loads the library until the process
  * exits.  The caller still passes every input and output.
  *
- * Same arguments, layouts, arithmetic and result as aflex_attn_decode.  Limits of the fixed
+ * Same arguments, layouts and arithmetic as aflex_attn_decode (the split of the work over CTAs
+ * differs, so results agree to rounding, not bit for bit).  What the kernel finds wrong while
+ * it runs (a length or page id out of range, an expired wait) is read with
+ * aflex_attn_decode_static_status below.  Limits of the fixed
  * scratch: batch * num_kv_heads <= 16384 (otherwise AFLEX_ERR_WORKSPACE is returned and
  * nothing is launched) and at most 320 persistent CTAs are used.  Other errors:
  * AFLEX_ERR_INVALID_ARG / AFLEX_ERR_UNSUPPORTED as for aflex_attn_decode, AFLEX_ERR_CUDA.
@@ -181,6 +184,22 @@ AFLEX_API aflex_status aflex_attn_decode(aflex_ctx* ctx, const aflex_attn_desc* 
  */
 AFLEX_API aflex_status aflex_attn_decode_static(const aflex_attn_desc* desc, const void* q, const aflex_kv* kv,
                                                 int batch, void* out, float* lse, void* stream);
+
+/*
+ * Device-side status of the calls of aflex_attn_decode_static on the current device (no
+ * counterpart in the paper either).  The kernel records what it meets while it runs in a status
+ * word of the fixed scratch -- AFLEX_ERR_BOUNDS: a sequence length outside
+ * [1, max_pages_per_seq * 16] (clamped; a sequence clamped to 0 gets no output) or a page id
+ * outside [0, num_pages) (page 0 is read instead); AFLEX_ERR_TIMEOUT: a bounded wait expired
+ * and rows are missing -- and aflex_attn_decode_static's own return value cannot carry it, since
+ * the call only enqueues work.  This call copies the word to *host_status on `stream`
+ * (one cudaMemcpyAsync, no allocation) and synchronises that stream; pass the stream the
+ * attention calls ran on.  Every aflex_attn_decode_static call re-zeroes the word before its
+ * kernel, so the value read is that of the last call enqueued before this one.  Returns
+ * AFLEX_ERR_INVALID_ARG for a null pointer or when no static call has been made on the current
+ * device yet, AFLEX_ERR_CUDA on a runtime error, else AFLEX_OK with *host_status set.
+ */
+AFLEX_API aflex_status aflex_attn_decode_static_status(int* host_status, void* stream);
 
 /*
  * Prefill (causal) attention: the attention operator of the prefill phase (the paper's "PA" pool; Section 1: in

@@ -24,7 +24,7 @@ EXPORTS = (
     "aflex_get_device_status", "aflex_attn_decode", "aflex_ffn_dense", "aflex_ffn_moe", "aflex_layer_step",
     "aflex_workspace_bytes", "aflex_linear", "aflex_set_attn_ctas", "aflex_set_attn_q_final", "aflex_num_kernel_kinds",
     "aflex_kernel_name", "aflex_launch_count", "aflex_profile_enable", "aflex_profile_read",
-    "aflex_trace_read", "aflex_attn_decode_static", "aflex_decoder_layers", "aflex_decoder_workspace_bytes",
+    "aflex_trace_read", "aflex_attn_decode_static", "aflex_attn_decode_static_status", "aflex_decoder_layers", "aflex_decoder_workspace_bytes",
     "aflex_add_rmsnorm", "aflex_rope_append", "aflex_attn_prefill", "aflex_af_decoder_layers", "aflex_af_workspace_bytes",
     "aflex_prefill_layers", "aflex_prefill_workspace_bytes",
     "aflex_eq2_layer_time", "aflex_curve_eval",
@@ -175,6 +175,8 @@ def load_library() -> ctypes.CDLL:
                                             ctypes.POINTER(ci)]
     lib.aflex_attn_decode_static.restype = ci
     lib.aflex_attn_decode_static.argtypes = [ctypes.POINTER(AttnDesc), vp, ctypes.POINTER(KV), ci, vp, vp, vp]
+    lib.aflex_attn_decode_static_status.restype = ci
+    lib.aflex_attn_decode_static_status.argtypes = [ctypes.POINTER(ci), vp]
     _lib = lib
     return lib
 
@@ -275,6 +277,17 @@ def attn_decode_static(desc: AttnDesc, q: torch.Tensor, kv: KV, out: torch.Tenso
                                       _stream(stream))
     if st != OK:
         raise AflexError(st, lib.aflex_status_string(st).decode(), _STATIC_ERRORS.get(st, "unknown error"))
+
+
+def attn_decode_static_status(stream=None) -> int:
+    """What the kernel of the last attn_decode_static call on this device recorded while it ran (OK,
+    ERR_BOUNDS for a clamped length or a redirected page id, ERR_TIMEOUT); synchronises the stream."""
+    lib = load_library()
+    v = ctypes.c_int(-1)
+    st = lib.aflex_attn_decode_static_status(ctypes.byref(v), _stream(stream))
+    if st != OK:
+        raise AflexError(st, lib.aflex_status_string(st).decode(), _STATIC_ERRORS.get(st, "unknown error"))
+    return int(v.value)
 
 
 # --------------------------------------------------------------------------- host-side decisions

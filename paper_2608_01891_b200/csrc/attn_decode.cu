@@ -117,9 +117,19 @@ struct Walker {
         b = r.b; prefix = r.prefix;
         len = usable_len(lens[b], max_pages); nu = (len + kUnitTokens - 1) / kUnitTokens + cost;
         const long long rel = pos - prefix * Hkv;
-        g = (int)(rel / nu); u = (int)(rel % nu);
+        if (nu > 0) { g = (int)(rel / nu); u = (int)(rel % nu); }
+        else { g = 0; u = 0; }                  // an item without any position (length 0, cost 0): skip_empty() steps over it
     }
     __device__ bool done() const { return pos >= end; }
+    // Step over list positions that hold no work: the `cost` empty positions charged in front of every item,
+    // and items that have no position at all (a sequence whose usable length is 0 when cost is 0).
+    __device__ void skip_empty() {
+        while (!done()) {
+            if (u < cost) advance(1);
+            else if (u >= nu) advance(0);
+            else break;
+        }
+    }
     // advance by n units inside the current item, moving to the next item / sequence when it ends
     __device__ void advance(int n) {
         pos += n; u += n;
@@ -229,7 +239,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             const int v = __shfl_up_sync(0xffffffffu, incl, off);
             if (lane >= off) incl += v;
         }
-        __shared__ int warp_tot[kAttnConsumerWarps + 1];
+        __shared__ int warp_tot[kAttnThreads / 32];
         if (lane == 31) warp_tot[warp] = incl;
         __syncthreads();
         int base = 0;
@@ -291,7 +301,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             locate(x0, rg0.b, rg0.prefix);
             Walker w0;
             w0.init(p, rg0);
-            while (!w0.done() && w0.u < w0.cost) w0.advance(1);
+            w0.skip_empty();
             pid0 = w0.done() ? 0 : page_id(w0);          // also warms the page-table line
         }
         // KV loads do not wait for the grid dependency: the only kernel of this library that writes the
@@ -317,7 +327,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                 else { rg.x0 = x0; rg.x1 = x1; rg.rid = rid; locate(x0, rg.b, rg.prefix); }
                 Walker wk;
                 wk.init(p, rg);
-                while (!wk.done() && wk.u < wk.cost) wk.advance(1);     // positions without work
+                wk.skip_empty();                                         // positions without work
                 // a range without any real unit is not handed to the consumers at all (every published
                 // range then holds at least one ring stage, which is what bounds the range ring)
                 if (!wk.done()) {
@@ -328,7 +338,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                 while (!wk.done()) {
                     const int g = wk.g, u = wk.u - wk.cost, len = wk.len;
                     wk.advance(1);
-                    while (!wk.done() && wk.u < wk.cost) wk.advance(1);
+                    wk.skip_empty();
                     const int pid_next = wk.done() ? 0 : page_id(wk);   // one unit ahead of the ring
                     if (!claimed && issued >= kAttnStages) { claim(); claimed = true; }
                     ++issued;
@@ -551,7 +561,6 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             if (rg.x1 <= rg.x0) break;
             Walker wk;
             wk.init(p, rg);
-            bool first_piece = true;            // a partial piece uses slot 0 if it is the range's first piece, else 1
 
         while (!wk.done() && !aborted) {
             // ---- one piece: units [u0, u0 + n) of item (b, g)
@@ -564,8 +573,9 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             const int n = max(wk.u + nv, cost) - cost - u0;
             wk.advance(nv);
             if (n <= 0) continue;                                            // only empty positions: no piece
-            const int slot = first_piece ? 0 : 1;
-            first_piece = false;
+            // A range holds at most two partial pieces: one of an item that began before the range (slot 0) and one
+            // of an item that begins inside it (slot 1).  The merge below locates a piece by the same predicate.
+            const int slot = rg.x0 < item_v0 ? 1 : 0;
 
             const int s_last = (s + n - 1) % kAttnStages;
             s = (s + n) % kAttnStages;
@@ -992,4 +1002,19 @@ extern "C" aflex_status aflex_attn_decode_static(const aflex_attn_desc* desc, co
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     if (desc->head_dim == 128) return attn_static_launch<128>(stt, desc, q, kv, batch, out, lse, st);
     return attn_static_launch<64>(stt, desc, q, kv, batch, out, lse, st);
+}
+
+extern "C" aflex_status aflex_attn_decode_static_status(int* host_status, void* stream) {
+    using namespace aflex;
+    if (!host_status) return AFLEX_ERR_INVALID_ARG;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return AFLEX_ERR_CUDA;
+    const StaticDeviceState& stt = g_static_state[dev];
+    if (stt.scratch == nullptr) return AFLEX_ERR_INVALID_ARG;     // no static call on this device yet
+    const int* status = reinterpret_cast<const int*>(reinterpret_cast<const float*>(stt.scratch) + kStaticOPartFloats + kStaticMlFloats) +
+                        kStaticMaxItems;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(host_status, status, sizeof(int), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    return e == cudaSuccess ? AFLEX_OK : AFLEX_ERR_CUDA;
 }

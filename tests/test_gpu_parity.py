@@ -341,6 +341,36 @@ def test_out_of_range_page_id_is_reported_not_dereferenced(ctx):
     assert row_rel_err(got, want) <= TOL_ATTN
 
 
+def zero_length_case(seed, n_seq, Hq, Hkv, D):
+    """Sequences of which about a third have device length 0 (first, last and runs in the middle included),
+    the rest long enough to be split over several CTAs.  Returns (q, kv, device lengths, valid rows)."""
+    rng = np.random.default_rng(seed)
+    true_lens = rng.integers(300, 2500, size=n_seq)
+    zero = rng.random(n_seq) < 0.35
+    zero[0] = zero[-1] = True
+    zero[n_seq // 2: n_seq // 2 + 3] = True
+    q, kv = make_case(n_seq, Hq, Hkv, D, true_lens.tolist(), seed=20 + seed, poison=True)
+    dev_lens = kv.seq_lens.clone()
+    dev_lens[torch.from_numpy(zero)] = 0
+    return q, kv, dev_lens, np.flatnonzero(~zero)
+
+
+@pytest.mark.parametrize("seed,Hq,Hkv,D", [(0, 64, 8, 128), (1, 8, 2, 64), (2, 32, 8, 128)])
+def test_zero_length_sequences_between_valid_rows_are_skipped_and_reported(ctx, seed, Hq, Hkv, D):
+    """A device-side length of 0 (outside the contract: lengths are >= 1) is clamped and reported; the row gets no
+    output and its neighbours are unaffected - whichever CTA range begins or ends on the empty item."""
+    q, kv, dev_lens, valid = zero_length_case(seed, 48, Hq, Hkv, D)
+    got, lse = run_attention(ctx, q, kv.k_cache, kv.v_cache, kv.page_table, dev_lens, Hq, Hkv, D, with_host_lens=False)
+    assert ctx.device_status() == AF.ERR_BOUNDS
+    want, want_lse = O.attn_decode(u16(q[valid]), u16(kv.k_cache), u16(kv.v_cache), kv.page_table.numpy()[valid],
+                                   kv.seq_lens.numpy()[valid])
+    assert row_rel_err(got[valid], want) <= TOL_ATTN
+    assert np.abs(lse[valid] - want_lse).max() <= TOL_LSE
+    skipped = np.setdiff1d(np.arange(len(dev_lens)), valid)
+    assert np.isnan(got[skipped]).all()                    # rows of empty sequences are left as they were
+    assert ctx.device_status() == AF.OK
+
+
 def test_moe_many_experts_top1_and_empty_experts(ctx):
     """E = 64 experts with 5 tokens: almost every expert is empty; K = 1 and K = 2."""
     T, H, I, E = 5, 128, 256, 64
