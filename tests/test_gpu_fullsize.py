@@ -1,6 +1,8 @@
 """Full-size parity: configurations 2-5 at their real sizes, in the launch configuration the
-benchmark times (aflex_layer_step with the configuration's microbatch depths), checked on
-sampled batch rows that the fp64 oracle computes one by one (rows are independent), plus
+benchmark times (aflex_layer_step with the configuration's microbatch depths).  The attention
+output of EVERY sequence is compared with the fp64 oracle; the layer output is compared on batch
+rows chosen to cover every token tile of every GEMM launch and, for the MoE layers, both ends of
+every expert's row segment (rows are independent, so the oracle computes them one by one); plus
 properties that hold at any size."""
 import numpy as np
 import pytest
@@ -16,12 +18,45 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
 
-def sampled_rows(lens: np.ndarray, extra: int = 1):
-    """Shortest, longest and `extra` seeded random rows."""
-    rows = {int(np.argmin(lens)), int(np.argmax(lens))}
-    rng = np.random.default_rng(12345)
-    while len(rows) < min(len(lens), 2 + extra):
-        rows.add(int(rng.integers(len(lens))))
+def near_equal_offsets(batch: int, M: int):
+    """The library's default microbatch split: near-equal, the first batch % M microbatches one row larger."""
+    base, extra = divmod(batch, M)
+    offs = [0]
+    for i in range(M):
+        offs.append(offs[-1] + base + (1 if i < extra else 0))
+    return offs
+
+
+def token_tile(rows: int) -> int:
+    """Token rows per GEMM tile as the library picks them: the fewest tiles of at most 256 rows, equal widths,
+    rounded up to 16 (grouped GEMMs cap a tile at 128 rows at decode sizes)."""
+    rows = max(rows, 16)
+    tiles = (rows + 255) // 256
+    return min(256, -(-(-(-rows // tiles)) // 16) * 16)
+
+
+def coverage_rows(cfg, lens: np.ndarray, logits):
+    """Batch rows chosen so that, for every microbatch depth the configuration is run at, every token tile of
+    every GEMM launch holds a compared row: the first and last row of every microbatch and of every token tile
+    inside it; for the MoE layers also the first and last assignment of every expert's row segment in every
+    microbatch and both sides of every 128-row chunk boundary inside a segment.  Plus the shortest and longest
+    context, a seeded random row and eight evenly spread rows."""
+    rows = {int(np.argmin(lens)), int(np.argmax(lens)), int(np.random.default_rng(12345).integers(len(lens)))}
+    rows.update(range(0, len(lens), max(1, len(lens) // 8)))                  # evenly spread as well
+    idx = O.moe_route(logits, cfg.top_k)[0] if cfg.num_experts else None
+    for M in cfg.microbatch_depths:
+        offs = near_equal_offsets(cfg.batch, M)
+        for r0, r1 in zip(offs, offs[1:]):
+            nt = token_tile(r1 - r0)
+            for t0 in range(r0, r1, nt):
+                rows.update((t0, min(r1, t0 + nt) - 1))
+            if idx is None:
+                continue
+            chunk = min(128, nt)
+            for e in range(cfg.num_experts):
+                seg = [t for t in range(r0, r1) if e in idx[t]]         # the segment's rows, in token order
+                for c0 in range(0, len(seg), chunk):
+                    rows.update((seg[c0], seg[min(len(seg), c0 + chunk) - 1]))
     return sorted(rows)
 
 
@@ -34,16 +69,25 @@ def oracle_rows(cfg, wl, rows):
                         logits=logits, top_k=cfg.top_k)
 
 
+def oracle_attention_all_rows(wl):
+    """The oracle's attention for EVERY sequence of the workload (the whole paged cache goes to the host)."""
+    kvh = wl["kvh"]
+    out, _ = O.attn_decode(u16(wl["q"]), u16(kvh.k_cache), u16(kvh.v_cache), kvh.page_table.numpy(), kvh.seq_lens.numpy())
+    return out
+
+
 @pytest.mark.parametrize("cid", [2, 3, 4, 5])
-def test_layer_step_full_size_sampled_rows(cid):
+def test_layer_step_full_size_all_attention_rows_and_tile_covering_ffn_rows(cid):
     cfg = IN.CONFIGS[cid]
     torch.cuda.set_device(0)
     wl = bench.build_workload(cfg, DEV)
     lens = wl["kvh"].seq_lens.numpy()
     ctx = AF.Context(0, AF.workspace_bytes(wl["layer"], cfg.batch, wl["kvh"].max_pages_per_seq))
     try:
-        rows = sampled_rows(lens)
-        want_a, want_y = oracle_rows(cfg, wl, rows)
+        rows = coverage_rows(cfg, lens, wl["logits"].cpu().numpy() if cfg.num_experts else None)
+        assert len(rows) >= (8 if cfg.num_experts == 0 else 16)
+        _, want_y = oracle_rows(cfg, wl, rows)
+        want_a_all = oracle_attention_all_rows(wl)
         a = torch.full_like(wl["q"], float("nan"))
         results = {}
         for M in cfg.microbatch_depths:
@@ -52,11 +96,9 @@ def test_layer_step_full_size_sampled_rows(cid):
             ctx.layer_step(wl["layer"], wl["q"], wl["kv"], wl["y"], M, None, wl["logits"], a)
             torch.cuda.synchronize()
             assert ctx.device_status() == AF.OK
-            ya, yy = f64(a[rows]), f64(wl["y"][rows])
-            assert row_rel_err(ya, want_a) <= TOL_ATTN, (cid, M)
-            assert row_rel_err(yy, want_y) <= TOL_FFN, (cid, M)
-            # any-size properties: every output finite; attention output inside the convex hull bound
-            assert torch.isfinite(wl["y"].float()).all() and torch.isfinite(a.float()).all()
+            assert row_rel_err(f64(a), want_a_all) <= TOL_ATTN, (cid, M)        # every sequence, every head
+            assert row_rel_err(f64(wl["y"][rows]), want_y) <= TOL_FFN, (cid, M)
+            assert torch.isfinite(wl["y"].float()).all()
             results[M] = wl["y"].float().cpu().numpy().astype(np.float64)
         # the result does not depend on the microbatch depth (to bf16 rounding of different GEMM plans)
         base = results[cfg.microbatch_depths[0]]
