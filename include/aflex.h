@@ -255,6 +255,18 @@ AFLEX_API aflex_status aflex_ffn_moe(aflex_ctx* ctx, const void* x, const float*
                                      const void* w_down, int T, int H, int I, int E, int top_k, void* y,
                                      int32_t* topk_idx, float* topk_gate, int32_t* expert_counts, void* stream);
 
+/*
+ * The routing and permutation steps of aflex_ffn_moe on their own (same kernel), with every integer
+ * result exported: topk_idx i32 [T][K] and topk_gate fp32 [T][K] as above; expert_counts i32 [E];
+ * expert_offsets i32 [E+1] = exclusive prefix of the counts (expert e owns permuted rows
+ * [offsets[e], offsets[e+1])); pos i32 [T][K] = permuted row of assignment (t,k) =
+ * offsets[e] + number of assignments (t',k') to the same expert e that precede (t,k) in (t,k) order.
+ * All pointers device, all required.  router_logits fp32 [T][E].  Integer results are exact.
+ */
+AFLEX_API aflex_status aflex_moe_route(aflex_ctx* ctx, const float* router_logits, int T, int E, int top_k,
+                                       int32_t* topk_idx, float* topk_gate, int32_t* expert_counts,
+                                       int32_t* expert_offsets, int32_t* pos, void* stream);
+
 /* ---- Layer step: A side, boundary, F side, as M interleaved microbatches ---
  *
  * Computes, for the whole batch,
@@ -299,8 +311,11 @@ AFLEX_API aflex_status aflex_layer_step(aflex_ctx* ctx, const aflex_layer_desc* 
 
 /*
  * Workspace bytes that suffice for aflex_attn_decode / aflex_ffn_* /
- * aflex_layer_step on this layer with up to max_batch rows and sequences of up
- * to 16*max_pages_per_seq tokens.  Pure host computation.
+ * aflex_layer_step on this layer with up to max_batch rows, on the CURRENT device
+ * (the scratch of the persistent kernels is per SM; with no device the figure is
+ * for a 148-SM part) and for any setting of aflex_set_attn_ctas.  The attention
+ * scratch is per CTA, not per context token: max_pages_per_seq must be >= 1 and
+ * is otherwise unused.  Host computation, nothing is enqueued.
  */
 AFLEX_API size_t aflex_workspace_bytes(const aflex_layer_desc* layer, int max_batch, int max_pages_per_seq);
 

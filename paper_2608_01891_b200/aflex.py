@@ -21,7 +21,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_
 # Every symbol include/aflex.h declares.
 EXPORTS = (
     "aflex_status_string", "aflex_version", "aflex_create", "aflex_destroy", "aflex_last_error",
-    "aflex_get_device_status", "aflex_attn_decode", "aflex_ffn_dense", "aflex_ffn_moe", "aflex_layer_step",
+    "aflex_get_device_status", "aflex_attn_decode", "aflex_ffn_dense", "aflex_ffn_moe", "aflex_moe_route", "aflex_layer_step",
     "aflex_workspace_bytes", "aflex_linear", "aflex_set_attn_ctas", "aflex_set_attn_q_final", "aflex_num_kernel_kinds",
     "aflex_kernel_name", "aflex_launch_count", "aflex_profile_enable", "aflex_profile_read",
     "aflex_trace_read", "aflex_attn_decode_static", "aflex_attn_decode_static_status", "aflex_decoder_layers", "aflex_decoder_workspace_bytes",
@@ -123,6 +123,8 @@ def load_library() -> ctypes.CDLL:
     lib.aflex_ffn_dense.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, vp, vp]
     lib.aflex_ffn_moe.restype = ci
     lib.aflex_ffn_moe.argtypes = [vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, vp, vp, vp, vp, vp]
+    lib.aflex_moe_route.restype = ci
+    lib.aflex_moe_route.argtypes = [vp, vp, ci, ci, ci, vp, vp, vp, vp, vp, vp]
     lib.aflex_layer_step.restype = ci
     lib.aflex_layer_step.argtypes = [vp, ctypes.POINTER(LayerDesc), vp, ctypes.POINTER(KV), ci, vp, ci,
                                      ctypes.POINTER(ctypes.c_int32), vp, vp, vp]
@@ -466,6 +468,13 @@ class Context:
         self._check(self._lib.aflex_ffn_moe(self._h, _ptr(x), _ptr(router_logits), _ptr(w_router), _ptr(w_gate),
                                             _ptr(w_up), _ptr(w_down), T, H, I, E, top_k, _ptr(y), _ptr(topk_idx),
                                             _ptr(topk_gate), _ptr(expert_counts), _stream(stream)))
+
+    def moe_route(self, router_logits, top_k: int, topk_idx, topk_gate, expert_counts, expert_offsets, pos,
+                  stream=None) -> None:
+        """Routing + permutation alone: idx/gate [T,K], counts [E], offsets [E+1], pos [T,K] (device tensors)."""
+        T, E = router_logits.shape
+        self._check(self._lib.aflex_moe_route(self._h, _ptr(router_logits), T, E, top_k, _ptr(topk_idx), _ptr(topk_gate),
+                                              _ptr(expert_counts), _ptr(expert_offsets), _ptr(pos), _stream(stream)))
 
     def layer_step(self, layer: LayerDesc, q, kv: KV, y, microbatch_depth: int = 1,
                    mb_offsets: Optional[Sequence[int]] = None, router_logits=None, attn_out=None,

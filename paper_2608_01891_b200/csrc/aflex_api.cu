@@ -467,6 +467,19 @@ aflex_status aflex_ffn_moe(aflex_ctx* ctx, const void* x, const float* router_lo
                    expert_counts, ctx->ws, ctx->ws_bytes, reinterpret_cast<cudaStream_t>(stream));
 }
 
+aflex_status aflex_moe_route(aflex_ctx* ctx, const float* router_logits, int T, int E, int top_k, int32_t* topk_idx,
+                             float* topk_gate, int32_t* expert_counts, int32_t* expert_offsets, int32_t* pos, void* stream) {
+    if (!ctx) return AFLEX_ERR_INVALID_ARG;
+    if (!router_logits || !topk_idx || !topk_gate || !expert_counts || !expert_offsets || !pos)
+        return set_error(ctx, AFLEX_ERR_INVALID_ARG, "moe route: null argument");
+    aflex_status s = validate_moe(ctx, T, 8, 8, E, top_k);
+    if (s != AFLEX_OK) return s;
+    MoeBuffers mb;
+    mb.idx = topk_idx; mb.gate = topk_gate; mb.counts = expert_counts; mb.offsets = expert_offsets; mb.pos = pos;
+    mb.logits = nullptr;
+    return moe_route_launch(ctx, router_logits, T, E, top_k, mb, reinterpret_cast<cudaStream_t>(stream));
+}
+
 // Workspace layout of the layer step: [A region | attention output a | boundary x | F region].
 // The A region (attention partials, W_o split-K partials) is used only on the attention stream,
 // the F region only on the FFN stream; a and x are indexed by batch row, so microbatches touch
@@ -508,10 +521,21 @@ LayerWs layer_ws(const aflex_layer_desc* L, int max_batch, size_t a_attn, int nu
 }
 }  // namespace
 
+// SM count the workspace queries size for: the current device's (the per-SM scratch of the persistent
+// kernels scales with it, and the entry points size the same regions from their ctx's device), or 148
+// when no device can be asked (a host without a GPU).
+static int query_num_sms() {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
+        return sms;
+    (void)cudaGetLastError();   // no device: not an error of this query
+    return 148;
+}
+
 size_t aflex_workspace_bytes(const aflex_layer_desc* layer, int max_batch, int max_pages_per_seq) {
     if (!layer || max_batch < 1 || max_pages_per_seq < 1) return 0;
     (void)max_pages_per_seq;   // the attention scratch is per CTA, not per context token
-    return layer_ws(layer, max_batch, attn_workspace_bytes(&layer->attn, 4096), 148).total;
+    return layer_ws(layer, max_batch, attn_workspace_bytes(&layer->attn, 4096), query_num_sms()).total;
 }
 
 aflex_status aflex_layer_step(aflex_ctx* ctx, const aflex_layer_desc* L, const void* q, const aflex_kv* kv, int batch,
@@ -648,7 +672,7 @@ DecoderWs decoder_ws(const aflex_decoder_desc* d, int max_batch, size_t a_attn, 
 
 size_t aflex_decoder_workspace_bytes(const aflex_decoder_desc* layer, int max_batch) {
     if (!layer || max_batch < 1) return 0;
-    return decoder_ws(layer, max_batch, attn_workspace_bytes(&layer->layer.attn, 4096), 148).total;
+    return decoder_ws(layer, max_batch, attn_workspace_bytes(&layer->layer.attn, 4096), query_num_sms()).total;
 }
 
 aflex_status aflex_add_rmsnorm(aflex_ctx* ctx, const void* res, const void* add, const void* w, int T, int H, float eps,
@@ -847,7 +871,7 @@ PrefillWs prefill_ws(const aflex_decoder_desc* d, int T, int num_sms) {
 
 size_t aflex_prefill_workspace_bytes(const aflex_decoder_desc* layer, int max_tokens) {
     if (!layer || max_tokens < 1) return 0;
-    return prefill_ws(layer, max_tokens, 148).total;
+    return prefill_ws(layer, max_tokens, query_num_sms()).total;
 }
 
 aflex_status aflex_prefill_layers(aflex_ctx* ctx, const aflex_decoder_desc* layers, const aflex_kv* kvs, int num_layers,
@@ -948,7 +972,7 @@ struct DeviceGuard {
 
 size_t aflex_af_workspace_bytes(const aflex_decoder_desc* layer, int max_batch, int ffn_side) {
     if (!layer || max_batch < 1) return 0;
-    const PairWs w = pair_ws(layer, max_batch, attn_workspace_bytes(&layer->layer.attn, 4096), 148);
+    const PairWs w = pair_ws(layer, max_batch, attn_workspace_bytes(&layer->layer.attn, 4096), query_num_sms());
     return ffn_side ? w.f_total : w.a_total;
 }
 

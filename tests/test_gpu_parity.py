@@ -177,6 +177,30 @@ def test_moe_routing_bit_exact_and_values(ctx, T, grid):
     assert row_rel_err(y, want_y) <= TOL_FFN
 
 
+@pytest.mark.parametrize("T,E,K,ties", [(1, 8, 2, False), (33, 8, 2, True), (256, 8, 2, False), (700, 8, 2, True),
+                                        (5, 64, 1, False), (1300, 16, 2, False), (300, 3, 1, True)])
+def test_moe_permutation_positions_are_exact(ctx, T, E, K, ties):
+    """Routing + permutation alone, every integer result against the oracle bit for bit: indices, per-expert
+    counts, segment offsets and the permuted position of every assignment (a bijection onto [0, T*K) sorted by
+    (expert, token, k))."""
+    g = torch.Generator().manual_seed(100 + T)
+    logits = torch.randint(-1, 2, (T, E), generator=g).float() if ties else torch.randn(T, E, generator=g)
+    i32 = lambda *s: torch.full(s, -7, dtype=torch.int32, device=DEV)
+    idx, counts, offsets, pos = i32(T, K), i32(E), i32(E + 1), i32(T, K)
+    gate = torch.zeros(T, K, device=DEV)
+    ctx.moe_route(logits.to(DEV), K, idx, gate, counts, offsets, pos)
+    torch.cuda.synchronize()
+    want_idx, want_gate = O.moe_route(logits.numpy(), K)
+    want_counts, want_offsets, want_pos = O.moe_permute(want_idx, E)
+    assert (idx.cpu().numpy() == want_idx).all()
+    assert (counts.cpu().numpy() == want_counts).all()
+    assert (offsets.cpu().numpy() == want_offsets).all()
+    assert (pos.cpu().numpy() == want_pos).all()
+    assert sorted(pos.cpu().numpy().ravel().tolist()) == list(range(T * K))
+    assert np.abs(gate.cpu().numpy() - want_gate).max() <= TOL_GATE
+    assert ctx.device_status() == AF.OK
+
+
 def test_moe_top1_and_router_weight_mode(ctx):
     T, H, I, E = 40, 256, 256, 4
     x = rand_bf16((T, H), 1.0, 1)
