@@ -127,6 +127,8 @@ def algorithmic_bytes(cfg, lens, M):
     if cfg.num_experts == 0:
         out["gateup_gemm"] = 2.0 * I * H * 2 + rows * (H + I) * 2
         out["down_gemm"] = 1.0 * H * I * 2 + rows * (I + H) * 2
+        # decode batches run gate/up and down (and, at depth 1, W_o in front of them) as phases of one kernel
+        out["gemm_chain"] = out["gateup_gemm"] + out["down_gemm"] + (out["linear_gemm"] if M == 1 else 0.0)
     else:
         E, K = cfg.num_experts, cfg.top_k
         out["moe_gateup_gemm"] = 2.0 * E * I * H * 2 + rows * K * (H + I) * 2
@@ -139,6 +141,7 @@ def algorithmic_flops(cfg, M):
     rows = B / M
     k = cfg.top_k if cfg.num_experts else 1
     return {"linear_gemm": 2.0 * rows * H * Hq * D, "gateup_gemm": 4.0 * rows * H * I, "down_gemm": 2.0 * rows * H * I,
+            "gemm_chain": 6.0 * rows * H * I + (2.0 * rows * H * Hq * D if M == 1 else 0.0),
             "moe_gateup_gemm": 4.0 * rows * k * H * I, "moe_down_gemm": 2.0 * rows * k * H * I}
 
 

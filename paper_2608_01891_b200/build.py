@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libaflex.so")
-SOURCES = ["aflex_api.cu", "attn_decode.cu", "attn_prefill.cu", "control.cu", "decoder.cu", "gemm_tcgen05.cu", "moe.cu"]
+SOURCES = ["aflex_api.cu", "attn_decode.cu", "attn_prefill.cu", "control.cu", "decoder.cu", "gemm_chain.cu", "gemm_tcgen05.cu", "moe.cu"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
          "-Xcompiler", "-fPIC,-fvisibility=hidden", "--expt-relaxed-constexpr"]

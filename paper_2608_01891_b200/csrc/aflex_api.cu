@@ -128,20 +128,38 @@ static aflex_status validate_ffn_dims(aflex_ctx* ctx, int T, int H, int I) {
 // ---- F side, shared by the stand-alone entry points and the layer step -----------------------
 static size_t dense_ws_bytes(int T, int H, int I, int num_sms) {
     const size_t gu = gateup_workspace_bytes(T, H, I, num_sms), dn = linear_workspace_bytes(T, I, H, num_sms);
-    return align256((size_t)T * I * 2) + (gu > dn ? gu : dn);
+    const size_t ch = chain_supported(T) ? chain_workspace_bytes(T, num_sms) : 0;
+    const size_t scratch = gu > dn ? (gu > ch ? gu : ch) : (dn > ch ? dn : ch);
+    return align256((size_t)T * I * 2) + scratch;
 }
 
 static aflex_status dense_run(aflex_ctx* ctx, const void* x, const void* wg, const void* wu, const void* wd, int T,
-                              int H, int I, void* y, char* ws, size_t ws_bytes, cudaStream_t st) {
+                              int H, int I, void* y, char* ws, size_t ws_bytes, cudaStream_t st,
+                              const ChainStep* pre = nullptr) {
     Arena arena(ws, ws_bytes);
     __nv_bfloat16* h = arena.take<__nv_bfloat16>((size_t)T * I);
     // the two GEMMs run back to back on one stream: they share one scratch region and one counter array
     const size_t gu = gateup_workspace_bytes(T, H, I, ctx->num_sms), dn = linear_workspace_bytes(T, I, H, ctx->num_sms);
-    const size_t scratch = gu > dn ? gu : dn;
+    const size_t ch = chain_supported(T) ? chain_workspace_bytes(T, ctx->num_sms) : 0;
+    const size_t scratch = gu > dn ? (gu > ch ? gu : ch) : (dn > ch ? dn : ch);
     char* sws = scratch ? arena.take<char>(scratch) : nullptr;
     if (arena.overflow)
         return set_error(ctx, AFLEX_ERR_WORKSPACE, "dense ffn: need %zu workspace bytes, have %zu",
                          dense_ws_bytes(T, H, I, ctx->num_sms), ws_bytes);
+    if (chain_supported(T)) {
+        // decode batch: gate/up and down as two phases of one persistent kernel (x_pre, when given, is a projection
+        // that produces x and becomes a phase in front of them)
+        ChainStep steps[3];
+        int n = 0;
+        if (pre) steps[n++] = *pre;
+        steps[n++] = ChainStep{x, wg, wu, H, I, h};
+        steps[n++] = ChainStep{h, wd, nullptr, I, H, y};
+        return chain_launch(ctx, steps, n, T, sws, scratch, st, ctx->chain_counters);
+    }
+    if (pre) {
+        aflex_status sp = linear_launch(ctx, pre->in, pre->w0, T, pre->K, pre->N, pre->out, sws, scratch, st, kKLinearGemm, ctx->counters_f);
+        if (sp != AFLEX_OK) return sp;
+    }
     aflex_status s = gateup_launch(ctx, x, wg, wu, T, H, I, h, sws, scratch, st, ctx->counters_f);
     if (s != AFLEX_OK) return s;
     return linear_launch(ctx, h, wd, T, I, H, y, sws, scratch, st, kKDownGemm, ctx->counters_f);
@@ -265,6 +283,8 @@ aflex_status aflex_create(aflex_ctx** out, int device, size_t workspace_bytes) {
     if (e == cudaSuccess) e = cudaMalloc(&ctx->counters_f, 2 * kStreamKMaxTiles * sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(ctx->counters_a, 0, 2 * kStreamKMaxTiles * sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(ctx->counters_f, 0, 2 * kStreamKMaxTiles * sizeof(int));
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->chain_counters, chain_counter_ints() * sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(ctx->chain_counters, 0, chain_counter_ints() * sizeof(int));
     if (e == cudaSuccess && getenv("AFLEX_TRACE") && atoi(getenv("AFLEX_TRACE")) > 0) {
         const size_t tb = (size_t)kTraceKernels * kTraceStride * sizeof(unsigned long long);
         e = cudaMalloc(&ctx->trace, tb);
@@ -313,6 +333,7 @@ aflex_status aflex_destroy(aflex_ctx* ctx) {
     if (ctx->counters_attn) cudaFree(ctx->counters_attn);
     if (ctx->counters_a) cudaFree(ctx->counters_a);
     if (ctx->counters_f) cudaFree(ctx->counters_f);
+    if (ctx->chain_counters) cudaFree(ctx->chain_counters);
     if (ctx->ws) cudaFree(ctx->ws);
     delete ctx;
     return AFLEX_OK;
@@ -333,6 +354,7 @@ aflex_status aflex_get_device_status(aflex_ctx* ctx, void* stream) {
         cudaMemsetAsync(ctx->counters_attn, 0, (kAttnCounterCap + 2) * sizeof(int), st);
         cudaMemsetAsync(ctx->counters_a, 0, 2 * kStreamKMaxTiles * sizeof(int), st);
         cudaMemsetAsync(ctx->counters_f, 0, 2 * kStreamKMaxTiles * sizeof(int), st);
+        cudaMemsetAsync(ctx->chain_counters, 0, chain_counter_ints() * sizeof(int), st);
         cudaStreamSynchronize(st);
     }
     if (v != 0) set_error(ctx, (aflex_status)v, "device status word = %d (%s)", v, aflex_status_string((aflex_status)v));
@@ -342,7 +364,7 @@ aflex_status aflex_get_device_status(aflex_ctx* ctx, void* stream) {
 static const char* kKernelNames[kKKindCount] = {
     "attn_decode", "linear_gemm", "down_gemm", "gateup_gemm", "router_logits",
     "moe_route", "moe_gather", "moe_gateup_gemm", "moe_down_gemm", "moe_combine",
-    "add_rmsnorm", "qkv_gemm", "rope_append", "attn_prefill"};
+    "add_rmsnorm", "qkv_gemm", "rope_append", "attn_prefill", "gemm_chain"};
 
 int aflex_num_kernel_kinds(void) { return kKKindCount; }
 
@@ -607,7 +629,9 @@ aflex_status aflex_layer_step(aflex_ctx* ctx, const aflex_layer_desc* L, const v
         const __nv_bfloat16* qi = reinterpret_cast<const __nv_bfloat16*>(q) + (size_t)r0 * Hq * D;
         s = attn_decode_launch(ctx, &L->attn, qi, &kvi, rows, a_buf + (size_t)r0 * A, nullptr, ws_a, w.a_attn, sa);
         if (s != AFLEX_OK) return s;
-        if (L->w_o) {
+        // M = 1, dense FFN, decode batch: W_o, gate/up and down are the three phases of one persistent kernel
+        const bool chain3 = serial && E == 0 && L->w_o && chain_supported(rows);
+        if (L->w_o && !chain3) {
             s = linear_launch(ctx, a_buf + (size_t)r0 * A, L->w_o, rows, A, H, x_buf + (size_t)r0 * H, ws_alin, w.a_lin, sa, kKLinearGemm, ctx->counters_a);
             if (s != AFLEX_OK) return s;
         }
@@ -620,7 +644,8 @@ aflex_status aflex_layer_step(aflex_ctx* ctx, const aflex_layer_desc* L, const v
         __nv_bfloat16* yi = reinterpret_cast<__nv_bfloat16*>(y) + (size_t)r0 * H;
         const __nv_bfloat16* xi = x_buf + (size_t)r0 * H;
         if (E == 0) {
-            s = dense_run(ctx, xi, L->w_gate, L->w_up, L->w_down, rows, H, I, yi, ws_f, w.f_total, sf);
+            const ChainStep wo_step{a_buf + (size_t)r0 * A, L->w_o, nullptr, A, H, x_buf + (size_t)r0 * H};
+            s = dense_run(ctx, xi, L->w_gate, L->w_up, L->w_down, rows, H, I, yi, ws_f, w.f_total, sf, chain3 ? &wo_step : nullptr);
         } else {
             s = moe_run(ctx, xi, router_logits ? router_logits + (size_t)r0 * E : nullptr, L->w_router, L->w_gate,
                         L->w_up, L->w_down, rows, H, I, E, K, yi, nullptr, nullptr, nullptr, ws_f, w.f_total, sf);

@@ -1,0 +1,623 @@
+// A chain of dependent decode-batch GEMMs as ONE persistent tcgen05 kernel, software-pipelined
+// across the GEMMs.
+//
+// At decode batch sizes (<= 64 token rows) the FFN side and the W_o projection are weight-streaming
+// kernels: the boundary projection x = a W_o^T, h = silu(x W_gate^T) .* (x W_up^T) and y = h W_down^T
+// each read their weights once and are bound by HBM.  Run as separate kernels, every boundary between
+// two of them leaves DRAM idle: the last CTAs of one kernel finish their shared-tile reduction while
+// the next kernel's CTAs cannot become resident beside them (shared memory), set up, and only then
+// request their first bytes.  Here the GEMMs are PHASES of one kernel, and no phase ever waits for
+// the whole of its predecessor:
+//
+//   * one CTA per SM stays resident for all phases; barriers, TMEM and the shared-memory ring are set
+//     up once and the ring keeps turning across phase boundaries;
+//   * the weight producer (warp 0) never waits for anything but a free ring stage: weights are inputs
+//     that no kernel writes;
+//   * every phase produces its output tiles in two SEGMENTS, one after the other (remainder tiles that
+//     are shared along K first, whole tiles second; a phase whose tiles are all shared is one segment,
+//     or optionally two halves).  A segment's output is complete - its shared-tile reductions included - while the next
+//     segment streams, and is announced through an epoch word;
+//   * a K step of phase p+1 reads 64 or 128 columns of phase p's output, i.e. the output of ONE tile of
+//     phase p.  Every piece of work of phase p+1 (a run of K steps of one tile in one CTA) visits the
+//     K steps fed by segment 0 of phase p first and those fed by segment 1 after (any K order gives the
+//     same sum up to rounding; the order is a fixed function of the piece, so results are bit-
+//     deterministic).  The activation producer (warp 6) waits (bounded) for segment 0's epoch before
+//     its first early step and for segment 1's epoch before its first late step - by which time the
+//     epilogue, the reduction and the slowest CTA of that segment have had the early steps' streaming
+//     time to finish;
+//   * per segment the tiles are dealt exactly like the stand-alone GEMM (gemm_sched.cuh): equal,
+//     contiguous shares of K steps, partials reduced in CTA order.
+//
+// Orientation as in gemm_tcgen05.cu: 128 weight rows are the MMA's M operand, the token rows its N
+// operand; the accumulator in TMEM is out^T (lane = weight row, column = token).
+//
+// A ring stage holds two 128x64 weight tiles and two activation tiles.  A gate/up phase uses them as
+// (gate tile, up tile, x tile) of one 64-wide K block with two accumulators; a linear phase as two
+// consecutive K blocks (w, w', x, x') of one accumulator, so that both phase kinds keep the whole ring
+// in flight.
+//
+// CTA = 7 warps: 0 weight producer, 1 MMA issuer (owns TMEM), 2..5 epilogue, 6 activation producer.
+// Every wait is bounded; on expiry the CTA raises AFLEX_ERR_TIMEOUT, drains and leaves.
+#include <cuda_bf16.h>
+#include <stdlib.h>
+
+#include "internal.h"
+#include "ptx.cuh"
+#include "gemm_sched.cuh"
+
+namespace aflex {
+
+constexpr int kChainThreads = 224;
+constexpr int kChainBlockM = 128;
+constexpr int kChainBlockK = 64;
+constexpr int kChainTileBytes = kChainBlockM * kChainBlockK * 2;   // one weight tile: 16 KB
+constexpr int kChainMaxStages = 8;
+constexpr int kChainMaxPhases = 3;
+constexpr int kChainSlots = 8;
+constexpr int kChainCounterInts = 8192;   // per half of the double-buffered counter array: per-tile counters, then the epoch words
+constexpr int kChainEpochBase = kChainCounterInts - 16;          // partial slots per CTA: [phase parity][segment][first / later unit]
+
+struct ChainPhase {
+    int gateup;        // 1: two weight matrices, SwiGLU epilogue; 0: plain linear
+    int N;             // weight rows (output features)
+    int K;             // reduction length
+    int ksteps;        // ring stages per tile: ceil(K / 64) (gate/up) or ceil(K / 128) (linear)
+    int seg_tiles[2];  // output tiles of segment 0 (ids 0 ..) and of segment 1 (ids seg_tiles[0] ..)
+    int n_early;       // K steps [0, n_early) read what the previous phase's segment 0 wrote (first phase: all)
+    int counter_base;  // first per-tile arrival counter of this phase
+    __nv_bfloat16* out;   // [T][N]
+};
+
+struct ChainParams {
+    int T;             // token rows (<= n_tile)
+    int n_tile;        // accumulator columns per matrix: T rounded up to 16
+    int box;           // token rows per activation box (TMA) = MMA N
+    int nphase;
+    int stages;
+    int tmem_cols;
+    ChainPhase ph[kChainMaxPhases];
+    float* partials;   // [grid][kChainSlots][2 * n_tile / 4][128 rows] float4
+    int* counters;     // two halves of kChainCounterInts ints, then the generation word.  A launch of generation g counts
+                       // in half g & 1 (per-tile arrival counters and, at kChainEpochBase, its epoch words: (phase, segment)
+                       // finished by so many CTAs; all zero on entry), zeroes the other half for its successor and bumps g
+    int* status;
+    unsigned long long* trace;   // optional [grid][32] timestamps (ns), or nullptr
+};
+
+struct ChainMaps {
+    CUtensorMap a0[kChainMaxPhases];   // weights (gate/up: W_gate)
+    CUtensorMap a1[kChainMaxPhases];   // gate/up: W_up; linear: unused (a0 again)
+    CUtensorMap b[kChainMaxPhases];    // the phase's input activations
+};
+
+struct __align__(8) ChainBarriers {
+    uint64_t full[kChainMaxStages];     // 2 arrivals (weight producer, activation producer) + their bytes
+    uint64_t empty[kChainMaxStages];
+    uint64_t tmem_full[2];
+    uint64_t tmem_empty[2];
+    uint32_t tmem_base;
+    volatile int abort;
+    volatile int gen;       // this launch's generation, published by the epilogue once the grid dependency has resolved (-1 before)
+};
+
+// The order in which a piece (logical K positions [j0, j1) of a tile with nK steps, n_early of them "early")
+// visits the actual K steps: its share of the early steps first, then its share of the late ones.  Over the
+// pieces of a tile the two shares partition [0, n_early) and [n_early, nK).
+struct StepOrder {
+    int eb0, n_early_here, late0;
+    __device__ StepOrder(int j0, int j1, int nK, int n_early) {
+        eb0 = (int)((long long)j0 * n_early / nK);
+        const int eb1 = (int)((long long)j1 * n_early / nK);
+        n_early_here = eb1 - eb0;
+        late0 = n_early + (j0 - eb0);
+    }
+    __device__ int actual(int i) const { return i < n_early_here ? eb0 + i : late0 + (i - n_early_here); }
+};
+
+__device__ __forceinline__ float chain_silu(float z) { return __fdividef(z, 1.0f + __expf(-z)); }
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+
+__global__ void __launch_bounds__(kChainThreads, 1)
+gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const ChainParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const int b_bytes = (p.n_tile * kChainBlockK * 2 + 1023) & ~1023;       // one activation tile slot
+    const int stage_bytes = 2 * kChainTileBytes + 2 * b_bytes;
+    ChainBarriers* bars = reinterpret_cast<ChainBarriers*>(smem + (size_t)p.stages * stage_bytes);
+    // epilogue staging: the output tile as [token][128 features] bf16, so that it leaves the SM in 16-byte pieces
+    __nv_bfloat16* stage_out = reinterpret_cast<__nv_bfloat16*>(smem + (size_t)p.stages * stage_bytes + 1024);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int grid = (int)gridDim.x;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; ++s) { mbar_init(&bars->full[s], 2); mbar_init(&bars->empty[s], 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&bars->tmem_full[b], 1); mbar_init(&bars->tmem_empty[b], 4); }
+        bars->abort = 0;
+        bars->gen = -1;
+        fence_mbar_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(&bars->tmem_base, (uint32_t)p.tmem_cols);
+        tmem_relinquish();
+    }
+    if (warp == 0 && lane == 0) {
+        for (int i = 0; i < p.nphase; ++i) { prefetch_tmap(&maps.a0[i]); if (p.ph[i].gateup) prefetch_tmap(&maps.a1[i]); }
+    }
+    if (warp == 6 && lane == 0) {
+        for (int i = 0; i < p.nphase; ++i) prefetch_tmap(&maps.b[i]);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+
+    const uint32_t tmem_base = bars->tmem_base;
+    const int buf_cols = 2 * p.n_tile;                   // TMEM columns per accumulator buffer (room for gate and up)
+    pdl_launch_dependents();
+    unsigned long long* tr = p.trace ? p.trace + (size_t)blockIdx.x * 32 : nullptr;
+    if (tr && threadIdx.x == 0) { tr[0] = global_timer_ns(); unsigned smid; asm volatile("mov.u32 %0, %%smid;" : "=r"(smid)); tr[3] = smid; }   // CTA running
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ weight producer
+        if (lane == 0) {
+            const uint64_t pol_w = policy_evict_first();      // every weight byte is read once
+            int s = 0; uint32_t ph = 0;
+            for (int pi = 0; pi < p.nphase && !bars->abort; ++pi) {
+                const ChainPhase& P = p.ph[pi];
+                for (int seg = 0; seg < 2 && !bars->abort; ++seg) {
+                    const Schedule sched(P.ksteps, 1, P.seg_tiles[seg], grid);
+                    UnitCursor cur(sched, blockIdx.x);
+                    WorkUnit wu;
+                    while (!bars->abort && cur.next(wu)) {
+                        const int row0 = (seg * P.seg_tiles[0] + wu.tile) * kChainBlockM;
+                        const StepOrder ord(wu.kb0, wu.kb1, P.ksteps, P.n_early);
+                        for (int i = 0; i < wu.kb1 - wu.kb0; ++i) {
+                            const int ks = ord.actual(i);
+                            if (!mbar_wait(&bars->empty[s], ph ^ 1)) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); break; }
+                            uint8_t* st = smem + (size_t)s * stage_bytes;
+                            mbar_expect_tx(&bars->full[s], 2u * kChainTileBytes);
+                            if (P.gateup) {
+                                tma_load_2d_hint(st, &maps.a0[pi], ks * kChainBlockK, row0, &bars->full[s], pol_w);
+                                tma_load_2d_hint(st + kChainTileBytes, &maps.a1[pi], ks * kChainBlockK, row0, &bars->full[s], pol_w);
+                            } else {
+                                tma_load_2d_hint(st, &maps.a0[pi], 2 * ks * kChainBlockK, row0, &bars->full[s], pol_w);
+                                tma_load_2d_hint(st + kChainTileBytes, &maps.a0[pi], (2 * ks + 1) * kChainBlockK, row0, &bars->full[s], pol_w);
+                            }
+                            if (++s == p.stages) { s = 0; ph ^= 1; }
+                        }
+                    }
+                }
+                if (tr) tr[4 + pi * 8 + 0] = global_timer_ns();       // phase's weight loads all issued
+            }
+            if (bars->abort) {
+                for (int i = 0; i < 200; ++i) __nanosleep(1000);     // loads land within microseconds; their barriers may never complete
+            }
+        }
+    } else if (warp == 6) {
+        // ------------------------------------------------------------ activation producer
+        if (lane == 0) {
+            const uint64_t pol_x = policy_evict_last();       // activations are re-read by every CTA
+            const uint32_t box_bytes = (uint32_t)(p.box * kChainBlockK * 2);
+            int s = 0; uint32_t ph = 0;
+            pdl_wait();                                       // the first phase's input comes from the preceding kernel
+            if (tr) tr[1] = global_timer_ns();
+            for (int pi = 0; pi < p.nphase && !bars->abort; ++pi) {
+                const ChainPhase& P = p.ph[pi];
+                bool ready[2] = {pi == 0, pi == 0};
+                // Segment e of the previous phase complete in every CTA, and visible to the TMA reads that follow.
+                auto need = [&](int e) -> bool {
+                    if (ready[e]) return true;
+                    const long long t_start = clock64();
+                    int gen;
+                    while ((gen = bars->gen) < 0 && clock64() - t_start < kWaitBudgetCycles) __nanosleep(20);
+                    if (gen < 0) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); return false; }
+                    const int* word = p.counters + (size_t)(gen & 1) * kChainCounterInts + kChainEpochBase + (pi - 1) * 2 + e;
+                    int seen;
+                    do {
+                        asm volatile("ld.acquire.gpu.b32 %0, [%1];" : "=r"(seen) : "l"(word) : "memory");
+                        if (seen >= grid) break;
+                        __nanosleep(20);
+                    } while (clock64() - t_start < kWaitBudgetCycles);
+                    if (seen < grid) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); return false; }
+                    fence_proxy_async_all();
+                    // every CTA's epilogue has read the generation by now (it signals only afterwards): one thread of the
+                    // grid moves it on for the next launch
+                    if (blockIdx.x == 0 && pi == 1 && !ready[0] && !ready[1]) p.counters[2 * kChainCounterInts] = (gen + 1) & 0x3fffffff;
+                    ready[e] = true;
+                    if (tr) tr[4 + pi * 8 + 1 + e] = global_timer_ns();   // input from segment e available
+                    return true;
+                };
+                for (int seg = 0; seg < 2 && !bars->abort; ++seg) {
+                    const Schedule sched(P.ksteps, 1, P.seg_tiles[seg], grid);
+                    UnitCursor cur(sched, blockIdx.x);
+                    WorkUnit wu;
+                    while (!bars->abort && cur.next(wu)) {
+                        const StepOrder ord(wu.kb0, wu.kb1, P.ksteps, P.n_early);
+                        for (int i = 0; i < wu.kb1 - wu.kb0; ++i) {
+                            const int ks = ord.actual(i);
+                            if (!need(ks < P.n_early ? 0 : 1)) break;
+                            if (!mbar_wait(&bars->empty[s], ph ^ 1)) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); break; }
+                            uint8_t* st = smem + (size_t)s * stage_bytes + 2 * kChainTileBytes;
+                            if (P.gateup) {
+                                mbar_expect_tx(&bars->full[s], box_bytes);
+                                tma_load_2d_hint(st, &maps.b[pi], ks * kChainBlockK, 0, &bars->full[s], pol_x);
+                            } else {
+                                mbar_expect_tx(&bars->full[s], 2u * box_bytes);
+                                tma_load_2d_hint(st, &maps.b[pi], 2 * ks * kChainBlockK, 0, &bars->full[s], pol_x);
+                                tma_load_2d_hint(st + b_bytes, &maps.b[pi], (2 * ks + 1) * kChainBlockK, 0, &bars->full[s], pol_x);
+                            }
+                            if (++s == p.stages) { s = 0; ph ^= 1; }
+                        }
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            int s = 0; uint32_t ph = 0;
+            int buf = 0; uint32_t acc_ph = 0;
+            const uint32_t idesc = umma_idesc_bf16(kChainBlockM, (uint32_t)p.box);
+            for (int pi = 0; pi < p.nphase && !bars->abort; ++pi) {
+                const ChainPhase& P = p.ph[pi];
+                for (int seg = 0; seg < 2 && !bars->abort; ++seg) {
+                    const Schedule sched(P.ksteps, 1, P.seg_tiles[seg], grid);
+                    UnitCursor cur(sched, blockIdx.x);
+                    WorkUnit wu;
+                    while (!bars->abort && cur.next(wu)) {
+                        if (!mbar_wait(&bars->tmem_empty[buf], acc_ph ^ 1)) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); break; }
+                        tc_fence_after();
+                        const uint32_t d0 = tmem_base + (uint32_t)(buf * buf_cols);
+                        for (int i = 0; i < wu.kb1 - wu.kb0; ++i) {
+                            if (!mbar_wait(&bars->full[s], ph)) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); break; }
+                            tc_fence_after();
+                            const uint32_t a_addr = smem_u32(smem + (size_t)s * stage_bytes);
+                            const uint64_t da0 = umma_desc_k_sw128(a_addr);
+                            const uint64_t da1 = umma_desc_k_sw128(a_addr + kChainTileBytes);
+                            const uint64_t db0 = umma_desc_k_sw128(a_addr + 2 * kChainTileBytes);
+                            const uint64_t db1 = umma_desc_k_sw128(a_addr + 2 * kChainTileBytes + b_bytes);
+                            if (P.gateup) {
+#pragma unroll
+                                for (int k = 0; k < kChainBlockK / 16; ++k) {
+                                    const uint32_t acc = (i > 0 || k > 0) ? 1u : 0u;
+                                    umma_bf16(d0, da0 + 2 * k, db0 + 2 * k, idesc, acc);
+                                    umma_bf16(d0 + (uint32_t)p.n_tile, da1 + 2 * k, db0 + 2 * k, idesc, acc);
+                                }
+                            } else {
+#pragma unroll
+                                for (int k = 0; k < kChainBlockK / 16; ++k)
+                                    umma_bf16(d0, da0 + 2 * k, db0 + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
+#pragma unroll
+                                for (int k = 0; k < kChainBlockK / 16; ++k)
+                                    umma_bf16(d0, da1 + 2 * k, db1 + 2 * k, idesc, 1u);
+                            }
+                            umma_commit(&bars->empty[s]);
+                            if (++s == p.stages) { s = 0; ph ^= 1; }
+                        }
+                        if (bars->abort) break;
+                        umma_commit(&bars->tmem_full[buf]);
+                        if (tr && wu.slot < 0) tr[18] = global_timer_ns();
+                        if (++buf == 2) { buf = 0; acc_ph ^= 1; }
+                    }
+                }
+                if (tr) tr[4 + pi * 8 + 3] = global_timer_ns();       // phase's last MMA issued
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue (warps 2..5)
+        const int lane_grp = warp & 3;
+        const int row = lane_grp * 32 + lane;
+        const int etid = threadIdx.x - 64;
+        const size_t slot_floats = (size_t)2 * p.n_tile * kChainBlockM;
+        int buf = 0; uint32_t acc_ph = 0;
+        pdl_wait();   // nothing is written (outputs, partials, counters) before the preceding kernels have completed
+        // The counters are double-buffered over launches: this launch counts in one half (zero on entry) and zeroes
+        // the other half, which the launch before it used and the launch after it will use.  Both neighbours are
+        // ordered against these stores by the grid dependency (the wait above; the next launch's own wait).
+        if (etid == 0) {
+            int g;
+            asm volatile("ld.relaxed.gpu.b32 %0, [%1];" : "=r"(g) : "l"(p.counters + 2 * kChainCounterInts) : "memory");
+            bars->gen = g;
+        }
+        asm volatile("bar.sync 2, 128;" ::: "memory");
+        int* const ctr = p.counters + (size_t)(bars->gen & 1) * kChainCounterInts;
+        {
+            int* other = p.counters + (size_t)((bars->gen & 1) ^ 1) * kChainCounterInts;
+            for (int i = (int)blockIdx.x * 128 + etid; i < kChainCounterInts; i += grid * 128) other[i] = 0;
+        }
+
+        for (int pi = 0; pi < p.nphase && !bars->abort; ++pi) {
+            const ChainPhase& P = p.ph[pi];
+            const int accs = P.gateup ? 2 : 1;
+            for (int seg = 0; seg < 2 && !bars->abort; ++seg) {
+                const Schedule sched(P.ksteps, 1, P.seg_tiles[seg], grid);
+                const int tile0 = seg * P.seg_tiles[0];                    // first tile id of this segment
+                int* counters = ctr + P.counter_base + tile0;
+                const int slot0 = ((pi & 1) * 2 + seg) * 2;                // this (phase parity, segment)'s pair of partial slots
+                int pend[2];
+                int npend = 0;
+
+                // Token rows [t_lo, t_hi) of the staged tile -> out[t][128 * tile ..], 16 bytes per thread and store; the
+                // trailing barrier frees the staging buffer for its next user.
+                auto store_rows = [&](int tile_g, int t_lo, int t_hi) {
+                    if (t_hi > p.T) t_hi = p.T;
+                    for (int c = t_lo * 16 + etid; c < t_hi * 16; c += 128) {
+                        const int t = c >> 4, part = c & 15;
+                        const int n = tile_g * kChainBlockM + part * 8;
+                        if (n < P.N)
+                            *reinterpret_cast<uint4*>(P.out + (size_t)t * P.N + n) = *reinterpret_cast<const uint4*>(stage_out + t * kChainBlockM + part * 8);
+                    }
+                    asm volatile("bar.sync 2, 128;" ::: "memory");
+                };
+
+                // This CTA's slice of a shared tile, summed over the pieces in CTA order (see gemm_tcgen05.cu).
+                auto run_reduce = [&](int tile) {
+                    const long long x0 = (long long)tile * P.ksteps;
+                    const int cf = sched.cta_of(x0);
+                    const int cl = sched.cta_of(x0 + P.ksteps - 1);
+                    const int np = cl - cf + 1, me = (int)blockIdx.x - cf;
+                    const int nred = (np > 1 && sched.share_begin(cl + 1) > x0 + P.ksteps) ? np - 1 : np;
+                    if (me >= nred) return;
+                    if (etid == 0) {
+                        const long long t_start = clock64();
+                        int seen;
+                        do {
+                            asm volatile("ld.acquire.gpu.b32 %0, [%1];" : "=r"(seen) : "l"(counters + tile) : "memory");
+                            if (seen >= np) break;
+                            __nanosleep(64);
+                        } while (clock64() - t_start < kWaitBudgetCycles);
+                        if (seen < np) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); }
+                    }
+                    asm volatile("bar.sync 2, 128;" ::: "memory");     // the acquire above, handed on to the other 127 threads
+                    if (tr && etid == 0) tr[30] = global_timer_ns();
+                    if (bars->abort) return;
+                    const bool cf_early = sched.share_begin(cf) < x0;
+                    // The parked accumulator is [column group of 4 tokens][128 rows] float4: reducer `me` takes whole column
+                    // groups, thread = weight row.  kE groups per round, every piece's loads of a round in flight together
+                    // (the loop is a chain of L2 round trips, not bandwidth).
+                    const int ncg = ((p.T + 15) / 16) * 4;
+                    const int cg_lo = ncg * me / nred, cg_hi = ncg * (me + 1) / nred;
+                    const int up_off = (p.n_tile >> 2) * kChainBlockM;
+                    constexpr int kE = 4;
+                    for (int c0 = cg_lo; c0 < cg_hi; c0 += kE) {
+                        float4 g[kE], u[kE];
+#pragma unroll
+                        for (int e = 0; e < kE; ++e) g[e] = u[e] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        for (int cb = cf; cb <= cl; cb += 4) {
+                            float4 a[kE][4];
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                const int cc = cb + q;
+                                if (cc <= cl) {
+                                    const int sl = slot0 + ((cc == cf && cf_early) ? 1 : 0);
+                                    const float4* part = reinterpret_cast<const float4*>(p.partials + ((size_t)cc * kChainSlots + sl) * slot_floats) + etid;
+#pragma unroll
+                                    for (int e = 0; e < kE; ++e)
+                                        if (c0 + e < cg_hi) a[e][q] = __ldcg(part + (c0 + e) * kChainBlockM);
+                                }
+                            }
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                if (cb + q <= cl) {
+#pragma unroll
+                                    for (int e = 0; e < kE; ++e)
+                                        if (c0 + e < cg_hi) { g[e].x += a[e][q].x; g[e].y += a[e][q].y; g[e].z += a[e][q].z; g[e].w += a[e][q].w; }
+                                }
+                            }
+                            if (accs == 2) {
+#pragma unroll
+                                for (int q = 0; q < 4; ++q) {
+                                    const int cc = cb + q;
+                                    if (cc <= cl) {
+                                        const int sl = slot0 + ((cc == cf && cf_early) ? 1 : 0);
+                                        const float4* part = reinterpret_cast<const float4*>(p.partials + ((size_t)cc * kChainSlots + sl) * slot_floats) + up_off + etid;
+#pragma unroll
+                                        for (int e = 0; e < kE; ++e)
+                                            if (c0 + e < cg_hi) a[e][q] = __ldcg(part + (c0 + e) * kChainBlockM);
+                                    }
+                                }
+#pragma unroll
+                                for (int q = 0; q < 4; ++q) {
+                                    if (cb + q <= cl) {
+#pragma unroll
+                                        for (int e = 0; e < kE; ++e)
+                                            if (c0 + e < cg_hi) { u[e].x += a[e][q].x; u[e].y += a[e][q].y; u[e].z += a[e][q].z; u[e].w += a[e][q].w; }
+                                    }
+                                }
+                            }
+                        }
+#pragma unroll
+                        for (int e = 0; e < kE; ++e) {
+                            if (c0 + e >= cg_hi) break;
+                            const float gf[4] = {g[e].x, g[e].y, g[e].z, g[e].w}, uf[4] = {u[e].x, u[e].y, u[e].z, u[e].w};
+#pragma unroll
+                            for (int k = 0; k < 4; ++k)
+                                stage_out[((c0 + e) * 4 + k) * kChainBlockM + etid] = __float2bfloat16_rn(P.gateup ? chain_silu(gf[k]) * uf[k] : gf[k]);
+                        }
+                    }
+                    asm volatile("bar.sync 2, 128;" ::: "memory");
+                    store_rows(tile0 + tile, cg_lo * 4, cg_hi * 4);
+                };
+
+                UnitCursor cur(sched, blockIdx.x);
+                WorkUnit wu;
+                while (!bars->abort && cur.next(wu)) {
+                    if (wu.slot < 0 && npend > 0) {
+                        for (int i = 0; i < npend; ++i) run_reduce(pend[i]);
+                        npend = 0;
+                        if (bars->abort) break;
+                    }
+                    if (!mbar_wait(&bars->tmem_full[buf], acc_ph)) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); break; }
+                    tc_fence_after();
+                    if (tr && etid == 0) tr[wu.slot < 0 ? 10 : 28] = global_timer_ns();
+                    const int n_local = (tile0 + wu.tile) * kChainBlockM + row;
+                    const bool n_ok = n_local < P.N;
+                    const uint32_t t0 = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(buf * buf_cols);
+                    if (wu.slot < 0) {
+                        for (int c0 = 0; c0 < p.T; c0 += 16) {
+                            uint32_t g[16], u[16];
+                            tmem_ld_32x32b_x16(t0 + (uint32_t)c0, g);
+                            if (P.gateup) tmem_ld_32x32b_x16(t0 + (uint32_t)(p.n_tile + c0), u);
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) {
+                                const float v = P.gateup ? chain_silu(__uint_as_float(g[j])) * __uint_as_float(u[j]) : __uint_as_float(g[j]);
+                                stage_out[(c0 + j) * kChainBlockM + row] = __float2bfloat16_rn(v);
+                            }
+                        }
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&bars->tmem_empty[buf]);
+                        asm volatile("bar.sync 2, 128;" ::: "memory");
+                        store_rows(tile0 + wu.tile, 0, p.T);
+                        if (tr && etid == 0) tr[11] = global_timer_ns();
+                    } else {
+                        uint4* mine = reinterpret_cast<uint4*>(p.partials + ((size_t)blockIdx.x * kChainSlots + slot0 + wu.slot) * slot_floats) + row;
+                        for (int a = 0; a < accs; ++a) {
+                            for (int c0 = 0; c0 < p.T; c0 += 16) {
+                                uint32_t g[16];
+                                tmem_ld_32x32b_x16(t0 + (uint32_t)(a * p.n_tile + c0), g);
+                                tmem_ld_wait();
+#pragma unroll
+                                for (int j = 0; j < 16; j += 4)
+                                    mine[(size_t)((a * p.n_tile + c0 + j) >> 2) * kChainBlockM] = make_uint4(g[j], g[j + 1], g[j + 2], g[j + 3]);
+                            }
+                        }
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&bars->tmem_empty[buf]);
+                        asm volatile("bar.sync 2, 128;" ::: "memory");
+                        if (etid == 0) {
+                            __threadfence();
+                            atomicAdd(&counters[wu.tile], 1);
+                            if (tr) tr[29] = global_timer_ns();
+                        }
+                        pend[npend++] = wu.tile;
+                    }
+                    if (++buf == 2) { buf = 0; acc_ph ^= 1; }
+                }
+                for (int i = 0; i < npend && !bars->abort; ++i) run_reduce(pend[i]);
+                // ---- this CTA's part of the segment's output is written: announce it to the next phase
+                if (pi + 1 < p.nphase) {
+                    // every path above ends with a barrier behind its last output store; the reader orders its TMA (async
+                    // proxy) reads behind its acquire of the epoch word with a proxy fence of its own
+                    if (tr && etid == 0) tr[26] = global_timer_ns();
+                    if (etid == 0 && !bars->abort) {
+                        __threadfence();
+                        atomicAdd(ctr + kChainEpochBase + pi * 2 + seg, 1);
+                    }
+                }
+                if (tr && etid == 0) tr[4 + pi * 8 + 4 + seg] = global_timer_ns();    // segment's output complete in this CTA
+            }
+        }
+    }
+
+    if (tr && threadIdx.x == 0) tr[2] = global_timer_ns();
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
+    }
+}
+
+// ----------------------------------------------------------------------------------------- host side
+static int chain_enabled() {
+    static int v = -1;
+    if (v < 0) { const char* e = getenv("AFLEX_FFN_CHAIN"); v = e ? atoi(e) : 1; }
+    return v;
+}
+
+// A phase whose tiles are all shared along K is one segment by default: cutting it in two halves puts two reductions
+// one behind the other in every CTA's epilogue, and on the W_o projection of the Qwen3-32B-shaped layer that costs more
+// (198.3 us per step) than the half-phase of overlap returns (195.4 us).  AFLEX_CHAIN_SPLIT=1 cuts (tuning).
+static int chain_split() {
+    static int v = -1;
+    if (v < 0) { const char* e = getenv("AFLEX_CHAIN_SPLIT"); v = e ? atoi(e) : 0; }
+    return v;
+}
+
+bool chain_supported(int T) { return chain_enabled() != 0 && T >= 1 && T <= kChainMaxRows; }
+
+static int chain_n_tile(int T) { return ((T < 16 ? 16 : T) + 15) / 16 * 16; }
+
+size_t chain_counter_ints() { return 2 * (size_t)kChainCounterInts + 64; }
+
+size_t chain_workspace_bytes(int T, int num_sms) {
+    return align256((size_t)num_sms * kChainSlots * 2 * chain_n_tile(T) * kChainBlockM * sizeof(float));
+}
+
+aflex_status chain_launch(aflex_ctx* ctx, const ChainStep* steps, int nsteps, int T, char* ws, size_t ws_bytes,
+                          cudaStream_t st, int* counters) {
+    if (nsteps < 1 || nsteps > kChainMaxPhases || !chain_supported(T))
+        return set_error(ctx, AFLEX_ERR_UNSUPPORTED, "gemm chain: %d steps at %d rows", nsteps, T);
+    ChainParams p;
+    ChainMaps maps;
+    p.T = T;
+    p.n_tile = chain_n_tile(T);
+    p.box = p.n_tile;
+    p.nphase = nsteps;
+    int cols = 32;
+    while (cols < 2 * 2 * p.n_tile) cols <<= 1;
+    p.tmem_cols = cols;
+    const int b_bytes = (p.n_tile * kChainBlockK * 2 + 1023) & ~1023;
+    const int stage_bytes = 2 * kChainTileBytes + 2 * b_bytes;
+    const int stage_out_bytes = p.n_tile * kChainBlockM * 2;
+    const int budget = kMaxDynamicSmem - 1024 - 1024 - stage_out_bytes - 256;
+    p.stages = budget / stage_bytes;
+    if (p.stages > kChainMaxStages) p.stages = kChainMaxStages;
+    { static int v = -1; if (v < 0) { const char* e = getenv("AFLEX_CHAIN_STAGES"); v = e ? atoi(e) : 0; } if (v >= 2 && v < p.stages) p.stages = v; }
+    if (p.stages < 2) return set_error(ctx, AFLEX_ERR_UNSUPPORTED, "gemm chain: no ring fits");
+    const size_t smem_bytes = (size_t)p.stages * stage_bytes + 1024 + stage_out_bytes + 1024 + 128;
+    const size_t need = chain_workspace_bytes(T, ctx->num_sms);
+    if (need > ws_bytes || ws == nullptr)
+        return set_error(ctx, AFLEX_ERR_WORKSPACE, "gemm chain: need %zu workspace bytes, have %zu", need, ws_bytes);
+    int base = 0;
+    const void* in = nullptr;
+    for (int i = 0; i < nsteps; ++i) {
+        const ChainStep& s = steps[i];
+        ChainPhase& P = p.ph[i];
+        P.gateup = s.w1 != nullptr;
+        P.N = s.N; P.K = s.K;
+        const int m_tiles = (s.N + kChainBlockM - 1) / kChainBlockM;
+        P.ksteps = P.gateup ? (s.K + kChainBlockK - 1) / kChainBlockK : (s.K + 2 * kChainBlockK - 1) / (2 * kChainBlockK);
+        // Segments: the remainder tiles (shared along K) first and the whole tiles second; when no CTA gets a whole
+        // tile, two halves - except in the last phase, whose output nobody in this kernel waits for.
+        const int grid = ctx->num_sms, whole = m_tiles / grid * grid, rem = m_tiles - whole;
+        if (whole > 0) { P.seg_tiles[0] = rem; P.seg_tiles[1] = whole; }
+        else if (i + 1 < nsteps && chain_split()) { P.seg_tiles[0] = (m_tiles + 1) / 2; P.seg_tiles[1] = m_tiles - P.seg_tiles[0]; }
+        else { P.seg_tiles[0] = m_tiles; P.seg_tiles[1] = 0; }
+        // K steps fed by the previous phase's segment 0 (its tile t is this phase's K columns [128 t, 128 t + 128))
+        if (i == 0) P.n_early = P.ksteps;
+        else {
+            const int e = (P.gateup ? 2 : 1) * p.ph[i - 1].seg_tiles[0];
+            P.n_early = e < P.ksteps ? e : P.ksteps;
+        }
+        P.counter_base = base;
+        base += m_tiles;
+        P.out = reinterpret_cast<__nv_bfloat16*>(s.out);
+        in = s.in;
+        if (!encode_tmap_2d_bf16(&maps.a0[i], s.w0, (uint64_t)s.N, (uint64_t)s.K, (uint64_t)s.K * 2, kChainBlockM, kChainBlockK, true) ||
+            !encode_tmap_2d_bf16(&maps.a1[i], P.gateup ? s.w1 : s.w0, (uint64_t)s.N, (uint64_t)s.K, (uint64_t)s.K * 2, kChainBlockM, kChainBlockK, true) ||
+            !encode_tmap_2d_bf16(&maps.b[i], in, (uint64_t)T, (uint64_t)s.K, (uint64_t)s.K * 2, (uint32_t)p.box, kChainBlockK, false))
+            return set_error(ctx, AFLEX_ERR_CUDA, "gemm chain: cuTensorMapEncodeTiled failed");
+    }
+    for (int i = nsteps; i < kChainMaxPhases; ++i) { p.ph[i] = p.ph[0]; maps.a0[i] = maps.a0[0]; maps.a1[i] = maps.a1[0]; maps.b[i] = maps.b[0]; }
+    p.partials = reinterpret_cast<float*>(ws);
+    if (base > kChainEpochBase) return set_error(ctx, AFLEX_ERR_UNSUPPORTED, "gemm chain: too many tiles");
+    p.counters = counters;
+    p.status = ctx->dev_status;
+    p.trace = ctx->trace ? ctx->trace + (size_t)(ctx->trace_slot++ % kTraceKernels) * kTraceStride : nullptr;
+
+    if (!ctx->chain_attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynamicSmem);
+        if (e != cudaSuccess) return check_cuda(ctx, e, "cudaFuncSetAttribute(gemm chain)");
+        ctx->chain_attr_set = true;
+    }
+    KernelScope scope(ctx, kKGemmChain, st);
+    return check_cuda(ctx, launch_pdl(gemm_chain_kernel, dim3((unsigned)ctx->num_sms), dim3(kChainThreads), smem_bytes, st, maps, p),
+                      "gemm_chain_kernel launch");
+}
+
+}  // namespace aflex

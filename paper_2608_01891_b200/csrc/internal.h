@@ -26,7 +26,7 @@ namespace aflex {
 enum KernelKind {
     kKAttnDecode = 0, kKLinearGemm, kKDownGemm, kKGateUpGemm, kKRouterLogits,
     kKMoeRoute, kKMoeGather, kKMoeGateUpGemm, kKMoeDownGemm, kKMoeCombine,
-    kKAddRmsNorm, kKQkvGemm, kKRopeAppend, kKAttnPrefill, kKKindCount
+    kKAddRmsNorm, kKQkvGemm, kKRopeAppend, kKAttnPrefill, kKGemmChain, kKKindCount
 };
 constexpr int kProfMaxSlots = 8192;
 struct ProfSlot { cudaEvent_t start, stop; int kind; };
@@ -43,6 +43,7 @@ struct aflex_ctx {
     int* counters_attn = nullptr; // per-(sequence, KV head) chunk arrival counters (zero between launches)
     int* counters_a = nullptr;    // per-tile arrival counters, attention-stream GEMMs (zero between launches)
     int* counters_f = nullptr;    // per-tile arrival counters, FFN-stream GEMMs
+    int* chain_counters = nullptr;   // arrival counters and epoch words of the GEMM chain kernel, double-buffered over launches
     cudaStream_t stream_a = nullptr, stream_f = nullptr;
     cudaEvent_t ev_entry = nullptr;
     cudaEvent_t ev_a[aflex::kMaxMicrobatches] = {};
@@ -52,6 +53,7 @@ struct aflex_ctx {
     bool attn_q_final = false;    // caller's promise (aflex_set_attn_q_final): q is never the output of the kernel just before
     bool attn_q_final_once = false;   // set by the layer chains for their own attention launch (q comes from the append kernel)
     bool gemm_attr_set[3] = {false, false, false};
+    bool chain_attr_set = false;
     bool attn_attr_set[2] = {false, false};
     bool prefill_attr_set[2] = {false, false};   // shared-memory limit raised for attn_prefill_kernel<64 / 128> on this device
     char err[512] = {0};
@@ -139,6 +141,19 @@ aflex_status linear_launch(aflex_ctx* ctx, const void* x, const void* w, int T, 
 size_t gateup_workspace_bytes(int T, int H, int I, int num_sms);
 aflex_status gateup_launch(aflex_ctx* ctx, const void* x, const void* w_gate, const void* w_up, int T, int H, int I,
                            void* h, char* ws, size_t ws_bytes, cudaStream_t st, int* counters);
+
+// ---- chain of dependent decode-batch GEMMs as one persistent kernel (gemm_chain.cu)
+// Step i computes out = in . w0^T (w1 == nullptr) or out = silu(in . w0^T) .* (in . w1^T); step i + 1 reads
+// step i's output.  in bf16 [T][K], w bf16 [N][K], out bf16 [T][N].  T <= kChainMaxRows.
+constexpr int kChainMaxRows = 64;
+struct ChainStep { const void* in; const void* w0; const void* w1; int K, N; void* out; };
+bool chain_supported(int T);
+size_t chain_workspace_bytes(int T, int num_sms);
+// `counters`: chain_counter_ints() zeroed ints reserved for the chain launches of one stream (double-buffered over
+// launches by a generation word the kernel itself keeps there: a launch counts in one half and zeroes the other).
+size_t chain_counter_ints();
+aflex_status chain_launch(aflex_ctx* ctx, const ChainStep* steps, int nsteps, int T, char* ws, size_t ws_bytes,
+                          cudaStream_t st, int* counters);
 
 // Grouped (per-expert) variants over permuted rows.  `offsets` is a device array [E+1]
 // (row segment of expert e = [offsets[e], offsets[e+1])); rows_max bounds any segment.
