@@ -52,6 +52,8 @@ constexpr int kBlockK = 64;    // bf16 elements per 128-byte swizzled row
 constexpr int kGemmThreads = 192;
 constexpr int kMaxStages = 8;
 constexpr int kMaxExperts = 64;
+constexpr int kStageTokens = 32;                             // token rows staged per round of the epilogue
+constexpr int kStageOutBytes = kStageTokens * 2 * kBlockM * 4;   // worst case: 256 fp32 features per token row
 
 struct GemmParams {
     int T;            // token rows of x (all experts' rows together for the grouped form)
@@ -163,6 +165,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
     constexpr int kABytes = kBlockM * kBlockK * 2;           // 16 KB
     const int stage_bytes = kNumA * kABytes + ((p.n_tile * kBlockK * 2 + 1023) & ~1023);
     GemmBarriers* bars = reinterpret_cast<GemmBarriers*>(smem + (size_t)p.stages * stage_bytes);
+    // Epilogue staging: kStageTokens token rows of the output tile, [token][tile's weight rows] in the output type, so
+    // that results leave the SM as 16-byte stores of consecutive features instead of one 2-byte store per value.
+    uint8_t* stage_out = smem + (size_t)p.stages * stage_bytes + ((sizeof(GemmBarriers) + 127) & ~(size_t)127);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -311,6 +316,33 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
         WorkUnit wu;
         pdl_wait();   // nothing is written before the predecessor grid has completed
 
+        // Geometry of the output tile in the staging buffer and in memory.
+        constexpr int kTileCols = (MODE == kLinear2) ? 2 * kBlockM : kBlockM;    // weight rows (output features) per tile
+        const int es = p.out_f32 ? 4 : 2;                                        // bytes per output element
+        const int per16 = 16 / es;                                               // elements per 16-byte store
+        const int cpr = kTileCols / per16;                                       // 16-byte pieces per staged token row
+        auto stage_put = [&](int tl, int col, float v) {                         // token row tl of the round, feature col of the tile
+            if (p.out_f32) reinterpret_cast<float*>(stage_out)[tl * kTileCols + col] = v;
+            else reinterpret_cast<__nv_bfloat16*>(stage_out)[tl * kTileCols + col] = __float2bfloat16_rn(v);
+        };
+        // Staged token rows [0, ntok) -> output rows t0 + .. (bounded by t_limit), features 128 * .. of the tile; the
+        // barriers order the staging writes before the reads and free the buffer for its next user.
+        auto stage_flush = [&](const TileCoord& c, int t0, int ntok) {
+            asm volatile("bar.sync 2, 128;" ::: "memory");
+            const int n0 = c.m_tile * p.tile_rows;
+            for (int i = etid; i < ntok * cpr; i += 128) {
+                const int tl = i / cpr, part = i - tl * cpr;
+                const int t = t0 + tl, n = n0 + part * per16;
+                if (t < c.out_row_limit && n < p.N) {
+                    const uint4 v = *reinterpret_cast<const uint4*>(stage_out + ((size_t)tl * kTileCols + part * per16) * es);
+                    uint8_t* dst = p.out_f32 ? reinterpret_cast<uint8_t*>(p.out_f32 + (size_t)t * p.N + n)
+                                             : reinterpret_cast<uint8_t*>(p.out_bf16 + (size_t)t * p.N + n);
+                    *reinterpret_cast<uint4*>(dst) = v;
+                }
+            }
+            asm volatile("bar.sync 2, 128;" ::: "memory");
+        };
+
         // A shared tile is finished by its contributors together (all of them but a last one that has another
         // shared tile to finish): once every piece is published (arrival counter == number of pieces; bounded
         // spin), reducer i sums the i-th slice of the tile over all pieces, in CTA order, and writes that slice
@@ -341,71 +373,69 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
             }
             asm volatile("bar.sync 2, 128;" ::: "memory");
             if (bars->abort) return;
-            __threadfence();
             const bool cf_early = sched.share_begin(cf) < x0;
-            const int n4 = ((pd.c.b_rows + 15) / 16) * 4 * kBlockM;     // float4 slots of one accumulator that were stored
-            const int lo = (int)((long long)n4 * me / nred), hi = (int)((long long)n4 * (me + 1) / nred);
-            const int up_off = (p.n_tile >> 2) * kBlockM;               // float4 offset of the "up" accumulator
-            // kElems float4 per thread and round, all pieces' loads of a round in flight together (the loop is
-            // bound by L2 latency, not bandwidth)
+            // The parked accumulators are [column group of 4 tokens][128 rows] float4.  Reducer `me` takes whole column
+            // groups, thread = accumulator row; kElems groups per round with every piece's loads of a round in flight
+            // together (the loop is bound by L2 latency, not bandwidth); kStageTokens tokens are staged per flush.
+            const int ncg = ((pd.c.b_rows + 15) / 16) * 4;
+            const int cg_lo = ncg * me / nred, cg_hi = ncg * (me + 1) / nred;
+            const int up_off = (p.n_tile >> 2) * kBlockM;               // float4 offset of the second accumulator
             constexpr int kElems = (kAccs == 1) ? 4 : 2;
-            for (int i0 = lo + etid; i0 < hi; i0 += kElems * 128) {
-                float4 g[kElems], u[kElems];
+            constexpr int kCgPerFlush = kStageTokens / 4;
+            for (int f0 = cg_lo; f0 < cg_hi; f0 += kCgPerFlush) {
+                const int f1 = min(cg_hi, f0 + kCgPerFlush);
+                for (int c0 = f0; c0 < f1; c0 += kElems) {
+                    float4 g[kElems], u[kElems];
 #pragma unroll
-                for (int e = 0; e < kElems; ++e) g[e] = u[e] = make_float4(0.f, 0.f, 0.f, 0.f);
-                for (int cb = cf; cb <= cl; cb += 4) {
-                    float4 a[kElems][4], b[kElems][4];
+                    for (int e = 0; e < kElems; ++e) g[e] = u[e] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    for (int cb = cf; cb <= cl; cb += 4) {
+                        float4 a[kElems][4], b[kElems][4];
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const int cc = cb + q;
-                        if (cc <= cl) {
-                            // only the first contributor's share can begin before the tile: then its piece is a
-                            // later unit of that CTA (slot 1); every other piece is a first unit (slot 0)
-                            const int sl = (cc == cf && cf_early) ? 1 : 0;
-                            const float4* part = reinterpret_cast<const float4*>(p.partials + ((size_t)cc * 2 + sl) * slot_floats);
+                        for (int q = 0; q < 4; ++q) {
+                            const int cc = cb + q;
+                            if (cc <= cl) {
+                                // only the first contributor's share can begin before the tile: then its piece is a
+                                // later unit of that CTA (slot 1); every other piece is a first unit (slot 0)
+                                const int sl = (cc == cf && cf_early) ? 1 : 0;
+                                const float4* part = reinterpret_cast<const float4*>(p.partials + ((size_t)cc * 2 + sl) * slot_floats) + etid;
 #pragma unroll
-                            for (int e = 0; e < kElems; ++e) {
-                                if (i0 + e * 128 < hi) {
-                                    a[e][q] = __ldcg(part + i0 + e * 128);
-                                    if (kAccs == 2) b[e][q] = __ldcg(part + up_off + i0 + e * 128);
+                                for (int e = 0; e < kElems; ++e) {
+                                    if (c0 + e < f1) {
+                                        a[e][q] = __ldcg(part + (size_t)(c0 + e) * kBlockM);
+                                        if (kAccs == 2) b[e][q] = __ldcg(part + up_off + (size_t)(c0 + e) * kBlockM);
+                                    }
+                                }
+                            }
+                        }
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            if (cb + q <= cl) {
+#pragma unroll
+                                for (int e = 0; e < kElems; ++e) {
+                                    if (c0 + e < f1) {
+                                        g[e].x += a[e][q].x; g[e].y += a[e][q].y; g[e].z += a[e][q].z; g[e].w += a[e][q].w;
+                                        if (kAccs == 2) { u[e].x += b[e][q].x; u[e].y += b[e][q].y; u[e].z += b[e][q].z; u[e].w += b[e][q].w; }
+                                    }
                                 }
                             }
                         }
                     }
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        if (cb + q <= cl) {
+                    for (int e = 0; e < kElems; ++e) {
+                        if (c0 + e >= f1) break;
+                        const float gf[4] = {g[e].x, g[e].y, g[e].z, g[e].w}, uf[4] = {u[e].x, u[e].y, u[e].z, u[e].w};
 #pragma unroll
-                            for (int e = 0; e < kElems; ++e) {
-                                if (i0 + e * 128 < hi) {
-                                    g[e].x += a[e][q].x; g[e].y += a[e][q].y; g[e].z += a[e][q].z; g[e].w += a[e][q].w;
-                                    if (kAccs == 2) { u[e].x += b[e][q].x; u[e].y += b[e][q].y; u[e].z += b[e][q].z; u[e].w += b[e][q].w; }
-                                }
+                        for (int k = 0; k < 4; ++k) {
+                            const int tl = (c0 + e - f0) * 4 + k;
+                            if (MODE == kGateUp) stage_put(tl, etid, silu_f32(gf[k]) * uf[k]);
+                            else {
+                                stage_put(tl, etid, gf[k]);
+                                if (MODE == kLinear2) stage_put(tl, etid + kBlockM, uf[k]);
                             }
                         }
                     }
                 }
-#pragma unroll
-                for (int e = 0; e < kElems; ++e) {
-                    const int idx = i0 + e * 128;
-                    if (idx >= hi) break;
-                    const float gf[4] = {g[e].x, g[e].y, g[e].z, g[e].w}, uf[4] = {u[e].x, u[e].y, u[e].z, u[e].w};
-                    const int r = idx & (kBlockM - 1), cg = idx / kBlockM;
-                    const int nl = pd.c.m_tile * p.tile_rows + r;
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        const int t = pd.c.b_row0 + cg * 4 + k;
-                        if (nl < p.N && t < pd.c.out_row_limit) {
-                            if (MODE == kGateUp) p.out_bf16[(size_t)t * p.N + nl] = __float2bfloat16_rn(silu_f32(gf[k]) * uf[k]);
-                            else if (MODE == kLinear2) {
-                                p.out_bf16[(size_t)t * p.N + nl] = __float2bfloat16_rn(gf[k]);
-                                if (nl + kBlockM < p.N) p.out_bf16[(size_t)t * p.N + nl + kBlockM] = __float2bfloat16_rn(uf[k]);
-                            }
-                            else if (p.out_f32) p.out_f32[(size_t)t * p.N + nl] = gf[k];
-                            else p.out_bf16[(size_t)t * p.N + nl] = __float2bfloat16_rn(gf[k]);
-                        }
-                    }
-                }
+                stage_flush(pd.c, pd.c.b_row0 + f0 * 4, (f1 - f0) * 4);
             }
             asm volatile("bar.sync 2, 128;" ::: "memory");
             if (etid == 0) {
@@ -432,51 +462,35 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
             const bool n_ok = n_local < p.N;
             const uint32_t t0 = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(buf * acc_cols);
             if (wu.slot < 0) {
-                // ---- whole K range in this CTA: epilogue straight from TMEM
-                for (int c0 = 0; c0 < c.b_rows; c0 += 16) {
-                    uint32_t g[16];
-                    tmem_ld_32x32b_x16(t0 + (uint32_t)c0, g);
-                    if (MODE == kGateUp) {
-                        uint32_t u[16];
-                        tmem_ld_32x32b_x16(t0 + (uint32_t)(p.n_tile + c0), u);
-                        tmem_ld_wait();
+                // ---- whole K range in this CTA: epilogue straight from TMEM, kStageTokens token columns per round
+                for (int tc = 0; tc < c.b_rows; tc += kStageTokens) {
+                    const int ntok = min(kStageTokens, c.b_rows - tc);
+                    for (int c0 = 0; c0 < ntok; c0 += 16) {
+                        uint32_t g[16];
+                        tmem_ld_32x32b_x16(t0 + (uint32_t)(tc + c0), g);
+                        if (MODE != kLinear) {
+                            uint32_t u[16];
+                            tmem_ld_32x32b_x16(t0 + (uint32_t)(p.n_tile + tc + c0), u);
+                            tmem_ld_wait();
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            const int t = c.b_row0 + c0 + j;
-                            if (n_ok && t < c.out_row_limit) {
-                                const float hv = silu_f32(__uint_as_float(g[j])) * __uint_as_float(u[j]);
-                                p.out_bf16[(size_t)t * p.N + n_local] = __float2bfloat16_rn(hv);
+                            for (int j = 0; j < 16; ++j) {
+                                if (MODE == kGateUp) stage_put(c0 + j, row, silu_f32(__uint_as_float(g[j])) * __uint_as_float(u[j]));
+                                else { stage_put(c0 + j, row, __uint_as_float(g[j])); stage_put(c0 + j, row + kBlockM, __uint_as_float(u[j])); }
                             }
-                        }
-                    } else if (MODE == kLinear2) {
-                        uint32_t u[16];
-                        tmem_ld_32x32b_x16(t0 + (uint32_t)(p.n_tile + c0), u);
-                        tmem_ld_wait();
-                        const bool n2_ok = n_local + kBlockM < p.N;        // the tile's second 128 weight rows
+                        } else {
+                            tmem_ld_wait();
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            const int t = c.b_row0 + c0 + j;
-                            if (t < c.out_row_limit) {
-                                if (n_ok) p.out_bf16[(size_t)t * p.N + n_local] = __float2bfloat16_rn(__uint_as_float(g[j]));
-                                if (n2_ok) p.out_bf16[(size_t)t * p.N + n_local + kBlockM] = __float2bfloat16_rn(__uint_as_float(u[j]));
-                            }
-                        }
-                    } else {
-                        tmem_ld_wait();
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            const int t = c.b_row0 + c0 + j;
-                            if (n_ok && t < c.out_row_limit) {
-                                const float v = __uint_as_float(g[j]);
-                                if (p.out_f32) p.out_f32[(size_t)t * p.N + n_local] = v;
-                                else p.out_bf16[(size_t)t * p.N + n_local] = __float2bfloat16_rn(v);
-                            }
+                            for (int j = 0; j < 16; ++j) stage_put(c0 + j, row, __uint_as_float(g[j]));
                         }
                     }
+                    if (tc + kStageTokens >= c.b_rows) {
+                        // the accumulator has been read in full: hand the TMEM buffer back before the stores
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&bars->tmem_empty[buf]);
+                    }
+                    stage_flush(c, c.b_row0 + tc, ntok);
                 }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&bars->tmem_empty[buf]);
             } else {
                 // ---- partial K range: park the fp32 accumulator as [column group of 4][row] float4 (a warp
                 //      stores / loads 512 contiguous bytes per instruction); the last arriver finishes the tile
@@ -626,12 +640,12 @@ static bool make_config(int mode, int T, int N, int K, int rows_max, int E, int 
     if (nostream < 0) { const char* e = getenv("AFLEX_GEMM_NOSTREAMK"); nostream = e ? atoi(e) : 0; }
     p.streamk = nostream ? 0 : (tiles_hi < 8LL * num_sms && tiles_hi <= kStreamKMaxTiles && (p.n_tile <= 128 || tiles_hi < 2LL * num_sms)) ? 1 : 0;
     const int cap = (p.streamk && p.n_tile <= 64 && mode != kLinear2) ? streaming_smem_budget() : kMaxDynamicSmem;
-    const int budget = cap - 1024 /*alignment slack*/ - (int)sizeof(GemmBarriers) - 256;
+    const int budget = cap - 1024 /*alignment slack*/ - (int)sizeof(GemmBarriers) - 256 - kStageOutBytes;
     int stages = budget / stage_bytes;
     if (stages > kMaxStages) stages = kMaxStages;
     if (stages < 2) stages = 2;
     p.stages = stages;
-    cfg->smem_bytes = (size_t)stages * stage_bytes + sizeof(GemmBarriers) + 1024 + 128;
+    cfg->smem_bytes = (size_t)stages * stage_bytes + sizeof(GemmBarriers) + 1024 + 256 + kStageOutBytes;
     if (cfg->smem_bytes > (size_t)kMaxDynamicSmem) return false;
     long long units = tiles_hi * p.kblocks;
     cfg->grid = (int)(units < num_sms ? units : num_sms);
