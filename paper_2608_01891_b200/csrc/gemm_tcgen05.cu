@@ -53,7 +53,6 @@ constexpr int kGemmThreads = 192;
 constexpr int kMaxStages = 8;
 constexpr int kMaxExperts = 64;
 constexpr int kStageTokens = 32;                             // token rows staged per round of the epilogue
-constexpr int kStageOutBytes = kStageTokens * 2 * kBlockM * 4;   // worst case: 256 fp32 features per token row
 
 struct GemmParams {
     int T;            // token rows of x (all experts' rows together for the grouped form)
@@ -583,7 +582,7 @@ static int linear_mode(int T, int N, int K) {
     return (n_tile >= 64 && n_tile <= 128 && (long long)N * K >= (64LL << 20)) ? kLinear2 : kLinear;
 }
 
-static bool make_config(int mode, int T, int N, int K, int rows_max, int E, int num_sms, GemmConfig* cfg) {
+static bool make_config(int mode, int T, int N, int K, int rows_max, int E, int num_sms, GemmConfig* cfg, bool out_f32 = false) {
     GemmParams& p = cfg->p;
     p.T = T; p.N = N; p.K = K;
     p.n_tile = pick_n_tile(rows_max);
@@ -639,13 +638,16 @@ static bool make_config(int mode, int T, int N, int K, int rows_max, int E, int 
     static int nostream = -1;   // AFLEX_GEMM_NOSTREAMK=1: whole tiles only (measurement of per-SM streaming rates)
     if (nostream < 0) { const char* e = getenv("AFLEX_GEMM_NOSTREAMK"); nostream = e ? atoi(e) : 0; }
     p.streamk = nostream ? 0 : (tiles_hi < 8LL * num_sms && tiles_hi <= kStreamKMaxTiles && (p.n_tile <= 128 || tiles_hi < 2LL * num_sms)) ? 1 : 0;
-    const int cap = (p.streamk && p.n_tile <= 64 && mode != kLinear2) ? streaming_smem_budget() : kMaxDynamicSmem;
-    const int budget = cap - 1024 /*alignment slack*/ - (int)sizeof(GemmBarriers) - 256 - kStageOutBytes;
+    // epilogue staging: kStageTokens token rows of the tile in the output type
+    const int stage_out_bytes = kStageTokens * (mode == kLinear2 ? 2 : 1) * kBlockM * (out_f32 ? 4 : 2);
+    int cap = (p.streamk && p.n_tile <= 64 && mode != kLinear2) ? streaming_smem_budget() + stage_out_bytes : kMaxDynamicSmem;
+    if (cap > kMaxDynamicSmem) cap = kMaxDynamicSmem;
+    const int budget = cap - 1024 /*alignment slack*/ - (int)sizeof(GemmBarriers) - 256 - stage_out_bytes;
     int stages = budget / stage_bytes;
     if (stages > kMaxStages) stages = kMaxStages;
     if (stages < 2) stages = 2;
     p.stages = stages;
-    cfg->smem_bytes = (size_t)stages * stage_bytes + sizeof(GemmBarriers) + 1024 + 256 + kStageOutBytes;
+    cfg->smem_bytes = (size_t)stages * stage_bytes + sizeof(GemmBarriers) + 1024 + 256 + stage_out_bytes;
     if (cfg->smem_bytes > (size_t)kMaxDynamicSmem) return false;
     long long units = tiles_hi * p.kblocks;
     cfg->grid = (int)(units < num_sms ? units : num_sms);
@@ -755,7 +757,7 @@ aflex_status gateup_launch(aflex_ctx* ctx, const void* x, const void* w_gate, co
 
 size_t grouped_workspace_bytes(int mode_gateup, int rows_total, int rows_max, int K, int N, int E, int num_sms) {
     GemmConfig cfg;
-    if (!make_config(mode_gateup ? kGateUp : kLinear, rows_total, N, K, rows_max, E, num_sms, &cfg)) return 0;
+    if (!make_config(mode_gateup ? kGateUp : kLinear, rows_total, N, K, rows_max, E, num_sms, &cfg, !mode_gateup)) return 0;
     return cfg.partial_bytes;
 }
 
@@ -786,7 +788,7 @@ aflex_status grouped_linear_launch(aflex_ctx* ctx, const void* hp, const void* w
                                    size_t ws_bytes, cudaStream_t st, int* counters) {
     if (E > kMaxExperts) return set_error(ctx, AFLEX_ERR_UNSUPPORTED, "num_experts > %d", kMaxExperts);
     GemmConfig cfg;
-    if (!make_config(kLinear, rows_total, N, K, rows_max, E, ctx->num_sms, &cfg))
+    if (!make_config(kLinear, rows_total, N, K, rows_max, E, ctx->num_sms, &cfg, true))
         return set_error(ctx, AFLEX_ERR_UNSUPPORTED, "grouped linear: no tile configuration fits");
     GemmParams& p = cfg.p;
     p.offsets = offsets;
