@@ -277,8 +277,8 @@ aflex_status aflex_create(aflex_ctx** out, int device, size_t workspace_bytes) {
     if (e == cudaSuccess) e = cudaMalloc(&ctx->ws, ctx->ws_bytes);
     if (e == cudaSuccess) e = cudaMalloc(&ctx->dev_status, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(ctx->dev_status, 0, sizeof(int));
-    if (e == cudaSuccess) e = cudaMalloc(&ctx->counters_attn, (kAttnCounterCap + 2) * sizeof(int));
-    if (e == cudaSuccess) e = cudaMemset(ctx->counters_attn, 0, (kAttnCounterCap + 2) * sizeof(int));
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->counters_attn, (kAttnCounterCap + 16) * sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(ctx->counters_attn, 0, (kAttnCounterCap + 16) * sizeof(int));
     if (e == cudaSuccess) e = cudaMalloc(&ctx->counters_a, 2 * kStreamKMaxTiles * sizeof(int));
     if (e == cudaSuccess) e = cudaMalloc(&ctx->counters_f, 2 * kStreamKMaxTiles * sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(ctx->counters_a, 0, 2 * kStreamKMaxTiles * sizeof(int));
@@ -351,7 +351,7 @@ aflex_status aflex_get_device_status(aflex_ctx* ctx, void* stream) {
     const int v = *ctx->host_status;
     if (v != 0) {
         // a kernel that gave up may have left arrival counters half-way: restore the all-zero state
-        cudaMemsetAsync(ctx->counters_attn, 0, (kAttnCounterCap + 2) * sizeof(int), st);
+        cudaMemsetAsync(ctx->counters_attn, 0, (kAttnCounterCap + 16) * sizeof(int), st);
         cudaMemsetAsync(ctx->counters_a, 0, 2 * kStreamKMaxTiles * sizeof(int), st);
         cudaMemsetAsync(ctx->counters_f, 0, 2 * kStreamKMaxTiles * sizeof(int), st);
         cudaMemsetAsync(ctx->chain_counters, 0, chain_counter_ints() * sizeof(int), st);

@@ -64,7 +64,8 @@ struct AttnParams {
     __nv_bfloat16* out;    // [B][Hq][D]
     float* lse;            // [B][Hq] or nullptr
     int* counters;         // [B][Hkv] piece-arrival counters, zero on entry and on exit
-    int* ticket;           // [2]: next dynamic chunk, CTAs finished; zero on entry and on exit (unused if dyn_pct == 0)
+    int* ticket;           // [2]: next dynamic chunk, CTAs finished; zero on entry and on exit, not shared with the launches
+                           // next to this one in the stream (unused if dyn_pct == 0)
     int dyn_pct;           // percent of the unit list handed out dynamically (0 = static shares only)
     int dyn_chunks;        // target number of dynamic chunks per CTA
     int kv_policy;         // 0: evict-first KV loads, 1: normal priority (tuning)
@@ -184,7 +185,8 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                    const AttnParams p) {
     constexpr int kHalves = D / 64;                 // 128-byte column blocks per row
     constexpr int kPageBytes = kPage * D * 2;       // one page of K (or V) for one KV head
-    constexpr int kStageBytes = 2 * kPagesPerStage * kPageBytes;
+    constexpr int kQBytes = 8 * D * 2;              // the (at most 8) query heads of one group: the block behind the pages
+    constexpr int kStageBytes = 2 * kPagesPerStage * kPageBytes + kQBytes;
     constexpr int kOpsPerStage = 2 * kPagesPerStage * kHalves;
     constexpr int kKSteps = D / 16;
 
@@ -306,11 +308,11 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         }
         // KV loads do not wait for the grid dependency: the only kernel of this library that writes the
         // cache (the K/V append) does not release its dependents early, so whatever precedes this launch
-        // in the stream has left the cache final.  The ticket, like everything else in global memory that
-        // an earlier attention launch may still be using, is touched only after pdl_wait.
+        // in the stream has left the cache final.  Neither do the chunk tickets: consecutive launches use
+        // different ticket words (four pairs in rotation, picked by the host), and a launch cannot start
+        // before the launch four back has completed, its words reset.
         bool waited = false;
         auto claim = [&]() {
-            if (!waited) { pdl_wait(); waited = true; }
             if (lane == 0) next_ticket = atomicAdd(&p.ticket[0], 1);
             next_ticket = __shfl_sync(0xffffffffu, next_ticket, 0);
         };
@@ -319,7 +321,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             // claim the chunk after this range while the range streams (the round trip hides behind it);
             // in the first range only once the ring has been filled
             bool claimed = sp.n2 == 0;
-            if (!claimed && waited) { claim(); claimed = true; }
+            if (!claimed && !first_range) { claim(); claimed = true; }
             int issued = 0;
             if (x1 > x0) {
                 AttnRange rg;
@@ -335,8 +337,11 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                     ++r;
                 }
                 int pid = wk.done() ? 0 : (first_range ? pid0 : page_id(wk));
+                int piece_b = -1, piece_g = -1;           // item of the piece being loaded (a new range starts a new piece)
                 while (!wk.done()) {
-                    const int g = wk.g, u = wk.u - wk.cost, len = wk.len;
+                    const int g = wk.g, u = wk.u - wk.cost, len = wk.len, b_now = wk.b;
+                    const bool piece_start = (b_now != piece_b) || (g != piece_g);
+                    piece_b = b_now; piece_g = g;
                     wk.advance(1);
                     wk.skip_empty();
                     const int pid_next = wk.done() ? 0 : page_id(wk);   // one unit ahead of the ring
@@ -350,7 +355,8 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                         break;
                     }
                     const int np = min(kPagesPerStage, (len - u * kUnitTokens + kPage - 1) / kPage);
-                    if (lane == 0) mbar_expect_tx(&sh->full[s], (uint32_t)(np * 2 * kPageBytes));
+                    const uint32_t q_bytes = piece_start ? (uint32_t)(p.G * D * 2) : 0u;
+                    if (lane == 0) mbar_expect_tx(&sh->full[s], (uint32_t)(np * 2 * kPageBytes) + q_bytes);
                     __syncwarp();
                     if (op_lane && pg < np) {
                         int id = pid;
@@ -358,6 +364,15 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                         uint8_t* dst = smem + s * kStageBytes + kv * (kPagesPerStage * kPageBytes) + pg * kPageBytes + hf * (kPage * 128);
                         const int row = (id * p.Hkv + g) * kPage;
                         tma_load_2d_hint(dst, kv ? &tmap_v : &tmap_k, hf * 64, row, &sh->full[s], pol_kv);
+                    }
+                    if (piece_start) {
+                        // The piece's queries (the G heads of the group are contiguous in q) travel with its first unit.
+                        // q may be the output of the kernel just before this one: unless the launcher knows better, the
+                        // first copy waits for the grid dependency (the KV loads above are already in flight).
+                        if (!p.q_final && !waited) { pdl_wait(); waited = true; }
+                        if (lane == 0)
+                            bulk_load_1d(smem + s * kStageBytes + 2 * kPagesPerStage * kPageBytes,
+                                         p.q + ((size_t)b_now * p.Hq + (size_t)g * p.G) * D, q_bytes, &sh->full[s]);
                     }
                     pid = pid_next;
                     if (++s == kAttnStages) { s = 0; ph ^= 1; }
@@ -378,7 +393,6 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             mbar_arrive(&sh->rng_ready[r % kRangeRing]);
             if (sp.n2 > 0) {
                 // last CTA out resets the ticket counters (every CTA has made its final claim by now)
-                if (!waited) pdl_wait();
                 __threadfence();
                 if (atomicAdd(&p.ticket[1], 1) == (int)gridDim.x - 1) { p.ticket[0] = 0; p.ticket[1] = 0; }
             }
@@ -390,7 +404,6 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         // does not release early, or the caller's promise) these warps wait for the grid dependency before
         // their first q load; the ring fills meanwhile.  They never write to global memory: a finished
         // piece's state goes to the epilogue warp through the piece's last stage buffer.
-        if (!p.q_final) pdl_wait();
         const int mi = lane >> 3, r8 = lane & 7;
         int s = 0;
         uint32_t ph = 0;
@@ -419,20 +432,9 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             wk.advance(nv);
             if (n <= 0) continue;                                            // only empty positions: no piece
 
-            // Q^T as the MMA's B operand: lane holds head (lane/4), d = 16*ks + 2*(lane%4) + {0,1} (+8)
+            // Q^T as the MMA's B operand: lane holds head (lane/4), d = 16*ks + 2*(lane%4) + {0,1} (+8); read from the
+            // piece's first stage, where the producer put the group's queries
             uint32_t qb[kKSteps][2];
-            {
-                const int h = lane >> 2;
-                const __nv_bfloat16* qrow = p.q + ((size_t)b * p.Hq + (size_t)g * p.G + (h < p.G ? h : 0)) * D;
-#pragma unroll
-                for (int ks = 0; ks < kKSteps; ++ks) {
-                    const int d0 = ks * 16 + 2 * (lane & 3);
-                    const uint32_t v0 = *reinterpret_cast<const uint32_t*>(qrow + d0);
-                    const uint32_t v1 = *reinterpret_cast<const uint32_t*>(qrow + d0 + 8);
-                    qb[ks][0] = h < p.G ? v0 : 0u;
-                    qb[ks][1] = h < p.G ? v1 : 0u;
-                }
-            }
             float o[kKSteps][4];
 #pragma unroll
             for (int i = 0; i < kKSteps; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
@@ -447,6 +449,18 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                     break;
                 }
                 if (tr && threadIdx.x == 0 && tr[3] == 0) tr[3] = global_timer_ns();     // first data landed
+                if (u == u0) {
+                    const int h = lane >> 2;
+                    const uint8_t* qs = smem + s * kStageBytes + 2 * kPagesPerStage * kPageBytes + (h < p.G ? h : 0) * (D * 2);
+#pragma unroll
+                    for (int ks = 0; ks < kKSteps; ++ks) {
+                        const int d0 = ks * 16 + 2 * (lane & 3);
+                        const uint32_t v0 = *reinterpret_cast<const uint32_t*>(qs + d0 * 2);
+                        const uint32_t v1 = *reinterpret_cast<const uint32_t*>(qs + (d0 + 8) * 2);
+                        qb[ks][0] = h < p.G ? v0 : 0u;
+                        qb[ks][1] = h < p.G ? v1 : 0u;
+                    }
+                }
                 const int nvalid = min(kPage, len - (u * kUnitTokens + warp * kPage));   // tokens of this warp's page
                 if (nvalid > 0) {
                     const uint32_t kpage = smem_u32(smem + s * kStageBytes + warp * kPageBytes);
@@ -826,7 +840,7 @@ static aflex_status attn_launch_t(aflex_ctx* ctx, const aflex_attn_desc* d, cons
     p.num_pages = kv->num_pages;
     const float scale = d->sm_scale != 0.f ? d->sm_scale : 1.0f / sqrtf((float)D);
     p.scale_log2 = scale * 1.4426950408889634f;
-    p.ticket = ctx->counters_attn + kAttnCounterCap;      // two ints past the per-item counters
+    p.ticket = ctx->counters_attn + kAttnCounterCap + 2 * (ctx->attn_launch_seq++ & 3u);   // past the per-item counters
     p.dyn_pct = attn_dyn_pct();
     p.dyn_chunks = attn_dyn_chunks();
     p.piece_cost = attn_piece_cost();
@@ -846,7 +860,7 @@ static aflex_status attn_launch_t(aflex_ctx* ctx, const aflex_attn_desc* d, cons
         !encode_tmap_2d_bf16(&tv, kv->v_cache, rows, D, (uint64_t)D * 2, kPage, 64, true))
         return set_error(ctx, AFLEX_ERR_CUDA, "attention: cuTensorMapEncodeTiled failed");
 
-    constexpr int kStageBytes = 2 * kPagesPerStage * kPage * D * 2;
+    constexpr int kStageBytes = 2 * kPagesPerStage * kPage * D * 2 + 8 * D * 2;
     const size_t smem = (size_t)kAttnStages * kStageBytes + sizeof(AttnShared) + 1024;
     const int ti = (D == 128) ? 1 : 0;
     if (!ctx->attn_attr_set[ti]) {
@@ -954,7 +968,7 @@ static aflex_status attn_static_launch(StaticDeviceState& stt, const aflex_attn_
     if (!encode_tmap_2d_bf16(&tk, kv->k_cache, rows, D, (uint64_t)D * 2, kPage, 64, true) ||
         !encode_tmap_2d_bf16(&tv, kv->v_cache, rows, D, (uint64_t)D * 2, kPage, 64, true))
         return AFLEX_ERR_CUDA;
-    constexpr int kStageBytes = 2 * kPagesPerStage * kPage * D * 2;
+    constexpr int kStageBytes = 2 * kPagesPerStage * kPage * D * 2 + 8 * D * 2;
     const size_t smem = (size_t)kAttnStages * kStageBytes + sizeof(AttnShared) + 1024;
     const int ti = (D == 128) ? 1 : 0;
     if (!stt.attr_set[ti]) {

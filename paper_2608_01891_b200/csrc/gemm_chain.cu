@@ -4,27 +4,32 @@
 // At decode batch sizes (<= 64 token rows) the FFN side and the W_o projection are weight-streaming
 // kernels: the boundary projection x = a W_o^T, h = silu(x W_gate^T) .* (x W_up^T) and y = h W_down^T
 // each read their weights once and are bound by HBM.  Run as separate kernels, every boundary between
-// two of them leaves DRAM idle: the last CTAs of one kernel finish their shared-tile reduction while
-// the next kernel's CTAs cannot become resident beside them (shared memory), set up, and only then
-// request their first bytes.  Here the GEMMs are PHASES of one kernel, and no phase ever waits for
-// the whole of its predecessor:
+// two of them leaves DRAM idle: the last CTAs of one kernel finish their shared-tile reduction (a chain
+// of half a dozen dependent L2 round trips, each 1 - 2 us while the memory system is busy) while the
+// next kernel's CTAs cannot become resident beside them (shared memory), set up, and only then request
+// their first bytes.  Here the GEMMs are PHASES of one kernel, and no phase waits for the whole of its
+// predecessor:
 //
 //   * one CTA per SM stays resident for all phases; barriers, TMEM and the shared-memory ring are set
 //     up once and the ring keeps turning across phase boundaries;
 //   * the weight producer (warp 0) never waits for anything but a free ring stage: weights are inputs
 //     that no kernel writes;
-//   * every phase produces its output tiles in two SEGMENTS, one after the other (remainder tiles that
-//     are shared along K first, whole tiles second; a phase whose tiles are all shared is one segment,
-//     or optionally two halves).  A segment's output is complete - its shared-tile reductions included - while the next
-//     segment streams, and is announced through an epoch word;
+//   * every phase produces its output tiles in up to four SEGMENTS, one after the other (remainder tiles
+//     that are shared along K first, whole tiles second; a phase whose tiles are all shared is cut into
+//     equal groups of tiles).  A segment's output is completed - its shared-tile reductions included -
+//     while the next segment streams, and is announced through an epoch word;
+//   * the reductions run on warps of their own (7..10): the epilogue warps only park fp32 partials and
+//     post a job through a shared-memory barrier, so a segment's reduction (waiting for the other
+//     contributors, summing in CTA order) never delays the parking of the next accumulators, and no
+//     epilogue thread ever executes a device-wide fence; a publisher thread releases each parked
+//     partial to the other CTAs at once, whatever the reducers are busy with;
 //   * a K step of phase p+1 reads 64 or 128 columns of phase p's output, i.e. the output of ONE tile of
-//     phase p.  Every piece of work of phase p+1 (a run of K steps of one tile in one CTA) visits the
-//     K steps fed by segment 0 of phase p first and those fed by segment 1 after (any K order gives the
-//     same sum up to rounding; the order is a fixed function of the piece, so results are bit-
-//     deterministic).  The activation producer (warp 6) waits (bounded) for segment 0's epoch before
-//     its first early step and for segment 1's epoch before its first late step - by which time the
-//     epilogue, the reduction and the slowest CTA of that segment have had the early steps' streaming
-//     time to finish;
+//     phase p.  Every piece of work of phase p+1 (a run of K steps of one tile in one CTA) visits its
+//     share of the K steps fed by segment 0 of phase p first, then of segment 1, and so on (any K order
+//     gives the same sum up to rounding; the order is a fixed function of the piece, so results are
+//     bit-deterministic).  The activation producer (warp 6) waits (bounded) for a segment's epoch only
+//     before the first step that needs it - by which time the reduction and the slowest CTA of that
+//     segment have had the earlier steps' streaming time to finish;
 //   * per segment the tiles are dealt exactly like the stand-alone GEMM (gemm_sched.cuh): equal,
 //     contiguous shares of K steps, partials reduced in CTA order.
 //
@@ -36,8 +41,8 @@
 // consecutive K blocks (w, w', x, x') of one accumulator, so that both phase kinds keep the whole ring
 // in flight.
 //
-// CTA = 7 warps: 0 weight producer, 1 MMA issuer (owns TMEM), 2..5 epilogue, 6 activation producer.
-// Every wait is bounded; on expiry the CTA raises AFLEX_ERR_TIMEOUT, drains and leaves.
+// CTA = 12 warps: 0 weight producer, 1 MMA issuer (owns TMEM), 2..5 epilogue, 6 activation producer,
+// 7..10 reducers, 11 publisher (releases parked partials to the other CTAs).  Every wait is bounded; on expiry the CTA raises AFLEX_ERR_TIMEOUT, drains and leaves.
 #include <cuda_bf16.h>
 #include <stdlib.h>
 
@@ -47,23 +52,28 @@
 
 namespace aflex {
 
-constexpr int kChainThreads = 224;
+constexpr int kChainThreads = 384;
 constexpr int kChainBlockM = 128;
 constexpr int kChainBlockK = 64;
 constexpr int kChainTileBytes = kChainBlockM * kChainBlockK * 2;   // one weight tile: 16 KB
 constexpr int kChainMaxStages = 8;
 constexpr int kChainMaxPhases = 3;
-constexpr int kChainSlots = 8;
+constexpr int kChainMaxSegs = 4;
+constexpr long long kChainIdleCycles = 4000;   // a wait for a free ring stage this long (~2 us) is a stall, not back-pressure
+constexpr int kChainSlots = 2 * kChainMaxSegs * 2;   // partial slots per CTA: [phase parity][segment][first / later unit]
 constexpr int kChainCounterInts = 8192;   // per half of the double-buffered counter array: per-tile counters, then the epoch words
-constexpr int kChainEpochBase = kChainCounterInts - 16;          // partial slots per CTA: [phase parity][segment][first / later unit]
+constexpr int kChainEpochBase = kChainCounterInts - 16;
+constexpr int kChainMaxJobs = 64;          // reduce jobs one CTA can post in a launch (<= 2 per segment, plus markers)
 
 struct ChainPhase {
     int gateup;        // 1: two weight matrices, SwiGLU epilogue; 0: plain linear
     int N;             // weight rows (output features)
     int K;             // reduction length
     int ksteps;        // ring stages per tile: ceil(K / 64) (gate/up) or ceil(K / 128) (linear)
-    int seg_tiles[2];  // output tiles of segment 0 (ids 0 ..) and of segment 1 (ids seg_tiles[0] ..)
-    int n_early;       // K steps [0, n_early) read what the previous phase's segment 0 wrote (first phase: all)
+    int nseg;          // segments in use (1..4)
+    int seg_tiles[kChainMaxSegs];   // output tiles per segment; segment g owns tile ids [sum of the earlier ones, + seg_tiles[g])
+    int cls_end[kChainMaxSegs];     // K steps [cls_end[g-1], cls_end[g]) read what segment g of the previous phase wrote
+                                    // (non-decreasing, last = ksteps; first phase: everything is class 0)
     int counter_base;  // first per-tile arrival counter of this phase
     __nv_bfloat16* out;   // [T][N]
 };
@@ -75,11 +85,14 @@ struct ChainParams {
     int nphase;
     int stages;
     int tmem_cols;
+    int l2_first_phase;   // first phase whose weights may be prefetched that way
+    int l2_ahead;      // ring stages' worth of weights the idle weight producer may prefetch into L2 beyond the ring (0 = off)
     ChainPhase ph[kChainMaxPhases];
     float* partials;   // [grid][kChainSlots][2 * n_tile / 4][128 rows] float4
     int* counters;     // two halves of kChainCounterInts ints, then the generation word.  A launch of generation g counts
                        // in half g & 1 (per-tile arrival counters and, at kChainEpochBase, its epoch words: (phase, segment)
-                       // finished by so many CTAs; all zero on entry), zeroes the other half for its successor and bumps g
+                       // finished by so many CTAs; all zero on entry), zeroes the other half for its
+                       // successor and bumps g
     int* status;
     unsigned long long* trace;   // optional [grid][32] timestamps (ns), or nullptr
 };
@@ -98,24 +111,48 @@ struct __align__(8) ChainBarriers {
     uint32_t tmem_base;
     volatile int abort;
     volatile int gen;       // this launch's generation, published by the epilogue once the grid dependency has resolved (-1 before)
+    uint64_t job_bar[kChainMaxJobs];    // job n is posted when the 128 epilogue threads have arrived on job_bar[n] (used once each)
+    volatile int cur_job, cur_gen;   // the reducers' current job and the generation, handed from their thread 0 to the others
+    volatile int job[kChainMaxJobs];   // (phase << 24) | (segment << 20) | kind << 16 | tile in the segment
 };
+static_assert(sizeof(ChainBarriers) <= 1024, "the staging buffers start 1 KB behind the barriers");
+constexpr int kJobReduce = 0, kJobSegEnd = 1, kJobExit = 2;
 
-// The order in which a piece (logical K positions [j0, j1) of a tile with nK steps, n_early of them "early")
-// visits the actual K steps: its share of the early steps first, then its share of the late ones.  Over the
-// pieces of a tile the two shares partition [0, n_early) and [n_early, nK).
+// The order in which a piece (logical K positions [j0, j1) of a tile with nK steps) visits the actual K steps:
+// its share of class 0's steps first, then of class 1's, ... (class g = actual steps [E[g-1], E[g])).  The shares
+// are defined by halving twice - classes {0,1} against {2,3}, then inside each half - with the rule
+// "positions [0, j) hold floor(j * n / m) steps of the first part", which is monotone in j, so over the pieces
+// of a tile the shares partition every class exactly.
 struct StepOrder {
-    int eb0, n_early_here, late0;
-    __device__ StepOrder(int j0, int j1, int nK, int n_early) {
-        eb0 = (int)((long long)j0 * n_early / nK);
-        const int eb1 = (int)((long long)j1 * n_early / nK);
-        n_early_here = eb1 - eb0;
-        late0 = n_early + (j0 - eb0);
+    int lo[kChainMaxSegs], len[kChainMaxSegs];
+    __device__ static int part(int j, int n, int m) { return m > 0 ? (int)((long long)j * n / m) : 0; }
+    __device__ StepOrder(int j0, int j1, int nK, const int* E) {
+        const int x0 = part(j0, E[1], nK), x1 = part(j1, E[1], nK);       // classes 0,1: index range [x0, x1) of [0, E1)
+        const int y0 = j0 - x0, y1 = j1 - x1;                              // classes 2,3: index range [y0, y1) of [0, nK - E1)
+        const int a0 = part(x0, E[0], E[1]), a1 = part(x1, E[0], E[1]);
+        lo[0] = a0; len[0] = a1 - a0;
+        lo[1] = E[0] + (x0 - a0); len[1] = (x1 - a1) - (x0 - a0);
+        const int c0 = part(y0, E[2] - E[1], nK - E[1]), c1 = part(y1, E[2] - E[1], nK - E[1]);
+        lo[2] = E[1] + c0; len[2] = c1 - c0;
+        lo[3] = E[2] + (y0 - c0); len[3] = (y1 - c1) - (y0 - c0);
     }
-    __device__ int actual(int i) const { return i < n_early_here ? eb0 + i : late0 + (i - n_early_here); }
+    __device__ int actual(int i) const {
+#pragma unroll
+        for (int g = 0; g < kChainMaxSegs - 1; ++g) {
+            if (i < len[g]) return lo[g] + i;
+            i -= len[g];
+        }
+        return lo[kChainMaxSegs - 1] + i;
+    }
 };
 
 __device__ __forceinline__ float chain_silu(float z) { return __fdividef(z, 1.0f + __expf(-z)); }
 __device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+__device__ __forceinline__ int seg_tile0(const ChainPhase& P, int seg) {
+    int t = 0;
+    for (int g = 0; g < seg; ++g) t += P.seg_tiles[g];
+    return t;
+}
 
 __global__ void __launch_bounds__(kChainThreads, 1)
 gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const ChainParams p) {
@@ -124,8 +161,10 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const ChainParams p) {
     const int b_bytes = (p.n_tile * kChainBlockK * 2 + 1023) & ~1023;       // one activation tile slot
     const int stage_bytes = 2 * kChainTileBytes + 2 * b_bytes;
     ChainBarriers* bars = reinterpret_cast<ChainBarriers*>(smem + (size_t)p.stages * stage_bytes);
-    // epilogue staging: the output tile as [token][128 features] bf16, so that it leaves the SM in 16-byte pieces
-    __nv_bfloat16* stage_out = reinterpret_cast<__nv_bfloat16*>(smem + (size_t)p.stages * stage_bytes + 1024);
+    // output staging, one buffer for the epilogue warps and one for the reducer warps: the output tile as
+    // [token][128 features] bf16, so that it leaves the SM in 16-byte pieces
+    __nv_bfloat16* stage_epi = reinterpret_cast<__nv_bfloat16*>(smem + (size_t)p.stages * stage_bytes + 1024);
+    __nv_bfloat16* stage_red = stage_epi + (size_t)p.n_tile * kChainBlockM;
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -136,6 +175,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const ChainParams p) {
         for (int b = 0; b < 2; ++b) { mbar_init(&bars->tmem_full[b], 1); mbar_init(&bars->tmem_empty[b], 4); }
         bars->abort = 0;
         bars->gen = -1;
+        for (int i = 0; i < kChainMaxJobs; ++i) mbar_init(&bars->job_bar[i], 128);
         fence_mbar_init();
     }
     if (warp == 1) {
@@ -154,9 +194,19 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const ChainParams p) {
 
     const uint32_t tmem_base = bars->tmem_base;
     const int buf_cols = 2 * p.n_tile;                   // TMEM columns per accumulator buffer (room for gate and up)
+    const size_t slot_floats = (size_t)2 * p.n_tile * kChainBlockM;
     pdl_launch_dependents();
     unsigned long long* tr = p.trace ? p.trace + (size_t)blockIdx.x * 32 : nullptr;
     if (tr && threadIdx.x == 0) { tr[0] = global_timer_ns(); unsigned smid; asm volatile("mov.u32 %0, %%smid;" : "=r"(smid)); tr[3] = smid; }   // CTA running
+
+    // The launch's generation, read from global memory by the epilogue after the grid dependency has resolved.
+    auto wait_gen = [&]() -> int {
+        const long long t_start = clock64();
+        int gen;
+        while ((gen = bars->gen) < 0 && !bars->abort && clock64() - t_start < kWaitBudgetCycles) __nanosleep(20);
+        if (gen < 0 && !bars->abort) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); }
+        return gen;
+    };
 
     if (warp == 0) {
         // ------------------------------------------------------------ weight producer
@@ -165,16 +215,44 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const ChainParams p) {
             int s = 0; uint32_t ph = 0;
             for (int pi = 0; pi < p.nphase && !bars->abort; ++pi) {
                 const ChainPhase& P = p.ph[pi];
-                for (int seg = 0; seg < 2 && !bars->abort; ++seg) {
+                for (int seg = 0; seg < P.nseg && !bars->abort; ++seg) {
                     const Schedule sched(P.ksteps, 1, P.seg_tiles[seg], grid);
+                    const int tile0 = seg_tile0(P, seg);
                     UnitCursor cur(sched, blockIdx.x);
                     WorkUnit wu;
                     while (!bars->abort && cur.next(wu)) {
-                        const int row0 = (seg * P.seg_tiles[0] + wu.tile) * kChainBlockM;
-                        const StepOrder ord(wu.kb0, wu.kb1, P.ksteps, P.n_early);
-                        for (int i = 0; i < wu.kb1 - wu.kb0; ++i) {
+                        const int row0 = (tile0 + wu.tile) * kChainBlockM;
+                        const StepOrder ord(wu.kb0, wu.kb1, P.ksteps, P.cls_end);
+                        const int L = wu.kb1 - wu.kb0;
+                        int pf = 0;                                   // steps of this unit already asked into L2
+                        for (int i = 0; i < L; ++i) {
                             const int ks = ord.actual(i);
-                            if (!mbar_wait(&bars->empty[s], ph ^ 1)) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); break; }
+                            if (!mbar_try_wait(&bars->empty[s], ph ^ 1)) {
+                                // No free stage.  In steady state one frees up every ~0.7 us.  A longer wait means the
+                                // consumers are held up (a phase's input is not there yet): nobody on this SM asks DRAM
+                                // for anything, so the wait can be spent pulling the next steps' weight tiles into L2.
+                                const long long t0w = clock64();
+                                bool ok = false;
+                                while (!(ok = mbar_try_wait(&bars->empty[s], ph ^ 1))) {
+                                    const long long dt = clock64() - t0w;
+                                    if (dt > kWaitBudgetCycles || bars->abort) break;
+                                    if (p.l2_ahead > 0 && pi >= p.l2_first_phase && dt > kChainIdleCycles) {
+                                        if (pf < i) pf = i;
+                                        if (pf < L && pf < i + p.l2_ahead) {
+                                            const int kp = ord.actual(pf);
+                                            if (P.gateup) {
+                                                tma_prefetch_l2_2d(&maps.a0[pi], kp * kChainBlockK, row0);
+                                                tma_prefetch_l2_2d(&maps.a1[pi], kp * kChainBlockK, row0);
+                                            } else {
+                                                tma_prefetch_l2_2d(&maps.a0[pi], 2 * kp * kChainBlockK, row0);
+                                                tma_prefetch_l2_2d(&maps.a0[pi], (2 * kp + 1) * kChainBlockK, row0);
+                                            }
+                                            ++pf;
+                                        }
+                                    }
+                                }
+                                if (!ok) { if (!bars->abort) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); } break; }
+                            }
                             uint8_t* st = smem + (size_t)s * stage_bytes;
                             mbar_expect_tx(&bars->full[s], 2u * kChainTileBytes);
                             if (P.gateup) {
@@ -202,41 +280,43 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const ChainParams p) {
             int s = 0; uint32_t ph = 0;
             pdl_wait();                                       // the first phase's input comes from the preceding kernel
             if (tr) tr[1] = global_timer_ns();
+            bool bumped = false;
             for (int pi = 0; pi < p.nphase && !bars->abort; ++pi) {
                 const ChainPhase& P = p.ph[pi];
-                bool ready[2] = {pi == 0, pi == 0};
+                int ready = pi == 0 ? kChainMaxSegs : 0;      // classes [0, ready) of this phase's input are complete
                 // Segment e of the previous phase complete in every CTA, and visible to the TMA reads that follow.
                 auto need = [&](int e) -> bool {
-                    if (ready[e]) return true;
-                    const long long t_start = clock64();
-                    int gen;
-                    while ((gen = bars->gen) < 0 && clock64() - t_start < kWaitBudgetCycles) __nanosleep(20);
-                    if (gen < 0) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); return false; }
-                    const int* word = p.counters + (size_t)(gen & 1) * kChainCounterInts + kChainEpochBase + (pi - 1) * 2 + e;
-                    int seen;
-                    do {
-                        asm volatile("ld.acquire.gpu.b32 %0, [%1];" : "=r"(seen) : "l"(word) : "memory");
-                        if (seen >= grid) break;
-                        __nanosleep(20);
-                    } while (clock64() - t_start < kWaitBudgetCycles);
-                    if (seen < grid) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); return false; }
-                    fence_proxy_async_all();
-                    // every CTA's epilogue has read the generation by now (it signals only afterwards): one thread of the
-                    // grid moves it on for the next launch
-                    if (blockIdx.x == 0 && pi == 1 && !ready[0] && !ready[1]) p.counters[2 * kChainCounterInts] = (gen + 1) & 0x3fffffff;
-                    ready[e] = true;
-                    if (tr) tr[4 + pi * 8 + 1 + e] = global_timer_ns();   // input from segment e available
+                    while (ready <= e) {
+                        const int gen = wait_gen();
+                        if (gen < 0) return false;
+                        const int* word = p.counters + (size_t)(gen & 1) * kChainCounterInts + kChainEpochBase + (pi - 1) * kChainMaxSegs + ready;
+                        const long long t_start = clock64();
+                        int seen;
+                        do {
+                            asm volatile("ld.acquire.gpu.b32 %0, [%1];" : "=r"(seen) : "l"(word) : "memory");
+                            if (seen >= grid) break;
+                            __nanosleep(20);
+                        } while (clock64() - t_start < kWaitBudgetCycles && !bars->abort);
+                        if (seen < grid) { if (!bars->abort) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); } return false; }
+                        fence_proxy_async_all();
+                        // every CTA's epilogue has read the generation by now (it signs off only afterwards): one thread of
+                        // the grid moves it on for the next launch
+                        if (blockIdx.x == 0 && !bumped) { p.counters[2 * kChainCounterInts] = (gen + 1) & 0x3fffffff; bumped = true; }
+                        if (tr && ready < 2) tr[4 + pi * 8 + 1 + ready] = global_timer_ns();   // input from segment `ready` available
+                        ++ready;
+                    }
                     return true;
                 };
-                for (int seg = 0; seg < 2 && !bars->abort; ++seg) {
+                for (int seg = 0; seg < P.nseg && !bars->abort; ++seg) {
                     const Schedule sched(P.ksteps, 1, P.seg_tiles[seg], grid);
                     UnitCursor cur(sched, blockIdx.x);
                     WorkUnit wu;
                     while (!bars->abort && cur.next(wu)) {
-                        const StepOrder ord(wu.kb0, wu.kb1, P.ksteps, P.n_early);
+                        const StepOrder ord(wu.kb0, wu.kb1, P.ksteps, P.cls_end);
                         for (int i = 0; i < wu.kb1 - wu.kb0; ++i) {
                             const int ks = ord.actual(i);
-                            if (!need(ks < P.n_early ? 0 : 1)) break;
+                            const int cls = ks < P.cls_end[0] ? 0 : ks < P.cls_end[1] ? 1 : ks < P.cls_end[2] ? 2 : 3;
+                            if (!need(cls)) break;
                             if (!mbar_wait(&bars->empty[s], ph ^ 1)) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); break; }
                             uint8_t* st = smem + (size_t)s * stage_bytes + 2 * kChainTileBytes;
                             if (P.gateup) {
@@ -252,6 +332,21 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const ChainParams p) {
                     }
                 }
             }
+            // a grid without any later phase step in CTA 0 still has to move the generation on
+            if (blockIdx.x == 0 && !bumped && !bars->abort && p.nphase > 1) {
+                const int gen = wait_gen();
+                if (gen >= 0) {
+                    const int* word = p.counters + (size_t)(gen & 1) * kChainCounterInts + kChainEpochBase;
+                    const long long t_start = clock64();
+                    int seen;
+                    do {
+                        asm volatile("ld.acquire.gpu.b32 %0, [%1];" : "=r"(seen) : "l"(word) : "memory");
+                        if (seen >= grid) break;
+                        __nanosleep(20);
+                    } while (clock64() - t_start < kWaitBudgetCycles && !bars->abort);
+                    if (seen >= grid) p.counters[2 * kChainCounterInts] = (gen + 1) & 0x3fffffff;
+                }
+            }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
@@ -261,7 +356,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const ChainParams p) {
             const uint32_t idesc = umma_idesc_bf16(kChainBlockM, (uint32_t)p.box);
             for (int pi = 0; pi < p.nphase && !bars->abort; ++pi) {
                 const ChainPhase& P = p.ph[pi];
-                for (int seg = 0; seg < 2 && !bars->abort; ++seg) {
+                for (int seg = 0; seg < P.nseg && !bars->abort; ++seg) {
                     const Schedule sched(P.ksteps, 1, P.seg_tiles[seg], grid);
                     UnitCursor cur(sched, blockIdx.x);
                     WorkUnit wu;
@@ -297,24 +392,34 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const ChainParams p) {
                         }
                         if (bars->abort) break;
                         umma_commit(&bars->tmem_full[buf]);
-                        if (tr && wu.slot < 0) tr[18] = global_timer_ns();
                         if (++buf == 2) { buf = 0; acc_ph ^= 1; }
                     }
                 }
                 if (tr) tr[4 + pi * 8 + 3] = global_timer_ns();       // phase's last MMA issued
             }
         }
-    } else {
+    } else if (warp >= 2 && warp <= 5) {
         // ------------------------------------------------------------ epilogue (warps 2..5)
+        // Whole tiles go from TMEM through the staging buffer to the output; partial accumulators are parked in the
+        // workspace and handed to the reducer warps as a job.  These warps never wait for another CTA.
         const int lane_grp = warp & 3;
         const int row = lane_grp * 32 + lane;
         const int etid = threadIdx.x - 64;
-        const size_t slot_floats = (size_t)2 * p.n_tile * kChainBlockM;
         int buf = 0; uint32_t acc_ph = 0;
+        int njobs = 0;
+        // Every epilogue thread calls this after its own stores of the job's data: the barrier's release / acquire hands
+        // those stores on to the publisher and the reducers, who put their device-wide fence behind them.
+        auto post = [&](int job) {
+            if (njobs < kChainMaxJobs) {
+                if (etid == 0) bars->job[njobs] = job;
+                mbar_arrive(&bars->job_bar[njobs]);
+                ++njobs;
+            }
+        };
         pdl_wait();   // nothing is written (outputs, partials, counters) before the preceding kernels have completed
-        // The counters are double-buffered over launches: this launch counts in one half (zero on entry) and zeroes
-        // the other half, which the launch before it used and the launch after it will use.  Both neighbours are
-        // ordered against these stores by the grid dependency (the wait above; the next launch's own wait).
+        // The counters are double-buffered over launches: this launch counts in half (generation & 1), zero on entry,
+        // and zeroes the other half, which the launch before it used and the launch after it will use.  Both
+        // neighbours are ordered against these stores by the grid dependency (the wait above; the next launch's own).
         if (etid == 0) {
             int g;
             asm volatile("ld.relaxed.gpu.b32 %0, [%1];" : "=r"(g) : "l"(p.counters + 2 * kChainCounterInts) : "memory");
@@ -327,132 +432,26 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const ChainParams p) {
             for (int i = (int)blockIdx.x * 128 + etid; i < kChainCounterInts; i += grid * 128) other[i] = 0;
         }
 
-        for (int pi = 0; pi < p.nphase && !bars->abort; ++pi) {
+        bool gave_up = false;
+        for (int pi = 0; pi < p.nphase && !gave_up; ++pi) {
             const ChainPhase& P = p.ph[pi];
             const int accs = P.gateup ? 2 : 1;
-            for (int seg = 0; seg < 2 && !bars->abort; ++seg) {
+            for (int seg = 0; seg < P.nseg && !gave_up; ++seg) {
                 const Schedule sched(P.ksteps, 1, P.seg_tiles[seg], grid);
-                const int tile0 = seg * P.seg_tiles[0];                    // first tile id of this segment
-                int* counters = ctr + P.counter_base + tile0;
-                const int slot0 = ((pi & 1) * 2 + seg) * 2;                // this (phase parity, segment)'s pair of partial slots
-                int pend[2];
-                int npend = 0;
-
-                // Token rows [t_lo, t_hi) of the staged tile -> out[t][128 * tile ..], 16 bytes per thread and store; the
-                // trailing barrier frees the staging buffer for its next user.
-                auto store_rows = [&](int tile_g, int t_lo, int t_hi) {
-                    if (t_hi > p.T) t_hi = p.T;
-                    for (int c = t_lo * 16 + etid; c < t_hi * 16; c += 128) {
-                        const int t = c >> 4, part = c & 15;
-                        const int n = tile_g * kChainBlockM + part * 8;
-                        if (n < P.N)
-                            *reinterpret_cast<uint4*>(P.out + (size_t)t * P.N + n) = *reinterpret_cast<const uint4*>(stage_out + t * kChainBlockM + part * 8);
-                    }
-                    asm volatile("bar.sync 2, 128;" ::: "memory");
-                };
-
-                // This CTA's slice of a shared tile, summed over the pieces in CTA order (see gemm_tcgen05.cu).
-                auto run_reduce = [&](int tile) {
-                    const long long x0 = (long long)tile * P.ksteps;
-                    const int cf = sched.cta_of(x0);
-                    const int cl = sched.cta_of(x0 + P.ksteps - 1);
-                    const int np = cl - cf + 1, me = (int)blockIdx.x - cf;
-                    const int nred = (np > 1 && sched.share_begin(cl + 1) > x0 + P.ksteps) ? np - 1 : np;
-                    if (me >= nred) return;
-                    if (etid == 0) {
-                        const long long t_start = clock64();
-                        int seen;
-                        do {
-                            asm volatile("ld.acquire.gpu.b32 %0, [%1];" : "=r"(seen) : "l"(counters + tile) : "memory");
-                            if (seen >= np) break;
-                            __nanosleep(64);
-                        } while (clock64() - t_start < kWaitBudgetCycles);
-                        if (seen < np) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); }
-                    }
-                    asm volatile("bar.sync 2, 128;" ::: "memory");     // the acquire above, handed on to the other 127 threads
-                    if (tr && etid == 0) tr[30] = global_timer_ns();
-                    if (bars->abort) return;
-                    const bool cf_early = sched.share_begin(cf) < x0;
-                    // The parked accumulator is [column group of 4 tokens][128 rows] float4: reducer `me` takes whole column
-                    // groups, thread = weight row.  kE groups per round, every piece's loads of a round in flight together
-                    // (the loop is a chain of L2 round trips, not bandwidth).
-                    const int ncg = ((p.T + 15) / 16) * 4;
-                    const int cg_lo = ncg * me / nred, cg_hi = ncg * (me + 1) / nred;
-                    const int up_off = (p.n_tile >> 2) * kChainBlockM;
-                    constexpr int kE = 4;
-                    for (int c0 = cg_lo; c0 < cg_hi; c0 += kE) {
-                        float4 g[kE], u[kE];
-#pragma unroll
-                        for (int e = 0; e < kE; ++e) g[e] = u[e] = make_float4(0.f, 0.f, 0.f, 0.f);
-                        for (int cb = cf; cb <= cl; cb += 4) {
-                            float4 a[kE][4];
-#pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                const int cc = cb + q;
-                                if (cc <= cl) {
-                                    const int sl = slot0 + ((cc == cf && cf_early) ? 1 : 0);
-                                    const float4* part = reinterpret_cast<const float4*>(p.partials + ((size_t)cc * kChainSlots + sl) * slot_floats) + etid;
-#pragma unroll
-                                    for (int e = 0; e < kE; ++e)
-                                        if (c0 + e < cg_hi) a[e][q] = __ldcg(part + (c0 + e) * kChainBlockM);
-                                }
-                            }
-#pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                if (cb + q <= cl) {
-#pragma unroll
-                                    for (int e = 0; e < kE; ++e)
-                                        if (c0 + e < cg_hi) { g[e].x += a[e][q].x; g[e].y += a[e][q].y; g[e].z += a[e][q].z; g[e].w += a[e][q].w; }
-                                }
-                            }
-                            if (accs == 2) {
-#pragma unroll
-                                for (int q = 0; q < 4; ++q) {
-                                    const int cc = cb + q;
-                                    if (cc <= cl) {
-                                        const int sl = slot0 + ((cc == cf && cf_early) ? 1 : 0);
-                                        const float4* part = reinterpret_cast<const float4*>(p.partials + ((size_t)cc * kChainSlots + sl) * slot_floats) + up_off + etid;
-#pragma unroll
-                                        for (int e = 0; e < kE; ++e)
-                                            if (c0 + e < cg_hi) a[e][q] = __ldcg(part + (c0 + e) * kChainBlockM);
-                                    }
-                                }
-#pragma unroll
-                                for (int q = 0; q < 4; ++q) {
-                                    if (cb + q <= cl) {
-#pragma unroll
-                                        for (int e = 0; e < kE; ++e)
-                                            if (c0 + e < cg_hi) { u[e].x += a[e][q].x; u[e].y += a[e][q].y; u[e].z += a[e][q].z; u[e].w += a[e][q].w; }
-                                    }
-                                }
-                            }
-                        }
-#pragma unroll
-                        for (int e = 0; e < kE; ++e) {
-                            if (c0 + e >= cg_hi) break;
-                            const float gf[4] = {g[e].x, g[e].y, g[e].z, g[e].w}, uf[4] = {u[e].x, u[e].y, u[e].z, u[e].w};
-#pragma unroll
-                            for (int k = 0; k < 4; ++k)
-                                stage_out[((c0 + e) * 4 + k) * kChainBlockM + etid] = __float2bfloat16_rn(P.gateup ? chain_silu(gf[k]) * uf[k] : gf[k]);
-                        }
-                    }
-                    asm volatile("bar.sync 2, 128;" ::: "memory");
-                    store_rows(tile0 + tile, cg_lo * 4, cg_hi * 4);
-                };
-
+                const int tile0 = seg_tile0(P, seg);
+                const int slot0 = ((pi & 1) * kChainMaxSegs + seg) * 2;    // this (phase parity, segment)'s pair of partial slots
                 UnitCursor cur(sched, blockIdx.x);
                 WorkUnit wu;
-                while (!bars->abort && cur.next(wu)) {
-                    if (wu.slot < 0 && npend > 0) {
-                        for (int i = 0; i < npend; ++i) run_reduce(pend[i]);
-                        npend = 0;
-                        if (bars->abort) break;
+                // (the four warps leave this loop together: every exit is decided on a predicate OR-ed across them)
+                while (cur.next(wu)) {
+                    if (bar_or(2, 128, bars->abort != 0)) { gave_up = true; break; }
+                    const bool ok = mbar_wait(&bars->tmem_full[buf], acc_ph);
+                    if (bar_or(2, 128, !ok)) {
+                        if (etid == 0) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); }
+                        gave_up = true;
+                        break;
                     }
-                    if (!mbar_wait(&bars->tmem_full[buf], acc_ph)) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); break; }
                     tc_fence_after();
-                    if (tr && etid == 0) tr[wu.slot < 0 ? 10 : 28] = global_timer_ns();
-                    const int n_local = (tile0 + wu.tile) * kChainBlockM + row;
-                    const bool n_ok = n_local < P.N;
                     const uint32_t t0 = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(buf * buf_cols);
                     if (wu.slot < 0) {
                         for (int c0 = 0; c0 < p.T; c0 += 16) {
@@ -463,15 +462,21 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const ChainParams p) {
 #pragma unroll
                             for (int j = 0; j < 16; ++j) {
                                 const float v = P.gateup ? chain_silu(__uint_as_float(g[j])) * __uint_as_float(u[j]) : __uint_as_float(g[j]);
-                                stage_out[(c0 + j) * kChainBlockM + row] = __float2bfloat16_rn(v);
+                                stage_epi[(c0 + j) * kChainBlockM + row] = __float2bfloat16_rn(v);
                             }
                         }
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive(&bars->tmem_empty[buf]);
                         asm volatile("bar.sync 2, 128;" ::: "memory");
-                        store_rows(tile0 + wu.tile, 0, p.T);
-                        if (tr && etid == 0) tr[11] = global_timer_ns();
+                        // token rows of the staged tile -> out[t][128 * tile ..], 16 bytes per thread and store
+                        for (int c = etid; c < p.T * 16; c += 128) {
+                            const int t = c >> 4, part = c & 15;
+                            const int n = (tile0 + wu.tile) * kChainBlockM + part * 8;
+                            if (n < P.N)
+                                *reinterpret_cast<uint4*>(P.out + (size_t)t * P.N + n) = *reinterpret_cast<const uint4*>(stage_epi + t * kChainBlockM + part * 8);
+                        }
+                        asm volatile("bar.sync 2, 128;" ::: "memory");
                     } else {
                         uint4* mine = reinterpret_cast<uint4*>(p.partials + ((size_t)blockIdx.x * kChainSlots + slot0 + wu.slot) * slot_floats) + row;
                         for (int a = 0; a < accs; ++a) {
@@ -487,28 +492,181 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const ChainParams p) {
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive(&bars->tmem_empty[buf]);
-                        asm volatile("bar.sync 2, 128;" ::: "memory");
-                        if (etid == 0) {
-                            __threadfence();
-                            atomicAdd(&counters[wu.tile], 1);
-                            if (tr) tr[29] = global_timer_ns();
-                        }
-                        pend[npend++] = wu.tile;
+                        post((pi << 24) | (seg << 20) | (kJobReduce << 16) | wu.tile);
                     }
                     if (++buf == 2) { buf = 0; acc_ph ^= 1; }
                 }
-                for (int i = 0; i < npend && !bars->abort; ++i) run_reduce(pend[i]);
-                // ---- this CTA's part of the segment's output is written: announce it to the next phase
-                if (pi + 1 < p.nphase) {
-                    // every path above ends with a barrier behind its last output store; the reader orders its TMA (async
-                    // proxy) reads behind its acquire of the epoch word with a proxy fence of its own
-                    if (tr && etid == 0) tr[26] = global_timer_ns();
-                    if (etid == 0 && !bars->abort) {
-                        __threadfence();
-                        atomicAdd(ctr + kChainEpochBase + pi * 2 + seg, 1);
+                // ---- this CTA's whole tiles of the segment are written (behind a barrier): sign off for the epilogue, and
+                //      tell the reducers that the segment has no more jobs
+                if (!gave_up) {
+                    post((pi << 24) | (seg << 20) | (kJobSegEnd << 16));
+                    if (tr && etid == 0 && seg < 2) tr[4 + pi * 8 + 4 + seg] = global_timer_ns();    // segment parked / written by this CTA's epilogue
+                }
+            }
+        }
+        post(kJobExit << 16);
+    } else if (warp >= 7 && warp <= 10) {
+        // ------------------------------------------------------------ reducers (warps 7..10)
+        // One job at a time, in the order the epilogue posted them: this CTA's slice of a shared tile, summed over the
+        // contributors' pieces in CTA order (bit-deterministic), staged and written; at a segment's end marker, the
+        // sign-off for the reducers.
+        const int rtid = threadIdx.x - 224;
+        volatile int& s_job = bars->cur_job;
+        volatile int& s_gen = bars->cur_gen;
+        pdl_wait();
+        int* ctr = nullptr;
+        int taken = 0;
+        // (the four warps move together: thread 0 takes every decision and hands it on through shared memory or an
+        // OR-ing barrier, so no exit can split the group in front of a barrier)
+        while (true) {
+            const bool got = taken < kChainMaxJobs && mbar_wait(&bars->job_bar[taken], 0);
+            if (rtid == 0) {
+                if (!got && !bars->abort) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); }
+                s_job = (!got || bars->abort) ? (kJobExit << 16) : bars->job[taken];
+                if (ctr == nullptr) s_gen = (!got || bars->abort) ? -1 : wait_gen();
+            }
+            asm volatile("bar.sync 3, 128;" ::: "memory");
+            const int job = s_job, gen = s_gen;
+            asm volatile("bar.sync 3, 128;" ::: "memory");     // everybody has read them before they are overwritten
+            ++taken;
+            const int kind = (job >> 16) & 0xf, pi = job >> 24, seg = (job >> 20) & 0xf, tile = job & 0xffff;
+            if (kind == kJobExit || gen < 0) break;
+            if (ctr == nullptr) ctr = p.counters + (size_t)(gen & 1) * kChainCounterInts;
+            const ChainPhase& P = p.ph[pi];
+            if (kind == kJobSegEnd) {
+                // The segment is complete in this CTA: its whole tiles were stored by the epilogue threads before they posted
+                // this marker, every reduce job ended with a barrier behind its last output store.  One sign-off for both.
+                if (rtid == 0 && pi + 1 < p.nphase) {
+                    __threadfence();
+                    atomicAdd(ctr + kChainEpochBase + pi * kChainMaxSegs + seg, 1);
+                }
+                if (tr && rtid == 0 && seg < 2) tr[26 + seg] = global_timer_ns();
+                continue;
+            }
+            const int accs = P.gateup ? 2 : 1;
+            const Schedule sched(P.ksteps, 1, P.seg_tiles[seg], grid);
+            const int tile0 = seg_tile0(P, seg);
+            const int* counters = ctr + P.counter_base + tile0;
+            const int slot0 = ((pi & 1) * kChainMaxSegs + seg) * 2;
+            const long long x0 = (long long)tile * P.ksteps;
+            const int cf = sched.cta_of(x0);
+            const int cl = sched.cta_of(x0 + P.ksteps - 1);
+            const int np = cl - cf + 1, me = (int)blockIdx.x - cf;
+            // A last contributor whose share runs on into the next tile has that tile to finish as well: it is excused here.
+            const int nred = (np > 1 && sched.share_begin(cl + 1) > x0 + P.ksteps) ? np - 1 : np;
+            if (me >= nred) continue;
+            bool failed = false;
+            if (rtid == 0) {
+                const long long t_start = clock64();
+                int seen;
+                do {
+                    asm volatile("ld.acquire.gpu.b32 %0, [%1];" : "=r"(seen) : "l"(counters + tile) : "memory");
+                    if (seen >= np) break;
+                    __nanosleep(40);
+                } while (clock64() - t_start < kWaitBudgetCycles && !bars->abort);
+                if (seen < np) { failed = true; if (!bars->abort) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); } }
+            }
+            // the barrier hands thread 0's acquire on to the other 127 threads, and its verdict with it
+            if (bar_or(3, 128, failed)) break;
+            const bool cf_early = sched.share_begin(cf) < x0;
+            // The parked accumulator is [column group of 4 tokens][128 rows] float4: reducer `me` takes whole column
+            // groups, thread = weight row.  kE groups per round, every piece's loads of a round in flight together
+            // (the loop is a chain of L2 round trips, not bandwidth).
+            const int ncg = ((p.T + 15) / 16) * 4;
+            const int cg_lo = ncg * me / nred, cg_hi = ncg * (me + 1) / nred;
+            const int up_off = (p.n_tile >> 2) * kChainBlockM;
+            constexpr int kE = 4;
+            for (int c0 = cg_lo; c0 < cg_hi; c0 += kE) {
+                float4 g[kE], u[kE];
+#pragma unroll
+                for (int e = 0; e < kE; ++e) g[e] = u[e] = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int cb = cf; cb <= cl; cb += 4) {
+                    float4 a[kE][4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const int cc = cb + q;
+                        if (cc <= cl) {
+                            const int sl = slot0 + ((cc == cf && cf_early) ? 1 : 0);
+                            const float4* part = reinterpret_cast<const float4*>(p.partials + ((size_t)cc * kChainSlots + sl) * slot_floats) + rtid;
+#pragma unroll
+                            for (int e = 0; e < kE; ++e)
+                                if (c0 + e < cg_hi) a[e][q] = __ldcg(part + (c0 + e) * kChainBlockM);
+                        }
+                    }
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        if (cb + q <= cl) {
+#pragma unroll
+                            for (int e = 0; e < kE; ++e)
+                                if (c0 + e < cg_hi) { g[e].x += a[e][q].x; g[e].y += a[e][q].y; g[e].z += a[e][q].z; g[e].w += a[e][q].w; }
+                        }
+                    }
+                    if (accs == 2) {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const int cc = cb + q;
+                            if (cc <= cl) {
+                                const int sl = slot0 + ((cc == cf && cf_early) ? 1 : 0);
+                                const float4* part = reinterpret_cast<const float4*>(p.partials + ((size_t)cc * kChainSlots + sl) * slot_floats) + up_off + rtid;
+#pragma unroll
+                                for (int e = 0; e < kE; ++e)
+                                    if (c0 + e < cg_hi) a[e][q] = __ldcg(part + (c0 + e) * kChainBlockM);
+                            }
+                        }
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            if (cb + q <= cl) {
+#pragma unroll
+                                for (int e = 0; e < kE; ++e)
+                                    if (c0 + e < cg_hi) { u[e].x += a[e][q].x; u[e].y += a[e][q].y; u[e].z += a[e][q].z; u[e].w += a[e][q].w; }
+                            }
+                        }
                     }
                 }
-                if (tr && etid == 0) tr[4 + pi * 8 + 4 + seg] = global_timer_ns();    // segment's output complete in this CTA
+#pragma unroll
+                for (int e = 0; e < kE; ++e) {
+                    if (c0 + e >= cg_hi) break;
+                    const float gf[4] = {g[e].x, g[e].y, g[e].z, g[e].w}, uf[4] = {u[e].x, u[e].y, u[e].z, u[e].w};
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        stage_red[((c0 + e) * 4 + k) * kChainBlockM + rtid] = __float2bfloat16_rn(P.gateup ? chain_silu(gf[k]) * uf[k] : gf[k]);
+                }
+            }
+            asm volatile("bar.sync 3, 128;" ::: "memory");
+            {
+                const int t_lo = cg_lo * 4, t_hi = min(cg_hi * 4, p.T);
+                for (int c = t_lo * 16 + rtid; c < t_hi * 16; c += 128) {
+                    const int t = c >> 4, part = c & 15;
+                    const int n = (tile0 + tile) * kChainBlockM + part * 8;
+                    if (n < P.N)
+                        *reinterpret_cast<uint4*>(P.out + (size_t)t * P.N + n) = *reinterpret_cast<const uint4*>(stage_red + t * kChainBlockM + part * 8);
+                }
+            }
+            asm volatile("bar.sync 3, 128;" ::: "memory");
+        }
+    }
+
+    else if (warp == 11) {
+        // ------------------------------------------------------------ publisher
+        // Releases every parked partial to the other CTAs as soon as the epilogue has posted it: the arrival counter of
+        // its tile is bumped behind a device-wide fence.  Kept apart from the reducers, which may be waiting for another
+        // CTA's partial at that moment - a wait that must never hold back this CTA's own partials.
+        if (lane == 0) {
+            pdl_wait();
+            int* ctr = nullptr;
+            for (int n = 0; n < kChainMaxJobs && !bars->abort; ++n) {
+                if (!mbar_wait(&bars->job_bar[n], 0)) { if (!bars->abort) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); } break; }
+                const int job = bars->job[n];
+                const int kind = (job >> 16) & 0xf, pi = job >> 24, seg = (job >> 20) & 0xf, tile = job & 0xffff;
+                if (kind == kJobExit) break;
+                if (kind != kJobReduce) continue;
+                if (ctr == nullptr) {
+                    const int gen = wait_gen();
+                    if (gen < 0) break;
+                    ctr = p.counters + (size_t)(gen & 1) * kChainCounterInts;
+                }
+                __threadfence();
+                atomicAdd(ctr + p.ph[pi].counter_base + seg_tile0(p.ph[pi], seg) + tile, 1);
             }
         }
     }
@@ -529,12 +687,14 @@ static int chain_enabled() {
     return v;
 }
 
-// A phase whose tiles are all shared along K is one segment by default: cutting it in two halves puts two reductions
-// one behind the other in every CTA's epilogue, and on the W_o projection of the Qwen3-32B-shaped layer that costs more
-// (198.3 us per step) than the half-phase of overlap returns (195.4 us).  AFLEX_CHAIN_SPLIT=1 cuts (tuning).
+// Groups of tiles a phase is cut into when all its tiles are shared along K and another phase follows: the later
+// groups stream while the earlier ones are reduced, and the next phase starts on the earlier groups' columns.
+// Measured on the Qwen3-32B-shaped layer (W_o: 40 tiles, 12 us of streaming): 1 / 2 / 4 groups -> 194.6 / 197.0 /
+// 213.0 us per step.  The phase is too short for it: every group adds up to two parked partials per CTA, and a group's
+// tile is then shared by 15 CTAs instead of 4.  One group is the default; AFLEX_CHAIN_SPLIT = 2 / 4 cuts (tuning).
 static int chain_split() {
     static int v = -1;
-    if (v < 0) { const char* e = getenv("AFLEX_CHAIN_SPLIT"); v = e ? atoi(e) : 0; }
+    if (v < 0) { const char* e = getenv("AFLEX_CHAIN_SPLIT"); v = e ? atoi(e) : 1; if (v < 1) v = 1; if (v > kChainMaxSegs) v = kChainMaxSegs; }
     return v;
 }
 
@@ -558,12 +718,14 @@ aflex_status chain_launch(aflex_ctx* ctx, const ChainStep* steps, int nsteps, in
     p.n_tile = chain_n_tile(T);
     p.box = p.n_tile;
     p.nphase = nsteps;
+    { static int v = -1; if (v < 0) { const char* e = getenv("AFLEX_CHAIN_L2_PHASE"); v = e ? atoi(e) : 1; } p.l2_first_phase = v; }
+    { static int v = -1; if (v < 0) { const char* e = getenv("AFLEX_CHAIN_L2_AHEAD"); v = e ? atoi(e) : 0; if (v < 0) v = 0; if (v > 64) v = 64; } p.l2_ahead = v; }
     int cols = 32;
     while (cols < 2 * 2 * p.n_tile) cols <<= 1;
     p.tmem_cols = cols;
     const int b_bytes = (p.n_tile * kChainBlockK * 2 + 1023) & ~1023;
     const int stage_bytes = 2 * kChainTileBytes + 2 * b_bytes;
-    const int stage_out_bytes = p.n_tile * kChainBlockM * 2;
+    const int stage_out_bytes = 2 * p.n_tile * kChainBlockM * 2;      // one staging buffer each for epilogue and reducers
     const int budget = kMaxDynamicSmem - 1024 - 1024 - stage_out_bytes - 256;
     p.stages = budget / stage_bytes;
     if (p.stages > kChainMaxStages) p.stages = kChainMaxStages;
@@ -583,16 +745,25 @@ aflex_status chain_launch(aflex_ctx* ctx, const ChainStep* steps, int nsteps, in
         const int m_tiles = (s.N + kChainBlockM - 1) / kChainBlockM;
         P.ksteps = P.gateup ? (s.K + kChainBlockK - 1) / kChainBlockK : (s.K + 2 * kChainBlockK - 1) / (2 * kChainBlockK);
         // Segments: the remainder tiles (shared along K) first and the whole tiles second; when no CTA gets a whole
-        // tile, two halves - except in the last phase, whose output nobody in this kernel waits for.
+        // tile, equal groups of tiles - except in the last phase, whose output nobody in this kernel waits for.
         const int grid = ctx->num_sms, whole = m_tiles / grid * grid, rem = m_tiles - whole;
-        if (whole > 0) { P.seg_tiles[0] = rem; P.seg_tiles[1] = whole; }
-        else if (i + 1 < nsteps && chain_split()) { P.seg_tiles[0] = (m_tiles + 1) / 2; P.seg_tiles[1] = m_tiles - P.seg_tiles[0]; }
-        else { P.seg_tiles[0] = m_tiles; P.seg_tiles[1] = 0; }
-        // K steps fed by the previous phase's segment 0 (its tile t is this phase's K columns [128 t, 128 t + 128))
-        if (i == 0) P.n_early = P.ksteps;
+        for (int g = 0; g < kChainMaxSegs; ++g) P.seg_tiles[g] = 0;
+        if (whole > 0) { P.nseg = 2; P.seg_tiles[0] = rem; P.seg_tiles[1] = whole; }
         else {
-            const int e = (P.gateup ? 2 : 1) * p.ph[i - 1].seg_tiles[0];
-            P.n_early = e < P.ksteps ? e : P.ksteps;
+            int ns = (i + 1 < nsteps) ? chain_split() : 1;
+            if (ns > m_tiles) ns = m_tiles;
+            P.nseg = ns;
+            for (int g = 0; g < ns; ++g) P.seg_tiles[g] = m_tiles * (g + 1) / ns - m_tiles * g / ns;
+        }
+        // K steps fed by the previous phase's segments (its tile t is this phase's K columns [128 t, 128 t + 128))
+        if (i == 0) { for (int g = 0; g < kChainMaxSegs; ++g) P.cls_end[g] = P.ksteps; }
+        else {
+            int tiles = 0;
+            for (int g = 0; g < kChainMaxSegs; ++g) {
+                tiles += p.ph[i - 1].seg_tiles[g];
+                const int e = (P.gateup ? 2 : 1) * tiles;
+                P.cls_end[g] = (e < P.ksteps && g + 1 < kChainMaxSegs) ? e : P.ksteps;
+            }
         }
         P.counter_base = base;
         base += m_tiles;

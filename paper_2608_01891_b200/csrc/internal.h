@@ -50,6 +50,7 @@ struct aflex_ctx {
     cudaEvent_t ev_f[aflex::kMaxMicrobatches] = {};   // F_{l,i} done (decoder chain)
     cudaEvent_t ev_f_done = nullptr, ev_a_done = nullptr;
     int attn_ctas = 0;            // persistent attention CTAs per launch; 0 = two per SM
+    unsigned attn_launch_seq = 0; // attention launches so far: picks the launch's pair of chunk-ticket words (four pairs in rotation)
     bool attn_q_final = false;    // caller's promise (aflex_set_attn_q_final): q is never the output of the kernel just before
     bool attn_q_final_once = false;   // set by the layer chains for their own attention launch (q comes from the append kernel)
     bool gemm_attr_set[3] = {false, false, false};
