@@ -590,6 +590,136 @@ def run_targets(args, cfg, wl, ctx, local_rank, device, peaks, stream):
     return out
 
 
+def run_plan(args, cfg, local_rank, device, peaks):
+    """The planner of Section 4.3 ("dynamic microbatch depth", "adaptive request batching") fed with stage-time curves
+    MEASURED on this GPU, and its predictions set against measured chain times.
+
+    1. t_F(rows): the FFN side alone (aflex_ffn_dense / aflex_ffn_moe, back to back) at several row counts.
+    2. t_layer(sub-batch): aflex_decoder_layers at depth 1 on sub-batches (prefixes of the batch, its shortest and
+       its longest sequences); t_A = t_layer - t_F(rows), fitted by least squares as a0 + a1 * context tokens +
+       a2 * rows, which gives the model's two attention curves.
+    3. aflex_pipeline_model with shared_memory_system = 1 (one GPU); for every depth of the configuration
+       aflex_pipeline_makespan's prediction for the near-equal split next to the measured chain time.
+    4. aflex_plan_microbatches: the depth / split it picks over all depths, and the best split at depth 2 alone;
+       both run, and the equal split at depth 2 beside it."""
+    from paper_2608_01891_b200 import aflex as AF
+    L = max(2, args.decoder_layers or 4)
+    B = cfg.batch
+    kvh = IN.make_paged_kv(cfg, device=device)
+    lens_all = kvh.seq_lens.numpy().astype(np.int64)
+    table_d = kvh.page_table.to(device)
+    attn = AF.attn_desc(cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim)
+    descs, caches, keep = [], [], []
+    for l in range(L):
+        w = IN.make_decoder_weights(cfg, l, device=device)
+        layer = AF.layer_desc(attn, cfg.hidden, cfg.inter, w.o, w.gate, w.up, w.down, cfg.num_experts, cfg.top_k, w.router)
+        descs.append(AF.decoder_desc(layer, w.qkv, w.ln_attn, w.ln_ffn, w.q_norm, w.k_norm, cfg.rms_eps, cfg.rope_theta))
+        caches.append((kvh.k_cache, kvh.v_cache) if l == 0 else (kvh.k_cache.clone(), kvh.v_cache.clone()))
+        keep.append(w)
+    ctx = AF.Context(local_rank, max(max(AF.decoder_workspace_bytes(d, B) for d in descs), 1 << 30))
+    stream = torch.cuda.current_stream()
+    x_all = IN.make_hidden(cfg, device=device)
+
+    def time_us(fn, n):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(n):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return 1e3 * e0.elapsed_time(e1) / n
+
+    def chain_us(rows_idx, M, offsets=None):
+        """Microseconds per layer of the chain over the sequences rows_idx (in that order)."""
+        idx = torch.as_tensor(np.asarray(rows_idx, dtype=np.int64))
+        tab = table_d.index_select(0, idx.to(device))
+        ln_h = kvh.seq_lens.index_select(0, idx).contiguous()
+        ln_d = ln_h.to(device)
+        kvs = [AF.make_kv(kc, vc, tab, ln_d, ln_h) for kc, vc in caches]
+        x = x_all.index_select(0, idx.to(device)).contiguous()
+        y = torch.empty_like(x)
+        us = time_us(lambda: ctx.decoder_layers(descs, kvs, x, y, M, offsets, stream), max(5, args.steps // 4))
+        return us / L
+
+    # ---- 1. FFN curve
+    w0 = keep[0]
+    f_rows = sorted({r for r in (8, 16, 32, 64, 128, 256, B // 4, B // 3, B // 2, B) if 1 <= r <= B})
+    f_us = []
+    for r in f_rows:
+        x = x_all[:r].contiguous()
+        y = torch.empty_like(x)
+        if cfg.num_experts == 0:
+            f_us.append(time_us(lambda: ctx.ffn_dense(x, w0.gate, w0.up, w0.down, y, stream), 20))
+        else:
+            f_us.append(time_us(lambda: ctx.ffn_moe(x, w0.gate, w0.up, w0.down, cfg.top_k, y, w_router=w0.router, stream=stream), 20))
+    t_f = lambda r: float(np.interp(r, f_rows, f_us))
+
+    # ---- 2. attention-side fit from depth-1 chain times on sub-batches
+    order = np.argsort(lens_all)
+    subs = []
+    for r in sorted({max(1, B // 8), max(1, B // 4), max(1, B // 2), max(1, 3 * B // 4), B}):
+        subs.append(list(range(r)))
+        if r < B:
+            subs.append(order[:r].tolist())
+            subs.append(order[-r:].tolist())
+    rows_fit, tok_fit, ta_fit, meas_fit = [], [], [], []
+    for sub in subs:
+        us = chain_us(sub, 1)
+        rows_fit.append(len(sub)); tok_fit.append(int(lens_all[sub].sum())); meas_fit.append(us)
+        ta_fit.append(us - t_f(len(sub)))
+    A = np.stack([np.ones(len(subs)), np.asarray(tok_fit, float), np.asarray(rows_fit, float)], axis=1)
+    coef, *_ = np.linalg.lstsq(A, np.asarray(ta_fit), rcond=None)
+    a0, a1, a2 = (float(c) for c in coef)
+    fit_err = float(np.max(np.abs(A @ coef - np.asarray(ta_fit)) / np.asarray(meas_fit)))
+    tok_hi = float(lens_all.sum())
+    model = AF.pipeline_model(([0.0, tok_hi], [a0, a0 + a1 * tok_hi]), ([0.0, float(B)], [0.0, a2 * B]),
+                              ([float(r) for r in f_rows], f_us), 0.0, 0.0, True)
+
+    # ---- 3. prediction against measurement, near-equal splits
+    def equal_offsets(M):
+        base, extra = divmod(B, M)
+        o = [0]
+        for i in range(M):
+            o.append(o[-1] + base + (1 if i < extra else 0))
+        return o
+
+    lens_list = lens_all.tolist()
+    depth_rows = []
+    for M in sorted(set(cfg.microbatch_depths) | {1, 2, 3, 4}):
+        if M > B:
+            continue
+        offs = equal_offsets(M)
+        pred = AF.pipeline_makespan(model, lens_list, offs, L) / L
+        meas = chain_us(list(range(B)), M, offs)
+        depth_rows.append({"M": M, "offsets": offs, "predicted_us_per_layer": round(pred, 1), "measured_us_per_layer": round(meas, 1),
+                           "error": round(pred / meas - 1.0, 4)})
+
+    # ---- 4. what the planner picks
+    gran = max(1, B // 16)
+    M_best, offs_best, pred_best = AF.plan_microbatches(model, lens_list, L, [1, 2, 3, 4], gran)
+    meas_best = chain_us(list(range(B)), M_best, offs_best)
+    _, offs2, pred2 = AF.plan_microbatches(model, lens_list, L, [2], gran)
+    meas2 = chain_us(list(range(B)), 2, offs2)
+    meas2_eq = next(r["measured_us_per_layer"] for r in depth_rows if r["M"] == 2)
+    assert ctx.device_status() == AF.OK
+    line = {"metric": "planner prediction against measured chain time", "unit": "us per layer", "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"config {cfg.cfg_id}: {cfg.name}, {L} chained decoder layers, one GPU (shared memory system)",
+                       "batch": B},
+            "ffn_curve": {"rows": f_rows, "us": [round(v, 1) for v in f_us]},
+            "attention_fit": {"a0_us": round(a0, 2), "us_per_1k_context_tokens": round(a1 * 1e3, 3), "us_per_row": round(a2, 3),
+                              "sub_batches": len(subs), "max_fit_error_of_layer_time": round(fit_err, 4)},
+            "depths": depth_rows,
+            "plan_all_depths": {"M": M_best, "offsets": offs_best, "predicted_us_per_layer": round(pred_best / L, 1),
+                                "measured_us_per_layer": round(meas_best, 1)},
+            "plan_depth_2": {"offsets": offs2, "predicted_us_per_layer": round(pred2 / L, 1), "measured_us_per_layer": round(meas2, 1),
+                             "equal_split_measured_us_per_layer": meas2_eq}}
+    print(json.dumps(line), flush=True)
+    ctx.close()
+
+
 def dataclasses_replace_dense(cfg):
     """The configuration's FFN shape as a dense FFN (MoE configurations: one expert's shape)."""
     import dataclasses
@@ -691,6 +821,10 @@ def main():
     ap.add_argument("--energy-ops", action="store_true",
                     help="instead of the layer step: time and NVML energy per token of attention, the dense FFN at "
                          "T = 32 and T = 2048 and the layer step, each alone, at the clocks the GPU is found at")
+    ap.add_argument("--plan", action="store_true",
+                    help="instead of the layer step: measure the stage-time curves of the configuration on this GPU, feed "
+                         "them to aflex_plan_microbatches / aflex_pipeline_makespan and set the predictions against "
+                         "measured aflex_decoder_layers times at every depth; prints one JSON line")
     ap.add_argument("--prefill", action="store_true",
                     help="instead of the layer step: prefill (causal) attention at the configuration's head shape over "
                          "several prompt mixes, TFLOP/s against the measured bf16 peaks")
@@ -738,13 +872,17 @@ def main():
         if rank == 0:
             (run_moe_sweep if cfg.num_experts > 0 else run_ffn_sweep)(args, cfg, local_rank, device, peaks)
         return
-    if args.decoder_layers > 0:
+    if args.decoder_layers > 0 and not args.plan:
         if rank == 0:
             run_decoder_chain(args, cfg, local_rank, device, peaks)
         return
     if args.energy_ops:
         if rank == 0:
             run_energy_ops(args, cfg, local_rank, device, peaks)
+        return
+    if args.plan:
+        if rank == 0:
+            run_plan(args, cfg, local_rank, device, peaks)
         return
     if args.prefill:
         if rank == 0:

@@ -243,6 +243,31 @@ def test_decoder_layers_match_oracle(cfg, L):
         ctx.close()
 
 
+def test_decoder_layers_with_planner_chosen_unequal_split_match_oracle():
+    """The split aflex_plan_microbatches picks is handed to aflex_decoder_layers as it comes.  With stage times
+    proportional to the work, the FFN side twice as slow as the attention side and one layer on separate pools, the
+    best two-microbatch split puts a third of the rows first (closed form pinned in the control-oracle tests): an
+    unequal, planner-made split.  The chain's result with it equals the oracle's, and (to rounding of the differently
+    sized GEMM launches) the depth-1 result."""
+    cfg = IN.LayerConfig(13, "tiny-plan", 12, 8, 2, 64, 256, 384, len_dist="uniform", len_lo=20, len_hi=90)
+    ch = Chain(cfg, 2)
+    lens = ch.kvh.seq_lens.numpy().tolist()
+    tokens = float(sum(lens))
+    model = AF.pipeline_model(([0.0, tokens], [0.0, 120.0]), ([0.0], [0.0]), ([0.0, 12.0], [0.0, 240.0]))
+    M, offsets, _ = AF.plan_microbatches(model, lens, 1, [2])
+    assert M == 2 and offsets[0] == 0 and offsets[2] == cfg.batch and 0 < offsets[1] < cfg.batch
+    assert offsets[1] != cfg.batch // 2                     # not the equal split
+    ctx = AF.Context(0, ch.workspace())
+    try:
+        outs, _, _ = ch.oracle()
+        got = _run_chain(ctx, ch, M, offsets)
+        assert row_rel_err(f64(got), outs[-1]) <= TOL_FFN * 2
+        one = _run_chain(ctx, ch, 1)
+        assert row_rel_err(f64(got), f64(one)) <= 1e-2
+    finally:
+        ctx.close()
+
+
 def test_decoder_layers_attention_sees_the_token_it_just_appended():
     """Sequences of 1-3 tokens: the appended K/V carries most of the softmax weight, so an attention
     that read the cache before the append would be far off."""
