@@ -720,6 +720,114 @@ def run_plan(args, cfg, local_rank, device, peaks):
     ctx.close()
 
 
+def af_pair_devices(world: int, rank: int, local_rank: int, device_count: int):
+    """Which GPUs the A/F pair measurement uses in a multi-GPU run: rank 0 alone drives it, with the Attention side on
+    its own GPU and the FFN side on the next local one; every other rank only waits.  Returns (attention device, FFN
+    device) for the rank that runs it, None for the ranks that wait, and a reason string when nobody runs it."""
+    if world < 2:
+        return "one GPU: not run (the pair needs two devices; both sides on one GPU are covered by the tests)"
+    if device_count < 2:
+        return "fewer than two visible devices: not run"
+    if rank != 0:
+        return None
+    return (local_rank, (local_rank + 1) % device_count)
+
+
+def wait_for_rank0(dist, host_group):
+    """Host-side rendezvous (gloo) behind the replica timing: the other ranks block here, off the GPU, while rank 0
+    measures the A/F pair on its own GPU and its neighbour's."""
+    dist.barrier(group=host_group)
+
+
+def run_af_pair_record(cfg, dev_a: int, dev_f: int, L: int, steps: int):
+    """One A/F pair inside a node (the paper's data plane, Section 4.3): Attention side on GPU dev_a, FFN side on GPU
+    dev_f, hidden states handed over by peer copies.  Per microbatch depth: microseconds per layer, checked bit for bit
+    against the same call with both contexts on dev_a; the measured time of one hand-over copy; Eq. 2's prediction
+    with the measured per-side kernel times and that t_comm."""
+    from paper_2608_01891_b200 import aflex as AF
+    da, df = f"cuda:{dev_a}", f"cuda:{dev_f}"
+    torch.cuda.set_device(dev_a)
+    kvh = IN.make_paged_kv(cfg, device=da)
+    table, lens = kvh.page_table.to(da), kvh.seq_lens.to(da)
+    attn = AF.attn_desc(cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim)
+    descs_pair, descs_one, kvs, keep = [], [], [], []
+    for l in range(L):
+        w = IN.make_decoder_weights(cfg, l, device=da)
+        f_side = [w.gate, w.up, w.down, w.ln_ffn, w.router]
+        f_far = [None if t is None else t.to(df) for t in f_side] if dev_f != dev_a else f_side
+        one = AF.layer_desc(attn, cfg.hidden, cfg.inter, w.o, w.gate, w.up, w.down, cfg.num_experts, cfg.top_k, w.router)
+        far = AF.layer_desc(attn, cfg.hidden, cfg.inter, w.o, f_far[0], f_far[1], f_far[2], cfg.num_experts, cfg.top_k, f_far[4])
+        descs_one.append(AF.decoder_desc(one, w.qkv, w.ln_attn, w.ln_ffn, w.q_norm, w.k_norm, cfg.rms_eps, cfg.rope_theta))
+        descs_pair.append(AF.decoder_desc(far, w.qkv, w.ln_attn, f_far[3], w.q_norm, w.k_norm, cfg.rms_eps, cfg.rope_theta))
+        kc, vc = (kvh.k_cache, kvh.v_cache) if l == 0 else (kvh.k_cache.clone(), kvh.v_cache.clone())
+        kvs.append(AF.make_kv(kc, vc, table, lens, kvh.seq_lens))
+        keep.append((w, f_far, kc, vc))
+    x = IN.make_hidden(cfg, device=da)
+    y_pair, y_one = torch.empty_like(x), torch.empty_like(x)
+    ctx_a = AF.Context(dev_a, max(AF.af_workspace_bytes(d, cfg.batch, False) for d in descs_pair))
+    ctx_f = AF.Context(dev_f, max(AF.af_workspace_bytes(d, cfg.batch, True) for d in descs_pair))
+    ctx_f1 = AF.Context(dev_a, max(AF.af_workspace_bytes(d, cfg.batch, True) for d in descs_one))
+    torch.cuda.set_device(dev_a)
+    stream = torch.cuda.current_stream()
+
+    def time_us(fn, n):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize(dev_a); torch.cuda.synchronize(dev_f)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(n):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize(dev_a); torch.cuda.synchronize(dev_f)
+        return 1e3 * e0.elapsed_time(e1) / n
+
+    rows = []
+    for M in (1, 2, 4):
+        if M > cfg.batch:
+            continue
+        AF.af_decoder_layers(ctx_a, ctx_f1, descs_one, kvs, x, y_one, M, None, stream)      # both sides on dev_a
+        torch.cuda.synchronize(dev_a)
+        AF.af_decoder_layers(ctx_a, ctx_f, descs_pair, kvs, x, y_pair, M, None, stream)     # the pair
+        torch.cuda.synchronize(dev_a); torch.cuda.synchronize(dev_f)
+        same = bool(torch.equal(y_one.view(torch.int16), y_pair.view(torch.int16)))
+        us = time_us(lambda: AF.af_decoder_layers(ctx_a, ctx_f, descs_pair, kvs, x, y_pair, M, None, stream), steps) / L
+        # per-side kernel time of one layer (event pair around every launch; no overlap counted)
+        ctx_a.profile_enable(True); ctx_f.profile_enable(True)
+        AF.af_decoder_layers(ctx_a, ctx_f, descs_pair, kvs, x, y_pair, M, None, stream)
+        torch.cuda.synchronize(dev_a); torch.cuda.synchronize(dev_f)
+        t_a = 1e3 * sum(v[0] for v in ctx_a.profile_read().values()) / L
+        torch.cuda.set_device(dev_f)
+        t_f = 1e3 * sum(v[0] for v in ctx_f.profile_read().values()) / L
+        torch.cuda.set_device(dev_a)
+        ctx_a.profile_enable(False); ctx_f.profile_enable(False)
+        # one hand-over: [rows of a microbatch][H] bf16 from the attention GPU into the FFN GPU's memory
+        r = -(-cfg.batch // M)
+        src = torch.empty(r, cfg.hidden, dtype=torch.bfloat16, device=da)
+        dst = torch.empty(r, cfg.hidden, dtype=torch.bfloat16, device=df)
+        # (20 copies captured into a CUDA graph, so that the device time of a copy is measured, not the host's issue rate)
+        g = torch.cuda.CUDAGraph()
+        cap = torch.cuda.Stream(device=da)
+        cap.wait_stream(stream)
+        with torch.cuda.graph(g, stream=cap):
+            for _ in range(20):
+                dst.copy_(src, non_blocking=True)
+        stream.wait_stream(cap)
+        t_copy = time_us(g.replay, 10) / 20
+        t_comm = 2.0 * M * t_copy                          # Eq. 2's t_comm: the whole batch, both directions
+        rows.append({"M": M, "us_per_layer": round(us, 1), "bit_identical_to_one_gpu_pair": same,
+                     "t_a_us": round(t_a, 1), "t_f_us": round(t_f, 1), "copy_us_per_boundary": round(t_copy, 2),
+                     "eq2_prediction_us": round(AF.eq2_layer_time(t_a, t_f, t_comm, M), 1)})
+    ok = ctx_a.device_status() == AF.OK
+    torch.cuda.set_device(dev_f)
+    ok = ok and ctx_f.device_status() == AF.OK
+    torch.cuda.set_device(dev_a)
+    for c in (ctx_f1, ctx_f, ctx_a):
+        c.close()
+    return {"config": cfg.cfg_id, "layers": L, "attention_gpu": dev_a, "ffn_gpu": dev_f, "device_status_ok": ok,
+            "transfer": "cudaMemcpyPeerAsync into the consumer's own memory; no kernel reads peer memory", "depths": rows}
+
+
 def dataclasses_replace_dense(cfg):
     """The configuration's FFN shape as a dense FFN (MoE configurations: one expert's shape)."""
     import dataclasses
@@ -821,6 +929,10 @@ def main():
     ap.add_argument("--energy-ops", action="store_true",
                     help="instead of the layer step: time and NVML energy per token of attention, the dense FFN at "
                          "T = 32 and T = 2048 and the layer step, each alone, at the clocks the GPU is found at")
+    ap.add_argument("--af-pair-record", type=int, default=-1, metavar="FFN_GPU",
+                    help="instead of the layer step: the A/F pair record of the multi-GPU run (configuration 3, 4 layers, "
+                         "depths 1 / 2 / 4) with the attention side on this GPU and the FFN side on GPU FFN_GPU (the "
+                         "same GPU is allowed); prints one JSON line")
     ap.add_argument("--plan", action="store_true",
                     help="instead of the layer step: measure the stage-time curves of the configuration on this GPU, feed "
                          "them to aflex_plan_microbatches / aflex_pipeline_makespan and set the predictions against "
@@ -863,9 +975,11 @@ def main():
     torch.cuda.set_device(local_rank)
     device = f"cuda:{local_rank}"
     dist = None
+    host_group = None
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device(device))
+        host_group = dist.new_group(backend="gloo")       # host-side rendezvous for the part only rank 0 runs
 
     peaks = load_peaks()
     if args.ffn_sweep:
@@ -883,6 +997,12 @@ def main():
     if args.plan:
         if rank == 0:
             run_plan(args, cfg, local_rank, device, peaks)
+        return
+    if args.af_pair_record >= 0:
+        if rank == 0:
+            print(json.dumps({"metric": "A/F pair across GPUs: us per decoder layer", "unit": "us", "dtype": "bf16",
+                              "data": "synthetic", "af_pair": run_af_pair_record(IN.CONFIGS[3 if args.config == 2 else args.config],
+                                                                                  local_rank, args.af_pair_record, 4, args.steps // 5 or 5)}), flush=True)
         return
     if args.prefill:
         if rank == 0:
@@ -1125,6 +1245,20 @@ def main():
             O.set_num_threads(threads)
             cpu["value_1_thread"] = len(rows) / dt1
 
+    # ---- the A/F pair across two GPUs (N >= 2 only): rank 0 drives its own GPU and the next one, the others wait on the host
+    af_pair = af_pair_devices(world, rank, local_rank, torch.cuda.device_count())
+    if world > 1:
+        barrier()                                          # every rank has finished its replica work
+        if isinstance(af_pair, tuple):
+            del wl
+            torch.cuda.empty_cache()
+            try:
+                af_pair = run_af_pair_record(IN.CONFIGS[3], af_pair[0], af_pair[1], 4, 10)
+            except Exception as exc:                       # never lose the headline line to the extra record
+                af_pair = {"failed": str(exc)[:300]}
+            torch.cuda.set_device(local_rank)
+        wait_for_rank0(dist, host_group)
+
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
@@ -1141,6 +1275,7 @@ def main():
             line["energy"] = energy
         if targets is not None:
             line["targets"] = targets
+        line["af_pair"] = af_pair
         print(json.dumps(line), flush=True)
     ctx.close()
     if dist is not None:
