@@ -915,6 +915,9 @@ def main():
     ap.add_argument("--ref-rows", type=int, default=0,
                     help="batch rows per reference/cpu-baseline sample (0 = about 15e9 multiply-adds of oracle work)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--quick", action="store_true",
+                    help="only the warm-up and the timed steps of the layer step, then a short JSON line (value, ms_per_step, "
+                         "gpu_launches): a small run with few launches, for a profiler")
     ap.add_argument("--ffn-sweep", action="store_true",
                     help="instead of the layer step: dense FFN (aflex_ffn_dense) at the configuration's weight shape "
                          "for T = 32..8192 tokens, TFLOP/s against the measured bf16 peak; prints one JSON line")
@@ -1051,6 +1054,19 @@ def main():
     sampler.start()
     ms_total = timed(step, args.steps)
     launches = ctx.launch_count() - launches0
+    if args.quick:
+        sampler.stop()
+        torch.cuda.synchronize()
+        assert ctx.device_status() == AF.OK, ctx.last_error()
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": whole_job_tokens_per_s(world, cfg.batch, ms_total / args.steps),
+                              "unit": "tokens/s", "ms_per_step": ms_total / args.steps, "steps": args.steps, "warmup": args.warmup,
+                              "gpu_launches": int(launches), "config": {"workload": f"config {cfg.cfg_id}: {cfg.name}", "quick": True}}),
+                  flush=True)
+        ctx.close()
+        if dist is not None:
+            dist.destroy_process_group()
+        return
     # the timed region can be shorter than one nvidia-smi sampling period: keep the same load
     # running (untimed) until the sampler has seen it
     if ms_total < 500:
@@ -1087,7 +1103,10 @@ def main():
         tr = json.load(open(ncu_traffic))
         key = f"config{cfg.cfg_id}/{dom}"
         if key in tr:
-            roofline["traffic"] = tr[key]
+            # one single-kernel, single-launch ncu capture of this kernel on this workload; the record says which
+            # commit's kernels were captured and how
+            roofline["traffic"] = tr[key]["bytes"]
+            roofline["traffic_source"] = {k: tr[key][k] for k in ("kernels_at_commit", "capture", "summary")}
 
     # ---- the two operators on their own: back-to-back calls of the public entry points over TWO alternating buffer
     #      sets (two copies of the KV cache for attention, two copies of the FFN weights), so that no launch can find
