@@ -165,6 +165,38 @@ static aflex_status dense_run(aflex_ctx* ctx, const void* x, const void* wg, con
     return linear_launch(ctx, h, wd, T, I, H, y, sws, scratch, st, kKDownGemm, ctx->counters_f);
 }
 
+// Decode batch, dense FFN, whole decoder layer: the output projection, the residual add, the RMS normalisation in
+// front of the FFN and the FFN itself as ONE chain launch.  a [T][A] is the attention output; resid [T][H] is updated in
+// place (resid += a W_o^T); xg [T][H] is scratch (the gain-weighted residual rows, the FFN's input before the row scale).
+// With next_qkv: the down projection's output is added to the residual rows as well, normalised for the NEXT layer
+// (gain next_gain, rows left in xn) and pushed through that layer's QKV projection (w_qkv [NQ][H] -> qkv [T][NQ]); y is
+// then not written.
+static aflex_status dense_fused_run(aflex_ctx* ctx, const void* a, const void* w_o, int A, void* resid, const void* gain, float eps,
+                                    void* xg, const void* wg, const void* wu, const void* wd, int T, int H, int I, void* y,
+                                    char* ws, size_t ws_bytes, cudaStream_t st, const void* next_gain = nullptr,
+                                    float next_eps = 0.f, void* xn = nullptr, const void* w_qkv = nullptr, int NQ = 0,
+                                    void* qkv = nullptr) {
+    Arena arena(ws, ws_bytes);
+    __nv_bfloat16* h = arena.take<__nv_bfloat16>((size_t)T * I);
+    const size_t scratch = chain_workspace_bytes(T, ctx->num_sms);
+    char* sws = arena.take<char>(scratch);
+    if (arena.overflow)
+        return set_error(ctx, AFLEX_ERR_WORKSPACE, "fused dense layer: need %zu workspace bytes, have %zu",
+                         dense_ws_bytes(T, H, I, ctx->num_sms), ws_bytes);
+    ChainStep steps[4];
+    steps[0] = ChainStep{a, w_o, nullptr, A, H, xg};
+    steps[0].resid_in = resid; steps[0].resid_out = resid; steps[0].gain = gain; steps[0].eps = eps;
+    steps[1] = ChainStep{xg, wg, wu, H, I, h};
+    if (w_qkv == nullptr) {
+        steps[2] = ChainStep{h, wd, nullptr, I, H, y};
+        return chain_launch(ctx, steps, 3, T, sws, scratch, st, ctx->chain_counters);
+    }
+    steps[2] = ChainStep{h, wd, nullptr, I, H, xn};
+    steps[2].resid_in = resid; steps[2].resid_out = resid; steps[2].gain = next_gain; steps[2].eps = next_eps;
+    steps[3] = ChainStep{xn, w_qkv, nullptr, H, NQ, qkv};
+    return chain_launch(ctx, steps, 4, T, sws, scratch, st, ctx->chain_counters);
+}
+
 static size_t moe_ws_bytes(int T, int H, int I, int E, int K, int num_sms) {
     const size_t R = (size_t)T * K;
     size_t b = 0;
@@ -660,6 +692,13 @@ aflex_status aflex_layer_step(aflex_ctx* ctx, const aflex_layer_desc* L, const v
     return check_cuda(ctx, e, "layer step: exit join");
 }
 
+// AFLEX_DECODER_FUSE=0: keep W_o, the residual add + RMS normalisation and the FFN as separate launches (tuning / comparison).
+static bool decoder_fuse() {
+    static int v = -1;
+    if (v < 0) { const char* e = getenv("AFLEX_DECODER_FUSE"); v = e ? atoi(e) : 1; }
+    return v != 0;
+}
+
 // ---- whole decoder layers ------------------------------------------------------------------
 // Workspace: [A scratch | resid | xn | qkv | q | a | o | xn2 | y | F scratch].  The row-indexed
 // buffers are touched by microbatch i only in rows of i, in the order A_{l,i} -> F_{l,i} ->
@@ -826,11 +865,26 @@ aflex_status aflex_decoder_layers(aflex_ctx* ctx, const aflex_decoder_desc* laye
                 e = cudaStreamWaitEvent(sa, ctx->ev_f[i], 0);     // F_{l-1,i} has returned this microbatch
                 if (e != cudaSuccess) return check_cuda(ctx, e, "decoder layers: F->A event");
             }
-            if (l == 0) s = add_rmsnorm_launch(ctx, reinterpret_cast<const bf*>(x_in) + oh, nullptr, d->w_ln_attn, rows, H, d->rms_eps, resid + oh, xn + oh, sa);
-            else s = add_rmsnorm_launch(ctx, resid + oh, yb + oh, d->w_ln_attn, rows, H, d->rms_eps, resid + oh, xn + oh, sa);
-            if (s != AFLEX_OK) return s;
-            s = linear_launch(ctx, xn + oh, d->w_qkv, rows, H, NQ, qkv + (size_t)r0 * NQ, ws_lin, w.a_lin, sa, kKQkvGemm, ctx->counters_a);
-            if (s != AFLEX_OK) return s;
+            // Decode batch with a dense FFN: W_o, the residual add, the FFN's RMS normalisation and the FFN are one chain
+            // launch on the FFN stream (the hand-over event then sits behind the attention kernel); when the next layer is
+            // of the same kind, the chain goes on through the FFN's residual add, that layer's first normalisation and its
+            // QKV projection, so that a layer is three launches: rotary + append, attention, the chain.
+            auto can_fuse = [&](int k) { return layers[k].layer.num_experts == 0 && chain_supported(rows) && decoder_fuse(); };
+            auto same_shape = [&](int k0, int k1) {      // same workspace layout, so one layer's chain can fill the next one's buffers
+                const aflex_layer_desc &x = layers[k0].layer, &y = layers[k1].layer;
+                return x.attn.num_q_heads == y.attn.num_q_heads && x.attn.num_kv_heads == y.attn.num_kv_heads &&
+                       x.attn.head_dim == y.attn.head_dim && x.hidden == y.hidden && x.inter == y.inter;
+            };
+            const bool fused = can_fuse(l);
+            const bool qkv_done = l > 0 && can_fuse(l - 1) && fused && same_shape(l - 1, l);      // the previous layer's chain made xn and qkv
+            const bool fuse_next = fused && l + 1 < num_layers && can_fuse(l + 1) && same_shape(l, l + 1);
+            if (!qkv_done) {
+                if (l == 0) s = add_rmsnorm_launch(ctx, reinterpret_cast<const bf*>(x_in) + oh, nullptr, d->w_ln_attn, rows, H, d->rms_eps, resid + oh, xn + oh, sa);
+                else s = add_rmsnorm_launch(ctx, resid + oh, yb + oh, d->w_ln_attn, rows, H, d->rms_eps, resid + oh, xn + oh, sa);
+                if (s != AFLEX_OK) return s;
+                s = linear_launch(ctx, xn + oh, d->w_qkv, rows, H, NQ, qkv + (size_t)r0 * NQ, ws_lin, w.a_lin, sa, kKQkvGemm, ctx->counters_a);
+                if (s != AFLEX_OK) return s;
+            }
             aflex_kv kvi = kvs[l];
             kvi.page_table = kvs[l].page_table + (size_t)r0 * kvs[l].max_pages_per_seq;
             kvi.seq_lens = kvs[l].seq_lens + r0;
@@ -840,17 +894,28 @@ aflex_status aflex_decoder_layers(aflex_ctx* ctx, const aflex_decoder_desc* laye
             ctx->attn_q_final_once = true;      // q was written by the append kernel, which does not release its dependents early
             s = attn_decode_launch(ctx, &L->attn, qb + (size_t)r0 * A, &kvi, rows, ab + (size_t)r0 * A, nullptr, ws_attn, w.a_attn, sa);
             if (s != AFLEX_OK) return s;
-            s = linear_launch(ctx, ab + (size_t)r0 * A, L->w_o, rows, A, H, ob + oh, ws_lin, w.a_lin, sa, kKLinearGemm, ctx->counters_a);
-            if (s != AFLEX_OK) return s;
+            if (!fused) {
+                s = linear_launch(ctx, ab + (size_t)r0 * A, L->w_o, rows, A, H, ob + oh, ws_lin, w.a_lin, sa, kKLinearGemm, ctx->counters_a);
+                if (s != AFLEX_OK) return s;
+            }
             if (!serial) {
                 e = cudaEventRecord(ctx->ev_a[i], sa);
                 if (e == cudaSuccess) e = cudaStreamWaitEvent(sf, ctx->ev_a[i], 0);
                 if (e != cudaSuccess) return check_cuda(ctx, e, "decoder layers: A->F event");
             }
             // ---- F_{l,i}
-            s = add_rmsnorm_launch(ctx, resid + oh, ob + oh, d->w_ln_ffn, rows, H, d->rms_eps, resid + oh, xn2 + oh, sf);
-            if (s != AFLEX_OK) return s;
-            if (E == 0) s = dense_run(ctx, xn2 + oh, L->w_gate, L->w_up, L->w_down, rows, H, I, yb + oh, ws_f, w.f_total, sf);
+            if (fused) {
+                const aflex_decoder_desc* dn = fuse_next ? &layers[l + 1] : nullptr;
+                const int NQn = dn ? (dn->layer.attn.num_q_heads + 2 * dn->layer.attn.num_kv_heads) * dn->layer.attn.head_dim : 0;
+                s = dense_fused_run(ctx, ab + (size_t)r0 * A, L->w_o, A, resid + oh, d->w_ln_ffn, d->rms_eps, xn2 + oh, L->w_gate, L->w_up,
+                                    L->w_down, rows, H, I, yb + oh, ws_f, w.f_total, sf, dn ? dn->w_ln_attn : nullptr, dn ? dn->rms_eps : 0.f,
+                                    xn + oh, dn ? dn->w_qkv : nullptr, NQn, dn ? qkv + (size_t)r0 * NQn : nullptr);
+            } else {
+                s = add_rmsnorm_launch(ctx, resid + oh, ob + oh, d->w_ln_ffn, rows, H, d->rms_eps, resid + oh, xn2 + oh, sf);
+                if (s != AFLEX_OK) return s;
+            }
+            if (fused) {}
+            else if (E == 0) s = dense_run(ctx, xn2 + oh, L->w_gate, L->w_up, L->w_down, rows, H, I, yb + oh, ws_f, w.f_total, sf);
             else s = moe_run(ctx, xn2 + oh, nullptr, L->w_router, L->w_gate, L->w_up, L->w_down, rows, H, I, E, L->top_k, yb + oh,
                              nullptr, nullptr, nullptr, ws_f, w.f_total, sf);
             if (s != AFLEX_OK) return s;

@@ -57,12 +57,13 @@ constexpr int kChainBlockM = 128;
 constexpr int kChainBlockK = 64;
 constexpr int kChainTileBytes = kChainBlockM * kChainBlockK * 2;   // one weight tile: 16 KB
 constexpr int kChainMaxStages = 8;
-constexpr int kChainMaxPhases = 3;
+constexpr int kChainMaxPhases = 4;
 constexpr int kChainMaxSegs = 4;
 constexpr long long kChainIdleCycles = 4000;   // a wait for a free ring stage this long (~2 us) is a stall, not back-pressure
 constexpr int kChainSlots = 2 * kChainMaxSegs * 2;   // partial slots per CTA: [phase parity][segment][first / later unit]
 constexpr int kChainCounterInts = 8192;   // per half of the double-buffered counter array: per-tile counters, then the epoch words
 constexpr int kChainEpochBase = kChainCounterInts - 16;
+constexpr int kChainMaxStatTiles = 512;    // tiles of a phase with the residual + normalisation epilogue (N <= 65536)
 constexpr int kChainMaxJobs = 64;          // reduce jobs one CTA can post in a launch (<= 2 per segment, plus markers)
 
 struct ChainPhase {
@@ -76,6 +77,15 @@ struct ChainPhase {
                                     // (non-decreasing, last = ksteps; first phase: everything is class 0)
     int counter_base;  // first per-tile arrival counter of this phase
     __nv_bfloat16* out;   // [T][N]
+    // Residual + normalisation epilogue (a linear phase in front of a normalised consumer): with o = bf16(in . w^T),
+    //   resid_out = bf16(o + resid_in),  out = bf16(resid_out * gain),  ss[tile][t] = sum over the tile's features of resid_out^2
+    // and the NEXT phase multiplies its accumulators by rsqrt(sum_tiles ss / N + eps) per token row: RMS normalisation
+    // with the row scale moved behind the GEMM, where it commutes ((r x) W^T = r (x W^T)).  gain == nullptr: off.
+    const __nv_bfloat16* resid_in;    // [T][N] (may alias resid_out)
+    __nv_bfloat16* resid_out;         // [T][N]
+    const __nv_bfloat16* gain;        // [N]
+    float eps;
+    int scale_rows;    // 1: this phase's accumulators take the per-row scale from the previous phase's statistics
 };
 
 struct ChainParams {
@@ -89,6 +99,7 @@ struct ChainParams {
     int l2_ahead;      // ring stages' worth of weights the idle weight producer may prefetch into L2 beyond the ring (0 = off)
     ChainPhase ph[kChainMaxPhases];
     float* partials;   // [grid][kChainSlots][2 * n_tile / 4][128 rows] float4
+    float* ss_part;    // [tiles of the normalised phase][n_tile]: per-tile sums of squares of the residual stream rows
     int* counters;     // two halves of kChainCounterInts ints, then the generation word.  A launch of generation g counts
                        // in half g & 1 (per-tile arrival counters and, at kChainEpochBase, its epoch words: (phase, segment)
                        // finished by so many CTAs; all zero on entry), zeroes the other half for its
@@ -165,6 +176,8 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const ChainParams p) {
     // [token][128 features] bf16, so that it leaves the SM in 16-byte pieces
     __nv_bfloat16* stage_epi = reinterpret_cast<__nv_bfloat16*>(smem + (size_t)p.stages * stage_bytes + 1024);
     __nv_bfloat16* stage_red = stage_epi + (size_t)p.n_tile * kChainBlockM;
+    float* rinv_epi = reinterpret_cast<float*>(stage_red + (size_t)p.n_tile * kChainBlockM);   // per-row scales, one copy per group
+    float* rinv_red = rinv_epi + 64;
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -206,6 +219,85 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const ChainParams p) {
         while ((gen = bars->gen) < 0 && !bars->abort && clock64() - t_start < kWaitBudgetCycles) __nanosleep(20);
         if (gen < 0 && !bars->abort) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); }
         return gen;
+    };
+
+    // Token rows [t_lo, t_hi) of a staged output tile -> memory, 16 bytes per thread and store.  `tid` = 0..127 inside
+    // the calling group (epilogue or reducers).  With the residual + normalisation epilogue the same pass adds the
+    // residual rows, writes them back, writes the gain-weighted rows for the next phase and reduces every row's sum of
+    // squares over the tile's 128 features (16 lanes hold one token row: a fixed-order shuffle reduction).
+    auto store_tokens = [&](const ChainPhase& P, const __nv_bfloat16* stage, int tile_g, int t_lo, int t_hi, int tid) {
+        if (t_hi > p.T) t_hi = p.T;
+        if (P.gain == nullptr) {
+            for (int c = t_lo * 16 + tid; c < t_hi * 16; c += 128) {
+                const int t = c >> 4, part = c & 15;
+                const int n = tile_g * kChainBlockM + part * 8;
+                if (n < P.N)
+                    *reinterpret_cast<uint4*>(P.out + (size_t)t * P.N + n) = *reinterpret_cast<const uint4*>(stage + t * kChainBlockM + part * 8);
+            }
+            return;
+        }
+        for (int c0 = t_lo * 16; c0 < t_hi * 16; c0 += 128) {
+            const int c = c0 + tid;
+            const int t = c >> 4, part = c & 15;
+            const int n = tile_g * kChainBlockM + part * 8;
+            const bool on = c < t_hi * 16 && n < P.N;
+            float ss = 0.f;
+            if (on) {
+                const uint4 o8 = *reinterpret_cast<const uint4*>(stage + t * kChainBlockM + part * 8);
+                const uint4 r8 = __ldcg(reinterpret_cast<const uint4*>(P.resid_in + (size_t)t * P.N + n));
+                const uint4 g8 = *reinterpret_cast<const uint4*>(P.gain + n);
+                const __nv_bfloat162* po = reinterpret_cast<const __nv_bfloat162*>(&o8);
+                const __nv_bfloat162* pr = reinterpret_cast<const __nv_bfloat162*>(&r8);
+                const __nv_bfloat162* pg = reinterpret_cast<const __nv_bfloat162*>(&g8);
+                uint4 res, xg;
+                __nv_bfloat162* ps = reinterpret_cast<__nv_bfloat162*>(&res);
+                __nv_bfloat162* px = reinterpret_cast<__nv_bfloat162*>(&xg);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const float2 fo = __bfloat1622float2(po[k]), fr = __bfloat1622float2(pr[k]), fg = __bfloat1622float2(pg[k]);
+                    ps[k] = __floats2bfloat162_rn(fo.x + fr.x, fo.y + fr.y);
+                    const float2 v = __bfloat1622float2(ps[k]);        // the residual stream as stored
+                    ss = fmaf(v.x, v.x, ss);
+                    ss = fmaf(v.y, v.y, ss);
+                    px[k] = __floats2bfloat162_rn(v.x * fg.x, v.y * fg.y);
+                }
+                *reinterpret_cast<uint4*>(P.resid_out + (size_t)t * P.N + n) = res;
+                *reinterpret_cast<uint4*>(P.out + (size_t)t * P.N + n) = xg;
+            }
+#pragma unroll
+            for (int off = 8; off > 0; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
+            if (c < t_hi * 16 && part == 0) p.ss_part[(size_t)tile_g * p.n_tile + t] = ss;
+        }
+    };
+    // The per-row scales of a phase whose input was left un-normalised by the previous phase: waits (bounded) until every
+    // segment of that phase is complete everywhere, then sums each row's per-tile statistics in tile order.  Called by
+    // all 128 threads of a group; false = gave up (uniformly).
+    auto load_row_scales = [&](int pi, const int* ctr, float* rinv, int tid, int bar_id) -> bool {
+        const ChainPhase& Q = p.ph[pi - 1];
+        bool failed = false;
+        if (tid == 0) {
+            for (int g = 0; g < Q.nseg && !failed; ++g) {
+                const long long t_start = clock64();
+                int seen;
+                do {
+                    asm volatile("ld.acquire.gpu.b32 %0, [%1];" : "=r"(seen) : "l"(ctr + kChainEpochBase + (pi - 1) * kChainMaxSegs + g) : "memory");
+                    if (seen >= grid) break;
+                    __nanosleep(40);
+                } while (clock64() - t_start < kWaitBudgetCycles && !bars->abort);
+                if (seen < grid) { failed = true; if (!bars->abort) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); } }
+            }
+        }
+        if (bar_or(bar_id, 128, failed)) return false;
+        if (tid < p.n_tile) {
+            int tiles = 0;
+            for (int g = 0; g < Q.nseg; ++g) tiles += Q.seg_tiles[g];
+            float ssum = 0.f;
+            for (int m = 0; m < tiles; ++m) ssum += __ldcg(p.ss_part + (size_t)m * p.n_tile + tid);
+            rinv[tid] = rsqrtf(ssum / (float)Q.N + Q.eps);
+        }
+        if (bar_id == 2) asm volatile("bar.sync 2, 128;" ::: "memory");
+        else asm volatile("bar.sync 3, 128;" ::: "memory");
+        return true;
     };
 
     if (warp == 0) {
@@ -436,6 +528,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const ChainParams p) {
         for (int pi = 0; pi < p.nphase && !gave_up; ++pi) {
             const ChainPhase& P = p.ph[pi];
             const int accs = P.gateup ? 2 : 1;
+            if (P.scale_rows && !load_row_scales(pi, ctr, rinv_epi, etid, 2)) { gave_up = true; break; }
             for (int seg = 0; seg < P.nseg && !gave_up; ++seg) {
                 const Schedule sched(P.ksteps, 1, P.seg_tiles[seg], grid);
                 const int tile0 = seg_tile0(P, seg);
@@ -461,7 +554,9 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const ChainParams p) {
                             tmem_ld_wait();
 #pragma unroll
                             for (int j = 0; j < 16; ++j) {
-                                const float v = P.gateup ? chain_silu(__uint_as_float(g[j])) * __uint_as_float(u[j]) : __uint_as_float(g[j]);
+                                const float r = P.scale_rows ? rinv_epi[c0 + j] : 1.0f;
+                                const float gv = r * __uint_as_float(g[j]);
+                                const float v = P.gateup ? chain_silu(gv) * (r * __uint_as_float(u[j])) : gv;
                                 stage_epi[(c0 + j) * kChainBlockM + row] = __float2bfloat16_rn(v);
                             }
                         }
@@ -469,13 +564,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const ChainParams p) {
                         __syncwarp();
                         if (lane == 0) mbar_arrive(&bars->tmem_empty[buf]);
                         asm volatile("bar.sync 2, 128;" ::: "memory");
-                        // token rows of the staged tile -> out[t][128 * tile ..], 16 bytes per thread and store
-                        for (int c = etid; c < p.T * 16; c += 128) {
-                            const int t = c >> 4, part = c & 15;
-                            const int n = (tile0 + wu.tile) * kChainBlockM + part * 8;
-                            if (n < P.N)
-                                *reinterpret_cast<uint4*>(P.out + (size_t)t * P.N + n) = *reinterpret_cast<const uint4*>(stage_epi + t * kChainBlockM + part * 8);
-                        }
+                        store_tokens(P, stage_epi, tile0 + wu.tile, 0, p.T, etid);
                         asm volatile("bar.sync 2, 128;" ::: "memory");
                     } else {
                         uint4* mine = reinterpret_cast<uint4*>(p.partials + ((size_t)blockIdx.x * kChainSlots + slot0 + wu.slot) * slot_floats) + row;
@@ -516,6 +605,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const ChainParams p) {
         pdl_wait();
         int* ctr = nullptr;
         int taken = 0;
+        int scales_of = -1;      // phase whose per-row scales sit in rinv_red
         // (the four warps move together: thread 0 takes every decision and hands it on through shared memory or an
         // OR-ing barrier, so no exit can split the group in front of a barrier)
         while (true) {
@@ -544,6 +634,10 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const ChainParams p) {
                 continue;
             }
             const int accs = P.gateup ? 2 : 1;
+            if (P.scale_rows && scales_of != pi) {
+                if (!load_row_scales(pi, ctr, rinv_red, rtid, 3)) break;
+                scales_of = pi;
+            }
             const Schedule sched(P.ksteps, 1, P.seg_tiles[seg], grid);
             const int tile0 = seg_tile0(P, seg);
             const int* counters = ctr + P.counter_base + tile0;
@@ -628,20 +722,15 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const ChainParams p) {
                     if (c0 + e >= cg_hi) break;
                     const float gf[4] = {g[e].x, g[e].y, g[e].z, g[e].w}, uf[4] = {u[e].x, u[e].y, u[e].z, u[e].w};
 #pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        stage_red[((c0 + e) * 4 + k) * kChainBlockM + rtid] = __float2bfloat16_rn(P.gateup ? chain_silu(gf[k]) * uf[k] : gf[k]);
+                    for (int k = 0; k < 4; ++k) {
+                        const int t = (c0 + e) * 4 + k;
+                        const float r = P.scale_rows ? rinv_red[t] : 1.0f;
+                        stage_red[t * kChainBlockM + rtid] = __float2bfloat16_rn(P.gateup ? chain_silu(r * gf[k]) * (r * uf[k]) : r * gf[k]);
+                    }
                 }
             }
             asm volatile("bar.sync 3, 128;" ::: "memory");
-            {
-                const int t_lo = cg_lo * 4, t_hi = min(cg_hi * 4, p.T);
-                for (int c = t_lo * 16 + rtid; c < t_hi * 16; c += 128) {
-                    const int t = c >> 4, part = c & 15;
-                    const int n = (tile0 + tile) * kChainBlockM + part * 8;
-                    if (n < P.N)
-                        *reinterpret_cast<uint4*>(P.out + (size_t)t * P.N + n) = *reinterpret_cast<const uint4*>(stage_red + t * kChainBlockM + part * 8);
-                }
-            }
+            store_tokens(P, stage_red, tile0 + tile, cg_lo * 4, cg_hi * 4, rtid);
             asm volatile("bar.sync 3, 128;" ::: "memory");
         }
     }
@@ -705,7 +794,8 @@ static int chain_n_tile(int T) { return ((T < 16 ? 16 : T) + 15) / 16 * 16; }
 size_t chain_counter_ints() { return 2 * (size_t)kChainCounterInts + 64; }
 
 size_t chain_workspace_bytes(int T, int num_sms) {
-    return align256((size_t)num_sms * kChainSlots * 2 * chain_n_tile(T) * kChainBlockM * sizeof(float));
+    return align256((size_t)num_sms * kChainSlots * 2 * chain_n_tile(T) * kChainBlockM * sizeof(float)) +
+           align256((size_t)kChainMaxStatTiles * chain_n_tile(T) * sizeof(float));
 }
 
 aflex_status chain_launch(aflex_ctx* ctx, const ChainStep* steps, int nsteps, int T, char* ws, size_t ws_bytes,
@@ -725,7 +815,7 @@ aflex_status chain_launch(aflex_ctx* ctx, const ChainStep* steps, int nsteps, in
     p.tmem_cols = cols;
     const int b_bytes = (p.n_tile * kChainBlockK * 2 + 1023) & ~1023;
     const int stage_bytes = 2 * kChainTileBytes + 2 * b_bytes;
-    const int stage_out_bytes = 2 * p.n_tile * kChainBlockM * 2;      // one staging buffer each for epilogue and reducers
+    const int stage_out_bytes = 2 * p.n_tile * kChainBlockM * 2 + 512;      // one staging buffer each for epilogue and reducers, and their per-row scales
     const int budget = kMaxDynamicSmem - 1024 - 1024 - stage_out_bytes - 256;
     p.stages = budget / stage_bytes;
     if (p.stages > kChainMaxStages) p.stages = kChainMaxStages;
@@ -768,6 +858,13 @@ aflex_status chain_launch(aflex_ctx* ctx, const ChainStep* steps, int nsteps, in
         P.counter_base = base;
         base += m_tiles;
         P.out = reinterpret_cast<__nv_bfloat16*>(s.out);
+        P.resid_in = reinterpret_cast<const __nv_bfloat16*>(s.resid_in);
+        P.resid_out = reinterpret_cast<__nv_bfloat16*>(s.resid_out);
+        P.gain = reinterpret_cast<const __nv_bfloat16*>(s.gain);
+        P.eps = s.eps;
+        P.scale_rows = (i > 0 && steps[i - 1].gain != nullptr) ? 1 : 0;
+        if (P.gain && (P.gateup || !P.resid_in || !P.resid_out || i + 1 >= nsteps || m_tiles > kChainMaxStatTiles))
+            return set_error(ctx, AFLEX_ERR_INVALID_ARG, "gemm chain: the residual + normalisation epilogue needs a linear step with a successor");
         in = s.in;
         if (!encode_tmap_2d_bf16(&maps.a0[i], s.w0, (uint64_t)s.N, (uint64_t)s.K, (uint64_t)s.K * 2, kChainBlockM, kChainBlockK, true) ||
             !encode_tmap_2d_bf16(&maps.a1[i], P.gateup ? s.w1 : s.w0, (uint64_t)s.N, (uint64_t)s.K, (uint64_t)s.K * 2, kChainBlockM, kChainBlockK, true) ||
@@ -776,6 +873,7 @@ aflex_status chain_launch(aflex_ctx* ctx, const ChainStep* steps, int nsteps, in
     }
     for (int i = nsteps; i < kChainMaxPhases; ++i) { p.ph[i] = p.ph[0]; maps.a0[i] = maps.a0[0]; maps.a1[i] = maps.a1[0]; maps.b[i] = maps.b[0]; }
     p.partials = reinterpret_cast<float*>(ws);
+    p.ss_part = reinterpret_cast<float*>(ws + align256((size_t)ctx->num_sms * kChainSlots * 2 * p.n_tile * kChainBlockM * sizeof(float)));
     if (base > kChainEpochBase) return set_error(ctx, AFLEX_ERR_UNSUPPORTED, "gemm chain: too many tiles");
     p.counters = counters;
     p.status = ctx->dev_status;

@@ -147,7 +147,13 @@ aflex_status gateup_launch(aflex_ctx* ctx, const void* x, const void* w_gate, co
 // Step i computes out = in . w0^T (w1 == nullptr) or out = silu(in . w0^T) .* (in . w1^T); step i + 1 reads
 // step i's output.  in bf16 [T][K], w bf16 [N][K], out bf16 [T][N].  T <= kChainMaxRows.
 constexpr int kChainMaxRows = 64;
-struct ChainStep { const void* in; const void* w0; const void* w1; int K, N; void* out; };
+struct ChainStep {
+    const void* in; const void* w0; const void* w1; int K, N; void* out;
+    // optional residual + normalisation epilogue of a linear step (w1 == nullptr) that has a successor:
+    //   resid_out = o + resid_in (o = the step's product, rounded to bf16), out = resid_out * gain (NOT yet divided by the
+    //   row's RMS), and the successor scales its accumulators by rsqrt(mean(resid_out^2) + eps) per row
+    const void* resid_in = nullptr; void* resid_out = nullptr; const void* gain = nullptr; float eps = 0.f;
+};
 bool chain_supported(int T);
 size_t chain_workspace_bytes(int T, int num_sms);
 // `counters`: chain_counter_ints() zeroed ints reserved for the chain launches of one stream (double-buffered over
