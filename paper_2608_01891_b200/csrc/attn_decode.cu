@@ -421,11 +421,8 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             wk.init(p, rg);
 
         while (!wk.done() && !aborted) {
-            // ---- one piece: units [u0, u0 + n) of item (b, g)
-            const int b = wk.b, g = wk.g, len = wk.len, cost = wk.cost;
-            const int nu = wk.nu - cost;                                     // real units of the item
-            const long long item_v0 = wk.prefix * p.Hkv + (long long)g * wk.nu;   // list position where the item starts
-            const long long item_x0 = item_v0 + cost;                        // ... where its real units start
+            // ---- one piece: units [u0, u0 + n) of one (sequence, KV head) item
+            const int len = wk.len, cost = wk.cost;
             const int nv = (int)min((long long)(wk.nu - wk.u), wk.end - wk.pos);
             const int u0 = max(wk.u, cost) - cost;                           // real unit range [u0, u0 + n)
             const int n = max(wk.u + nv, cost) - cost - u0;
@@ -578,7 +575,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
 
         while (!wk.done() && !aborted) {
             // ---- one piece: units [u0, u0 + n) of item (b, g)
-            const int b = wk.b, g = wk.g, len = wk.len, cost = wk.cost;
+            const int b = wk.b, g = wk.g, cost = wk.cost;
             const int nu = wk.nu - cost;                                     // real units of the item
             const long long item_v0 = wk.prefix * p.Hkv + (long long)g * wk.nu;   // list position where the item starts
             const long long item_x0 = item_v0 + cost;                        // ... where its real units start

@@ -350,6 +350,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
         struct PendingTile { int tile; TileCoord c; };
         PendingTile pend[2];
         int npend = 0;
+        bool gave_up = false;
         auto run_reduce = [&](const PendingTile& pd) {
             const long long x0 = (long long)pd.tile * p.kblocks;
             const int cf = sched.cta_of(x0);
@@ -360,6 +361,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
             // at the very end, where everybody else waits for the kernel's last CTA.
             const int nred = (np > 1 && sched.share_begin(cl + 1) > x0 + p.kblocks) ? np - 1 : np;
             if (me >= nred) return;
+            bool failed = false;
             if (etid == 0) {
                 const long long t_start = clock64();
                 int seen;
@@ -368,10 +370,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
                     if (seen >= np) break;
                     __nanosleep(64);
                 } while (clock64() - t_start < kWaitBudgetCycles);
-                if (seen < np) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); }
+                if (seen < np) { failed = true; bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); }
             }
-            asm volatile("bar.sync 2, 128;" ::: "memory");
-            if (bars->abort) return;
+            // the barrier hands thread 0's acquire on to the other 127 threads, and its verdict with it: the four warps
+            // leave together or not at all (there are barriers further down)
+            if (bar_or(2, 128, failed)) { gave_up = true; return; }
             const bool cf_early = sched.share_begin(cf) < x0;
             // The parked accumulators are [column group of 4 tokens][128 rows] float4.  Reducer `me` takes whole column
             // groups, thread = accumulator row; kElems groups per round with every piece's loads of a round in flight
@@ -446,19 +449,25 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
             }
         };
 
-        while (!bars->abort && cur.next(wu)) {
+        // (every exit from this loop is decided on a predicate OR-ed across the four epilogue warps: the loop body holds
+        // barriers, and a warp that left alone would leave the others waiting at one for good)
+        while (cur.next(wu)) {
+            if (bar_or(2, 128, bars->abort != 0)) { gave_up = true; break; }
             const TileCoord c = tiles.get(wu.tile);
             if (wu.slot < 0 && npend > 0) {
                 // shared tiles come first: before waiting for the first whole tile, finish this CTA's part
                 // of the shared tiles (the main loop of the whole tile runs meanwhile)
-                for (int i = 0; i < npend; ++i) run_reduce(pend[i]);
+                for (int i = 0; i < npend && !gave_up; ++i) run_reduce(pend[i]);
                 npend = 0;
-                if (bars->abort) break;
+                if (gave_up) break;
             }
-            if (!mbar_wait(&bars->tmem_full[buf], acc_ph)) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); break; }
+            const bool full_ok = mbar_wait(&bars->tmem_full[buf], acc_ph);
+            if (bar_or(2, 128, !full_ok)) {
+                if (etid == 0) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); }
+                gave_up = true;
+                break;
+            }
             tc_fence_after();
-            const int n_local = c.m_tile * p.tile_rows + row;    // output feature inside the expert
-            const bool n_ok = n_local < p.N;
             const uint32_t t0 = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(buf * acc_cols);
             if (wu.slot < 0) {
                 // ---- whole K range in this CTA: epilogue straight from TMEM, kStageTokens token columns per round
@@ -521,7 +530,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
             }
             if (++buf == p.nbuf) { buf = 0; acc_ph ^= 1; }
         }
-        for (int i = 0; i < npend; ++i) run_reduce(pend[i]);
+        for (int i = 0; i < npend && !gave_up; ++i) run_reduce(pend[i]);
     }
 
     if (tr && threadIdx.x == 64) tr[5] = global_timer_ns();          // epilogue finished
