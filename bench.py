@@ -1140,8 +1140,9 @@ def main():
             for _ in range(4):
                 fn()
             us = 1e3 * timed(fn, args.steps) / args.steps
+            ab1, fl1 = algorithmic_bytes(cfg, lens_np, 1), algorithmic_flops(cfg, 1)     # these calls take the whole batch at once
             if name == "attn_decode":
-                byts = abytes["attn_decode"] * M
+                byts = ab1["attn_decode"]
                 operators[name] = {"us": round(us, 2), "gbs": round(byts / us / 1e3, 1),
                                    "frac_hbm_measured": round(byts / us / 1e3 / peaks["hbm_gbs"], 4),
                                    "frac_hbm_nominal_8tbs": round(byts / us / 1e3 / 8000.0, 4),
@@ -1152,7 +1153,7 @@ def main():
                     operators[name]["frac_hbm_nominal_8tbs_event_pair"] = round(byts / ep / 1e3 / 8000.0, 4)
             else:
                 g, d = ("gateup_gemm", "down_gemm") if cfg.num_experts == 0 else ("moe_gateup_gemm", "moe_down_gemm")
-                byts, fl = (abytes[g] + abytes[d]) * M, (aflops[g] + aflops[d]) * M
+                byts, fl = ab1[g] + ab1[d], fl1[g] + fl1[d]
                 operators[name] = {"us": round(us, 2), "weight_stream_gbs": round(byts / us / 1e3, 1),
                                    "frac_hbm_measured": round(byts / us / 1e3 / peaks["hbm_gbs"], 4),
                                    "tflops": round(fl / us / 1e6, 1), "frac_bf16_burst": round(fl / us / 1e6 / peaks["bf16_tflops"], 4),
