@@ -1,7 +1,7 @@
 // A chain of dependent decode-batch GEMMs as ONE persistent tcgen05 kernel, software-pipelined
 // across the GEMMs.
 //
-// At decode batch sizes (<= 64 token rows) the FFN side and the W_o projection are weight-streaming
+// At decode batch sizes (<= 64 token rows by default) the FFN side and the W_o projection are weight-streaming
 // kernels: the boundary projection x = a W_o^T, h = silu(x W_gate^T) .* (x W_up^T) and y = h W_down^T
 // each read their weights once and are bound by HBM.  Run as separate kernels, every boundary between
 // two of them leaves DRAM idle: the last CTAs of one kernel finish their shared-tile reduction (a chain
@@ -64,6 +64,7 @@ constexpr int kChainSlots = 2 * kChainMaxSegs * 2;   // partial slots per CTA: [
 constexpr int kChainCounterInts = 8192;   // per half of the double-buffered counter array: per-tile counters, then the epoch words
 constexpr int kChainEpochBase = kChainCounterInts - 16;
 constexpr int kChainMaxStatTiles = 512;    // tiles of a phase with the residual + normalisation epilogue (N <= 65536)
+constexpr int kChainStageTokens = 32;       // token rows of an output tile staged per round (the staging buffers' height)
 constexpr int kChainMaxJobs = 64;          // reduce jobs one CTA can post in a launch (<= 2 per segment, plus markers)
 
 struct ChainPhase {
@@ -175,9 +176,9 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const ChainParams p) {
     // output staging, one buffer for the epilogue warps and one for the reducer warps: the output tile as
     // [token][128 features] bf16, so that it leaves the SM in 16-byte pieces
     __nv_bfloat16* stage_epi = reinterpret_cast<__nv_bfloat16*>(smem + (size_t)p.stages * stage_bytes + 1024);
-    __nv_bfloat16* stage_red = stage_epi + (size_t)p.n_tile * kChainBlockM;
-    float* rinv_epi = reinterpret_cast<float*>(stage_red + (size_t)p.n_tile * kChainBlockM);   // per-row scales, one copy per group
-    float* rinv_red = rinv_epi + 64;
+    __nv_bfloat16* stage_red = stage_epi + (size_t)kChainStageTokens * kChainBlockM;
+    float* rinv_epi = reinterpret_cast<float*>(stage_red + (size_t)kChainStageTokens * kChainBlockM);   // per-row scales, one copy per group
+    float* rinv_red = rinv_epi + kChainMaxRows;
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -225,7 +226,9 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const ChainParams p) {
     // the calling group (epilogue or reducers).  With the residual + normalisation epilogue the same pass adds the
     // residual rows, writes them back, writes the gain-weighted rows for the next phase and reduces every row's sum of
     // squares over the tile's 128 features (16 lanes hold one token row: a fixed-order shuffle reduction).
-    auto store_tokens = [&](const ChainPhase& P, const __nv_bfloat16* stage, int tile_g, int t_lo, int t_hi, int tid) {
+    // (the staging buffer holds token rows t_lo .. : row t of the tile sits in staged row t - t_lo)
+    auto store_tokens = [&](const ChainPhase& P, const __nv_bfloat16* stage_at_t0, int tile_g, int t_lo, int t_hi, int tid) {
+        const __nv_bfloat16* stage = stage_at_t0 - (size_t)t_lo * kChainBlockM;
         if (t_hi > p.T) t_hi = p.T;
         if (P.gain == nullptr) {
             for (int c = t_lo * 16 + tid; c < t_hi * 16; c += 128) {
@@ -547,25 +550,31 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const ChainParams p) {
                     tc_fence_after();
                     const uint32_t t0 = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(buf * buf_cols);
                     if (wu.slot < 0) {
-                        for (int c0 = 0; c0 < p.T; c0 += 16) {
-                            uint32_t g[16], u[16];
-                            tmem_ld_32x32b_x16(t0 + (uint32_t)c0, g);
-                            if (P.gateup) tmem_ld_32x32b_x16(t0 + (uint32_t)(p.n_tile + c0), u);
-                            tmem_ld_wait();
+                        for (int tc = 0; tc < p.T; tc += kChainStageTokens) {          // kChainStageTokens token columns per round
+                            const int ntok = min(kChainStageTokens, p.T - tc);
+                            for (int c0 = 0; c0 < ntok; c0 += 16) {
+                                uint32_t g[16], u[16];
+                                tmem_ld_32x32b_x16(t0 + (uint32_t)(tc + c0), g);
+                                if (P.gateup) tmem_ld_32x32b_x16(t0 + (uint32_t)(p.n_tile + tc + c0), u);
+                                tmem_ld_wait();
 #pragma unroll
-                            for (int j = 0; j < 16; ++j) {
-                                const float r = P.scale_rows ? rinv_epi[c0 + j] : 1.0f;
-                                const float gv = r * __uint_as_float(g[j]);
-                                const float v = P.gateup ? chain_silu(gv) * (r * __uint_as_float(u[j])) : gv;
-                                stage_epi[(c0 + j) * kChainBlockM + row] = __float2bfloat16_rn(v);
+                                for (int j = 0; j < 16; ++j) {
+                                    const float r = P.scale_rows ? rinv_epi[tc + c0 + j] : 1.0f;
+                                    const float gv = r * __uint_as_float(g[j]);
+                                    const float v = P.gateup ? chain_silu(gv) * (r * __uint_as_float(u[j])) : gv;
+                                    stage_epi[(c0 + j) * kChainBlockM + row] = __float2bfloat16_rn(v);
+                                }
                             }
+                            if (tc + kChainStageTokens >= p.T) {
+                                // the accumulator has been read in full: hand the TMEM buffer back before the stores
+                                tc_fence_before();
+                                __syncwarp();
+                                if (lane == 0) mbar_arrive(&bars->tmem_empty[buf]);
+                            }
+                            asm volatile("bar.sync 2, 128;" ::: "memory");
+                            store_tokens(P, stage_epi, tile0 + wu.tile, tc, tc + ntok, etid);
+                            asm volatile("bar.sync 2, 128;" ::: "memory");
                         }
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(&bars->tmem_empty[buf]);
-                        asm volatile("bar.sync 2, 128;" ::: "memory");
-                        store_tokens(P, stage_epi, tile0 + wu.tile, 0, p.T, etid);
-                        asm volatile("bar.sync 2, 128;" ::: "memory");
                     } else {
                         uint4* mine = reinterpret_cast<uint4*>(p.partials + ((size_t)blockIdx.x * kChainSlots + slot0 + wu.slot) * slot_floats) + row;
                         for (int a = 0; a < accs; ++a) {
@@ -670,7 +679,10 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const ChainParams p) {
             const int cg_lo = ncg * me / nred, cg_hi = ncg * (me + 1) / nred;
             const int up_off = (p.n_tile >> 2) * kChainBlockM;
             constexpr int kE = 4;
-            for (int c0 = cg_lo; c0 < cg_hi; c0 += kE) {
+            constexpr int kCgPerFlush = kChainStageTokens / 4;
+            for (int f0 = cg_lo; f0 < cg_hi; f0 += kCgPerFlush) {
+            const int f1 = min(cg_hi, f0 + kCgPerFlush);
+            for (int c0 = f0; c0 < f1; c0 += kE) {
                 float4 g[kE], u[kE];
 #pragma unroll
                 for (int e = 0; e < kE; ++e) g[e] = u[e] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -684,7 +696,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const ChainParams p) {
                             const float4* part = reinterpret_cast<const float4*>(p.partials + ((size_t)cc * kChainSlots + sl) * slot_floats) + rtid;
 #pragma unroll
                             for (int e = 0; e < kE; ++e)
-                                if (c0 + e < cg_hi) a[e][q] = __ldcg(part + (c0 + e) * kChainBlockM);
+                                if (c0 + e < f1) a[e][q] = __ldcg(part + (c0 + e) * kChainBlockM);
                         }
                     }
 #pragma unroll
@@ -692,7 +704,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const ChainParams p) {
                         if (cb + q <= cl) {
 #pragma unroll
                             for (int e = 0; e < kE; ++e)
-                                if (c0 + e < cg_hi) { g[e].x += a[e][q].x; g[e].y += a[e][q].y; g[e].z += a[e][q].z; g[e].w += a[e][q].w; }
+                                if (c0 + e < f1) { g[e].x += a[e][q].x; g[e].y += a[e][q].y; g[e].z += a[e][q].z; g[e].w += a[e][q].w; }
                         }
                     }
                     if (accs == 2) {
@@ -704,7 +716,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const ChainParams p) {
                                 const float4* part = reinterpret_cast<const float4*>(p.partials + ((size_t)cc * kChainSlots + sl) * slot_floats) + up_off + rtid;
 #pragma unroll
                                 for (int e = 0; e < kE; ++e)
-                                    if (c0 + e < cg_hi) a[e][q] = __ldcg(part + (c0 + e) * kChainBlockM);
+                                    if (c0 + e < f1) a[e][q] = __ldcg(part + (c0 + e) * kChainBlockM);
                             }
                         }
 #pragma unroll
@@ -712,26 +724,27 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const ChainParams p) {
                             if (cb + q <= cl) {
 #pragma unroll
                                 for (int e = 0; e < kE; ++e)
-                                    if (c0 + e < cg_hi) { u[e].x += a[e][q].x; u[e].y += a[e][q].y; u[e].z += a[e][q].z; u[e].w += a[e][q].w; }
+                                    if (c0 + e < f1) { u[e].x += a[e][q].x; u[e].y += a[e][q].y; u[e].z += a[e][q].z; u[e].w += a[e][q].w; }
                             }
                         }
                     }
                 }
 #pragma unroll
                 for (int e = 0; e < kE; ++e) {
-                    if (c0 + e >= cg_hi) break;
+                    if (c0 + e >= f1) break;
                     const float gf[4] = {g[e].x, g[e].y, g[e].z, g[e].w}, uf[4] = {u[e].x, u[e].y, u[e].z, u[e].w};
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {
                         const int t = (c0 + e) * 4 + k;
                         const float r = P.scale_rows ? rinv_red[t] : 1.0f;
-                        stage_red[t * kChainBlockM + rtid] = __float2bfloat16_rn(P.gateup ? chain_silu(r * gf[k]) * (r * uf[k]) : r * gf[k]);
+                        stage_red[(t - f0 * 4) * kChainBlockM + rtid] = __float2bfloat16_rn(P.gateup ? chain_silu(r * gf[k]) * (r * uf[k]) : r * gf[k]);
                     }
                 }
             }
             asm volatile("bar.sync 3, 128;" ::: "memory");
-            store_tokens(P, stage_red, tile0 + tile, cg_lo * 4, cg_hi * 4, rtid);
+            store_tokens(P, stage_red, tile0 + tile, f0 * 4, f1 * 4, rtid);
             asm volatile("bar.sync 3, 128;" ::: "memory");
+            }
         }
     }
 
@@ -787,7 +800,17 @@ static int chain_split() {
     return v;
 }
 
-bool chain_supported(int T) { return chain_enabled() != 0 && T >= 1 && T <= kChainMaxRows; }
+// The largest batch that takes the chain kernel.  The kernel itself handles up to kChainMaxRows = 128 token rows, but
+// above 64 a ring stage is 64 KB and only three fit: measured at the Qwen3-32B shape with 128 rows, 152.9 us for the FFN
+// against 142.4 us as two launches of the stand-alone GEMM, and 403.9 against 397.3 us for the configuration-3 step.
+// So 64 is the default; AFLEX_CHAIN_MAX_ROWS (<= 128) moves it (tuning / comparison).
+static int chain_max_rows() {
+    static int v = -1;
+    if (v < 0) { const char* e = getenv("AFLEX_CHAIN_MAX_ROWS"); v = e ? atoi(e) : 64; if (v > kChainMaxRows) v = kChainMaxRows; if (v < 0) v = 0; }
+    return v;
+}
+
+bool chain_supported(int T) { return chain_enabled() != 0 && T >= 1 && T <= chain_max_rows(); }
 
 static int chain_n_tile(int T) { return ((T < 16 ? 16 : T) + 15) / 16 * 16; }
 
@@ -815,7 +838,7 @@ aflex_status chain_launch(aflex_ctx* ctx, const ChainStep* steps, int nsteps, in
     p.tmem_cols = cols;
     const int b_bytes = (p.n_tile * kChainBlockK * 2 + 1023) & ~1023;
     const int stage_bytes = 2 * kChainTileBytes + 2 * b_bytes;
-    const int stage_out_bytes = 2 * p.n_tile * kChainBlockM * 2 + 512;      // one staging buffer each for epilogue and reducers, and their per-row scales
+    const int stage_out_bytes = 2 * kChainStageTokens * kChainBlockM * 2 + 2 * kChainMaxRows * 4;      // one staging buffer each for epilogue and reducers, and their per-row scales
     const int budget = kMaxDynamicSmem - 1024 - 1024 - stage_out_bytes - 256;
     p.stages = budget / stage_bytes;
     if (p.stages > kChainMaxStages) p.stages = kChainMaxStages;

@@ -146,7 +146,7 @@ aflex_status gateup_launch(aflex_ctx* ctx, const void* x, const void* w_gate, co
 // ---- chain of dependent decode-batch GEMMs as one persistent kernel (gemm_chain.cu)
 // Step i computes out = in . w0^T (w1 == nullptr) or out = silu(in . w0^T) .* (in . w1^T); step i + 1 reads
 // step i's output.  in bf16 [T][K], w bf16 [N][K], out bf16 [T][N].  T <= kChainMaxRows.
-constexpr int kChainMaxRows = 64;
+constexpr int kChainMaxRows = 128;
 struct ChainStep {
     const void* in; const void* w0; const void* w1; int K, N; void* out;
     // optional residual + normalisation epilogue of a linear step (w1 == nullptr) that has a successor:

@@ -120,7 +120,7 @@ def test_linear_matches_oracle(ctx, T, K, N):
     assert row_rel_err(f64(y), want) <= TOL_FFN
 
 
-@pytest.mark.parametrize("T", [1, 3, 4, 32, 33, 300, 384, 530])
+@pytest.mark.parametrize("T", [1, 3, 4, 32, 33, 64, 65, 100, 128, 129, 300, 384, 530])
 def test_dense_ffn_config1_shapes(ctx, T):
     cfg = IN.CONFIGS[1]
     x = IN.make_x(cfg, tokens=T)
