@@ -134,6 +134,26 @@ def test_dense_ffn_config1_shapes(ctx, T):
     assert row_rel_err(f64(y), want) <= TOL_FFN
 
 
+@pytest.mark.parametrize("T,H,I", [(20, 320, 448), (7, 64, 8), (48, 1096, 2056), (64, 8, 136), (33, 192, 19000)])
+def test_dense_ffn_decode_batch_odd_shapes(ctx, T, H, I):
+    """Decode batches go through the persistent GEMM chain kernel: reduction lengths that are an odd number of 64-wide
+    K blocks (its linear phases step two blocks at a time; the missing half block is read as zeros), reduction lengths
+    and feature counts below one tile, feature counts that are not a multiple of 128, and a phase with more tiles
+    than SMs (whole tiles and shared remainder tiles in one phase)."""
+    x, wg = rand_bf16((T, H), 1.0, 31), rand_bf16((I, H), 1.5 / np.sqrt(H), 32)
+    wu, wd = rand_bf16((I, H), 1.0 / np.sqrt(H), 33), rand_bf16((H, I), 1.0 / np.sqrt(I), 34)
+    y = torch.full((T, H), float("nan"), dtype=torch.bfloat16, device=DEV)
+    ctx.ffn_dense(x.to(DEV), wg.to(DEV), wu.to(DEV), wd.to(DEV), y)
+    torch.cuda.synchronize()
+    want = O.ffn_dense(u16(x), u16(wg), u16(wu), u16(wd))
+    assert row_rel_err(f64(y), want) <= TOL_FFN
+    y2 = torch.full_like(y, float("nan"))
+    ctx.ffn_dense(x.to(DEV), wg.to(DEV), wu.to(DEV), wd.to(DEV), y2)
+    torch.cuda.synchronize()
+    assert torch.equal(y.view(torch.int16), y2.view(torch.int16))          # bit-deterministic, launch after launch
+    assert ctx.device_status() == AF.OK
+
+
 def test_dense_ffn_zero_gate_gives_zero(ctx):
     T, H, I = 5, 128, 256
     x, wu, wd = rand_bf16((T, H), 1.0, 1), rand_bf16((I, H), 0.1, 2), rand_bf16((H, I), 0.1, 3)
