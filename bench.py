@@ -237,7 +237,7 @@ def run_ffn_sweep(args, cfg, local_rank, device, peaks):
     sampler = ClockSampler(local_rank)
     sampler.start()
     rows = []
-    for T in (32, 64, 128, 256, 512, 1024, 2048, 4096, 8192):
+    for T in ([args.ffn_tokens] if args.ffn_tokens > 0 else (32, 64, 128, 256, 512, 1024, 2048, 4096, 8192)):
         x = IN.make_x(dense, device=device, tokens=T)
         y = torch.empty(T, H, dtype=torch.bfloat16, device=device)
         for _ in range(max(3, args.warmup)):
@@ -258,6 +258,11 @@ def run_ffn_sweep(args, cfg, local_rank, device, peaks):
                      "frac_bf16_sustained": round(flops / us / 1e6 / peaks["bf16_tflops_sustained"], 4),
                      "weight_stream_gbs": round(wbytes / us / 1e3, 1),
                      "frac_hbm": round(wbytes / us / 1e3 / peaks["hbm_gbs"], 4)})
+        ctx.profile_enable(True)                       # per kernel under event pairs (serialised: no launch overlap)
+        for _ in range(3):
+            ctx.ffn_dense(x, wg, wu, wd, y, stream)
+        rows[-1]["kernels_us"] = {k: round(1e3 * v[0] / v[1], 1) for k, v in ctx.profile_read().items()}
+        ctx.profile_enable(False)
     assert ctx.device_status() == AF.OK
     line = {"metric": "dense FFN throughput vs tokens (Qwen3-32B FFN shape)" if cfg.cfg_id in (2, 3) else
             f"dense FFN throughput vs tokens (H={H}, I={I})", "unit": "TFLOP/s", "dtype": "bf16", "data": "synthetic",
@@ -921,6 +926,7 @@ def main():
     ap.add_argument("--ffn-sweep", action="store_true",
                     help="instead of the layer step: dense FFN (aflex_ffn_dense) at the configuration's weight shape "
                          "for T = 32..8192 tokens, TFLOP/s against the measured bf16 peak; prints one JSON line")
+    ap.add_argument("--ffn-tokens", type=int, default=0, help="with --ffn-sweep: only this token count")
     ap.add_argument("--decoder-layers", type=int, default=0,
                     help="instead of the layer step: chain this many whole decoder layers (aflex_decoder_layers) at "
                          "every microbatch depth of the configuration; prints one JSON line")

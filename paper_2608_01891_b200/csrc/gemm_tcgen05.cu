@@ -153,7 +153,7 @@ struct __align__(8) GemmBarriers {
 
 __device__ __forceinline__ float silu_f32(float z) { return __fdividef(z, 1.0f + __expf(-z)); }
 
-template <int MODE>
+template <int MODE, bool PAIR>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__ CUtensorMap tmap_a1,
             const __grid_constant__ TmapSetB tmaps_b, const GemmParams p) {
@@ -162,7 +162,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     constexpr int kNumA = (MODE == kLinear) ? 1 : 2;
     constexpr int kABytes = kBlockM * kBlockK * 2;           // 16 KB
-    const int stage_bytes = kNumA * kABytes + ((p.n_tile * kBlockK * 2 + 1023) & ~1023);
+    // (a CTA of a pair holds half of the token rows of the activation tile)
+    const int stage_bytes = kNumA * kABytes + (((PAIR ? p.n_tile / 2 : p.n_tile) * kBlockK * 2 + 1023) & ~1023);
+    // Pair form: CTAs 2c and 2c + 1 are pair c of the schedule; rank 0 issues the MMAs of both.
+    const int rank = PAIR ? (int)cluster_cta_rank() : 0;
+    const int cid = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
     GemmBarriers* bars = reinterpret_cast<GemmBarriers*>(smem + (size_t)p.stages * stage_bytes);
     // Epilogue staging: kStageTokens token rows of the output tile, [token][tile's weight rows] in the output type, so
     // that results leave the SM as 16-byte stores of consecutive features instead of one 2-byte store per value.
@@ -173,7 +177,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&bars->tmem_full[b], 1); mbar_init(&bars->tmem_empty[b], 4); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&bars->tmem_full[b], 1); mbar_init(&bars->tmem_empty[b], PAIR ? 8 : 4); }
         bars->abort = 0;
         fence_mbar_init();
     }
@@ -184,8 +188,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
         for (int i = threadIdx.x; i <= p.num_experts; i += blockDim.x) bars->seg[i] = p.offsets[i];
     }
     if (warp == 1) {
-        tmem_alloc(&bars->tmem_base, (uint32_t)p.tmem_cols);
-        tmem_relinquish();
+        if (PAIR) { tmem_alloc_pair(&bars->tmem_base, (uint32_t)p.tmem_cols); tmem_relinquish_pair(); }
+        else { tmem_alloc(&bars->tmem_base, (uint32_t)p.tmem_cols); tmem_relinquish(); }
     }
     if (warp == 0 && lane == 0) {
         prefetch_tmap(&tmap_a0);
@@ -193,14 +197,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
         for (int i = 0; i <= box_index(p.n_tile); ++i) prefetch_tmap(&tmaps_b.m[i]);
     }
     tc_fence_before();
-    __syncthreads();
+    if (PAIR) cluster_sync_all();      // the peer's barriers are initialised before anything signals them
+    else __syncthreads();
     tc_fence_after();
 
     const uint32_t tmem_base = bars->tmem_base;
     const TileIter tiles(p, bars->seg);
     constexpr int kAccs = (MODE == kLinear) ? 1 : 2;
     const int acc_cols = kAccs * p.n_tile;   // TMEM columns per accumulator buffer
-    const Schedule sched(p.kblocks, p.streamk, tiles.total, (int)gridDim.x);
+    const Schedule sched(p.kblocks, p.streamk, tiles.total, PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x);
     pdl_launch_dependents();
     unsigned long long* tr = p.trace ? p.trace + (size_t)blockIdx.x * 8 : nullptr;
     if (tr && threadIdx.x == 0) tr[0] = global_timer_ns();           // CTA running
@@ -212,8 +217,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
             const uint64_t pol_w = p.w_reuse ? policy_evict_normal() : policy_evict_first();
             const uint64_t pol_x = policy_evict_last();    // activations: re-read by every tile
             int s = 0; uint32_t ph = 0;
-            UnitCursor cur(sched, blockIdx.x);
+            UnitCursor cur(sched, cid);
             WorkUnit wu;
+            // Pair form: both CTAs' loads of a stage are counted on the even CTA's barrier (it issues the MMAs).
+            auto load = [&](void* dst, const CUtensorMap* tm, int x, int y, int stage, uint64_t pol) {
+                if (PAIR) tma_load_2d_hint_pair(dst, tm, x, y, cluster_map_shared(smem_u32(&bars->full[stage]), 0), pol);
+                else tma_load_2d_hint(dst, tm, x, y, &bars->full[stage], pol);
+            };
+            const int a_off = rank * kBlockM;                      // this CTA's weight rows inside a pair tile
             // The first `stages` K blocks find the ring empty: their weight tiles are requested at once,
             // before the grid-dependency wait; their activation tiles follow after it.
             int primed = 0;
@@ -222,15 +233,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
             while (!bars->abort && cur.next(wu)) {
                 const TileCoord c = tiles.get(wu.tile);
                 const int bi = box_index(c.b_rows);
-                const uint32_t tx = (uint32_t)(kNumA * kABytes + box_rows(c.b_rows, p.n_tile) * kBlockK * 2);
+                const int box = box_rows(c.b_rows, p.n_tile);
+                const uint32_t tx = (uint32_t)((PAIR ? 2 : 1) * kNumA * kABytes + box * kBlockK * 2);   // both CTAs' bytes
+                const int b_row = c.b_row0 + (PAIR ? rank * (box >> 1) : 0);
                 for (int kb = wu.kb0; kb < wu.kb1; ++kb) {
                     if (primed < p.stages) {
                         uint8_t* st = smem + (size_t)primed * stage_bytes;
-                        mbar_expect_tx(&bars->full[primed], tx);
-                        tma_load_2d_hint(st, &tmap_a0, kb * kBlockK, c.a_row0, &bars->full[primed], pol_w);
-                        if (kNumA == 2) tma_load_2d_hint(st + kABytes, MODE == kGateUp ? &tmap_a1 : &tmap_a0, kb * kBlockK,
-                                                         c.a_row0 + (MODE == kGateUp ? 0 : kBlockM), &bars->full[primed], pol_w);
-                        pend_kb[primed] = kb; pend_row[primed] = c.b_row0; pend_box[primed] = bi;
+                        if (rank == 0) mbar_expect_tx(&bars->full[primed], tx);
+                        load(st, &tmap_a0, kb * kBlockK, c.a_row0 + a_off, primed, pol_w);
+                        if (kNumA == 2) load(st + kABytes, MODE == kGateUp ? &tmap_a1 : &tmap_a0, kb * kBlockK,
+                                             c.a_row0 + a_off + (MODE == kGateUp ? 0 : kBlockM), primed, pol_w);
+                        pend_kb[primed] = kb; pend_row[primed] = b_row; pend_box[primed] = bi;
                         ++primed;
                         if (++s == p.stages) { s = 0; ph ^= 1; }
                         continue;
@@ -240,17 +253,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
                         pdl_wait();
                         if (tr) tr[2] = global_timer_ns();           // dependency satisfied
                         for (int i = 0; i < primed; ++i)
-                            tma_load_2d_hint(smem + (size_t)i * stage_bytes + kNumA * kABytes, &tmaps_b.m[pend_box[i]],
-                                             pend_kb[i] * kBlockK, pend_row[i], &bars->full[i], pol_x);
+                            load(smem + (size_t)i * stage_bytes + kNumA * kABytes, &tmaps_b.m[pend_box[i]],
+                                 pend_kb[i] * kBlockK, pend_row[i], i, pol_x);
                         waited = true;
                     }
                     if (!mbar_wait(&bars->empty[s], ph ^ 1)) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); break; }
                     uint8_t* st = smem + (size_t)s * stage_bytes;
-                    mbar_expect_tx(&bars->full[s], tx);
-                    tma_load_2d_hint(st, &tmap_a0, kb * kBlockK, c.a_row0, &bars->full[s], pol_w);
-                    if (kNumA == 2) tma_load_2d_hint(st + kABytes, MODE == kGateUp ? &tmap_a1 : &tmap_a0, kb * kBlockK,
-                                                     c.a_row0 + (MODE == kGateUp ? 0 : kBlockM), &bars->full[s], pol_w);
-                    tma_load_2d_hint(st + kNumA * kABytes, &tmaps_b.m[bi], kb * kBlockK, c.b_row0, &bars->full[s], pol_x);
+                    if (rank == 0) mbar_expect_tx(&bars->full[s], tx);
+                    load(st, &tmap_a0, kb * kBlockK, c.a_row0 + a_off, s, pol_w);
+                    if (kNumA == 2) load(st + kABytes, MODE == kGateUp ? &tmap_a1 : &tmap_a0, kb * kBlockK,
+                                         c.a_row0 + a_off + (MODE == kGateUp ? 0 : kBlockM), s, pol_w);
+                    load(st + kNumA * kABytes, &tmaps_b.m[bi], kb * kBlockK, b_row, s, pol_x);
                     if (++s == p.stages) { s = 0; ph ^= 1; }
                 }
             }
@@ -258,23 +271,24 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
             if (!waited) {
                 pdl_wait();
                 for (int i = 0; i < primed; ++i)
-                    tma_load_2d_hint(smem + (size_t)i * stage_bytes + kNumA * kABytes, &tmaps_b.m[pend_box[i]],
-                                     pend_kb[i] * kBlockK, pend_row[i], &bars->full[i], pol_x);
+                    load(smem + (size_t)i * stage_bytes + kNumA * kABytes, &tmaps_b.m[pend_box[i]],
+                         pend_kb[i] * kBlockK, pend_row[i], i, pol_x);
             }
-            // On abort wait (bounded) for loads still in flight before the CTA leaves.
-            if (bars->abort) {
+            // On abort wait (bounded) for loads still in flight before the CTA leaves (the even CTA of a pair waits
+            // for its peer's too: they are counted on its barriers, and the peer leaves after it).
+            if (bars->abort && rank == 0) {
                 for (int i = 0; i < p.stages; ++i) (void)mbar_wait(&bars->full[i], 0);
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        if (lane == 0 && rank == 0) {
             int s = 0; uint32_t ph = 0;
             int buf = 0; uint32_t acc_ph = 0;
-            UnitCursor cur(sched, blockIdx.x);
+            UnitCursor cur(sched, cid);
             WorkUnit wu;
             while (!bars->abort && cur.next(wu)) {
-                const uint32_t idesc = umma_idesc_bf16(kBlockM, (uint32_t)box_rows(tiles.get(wu.tile).b_rows, p.n_tile));
+                const uint32_t idesc = umma_idesc_bf16(PAIR ? 2 * kBlockM : kBlockM, (uint32_t)box_rows(tiles.get(wu.tile).b_rows, p.n_tile));
                 if (!mbar_wait(&bars->tmem_empty[buf], acc_ph ^ 1)) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); break; }
                 tc_fence_after();
                 const uint32_t d0 = tmem_base + (uint32_t)(buf * acc_cols);
@@ -288,17 +302,20 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
                     for (int k = 0; k < kBlockK / 16; ++k) {
                         const uint32_t acc = (kb > wu.kb0 || k > 0) ? 1u : 0u;
                         // advancing 16 bf16 along K inside the swizzled row = +32 bytes = +2 in 16-byte units
-                        umma_bf16(d0, da0 + 2 * k, db + 2 * k, idesc, acc);
+                        if (PAIR) umma_bf16_pair(d0, da0 + 2 * k, db + 2 * k, idesc, acc);
+                        else umma_bf16(d0, da0 + 2 * k, db + 2 * k, idesc, acc);
                         if (kNumA == 2) {
                             const uint64_t da1 = umma_desc_k_sw128(a_addr + kABytes);
-                            umma_bf16(d0 + (uint32_t)p.n_tile, da1 + 2 * k, db + 2 * k, idesc, acc);
+                            if (PAIR) umma_bf16_pair(d0 + (uint32_t)p.n_tile, da1 + 2 * k, db + 2 * k, idesc, acc);
+                            else umma_bf16(d0 + (uint32_t)p.n_tile, da1 + 2 * k, db + 2 * k, idesc, acc);
                         }
                     }
-                    umma_commit(&bars->empty[s]);   // smem stage reusable once these MMAs retire
+                    // smem stage reusable once these MMAs retire (in both CTAs of a pair)
+                    if (PAIR) umma_commit_pair(&bars->empty[s]); else umma_commit(&bars->empty[s]);
                     if (++s == p.stages) { s = 0; ph ^= 1; }
                 }
                 if (bars->abort) break;
-                umma_commit(&bars->tmem_full[buf]);  // accumulator complete
+                if (PAIR) umma_commit_pair(&bars->tmem_full[buf]); else umma_commit(&bars->tmem_full[buf]);  // accumulator complete
                 if (tr) tr[4] = global_timer_ns();                   // last MMA of the unit issued
                 if (++buf == p.nbuf) { buf = 0; acc_ph ^= 1; }
             }
@@ -311,8 +328,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
         const int cols = kAccs * p.n_tile;             // fp32 values per accumulator row
         const size_t slot_floats = (size_t)cols * kBlockM;
         int buf = 0; uint32_t acc_ph = 0;
-        UnitCursor cur(sched, blockIdx.x);
+        UnitCursor cur(sched, cid);
         WorkUnit wu;
+        // Handing an accumulator buffer back: to the MMA issuer's barrier, which in a pair is the even CTA's.
+        auto release_tmem = [&](int b) {
+            if (PAIR) mbar_arrive_cluster(cluster_map_shared(smem_u32(&bars->tmem_empty[b]), 0));
+            else mbar_arrive(&bars->tmem_empty[b]);
+        };
+        // Counters of a shared tile: in a pair each CTA finishes its own 128 rows with the same-rank CTAs of the other pairs.
+        auto ctile = [&](int tile) { return PAIR ? tile * 2 + rank : tile; };
         pdl_wait();   // nothing is written before the predecessor grid has completed
 
         // Geometry of the output tile in the staging buffer and in memory.
@@ -328,7 +352,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
         // barriers order the staging writes before the reads and free the buffer for its next user.
         auto stage_flush = [&](const TileCoord& c, int t0, int ntok) {
             asm volatile("bar.sync 2, 128;" ::: "memory");
-            const int n0 = c.m_tile * p.tile_rows;
+            const int n0 = c.m_tile * p.tile_rows + rank * kBlockM;
             for (int i = etid; i < ntok * cpr; i += 128) {
                 const int tl = i / cpr, part = i - tl * cpr;
                 const int t = t0 + tl, n = n0 + part * per16;
@@ -355,7 +379,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
             const long long x0 = (long long)pd.tile * p.kblocks;
             const int cf = sched.cta_of(x0);
             const int cl = sched.cta_of(x0 + p.kblocks - 1);
-            const int np = cl - cf + 1, me = (int)blockIdx.x - cf;
+            const int np = cl - cf + 1, me = cid - cf;
             // A last contributor whose share runs on into the next tile has a second shared tile to finish (as that
             // tile's first contributor): it is excused here, so that no CTA does two reductions one after the other
             // at the very end, where everybody else waits for the kernel's last CTA.
@@ -366,7 +390,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
                 const long long t_start = clock64();
                 int seen;
                 do {
-                    asm volatile("ld.acquire.gpu.b32 %0, [%1];" : "=r"(seen) : "l"(p.counters + pd.tile) : "memory");
+                    asm volatile("ld.acquire.gpu.b32 %0, [%1];" : "=r"(seen) : "l"(p.counters + ctile(pd.tile)) : "memory");
                     if (seen >= np) break;
                     __nanosleep(64);
                 } while (clock64() - t_start < kWaitBudgetCycles);
@@ -399,7 +423,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
                                 // only the first contributor's share can begin before the tile: then its piece is a
                                 // later unit of that CTA (slot 1); every other piece is a first unit (slot 0)
                                 const int sl = (cc == cf && cf_early) ? 1 : 0;
-                                const float4* part = reinterpret_cast<const float4*>(p.partials + ((size_t)cc * 2 + sl) * slot_floats) + etid;
+                                const size_t who = PAIR ? (size_t)cc * 2 + rank : (size_t)cc;      // the CTA that parked the piece
+                                const float4* part = reinterpret_cast<const float4*>(p.partials + (who * 2 + sl) * slot_floats) + etid;
 #pragma unroll
                                 for (int e = 0; e < kElems; ++e) {
                                     if (c0 + e < f1) {
@@ -441,10 +466,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
             }
             asm volatile("bar.sync 2, 128;" ::: "memory");
             if (etid == 0) {
-                const int done = atomicAdd(&p.counters[kStreamKMaxTiles + pd.tile], 1);
+                const int done = atomicAdd(&p.counters[kStreamKMaxTiles + ctile(pd.tile)], 1);
                 if (done == nred - 1) {   // every reducer has read what it needs: clean up for the next launch
-                    p.counters[pd.tile] = 0;
-                    p.counters[kStreamKMaxTiles + pd.tile] = 0;
+                    p.counters[ctile(pd.tile)] = 0;
+                    p.counters[kStreamKMaxTiles + ctile(pd.tile)] = 0;
                 }
             }
         };
@@ -495,7 +520,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
                         // the accumulator has been read in full: hand the TMEM buffer back before the stores
                         tc_fence_before();
                         __syncwarp();
-                        if (lane == 0) mbar_arrive(&bars->tmem_empty[buf]);
+                        if (lane == 0) release_tmem(buf);
                     }
                     stage_flush(c, c.b_row0 + tc, ntok);
                 }
@@ -514,14 +539,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&bars->tmem_empty[buf]);   // TMEM buffer is free again
+                if (lane == 0) release_tmem(buf);   // TMEM buffer is free again
                 // publish: all 128 rows stored (CTA barrier), then one thread releases them device-wide
                 // and bumps the tile counter.  The reduction itself is deferred (see run_reduce).
                 asm volatile("bar.sync 2, 128;" ::: "memory");
                 if (etid == 0) {
                     if (tr) tr[6] = global_timer_ns();               // partial stored, about to publish
                     __threadfence();
-                    atomicAdd(&p.counters[wu.tile], 1);
+                    atomicAdd(&p.counters[ctile(wu.tile)], 1);
                     if (tr) tr[7] = global_timer_ns();               // published
                 }
                 pend[npend].tile = wu.tile;
@@ -535,10 +560,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
 
     if (tr && threadIdx.x == 64) tr[5] = global_timer_ns();          // epilogue finished
     tc_fence_before();
-    __syncthreads();
+    // A pair leaves together: the peer's shared memory, barriers and TMEM are in use until both are done.
+    if (PAIR) cluster_sync_all();
+    else __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
+        if (PAIR) tmem_dealloc_pair(tmem_base, (uint32_t)p.tmem_cols);
+        else tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
     }
 }
 
@@ -557,6 +585,7 @@ static int pick_n_tile(int rows_max) {
 
 struct GemmConfig {
     GemmParams p;
+    bool pair;          // CTA pairs (cta_group::2): a 256-weight-row tile per pair, half of the token rows loaded by each CTA
     size_t smem_bytes;
     size_t partial_bytes;
     int grid;
@@ -579,6 +608,19 @@ static int streaming_smem_budget() {
 // Plain linear GEMMs take two weight-row tiles per CTA tile (kLinear2) when the activation tile is as
 // large as a weight tile's K slice or close to it (64..128 token rows) and the weight matrix is large:
 // the activation bytes that go from L2 to shared memory per weight byte are halved.  AFLEX_GEMM_DUAL = 0 / 1 forces it off / on (tuning).
+// CTA pairs pay where the activation tile takes a large part of a pipeline stage, so that too few weight bytes are in
+// flight per SM to cover the DRAM latency: from this token-tile width on (dense form).  AFLEX_GEMM_PAIR: 0 = never,
+// n >= 16 = from n token rows per tile on (tuning).
+static int pair_from_rows() {
+    static int v = -1;
+    if (v < 0) { const char* e = getenv("AFLEX_GEMM_PAIR"); v = e ? atoi(e) : 192; }
+    return v;
+}
+static bool use_pair(int T, int N, int E, int num_sms) {
+    const int from = pair_from_rows();
+    return from >= 16 && E == 0 && pick_n_tile(T) >= from && N >= 2 * kBlockM && num_sms >= 2;
+}
+
 static int linear_mode(int T, int N, int K) {
     static int force = -2;
     if (force == -2) { const char* e = getenv("AFLEX_GEMM_DUAL"); force = e ? atoi(e) : -1; }
@@ -586,6 +628,7 @@ static int linear_mode(int T, int N, int K) {
     if (force == 0) return kLinear;
     if (force == 1) return kLinear2;
     const int n_tile = pick_n_tile(T);
+    if (pair_from_rows() >= 16 && n_tile >= pair_from_rows()) return kLinear;   // the pair form halves the activation bytes itself
     // measured at the Qwen3-32B shapes: pays on the long down projection (70.6 -> 66.3 us at 128 rows), not on
     // the short W_o / QKV projections, whose time is fixed cost rather than streaming
     return (n_tile >= 64 && n_tile <= 128 && (long long)N * K >= (64LL << 20)) ? kLinear2 : kLinear;
@@ -615,7 +658,8 @@ static bool make_config(int mode, int T, int N, int K, int rows_max, int E, int 
         if (cap < 0) { const char* e = getenv("AFLEX_GEMM_NTILE_CAP"); cap = e ? atoi(e) : 0; }
         if (cap >= 16 && p.n_tile > cap) p.n_tile = cap / 16 * 16;
     }
-    p.tile_rows = (mode == kLinear2) ? 2 * kBlockM : kBlockM;
+    cfg->pair = mode != kLinear2 && use_pair(rows_max, N, E, num_sms) && p.n_tile >= pair_from_rows();
+    p.tile_rows = (mode == kLinear2 || cfg->pair) ? 2 * kBlockM : kBlockM;
     p.m_tiles = (N + p.tile_rows - 1) / p.tile_rows;
     p.n_tiles = (T + p.n_tile - 1) / p.n_tile;
     p.kblocks = (K + kBlockK - 1) / kBlockK;
@@ -640,13 +684,14 @@ static bool make_config(int mode, int T, int N, int K, int rows_max, int E, int 
     while (cols < p.nbuf * acc_cols) cols <<= 1;
     p.tmem_cols = cols;
     const int a_bytes = accs * kBlockM * kBlockK * 2;
-    const int stage_bytes = a_bytes + round_up(p.n_tile * kBlockK * 2, 1024);
+    const int stage_bytes = a_bytes + round_up((cfg->pair ? p.n_tile / 2 : p.n_tile) * kBlockK * 2, 1024);
     // few tiles per SM: share the remainder tiles along K; many: whole tiles round-robin.  Wide tiles
     // (large T, compute-bound) make the shared tiles' partials big, so they are shared only when whole
     // tiles alone would leave most SMs idle.
     static int nostream = -1;   // AFLEX_GEMM_NOSTREAMK=1: whole tiles only (measurement of per-SM streaming rates)
     if (nostream < 0) { const char* e = getenv("AFLEX_GEMM_NOSTREAMK"); nostream = e ? atoi(e) : 0; }
-    p.streamk = nostream ? 0 : (tiles_hi < 8LL * num_sms && tiles_hi <= kStreamKMaxTiles && (p.n_tile <= 128 || tiles_hi < 2LL * num_sms)) ? 1 : 0;
+    const long long workers = cfg->pair ? num_sms / 2 : num_sms;      // CTAs, or CTA pairs, that share the tile list
+    p.streamk = nostream ? 0 : (tiles_hi < 8LL * workers && tiles_hi <= kStreamKMaxTiles && (p.n_tile <= 128 || tiles_hi < 2LL * workers)) ? 1 : 0;
     // epilogue staging: kStageTokens token rows of the tile in the output type
     const int stage_out_bytes = kStageTokens * (mode == kLinear2 ? 2 : 1) * kBlockM * (out_f32 ? 4 : 2);
     int cap = (p.streamk && p.n_tile <= 64 && mode != kLinear2) ? streaming_smem_budget() + stage_out_bytes : kMaxDynamicSmem;
@@ -659,28 +704,35 @@ static bool make_config(int mode, int T, int N, int K, int rows_max, int E, int 
     cfg->smem_bytes = (size_t)stages * stage_bytes + sizeof(GemmBarriers) + 1024 + 256 + stage_out_bytes;
     if (cfg->smem_bytes > (size_t)kMaxDynamicSmem) return false;
     long long units = tiles_hi * p.kblocks;
-    cfg->grid = (int)(units < num_sms ? units : num_sms);
+    if (cfg->pair) {
+        const int pairs = num_sms / 2;
+        cfg->grid = 2 * (int)(units < pairs ? units : pairs);
+        if (2 * tiles_hi > kStreamKMaxTiles) return false;             // each CTA of a pair has its own tile counters
+    } else {
+        cfg->grid = (int)(units < num_sms ? units : num_sms);
+    }
     if (cfg->grid < 1) cfg->grid = 1;
     cfg->partial_bytes = p.streamk ? align256((size_t)cfg->grid * 2 * accs * p.n_tile * kBlockM * sizeof(float)) : 0;
     return true;
 }
 
-static bool encode_b_set(TmapSetB* set, const void* base, uint64_t rows, uint64_t K, int n_tile) {
+static bool encode_b_set(TmapSetB* set, const void* base, uint64_t rows, uint64_t K, int n_tile, bool pair = false) {
     for (int i = 0; i < 5; ++i) {
-        const uint32_t box = (uint32_t)((16 << i) < n_tile ? (16 << i) : n_tile);   // same rule as box_rows()
+        uint32_t box = (uint32_t)((16 << i) < n_tile ? (16 << i) : n_tile);   // same rule as box_rows()
+        if (pair) box >>= 1;                                                  // each CTA of a pair loads half of the rows
         if (!encode_tmap_2d_bf16(&set->m[i], base, rows, K, K * 2, box, kBlockK, false)) return false;
     }
     return true;
 }
 
-template <int MODE>
+template <int MODE, bool PAIR = false>
 static aflex_status launch_gemm(aflex_ctx* ctx, const GemmConfig& cfg, const CUtensorMap& ta0, const CUtensorMap& ta1,
                                 const TmapSetB& tb, cudaStream_t st, int kind) {
-    if (!ctx->gemm_attr_set[MODE]) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (!ctx->gemm_attr_set[MODE + (PAIR ? 3 : 0)]) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_kernel<MODE, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              kMaxDynamicSmem);
         if (e != cudaSuccess) return check_cuda(ctx, e, "cudaFuncSetAttribute(gemm)");
-        ctx->gemm_attr_set[MODE] = true;
+        ctx->gemm_attr_set[MODE + (PAIR ? 3 : 0)] = true;
     }
     KernelScope scope(ctx, kind, st);
     cudaLaunchConfig_t lc = {};
@@ -688,12 +740,19 @@ static aflex_status launch_gemm(aflex_ctx* ctx, const GemmConfig& cfg, const CUt
     lc.blockDim = dim3(kGemmThreads);
     lc.dynamicSmemBytes = cfg.smem_bytes;
     lc.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     lc.attrs = attr;
     lc.numAttrs = 1;
-    return check_cuda(ctx, cudaLaunchKernelEx(&lc, gemm_kernel<MODE>, ta0, ta1, tb, cfg.p), "gemm_kernel launch");
+    if (PAIR) {
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = 2;
+        attr[1].val.clusterDim.y = 1;
+        attr[1].val.clusterDim.z = 1;
+        lc.numAttrs = 2;
+    }
+    return check_cuda(ctx, cudaLaunchKernelEx(&lc, gemm_kernel<MODE, PAIR>, ta0, ta1, tb, cfg.p), "gemm_kernel launch");
 }
 
 static aflex_status bind_scratch(aflex_ctx* ctx, GemmConfig& cfg, char* ws, size_t ws_bytes, int* counters,
@@ -732,8 +791,9 @@ aflex_status linear_launch(aflex_ctx* ctx, const void* x, const void* w, int T, 
     CUtensorMap ta;
     TmapSetB tb;
     if (!encode_tmap_2d_bf16(&ta, w, (uint64_t)N, (uint64_t)K, (uint64_t)K * 2, kBlockM, kBlockK, true) ||
-        !encode_b_set(&tb, x, (uint64_t)T, (uint64_t)K, p.n_tile))
+        !encode_b_set(&tb, x, (uint64_t)T, (uint64_t)K, p.n_tile, cfg.pair))
         return set_error(ctx, AFLEX_ERR_CUDA, "linear: cuTensorMapEncodeTiled failed");
+    if (cfg.pair) return launch_gemm<kLinear, true>(ctx, cfg, ta, ta, tb, st, kind);
     if (mode == kLinear2) return launch_gemm<kLinear2>(ctx, cfg, ta, ta, tb, st, kind);
     return launch_gemm<kLinear>(ctx, cfg, ta, ta, tb, st, kind);
 }
@@ -759,8 +819,9 @@ aflex_status gateup_launch(aflex_ctx* ctx, const void* x, const void* w_gate, co
     TmapSetB tb;
     if (!encode_tmap_2d_bf16(&tg, w_gate, (uint64_t)I, (uint64_t)H, (uint64_t)H * 2, kBlockM, kBlockK, true) ||
         !encode_tmap_2d_bf16(&tu, w_up, (uint64_t)I, (uint64_t)H, (uint64_t)H * 2, kBlockM, kBlockK, true) ||
-        !encode_b_set(&tb, x, (uint64_t)T, (uint64_t)H, p.n_tile))
+        !encode_b_set(&tb, x, (uint64_t)T, (uint64_t)H, p.n_tile, cfg.pair))
         return set_error(ctx, AFLEX_ERR_CUDA, "gate/up: cuTensorMapEncodeTiled failed");
+    if (cfg.pair) return launch_gemm<kGateUp, true>(ctx, cfg, tg, tu, tb, st, kKGateUpGemm);
     return launch_gemm<kGateUp>(ctx, cfg, tg, tu, tb, st, kKGateUpGemm);
 }
 

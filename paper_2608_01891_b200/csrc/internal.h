@@ -53,7 +53,7 @@ struct aflex_ctx {
     unsigned attn_launch_seq = 0; // attention launches so far: picks the launch's pair of chunk-ticket words (four pairs in rotation)
     bool attn_q_final = false;    // caller's promise (aflex_set_attn_q_final): q is never the output of the kernel just before
     bool attn_q_final_once = false;   // set by the layer chains for their own attention launch (q comes from the append kernel)
-    bool gemm_attr_set[3] = {false, false, false};
+    bool gemm_attr_set[6] = {false, false, false, false, false, false};   // [mode + 3 * pair form]
     bool chain_attr_set = false;
     bool attn_attr_set[2] = {false, false};
     bool prefill_attr_set[2] = {false, false};   // shared-memory limit raised for attn_prefill_kernel<64 / 128> on this device

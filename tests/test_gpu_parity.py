@@ -110,7 +110,11 @@ def test_attention_custom_scale_and_zero_query(ctx):
 # ------------------------------------------------------------------------------- GEMMs / dense FFN
 @pytest.mark.parametrize("T,K,N", [(1, 64, 128), (4, 512, 512), (32, 1376, 512), (33, 520, 264), (130, 8192, 640),
                                    (300, 256, 136), (384, 320, 264), (700, 128, 136),
-                                   (100, 16384, 4104), (64, 8200, 8328)])   # large weights: two weight tiles per CTA tile
+                                   (100, 16384, 4104), (64, 8200, 8328),    # large weights: two weight tiles per CTA tile
+                                   # token tiles of 192 rows and more run on CTA pairs (256 weight rows per pair):
+                                   # a ragged second pair tile and ragged K; tiles shared along K by several pairs;
+                                   # several token tiles with a ragged last one; fewer pair tiles than pairs
+                                   (200, 520, 264), (256, 8192, 640), (1000, 1024, 1160), (192, 64, 256)])
 def test_linear_matches_oracle(ctx, T, K, N):
     x, w = rand_bf16((T, K), 1.0, 1), rand_bf16((N, K), 0.05, 2)
     y = torch.full((T, N), float("nan"), dtype=torch.bfloat16, device=DEV)
@@ -120,7 +124,7 @@ def test_linear_matches_oracle(ctx, T, K, N):
     assert row_rel_err(f64(y), want) <= TOL_FFN
 
 
-@pytest.mark.parametrize("T", [1, 3, 4, 32, 33, 64, 65, 100, 128, 129, 300, 384, 530])
+@pytest.mark.parametrize("T", [1, 3, 4, 32, 33, 64, 65, 100, 128, 129, 192, 200, 250, 256, 300, 384, 512, 530, 1000])
 def test_dense_ffn_config1_shapes(ctx, T):
     cfg = IN.CONFIGS[1]
     x = IN.make_x(cfg, tokens=T)
@@ -151,6 +155,24 @@ def test_dense_ffn_decode_batch_odd_shapes(ctx, T, H, I):
     ctx.ffn_dense(x.to(DEV), wg.to(DEV), wu.to(DEV), wd.to(DEV), y2)
     torch.cuda.synchronize()
     assert torch.equal(y.view(torch.int16), y2.view(torch.int16))          # bit-deterministic, launch after launch
+    assert ctx.device_status() == AF.OK
+
+
+@pytest.mark.parametrize("T,H,I", [(256, 1024, 2816), (208, 320, 3000), (600, 512, 1376)])
+def test_dense_ffn_cta_pair_shapes_are_bit_deterministic(ctx, T, H, I):
+    """Token tiles of 192 rows and more run on CTA pairs: tiles shared along K by several pairs (more K steps than a
+    pair's share), feature counts that are not a multiple of the pair's 256 weight rows, several token tiles."""
+    x, wg = rand_bf16((T, H), 1.0, 41), rand_bf16((I, H), 1.5 / np.sqrt(H), 42)
+    wu, wd = rand_bf16((I, H), 1.0 / np.sqrt(H), 43), rand_bf16((H, I), 1.0 / np.sqrt(I), 44)
+    y = torch.full((T, H), float("nan"), dtype=torch.bfloat16, device=DEV)
+    ctx.ffn_dense(x.to(DEV), wg.to(DEV), wu.to(DEV), wd.to(DEV), y)
+    torch.cuda.synchronize()
+    want = O.ffn_dense(u16(x), u16(wg), u16(wu), u16(wd))
+    assert row_rel_err(f64(y), want) <= TOL_FFN
+    y2 = torch.full_like(y, float("nan"))
+    ctx.ffn_dense(x.to(DEV), wg.to(DEV), wu.to(DEV), wd.to(DEV), y2)
+    torch.cuda.synchronize()
+    assert torch.equal(y.view(torch.int16), y2.view(torch.int16))
     assert ctx.device_status() == AF.OK
 
 
