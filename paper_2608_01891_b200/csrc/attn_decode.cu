@@ -661,24 +661,8 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                 }
                 continue;
             }
-            // ---- partial piece: park it in the range's slot, bump the item's counter
-            {
-                float* op = p.o_part + ((size_t)rg.rid * 2 + slot) * 8 * D;
-                float* mlp = p.ml_part + ((size_t)rg.rid * 2 + slot) * 8 * 2;
-#pragma unroll
-                for (int mt = 0; mt < kKSteps; ++mt) {
-                    op[(h0) * D + mt * 16 + dr] = o[mt][0];
-                    op[(h0 + 1) * D + mt * 16 + dr] = o[mt][1];
-                    op[(h0) * D + mt * 16 + dr + 8] = o[mt][2];
-                    op[(h0 + 1) * D + mt * 16 + dr + 8] = o[mt][3];
-                }
-                if (dr == 0) {
-                    mlp[h0 * 2] = m0; mlp[h0 * 2 + 1] = l0;
-                    mlp[(h0 + 1) * 2] = m1; mlp[(h0 + 1) * 2 + 1] = l1;
-                }
-            }
-            __syncwarp();
-            // pieces of this item: static shares cf..cl over [item_x0, min(item_x1, U1)), then dynamic chunks jf..jl
+            // ---- partial piece.  Pieces of this item: static shares cf..cl over [item_x0, min(item_x1, U1)), then
+            // dynamic chunks jf..jl; `mine` is this piece's place in that list.
             const long long item_x1 = item_x0 + nu;
             int cf = 0, cl = -1, jf = 0, jl = -1;
             if (item_x0 < sp.U1) {
@@ -690,90 +674,96 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                 jf = (int)((dyn_x0 - sp.U1) / sp.K2);
                 jl = (int)((item_x1 - 1 - sp.U1) / sp.K2);
             }
-            const int expected = (cl - cf + 1) + (jl - jf + 1);
-            int last = 0;
-            if (lane == 0) {
-                __threadfence();
-                last = (atomicAdd(&p.counters[b * p.Hkv + g], 1) == expected - 1) ? 1 : 0;
-            }
-            last = __shfl_sync(0xffffffffu, last, 0);
-            if (!last) continue;
-            // ---- last arriver: merge the item's pieces in list order (one pass, running maximum).
-            // Lane owns d = 4*lane + 128*j .. +3 of every head: all loads of a piece are independent.
-            // A piece sits in slot 0 of its range unless other units of the range precede it (slot 1):
-            // that can only happen for the first static share and for the first dynamic chunk.
-            __threadfence();
-            constexpr int kVec = D / 128 > 0 ? D / 128 : 1;      // float4 per head per lane (D = 64: lanes 16.. idle)
-            const bool lane_on = lane * 4 < D;
-            float M[8], L[8];
-            float4 acc[8][kVec];
-#pragma unroll
-            for (int h = 0; h < 8; ++h) {
-                M[h] = kNegBig; L[h] = 0.f;
-#pragma unroll
-                for (int j = 0; j < kVec; ++j) acc[h][j] = make_float4(0.f, 0.f, 0.f, 0.f);
-            }
             const int n_static = cl - cf + 1;
+            const int expected = n_static + (jl - jf + 1);
+            const int mine = rg.rid < G ? rg.rid - cf : n_static + (rg.rid - G - jf);
+            int* counter = p.counters + b * p.Hkv + g;
+            // Whoever finds all other pieces published finishes the item.  Usually that is known before anything is
+            // written: the other pieces of an item that ends a CTA's share were computed at the start of the next
+            // CTA's share, long ago.  Then this piece stays in registers: no partial store, no fence, no atomic.
+            int seen = 0;
+            if (lane == 0) asm volatile("ld.acquire.gpu.b32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
+            seen = __shfl_sync(0xffffffffu, seen, 0);
+            if (seen != expected - 1) {
+                // park the piece in the range's slot (as the lanes hold it: [k step][lane][4]), bump the item's counter
+                float4* op = reinterpret_cast<float4*>(p.o_part + ((size_t)rg.rid * 2 + slot) * 8 * D) + lane;
+                float* mlp = p.ml_part + ((size_t)rg.rid * 2 + slot) * 8 * 2;
+#pragma unroll
+                for (int mt = 0; mt < kKSteps; ++mt) op[mt * 32] = make_float4(o[mt][0], o[mt][1], o[mt][2], o[mt][3]);
+                if (dr == 0) *reinterpret_cast<float4*>(mlp + 2 * h0) = make_float4(m0, l0, m1, l1);
+                __syncwarp();
+                int last = 0;
+                if (lane == 0) {
+                    __threadfence();
+                    last = (atomicAdd(counter, 1) == expected - 1) ? 1 : 0;
+                }
+                last = __shfl_sync(0xffffffffu, last, 0);
+                if (!last) continue;
+                __threadfence();
+            }
+            // ---- merge the item's pieces in list order (running maximum), this piece from registers, the others
+            // from their slots.  A piece sits in slot 0 of its range unless other units of the range precede it
+            // (slot 1): that can only happen for the first static share and for the first dynamic chunk.
+            float acc[kKSteps][4];
+#pragma unroll
+            for (int mt = 0; mt < kKSteps; ++mt) { acc[mt][0] = acc[mt][1] = acc[mt][2] = acc[mt][3] = 0.f; }
+            float M0 = kNegBig, M1 = kNegBig, L0 = 0.f, L1 = 0.f;
             for (int i = 0; i < expected; ++i) {
-                int rid_i, sl;
-                if (i < n_static) {
-                    rid_i = cf + i;
-                    sl = (i == 0 && share_begin(sp.U1, cf, sp.Ge1) < item_v0) ? 1 : 0;
+                float pm0, pl0, pm1, pl1;
+                float4 po[kKSteps];
+                if (i == mine) {
+                    pm0 = m0; pl0 = l0; pm1 = m1; pl1 = l1;
+#pragma unroll
+                    for (int mt = 0; mt < kKSteps; ++mt) po[mt] = make_float4(o[mt][0], o[mt][1], o[mt][2], o[mt][3]);
                 } else {
-                    const int j = jf + (i - n_static);
-                    rid_i = G + j;
-                    sl = (j == jf && sp.U1 + (long long)jf * sp.K2 < max(item_v0, sp.U1)) ? 1 : 0;
-                }
-                const size_t base = ((size_t)rid_i * 2 + sl) * 8;
-                float2 ml[8];
-                float4 o4[8][kVec];
-#pragma unroll
-                for (int h = 0; h < 8; ++h) {
-                    if (h < p.G) {
-                        ml[h] = __ldcg(reinterpret_cast<const float2*>(p.ml_part + (base + h) * 2));
-#pragma unroll
-                        for (int j = 0; j < kVec; ++j)
-                            if (lane_on) o4[h][j] = __ldcg(reinterpret_cast<const float4*>(p.o_part + (base + h) * D + lane * 4 + j * 128));
+                    int rid_i, sl;
+                    if (i < n_static) {
+                        rid_i = cf + i;
+                        sl = (i == 0 && share_begin(sp.U1, cf, sp.Ge1) < item_v0) ? 1 : 0;
+                    } else {
+                        const int j = jf + (i - n_static);
+                        rid_i = G + j;
+                        sl = (j == jf && sp.U1 + (long long)jf * sp.K2 < max(item_v0, sp.U1)) ? 1 : 0;
                     }
+                    const size_t base = ((size_t)rid_i * 2 + sl) * 8;
+                    const float4 ml = __ldcg(reinterpret_cast<const float4*>(p.ml_part + base * 2 + 2 * h0));
+                    const float4* src = reinterpret_cast<const float4*>(p.o_part + base * D) + lane;
+#pragma unroll
+                    for (int mt = 0; mt < kKSteps; ++mt) po[mt] = __ldcg(src + mt * 32);
+                    pm0 = ml.x; pl0 = ml.y; pm1 = ml.z; pl1 = ml.w;
                 }
+                const float mn0 = fmaxf(M0, pm0), mn1 = fmaxf(M1, pm1);
+                const float a0 = fast_exp2(M0 - mn0), a1 = fast_exp2(M1 - mn1);
+                const float b0 = fast_exp2(pm0 - mn0), b1 = fast_exp2(pm1 - mn1);
+                M0 = mn0; M1 = mn1;
+                L0 = L0 * a0 + pl0 * b0;
+                L1 = L1 * a1 + pl1 * b1;
 #pragma unroll
-                for (int h = 0; h < 8; ++h) {
-                    if (h < p.G) {
-                        const float mn = fmaxf(M[h], ml[h].x);
-                        const float fa = fast_exp2(M[h] - mn), fb = fast_exp2(ml[h].x - mn);
-                        M[h] = mn;
-                        L[h] = L[h] * fa + ml[h].y * fb;
-#pragma unroll
-                        for (int j = 0; j < kVec; ++j) {
-                            if (lane_on) {
-                                acc[h][j].x = acc[h][j].x * fa + o4[h][j].x * fb;
-                                acc[h][j].y = acc[h][j].y * fa + o4[h][j].y * fb;
-                                acc[h][j].z = acc[h][j].z * fa + o4[h][j].z * fb;
-                                acc[h][j].w = acc[h][j].w * fa + o4[h][j].w * fb;
-                            }
-                        }
-                    }
+                for (int mt = 0; mt < kKSteps; ++mt) {
+                    acc[mt][0] = acc[mt][0] * a0 + po[mt].x * b0;
+                    acc[mt][1] = acc[mt][1] * a1 + po[mt].y * b1;
+                    acc[mt][2] = acc[mt][2] * a0 + po[mt].z * b0;
+                    acc[mt][3] = acc[mt][3] * a1 + po[mt].w * b1;
                 }
             }
+            if (h0 < p.G) {
+                const float i0 = 1.0f / L0, i1 = 1.0f / L1;
+                __nv_bfloat16* out0 = p.out + ((size_t)b * p.Hq + hq0) * D;
 #pragma unroll
-            for (int h = 0; h < 8; ++h) {
-                if (h < p.G) {
-                    const float inv = 1.0f / L[h];
-                    const size_t hq = (size_t)g * p.G + h;
-#pragma unroll
-                    for (int j = 0; j < kVec; ++j) {
-                        if (lane_on) {
-                            __nv_bfloat162 lo = __floats2bfloat162_rn(acc[h][j].x * inv, acc[h][j].y * inv);
-                            __nv_bfloat162 hi = __floats2bfloat162_rn(acc[h][j].z * inv, acc[h][j].w * inv);
-                            uint2 pk;
-                            pk.x = *reinterpret_cast<uint32_t*>(&lo);
-                            pk.y = *reinterpret_cast<uint32_t*>(&hi);
-                            *reinterpret_cast<uint2*>(p.out + ((size_t)b * p.Hq + hq) * D + lane * 4 + j * 128) = pk;
-                        }
+                for (int mt = 0; mt < kKSteps; ++mt) {
+                    out0[mt * 16 + dr] = __float2bfloat16_rn(acc[mt][0] * i0);
+                    out0[mt * 16 + dr + 8] = __float2bfloat16_rn(acc[mt][2] * i0);
+                    if (h0 + 1 < p.G) {
+                        out0[D + mt * 16 + dr] = __float2bfloat16_rn(acc[mt][1] * i1);
+                        out0[D + mt * 16 + dr + 8] = __float2bfloat16_rn(acc[mt][3] * i1);
                     }
-                    if (p.lse != nullptr && lane == 0) p.lse[(size_t)b * p.Hq + hq] = (M[h] + log2f(L[h])) * 0.6931471805599453f;
+                }
+                if (p.lse != nullptr && dr == 0) {
+                    p.lse[(size_t)b * p.Hq + hq0] = (M0 + log2f(L0)) * 0.6931471805599453f;
+                    if (h0 + 1 < p.G) p.lse[(size_t)b * p.Hq + hq0 + 1] = (M1 + log2f(L1)) * 0.6931471805599453f;
                 }
             }
+            __syncwarp();
             if (lane == 0) p.counters[b * p.Hkv + g] = 0;   // clean for the next launch
         }
         }
