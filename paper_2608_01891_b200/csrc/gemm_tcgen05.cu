@@ -33,7 +33,8 @@
 // before its predecessor has drained; weight tiles (which no kernel writes) are prefetched into
 // the pipeline before the grid-dependency wait, activation tiles only after it.
 //
-// CTA = 6 warps: warp 0 TMA producer, warp 1 MMA issuer (owns TMEM), warps 2..5 epilogue.
+// CTA = 10 warps: warp 0 TMA producer, warp 1 MMA issuer (owns TMEM), warps 2..9 epilogue (a warp reads the TMEM lanes
+// of its quadrant, warp index mod 4; the two warps of a quadrant take alternate groups of 16 token columns).
 // All waits are bounded.
 #include <cuda_bf16.h>
 #include <stdio.h>
@@ -49,7 +50,9 @@ enum GemmMode { kLinear = 0, kGateUp = 1, kLinear2 = 2 };
 
 constexpr int kBlockM = 128;   // weight rows per tile (UMMA M)
 constexpr int kBlockK = 64;    // bf16 elements per 128-byte swizzled row
-constexpr int kGemmThreads = 192;
+constexpr int kEpiWarps = 8;                                 // epilogue warps: two per TMEM lane quadrant, each pair splits the token columns
+constexpr int kEpiThreads = kEpiWarps * 32;
+constexpr int kGemmThreads = 64 + kEpiThreads;
 constexpr int kMaxStages = 8;
 constexpr int kMaxExperts = 64;
 constexpr int kStageTokens = 32;                             // token rows staged per round of the epilogue
@@ -177,7 +180,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&bars->tmem_full[b], 1); mbar_init(&bars->tmem_empty[b], PAIR ? 8 : 4); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&bars->tmem_full[b], 1); mbar_init(&bars->tmem_empty[b], (PAIR ? 2 : 1) * kEpiWarps); }
         bars->abort = 0;
         fence_mbar_init();
     }
@@ -321,10 +324,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
             }
         }
     } else {
-        // ------------------------------------------------------------ epilogue (warps 2..5)
+        // ------------------------------------------------------------ epilogue (warps 2..9)
         const int lane_grp = warp & 3;                 // TMEM lanes [32*lane_grp, +32) belong to this warp
+        const int chalf = (warp - 2) >> 2;             // which of the quadrant's two warps: takes column groups chalf, chalf + 2, ..
         const int row = lane_grp * 32 + lane;          // accumulator row = weight row inside the tile
-        const int etid = threadIdx.x - 64;             // 0..127 among the epilogue threads
+        const int etid = threadIdx.x - 64;             // 0..255 among the epilogue threads
         const int cols = kAccs * p.n_tile;             // fp32 values per accumulator row
         const size_t slot_floats = (size_t)cols * kBlockM;
         int buf = 0; uint32_t acc_ph = 0;
@@ -351,9 +355,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
         // Staged token rows [0, ntok) -> output rows t0 + .. (bounded by t_limit), features 128 * .. of the tile; the
         // barriers order the staging writes before the reads and free the buffer for its next user.
         auto stage_flush = [&](const TileCoord& c, int t0, int ntok) {
-            asm volatile("bar.sync 2, 128;" ::: "memory");
+            asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads) : "memory");
             const int n0 = c.m_tile * p.tile_rows + rank * kBlockM;
-            for (int i = etid; i < ntok * cpr; i += 128) {
+            for (int i = etid; i < ntok * cpr; i += kEpiThreads) {
                 const int tl = i / cpr, part = i - tl * cpr;
                 const int t = t0 + tl, n = n0 + part * per16;
                 if (t < c.out_row_limit && n < p.N) {
@@ -363,7 +367,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
                     *reinterpret_cast<uint4*>(dst) = v;
                 }
             }
-            asm volatile("bar.sync 2, 128;" ::: "memory");
+            asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads) : "memory");
         };
 
         // A shared tile is finished by its contributors together (all of them but a last one that has another
@@ -398,7 +402,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
             }
             // the barrier hands thread 0's acquire on to the other 127 threads, and its verdict with it: the four warps
             // leave together or not at all (there are barriers further down)
-            if (bar_or(2, 128, failed)) { gave_up = true; return; }
+            if (bar_or(2, kEpiThreads, failed)) { gave_up = true; return; }
             const bool cf_early = sched.share_begin(cf) < x0;
             // The parked accumulators are [column group of 4 tokens][128 rows] float4.  Reducer `me` takes whole column
             // groups, thread = accumulator row; kElems groups per round with every piece's loads of a round in flight
@@ -410,7 +414,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
             constexpr int kCgPerFlush = kStageTokens / 4;
             for (int f0 = cg_lo; f0 < cg_hi; f0 += kCgPerFlush) {
                 const int f1 = min(cg_hi, f0 + kCgPerFlush);
-                for (int c0 = f0; c0 < f1; c0 += kElems) {
+                for (int c0 = f0 + chalf * kElems; c0 < f1; c0 += 2 * kElems) {
                     float4 g[kElems], u[kElems];
 #pragma unroll
                     for (int e = 0; e < kElems; ++e) g[e] = u[e] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -424,7 +428,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
                                 // later unit of that CTA (slot 1); every other piece is a first unit (slot 0)
                                 const int sl = (cc == cf && cf_early) ? 1 : 0;
                                 const size_t who = PAIR ? (size_t)cc * 2 + rank : (size_t)cc;      // the CTA that parked the piece
-                                const float4* part = reinterpret_cast<const float4*>(p.partials + (who * 2 + sl) * slot_floats) + etid;
+                                const float4* part = reinterpret_cast<const float4*>(p.partials + (who * 2 + sl) * slot_floats) + row;
 #pragma unroll
                                 for (int e = 0; e < kElems; ++e) {
                                     if (c0 + e < f1) {
@@ -454,17 +458,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
 #pragma unroll
                         for (int k = 0; k < 4; ++k) {
                             const int tl = (c0 + e - f0) * 4 + k;
-                            if (MODE == kGateUp) stage_put(tl, etid, silu_f32(gf[k]) * uf[k]);
+                            if (MODE == kGateUp) stage_put(tl, row, silu_f32(gf[k]) * uf[k]);
                             else {
-                                stage_put(tl, etid, gf[k]);
-                                if (MODE == kLinear2) stage_put(tl, etid + kBlockM, uf[k]);
+                                stage_put(tl, row, gf[k]);
+                                if (MODE == kLinear2) stage_put(tl, row + kBlockM, uf[k]);
                             }
                         }
                     }
                 }
                 stage_flush(pd.c, pd.c.b_row0 + f0 * 4, (f1 - f0) * 4);
             }
-            asm volatile("bar.sync 2, 128;" ::: "memory");
+            asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads) : "memory");
             if (etid == 0) {
                 const int done = atomicAdd(&p.counters[kStreamKMaxTiles + ctile(pd.tile)], 1);
                 if (done == nred - 1) {   // every reducer has read what it needs: clean up for the next launch
@@ -477,7 +481,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
         // (every exit from this loop is decided on a predicate OR-ed across the four epilogue warps: the loop body holds
         // barriers, and a warp that left alone would leave the others waiting at one for good)
         while (cur.next(wu)) {
-            if (bar_or(2, 128, bars->abort != 0)) { gave_up = true; break; }
+            if (bar_or(2, kEpiThreads, bars->abort != 0)) { gave_up = true; break; }
             const TileCoord c = tiles.get(wu.tile);
             if (wu.slot < 0 && npend > 0) {
                 // shared tiles come first: before waiting for the first whole tile, finish this CTA's part
@@ -487,7 +491,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
                 if (gave_up) break;
             }
             const bool full_ok = mbar_wait(&bars->tmem_full[buf], acc_ph);
-            if (bar_or(2, 128, !full_ok)) {
+            if (bar_or(2, kEpiThreads, !full_ok)) {
                 if (etid == 0) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); }
                 gave_up = true;
                 break;
@@ -498,7 +502,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
                 // ---- whole K range in this CTA: epilogue straight from TMEM, kStageTokens token columns per round
                 for (int tc = 0; tc < c.b_rows; tc += kStageTokens) {
                     const int ntok = min(kStageTokens, c.b_rows - tc);
-                    for (int c0 = 0; c0 < ntok; c0 += 16) {
+                    for (int c0 = 16 * chalf; c0 < ntok; c0 += 32) {
                         uint32_t g[16];
                         tmem_ld_32x32b_x16(t0 + (uint32_t)(tc + c0), g);
                         if (MODE != kLinear) {
@@ -528,7 +532,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
                 // ---- partial K range: park the fp32 accumulator as [column group of 4][row] float4 (a warp
                 //      stores / loads 512 contiguous bytes per instruction); the last arriver finishes the tile
                 uint4* mine = reinterpret_cast<uint4*>(p.partials + ((size_t)blockIdx.x * 2 + wu.slot) * slot_floats) + row;
-                for (int c0 = 0; c0 < cols; c0 += 16) {
+                for (int c0 = 16 * chalf; c0 < cols; c0 += 32) {
                     if ((c0 % p.n_tile) >= c.b_rows) continue;   // token columns beyond the tile's valid rows
                     uint32_t g[16];
                     tmem_ld_32x32b_x16(t0 + (uint32_t)c0, g);
@@ -542,7 +546,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
                 if (lane == 0) release_tmem(buf);   // TMEM buffer is free again
                 // publish: all 128 rows stored (CTA barrier), then one thread releases them device-wide
                 // and bumps the tile counter.  The reduction itself is deferred (see run_reduce).
-                asm volatile("bar.sync 2, 128;" ::: "memory");
+                asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads) : "memory");
                 if (etid == 0) {
                     if (tr) tr[6] = global_timer_ns();               // partial stored, about to publish
                     __threadfence();
