@@ -695,7 +695,16 @@ static bool make_config(int mode, int T, int N, int K, int rows_max, int E, int 
     static int nostream = -1;   // AFLEX_GEMM_NOSTREAMK=1: whole tiles only (measurement of per-SM streaming rates)
     if (nostream < 0) { const char* e = getenv("AFLEX_GEMM_NOSTREAMK"); nostream = e ? atoi(e) : 0; }
     const long long workers = cfg->pair ? num_sms / 2 : num_sms;      // CTAs, or CTA pairs, that share the tile list
-    p.streamk = nostream ? 0 : (tiles_hi < 8LL * workers && tiles_hi <= kStreamKMaxTiles && (p.n_tile <= 128 || tiles_hi < 2LL * workers)) ? 1 : 0;
+    // ... or, for the dense single-accumulator form (128 KB partials, double-buffered TMEM), when whole tiles in rounds
+    // would leave more than a tenth of the last round's CTAs idle: the down projection at 2048 tokens is 160 tiles on 74
+    // pairs, three rounds for 2.16 rounds of work (465 -> 380 us with the remainder shared along K).  Gate/up (two
+    // accumulators: 256 KB partials, no second buffer) and the grouped form measured slower that way.
+    // AFLEX_GEMM_STREAMK_WIDE=0 switches it off (tuning).
+    static int wide_sk = -1;
+    if (wide_sk < 0) { const char* e = getenv("AFLEX_GEMM_STREAMK_WIDE"); wide_sk = e ? atoi(e) : 1; }
+    const long long rounds = (tiles_hi + workers - 1) / workers;
+    const bool wide_share = wide_sk != 0 && E == 0 && mode == kLinear && tiles_hi * 10 < rounds * workers * 9;
+    p.streamk = nostream ? 0 : (tiles_hi < 8LL * workers && tiles_hi <= kStreamKMaxTiles && (p.n_tile <= 128 || wide_share || tiles_hi < 2LL * workers)) ? 1 : 0;
     // epilogue staging: kStageTokens token rows of the tile in the output type
     const int stage_out_bytes = kStageTokens * (mode == kLinear2 ? 2 : 1) * kBlockM * (out_f32 ? 4 : 2);
     int cap = (p.streamk && p.n_tile <= 64 && mode != kLinear2) ? streaming_smem_budget() + stage_out_bytes : kMaxDynamicSmem;
