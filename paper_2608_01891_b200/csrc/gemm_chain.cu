@@ -669,7 +669,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const ChainParams p) {
                 } while (clock64() - t_start < kWaitBudgetCycles && !bars->abort);
                 if (seen < np) { failed = true; if (!bars->abort) { bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); } }
             }
-            // the barrier hands thread 0's acquire on to the other 127 threads, and its verdict with it
+            // the barrier hands thread 0's acquire on to the other 127 threads, and its decision with it
             if (bar_or(3, 128, failed)) break;
             const bool cf_early = sched.share_begin(cf) < x0;
             // The parked accumulator is [column group of 4 tokens][128 rows] float4: reducer `me` takes whole column

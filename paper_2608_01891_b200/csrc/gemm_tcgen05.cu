@@ -400,7 +400,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__
                 } while (clock64() - t_start < kWaitBudgetCycles);
                 if (seen < np) { failed = true; bars->abort = 1; atomicExch(p.status, AFLEX_ERR_TIMEOUT); }
             }
-            // the barrier hands thread 0's acquire on to the other 127 threads, and its verdict with it: the four warps
+            // the barrier hands thread 0's acquire on to the other epilogue threads, and its decision with it: the warps
             // leave together or not at all (there are barriers further down)
             if (bar_or(2, kEpiThreads, failed)) { gave_up = true; return; }
             const bool cf_early = sched.share_begin(cf) < x0;
