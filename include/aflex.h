@@ -274,11 +274,16 @@ AFLEX_API aflex_status aflex_moe_route(aflex_ctx* ctx, const float* router_logit
  *     x = a W_o^T   (x = a if w_o == NULL, which requires Hq*D == hidden)
  *     y = dense FFN(x)  or  MoE FFN(x, router)   bf16 [B][hidden]
  * scheduled as in the paper's interleaved A/F pipeline (Section 4.3, Eq. 2):
- * the batch is cut into M contiguous microbatches; A_i (attention + W_o) is
- * enqueued on the ctx's attention stream, F_i on its FFN stream as soon as A_i
- * has finished, so A_{i+1} overlaps F_i.  M = 1 runs A then F serially.  Both
- * "sides" live on one GPU here, so the transfer term of Eq. 2 is zero.
- * The result does not depend on M or on the split.
+ * the batch is cut into M contiguous microbatches, enqueued in the pipeline's
+ * order A_0, F_0, A_1, F_1, ...  Both "sides" live on one GPU here, so the
+ * transfer term of Eq. 2 is zero, and every kernel of either side fills the
+ * whole GPU: by default everything goes on the caller's stream, where each
+ * kernel starts (programmatic dependent launch) while its predecessor drains.
+ * With aflex_set_interleave_streams(ctx, 1) A_i (attention + W_o) is enqueued
+ * on the ctx's attention stream and F_i on its FFN stream as soon as A_i has
+ * finished, so that A_{i+1} may overlap F_i as on two pools; on one B200 that
+ * form measured 1 - 4 % slower.  M = 1 always runs A then F on the caller's
+ * stream.  The result does not depend on M, on the split or on the form.
  */
 typedef struct {
     aflex_attn_desc attn;
@@ -337,6 +342,12 @@ AFLEX_API aflex_status aflex_set_attn_ctas(aflex_ctx* ctx, int ctas);
  * computing while the preceding kernel drains.  q written by aflex_rope_append, by a caller's kernel, by a copy,
  * or resident from earlier work satisfies the promise. */
 AFLEX_API aflex_status aflex_set_attn_q_final(aflex_ctx* ctx, int on);
+
+/* How aflex_layer_step enqueues M >= 2 microbatches (default off; AFLEX_MB_STREAMS=2 in the
+ * environment when the ctx is created turns it on).  on != 0: A_i on the ctx's attention stream, F_i on its FFN stream behind an
+ * event, both joined to the caller's stream at entry and exit.  on == 0: all kernels on the caller's stream in the
+ * order A_0, F_0, A_1, F_1, ...  Host-side choice only; the results are the same. */
+AFLEX_API aflex_status aflex_set_interleave_streams(aflex_ctx* ctx, int on);
 
 /* ---- Whole decoder layers, chained (Section 4.3, "Interleaved A/F Pipeline") -------------
  *

@@ -22,7 +22,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_
 EXPORTS = (
     "aflex_status_string", "aflex_version", "aflex_create", "aflex_destroy", "aflex_last_error",
     "aflex_get_device_status", "aflex_attn_decode", "aflex_ffn_dense", "aflex_ffn_moe", "aflex_moe_route", "aflex_layer_step",
-    "aflex_workspace_bytes", "aflex_linear", "aflex_set_attn_ctas", "aflex_set_attn_q_final", "aflex_num_kernel_kinds",
+    "aflex_workspace_bytes", "aflex_linear", "aflex_set_attn_ctas", "aflex_set_attn_q_final", "aflex_set_interleave_streams", "aflex_num_kernel_kinds",
     "aflex_kernel_name", "aflex_launch_count", "aflex_profile_enable", "aflex_profile_read",
     "aflex_trace_read", "aflex_attn_decode_static", "aflex_attn_decode_static_status", "aflex_decoder_layers", "aflex_decoder_workspace_bytes",
     "aflex_add_rmsnorm", "aflex_rope_append", "aflex_attn_prefill", "aflex_af_decoder_layers", "aflex_af_workspace_bytes",
@@ -113,6 +113,8 @@ def load_library() -> ctypes.CDLL:
     lib.aflex_set_attn_ctas.argtypes = [vp, ci]
     lib.aflex_set_attn_q_final.restype = ci
     lib.aflex_set_attn_q_final.argtypes = [vp, ci]
+    lib.aflex_set_interleave_streams.restype = ci
+    lib.aflex_set_interleave_streams.argtypes = [vp, ci]
     lib.aflex_attn_decode.restype = ci
     lib.aflex_attn_decode.argtypes = [vp, ctypes.POINTER(AttnDesc), vp, ctypes.POINTER(KV), ci, vp, vp, vp]
     lib.aflex_attn_prefill.restype = ci
@@ -432,6 +434,10 @@ class Context:
     def set_attn_q_final(self, on: bool) -> None:
         """Promise that q is never produced by the library kernel enqueued directly before an attention call."""
         self._check(self._lib.aflex_set_attn_q_final(self._h, 1 if on else 0))
+
+    def set_interleave_streams(self, on: bool) -> None:
+        """layer_step with M >= 2: A side and F side on the ctx's two streams (True) or everything on the caller's stream."""
+        self._check(self._lib.aflex_set_interleave_streams(self._h, 1 if on else 0))
 
     def set_attn_ctas(self, ctas: int) -> None:
         self._check(self._lib.aflex_set_attn_ctas(self._h, ctas))

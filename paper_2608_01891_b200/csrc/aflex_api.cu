@@ -295,6 +295,7 @@ aflex_status aflex_create(aflex_ctx** out, int device, size_t workspace_bytes) {
     aflex_ctx* ctx = new (std::nothrow) aflex_ctx();
     if (!ctx) return AFLEX_ERR_CUDA;
     ctx->device = device;
+    { const char* ev = getenv("AFLEX_MB_STREAMS"); ctx->mb_two_streams = ev && atoi(ev) == 2; }
     ctx->ws_bytes = workspace_bytes ? align256(workspace_bytes) : kDefaultWorkspace;
     cudaError_t e = cudaSetDevice(device);
     cudaDeviceProp prop;
@@ -456,6 +457,12 @@ aflex_status aflex_trace_read(aflex_ctx* ctx, unsigned long long* host_out, int 
 aflex_status aflex_set_attn_q_final(aflex_ctx* ctx, int on) {
     if (!ctx) return AFLEX_ERR_INVALID_ARG;
     ctx->attn_q_final = on != 0;
+    return AFLEX_OK;
+}
+
+aflex_status aflex_set_interleave_streams(aflex_ctx* ctx, int on) {
+    if (!ctx) return AFLEX_ERR_INVALID_ARG;
+    ctx->mb_two_streams = on != 0;
     return AFLEX_OK;
 }
 
@@ -638,9 +645,11 @@ aflex_status aflex_layer_step(aflex_ctx* ctx, const aflex_layer_desc* L, const v
 
     cudaStream_t user = reinterpret_cast<cudaStream_t>(stream);
     // M = 1 is A then F in series (Eq. 2, first case): everything goes on the caller's stream, where
-    // consecutive kernels chain through programmatic dependent launch.  M >= 2 uses the ctx's
-    // attention and FFN streams, joined to the caller's stream on entry and exit.
-    const bool serial = (M == 1);
+    // consecutive kernels chain through programmatic dependent launch.  So does M >= 2 by default, in the
+    // order A_0, F_0, A_1, F_1, ...: on one GPU a kernel of either side fills every SM, so the sides cannot
+    // run at the same time and the chained launches have the shorter boundaries.  On request M >= 2 uses the
+    // ctx's attention and FFN streams, joined to the caller's stream on entry and exit.
+    const bool serial = (M == 1) || !ctx->mb_two_streams;
     cudaStream_t sa = serial ? user : ctx->stream_a, sf = serial ? user : ctx->stream_f;
     cudaError_t e = cudaSuccess;
     if (!serial) {

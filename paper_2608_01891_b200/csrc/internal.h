@@ -51,6 +51,7 @@ struct aflex_ctx {
     cudaEvent_t ev_f_done = nullptr, ev_a_done = nullptr;
     int attn_ctas = 0;            // persistent attention CTAs per launch; 0 = two per SM
     unsigned attn_launch_seq = 0; // attention launches so far: picks the launch's pair of chunk-ticket words (four pairs in rotation)
+    bool mb_two_streams = false;  // aflex_layer_step, M >= 2: A side and F side on the ctx's two streams (else all on the caller's)
     bool attn_q_final = false;    // caller's promise (aflex_set_attn_q_final): q is never the output of the kernel just before
     bool attn_q_final_once = false;   // set by the layer chains for their own attention launch (q comes from the append kernel)
     bool gemm_attr_set[6] = {false, false, false, false, false, false};   // [mode + 3 * pair form]

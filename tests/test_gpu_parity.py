@@ -281,7 +281,18 @@ def run_layer(ctx, cfg, q, kv, wo, wg, wu, wd, M, offsets=None, logits=None, wan
     return f64(y), (f64(a) if want_attn else None)
 
 
-def test_layer_step_config1_all_depths(ctx):
+@pytest.mark.parametrize("two_streams", [False, True])
+def test_layer_step_config1_all_depths(ctx, two_streams):
+    """Both forms of the M >= 2 schedule: everything on the caller's stream (default), and A side / F side on the ctx's
+    two streams."""
+    ctx.set_interleave_streams(two_streams)
+    try:
+        _layer_step_config1_all_depths(ctx)
+    finally:
+        ctx.set_interleave_streams(False)
+
+
+def _layer_step_config1_all_depths(ctx):
     cfg = IN.CONFIGS[1]
     kv = IN.make_paged_kv(cfg, poison=True)
     q, wo = IN.make_q(cfg), IN.make_wo(cfg)
@@ -300,7 +311,16 @@ def test_layer_step_config1_all_depths(ctx):
         assert row_rel_err(y, ys[0]) <= 1e-2       # independent of M and of the split (to bf16 rounding)
 
 
-def test_layer_step_small_moe_all_depths(ctx):
+@pytest.mark.parametrize("two_streams", [False, True])
+def test_layer_step_small_moe_all_depths(ctx, two_streams):
+    ctx.set_interleave_streams(two_streams)
+    try:
+        _layer_step_small_moe_all_depths(ctx)
+    finally:
+        ctx.set_interleave_streams(False)
+
+
+def _layer_step_small_moe_all_depths(ctx):
     cfg = IN.LayerConfig(91, "small-moe", 12, 8, 2, 128, 256, 384, num_experts=8, top_k=2,
                          len_lo=1, len_hi=700)
     kv = IN.make_paged_kv(cfg)
@@ -538,10 +558,18 @@ def test_attention_waits_for_a_query_produced_by_the_preceding_gemm(ctx):
     assert ctx.device_status() == AF.OK
 
 
-@pytest.mark.parametrize("M", [1, 2])
-def test_layer_step_replays_from_a_cuda_graph(ctx, M):
-    """The layer step (one stream at M = 1, the ctx's two streams joined to the caller's at M >= 2) captured
-    into a CUDA graph after a warm-up call, replayed twice: same bits as the eager call."""
+@pytest.mark.parametrize("M,two_streams", [(1, False), (2, False), (2, True)])
+def test_layer_step_replays_from_a_cuda_graph(ctx, M, two_streams):
+    """The layer step (everything on the caller's stream, or at M >= 2 the ctx's two streams joined to the caller's)
+    captured into a CUDA graph after a warm-up call, replayed twice: same bits as the eager call."""
+    ctx.set_interleave_streams(two_streams)
+    try:
+        _layer_step_replays_from_a_cuda_graph(ctx, M)
+    finally:
+        ctx.set_interleave_streams(False)
+
+
+def _layer_step_replays_from_a_cuda_graph(ctx, M):
     cfg = IN.CONFIGS[1]
     kvh = IN.make_paged_kv(cfg)
     kv = AF.make_kv(kvh.k_cache.to(DEV), kvh.v_cache.to(DEV), kvh.page_table.to(DEV), kvh.seq_lens.to(DEV), kvh.seq_lens)
