@@ -838,6 +838,8 @@ aflex_status aflex_decoder_layers(aflex_ctx* ctx, const aflex_decoder_desc* laye
     if (s != AFLEX_OK) return s;
 
     cudaStream_t user = reinterpret_cast<cudaStream_t>(stream);
+    // (always two streams at M >= 2 here: with the layer's small attention-side kernels between the big ones the
+    //  two-stream form measured equal on the dense configurations and 4 - 5 % faster on the MoE ones)
     const bool serial = (M == 1);
     cudaStream_t sa = serial ? user : ctx->stream_a, sf = serial ? user : ctx->stream_f;
     cudaError_t e = cudaSuccess;
